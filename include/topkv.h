@@ -1,0 +1,201 @@
+/*
+ * topkv.h — C ABI of the TopKV data plane for one B200 (sm_100a).
+ *
+ * The library moves ONE LAYER of a batch's paged KV cache between a paged block
+ * pool and a contiguous "wire" buffer, the unit that the paper's pipelined
+ * layer-by-layer transfer sends while later layers still compute (§5.2), in the
+ * contiguous serialised layout that lets a link move it as one DMA (§3.4).
+ *
+ *   pack    : paged pool  -> contiguous wire      (prefill side)
+ *   unpack  : contiguous wire -> paged pool       (decode side, own block table)
+ *   *_host  : the same with the wire in pinned host memory (the PCIe leg, §3.3)
+ *
+ * Elements are opaque `elem_bytes`-wide words (FP16 in the paper, §2.2; bf16 in
+ * the benchmark shapes): bytes are moved, never interpreted, so every result is
+ * bit-exact by construction.
+ *
+ * Notation (follows the paper's Eq. 1 where it has a symbol):
+ *   L layers, h_kv = num_kv_heads (H), d_h = head_dim (D), b_p = elem_bytes (E),
+ *   F = kv_factor (2: separate K and V planes; 1: a single MLA latent row, §5.3),
+ *   P = page_tokens, R = requests, s_r = seq_lens[r], cu_r = sum_{q<r} s_q,
+ *   T = cu_R, row_bytes = H*D*E, N_layer = T*F*row_bytes.
+ *
+ * Pool addressing (bytes):
+ *   poff(l,p,c,t,h,d) = l*pool_layer_stride + p*pool_page_stride + c*pool_kv_stride
+ *                     + t*pool_token_stride + h*pool_head_stride + d*E
+ * Wire addressing (bytes), per layer slab:
+ *   TOKEN_KV : woff(r,i,c,h,d) = ((cu_r + i)*F + c)*row_bytes + (h*D + d)*E
+ *   PLANAR   : woff(r,i,c,h,d) = (c*T + cu_r + i)*row_bytes   + (h*D + d)*E
+ * TOKEN_KV is the batched order [request][token][K|V][head][dim]; PLANAR is the
+ * paper's "K tensor then V tensor, each [seq_len][kv_heads][head_dim]" (§3.4).
+ * The wire slab of layer l starts at wire + l*wire_layer_stride.
+ *
+ * pack   : for r<R, i<s_r, c<F, h<H, d<D : wire[woff(r,i,c,h,d)] = pool[poff(l, bt[r][i/P], c, i%P, h, d)]
+ * unpack : for the same index set        : pool[poff(l, bt[r][i/P], c, i%P, h, d)] = wire[woff(r,i,c,h,d)]
+ *          and every other pool byte keeps its value.
+ *
+ * Ownership: the caller owns every buffer. The entry points below allocate
+ * nothing, free nothing and only enqueue work on `stream`; results are valid
+ * once the caller has synchronised with the stream. All `const void*`/`void*`
+ * arguments are DEVICE pointers unless their name starts with `h_`.
+ *
+ * Errors: every int-returning function returns TOPKV_OK (0) or a negative
+ * topkv_status. When an error is returned nothing has been launched.
+ */
+#ifndef TOPKV_H_
+#define TOPKV_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* A CUDA stream handle (cudaStream_t). Declared opaquely so that this header
+ * compiles without the CUDA toolkit. */
+typedef struct CUstream_st* topkv_stream_t;
+
+typedef enum topkv_status {
+  TOPKV_OK = 0,
+  TOPKV_ERR_INVALID_ARG = -1,        /* NULL pointer, negative count, struct_size mismatch   */
+  TOPKV_ERR_LAYER_RANGE = -2,        /* layer not in [0, num_layers)                          */
+  TOPKV_ERR_ALIGNMENT = -3,          /* a base, stride or row_bytes is not a multiple of 16 B */
+  TOPKV_ERR_CAPACITY = -4,           /* wire / host / staging buffer smaller than N_layer     */
+  TOPKV_ERR_UNSUPPORTED_LAYOUT = -5, /* descriptor is self-inconsistent or not supported      */
+  TOPKV_ERR_CUDA = -6                /* a CUDA call failed; see topkv_last_cuda_error()       */
+} topkv_status;
+
+enum { TOPKV_KIND_GQA = 0, TOPKV_KIND_MLA = 1 };
+enum { TOPKV_WIRE_TOKEN_KV = 0, TOPKV_WIRE_PLANAR = 1 };
+
+/* Describes one paged pool and the wire format. All strides are in bytes; the
+ * head_dim axis is always contiguous. */
+typedef struct topkv_layout {
+  uint32_t struct_size;     /* = sizeof(topkv_layout); guards against ABI drift          */
+  uint32_t kind;            /* TOPKV_KIND_GQA or TOPKV_KIND_MLA (informational; F rules)  */
+  uint32_t num_layers;      /* L                                                          */
+  uint32_t kv_factor;       /* F: 2 = K and V planes, 1 = one latent row per token (§5.3) */
+  uint32_t num_kv_heads;    /* H (1 for MLA)                                              */
+  uint32_t head_dim;        /* D (576 = 512 + 64 for the DeepSeek-V3 latent, §5.3)        */
+  uint32_t elem_bytes;      /* E = b_p of Eq. 1 (2 for FP16 / bf16)                       */
+  uint32_t page_tokens;     /* P                                                          */
+  uint32_t wire_order;      /* TOPKV_WIRE_TOKEN_KV or TOPKV_WIRE_PLANAR                   */
+  uint32_t reserved;        /* must be 0                                                  */
+  int64_t num_pool_pages;   /* pages per layer slab                                       */
+  int64_t pool_layer_stride;
+  int64_t pool_page_stride;
+  int64_t pool_kv_stride;   /* ignored when F == 1                                        */
+  int64_t pool_token_stride;
+  int64_t pool_head_stride; /* ignored when H == 1                                        */
+  int64_t wire_layer_stride;/* bytes between wire slabs; 0 = caller passes layer's slab   */
+} topkv_layout;
+
+/* One batch of requests. block_table and seq_lens do not depend on the layer
+ * (a page id addresses the same page slot in every layer slab). */
+typedef struct topkv_batch {
+  uint32_t struct_size;          /* = sizeof(topkv_batch)                                   */
+  int32_t num_requests;          /* R >= 0                                                  */
+  int32_t max_pages_per_req;     /* block-table row width (columns)                         */
+  int32_t reserved;              /* must be 0                                               */
+  const int32_t* block_table;    /* DEVICE int32 [R][max_pages_per_req]; columns at or past */
+                                 /* ceil(s_r/P) are ignored (conventionally -1)             */
+  const int32_t* seq_lens;       /* DEVICE int32 [R], each in [0, max_pages_per_req*P]      */
+  const int64_t* cu_seq_lens;    /* DEVICE int64 [R+1] from topkv_build_plan, or NULL: then */
+                                 /* each CTA derives it (allowed for R <= TOPKV_MAX_INLINE_R)*/
+  int64_t total_tokens;          /* T if the host knows it, else -1. When -1 the capacity   */
+                                 /* checks are skipped and the caller guarantees them.      */
+} topkv_batch;
+
+/* Largest R for which cu_seq_lens may be NULL. */
+#define TOPKV_MAX_INLINE_R 1024
+
+/* ---- the four hot-path calls (§3.4 layout, issued per layer as in §5.2) -------------- */
+
+/* Gathers layer `layer` of the batch from the paged pool `src_pool` (base of layer 0) into
+ * the wire slab at d_wire + layer*wire_layer_stride. wire_capacity_bytes is the size of the
+ * whole buffer behind d_wire. Enqueues one kernel on `stream`. */
+int topkv_pack_layer(int layer, const void* src_pool, const topkv_layout* layout,
+                     const topkv_batch* batch, void* d_wire, int64_t wire_capacity_bytes,
+                     topkv_stream_t stream);
+
+/* Inverse of topkv_pack_layer: scatters the wire slab into `dst_pool` through the batch's
+ * (destination) block table. Pool bytes that no valid token addresses are not written.
+ * Precondition (unchecked on the device): no two requests share a destination page. */
+int topkv_unpack_layer(int layer, void* dst_pool, const topkv_layout* layout,
+                       const topkv_batch* batch, const void* d_wire, int64_t wire_bytes,
+                       topkv_stream_t stream);
+
+/* pack with the wire slab landing in caller-owned PINNED host memory `h_pinned`
+ * (slab of layer l at h_pinned + l*wire_layer_stride), the PCIe leg of §3.3.
+ *   d_staging != NULL : kernel packs into d_staging (>= N_layer bytes, device), then one
+ *                       cudaMemcpyAsync device->host on the same stream (copy engine).
+ *   d_staging == NULL : the kernel stores straight into the mapped pinned buffer; h_pinned
+ *                       must be device-accessible at the same address (cudaHostAlloc under
+ *                       unified addressing). Requires batch->total_tokens >= 0 only for the
+ *                       staged form (the copy size must be known on the host). */
+int topkv_pack_layer_to_host(int layer, const void* src_pool, const topkv_layout* layout,
+                             const topkv_batch* batch, void* h_pinned,
+                             int64_t host_capacity_bytes, void* d_staging,
+                             int64_t staging_capacity_bytes, topkv_stream_t stream);
+
+/* unpack with the wire slab read from pinned host memory; same two forms as above
+ * (host->device copy into d_staging then unpack, or direct mapped loads). */
+int topkv_unpack_layer_from_host(int layer, void* dst_pool, const topkv_layout* layout,
+                                 const topkv_batch* batch, const void* h_pinned,
+                                 int64_t host_bytes, void* d_staging,
+                                 int64_t staging_capacity_bytes, topkv_stream_t stream);
+
+/* ---- plan (layer-invariant, once per batch) ------------------------------------------ */
+
+/* Writes the exclusive prefix sum of seq_lens to d_cu_seq_lens (DEVICE int64 [R+1]). */
+int topkv_build_plan(const topkv_batch* batch, int64_t* d_cu_seq_lens, topkv_stream_t stream);
+
+/* Host-side validator for tests and debugging: h_block_table [R][max_pages] and
+ * h_seq_lens [R] are HOST copies. Checks seq_len range, that every used page id lies in
+ * [0, num_pool_pages) and, when require_disjoint != 0, that no page id is used twice
+ * (the unpack precondition). Returns TOPKV_OK or TOPKV_ERR_INVALID_ARG. */
+int topkv_validate_batch_host(const topkv_layout* layout, int32_t num_requests,
+                              int32_t max_pages_per_req, const int32_t* h_block_table,
+                              const int32_t* h_seq_lens, int require_disjoint);
+
+/* ---- size bookkeeping ------------------------------------------------------------------ */
+
+/* Fills the stride fields of *layout for the default page-major pool
+ * pool[l][page][c][t][h][d] from its shape fields; wire_layer_stride is left untouched. */
+int topkv_layout_default_strides(topkv_layout* layout);
+
+/* N_layer = total_tokens * F * H * D * E, or a negative topkv_status. */
+int64_t topkv_wire_layer_bytes(const topkv_layout* layout, int64_t total_tokens);
+
+/* Eq. 1 with the §5.3 MLA rule: F * L * H * D * seq_len * E bytes for one sequence. */
+int64_t topkv_kv_bytes(const topkv_layout* layout, int64_t seq_len);
+
+/* ---- CPU-side analytic helpers (context only; no GPU work) ------------------------------- */
+
+/* Eq. 2: bytes / bandwidth + setup latency, in seconds. */
+double topkv_model_transfer_s(double bytes, double bandwidth_bytes_per_s, double setup_s);
+
+/* Eq. 3: T_eff = max(t_last, t_xfer - t_rem). */
+double topkv_model_t_eff_s(double t_last_s, double t_xfer_s, double t_rem_s);
+
+/* Fraction of t_xfer hidden behind the (layers-1) layers still computing after the first
+ * layer's cache is ready (§5.2 worked example): min(1, (layers-1)*t_layer / t_xfer). */
+double topkv_model_hidden_fraction(int layers, double t_layer_compute_s, double t_xfer_total_s);
+
+/* ---- diagnostics ------------------------------------------------------------------------ */
+
+const char* topkv_strerror(int status);
+int topkv_version(void);
+/* cudaError_t of the most recent failing CUDA call made by this library on this thread. */
+int topkv_last_cuda_error(void);
+/* Number of kernels this library has launched in this process (all threads). */
+int64_t topkv_kernel_launch_count(void);
+/* Selects the kernel family used by the four hot calls: 0 = vectorised load/store,
+ * 1 = bulk-async copies staged through shared memory. Returns the previous value, or
+ * TOPKV_ERR_INVALID_ARG. Process-wide; intended for benchmarking, not for the hot path. */
+int topkv_set_kernel_variant(int variant);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TOPKV_H_ */

@@ -1,0 +1,207 @@
+"""CPU oracle for the paged-KV pack / unpack path — TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import this
+package; the product library never does, and this package never imports the product.
+
+The arithmetic lives in ``topkv_oracle.c`` (plain C, the definition written out); this
+module compiles it with gcc on first use and wraps it for numpy arrays. Symbols follow the
+paper: ``L`` layers, ``h_kv`` KV heads, ``d_h`` head dim, ``b_p`` bytes per element (Eq. 1),
+``F`` = 2 for separate K and V tensors and 1 for a single MLA latent (§5.3).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+WIRE_TOKEN_KV = 0
+WIRE_PLANAR = 1
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "topkv_oracle.c")
+_HDR = os.path.join(_HERE, "topkv_oracle.h")
+_SO = os.path.join(_HERE, "libtopkv_oracle.so")
+
+
+def build(force: bool = False) -> str:
+    """Compiles the C oracle with gcc (no CUDA involved) and returns the path of the .so."""
+    stale = (not os.path.exists(_SO)) or any(
+        os.path.getmtime(p) > os.path.getmtime(_SO) for p in (_SRC, _HDR))
+    if force or stale:
+        tmp = _SO + f".{os.getpid()}.tmp"
+        subprocess.check_call(["gcc", "-O2", "-Wall", "-Wextra", "-shared", "-fPIC", "-o", tmp,
+                               _SRC, "-lpthread"])
+        os.replace(tmp, _SO)
+    return _SO
+
+
+class _Geom(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int64) for n in (
+        "L", "F", "h_kv", "d_h", "b_p", "P", "S_layer", "S_page", "S_kv", "S_tok", "S_head",
+        "W_layer", "wire_order")]
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        i64, f64, vp = ctypes.c_int64, ctypes.c_double, ctypes.c_void_p
+        lib.oracle_kv_bytes.restype = i64
+        lib.oracle_kv_bytes.argtypes = [i64] * 6
+        lib.oracle_transfer_s.restype = f64
+        lib.oracle_transfer_s.argtypes = [f64] * 3
+        lib.oracle_t_eff.restype = f64
+        lib.oracle_t_eff.argtypes = [f64] * 3
+        lib.oracle_hidden_fraction.restype = f64
+        lib.oracle_hidden_fraction.argtypes = [i64, f64, f64]
+        gp = ctypes.POINTER(_Geom)
+        for name in ("oracle_pack_ref", "oracle_unpack_ref"):
+            fn = getattr(lib, name)
+            fn.restype = None
+            fn.argtypes = [gp, i64, vp, i64, i64, vp, vp, vp]
+        for name in ("oracle_pack_rows", "oracle_unpack_rows"):
+            fn = getattr(lib, name)
+            fn.restype = None
+            fn.argtypes = [gp, i64, vp, i64, i64, vp, vp, vp, ctypes.c_int]
+        _lib = lib
+    return _lib
+
+
+@dataclass
+class Geom:
+    """Shape of one paged pool and of the wire format. Strides are in bytes."""
+    L: int
+    F: int
+    h_kv: int
+    d_h: int
+    b_p: int
+    P: int
+    num_pages: int
+    wire_order: int = WIRE_TOKEN_KV
+    S_layer: int = 0
+    S_page: int = 0
+    S_kv: int = 0
+    S_tok: int = 0
+    S_head: int = 0
+    W_layer: int = 0
+
+    def __post_init__(self):
+        if self.S_page == 0:  # default pool: pool[l][page][c][t][h][d], dim contiguous
+            self.S_head = self.d_h * self.b_p
+            self.S_tok = self.h_kv * self.S_head
+            self.S_kv = self.P * self.S_tok
+            self.S_page = self.F * self.S_kv
+            self.S_layer = self.num_pages * self.S_page
+
+    @property
+    def row_bytes(self) -> int:
+        return self.h_kv * self.d_h * self.b_p
+
+    def wire_layer_bytes(self, T: int) -> int:
+        """Bytes of one layer's wire slab for T tokens: every token carries F rows (§3.4)."""
+        return T * self.F * self.row_bytes
+
+    def pool_bytes(self) -> int:
+        return self.L * self.S_layer
+
+    def _c(self) -> _Geom:
+        return _Geom(self.L, self.F, self.h_kv, self.d_h, self.b_p, self.P, self.S_layer,
+                     self.S_page, self.S_kv, self.S_tok, self.S_head, self.W_layer,
+                     self.wire_order)
+
+
+def kv_bytes(L: int, h_kv: int, d_h: int, s: int, b_p: int = 2, F: int = 2) -> int:
+    """Eq. 1 (F = 2), or the MLA form without the K/V factor (F = 1, §5.3)."""
+    return int(_load().oracle_kv_bytes(F, L, h_kv, d_h, s, b_p))
+
+
+def transfer_s(S_bytes: float, B_bytes_per_s: float, L_m_s: float = 0.0) -> float:
+    """Eq. 2."""
+    return float(_load().oracle_transfer_s(S_bytes, B_bytes_per_s, L_m_s))
+
+
+def t_eff(T_last: float, T_xfer: float, T_rem: float) -> float:
+    """Eq. 3."""
+    return float(_load().oracle_t_eff(T_last, T_xfer, T_rem))
+
+
+def hidden_fraction(L: int, t_layer: float, T_xfer: float) -> float:
+    """§5.2 worked example: min(1, (L-1)*t_layer / T_xfer)."""
+    return float(_load().oracle_hidden_fraction(L, t_layer, T_xfer))
+
+
+def _u8(a: np.ndarray, writable: bool) -> np.ndarray:
+    assert a.dtype == np.uint8 and a.ndim == 1 and a.flags.c_contiguous
+    if writable:
+        assert a.flags.writeable
+    return a
+
+
+def _tables(bt: np.ndarray, sl: np.ndarray):
+    bt = np.ascontiguousarray(bt, dtype=np.int32)
+    sl = np.ascontiguousarray(sl, dtype=np.int32)
+    assert bt.ndim == 2 and sl.ndim == 1 and bt.shape[0] == sl.shape[0]
+    return bt, sl
+
+
+def _check_extent(g: Geom, layer: int, pool: np.ndarray, bt, sl, wire: np.ndarray):
+    """Guards the C loops: every offset they will form must lie inside the arrays."""
+    T = int(sl.sum())
+    need_wire = layer * g.W_layer + g.wire_layer_bytes(T)
+    assert wire.size >= need_wire, (wire.size, need_wire)
+    assert 0 <= layer < g.L
+    for r in range(sl.shape[0]):
+        n = -(-int(sl[r]) // g.P)
+        assert n <= bt.shape[1]
+        if n:
+            used = bt[r, :n]
+            assert used.min() >= 0
+            last = (layer * g.S_layer + int(used.max()) * g.S_page + (g.F - 1) * g.S_kv
+                    + (g.P - 1) * g.S_tok + (g.h_kv - 1) * g.S_head + g.d_h * g.b_p)
+            assert pool.size >= last, (pool.size, last)
+
+
+def pack(g: Geom, layer: int, pool: np.ndarray, bt: np.ndarray, sl: np.ndarray,
+         wire: np.ndarray | None = None, impl: str = "ref", threads: int = 1) -> np.ndarray:
+    """wire <- pool through the block table. ``pool`` is the uint8 view from layer 0's base,
+    ``wire`` the uint8 view from layer 0's slab (allocated, zero-filled, if None)."""
+    bt, sl = _tables(bt, sl)
+    T = int(sl.sum())
+    if wire is None:
+        wire = np.zeros(layer * g.W_layer + g.wire_layer_bytes(T), dtype=np.uint8)
+    _u8(pool, False), _u8(wire, True)
+    _check_extent(g, layer, pool, bt, sl, wire)
+    cg = g._c()
+    args = (ctypes.byref(cg), layer, pool.ctypes.data, sl.shape[0], bt.shape[1],
+            bt.ctypes.data, sl.ctypes.data, wire.ctypes.data)
+    if impl == "ref":
+        _load().oracle_pack_ref(*args)
+    elif impl == "rows":
+        _load().oracle_pack_rows(*args, threads)
+    else:
+        raise ValueError(impl)
+    return wire
+
+
+def unpack(g: Geom, layer: int, pool: np.ndarray, bt: np.ndarray, sl: np.ndarray,
+           wire: np.ndarray, impl: str = "ref", threads: int = 1) -> np.ndarray:
+    """pool <- wire through the block table, in place; untouched pool bytes keep their value."""
+    bt, sl = _tables(bt, sl)
+    _u8(pool, True), _u8(wire, False)
+    _check_extent(g, layer, pool, bt, sl, wire)
+    cg = g._c()
+    args = (ctypes.byref(cg), layer, pool.ctypes.data, sl.shape[0], bt.shape[1],
+            bt.ctypes.data, sl.ctypes.data, wire.ctypes.data)
+    if impl == "ref":
+        _load().oracle_unpack_ref(*args)
+    elif impl == "rows":
+        _load().oracle_unpack_rows(*args, threads)
+    else:
+        raise ValueError(impl)
+    return pool

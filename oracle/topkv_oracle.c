@@ -1,0 +1,155 @@
+/*
+ * CPU oracle (see topkv_oracle.h). TEST INFRASTRUCTURE ONLY.
+ *
+ * Pinned by tests/test_oracle_*.py against: the values of Table 1 and Table 4, the §5.2
+ * worked example, a hand-derived miniature, an independently derived inverse index map,
+ * memcpy / row-gather special cases, and round-trip and permutation invariants.
+ * Unpinned parts: none in this file.
+ */
+#include "topkv_oracle.h"
+
+#include <pthread.h>
+#include <stdlib.h>
+#include <string.h>
+
+int64_t oracle_kv_bytes(int64_t F, int64_t L, int64_t h_kv, int64_t d_h, int64_t s, int64_t b_p) {
+  return F * L * h_kv * d_h * s * b_p; /* Eq. 1 with the leading 2 generalised to F (§5.3) */
+}
+
+double oracle_transfer_s(double S_bytes, double B, double L_m) { return S_bytes / B + L_m; } /* Eq. 2 */
+
+double oracle_t_eff(double T_last, double T_xfer, double T_rem) { /* Eq. 3 */
+  double d = T_xfer - T_rem;
+  return T_last > d ? T_last : d;
+}
+
+double oracle_hidden_fraction(int64_t L, double t_layer, double T_xfer) {
+  double T_rem = (double)(L - 1) * t_layer; /* compute left once the first layer is done */
+  double f = T_rem / T_xfer;
+  return f > 1.0 ? 1.0 : f;
+}
+
+/* Pool byte offset of element (l, page, c, t, h, d), byte b. */
+static int64_t poff(const oracle_geom* g, int64_t l, int64_t page, int64_t c, int64_t t,
+                    int64_t h, int64_t d, int64_t b) {
+  return l * g->S_layer + page * g->S_page + c * g->S_kv + t * g->S_tok + h * g->S_head +
+         d * g->b_p + b;
+}
+
+/* Wire byte offset of element (l, global token n = cu_r + i, c, h, d), byte b; T = total tokens. */
+static int64_t woff(const oracle_geom* g, int64_t l, int64_t n, int64_t T, int64_t c, int64_t h,
+                    int64_t d, int64_t b) {
+  int64_t row_bytes = g->h_kv * g->d_h * g->b_p;
+  int64_t row = (g->wire_order == ORACLE_WIRE_PLANAR) ? (c * T + n) : (n * g->F + c);
+  return l * g->W_layer + row * row_bytes + (h * g->d_h + d) * g->b_p + b;
+}
+
+static int64_t total_tokens(int64_t R, const int32_t* sl) {
+  int64_t T = 0;
+  for (int64_t r = 0; r < R; ++r) T += sl[r];
+  return T;
+}
+
+void oracle_pack_ref(const oracle_geom* g, int64_t layer, const uint8_t* pool, int64_t R,
+                     int64_t maxp, const int32_t* bt, const int32_t* sl, uint8_t* wire) {
+  int64_t T = total_tokens(R, sl);
+  int64_t cu = 0;
+  for (int64_t r = 0; r < R; ++r) {
+    for (int64_t i = 0; i < sl[r]; ++i) {
+      int64_t page = bt[r * maxp + i / g->P];
+      int64_t t = i % g->P;
+      for (int64_t c = 0; c < g->F; ++c)
+        for (int64_t h = 0; h < g->h_kv; ++h)
+          for (int64_t d = 0; d < g->d_h; ++d)
+            for (int64_t b = 0; b < g->b_p; ++b)
+              wire[woff(g, layer, cu + i, T, c, h, d, b)] = pool[poff(g, layer, page, c, t, h, d, b)];
+    }
+    cu += sl[r];
+  }
+}
+
+void oracle_unpack_ref(const oracle_geom* g, int64_t layer, uint8_t* pool, int64_t R,
+                       int64_t maxp, const int32_t* bt, const int32_t* sl, const uint8_t* wire) {
+  int64_t T = total_tokens(R, sl);
+  int64_t cu = 0;
+  for (int64_t r = 0; r < R; ++r) {
+    for (int64_t i = 0; i < sl[r]; ++i) {
+      int64_t page = bt[r * maxp + i / g->P];
+      int64_t t = i % g->P;
+      for (int64_t c = 0; c < g->F; ++c)
+        for (int64_t h = 0; h < g->h_kv; ++h)
+          for (int64_t d = 0; d < g->d_h; ++d)
+            for (int64_t b = 0; b < g->b_p; ++b)
+              pool[poff(g, layer, page, c, t, h, d, b)] = wire[woff(g, layer, cu + i, T, c, h, d, b)];
+    }
+    cu += sl[r];
+  }
+}
+
+/* ---- row-memcpy form, threaded over requests ---------------------------------------- */
+
+typedef struct job {
+  const oracle_geom* g;
+  int64_t layer, R, maxp, T;
+  const int32_t *bt, *sl;
+  const int64_t* cu;
+  uint8_t* pool; /* written by unpack only */
+  uint8_t* wire; /* written by pack only   */
+  int pack;
+  int64_t r_begin, r_end;
+} job;
+
+static void* run_job(void* arg) {
+  job* j = (job*)arg;
+  const oracle_geom* g = j->g;
+  size_t head_bytes = (size_t)(g->d_h * g->b_p);
+  for (int64_t r = j->r_begin; r < j->r_end; ++r) {
+    for (int64_t i = 0; i < j->sl[r]; ++i) {
+      int64_t page = j->bt[r * j->maxp + i / g->P];
+      int64_t t = i % g->P;
+      for (int64_t c = 0; c < g->F; ++c)
+        for (int64_t h = 0; h < g->h_kv; ++h) {
+          uint8_t* p = j->pool + poff(g, j->layer, page, c, t, h, 0, 0);
+          uint8_t* w = j->wire + woff(g, j->layer, j->cu[r] + i, j->T, c, h, 0, 0);
+          if (j->pack) memcpy(w, p, head_bytes);
+          else memcpy(p, w, head_bytes);
+        }
+    }
+  }
+  return NULL;
+}
+
+static void run_rows(const oracle_geom* g, int64_t layer, uint8_t* pool, int64_t R, int64_t maxp,
+                     const int32_t* bt, const int32_t* sl, uint8_t* wire, int threads, int pack) {
+  if (threads < 1) threads = 1;
+  if (threads > 256) threads = 256;
+  if (R < threads) threads = R > 0 ? (int)R : 1;
+  int64_t* cu = (int64_t*)malloc(sizeof(int64_t) * (size_t)(R + 1));
+  cu[0] = 0;
+  for (int64_t r = 0; r < R; ++r) cu[r + 1] = cu[r] + sl[r];
+  job jobs[256];
+  pthread_t tid[256];
+  for (int k = 0; k < threads; ++k) {
+    job* j = &jobs[k];
+    j->g = g; j->layer = layer; j->R = R; j->maxp = maxp; j->T = cu[R];
+    j->bt = bt; j->sl = sl; j->cu = cu; j->pool = pool; j->wire = wire; j->pack = pack;
+    j->r_begin = R * k / threads;
+    j->r_end = R * (k + 1) / threads;
+  }
+  for (int k = 1; k < threads; ++k) pthread_create(&tid[k], NULL, run_job, &jobs[k]);
+  run_job(&jobs[0]);
+  for (int k = 1; k < threads; ++k) pthread_join(tid[k], NULL);
+  free(cu);
+}
+
+void oracle_pack_rows(const oracle_geom* g, int64_t layer, const uint8_t* pool, int64_t R,
+                      int64_t maxp, const int32_t* bt, const int32_t* sl, uint8_t* wire,
+                      int threads) {
+  run_rows(g, layer, (uint8_t*)pool, R, maxp, bt, sl, wire, threads, 1);
+}
+
+void oracle_unpack_rows(const oracle_geom* g, int64_t layer, uint8_t* pool, int64_t R,
+                        int64_t maxp, const int32_t* bt, const int32_t* sl, const uint8_t* wire,
+                        int threads) {
+  run_rows(g, layer, pool, R, maxp, bt, sl, (uint8_t*)wire, threads, 0);
+}

@@ -1,0 +1,51 @@
+/*
+ * CPU oracle for the paged-KV pack / unpack path. TEST INFRASTRUCTURE ONLY: it is
+ * called by the tests, by the smoke check and by the benchmark's CPU-baseline leg,
+ * never by the product library, with which it shares no code and no header.
+ *
+ * Everything here is the plain definition written out (the result of pack/unpack is
+ * exactly defined, bit for bit), in the paper's notation:
+ *   L layers, h_kv KV heads, d_h head dim, b_p bytes per element (Eq. 1),
+ *   F = 2 for separate K and V tensors, 1 for a single MLA latent (§5.3).
+ * Serialised layout: per layer, rows of [kv_heads][head_dim] elements, contiguous (§3.4).
+ */
+#ifndef TOPKV_ORACLE_H_
+#define TOPKV_ORACLE_H_
+#include <stdint.h>
+
+enum { ORACLE_WIRE_TOKEN_KV = 0, ORACLE_WIRE_PLANAR = 1 };
+
+typedef struct oracle_geom {
+  int64_t L, F, h_kv, d_h, b_p; /* Eq. 1 symbols (+ F)                            */
+  int64_t P;                    /* tokens per page                                */
+  int64_t S_layer, S_page, S_kv, S_tok, S_head; /* pool strides, bytes            */
+  int64_t W_layer;              /* bytes between wire slabs of consecutive layers */
+  int64_t wire_order;           /* ORACLE_WIRE_*                                  */
+} oracle_geom;
+
+/* Eq. 1 (F = 2) and its MLA form (F = 1, §5.3): F * L * h_kv * d_h * s * b_p. */
+int64_t oracle_kv_bytes(int64_t F, int64_t L, int64_t h_kv, int64_t d_h, int64_t s, int64_t b_p);
+
+/* Eq. 2. */
+double oracle_transfer_s(double S_bytes, double B_bytes_per_s, double L_m_s);
+/* Eq. 3. */
+double oracle_t_eff(double T_last, double T_xfer, double T_rem);
+/* §5.2 worked example: share of T_xfer covered by the (L-1) layers still computing. */
+double oracle_hidden_fraction(int64_t L, double t_layer, double T_xfer);
+
+/* Byte-by-byte definition, one thread. `pool` is the base of layer 0, `wire` the base of
+ * the wire slab of layer 0; bt is int32 [R][maxp] (host), sl is int32 [R] (host). */
+void oracle_pack_ref(const oracle_geom* g, int64_t layer, const uint8_t* pool, int64_t R,
+                     int64_t maxp, const int32_t* bt, const int32_t* sl, uint8_t* wire);
+void oracle_unpack_ref(const oracle_geom* g, int64_t layer, uint8_t* pool, int64_t R,
+                       int64_t maxp, const int32_t* bt, const int32_t* sl, const uint8_t* wire);
+
+/* Same definition, one memcpy per (request, token, plane, head) row of d_h*b_p bytes,
+ * requests split over `threads` POSIX threads. */
+void oracle_pack_rows(const oracle_geom* g, int64_t layer, const uint8_t* pool, int64_t R,
+                      int64_t maxp, const int32_t* bt, const int32_t* sl, uint8_t* wire,
+                      int threads);
+void oracle_unpack_rows(const oracle_geom* g, int64_t layer, uint8_t* pool, int64_t R,
+                        int64_t maxp, const int32_t* bt, const int32_t* sl, const uint8_t* wire,
+                        int threads);
+#endif

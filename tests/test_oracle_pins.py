@@ -1,0 +1,372 @@
+"""Pins the CPU oracle to things other than itself: values the paper prints, a hand-derived
+miniature, an independently derived inverse index map, library special cases and invariants.
+No GPU and no product code is involved here."""
+import bisect
+
+import numpy as np
+import pytest
+
+import oracle
+from oracle import Geom, WIRE_PLANAR, WIRE_TOKEN_KV
+from paper_2607_28633_b200 import workloads as wl
+
+
+# ---------------------------------------------------------------------------- closed forms
+
+def test_table1_kv_sizes(golden):
+    g = golden("paper_values.txt")
+    s, bp = int(g["seq_len"]), int(g["bytes_per_elem"])
+    llama = oracle.kv_bytes(int(g["table1.llama3_70b.layers"]), int(g["table1.llama3_70b.kv_heads"]),
+                            int(g["table1.llama3_70b.head_dim"]), s, bp)
+    assert llama == 1_342_177_280                      # 2*80*8*128*4096*2
+    assert round(llama / 1e9, 1) == float(g["table1.llama3_70b.gb"])
+    mix = oracle.kv_bytes(int(g["table1.mixtral.layers"]), int(g["table1.mixtral.kv_heads"]),
+                          int(g["table1.mixtral.head_dim"]), s, bp)
+    assert mix == 939_524_096
+    assert round(mix / 1e9, 2) == float(g["table1.mixtral.gb"])
+    # MLA: one latent, no K/V factor (§5.3). The printed 0.27 is the binary-GB reading of
+    # 287,834,112 B (0.268 GiB); the decimal reading is 0.288 GB, 7 % above the print.
+    mla = oracle.kv_bytes(int(g["table1.dsv3.layers"]), int(g["table1.dsv3.kv_heads"]),
+                          int(g["table1.dsv3.head_dim"]), s, bp, F=1)
+    assert mla == 287_834_112
+    assert round(mla / 2**30, 2) == float(g["table1.dsv3.gb"])
+    assert abs(mla / 1e9 - float(g["table1.dsv3.gb"])) / float(g["table1.dsv3.gb"]) < 0.07
+    # Had the factor 2 been kept for MLA the print would be missed by 2x:
+    assert round(oracle.kv_bytes(61, 1, 576, s, bp, F=2) / 2**30, 2) != float(g["table1.dsv3.gb"])
+
+
+def test_mla_reduction(golden):
+    g = golden("paper_values.txt")
+    per_tok_mha = oracle.kv_bytes(1, 128, 128, 1, 1, F=2)
+    per_tok_mla = oracle.kv_bytes(1, 1, 576, 1, 1, F=1)
+    assert per_tok_mha == int(g["mha.elems_per_token_layer"])
+    assert per_tok_mla == int(g["mla.elems_per_token_layer"])
+    assert round(per_tok_mha / per_tok_mla) == int(g["mla.reduction"])
+
+
+def test_table4_latencies(golden):
+    g = golden("paper_values.txt")
+    S = float(g["table1.llama3_70b.gb"]) * 1e9
+    for mode in ("nvlink", "pcie", "rdma", "tcp"):
+        ms = oracle.transfer_s(S, float(g[f"table4.{mode}.gbps"]) * 1e9) * 1e3
+        want = float(g[f"table4.{mode}.ms"])
+        assert round(ms, 1 if want < 10 else 0) == want, (mode, ms)
+    assert round(oracle.transfer_s(S, 50e9) * 1e3) == float(g["s22.rate50.ms"])
+    assert round(oracle.transfer_s(S, 900e9) * 1e3, 1) == float(g["s22.rate900.ms"])
+    S_mla = float(g["table1.dsv3.gb"]) * 1e9
+    assert round(oracle.transfer_s(S_mla, 450e9) * 1e3, 1) == float(g["mla.nvlink_ms"])
+    assert round(oracle.transfer_s(S_mla, 25e9) * 1e3) == float(g["mla.rdma_ms"])
+    # setup latency is additive (Eq. 2)
+    assert oracle.transfer_s(1e9, 1e9, 0.25) == pytest.approx(1.25)
+    assert round(25e9 / S, 1) == float(g["demand.ib_req_per_s"])
+
+
+def test_overlap_example(golden):
+    g = golden("paper_values.txt")
+    L, t_layer = int(g["overlap.layers"]), float(g["overlap.layer_ms"]) * 1e-3
+    assert (L - 1) * t_layer * 1e3 == pytest.approx(float(g["overlap.t_rem_ms"]))
+    for mode in ("rdma", "nvlink", "pcie"):
+        T_xfer = float(g[f"table4.{mode}.ms"]) * 1e-3
+        pct = round(100 * oracle.hidden_fraction(L, t_layer, T_xfer))
+        assert pct == int(g[f"overlap.{mode}_hidden_pct"]), mode
+    # Eq. 3: the part of the RDMA transfer that sticks out is 52 - 39.5 = 12.5 ms ...
+    assert oracle.t_eff(0.5e-3, 52e-3, 39.5e-3) == pytest.approx(12.5e-3)
+    # ... and a transfer shorter than the remaining compute floors at T_last.
+    assert oracle.t_eff(0.5e-3, 26e-3, 39.5e-3) == pytest.approx(0.5e-3)
+    assert oracle.t_eff(0.5e-3, 2.9e-3, 39.5e-3) == pytest.approx(0.5e-3)
+
+
+def test_layer_slabs_sum_to_eq1():
+    g = Geom(L=80, F=2, h_kv=8, d_h=128, b_p=2, P=16, num_pages=1)
+    assert g.wire_layer_bytes(4096) == 16_777_216
+    assert 80 * g.wire_layer_bytes(4096) == oracle.kv_bytes(80, 8, 128, 4096)
+    m = Geom(L=61, F=1, h_kv=1, d_h=576, b_p=2, P=64, num_pages=1)
+    assert m.wire_layer_bytes(4096) == 4_718_592
+    assert 61 * m.wire_layer_bytes(4096) == oracle.kv_bytes(61, 1, 576, 4096, F=1)
+
+
+# ---------------------------------------------------------------------------- miniature
+
+def _rows(txt):
+    return [int(x) for x in txt.split()]
+
+
+def _mini():
+    g = Geom(L=1, F=2, h_kv=1, d_h=8, b_p=2, P=2, num_pages=4)
+    assert (g.S_tok, g.S_kv, g.S_page, g.S_layer) == (16, 32, 64, 256)
+    pool = (np.arange(256) % 251).astype(np.uint8)
+    sl = np.array([3, 1], dtype=np.int32)
+    bt_src = np.array([[2, 0], [3, -1]], dtype=np.int32)
+    bt_dst = np.array([[1, 3], [0, -1]], dtype=np.int32)
+    return g, pool, sl, bt_src, bt_dst
+
+
+@pytest.mark.parametrize("impl", ["ref", "rows"])
+def test_miniature_pack(golden, impl):
+    gold = golden("miniature_pack.txt")
+    g, pool, sl, bt_src, _ = _mini()
+    for order, key in ((WIRE_TOKEN_KV, "wire_token_kv_rows"), (WIRE_PLANAR, "wire_planar_rows")):
+        g.wire_order = order
+        wire = oracle.pack(g, 0, pool, bt_src, sl, impl=impl)
+        want = np.concatenate([pool[o:o + 16] for o in _rows(gold[key])])
+        assert wire.size == 128 and np.array_equal(wire, want), key
+    # rows that must never reach the wire: poison them, the wire must not change
+    g.wire_order = WIRE_TOKEN_KV
+    before = oracle.pack(g, 0, pool, bt_src, sl, impl=impl)
+    poisoned = pool.copy()
+    for o in _rows(gold["never_read_rows"]):
+        poisoned[o:o + 16] ^= 0xFF
+    assert np.array_equal(oracle.pack(g, 0, poisoned, bt_src, sl, impl=impl), before)
+
+
+@pytest.mark.parametrize("impl", ["ref", "rows"])
+def test_miniature_unpack(golden, impl):
+    gold = golden("miniature_pack.txt")
+    g, pool, sl, bt_src, bt_dst = _mini()
+    wire = oracle.pack(g, 0, pool, bt_src, sl, impl=impl)
+    dst = np.full(256, 0xEE, dtype=np.uint8)
+    oracle.unpack(g, 0, dst, bt_dst, sl, wire, impl=impl)
+    for k, o in enumerate(_rows(gold["unpack_dst_rows"])):
+        assert np.array_equal(dst[o:o + 16], wire[16 * k:16 * k + 16]), (k, o)
+    for o in _rows(gold["unpack_untouched"]):
+        assert (dst[o:o + 16] == 0xEE).all(), o
+    touched = set(_rows(gold["unpack_dst_rows"])) | set(_rows(gold["unpack_untouched"]))
+    assert touched == set(range(0, 256, 16))
+
+
+# ---------------------------------------------------------------- independent inverse map
+
+def inverse_pack(g: Geom, layer, pool, bt, sl):
+    """Second derivation of pack, written from the wire side: walks the wire bytes in order
+    and inverts the layout (wire byte k -> request, token, plane, head, dim, byte) by div/mod
+    and a binary search in the prefix sums. Shares nothing with the C loops."""
+    cu = np.concatenate([[0], np.cumsum(sl.astype(np.int64))]).tolist()
+    T = cu[-1]
+    row = g.h_kv * g.d_h * g.b_p
+    n_bytes = T * g.F * row
+    out = np.zeros(layer * g.W_layer + n_bytes, dtype=np.uint8)
+    for k in range(n_bytes):
+        q, inner = divmod(k, row)
+        if g.wire_order == WIRE_PLANAR:
+            c, n = divmod(q, T)
+        else:
+            n, c = divmod(q, g.F)
+        r = bisect.bisect_right(cu, n) - 1
+        i = n - cu[r]
+        e, b = divmod(inner, g.b_p)
+        h, d = divmod(e, g.d_h)
+        page = int(bt[r, i // g.P])
+        src = (layer * g.S_layer + page * g.S_page + c * g.S_kv + (i % g.P) * g.S_tok
+               + h * g.S_head + d * g.b_p + b)
+        out[layer * g.W_layer + k] = pool[src]
+    return out
+
+
+def _random_case(seed, F, h_kv, d_h, P, strided):
+    rng = np.random.default_rng(seed)
+    L, b_p = 2, 2
+    R = int(rng.integers(1, 5))
+    sl = rng.integers(0, 3 * P + 2, size=R).astype(np.int32)
+    if seed % 3 == 0:
+        sl[int(rng.integers(0, R))] = 0                      # an empty request
+    pages = (sl + P - 1) // P
+    maxp = max(int(pages.max()), 1) + 1
+    npages = int(pages.sum()) + 3
+    g = Geom(L=L, F=F, h_kv=h_kv, d_h=d_h, b_p=b_p, P=P, num_pages=npages)
+    if strided:  # plane-major pool with padded tokens: pool[l][c][page][t(+pad)][h][d]
+        g.S_head = d_h * b_p
+        g.S_tok = h_kv * g.S_head + 16
+        g.S_page = P * g.S_tok
+        g.S_kv = npages * g.S_page
+        g.S_layer = F * g.S_kv + 32
+    T = int(sl.sum())
+    g.W_layer = g.wire_layer_bytes(T) + 48
+    perm = rng.permutation(npages)
+    bt = np.full((R, maxp), -1, dtype=np.int32)
+    pos = 0
+    for r in range(R):
+        bt[r, :pages[r]] = perm[pos:pos + pages[r]]
+        pos += pages[r]
+    pool = rng.integers(0, 256, size=g.L * g.S_layer, dtype=np.uint8)
+    return g, pool, bt, sl
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_pack_matches_inverse_map(seed):
+    F = 1 if seed % 4 == 3 else 2
+    h_kv, d_h, P = [(2, 8, 4), (1, 24, 3), (3, 8, 2), (1, 40, 5)][seed % 4]
+    g, pool, bt, sl = _random_case(seed, F, h_kv, d_h, P, strided=seed % 2 == 1)
+    for order in (WIRE_TOKEN_KV, WIRE_PLANAR):
+        g.wire_order = order
+        for layer in range(g.L):
+            want = inverse_pack(g, layer, pool, bt, sl)
+            for impl in ("ref", "rows"):
+                got = oracle.pack(g, layer, pool, bt, sl, wire=np.zeros_like(want), impl=impl,
+                                  threads=3)
+                assert np.array_equal(got, want), (order, layer, impl)
+
+
+# ---------------------------------------------------------------- library special cases
+
+def test_identity_table_is_memcpy():
+    # full pages, identity block table, one plane per page run => the wire is the slab prefix
+    g = Geom(L=3, F=1, h_kv=1, d_h=24, b_p=2, P=4, num_pages=10)
+    pool = np.random.default_rng(1).integers(0, 256, g.pool_bytes(), dtype=np.uint8)
+    sl = np.array([8, 12, 4], dtype=np.int32)
+    bt = np.array([[0, 1, -1], [2, 3, 4], [5, -1, -1]], dtype=np.int32)
+    for layer in range(3):
+        wire = oracle.pack(g, layer, pool, bt, sl)
+        lo = layer * g.S_layer
+        assert np.array_equal(wire, pool[lo:lo + 24 * g.row_bytes])
+
+
+def test_page_size_one_is_row_gather():
+    # P = 1, PLANAR: K plane == pool rows fancy-indexed by the flattened block table
+    g = Geom(L=1, F=2, h_kv=2, d_h=8, b_p=2, P=1, num_pages=32, wire_order=WIRE_PLANAR)
+    rng = np.random.default_rng(2)
+    pool = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
+    sl = np.array([5, 0, 7], dtype=np.int32)
+    perm = rng.permutation(32).astype(np.int32)
+    bt = np.full((3, 7), -1, dtype=np.int32)
+    bt[0, :5], bt[2, :7] = perm[:5], perm[5:12]
+    flat = np.concatenate([bt[0, :5], bt[2, :7]])
+    pages = pool.reshape(32, 2, g.row_bytes)          # [page][K|V][row]
+    wire = oracle.pack(g, 0, pool, bt, sl)
+    assert np.array_equal(wire[:12 * g.row_bytes], pages[flat, 0].reshape(-1))
+    assert np.array_equal(wire[12 * g.row_bytes:], pages[flat, 1].reshape(-1))
+
+
+def test_numpy_gather_third_opinion_cfg1():
+    # the tiny benchmark configuration against a vectorised numpy formulation
+    b = wl.make_batch(wl.CFG1)
+    s = b.spec
+    g = Geom(L=s.L, F=s.F, h_kv=s.H, d_h=s.D, b_p=s.E, P=s.P, num_pages=b.num_pool_pages)
+    assert b.total_tokens == 436 and b.pages_needed == 29
+    assert g.wire_layer_bytes(b.total_tokens) == 1_785_856
+    g.W_layer = g.wire_layer_bytes(b.total_tokens)
+    pool = wl.fill_numpy(g.pool_bytes(), b.seeds["data"])
+    view = pool.reshape(s.L, b.num_pool_pages, s.F, s.P, g.row_bytes)
+    for layer in range(s.L):
+        parts = []
+        for r in range(s.R):
+            i = np.arange(b.seq_lens[r])
+            pg = b.src_block_table[r, i // s.P]
+            parts.append(view[layer, pg, :, i % s.P, :])       # [tok][K|V][row]
+        want = np.concatenate(parts).reshape(-1)
+        wire = np.zeros(s.L * g.W_layer, dtype=np.uint8)
+        for impl in ("ref", "rows"):
+            got = oracle.pack(g, layer, pool, b.src_block_table, b.seq_lens, wire=wire.copy(),
+                              impl=impl, threads=4)
+            assert np.array_equal(got[layer * g.W_layer:(layer + 1) * g.W_layer], want)
+            other = got.copy()
+            other[layer * g.W_layer:(layer + 1) * g.W_layer] = 0
+            assert not other.any()                              # only this layer's slab written
+
+
+def test_mla_is_gqa_with_one_plane():
+    rng = np.random.default_rng(5)
+    g1 = Geom(L=1, F=1, h_kv=1, d_h=576, b_p=2, P=4, num_pages=6)
+    # the same bytes seen as a 9-head, 64-dim, single-plane cache
+    g2 = Geom(L=1, F=1, h_kv=9, d_h=64, b_p=2, P=4, num_pages=6)
+    pool = rng.integers(0, 256, g1.pool_bytes(), dtype=np.uint8)
+    sl = np.array([6, 9], dtype=np.int32)
+    bt = np.array([[4, 1, -1], [0, 5, 2]], dtype=np.int32)
+    assert np.array_equal(oracle.pack(g1, 0, pool, bt, sl), oracle.pack(g2, 0, pool, bt, sl))
+
+
+# ---------------------------------------------------------------- invariants
+
+@pytest.mark.parametrize("seed", range(6))
+def test_round_trip_and_untouched(seed):
+    g, pool, bt_src, sl = _random_case(100 + seed, 2, 2, 8, 4, strided=seed % 2 == 0)
+    rng = np.random.default_rng(seed)
+    pages = (sl + g.P - 1) // g.P
+    perm = rng.permutation(g.num_pages)
+    bt_dst = np.full_like(bt_src, -1)
+    pos = 0
+    for r in range(sl.shape[0]):
+        bt_dst[r, :pages[r]] = perm[pos:pos + pages[r]]
+        pos += pages[r]
+    for order in (WIRE_TOKEN_KV, WIRE_PLANAR):
+        g.wire_order = order
+        for layer in range(g.L):
+            wire = oracle.pack(g, layer, pool, bt_src, sl)
+            fill = rng.integers(0, 256, pool.size, dtype=np.uint8)
+            dst = fill.copy()
+            oracle.unpack(g, layer, dst, bt_dst, sl, wire)
+            # pack(dst) gives back the same wire
+            again = oracle.pack(g, layer, dst, bt_dst, sl)
+            assert np.array_equal(again, wire)
+            # number of changed-or-addressed bytes: exactly the valid rows were written
+            mask = np.zeros(pool.size, dtype=bool)
+            for r in range(sl.shape[0]):
+                for i in range(sl[r]):
+                    for c in range(g.F):
+                        for h in range(g.h_kv):
+                            o = (layer * g.S_layer + int(bt_dst[r, i // g.P]) * g.S_page
+                                 + c * g.S_kv + (i % g.P) * g.S_tok + h * g.S_head)
+                            mask[o:o + g.d_h * g.b_p] = True
+            assert np.array_equal(dst[~mask], fill[~mask])
+            assert mask.sum() == g.wire_layer_bytes(int(sl.sum()))
+    # unpack through the SOURCE table into a copy of the source is the identity
+    g.wire_order = WIRE_TOKEN_KV
+    same = pool.copy()
+    oracle.unpack(g, 0, same, bt_src, sl, oracle.pack(g, 0, pool, bt_src, sl))
+    assert np.array_equal(same, pool)
+
+
+def test_consistent_page_permutation_leaves_wire_unchanged():
+    g, pool, bt, sl = _random_case(7, 2, 2, 8, 4, strided=False)
+    sigma = np.random.default_rng(3).permutation(g.num_pages)        # old page -> new page
+    view = pool.reshape(g.L, g.num_pages, g.S_page)
+    moved = np.empty_like(view)
+    moved[:, sigma] = view
+    bt2 = np.where(bt >= 0, sigma[np.clip(bt, 0, None)], -1).astype(np.int32)
+    for layer in range(g.L):
+        assert np.array_equal(oracle.pack(g, layer, pool, bt, sl),
+                              oracle.pack(g, layer, moved.reshape(-1), bt2, sl))
+
+
+def test_wire_rows_are_the_valid_source_rows():
+    g, pool, bt, sl = _random_case(9, 2, 1, 8, 4, strided=False)
+    wire = oracle.pack(g, 0, pool, bt, sl)
+    rows_w = sorted(bytes(wire[o:o + g.row_bytes]) for o in range(0, wire.size, g.row_bytes))
+    rows_s = []
+    for r in range(sl.shape[0]):
+        for i in range(sl[r]):
+            for c in range(g.F):
+                o = int(bt[r, i // g.P]) * g.S_page + c * g.S_kv + (i % g.P) * g.S_tok
+                rows_s.append(bytes(pool[o:o + g.row_bytes]))
+    assert rows_w == sorted(rows_s)
+
+
+def test_concatenated_batches_concatenate_wires():
+    seed = 11
+    while True:
+        g, pool, bt, sl = _random_case(seed, 2, 2, 8, 4, strided=False)
+        R = sl.shape[0]
+        if R >= 2:
+            break
+        seed += 1
+    k = R // 2
+    a = oracle.pack(g, 0, pool, bt[:k], sl[:k])
+    b = oracle.pack(g, 0, pool, bt[k:], sl[k:])
+    assert np.array_equal(np.concatenate([a, b]), oracle.pack(g, 0, pool, bt, sl))
+
+
+def test_rows_impl_threads_agree_with_ref_on_cfg1():
+    b = wl.make_batch(wl.CFG1)
+    s = b.spec
+    g = Geom(L=s.L, F=s.F, h_kv=s.H, d_h=s.D, b_p=s.E, P=s.P, num_pages=b.num_pool_pages)
+    pool = wl.fill_numpy(g.pool_bytes(), b.seeds["data"])
+    for order in (WIRE_TOKEN_KV, WIRE_PLANAR):
+        g.wire_order = order
+        ref = oracle.pack(g, 1, pool, b.src_block_table, b.seq_lens)
+        for th in (1, 2, 8):
+            assert np.array_equal(ref, oracle.pack(g, 1, pool, b.src_block_table, b.seq_lens,
+                                                   impl="rows", threads=th))
+        dst_a = wl.fill_numpy(g.pool_bytes(), b.seeds["dst_fill"])
+        dst_b = dst_a.copy()
+        oracle.unpack(g, 1, dst_a, b.dst_block_table, b.seq_lens, ref)
+        oracle.unpack(g, 1, dst_b, b.dst_block_table, b.seq_lens, ref, impl="rows", threads=3)
+        assert np.array_equal(dst_a, dst_b)
