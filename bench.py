@@ -1,0 +1,525 @@
+#!/usr/bin/env python
+"""Benchmark of the TopKV data plane on B200.
+
+A "step" is one pass of the hot path over one synthetic batch: the plan (prefix sums), then
+pack of every layer, then unpack of every layer, device to device. The headline workload is
+the Llama-3-8B-shaped cache (16 requests, 512..4096 tokens, 32 layers). The same JSON line
+also carries the host-leg (PCIe) figure as ``e2e``, the live roofline of the pack kernel, the
+CPU oracle timed on this machine as ``cpu_baseline``, and, at one GPU, the other benchmark shapes
+(70B GQA with its host leg, DeepSeek-V3 MLA) and the side-stream overlap run under ``extra``.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--extras ...]
+
+With N > 1 (launched by torchrun) every rank runs its own batch (weak scaling, no data-path
+collective); the time is the max over ranks, the value the sum of bytes over that time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "kv_pack_unpack_GBps"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic of one pack launch relative to its algorithmic bytes, from the ncu capture
+# summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over 2*N_layer).
+# None until a capture exists.
+NCU_TRAFFIC_RATIO = None
+
+
+def measured_peak_gbs():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (6650 GB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap,power.draw")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.t.join(timeout=2)
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx = float(r[1])
+                for n, v in zip(names, r[2:6]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                pass
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def host_cores():
+    return len(os.sched_getaffinity(0))
+
+
+def oracle_sample(spec, batch, seconds_target=12.0):
+    """Times the CPU oracle (row-memcpy form, all cores) on whole layers of this workload until
+    about ``seconds_target`` of wall time has passed. Returns (GB/s, layers timed, cores)."""
+    import numpy as np
+    import oracle
+    from paper_2607_28633_b200 import workloads as wl
+    cores = host_cores()
+    g = oracle.Geom(L=1, F=spec.F, h_kv=spec.H, d_h=spec.D, b_p=spec.E, P=spec.P,
+                    num_pages=batch.num_pool_pages)
+    src = wl.fill_numpy(g.pool_bytes(), batch.seeds["data"], raw_bits=True)
+    dst = np.zeros_like(src)
+    n_layer = g.wire_layer_bytes(batch.total_tokens)
+    wire = np.zeros(n_layer, dtype=np.uint8)
+    oracle.pack(g, 0, src, batch.src_block_table, batch.seq_lens, wire=wire, impl="rows",
+                threads=cores)  # touch every page once (first-touch faults are not the oracle)
+    oracle.unpack(g, 0, dst, batch.dst_block_table, batch.seq_lens, wire, impl="rows", threads=cores)
+    t0, n = time.perf_counter(), 0
+    while True:
+        oracle.pack(g, 0, src, batch.src_block_table, batch.seq_lens, wire=wire, impl="rows",
+                    threads=cores)
+        oracle.unpack(g, 0, dst, batch.dst_block_table, batch.seq_lens, wire, impl="rows",
+                      threads=cores)
+        n += 1
+        dt = time.perf_counter() - t0
+        if dt >= seconds_target or n >= 64:
+            break
+    return 4.0 * n_layer * n / dt / 1e9, n, cores, dt
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle as it stands, on this machine's host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2607_28633_b200 import workloads as wl
+    spec = wl.CFG2
+    batch = wl.make_batch(spec)
+    per_step = max(1.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        oracle_sample(spec, batch, seconds_target=per_step)
+    vals, times = [], []
+    for _ in range(args.steps):
+        v, n, cores, dt = oracle_sample(spec, batch, seconds_target=per_step)
+        vals.append(v)
+        times.append(dt / n * spec.L)   # a full step = all L layers at the sampled rate
+    value = statistics.mean(vals)
+    sample = f"{n} layer(s) of {spec.L} per step (pack+unpack), rows-memcpy oracle, {cores} threads"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": UNIT,
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": round(statistics.mean(times) * 1e3, 3), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": workload_config(spec, batch),
+        "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0,
+                "d2h_bytes_per_step": 0},
+    }))
+
+
+def workload_config(spec, batch):
+    return {"workload": spec.name, "note": spec.note, "layers": spec.L, "requests": spec.R,
+            "total_tokens": batch.total_tokens, "page_tokens": spec.P,
+            "wire_bytes_per_layer": batch.total_tokens * spec.tok_bytes,
+            "pool_pages": batch.num_pool_pages,
+            "l2": "inputs larger than L2: every layer touches distinct memory and all packs "
+                  "precede all unpacks, so no slab is re-read from L2"}
+
+
+def time_phase(stream, fn):
+    import torch
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    fn()
+    b.record(stream)
+    return a, b
+
+
+def bench_d2d(w, stream, steps, warmup, barrier):
+    """Times K steps of plan + pack(all layers) + unpack(all layers). Returns per-step ms
+    (whole region / K), and the summed pack-phase and unpack-phase ms."""
+    import torch
+    from paper_2607_28633_b200 import binding as tk
+    L = w.layers
+    plan_batch = tk.make_batch(w.src_bt, w.seq_lens)
+
+    def step(rec):
+        tk.check(tk.topkv_build_plan(plan_batch, w.cu, stream))
+        e0 = torch.cuda.Event(enable_timing=True); e0.record(stream)
+        for l in range(L):
+            w.pack(l, stream)
+        e1 = torch.cuda.Event(enable_timing=True); e1.record(stream)
+        for l in range(L):
+            w.unpack(l, stream)
+        e2 = torch.cuda.Event(enable_timing=True); e2.record(stream)
+        if rec is not None:
+            rec.append((e0, e1, e2))
+
+    for _ in range(warmup):
+        step(None)
+    stream.synchronize()
+    barrier()
+    rec = []
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = tk.topkv_kernel_launch_count()
+    t0.record(stream)
+    for _ in range(steps):
+        step(rec)
+    t1.record(stream)
+    stream.synchronize()
+    launches = tk.topkv_kernel_launch_count() - launches0
+    total_ms = t0.elapsed_time(t1)
+    pack_ms = sum(a.elapsed_time(b) for a, b, _ in rec)
+    unpack_ms = sum(b.elapsed_time(c) for _, b, c in rec)
+    return total_ms / steps, pack_ms / steps, unpack_ms / steps, launches
+
+
+def bench_host_leg(w, stream, pinned, staging, steps, warmup, barrier, slots):
+    """pack_to_host for all layers then unpack_from_host for all layers, through pinned host
+    memory (``slots`` slabs used as a ring). Returns ms per step and the two phase times."""
+    import ctypes
+    import torch
+    from paper_2607_28633_b200 import binding as tk
+    L, n = w.layers, w.n_layer
+    lo = type(w.layout)()
+    ctypes.memmove(ctypes.byref(lo), ctypes.byref(w.layout), ctypes.sizeof(lo))
+    lo.wire_layer_stride = 0
+    cap = 0 if staging is None else staging.numel()
+
+    def step(rec):
+        e0 = torch.cuda.Event(enable_timing=True); e0.record(stream)
+        for l in range(L):
+            slab = pinned[(l % slots) * n:(l % slots + 1) * n]
+            tk.check(tk.topkv_pack_layer_to_host(l, w.src_pool, lo, w.src_batch, slab, n, staging,
+                                                 cap, stream))
+        e1 = torch.cuda.Event(enable_timing=True); e1.record(stream)
+        for l in range(L):
+            slab = pinned[(l % slots) * n:(l % slots + 1) * n]
+            tk.check(tk.topkv_unpack_layer_from_host(l, w.dst_pool, lo, w.dst_batch, slab, n,
+                                                     staging, cap, stream))
+        e2 = torch.cuda.Event(enable_timing=True); e2.record(stream)
+        if rec is not None:
+            rec.append((e0, e1, e2))
+
+    for _ in range(warmup):
+        step(None)
+    stream.synchronize()
+    barrier()
+    rec = []
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record(stream)
+    for _ in range(steps):
+        step(rec)
+    t1.record(stream)
+    stream.synchronize()
+    total = t0.elapsed_time(t1) / steps
+    to_host = sum(a.elapsed_time(b) for a, b, _ in rec) / steps
+    from_host = sum(b.elapsed_time(c) for _, b, c in rec) / steps
+    return total, to_host, from_host
+
+
+def pinned_copy_baseline(dev, stream, nbytes, reps=5):
+    """cudaMemcpyAsync of one slab between pinned host and device memory (torch copy_), GB/s."""
+    import torch
+    h = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
+    d = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    out = {}
+    with torch.cuda.stream(stream):
+        for name, (dst, src) in (("d2h", (h, d)), ("h2d", (d, h))):
+            dst.copy_(src, non_blocking=True)
+            stream.synchronize()
+            best = 1e30
+            for _ in range(reps):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                dst.copy_(src, non_blocking=True)
+                b.record(stream)
+                stream.synchronize()
+                best = min(best, a.elapsed_time(b))
+            out[name] = nbytes / (best * 1e-3) / 1e9
+    return out
+
+
+def device_copy_baseline(dev, stream, nbytes, reps=10):
+    """Plain device-to-device copy of nbytes (torch copy_), read+write GB/s, best of reps."""
+    import torch
+    a_ = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    b_ = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    best = 1e30
+    with torch.cuda.stream(stream):
+        for _ in range(3):
+            b_.copy_(a_)
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            b_.copy_(a_)
+            b.record(stream)
+            stream.synchronize()
+            best = min(best, a.elapsed_time(b))
+    return 2 * nbytes / (best * 1e-3) / 1e9
+
+
+def run_extra(name, dev, stream, args, peak):
+    """Other benchmark shapes at one GPU; returns a dict for the ``extra`` object."""
+    import torch
+    from paper_2607_28633_b200 import harness, overlap
+    from paper_2607_28633_b200 import workloads as wl
+    spec = wl.ALL[name]
+    nobar = lambda: None
+    out = {"workload": spec.name}
+    if name in ("cfg3", "cfg4"):
+        w = harness.setup(spec, dev, fill_dst=False)
+        ms, pack_ms, unpack_ms, _ = bench_d2d(w, stream, args.steps, args.warmup, nobar)
+        traffic = 2.0 * w.n_layer * w.layers
+        out.update({"pack_GBps": round(traffic / (pack_ms * 1e-3) / 1e9, 1),
+                    "unpack_GBps": round(traffic / (unpack_ms * 1e-3) / 1e9, 1),
+                    "pack_frac_of_peak": round(traffic / (pack_ms * 1e-3) / 1e9 / peak, 4),
+                    "unpack_frac_of_peak": round(traffic / (unpack_ms * 1e-3) / 1e9 / peak, 4),
+                    "ms_per_step": round(ms, 4), "wire_bytes_per_layer": w.n_layer,
+                    "layers": w.layers})
+        if name == "cfg3":
+            slots = w.layers
+            try:
+                pinned = torch.empty(slots * w.n_layer, dtype=torch.uint8, pin_memory=True)
+            except Exception:
+                slots = 4
+                pinned = torch.empty(slots * w.n_layer, dtype=torch.uint8, pin_memory=True)
+            staging = torch.empty(w.n_layer, dtype=torch.uint8, device=dev)
+            base = pinned_copy_baseline(dev, stream, w.n_layer)
+            hs = max(1, min(args.steps, 3))
+            for form, st in (("staged", staging), ("direct", None)):
+                _, th, fh = bench_host_leg(w, stream, pinned, st, hs, 1, nobar, slots)
+                d2h = w.n_layer * w.layers / (th * 1e-3) / 1e9
+                h2d = w.n_layer * w.layers / (fh * 1e-3) / 1e9
+                out[f"host_leg_{form}"] = {
+                    "to_host_GBps": round(d2h, 2), "from_host_GBps": round(h2d, 2),
+                    "to_host_frac_of_pinned_copy": round(d2h / base["d2h"], 4),
+                    "from_host_frac_of_pinned_copy": round(h2d / base["h2d"], 4)}
+            out["pinned_copy_GBps"] = {k: round(v, 2) for k, v in base.items()}
+            out["pinned_slots"] = slots
+            del pinned, staging
+        del w
+    elif name == "cfg5":
+        w = harness.setup(spec, dev, need_dst=False, need_wire=False)
+        slots = w.layers
+        try:
+            pinned = torch.empty(slots * w.n_layer, dtype=torch.uint8, pin_memory=True)
+        except Exception:
+            slots = 8
+            pinned = torch.empty(slots * w.n_layer, dtype=torch.uint8, pin_memory=True)
+        staging = torch.empty(w.n_layer, dtype=torch.uint8, device=dev)
+        pre = overlap.PrefillStandIn(dev, w.batch.seeds["data"] + 50)
+        best = None
+        for form, st in (("staged", staging), ("direct", None)):
+            r = overlap.run_overlap(w, pinned, st, pre, slots=slots)
+            d = r.as_dict()
+            d["form"] = form
+            d["hidden_model"] = round(min(1.0, (r.layers - 1) * r.t_layer_compute_ms
+                                          / r.t_xfer_serial_ms), 6)
+            d["prefill_tflops_alone"] = round(pre.flop_per_layer / (r.t_layer_compute_ms * 1e-3)
+                                              / 1e12, 1)
+            out[form] = d
+            if best is None or d["hidden"] > out[best]["hidden"]:
+                best = form
+        out["best_form"] = best
+        out["hidden_fraction"] = out[best]["hidden"]
+        out["pinned_slots"] = slots
+        del w, pinned, staging, pre
+    torch.cuda.empty_cache()
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="topkv", choices=["topkv", "reference"])
+    ap.add_argument("--extras", default="cfg5,cfg3,cfg4",
+                    help="comma list of extra workloads measured at one GPU ('' for none)")
+    ap.add_argument("--variant", type=int, default=None, help="kernel family (see topkv.h)")
+    ap.add_argument("--layers", type=int, default=None, help="fewer layers (profiling only)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import __graft_entry__ as entry
+    from paper_2607_28633_b200 import binding as tk
+    from paper_2607_28633_b200 import harness
+    from paper_2607_28633_b200 import workloads as wl
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the TopKV path has no CPU fallback")
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if rank == 0:
+        entry.build()
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.barrier()
+    tk.lib()
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    if args.variant is not None:
+        tk.check(tk.topkv_set_kernel_variant(args.variant))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    def max_over_ranks(x: float) -> float:
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def sum_over_ranks(x: float) -> float:
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        return float(t.item())
+
+    peak, peak_src = measured_peak_gbs()
+    spec = wl.CFG2 if args.layers is None else wl.with_layers(wl.CFG2, args.layers)
+    w = harness.setup(spec, dev, rank=rank, fill_dst=False)
+    stream = torch.cuda.Stream(dev)
+    L, n_layer = w.layers, w.n_layer
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    ms, pack_ms, unpack_ms, launches = bench_d2d(w, stream, args.steps, args.warmup, barrier)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+
+    ms_max = max_over_ranks(ms)
+    bytes_step_all = sum_over_ranks(4.0 * n_layer * L)        # pack r+w, unpack r+w
+    value = bytes_step_all / (ms_max * 1e-3) / 1e9
+    pack_launch_ms = pack_ms / L
+    unpack_launch_ms = unpack_ms / L
+    achieved = 2.0 * n_layer / (pack_launch_ms * 1e-3) / 1e9
+    achieved_unpack = 2.0 * n_layer / (unpack_launch_ms * 1e-3) / 1e9
+
+    e2e = None
+    if not args.no_e2e:
+        slots = L
+        try:
+            pinned = torch.empty(slots * n_layer, dtype=torch.uint8, pin_memory=True)
+        except Exception:
+            slots = 4
+            pinned = torch.empty(slots * n_layer, dtype=torch.uint8, pin_memory=True)
+        staging = torch.empty(n_layer, dtype=torch.uint8, device=dev)
+        hs = max(1, min(args.steps, 3))
+        ems, th, fh = bench_host_leg(w, stream, pinned, staging, hs, 1, barrier, slots)
+        ems_max = max_over_ranks(ems)
+        e2e = {"value": round(bytes_step_all / (ems_max * 1e-3) / 1e9, 3), "unit": UNIT,
+               "h2d_bytes_per_step": n_layer * L, "d2h_bytes_per_step": n_layer * L,
+               "form": "staged (kernel + copy engine)", "steps": hs,
+               "to_host_link_GBps": round(n_layer * L / (th * 1e-3) / 1e9, 2),
+               "from_host_link_GBps": round(n_layer * L / (fh * 1e-3) / 1e9, 2)}
+        del pinned, staging
+
+    extra = {}
+    if rank == 0 and world == 1:
+        extra["device_copy_GBps_same_bytes"] = round(device_copy_baseline(dev, stream, n_layer), 1)
+    batch = w.batch
+    del w
+    torch.cuda.empty_cache()
+    if world == 1 and args.extras:
+        for name in [x for x in args.extras.split(",") if x]:
+            try:
+                extra[name] = run_extra(name, dev, stream, args, peak)
+            except Exception as e:  # an extra must not take the headline line down
+                extra[name] = {"error": f"{type(e).__name__}: {e}"}
+                torch.cuda.empty_cache()
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, n, cores, dt = oracle_sample(wl.CFG2, wl.make_batch(wl.CFG2), seconds_target=12.0)
+        cpu = {"value": round(v, 3), "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"{n} layer(s) of {wl.CFG2.L} of this workload, pack+unpack, "
+                         f"rows-memcpy oracle, {dt:.1f} s"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_max, 4),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
+            "data": "synthetic", "config": workload_config(spec, batch),
+            "gpu_launches": int(launches), "clocks": clocks,
+            "roofline": {"bound": "hbm", "kernel": "topkv_page_copy_kernel (pack)",
+                         "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                         "frac": round(achieved / peak, 4), "peak_source": peak_src,
+                         "frac_of_8000_spec": round(achieved / 8000.0, 4),
+                         "bytes_per_launch": 2 * n_layer,
+                         "launch_ms": round(pack_launch_ms, 5),
+                         "traffic": (None if NCU_TRAFFIC_RATIO is None
+                                     else int(NCU_TRAFFIC_RATIO * 2 * n_layer)),
+                         "unpack_achieved": round(achieved_unpack, 1),
+                         "unpack_frac": round(achieved_unpack / peak, 4)},
+            "e2e": e2e, "cpu_baseline": cpu, "extra": extra,
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

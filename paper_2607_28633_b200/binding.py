@@ -1,0 +1,244 @@
+"""ctypes binding of the TopKV C-ABI library (``include/topkv.h``).
+
+Argument marshalling only: every function below has the name and the argument order of the
+C entry point it calls, accepts torch tensors (their ``data_ptr()`` is passed) or raw integer
+addresses, and returns the C status code unchanged. ``check()`` turns a negative status into
+an exception. The library is loaded on first use; if it has not been built this module
+raises — there is no fallback implementation.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import c_double, c_int, c_int32, c_int64, c_uint32, c_void_p
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtopkv.so")
+
+TOPKV_OK = 0
+TOPKV_ERR_INVALID_ARG = -1
+TOPKV_ERR_LAYER_RANGE = -2
+TOPKV_ERR_ALIGNMENT = -3
+TOPKV_ERR_CAPACITY = -4
+TOPKV_ERR_UNSUPPORTED_LAYOUT = -5
+TOPKV_ERR_CUDA = -6
+
+TOPKV_KIND_GQA, TOPKV_KIND_MLA = 0, 1
+TOPKV_WIRE_TOKEN_KV, TOPKV_WIRE_PLANAR = 0, 1
+TOPKV_MAX_INLINE_R = 1024
+
+# every symbol include/topkv.h declares
+EXPORTS = (
+    "topkv_pack_layer", "topkv_unpack_layer", "topkv_pack_layer_to_host",
+    "topkv_unpack_layer_from_host", "topkv_build_plan", "topkv_validate_batch_host",
+    "topkv_layout_default_strides", "topkv_wire_layer_bytes", "topkv_kv_bytes",
+    "topkv_model_transfer_s", "topkv_model_t_eff_s", "topkv_model_hidden_fraction",
+    "topkv_strerror", "topkv_version", "topkv_last_cuda_error", "topkv_kernel_launch_count",
+    "topkv_set_kernel_variant",
+)
+
+
+class topkv_layout(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", c_uint32), ("kind", c_uint32), ("num_layers", c_uint32),
+        ("kv_factor", c_uint32), ("num_kv_heads", c_uint32), ("head_dim", c_uint32),
+        ("elem_bytes", c_uint32), ("page_tokens", c_uint32), ("wire_order", c_uint32),
+        ("reserved", c_uint32), ("num_pool_pages", c_int64), ("pool_layer_stride", c_int64),
+        ("pool_page_stride", c_int64), ("pool_kv_stride", c_int64),
+        ("pool_token_stride", c_int64), ("pool_head_stride", c_int64),
+        ("wire_layer_stride", c_int64),
+    ]
+
+
+class topkv_batch(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", c_uint32), ("num_requests", c_int32), ("max_pages_per_req", c_int32),
+        ("reserved", c_int32), ("block_table", c_void_p), ("seq_lens", c_void_p),
+        ("cu_seq_lens", c_void_p), ("total_tokens", c_int64),
+    ]
+
+
+class TopkvError(RuntimeError):
+    def __init__(self, status: int):
+        self.status = status
+        super().__init__(f"topkv status {status}: {topkv_strerror(status)}")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libtopkv.so (built by ``__graft_entry__.build()``); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} not found: build the CUDA library first "
+                "(python -c 'import __graft_entry__ as g; g.build()'); there is no CPU fallback")
+        L = ctypes.CDLL(LIB_PATH)
+        lp, bp = ctypes.POINTER(topkv_layout), ctypes.POINTER(topkv_batch)
+        L.topkv_pack_layer.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p]
+        L.topkv_unpack_layer.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p]
+        L.topkv_pack_layer_to_host.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64,
+                                               c_void_p, c_int64, c_void_p]
+        L.topkv_unpack_layer_from_host.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64,
+                                                   c_void_p, c_int64, c_void_p]
+        L.topkv_build_plan.argtypes = [bp, c_void_p, c_void_p]
+        L.topkv_validate_batch_host.argtypes = [lp, c_int32, c_int32, c_void_p, c_void_p, c_int]
+        L.topkv_layout_default_strides.argtypes = [lp]
+        L.topkv_wire_layer_bytes.argtypes = [lp, c_int64]
+        L.topkv_wire_layer_bytes.restype = c_int64
+        L.topkv_kv_bytes.argtypes = [lp, c_int64]
+        L.topkv_kv_bytes.restype = c_int64
+        L.topkv_model_transfer_s.argtypes = [c_double] * 3
+        L.topkv_model_transfer_s.restype = c_double
+        L.topkv_model_t_eff_s.argtypes = [c_double] * 3
+        L.topkv_model_t_eff_s.restype = c_double
+        L.topkv_model_hidden_fraction.argtypes = [c_int, c_double, c_double]
+        L.topkv_model_hidden_fraction.restype = c_double
+        L.topkv_strerror.argtypes = [c_int]
+        L.topkv_strerror.restype = ctypes.c_char_p
+        L.topkv_kernel_launch_count.restype = c_int64
+        L.topkv_set_kernel_variant.argtypes = [c_int]
+        _lib = L
+    return _lib
+
+
+def _ptr(x) -> int | None:
+    """torch tensor / numpy array / int / None -> address."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "data_ptr"):
+        return x.data_ptr()
+    if hasattr(x, "ctypes"):
+        return x.ctypes.data
+    raise TypeError(type(x))
+
+
+def _stream(s) -> int | None:
+    if s is None:
+        return None
+    if isinstance(s, int):
+        return s or None
+    return s.cuda_stream or None  # torch.cuda.Stream
+
+
+def check(status: int) -> int:
+    if status < 0:
+        raise TopkvError(status)
+    return status
+
+
+# ---- constructors for the two descriptors -------------------------------------------------
+
+def make_layout(L: int, F: int, H: int, D: int, E: int, P: int, num_pool_pages: int,
+                wire_order: int = TOPKV_WIRE_TOKEN_KV, wire_layer_stride: int = 0,
+                kind: int | None = None) -> topkv_layout:
+    """Layout of the default page-major pool pool[l][page][c][t][h][d]."""
+    lo = topkv_layout()
+    lo.struct_size = ctypes.sizeof(topkv_layout)
+    lo.kind = (TOPKV_KIND_MLA if F == 1 and H == 1 else TOPKV_KIND_GQA) if kind is None else kind
+    lo.num_layers, lo.kv_factor, lo.num_kv_heads, lo.head_dim = L, F, H, D
+    lo.elem_bytes, lo.page_tokens, lo.wire_order = E, P, wire_order
+    lo.num_pool_pages = num_pool_pages
+    lo.wire_layer_stride = wire_layer_stride
+    check(topkv_layout_default_strides(lo))
+    return lo
+
+
+def make_batch(block_table, seq_lens, total_tokens: int = -1, cu_seq_lens=None) -> topkv_batch:
+    """block_table: device int32 [R][maxp]; seq_lens: device int32 [R]. The caller keeps the
+    tensors alive for as long as the descriptor is in use."""
+    b = topkv_batch()
+    b.struct_size = ctypes.sizeof(topkv_batch)
+    b.num_requests = int(block_table.shape[0])
+    b.max_pages_per_req = int(block_table.shape[1]) if block_table.ndim == 2 else 0
+    b.block_table = _ptr(block_table)
+    b.seq_lens = _ptr(seq_lens)
+    b.cu_seq_lens = _ptr(cu_seq_lens)
+    b.total_tokens = total_tokens
+    return b
+
+
+# ---- the C entry points, same names, same order ---------------------------------------------
+
+def topkv_pack_layer(layer, src_pool, layout, batch, d_wire, wire_capacity_bytes, stream=None):
+    return lib().topkv_pack_layer(layer, _ptr(src_pool), ctypes.byref(layout), ctypes.byref(batch),
+                                  _ptr(d_wire), wire_capacity_bytes, _stream(stream))
+
+
+def topkv_unpack_layer(layer, dst_pool, layout, batch, d_wire, wire_bytes, stream=None):
+    return lib().topkv_unpack_layer(layer, _ptr(dst_pool), ctypes.byref(layout),
+                                    ctypes.byref(batch), _ptr(d_wire), wire_bytes, _stream(stream))
+
+
+def topkv_pack_layer_to_host(layer, src_pool, layout, batch, h_pinned, host_capacity_bytes,
+                             d_staging, staging_capacity_bytes, stream=None):
+    return lib().topkv_pack_layer_to_host(layer, _ptr(src_pool), ctypes.byref(layout),
+                                          ctypes.byref(batch), _ptr(h_pinned), host_capacity_bytes,
+                                          _ptr(d_staging), staging_capacity_bytes, _stream(stream))
+
+
+def topkv_unpack_layer_from_host(layer, dst_pool, layout, batch, h_pinned, host_bytes, d_staging,
+                                 staging_capacity_bytes, stream=None):
+    return lib().topkv_unpack_layer_from_host(layer, _ptr(dst_pool), ctypes.byref(layout),
+                                              ctypes.byref(batch), _ptr(h_pinned), host_bytes,
+                                              _ptr(d_staging), staging_capacity_bytes,
+                                              _stream(stream))
+
+
+def topkv_build_plan(batch, d_cu_seq_lens, stream=None):
+    return lib().topkv_build_plan(ctypes.byref(batch), _ptr(d_cu_seq_lens), _stream(stream))
+
+
+def topkv_validate_batch_host(layout, num_requests, max_pages_per_req, h_block_table, h_seq_lens,
+                              require_disjoint):
+    return lib().topkv_validate_batch_host(ctypes.byref(layout), num_requests, max_pages_per_req,
+                                           _ptr(h_block_table), _ptr(h_seq_lens),
+                                           int(require_disjoint))
+
+
+def topkv_layout_default_strides(layout):
+    return lib().topkv_layout_default_strides(ctypes.byref(layout))
+
+
+def topkv_wire_layer_bytes(layout, total_tokens):
+    return lib().topkv_wire_layer_bytes(ctypes.byref(layout), total_tokens)
+
+
+def topkv_kv_bytes(layout, seq_len):
+    return lib().topkv_kv_bytes(ctypes.byref(layout), seq_len)
+
+
+def topkv_model_transfer_s(nbytes, bandwidth_bytes_per_s, setup_s=0.0):
+    return lib().topkv_model_transfer_s(nbytes, bandwidth_bytes_per_s, setup_s)
+
+
+def topkv_model_t_eff_s(t_last_s, t_xfer_s, t_rem_s):
+    return lib().topkv_model_t_eff_s(t_last_s, t_xfer_s, t_rem_s)
+
+
+def topkv_model_hidden_fraction(layers, t_layer_compute_s, t_xfer_total_s):
+    return lib().topkv_model_hidden_fraction(layers, t_layer_compute_s, t_xfer_total_s)
+
+
+def topkv_strerror(status):
+    return lib().topkv_strerror(status).decode()
+
+
+def topkv_version():
+    return lib().topkv_version()
+
+
+def topkv_last_cuda_error():
+    return lib().topkv_last_cuda_error()
+
+
+def topkv_kernel_launch_count():
+    return lib().topkv_kernel_launch_count()
+
+
+def topkv_set_kernel_variant(variant):
+    return lib().topkv_set_kernel_variant(variant)

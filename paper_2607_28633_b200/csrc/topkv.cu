@@ -1,0 +1,511 @@
+// TopKV data plane for B200 (sm_100a): per-layer pack / unpack of a paged KV cache to and
+// from a contiguous wire slab (§3.4 layout, sent layer by layer as in §5.2), and the
+// pinned-host PCIe leg (§3.3). Pure byte movement: no arithmetic on the elements.
+//
+// The product path lives entirely in this file and topkv_host.cpp; it never calls the CPU
+// oracle. All entry points are declared and documented in include/topkv.h.
+#include "topkv.h"
+
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdint>
+#include <cstring>
+
+namespace {
+
+// ------------------------------------------------------------------------------------------
+// Kernel parameters (plain data, passed by value).
+// A "unit" is the largest run of bytes that is contiguous on both sides for one
+// (token, plane): the whole [head][dim] row when heads are contiguous in the pool,
+// otherwise one head (U = H units per row).
+// ------------------------------------------------------------------------------------------
+struct KParams {
+  uint8_t* pool;          // base of this layer's pool slab
+  uint8_t* wire;          // base of this layer's wire slab (device, or mapped pinned host)
+  const int32_t* bt;      // [R][maxp]
+  const int32_t* sl;      // [R]
+  const int64_t* cu;      // [R+1] or nullptr
+  int64_t T;              // total tokens or -1
+  int64_t S_page, S_kv, S_tok, S_unit;  // pool strides, bytes
+  int R, maxp, P;
+  int U;                  // units per (token, plane)
+  int unit_chunks;        // VEC-byte chunks per unit
+  int planar;             // wire order
+};
+
+constexpr int kThreads = 256;
+constexpr int kUnroll16 = 8;  // vectors in flight per thread, 16-byte vectors
+constexpr int kUnroll32 = 4;  // and 32-byte vectors
+
+// Streaming vector accesses: every byte is touched exactly once, so neither side should
+// displace anything useful from L1 / L2. Vec<32> uses the 256-bit global accesses of sm_100.
+template <int VEC>
+struct Vec;
+template <>
+struct Vec<16> {
+  uint32_t v[4];
+  __device__ __forceinline__ void load(const uint8_t* p) {
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3])
+                 : "l"(p));
+  }
+  __device__ __forceinline__ void store(uint8_t* p) const {
+    asm volatile("st.global.L1::no_allocate.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v[0]),
+                 "r"(v[1]), "r"(v[2]), "r"(v[3])
+                 : "memory");
+  }
+};
+template <>
+struct Vec<32> {
+  uint32_t v[8];
+  __device__ __forceinline__ void load(const uint8_t* p) {
+    asm volatile(
+        "ld.global.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+          "=r"(v[7])
+        : "l"(p));
+  }
+  __device__ __forceinline__ void store(uint8_t* p) const {
+    asm volatile(
+        "st.global.L1::no_allocate.L2::evict_first.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p),
+        "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+        : "memory");
+  }
+};
+
+// Sum of sl[0..n) over the CTA, result broadcast to all threads. n <= TOPKV_MAX_INLINE_R.
+__device__ __forceinline__ int64_t block_prefix(const int32_t* __restrict__ sl, int n, int r_split,
+                                                int64_t* total_out) {
+  // returns sum_{q < r_split} sl[q]; *total_out = sum_{q < n} sl[q]
+  __shared__ int64_t s_part[2][kThreads / 32];
+  int64_t below = 0, all = 0;
+  for (int q = threadIdx.x; q < n; q += kThreads) {
+    int64_t v = sl[q];
+    all += v;
+    if (q < r_split) below += v;
+  }
+  for (int o = 16; o > 0; o >>= 1) {
+    below += __shfl_xor_sync(0xffffffffu, below, o);
+    all += __shfl_xor_sync(0xffffffffu, all, o);
+  }
+  if ((threadIdx.x & 31) == 0) {
+    s_part[0][threadIdx.x >> 5] = below;
+    s_part[1][threadIdx.x >> 5] = all;
+  }
+  __syncthreads();
+  below = 0;
+  all = 0;
+#pragma unroll
+  for (int w = 0; w < kThreads / 32; ++w) {
+    below += s_part[0][w];
+    all += s_part[1][w];
+  }
+  *total_out = all;
+  return below;
+}
+
+// One CTA per (request, page column). F: planes per token; PACK: pool -> wire, else
+// wire -> pool; MERGED: the valid tokens of a page form one contiguous run per plane on
+// both sides (MLA rows, or PLANAR wire with a token-contiguous pool).
+template <int F, bool PACK, bool MERGED, int VEC>
+__global__ void __launch_bounds__(kThreads)
+topkv_page_copy_kernel(const KParams p) {
+  const int slot = blockIdx.x;
+  const int r = slot / p.maxp;
+  const int j = slot - r * p.maxp;
+  const int s_r = p.sl[r];
+  const int first = j * p.P;
+  if (first >= s_r) return;
+  const int v = min(p.P, s_r - first);  // valid tokens in this page
+
+  int64_t cu_r, T = p.T;
+  if (p.cu != nullptr) {
+    cu_r = p.cu[r];
+    if (p.planar && T < 0) T = p.cu[p.R];
+  } else {
+    int64_t total;
+    cu_r = block_prefix(p.sl, (p.planar && T < 0) ? p.R : r, r, &total);
+    if (p.planar && T < 0) T = total;
+  }
+  const int64_t page = p.bt[(int64_t)r * p.maxp + j];
+  uint8_t* pool_page = p.pool + page * p.S_page;
+  const int64_t n0 = cu_r + first;  // global index of the page's first token
+  const int64_t unit_bytes = (int64_t)p.unit_chunks * VEC;
+  constexpr int kUnroll = VEC == 32 ? kUnroll32 : kUnroll16;
+  const int tid = threadIdx.x;
+
+  if (MERGED) {
+    // F runs of v * row bytes each (U == 1 here).
+    const int n = v * p.unit_chunks;
+#pragma unroll
+    for (int c = 0; c < F; ++c) {
+      uint8_t* a = pool_page + c * p.S_kv;
+      uint8_t* b = p.wire + ((p.planar ? c * T : 0) + n0) * unit_bytes;  // not planar => F == 1
+      const uint8_t* src = PACK ? a : b;
+      uint8_t* dst = PACK ? b : a;
+      for (int w0 = tid; w0 < n; w0 += kThreads * kUnroll) {
+        Vec<VEC> buf[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+          const int w = w0 + u * kThreads;
+          if (w < n) buf[u].load(src + (int64_t)w * VEC);
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+          const int w = w0 + u * kThreads;
+          if (w < n) buf[u].store(dst + (int64_t)w * VEC);
+        }
+      }
+    }
+    return;
+  }
+
+  // Units of this page in wire order: q = (t*F + c)*U + h  (TOKEN_KV), or
+  // q = (c*v + t)*U + h (PLANAR). `tpu` threads cooperate on one unit.
+  const int nunits = v * F * p.U;
+  const int tpu = min(p.unit_chunks, kThreads);
+  const int groups = kThreads / tpu;
+  const int my_g = tid / tpu;
+  const int my_w = tid - my_g * tpu;
+  if (my_g >= groups) return;
+  uint8_t* wire_page = p.wire + n0 * F * p.U * unit_bytes;  // TOKEN_KV: the page is one run
+
+  for (int q0 = my_g; q0 < nunits; q0 += groups * kUnroll) {
+    for (int w = my_w; w < p.unit_chunks; w += tpu) {
+      Vec<VEC> buf[kUnroll];
+      uint8_t* a[kUnroll];
+      uint8_t* b[kUnroll];
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        const int q = q0 + u * groups;
+        int h = 0, tc = q;
+        if (p.U > 1) {
+          tc = q / p.U;
+          h = q - tc * p.U;
+        }
+        int c, t;
+        if (p.planar) {
+          c = (F > 1 && tc >= v) ? 1 : 0;
+          t = tc - c * v;
+          b[u] = p.wire + (((int64_t)c * T + n0 + t) * p.U + h) * unit_bytes + (int64_t)w * VEC;
+        } else {
+          t = tc / F;
+          c = tc - t * F;
+          b[u] = wire_page + (int64_t)q * unit_bytes + (int64_t)w * VEC;
+        }
+        a[u] = pool_page + c * p.S_kv + t * p.S_tok + h * p.S_unit + (int64_t)w * VEC;
+        if (q < nunits) buf[u].load(PACK ? a[u] : b[u]);
+      }
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        const int q = q0 + u * groups;
+        if (q < nunits) buf[u].store(PACK ? b[u] : a[u]);
+      }
+    }
+  }
+}
+
+// Exclusive prefix sum of seq_lens into int64 [R+1]; one CTA, any R.
+__global__ void __launch_bounds__(kThreads)
+topkv_plan_kernel(const int32_t* __restrict__ sl, int R, int64_t* __restrict__ cu) {
+  __shared__ int64_t s_warp[kThreads / 32];
+  __shared__ int64_t s_carry;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  if (tid == 0) s_carry = 0;
+  __syncthreads();
+  for (int base = 0; base < R; base += kThreads) {
+    const int q = base + tid;
+    const int64_t x = q < R ? (int64_t)sl[q] : 0;
+    int64_t inc = x;  // inclusive scan inside the warp
+    for (int o = 1; o < 32; o <<= 1) {
+      const int64_t y = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += y;
+    }
+    if (lane == 31) s_warp[wid] = inc;
+    __syncthreads();
+    int64_t before = s_carry;
+    for (int w = 0; w < wid; ++w) before += s_warp[w];
+    if (q < R) cu[q] = before + inc - x;
+    __syncthreads();
+    if (tid == kThreads - 1) s_carry = before + inc;
+    __syncthreads();
+  }
+  if (tid == 0) cu[R] = s_carry;
+}
+
+// ------------------------------------------------------------------------------------------
+// Host side
+// ------------------------------------------------------------------------------------------
+thread_local int g_last_cuda_error = 0;
+std::atomic<int64_t> g_launches{0};
+std::atomic<int> g_variant{0};
+
+inline bool mult16(int64_t x) { return (x & 15) == 0; }
+inline bool mult16p(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+int cuda_fail(cudaError_t e) {
+  g_last_cuda_error = static_cast<int>(e);
+  return TOPKV_ERR_CUDA;
+}
+
+struct Resolved {
+  int64_t row_bytes;   // H*D*E
+  int64_t unit_bytes;  // contiguous unit
+  int U;
+  bool merged;
+};
+
+int check_layout(const topkv_layout* lo, Resolved* out) {
+  if (lo == nullptr || lo->struct_size != sizeof(topkv_layout)) return TOPKV_ERR_INVALID_ARG;
+  if (lo->reserved != 0) return TOPKV_ERR_INVALID_ARG;
+  if (lo->num_layers == 0 || lo->num_kv_heads == 0 || lo->head_dim == 0 || lo->elem_bytes == 0 ||
+      lo->page_tokens == 0 || lo->num_pool_pages <= 0)
+    return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  if (lo->kv_factor != 1 && lo->kv_factor != 2) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  if (lo->wire_order != TOPKV_WIRE_TOKEN_KV && lo->wire_order != TOPKV_WIRE_PLANAR)
+    return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  if (lo->kind != TOPKV_KIND_GQA && lo->kind != TOPKV_KIND_MLA) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  if (lo->kind == TOPKV_KIND_MLA && lo->kv_factor != 1) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  const int64_t head_bytes = (int64_t)lo->head_dim * lo->elem_bytes;
+  const int64_t row_bytes = head_bytes * lo->num_kv_heads;
+  if (row_bytes > (1ll << 30)) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  const bool heads_contig = lo->num_kv_heads == 1 || lo->pool_head_stride == head_bytes;
+  const int64_t unit = heads_contig ? row_bytes : head_bytes;
+  if (lo->pool_page_stride <= 0 || lo->pool_token_stride < unit || lo->pool_layer_stride <= 0 ||
+      (lo->kv_factor > 1 && lo->pool_kv_stride <= 0) ||
+      (!heads_contig && lo->pool_head_stride < head_bytes) || lo->wire_layer_stride < 0)
+    return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  if (!mult16(unit) || !mult16(lo->pool_page_stride) || !mult16(lo->pool_token_stride) ||
+      !mult16(lo->pool_layer_stride) || (lo->kv_factor > 1 && !mult16(lo->pool_kv_stride)) ||
+      (!heads_contig && !mult16(lo->pool_head_stride)) || !mult16(lo->wire_layer_stride))
+    return TOPKV_ERR_ALIGNMENT;
+  out->row_bytes = row_bytes;
+  out->unit_bytes = unit;
+  out->U = heads_contig ? 1 : (int)lo->num_kv_heads;
+  out->merged = heads_contig && lo->pool_token_stride == row_bytes &&
+                (lo->kv_factor == 1 || lo->wire_order == TOPKV_WIRE_PLANAR);
+  return TOPKV_OK;
+}
+
+int check_batch(const topkv_layout* lo, const topkv_batch* b) {
+  if (b == nullptr || b->struct_size != sizeof(topkv_batch) || b->reserved != 0)
+    return TOPKV_ERR_INVALID_ARG;
+  if (b->num_requests < 0 || b->max_pages_per_req < 0 || b->total_tokens < -1)
+    return TOPKV_ERR_INVALID_ARG;
+  if (b->num_requests > 0 && b->max_pages_per_req > 0) {
+    if (b->block_table == nullptr || b->seq_lens == nullptr) return TOPKV_ERR_INVALID_ARG;
+    if (b->cu_seq_lens == nullptr && b->num_requests > TOPKV_MAX_INLINE_R)
+      return TOPKV_ERR_INVALID_ARG;
+    if ((int64_t)b->num_requests * b->max_pages_per_req > 0x7fffffffll) return TOPKV_ERR_INVALID_ARG;
+    if (b->total_tokens > (int64_t)b->num_requests * b->max_pages_per_req * lo->page_tokens)
+      return TOPKV_ERR_INVALID_ARG;
+  }
+  return TOPKV_OK;
+}
+
+// Validates everything and fills the kernel parameters for one layer. `wire_base` is the base
+// of the whole wire buffer (layer 0's slab) of `capacity` bytes.
+int prepare(int layer, const void* pool, const topkv_layout* lo, const topkv_batch* b,
+            const void* wire_base, int64_t capacity, int64_t wire_layer_stride, KParams* kp,
+            Resolved* rs, int64_t* n_layer_out) {
+  int st = check_layout(lo, rs);
+  if (st != TOPKV_OK) return st;
+  st = check_batch(lo, b);
+  if (st != TOPKV_OK) return st;
+  if (layer < 0 || (uint32_t)layer >= lo->num_layers) return TOPKV_ERR_LAYER_RANGE;
+  if (pool == nullptr || wire_base == nullptr || capacity < 0) return TOPKV_ERR_INVALID_ARG;
+  if (!mult16p(pool) || !mult16p(wire_base)) return TOPKV_ERR_ALIGNMENT;
+  int64_t n_layer = -1;
+  if (b->total_tokens >= 0) {
+    n_layer = b->total_tokens * lo->kv_factor * rs->row_bytes;
+    if ((int64_t)layer * wire_layer_stride + n_layer > capacity) return TOPKV_ERR_CAPACITY;
+  }
+  *n_layer_out = n_layer;
+  kp->pool = const_cast<uint8_t*>(static_cast<const uint8_t*>(pool)) + (int64_t)layer * lo->pool_layer_stride;
+  kp->wire = const_cast<uint8_t*>(static_cast<const uint8_t*>(wire_base)) + (int64_t)layer * wire_layer_stride;
+  kp->bt = b->block_table;
+  kp->sl = b->seq_lens;
+  kp->cu = b->cu_seq_lens;
+  kp->T = b->total_tokens;
+  kp->S_page = lo->pool_page_stride;
+  kp->S_kv = lo->kv_factor > 1 ? lo->pool_kv_stride : 0;
+  kp->S_tok = lo->pool_token_stride;
+  kp->S_unit = rs->U > 1 ? lo->pool_head_stride : 0;
+  kp->R = b->num_requests;
+  kp->maxp = b->max_pages_per_req;
+  kp->P = (int)lo->page_tokens;
+  kp->U = rs->U;
+  kp->unit_chunks = (int)(rs->unit_bytes / 16);
+  kp->planar = lo->wire_order == TOPKV_WIRE_PLANAR;
+  return TOPKV_OK;
+}
+
+template <bool PACK, int VEC>
+void launch_vec(const KParams& kp, bool merged, int F, dim3 grid, cudaStream_t stream) {
+  const dim3 block(kThreads);
+  if (merged) {
+    if (F == 1) topkv_page_copy_kernel<1, PACK, true, VEC><<<grid, block, 0, stream>>>(kp);
+    else topkv_page_copy_kernel<2, PACK, true, VEC><<<grid, block, 0, stream>>>(kp);
+  } else {
+    if (F == 1) topkv_page_copy_kernel<1, PACK, false, VEC><<<grid, block, 0, stream>>>(kp);
+    else topkv_page_copy_kernel<2, PACK, false, VEC><<<grid, block, 0, stream>>>(kp);
+  }
+}
+
+template <bool PACK>
+int launch_copy(KParams kp, const Resolved& rs, int F, cudaStream_t stream) {
+  const int64_t slots = (int64_t)kp.R * kp.maxp;
+  if (slots == 0) return TOPKV_OK;
+  const dim3 grid((unsigned)slots);
+  // 32-byte vectors when every address the kernel can form is 32-byte aligned
+  const bool wide = ((reinterpret_cast<uintptr_t>(kp.pool) | reinterpret_cast<uintptr_t>(kp.wire) |
+                      (uintptr_t)kp.S_page | (uintptr_t)kp.S_kv | (uintptr_t)kp.S_tok |
+                      (uintptr_t)kp.S_unit | (uintptr_t)rs.unit_bytes) & 31) == 0;
+  if (wide) {
+    kp.unit_chunks = (int)(rs.unit_bytes / 32);
+    launch_vec<PACK, 32>(kp, rs.merged, F, grid, stream);
+  } else {
+    kp.unit_chunks = (int)(rs.unit_bytes / 16);
+    launch_vec<PACK, 16>(kp, rs.merged, F, grid, stream);
+  }
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return TOPKV_OK;
+}
+
+// Device-visible address of a pinned host buffer (identity under unified addressing, but
+// asked for explicitly so that pageable memory is refused instead of faulting).
+int mapped_device_pointer(const void* h, void** d) {
+  cudaPointerAttributes attr;
+  cudaError_t e = cudaPointerGetAttributes(&attr, h);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return cuda_fail(e);
+  }
+  if (attr.type != cudaMemoryTypeHost || attr.devicePointer == nullptr) return TOPKV_ERR_INVALID_ARG;
+  *d = attr.devicePointer;
+  return TOPKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int topkv_pack_layer(int layer, const void* src_pool, const topkv_layout* layout,
+                     const topkv_batch* batch, void* d_wire, int64_t wire_capacity_bytes,
+                     topkv_stream_t stream) {
+  KParams kp;
+  Resolved rs;
+  int64_t n_layer;
+  const int st = prepare(layer, src_pool, layout, batch, d_wire, wire_capacity_bytes,
+                         layout ? layout->wire_layer_stride : 0, &kp, &rs, &n_layer);
+  if (st != TOPKV_OK) return st;
+  return launch_copy<true>(kp, rs, (int)layout->kv_factor, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int topkv_unpack_layer(int layer, void* dst_pool, const topkv_layout* layout,
+                       const topkv_batch* batch, const void* d_wire, int64_t wire_bytes,
+                       topkv_stream_t stream) {
+  KParams kp;
+  Resolved rs;
+  int64_t n_layer;
+  const int st = prepare(layer, dst_pool, layout, batch, d_wire, wire_bytes,
+                         layout ? layout->wire_layer_stride : 0, &kp, &rs, &n_layer);
+  if (st != TOPKV_OK) return st;
+  return launch_copy<false>(kp, rs, (int)layout->kv_factor, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int topkv_pack_layer_to_host(int layer, const void* src_pool, const topkv_layout* layout,
+                             const topkv_batch* batch, void* h_pinned, int64_t host_capacity_bytes,
+                             void* d_staging, int64_t staging_capacity_bytes,
+                             topkv_stream_t stream) {
+  KParams kp;
+  Resolved rs;
+  int64_t n_layer;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (d_staging == nullptr) {  // direct stores into the mapped pinned buffer
+    int st = prepare(layer, src_pool, layout, batch, h_pinned, host_capacity_bytes,
+                     layout ? layout->wire_layer_stride : 0, &kp, &rs, &n_layer);
+    if (st != TOPKV_OK) return st;
+    void* dev = nullptr;
+    st = mapped_device_pointer(h_pinned, &dev);
+    if (st != TOPKV_OK) return st;
+    kp.wire = static_cast<uint8_t*>(dev) + (int64_t)layer * layout->wire_layer_stride;
+    return launch_copy<true>(kp, rs, (int)layout->kv_factor, s);
+  }
+  // staged: pack this layer into the staging slab, then one copy-engine transfer
+  if (batch != nullptr && batch->struct_size == sizeof(topkv_batch) && batch->total_tokens < 0)
+    return TOPKV_ERR_INVALID_ARG;
+  int st = prepare(layer, src_pool, layout, batch, h_pinned, host_capacity_bytes,
+                   layout ? layout->wire_layer_stride : 0, &kp, &rs, &n_layer);
+  if (st != TOPKV_OK) return st;
+  if (!mult16p(d_staging)) return TOPKV_ERR_ALIGNMENT;
+  if (staging_capacity_bytes < n_layer) return TOPKV_ERR_CAPACITY;
+  uint8_t* host_slab = kp.wire;
+  kp.wire = static_cast<uint8_t*>(d_staging);
+  st = launch_copy<true>(kp, rs, (int)layout->kv_factor, s);
+  if (st != TOPKV_OK) return st;
+  if (n_layer > 0) {
+    const cudaError_t e = cudaMemcpyAsync(host_slab, d_staging, (size_t)n_layer, cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  return TOPKV_OK;
+}
+
+int topkv_unpack_layer_from_host(int layer, void* dst_pool, const topkv_layout* layout,
+                                 const topkv_batch* batch, const void* h_pinned, int64_t host_bytes,
+                                 void* d_staging, int64_t staging_capacity_bytes,
+                                 topkv_stream_t stream) {
+  KParams kp;
+  Resolved rs;
+  int64_t n_layer;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (d_staging == nullptr) {  // direct loads from the mapped pinned buffer
+    int st = prepare(layer, dst_pool, layout, batch, h_pinned, host_bytes,
+                     layout ? layout->wire_layer_stride : 0, &kp, &rs, &n_layer);
+    if (st != TOPKV_OK) return st;
+    void* dev = nullptr;
+    st = mapped_device_pointer(h_pinned, &dev);
+    if (st != TOPKV_OK) return st;
+    kp.wire = static_cast<uint8_t*>(dev) + (int64_t)layer * layout->wire_layer_stride;
+    return launch_copy<false>(kp, rs, (int)layout->kv_factor, s);
+  }
+  if (batch != nullptr && batch->struct_size == sizeof(topkv_batch) && batch->total_tokens < 0)
+    return TOPKV_ERR_INVALID_ARG;
+  int st = prepare(layer, dst_pool, layout, batch, h_pinned, host_bytes,
+                   layout ? layout->wire_layer_stride : 0, &kp, &rs, &n_layer);
+  if (st != TOPKV_OK) return st;
+  if (!mult16p(d_staging)) return TOPKV_ERR_ALIGNMENT;
+  if (staging_capacity_bytes < n_layer) return TOPKV_ERR_CAPACITY;
+  if (n_layer > 0) {
+    const cudaError_t e = cudaMemcpyAsync(d_staging, kp.wire, (size_t)n_layer, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  kp.wire = static_cast<uint8_t*>(d_staging);
+  return launch_copy<false>(kp, rs, (int)layout->kv_factor, s);
+}
+
+int topkv_build_plan(const topkv_batch* batch, int64_t* d_cu_seq_lens, topkv_stream_t stream) {
+  if (batch == nullptr || batch->struct_size != sizeof(topkv_batch) || d_cu_seq_lens == nullptr)
+    return TOPKV_ERR_INVALID_ARG;
+  if (batch->num_requests < 0 || (batch->num_requests > 0 && batch->seq_lens == nullptr))
+    return TOPKV_ERR_INVALID_ARG;
+  topkv_plan_kernel<<<1, kThreads, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+      batch->seq_lens, batch->num_requests, d_cu_seq_lens);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return TOPKV_OK;
+}
+
+int topkv_last_cuda_error(void) { return g_last_cuda_error; }
+int64_t topkv_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int topkv_set_kernel_variant(int variant) {
+  if (variant < 0 || variant > 1) return TOPKV_ERR_INVALID_ARG;
+  return g_variant.exchange(variant);
+}
+
+}  // extern "C"

@@ -1,0 +1,170 @@
+"""CPU checks of the C-ABI library: it loads, exports every declared symbol, its host-side
+logic (argument validation, size bookkeeping, analytic helpers, batch validator) behaves as
+the header says, and a launch without a GPU fails loudly instead of falling back."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import __graft_entry__ as entry
+from paper_2607_28633_b200 import binding as tk
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    entry.build()
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "topkv.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(topkv_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_exports_every_declared_symbol():
+    names = _declared_symbols()
+    assert len(names) >= 17
+    assert sorted(tk.EXPORTS) == names
+    lib = tk.lib()
+    for n in names:
+        assert getattr(lib, n) is not None
+    assert tk.topkv_version() >= 100
+
+
+def test_struct_sizes_match_header():
+    # natural alignment of the C structs: 10 x u32 + 7 x i64, and 4 x 32-bit + 3 ptr + i64
+    assert ctypes.sizeof(tk.topkv_layout) == 96
+    assert ctypes.sizeof(tk.topkv_batch) == 48
+
+
+def _gqa(L=4, pages=64, **kw):
+    return tk.make_layout(L, 2, 8, 128, 2, 16, pages, **kw)
+
+
+def test_default_strides_and_sizes(golden):
+    lo = _gqa()
+    assert (lo.pool_head_stride, lo.pool_token_stride, lo.pool_kv_stride, lo.pool_page_stride,
+            lo.pool_layer_stride) == (256, 2048, 32768, 65536, 64 * 65536)
+    mla = tk.make_layout(61, 1, 1, 576, 2, 64, 10)
+    assert mla.kind == tk.TOPKV_KIND_MLA and mla.pool_page_stride == 73728
+    g = golden("paper_values.txt")
+    s = int(g["seq_len"])
+    l70 = tk.make_layout(80, 2, 8, 128, 2, 16, 1)
+    assert tk.topkv_kv_bytes(l70, s) == 1_342_177_280            # Table 1: 1.3 GB
+    assert round(tk.topkv_kv_bytes(l70, s) / 1e9, 1) == float(g["table1.llama3_70b.gb"])
+    assert tk.topkv_kv_bytes(mla, s) == 287_834_112              # Table 1: 0.27 (binary) GB
+    assert tk.topkv_kv_bytes(tk.make_layout(56, 2, 8, 128, 2, 16, 1), s) == 939_524_096
+    assert tk.topkv_wire_layer_bytes(l70, s) * 80 == tk.topkv_kv_bytes(l70, s)
+    assert tk.topkv_wire_layer_bytes(l70, -1) == tk.TOPKV_ERR_INVALID_ARG
+
+
+def test_model_helpers(golden):
+    g = golden("paper_values.txt")
+    S = 1.3e9
+    for mode in ("nvlink", "pcie", "rdma", "tcp"):
+        ms = tk.topkv_model_transfer_s(S, float(g[f"table4.{mode}.gbps"]) * 1e9) * 1e3
+        want = float(g[f"table4.{mode}.ms"])
+        assert round(ms, 1 if want < 10 else 0) == want
+    assert round(100 * tk.topkv_model_hidden_fraction(80, 0.5e-3, 52e-3)) == 76
+    assert tk.topkv_model_hidden_fraction(80, 0.5e-3, 26e-3) == 1.0
+    assert tk.topkv_model_t_eff_s(0.5e-3, 52e-3, 39.5e-3) == pytest.approx(12.5e-3)
+    assert tk.topkv_model_t_eff_s(0.5e-3, 2.9e-3, 39.5e-3) == pytest.approx(0.5e-3)
+
+
+class _FakeTensor:
+    """Stands in for a device tensor on a GPU-less box: only an address and a shape."""
+    def __init__(self, addr, shape):
+        self._a, self.shape, self.ndim = addr, shape, len(shape)
+
+    def data_ptr(self):
+        return self._a
+
+
+def _batch(R=4, maxp=16, T=436):
+    return tk.make_batch(_FakeTensor(0x10000, (R, maxp)), _FakeTensor(0x20000, (R,)), T)
+
+
+def test_argument_validation_without_gpu():
+    lo, b = _gqa(wire_layer_stride=1_785_856), _batch()
+    pool, wire, cap = 0x7000000, 0x9000000, 4 * 1_785_856
+    P = tk.topkv_pack_layer
+    assert P(-1, pool, lo, b, wire, cap) == tk.TOPKV_ERR_LAYER_RANGE
+    assert P(4, pool, lo, b, wire, cap) == tk.TOPKV_ERR_LAYER_RANGE
+    assert P(0, None, lo, b, wire, cap) == tk.TOPKV_ERR_INVALID_ARG
+    assert P(0, pool, lo, b, None, cap) == tk.TOPKV_ERR_INVALID_ARG
+    assert P(0, pool + 8, lo, b, wire, cap) == tk.TOPKV_ERR_ALIGNMENT
+    assert P(0, pool, lo, b, wire + 4, cap) == tk.TOPKV_ERR_ALIGNMENT
+    assert P(3, pool, lo, b, wire, cap - 1) == tk.TOPKV_ERR_CAPACITY
+    assert tk.topkv_unpack_layer(3, pool, lo, b, wire, cap - 1) == tk.TOPKV_ERR_CAPACITY
+    bad = _gqa(); bad.struct_size = 8
+    assert P(0, pool, bad, b, wire, cap) == tk.TOPKV_ERR_INVALID_ARG
+    bad = _gqa(); bad.kv_factor = 3
+    assert P(0, pool, bad, b, wire, cap) == tk.TOPKV_ERR_UNSUPPORTED_LAYOUT
+    bad = _gqa(); bad.wire_order = 7
+    assert P(0, pool, bad, b, wire, cap) == tk.TOPKV_ERR_UNSUPPORTED_LAYOUT
+    bad = _gqa(); bad.pool_token_stride = 2048 + 8
+    assert P(0, pool, bad, b, wire, cap) == tk.TOPKV_ERR_ALIGNMENT
+    bad = tk.make_layout(2, 2, 1, 4, 2, 16, 8)               # 8-byte rows
+    assert P(0, pool, bad, b, wire, cap) == tk.TOPKV_ERR_ALIGNMENT
+    bb = _batch(); bb.struct_size = 4
+    assert P(0, pool, lo, bb, wire, cap) == tk.TOPKV_ERR_INVALID_ARG
+    bb = _batch(); bb.seq_lens = None
+    assert P(0, pool, lo, bb, wire, cap) == tk.TOPKV_ERR_INVALID_ARG
+    bb = _batch(R=tk.TOPKV_MAX_INLINE_R + 1, T=-1)          # no plan for a large batch
+    assert P(0, pool, lo, bb, wire, cap) == tk.TOPKV_ERR_INVALID_ARG
+    bb = _batch(T=4 * 16 * 16 + 1)                          # more tokens than the table can hold
+    assert P(0, pool, lo, bb, wire, cap) == tk.TOPKV_ERR_INVALID_ARG
+    # staged host leg needs the copy size on the host and a big enough staging slab
+    H = tk.topkv_pack_layer_to_host
+    assert H(0, pool, lo, _batch(T=-1), wire, cap, 0xA000000, cap) == tk.TOPKV_ERR_INVALID_ARG
+    assert H(0, pool, lo, b, wire, cap, 0xA000000, 1_785_855) == tk.TOPKV_ERR_CAPACITY
+    assert tk.topkv_unpack_layer_from_host(0, pool, lo, b, wire, cap, 0xA000008, cap) \
+        == tk.TOPKV_ERR_ALIGNMENT
+    assert tk.topkv_build_plan(b, None) == tk.TOPKV_ERR_INVALID_ARG
+    for code in range(-6, 1):
+        assert tk.topkv_strerror(code) != "unknown status"
+    assert tk.topkv_set_kernel_variant(99) == tk.TOPKV_ERR_INVALID_ARG
+
+
+def test_empty_batches_launch_nothing():
+    lo = _gqa(wire_layer_stride=0)
+    before = tk.topkv_kernel_launch_count()
+    b = tk.make_batch(_FakeTensor(0, (0, 16)), _FakeTensor(0, (0,)), 0)
+    assert tk.topkv_pack_layer(0, 0x7000000, lo, b, 0x9000000, 0) == tk.TOPKV_OK
+    assert tk.topkv_unpack_layer(0, 0x7000000, lo, b, 0x9000000, 0) == tk.TOPKV_OK
+    assert tk.topkv_kernel_launch_count() == before
+
+
+def test_no_cpu_fallback_without_device():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("GPU present; the launch would succeed")
+    lo, b = _gqa(wire_layer_stride=1_785_856), _batch()
+    st = tk.topkv_pack_layer(0, 0x7000000, lo, b, 0x9000000, 4 * 1_785_856)
+    assert st == tk.TOPKV_ERR_CUDA and tk.topkv_last_cuda_error() != 0
+    with pytest.raises(tk.TopkvError):
+        tk.check(st)
+
+
+def test_validate_batch_host():
+    lo = _gqa(pages=8)
+    sl = np.array([17, 32, 0], dtype=np.int32)
+    bt = np.array([[3, 5], [0, 1], [-1, -1]], dtype=np.int32)
+    V = tk.topkv_validate_batch_host
+    assert V(lo, 3, 2, bt, sl, 1) == tk.TOPKV_OK
+    bad = bt.copy(); bad[1, 1] = 8
+    assert V(lo, 3, 2, bad, sl, 0) == tk.TOPKV_ERR_INVALID_ARG      # page id out of range
+    bad = bt.copy(); bad[0, 1] = -1
+    assert V(lo, 3, 2, bad, sl, 0) == tk.TOPKV_ERR_INVALID_ARG      # used column is padding
+    bad = bt.copy(); bad[1, 0] = 3
+    assert V(lo, 3, 2, bad, sl, 0) == tk.TOPKV_OK                   # shared source page: allowed
+    assert V(lo, 3, 2, bad, sl, 1) == tk.TOPKV_ERR_INVALID_ARG      # shared destination page
+    long = sl.copy(); long[0] = 33
+    assert V(lo, 3, 2, bt, long, 0) == tk.TOPKV_ERR_INVALID_ARG     # longer than the table row
+    short = sl.copy(); short[0] = 16                               # ignores the unused column
+    ok = bt.copy(); ok[0, 1] = -1
+    assert V(lo, 3, 2, ok, short, 1) == tk.TOPKV_OK

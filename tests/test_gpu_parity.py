@@ -1,0 +1,324 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle, byte for byte
+(pure byte movement: the bar is bit-exact everywhere)."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+import oracle
+from oracle import Geom
+from paper_2607_28633_b200 import binding as tk
+from paper_2607_28633_b200 import harness
+from paper_2607_28633_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dev():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    import __graft_entry__ as entry
+    entry.build()
+    return torch.device("cuda:0")
+
+
+def _geom(spec, npages, L, wire_order, W_layer):
+    return Geom(L=L, F=spec.F, h_kv=spec.H, d_h=spec.D, b_p=spec.E, P=spec.P, num_pages=npages,
+                wire_order=wire_order, W_layer=W_layer)
+
+
+# -------------------------------------------------------------------- cfg1, every option
+
+@pytest.mark.parametrize("wire_order", [tk.TOPKV_WIRE_TOKEN_KV, tk.TOPKV_WIRE_PLANAR])
+@pytest.mark.parametrize("use_plan", [True, False])
+@pytest.mark.parametrize("know_T", [True, False])
+def test_cfg1_pack_unpack(dev, wire_order, use_plan, know_T):
+    w = harness.setup(wl.CFG1, dev, wire_order=wire_order, use_plan=use_plan)
+    b, s = w.batch, w.batch.spec
+    if not know_T:
+        w.src_batch.total_tokens = -1
+        w.dst_batch.total_tokens = -1
+    g = _geom(s, b.num_pool_pages, s.L, wire_order, w.n_layer)
+    src_h = w.src_pool.cpu().numpy()
+    dst_h = w.dst_pool.cpu().numpy()
+    stream = torch.cuda.Stream(dev)
+    for layer in range(s.L):
+        w.pack(layer, stream)
+        w.unpack(layer, stream)
+    stream.synchronize()
+    want_wire = np.zeros(s.L * w.n_layer, dtype=np.uint8)
+    for layer in range(s.L):
+        oracle.pack(g, layer, src_h, b.src_block_table, b.seq_lens, wire=want_wire)
+        oracle.unpack(g, layer, dst_h, b.dst_block_table, b.seq_lens, want_wire)
+    assert np.array_equal(w.wire.cpu().numpy(), want_wire)
+    assert np.array_equal(w.dst_pool.cpu().numpy(), dst_h)
+    assert np.array_equal(w.src_pool.cpu().numpy(), src_h)          # source untouched
+
+
+def test_build_plan(dev):
+    for R in (1, 5, 255, 256, 257, 1000, 3000):
+        sl = np.random.default_rng(R).integers(0, 9000, size=R).astype(np.int32)
+        d_sl = torch.from_numpy(sl).to(dev)
+        cu = torch.full((R + 1,), -7, dtype=torch.int64, device=dev)
+        b = tk.make_batch(torch.zeros((R, 1), dtype=torch.int32, device=dev), d_sl)
+        tk.check(tk.topkv_build_plan(b, cu))
+        torch.cuda.synchronize()
+        want = np.concatenate([[0], np.cumsum(sl.astype(np.int64))])
+        assert np.array_equal(cu.cpu().numpy(), want)
+
+
+# -------------------------------------------------------------------- random small cases
+
+def _case(seed):
+    """Random geometry, including strided pools, head-split rows, 16-byte-only alignment,
+    empty requests, full last pages and single tokens."""
+    rng = np.random.default_rng(seed)
+    F = int(rng.integers(1, 3))
+    H = int(rng.choice([1, 2, 4, 8]))
+    D = int(rng.choice([8, 24, 64, 72, 128, 576]))
+    P = int(rng.choice([1, 3, 16, 64]))
+    E = 2
+    L = 2
+    R = int(rng.integers(1, 7))
+    sl = rng.integers(0, 4 * P + 2, size=R).astype(np.int32)
+    if seed % 5 == 0:
+        sl[rng.integers(0, R)] = 0
+    if seed % 5 == 1:
+        sl[rng.integers(0, R)] = P * int(rng.integers(1, 4))
+    if seed % 7 == 2:
+        sl[:] = 0
+    pages = (sl + P - 1) // P
+    maxp = max(int(pages.max()), 1) + int(rng.integers(0, 3))
+    npages = int(pages.sum()) + int(rng.integers(1, 5))
+    g = Geom(L=L, F=F, h_kv=H, d_h=D, b_p=E, P=P, num_pages=npages)
+    style = seed % 4
+    if style == 1:      # padded token stride (keeps heads contiguous)
+        g.S_tok = H * D * E + 16 * int(rng.integers(1, 3))
+        g.S_kv = P * g.S_tok
+        g.S_page = F * g.S_kv + 32
+        g.S_layer = npages * g.S_page
+    elif style == 2:    # head-major inside the page: pool[l][page][c][h][t][d]
+        g.S_tok = D * E
+        g.S_head = P * g.S_tok
+        g.S_kv = H * g.S_head
+        g.S_page = F * g.S_kv
+        g.S_layer = npages * g.S_page
+    elif style == 3:    # plane-major pool: pool[l][c][page][t][h][d]
+        g.S_page = P * g.S_tok
+        g.S_kv = npages * g.S_page
+        g.S_layer = F * g.S_kv + 16
+    g.wire_order = int(rng.integers(0, 2))
+    T = int(sl.sum())
+    g.W_layer = g.wire_layer_bytes(T) + 16 * int(rng.integers(0, 3))
+    bt_s = np.full((R, maxp), -1, dtype=np.int32)
+    bt_d = np.full((R, maxp), -1, dtype=np.int32)
+    ps, pd, pos = rng.permutation(npages), rng.permutation(npages), 0
+    for r in range(R):
+        bt_s[r, :pages[r]] = ps[pos:pos + pages[r]]
+        bt_d[r, :pages[r]] = pd[pos:pos + pages[r]]
+        pos += pages[r]
+    return g, sl, bt_s, bt_d, rng
+
+
+def _layout_from_geom(g: Geom):
+    lo = tk.make_layout(g.L, g.F, g.h_kv, g.d_h, g.b_p, g.P, g.num_pages, wire_order=g.wire_order,
+                        wire_layer_stride=g.W_layer,
+                        kind=tk.TOPKV_KIND_GQA)
+    lo.pool_layer_stride, lo.pool_page_stride, lo.pool_kv_stride = g.S_layer, g.S_page, g.S_kv
+    lo.pool_token_stride, lo.pool_head_stride = g.S_tok, g.S_head
+    return lo
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_random_geometries(dev, seed):
+    g, sl, bt_s, bt_d, rng = _case(seed)
+    lo = _layout_from_geom(g)
+    T = int(sl.sum())
+    guard = 64
+    skew = 16 * (seed % 2)                     # odd seeds: 16-byte (not 32-byte) aligned bases
+    src_h = rng.integers(0, 256, g.L * g.S_layer, dtype=np.uint8)
+    fill_h = rng.integers(0, 256, g.L * g.S_layer, dtype=np.uint8)
+    wire_len = g.L * g.W_layer + 32            # slack for the last layer's padding
+    src_buf = torch.zeros(src_h.size + skew, dtype=torch.uint8, device=dev)
+    src = src_buf[skew:]
+    src.copy_(torch.from_numpy(src_h))
+    dst_buf = torch.zeros(fill_h.size + skew, dtype=torch.uint8, device=dev)
+    dst = dst_buf[skew:]
+    dst.copy_(torch.from_numpy(fill_h))
+    wire_buf = torch.full((guard + wire_len + guard + skew,), 0xA5, dtype=torch.uint8, device=dev)
+    wire = wire_buf[guard + skew:guard + skew + wire_len]
+    d_sl = torch.from_numpy(sl).to(dev)
+    d_bs, d_bd = torch.from_numpy(bt_s).to(dev), torch.from_numpy(bt_d).to(dev)
+    know_T = seed % 3 != 0
+    bs = tk.make_batch(d_bs, d_sl, T if know_T else -1)
+    bd = tk.make_batch(d_bd, d_sl, T if know_T else -1)
+    assert tk.topkv_validate_batch_host(lo, len(sl), bt_s.shape[1], bt_s, sl, 0) == tk.TOPKV_OK
+    assert tk.topkv_validate_batch_host(lo, len(sl), bt_d.shape[1], bt_d, sl, 1) == tk.TOPKV_OK
+    for layer in range(g.L):
+        tk.check(tk.topkv_pack_layer(layer, src, lo, bs, wire, wire.numel()))
+        tk.check(tk.topkv_unpack_layer(layer, dst, lo, bd, wire, wire.numel()))
+    torch.cuda.synchronize()
+    want_wire = np.full(wire_len, 0xA5, dtype=np.uint8)
+    want_dst = fill_h.copy()
+    for layer in range(g.L):
+        oracle.pack(g, layer, src_h, bt_s, sl, wire=want_wire)
+        oracle.unpack(g, layer, want_dst, bt_d, sl, want_wire)
+    got = wire_buf.cpu().numpy()
+    assert (got[:guard + skew] == 0xA5).all() and (got[guard + skew + wire_len:] == 0xA5).all()
+    assert np.array_equal(got[guard + skew:guard + skew + wire_len], want_wire)
+    assert np.array_equal(dst.cpu().numpy(), want_dst)
+
+
+def test_many_short_requests_inline_and_planned(dev):
+    """R at the inline limit (each CTA derives the prefix sum) and beyond it (plan required)."""
+    for R, planned in ((tk.TOPKV_MAX_INLINE_R, False), (tk.TOPKV_MAX_INLINE_R, True), (2500, True)):
+        rng = np.random.default_rng(R + planned)
+        g = Geom(L=1, F=2, h_kv=2, d_h=64, b_p=2, P=16, num_pages=2 * R + 5)
+        sl = rng.integers(0, 33, size=R).astype(np.int32)
+        pages = (sl + 15) // 16
+        bt = np.full((R, 3), -1, dtype=np.int32)
+        perm, pos = rng.permutation(g.num_pages), 0
+        for r in range(R):
+            bt[r, :pages[r]] = perm[pos:pos + pages[r]]
+            pos += pages[r]
+        T = int(sl.sum())
+        for order in (0, 1):
+            g.wire_order = order
+            lo = _layout_from_geom(g)
+            src_h = rng.integers(0, 256, g.S_layer, dtype=np.uint8)
+            src = torch.from_numpy(src_h).to(dev)
+            wire = torch.zeros(g.wire_layer_bytes(T), dtype=torch.uint8, device=dev)
+            d_sl, d_bt = torch.from_numpy(sl).to(dev), torch.from_numpy(bt).to(dev)
+            cu = None
+            if planned:
+                cu = torch.zeros(R + 1, dtype=torch.int64, device=dev)
+                tk.check(tk.topkv_build_plan(tk.make_batch(d_bt, d_sl), cu))
+            b = tk.make_batch(d_bt, d_sl, -1, cu)
+            tk.check(tk.topkv_pack_layer(0, src, lo, b, wire, wire.numel()))
+            torch.cuda.synchronize()
+            want = oracle.pack(g, 0, src_h, bt, sl, impl="rows", threads=4)
+            assert np.array_equal(wire.cpu().numpy(), want)
+    # without a plan a batch beyond the inline limit is refused, nothing is launched
+    b = tk.make_batch(d_bt, d_sl, -1, None)
+    assert tk.topkv_pack_layer(0, src, lo, b, wire, wire.numel()) == tk.TOPKV_ERR_INVALID_ARG
+
+
+# -------------------------------------------------------------------- benchmark shapes
+
+def _check_layers(w, layers, dev, threads=8):
+    """pack + unpack the given layers and compare each slab with the oracle."""
+    b, s = w.batch, w.batch.spec
+    g = _geom(s, b.num_pool_pages, 1, w.layout.wire_order, 0)      # one-slab view
+    slab = w.slab_bytes
+    for layer in layers:
+        src_h = harness.layer_slab_to_numpy(w.src_pool, slab, layer)
+        dst_h = harness.layer_slab_to_numpy(w.dst_pool, slab, layer)
+        w.pack(layer)
+        w.unpack(layer)
+        torch.cuda.synchronize()
+        want = oracle.pack(g, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=threads)
+        got = w.wire[layer * w.n_layer:(layer + 1) * w.n_layer].cpu().numpy()
+        assert np.array_equal(got, want), f"pack layer {layer}"
+        oracle.unpack(g, 0, dst_h, b.dst_block_table, b.seq_lens, want, impl="rows", threads=threads)
+        assert np.array_equal(harness.layer_slab_to_numpy(w.dst_pool, slab, layer), dst_h), \
+            f"unpack layer {layer}"
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg4"])
+def test_bench_shapes_reduced_layers(dev, name):
+    spec = wl.ALL[name]
+    w = harness.setup(spec, dev, layers=3)
+    assert w.batch.spec.R == spec.R
+    _check_layers(w, range(3), dev)
+    del w
+    torch.cuda.empty_cache()
+
+
+def test_cfg2_full_size_sampled_layers(dev):
+    """The launch configuration bench.py times (all 32 layers resident), three layers checked
+    in full against the oracle and every other layer's wire by a sampled-row comparison."""
+    spec = wl.CFG2
+    w = harness.setup(spec, dev)
+    _check_layers(w, [0, 17, spec.L - 1], dev)
+    b, s = w.batch, spec
+    rng = np.random.default_rng(7)
+    cu = np.concatenate([[0], np.cumsum(b.seq_lens.astype(np.int64))])
+    for layer in range(spec.L):
+        w.pack(layer)
+    torch.cuda.synchronize()
+    for layer in range(spec.L):
+        # sampled tokens, each computed one by one from the definition
+        for _ in range(16):
+            r = int(rng.integers(0, s.R))
+            i = int(rng.integers(0, b.seq_lens[r]))
+            page = int(b.src_block_table[r, i // s.P])
+            for c in range(s.F):
+                po = (layer * w.slab_bytes + page * s.page_bytes + c * s.P * s.row_bytes
+                      + (i % s.P) * s.row_bytes)
+                wo = layer * w.n_layer + ((cu[r] + i) * s.F + c) * s.row_bytes
+                assert torch.equal(w.src_pool[po:po + s.row_bytes], w.wire[wo:wo + s.row_bytes])
+    del w
+    torch.cuda.empty_cache()
+
+
+# -------------------------------------------------------------------- host leg
+
+@pytest.mark.parametrize("staged", [True, False])
+def test_host_leg_cfg1(dev, staged):
+    w = harness.setup(wl.CFG1, dev)
+    b, s = w.batch, w.batch.spec
+    g = _geom(s, b.num_pool_pages, s.L, 0, w.n_layer)
+    src_h, dst_h = w.src_pool.cpu().numpy(), w.dst_pool.cpu().numpy()
+    pinned = torch.full((s.L * w.n_layer,), 0x5A, dtype=torch.uint8).pin_memory()
+    staging = torch.zeros(w.n_layer, dtype=torch.uint8, device=dev) if staged else None
+    stream = torch.cuda.Stream(dev)
+    for layer in range(s.L):
+        w.pack_to_host(layer, pinned, staging, stream)
+    stream.synchronize()
+    want_wire = np.zeros(s.L * w.n_layer, dtype=np.uint8)
+    for layer in range(s.L):
+        oracle.pack(g, layer, src_h, b.src_block_table, b.seq_lens, wire=want_wire)
+    assert np.array_equal(pinned.numpy(), want_wire)
+    for layer in range(s.L):
+        w.unpack_from_host(layer, pinned, staging, stream)
+    stream.synchronize()
+    for layer in range(s.L):
+        oracle.unpack(g, layer, dst_h, b.dst_block_table, b.seq_lens, want_wire)
+    assert np.array_equal(w.dst_pool.cpu().numpy(), dst_h)
+
+
+def test_host_leg_refuses_pageable_memory(dev):
+    w = harness.setup(wl.CFG1, dev)
+    pageable = torch.zeros(w.batch.spec.L * w.n_layer, dtype=torch.uint8)
+    st = tk.topkv_pack_layer_to_host(0, w.src_pool, w.layout, w.src_batch, pageable,
+                                     pageable.numel(), None, 0)
+    assert st in (tk.TOPKV_ERR_INVALID_ARG, tk.TOPKV_ERR_CUDA)
+    torch.cuda.synchronize()
+
+
+def test_host_leg_cfg3_shape_two_layers(dev):
+    """The 70B shape's per-layer slab (128 MiB) through pinned memory, both forms."""
+    w = harness.setup(wl.CFG3, dev, layers=2)
+    b, s = w.batch, w.batch.spec
+    g = _geom(s, b.num_pool_pages, 1, 0, 0)
+    pinned = torch.zeros(2 * w.n_layer, dtype=torch.uint8).pin_memory()
+    staging = torch.zeros(w.n_layer, dtype=torch.uint8, device=dev)
+    for staged, layer in ((True, 0), (False, 1)):
+        w.pack_to_host(layer, pinned, staging if staged else None)
+        torch.cuda.synchronize()
+        src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, layer)
+        want = oracle.pack(g, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=8)
+        assert np.array_equal(pinned[layer * w.n_layer:(layer + 1) * w.n_layer].numpy(), want)
+        dst_h = harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, layer)
+        w.unpack_from_host(layer, pinned, None if staged else staging)   # the other form back
+        torch.cuda.synchronize()
+        oracle.unpack(g, 0, dst_h, b.dst_block_table, b.seq_lens, want, impl="rows", threads=8)
+        assert np.array_equal(harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, layer), dst_h)
+    del w
+    torch.cuda.empty_cache()
+
+
+def test_smoke_entry(dev):
+    import __graft_entry__ as entry
+    entry.smoke()
