@@ -60,7 +60,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                 "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+                 "-i", str(self.index), "-lms", "50"], stdout=subprocess.PIPE, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
         except Exception:
@@ -123,7 +123,7 @@ def oracle_sample(spec, batch, seconds_target=12.0):
                       threads=cores)
         n += 1
         dt = time.perf_counter() - t0
-        if dt >= seconds_target or n >= 64:
+        if dt >= seconds_target:
             break
     return 4.0 * n_layer * n / dt / 1e9, n, cores, dt
 
@@ -361,7 +361,8 @@ def run_extra(name, dev, stream, args, peak):
             d["prefill_tflops_alone"] = round(pre.flop_per_layer / (r.t_layer_compute_ms * 1e-3)
                                               / 1e12, 1)
             out[form] = d
-            if best is None or d["hidden"] > out[best]["hidden"]:
+            # prefer the form that disturbs the prefill least among those that hide >= 95 %
+            if best is None or (d["hidden"] >= 0.95 and d["slowdown"] < out[best]["slowdown"]):
                 best = form
         out["best_form"] = best
         out["hidden_fraction"] = out[best]["hidden"]

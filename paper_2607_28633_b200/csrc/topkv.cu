@@ -272,7 +272,8 @@ int check_layout(const topkv_layout* lo, Resolved* out) {
   if (row_bytes > (1ll << 30)) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
   const bool heads_contig = lo->num_kv_heads == 1 || lo->pool_head_stride == head_bytes;
   const int64_t unit = heads_contig ? row_bytes : head_bytes;
-  if (lo->pool_page_stride <= 0 || lo->pool_token_stride < unit || lo->pool_layer_stride <= 0 ||
+  if (lo->pool_page_stride <= 0 || lo->pool_layer_stride <= 0 ||
+      (lo->page_tokens > 1 && lo->pool_token_stride < unit) ||
       (lo->kv_factor > 1 && lo->pool_kv_stride <= 0) ||
       (!heads_contig && lo->pool_head_stride < head_bytes) || lo->wire_layer_stride < 0)
     return TOPKV_ERR_UNSUPPORTED_LAYOUT;
@@ -283,7 +284,7 @@ int check_layout(const topkv_layout* lo, Resolved* out) {
   out->row_bytes = row_bytes;
   out->unit_bytes = unit;
   out->U = heads_contig ? 1 : (int)lo->num_kv_heads;
-  out->merged = heads_contig && lo->pool_token_stride == row_bytes &&
+  out->merged = heads_contig && (lo->page_tokens == 1 || lo->pool_token_stride == row_bytes) &&
                 (lo->kv_factor == 1 || lo->wire_order == TOPKV_WIRE_PLANAR);
   return TOPKV_OK;
 }
