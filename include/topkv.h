@@ -145,6 +145,38 @@ int topkv_unpack_layer_from_host(int layer, void* dst_pool, const topkv_layout* 
                                  int64_t host_bytes, void* d_staging,
                                  int64_t staging_capacity_bytes, topkv_stream_t stream);
 
+/* ---- allocation-free host leg -------------------------------------------------------------- */
+
+/* Size of the library's built-in staging slab (bytes). Every GPU that loads the library
+ * reserves this much device memory until the process exits. */
+#define TOPKV_NOALLOC_STAGING_BYTES (8 * 1024 * 1024)
+
+/* (No counterpart in the paper: this exists for callers, not for the method.)
+ *
+ * Staged form of topkv_pack_layer_to_host for callers that cannot provide a staging slab
+ * because they are not allowed to allocate device memory: code running inside another
+ * framework's memory pool with a fixed budget, plug-ins loaded after that pool has claimed
+ * the GPU, and paths where a cudaMalloc would stall the device (it synchronises) in the
+ * middle of serving. The staging slab is a fixed array inside the library's own device image,
+ * so this call performs no cudaMalloc / cudaFree and calls no allocating routine.
+ *
+ * Same result as topkv_pack_layer_to_host with a caller staging slab: layer `layer` is packed
+ * into the built-in slab, then copied to h_pinned + layer*wire_layer_stride by the copy
+ * engine, all on `stream`. batch->total_tokens must be known (>= 0).
+ *
+ * Limits and rules:
+ *  - N_layer must not exceed TOPKV_NOALLOC_STAGING_BYTES, else TOPKV_ERR_CAPACITY is returned
+ *    and nothing is launched.
+ *  - The first call on each device looks up the slab's device address (once per device, with
+ *    that device current). Make that first call outside any stream capture.
+ *  - There is ONE slab per device, shared by every call and every stream, and it keeps the
+ *    previous call's bytes. Nothing in it needs to start at zero (each call overwrites the
+ *    N_layer bytes it then copies out), but two calls whose GPU work may overlap (different
+ *    streams, no ordering between them) race on it: order them on one stream or with events. */
+int topkv_pack_layer_to_host_noalloc(int layer, const void* src_pool, const topkv_layout* layout,
+                                     const topkv_batch* batch, void* h_pinned,
+                                     int64_t host_capacity_bytes, topkv_stream_t stream);
+
 /* ---- plan (layer-invariant, once per batch) ------------------------------------------ */
 
 /* Writes the exclusive prefix sum of seq_lens to d_cu_seq_lens (DEVICE int64 [R+1]). */

@@ -26,6 +26,7 @@ TOPKV_ERR_CUDA = -6
 TOPKV_KIND_GQA, TOPKV_KIND_MLA = 0, 1
 TOPKV_WIRE_TOKEN_KV, TOPKV_WIRE_PLANAR = 0, 1
 TOPKV_MAX_INLINE_R = 1024
+TOPKV_NOALLOC_STAGING_BYTES = 8 * 1024 * 1024
 
 # every symbol include/topkv.h declares
 EXPORTS = (
@@ -34,7 +35,7 @@ EXPORTS = (
     "topkv_layout_default_strides", "topkv_wire_layer_bytes", "topkv_kv_bytes",
     "topkv_model_transfer_s", "topkv_model_t_eff_s", "topkv_model_hidden_fraction",
     "topkv_strerror", "topkv_version", "topkv_last_cuda_error", "topkv_kernel_launch_count",
-    "topkv_set_kernel_variant",
+    "topkv_set_kernel_variant", "topkv_pack_layer_to_host_noalloc",
 )
 
 
@@ -84,6 +85,8 @@ def lib() -> ctypes.CDLL:
         L.topkv_unpack_layer_from_host.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64,
                                                    c_void_p, c_int64, c_void_p]
         L.topkv_build_plan.argtypes = [bp, c_void_p, c_void_p]
+        L.topkv_pack_layer_to_host_noalloc.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64,
+                                                       c_void_p]
         L.topkv_validate_batch_host.argtypes = [lp, c_int32, c_int32, c_void_p, c_void_p, c_int]
         L.topkv_layout_default_strides.argtypes = [lp]
         L.topkv_wire_layer_bytes.argtypes = [lp, c_int64]
@@ -187,6 +190,16 @@ def topkv_unpack_layer_from_host(layer, dst_pool, layout, batch, h_pinned, host_
                                               ctypes.byref(batch), _ptr(h_pinned), host_bytes,
                                               _ptr(d_staging), staging_capacity_bytes,
                                               _stream(stream))
+
+
+def topkv_pack_layer_to_host_noalloc(layer, src_pool, layout, batch, h_pinned,
+                                     host_capacity_bytes, stream=None):
+    """Staged pack-to-host for callers that may not allocate device memory: the staging slab
+    is the library's built-in TOPKV_NOALLOC_STAGING_BYTES array. One slab per device, shared by
+    all calls; make the first call on a device outside stream capture."""
+    return lib().topkv_pack_layer_to_host_noalloc(
+        layer, _ptr(src_pool), ctypes.byref(layout), ctypes.byref(batch), _ptr(h_pinned),
+        host_capacity_bytes, _stream(stream))
 
 
 def topkv_build_plan(batch, d_cu_seq_lens, stream=None):

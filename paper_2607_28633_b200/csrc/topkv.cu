@@ -11,6 +11,7 @@
 #include <atomic>
 #include <cstdint>
 #include <cstring>
+#include <mutex>
 
 namespace {
 
@@ -390,6 +391,36 @@ int mapped_device_pointer(const void* h, void** d) {
   return TOPKV_OK;
 }
 
+// ---- built-in staging slab of topkv_pack_layer_to_host_noalloc ---------------------------
+// Lives in the library's device image: present on every GPU that loads the library, shared by
+// all calls. In host code the name below is only a handle; the device address comes from
+// cudaGetSymbolAddress, looked up once per device.
+static __device__ __align__(256) unsigned char g_noalloc_staging[TOPKV_NOALLOC_STAGING_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+void* g_noalloc_addr[kMaxDevices] = {};
+
+int noalloc_staging_address(void** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev < 0 || dev >= kMaxDevices) return TOPKV_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (g_noalloc_addr[dev] == nullptr) {
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_noalloc_staging);  // address on the CURRENT device
+    if (e != cudaSuccess) {
+      cudaGetLastError();
+      return cuda_fail(e);
+    }
+    if (ptr == nullptr) return TOPKV_ERR_CUDA;
+    g_noalloc_addr[dev] = ptr;
+  }
+  *out = g_noalloc_addr[dev];
+  return TOPKV_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -486,6 +517,33 @@ int topkv_unpack_layer_from_host(int layer, void* dst_pool, const topkv_layout* 
   }
   kp.wire = static_cast<uint8_t*>(d_staging);
   return launch_copy<false>(kp, rs, (int)layout->kv_factor, s);
+}
+
+int topkv_pack_layer_to_host_noalloc(int layer, const void* src_pool, const topkv_layout* layout,
+                                     const topkv_batch* batch, void* h_pinned,
+                                     int64_t host_capacity_bytes, topkv_stream_t stream) {
+  KParams kp;
+  Resolved rs;
+  int64_t n_layer;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (batch != nullptr && batch->struct_size == sizeof(topkv_batch) && batch->total_tokens < 0)
+    return TOPKV_ERR_INVALID_ARG;
+  int st = prepare(layer, src_pool, layout, batch, h_pinned, host_capacity_bytes,
+                   layout ? layout->wire_layer_stride : 0, &kp, &rs, &n_layer);
+  if (st != TOPKV_OK) return st;
+  if (n_layer > (int64_t)TOPKV_NOALLOC_STAGING_BYTES) return TOPKV_ERR_CAPACITY;
+  void* staging = nullptr;
+  st = noalloc_staging_address(&staging);  // first call on this device: symbol lookup
+  if (st != TOPKV_OK) return st;
+  uint8_t* host_slab = kp.wire;
+  kp.wire = static_cast<uint8_t*>(staging);  // the device address, never the host-side handle
+  st = launch_copy<true>(kp, rs, (int)layout->kv_factor, s);
+  if (st != TOPKV_OK) return st;
+  if (n_layer > 0) {
+    const cudaError_t e = cudaMemcpyAsync(host_slab, staging, (size_t)n_layer, cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  return TOPKV_OK;
 }
 
 int topkv_build_plan(const topkv_batch* batch, int64_t* d_cu_seq_lens, topkv_stream_t stream) {
