@@ -96,7 +96,7 @@ typedef struct topkv_batch {
   uint32_t struct_size;          /* = sizeof(topkv_batch)                                   */
   int32_t num_requests;          /* R >= 0                                                  */
   int32_t max_pages_per_req;     /* block-table row width (columns)                         */
-  int32_t reserved;              /* must be 0                                               */
+  uint32_t flags;                /* 0 or TOPKV_FLAG_OVERLAP_PREVIOUS                        */
   const int32_t* block_table;    /* DEVICE int32 [R][max_pages_per_req]; columns at or past */
                                  /* ceil(s_r/P) are ignored (conventionally -1)             */
   const int32_t* seq_lens;       /* DEVICE int32 [R], each in [0, max_pages_per_req*P]      */
@@ -105,6 +105,17 @@ typedef struct topkv_batch {
   int64_t total_tokens;          /* T if the host knows it, else -1. When -1 the capacity   */
                                  /* checks are skipped and the caller guarantees them.      */
 } topkv_batch;
+
+/* topkv_batch.flags. Every copy kernel is launched so that it may become resident while the
+ * previous kernel of the stream drains, but by default it touches memory only after that
+ * kernel has finished. With TOPKV_FLAG_OVERLAP_PREVIOUS the caller declares that this call
+ * reads nothing and overwrites nothing that the kernels enqueued before it on `stream` write
+ * or read, back to the most recent call made WITHOUT the flag (or the most recent non-kernel
+ * operation, e.g. a copy or an event wait, which is always honoured). The call's kernel may
+ * then move data while those kernels finish their tails, e.g. pack of layer l+1 behind pack
+ * of layer l. Completion stays in stream order: whatever is enqueued after the call starts
+ * only after all of them are done. */
+#define TOPKV_FLAG_OVERLAP_PREVIOUS 1u
 
 /* Largest R for which cu_seq_lens may be NULL. */
 #define TOPKV_MAX_INLINE_R 1024
@@ -220,6 +231,10 @@ const char* topkv_strerror(int status);
 int topkv_version(void);
 /* cudaError_t of the most recent failing CUDA call made by this library on this thread. */
 int topkv_last_cuda_error(void);
+/* Synchronises the device and returns the error bits kernels of this library have raised on
+ * the current device since the library was loaded (0 = none; bit 0 = a bounded wait inside a
+ * kernel ran out, its output is incomplete), or a negative topkv_status. */
+int topkv_device_error_flags(void);
 /* Number of kernels this library has launched in this process (all threads). */
 int64_t topkv_kernel_launch_count(void);
 /* Selects the kernel family used by the four hot calls: 0 = vectorised load/store,

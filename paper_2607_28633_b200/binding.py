@@ -26,6 +26,7 @@ TOPKV_ERR_CUDA = -6
 TOPKV_KIND_GQA, TOPKV_KIND_MLA = 0, 1
 TOPKV_WIRE_TOKEN_KV, TOPKV_WIRE_PLANAR = 0, 1
 TOPKV_MAX_INLINE_R = 1024
+TOPKV_FLAG_OVERLAP_PREVIOUS = 1
 TOPKV_NOALLOC_STAGING_BYTES = 8 * 1024 * 1024
 
 # every symbol include/topkv.h declares
@@ -35,7 +36,7 @@ EXPORTS = (
     "topkv_layout_default_strides", "topkv_wire_layer_bytes", "topkv_kv_bytes",
     "topkv_model_transfer_s", "topkv_model_t_eff_s", "topkv_model_hidden_fraction",
     "topkv_strerror", "topkv_version", "topkv_last_cuda_error", "topkv_kernel_launch_count",
-    "topkv_set_kernel_variant", "topkv_pack_layer_to_host_noalloc",
+    "topkv_set_kernel_variant", "topkv_pack_layer_to_host_noalloc", "topkv_device_error_flags",
 )
 
 
@@ -54,7 +55,7 @@ class topkv_layout(ctypes.Structure):
 class topkv_batch(ctypes.Structure):
     _fields_ = [
         ("struct_size", c_uint32), ("num_requests", c_int32), ("max_pages_per_req", c_int32),
-        ("reserved", c_int32), ("block_table", c_void_p), ("seq_lens", c_void_p),
+        ("flags", c_uint32), ("block_table", c_void_p), ("seq_lens", c_void_p),
         ("cu_seq_lens", c_void_p), ("total_tokens", c_int64),
     ]
 
@@ -151,7 +152,8 @@ def make_layout(L: int, F: int, H: int, D: int, E: int, P: int, num_pool_pages: 
     return lo
 
 
-def make_batch(block_table, seq_lens, total_tokens: int = -1, cu_seq_lens=None) -> topkv_batch:
+def make_batch(block_table, seq_lens, total_tokens: int = -1, cu_seq_lens=None,
+               flags: int = 0) -> topkv_batch:
     """block_table: device int32 [R][maxp]; seq_lens: device int32 [R]. The caller keeps the
     tensors alive for as long as the descriptor is in use."""
     b = topkv_batch()
@@ -162,6 +164,7 @@ def make_batch(block_table, seq_lens, total_tokens: int = -1, cu_seq_lens=None) 
     b.seq_lens = _ptr(seq_lens)
     b.cu_seq_lens = _ptr(cu_seq_lens)
     b.total_tokens = total_tokens
+    b.flags = flags
     return b
 
 
@@ -247,6 +250,10 @@ def topkv_version():
 
 def topkv_last_cuda_error():
     return lib().topkv_last_cuda_error()
+
+
+def topkv_device_error_flags():
+    return lib().topkv_device_error_flags()
 
 
 def topkv_kernel_launch_count():

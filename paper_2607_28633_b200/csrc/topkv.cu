@@ -8,6 +8,10 @@
 
 #include <cuda_runtime.h>
 
+#include "topkv_bulk.cuh"
+#include "topkv_common.cuh"
+
+#include <algorithm>
 #include <atomic>
 #include <cstdint>
 #include <cstring>
@@ -15,25 +19,7 @@
 
 namespace {
 
-// ------------------------------------------------------------------------------------------
-// Kernel parameters (plain data, passed by value).
-// A "unit" is the largest run of bytes that is contiguous on both sides for one
-// (token, plane): the whole [head][dim] row when heads are contiguous in the pool,
-// otherwise one head (U = H units per row).
-// ------------------------------------------------------------------------------------------
-struct KParams {
-  uint8_t* pool;          // base of this layer's pool slab
-  uint8_t* wire;          // base of this layer's wire slab (device, or mapped pinned host)
-  const int32_t* bt;      // [R][maxp]
-  const int32_t* sl;      // [R]
-  const int64_t* cu;      // [R+1] or nullptr
-  int64_t T;              // total tokens or -1
-  int64_t S_page, S_kv, S_tok, S_unit;  // pool strides, bytes
-  int R, maxp, P;
-  int U;                  // units per (token, plane)
-  int unit_chunks;        // VEC-byte chunks per unit
-  int planar;             // wire order
-};
+using namespace topkv;
 
 constexpr int kThreads = 256;
 constexpr int kUnroll16 = 8;  // vectors in flight per thread, 16-byte vectors
@@ -110,8 +96,7 @@ __device__ __forceinline__ int64_t block_prefix(const int32_t* __restrict__ sl, 
 // wire -> pool; MERGED: the valid tokens of a page form one contiguous run per plane on
 // both sides (MLA rows, or PLANAR wire with a token-contiguous pool).
 template <int F, bool PACK, bool MERGED, int VEC>
-__global__ void __launch_bounds__(kThreads)
-topkv_page_copy_kernel(const KParams p) {
+__device__ __forceinline__ void copy_page(const KParams& p) {
   const int slot = blockIdx.x;
   const int r = slot / p.maxp;
   const int j = slot - r * p.maxp;
@@ -207,6 +192,14 @@ topkv_page_copy_kernel(const KParams p) {
   }
 }
 
+template <int F, bool PACK, bool MERGED, int VEC>
+__global__ void __launch_bounds__(kThreads)
+topkv_page_copy_kernel(const KParams p) {
+  pdl_prologue(p.overlap);
+  copy_page<F, PACK, MERGED, VEC>(p);
+  pdl_epilogue(p.overlap);
+}
+
 // Exclusive prefix sum of seq_lens into int64 [R+1]; one CTA, any R.
 __global__ void __launch_bounds__(kThreads)
 topkv_plan_kernel(const int32_t* __restrict__ sl, int R, int64_t* __restrict__ cu) {
@@ -291,7 +284,8 @@ int check_layout(const topkv_layout* lo, Resolved* out) {
 }
 
 int check_batch(const topkv_layout* lo, const topkv_batch* b) {
-  if (b == nullptr || b->struct_size != sizeof(topkv_batch) || b->reserved != 0)
+  if (b == nullptr || b->struct_size != sizeof(topkv_batch) ||
+      (b->flags & ~(uint32_t)TOPKV_FLAG_OVERLAP_PREVIOUS) != 0)
     return TOPKV_ERR_INVALID_ARG;
   if (b->num_requests < 0 || b->max_pages_per_req < 0 || b->total_tokens < -1)
     return TOPKV_ERR_INVALID_ARG;
@@ -340,6 +334,7 @@ int prepare(int layer, const void* pool, const topkv_layout* lo, const topkv_bat
   kp->U = rs->U;
   kp->unit_chunks = (int)(rs->unit_bytes / 16);
   kp->planar = lo->wire_order == TOPKV_WIRE_PLANAR;
+  kp->overlap = (b->flags & TOPKV_FLAG_OVERLAP_PREVIOUS) ? 1 : 0;
   return TOPKV_OK;
 }
 
@@ -347,29 +342,101 @@ template <bool PACK, int VEC>
 void launch_vec(const KParams& kp, bool merged, int F, dim3 grid, cudaStream_t stream) {
   const dim3 block(kThreads);
   if (merged) {
-    if (F == 1) topkv_page_copy_kernel<1, PACK, true, VEC><<<grid, block, 0, stream>>>(kp);
-    else topkv_page_copy_kernel<2, PACK, true, VEC><<<grid, block, 0, stream>>>(kp);
+    if (F == 1) launch_pdl(topkv_page_copy_kernel<1, PACK, true, VEC>, grid, block, 0, stream, kp);
+    else launch_pdl(topkv_page_copy_kernel<2, PACK, true, VEC>, grid, block, 0, stream, kp);
   } else {
-    if (F == 1) topkv_page_copy_kernel<1, PACK, false, VEC><<<grid, block, 0, stream>>>(kp);
-    else topkv_page_copy_kernel<2, PACK, false, VEC><<<grid, block, 0, stream>>>(kp);
+    if (F == 1) launch_pdl(topkv_page_copy_kernel<1, PACK, false, VEC>, grid, block, 0, stream, kp);
+    else launch_pdl(topkv_page_copy_kernel<2, PACK, false, VEC>, grid, block, 0, stream, kp);
   }
+}
+
+// ---- bulk-async family -------------------------------------------------------------------
+constexpr int kSmemBudget = 227 * 1024;   // opt-in dynamic shared memory per CTA on sm_100
+constexpr int kStageTarget = 36 * 1024;   // bytes of payload per ring stage
+
+struct DeviceInfo {
+  int sms = 0;
+  bool attr_set[4] = {false, false, false, false};
+};
+std::mutex g_devinfo_mutex;
+DeviceInfo g_devinfo[64];
+
+template <int F, bool PACK>
+int bulk_prepare_device(int* sms_out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev < 0 || dev >= 64) return TOPKV_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_devinfo_mutex);
+  DeviceInfo& di = g_devinfo[dev];
+  if (di.sms == 0) {
+    e = cudaDeviceGetAttribute(&di.sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  const int idx = (F - 1) * 2 + (PACK ? 1 : 0);
+  if (!di.attr_set[idx]) {
+    e = cudaFuncSetAttribute(topkv_bulk_kernel<F, PACK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kSmemBudget);
+    if (e != cudaSuccess) return cuda_fail(e);
+    di.attr_set[idx] = true;
+  }
+  *sms_out = di.sms;
+  return TOPKV_OK;
+}
+
+// Launches the bulk-async kernel when the shape fits its shared-memory ring; *handled tells
+// the caller whether it did (otherwise the vectorised family takes over).
+template <bool PACK>
+int launch_bulk(const KParams& kp0, const Resolved& rs, int F, cudaStream_t stream, bool* handled) {
+  *handled = false;
+  if (kp0.R > kBulkMaxR) return TOPKV_OK;
+  const int64_t tok_bytes = (int64_t)F * rs.row_bytes;
+  if (tok_bytes > kStageTarget || rs.unit_bytes > 0x7fffffff) return TOPKV_OK;
+  BulkParams bp;
+  bp.k = kp0;
+  bp.k.unit_chunks = (int)(rs.unit_bytes / 16);
+  bp.tpc = (int)std::min<int64_t>(kp0.P, kStageTarget / tok_bytes);
+  bp.cpp = (kp0.P + bp.tpc - 1) / bp.tpc;
+  bp.tpc = (kp0.P + bp.cpp - 1) / bp.cpp;  // even split of the page
+  bp.stage_bytes = (int)((bp.tpc * tok_bytes + 127) / 128 * 128);
+  bp.merged = rs.merged ? 1 : 0;
+  const int fixed = kBulkWarps * kBulkMaxStages * (int)(sizeof(uint64_t) + sizeof(ItemDesc)) +
+                    2 * (kp0.R + 1) * (int)sizeof(int32_t);
+  bp.nstages = std::min(kBulkMaxStages, (kSmemBudget - fixed) / (kBulkWarps * bp.stage_bytes));
+  if (bp.nstages < 2) return TOPKV_OK;
+  const size_t smem = (size_t)kBulkWarps * bp.nstages * bp.stage_bytes + fixed;
+  int sms = 0;
+  int st = (F == 1) ? bulk_prepare_device<1, PACK>(&sms) : bulk_prepare_device<2, PACK>(&sms);
+  if (st != TOPKV_OK) return st;
+  const dim3 grid((unsigned)sms), block(kBulkThreads);
+  if (F == 1) launch_pdl(topkv_bulk_kernel<1, PACK>, grid, block, smem, stream, bp);
+  else launch_pdl(topkv_bulk_kernel<2, PACK>, grid, block, smem, stream, bp);
+  *handled = true;
+  return TOPKV_OK;
 }
 
 template <bool PACK>
 int launch_copy(KParams kp, const Resolved& rs, int F, cudaStream_t stream) {
   const int64_t slots = (int64_t)kp.R * kp.maxp;
   if (slots == 0) return TOPKV_OK;
-  const dim3 grid((unsigned)slots);
-  // 32-byte vectors when every address the kernel can form is 32-byte aligned
-  const bool wide = ((reinterpret_cast<uintptr_t>(kp.pool) | reinterpret_cast<uintptr_t>(kp.wire) |
-                      (uintptr_t)kp.S_page | (uintptr_t)kp.S_kv | (uintptr_t)kp.S_tok |
-                      (uintptr_t)kp.S_unit | (uintptr_t)rs.unit_bytes) & 31) == 0;
-  if (wide) {
-    kp.unit_chunks = (int)(rs.unit_bytes / 32);
-    launch_vec<PACK, 32>(kp, rs.merged, F, grid, stream);
-  } else {
-    kp.unit_chunks = (int)(rs.unit_bytes / 16);
-    launch_vec<PACK, 16>(kp, rs.merged, F, grid, stream);
+  bool handled = false;
+  if (g_variant.load(std::memory_order_relaxed) == 1) {
+    const int st = launch_bulk<PACK>(kp, rs, F, stream, &handled);
+    if (st != TOPKV_OK) return st;
+  }
+  if (!handled) {
+    const dim3 grid((unsigned)slots);
+    // 32-byte vectors when every address the kernel can form is 32-byte aligned
+    const bool wide = ((reinterpret_cast<uintptr_t>(kp.pool) | reinterpret_cast<uintptr_t>(kp.wire) |
+                        (uintptr_t)kp.S_page | (uintptr_t)kp.S_kv | (uintptr_t)kp.S_tok |
+                        (uintptr_t)kp.S_unit | (uintptr_t)rs.unit_bytes) & 31) == 0;
+    if (wide) {
+      kp.unit_chunks = (int)(rs.unit_bytes / 32);
+      launch_vec<PACK, 32>(kp, rs.merged, F, grid, stream);
+    } else {
+      kp.unit_chunks = (int)(rs.unit_bytes / 16);
+      launch_vec<PACK, 16>(kp, rs.merged, F, grid, stream);
+    }
   }
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
@@ -560,6 +627,13 @@ int topkv_build_plan(const topkv_batch* batch, int64_t* d_cu_seq_lens, topkv_str
 }
 
 int topkv_last_cuda_error(void) { return g_last_cuda_error; }
+
+int topkv_device_error_flags(void) {
+  int flags = 0;
+  const cudaError_t e = cudaMemcpyFromSymbol(&flags, g_device_error_flags, sizeof(int));
+  if (e != cudaSuccess) return cuda_fail(e);
+  return flags;
+}
 int64_t topkv_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 int topkv_set_kernel_variant(int variant) {

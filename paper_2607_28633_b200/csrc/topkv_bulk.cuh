@@ -82,6 +82,7 @@ template <int F, bool PACK>
 __global__ void __launch_bounds__(kBulkThreads, 1) topkv_bulk_kernel(const BulkParams bp) {
   extern __shared__ __align__(128) uint8_t smem[];
   const KParams& p = bp.k;
+  pdl_prologue(p.overlap);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int S = bp.nstages;
 
@@ -264,6 +265,7 @@ __global__ void __launch_bounds__(kBulkThreads, 1) topkv_bulk_kernel(const BulkP
   }
   if (failed && lane == 0) atomicOr(&g_device_error_flags, 1);
   bulk_wait_all();
+  pdl_epilogue(p.overlap);
 }
 
 }  // namespace topkv

@@ -1,0 +1,68 @@
+// Types shared by the TopKV kernels (device side) and their host launchers.
+#pragma once
+#include <cstdint>
+
+#include <cuda_runtime.h>
+
+#include "topkv.h"
+
+namespace topkv {
+
+// ------------------------------------------------------------------------------------------
+// Kernel parameters (plain data, passed by value).
+// A "unit" is the largest run of bytes that is contiguous on both sides for one
+// (token, plane): the whole [head][dim] row when heads are contiguous in the pool,
+// otherwise one head (U = H units per row).
+// ------------------------------------------------------------------------------------------
+struct KParams {
+  uint8_t* pool;          // base of this layer's pool slab
+  uint8_t* wire;          // base of this layer's wire slab (device, or mapped pinned host)
+  const int32_t* bt;      // [R][maxp]
+  const int32_t* sl;      // [R]
+  const int64_t* cu;      // [R+1] or nullptr
+  int64_t T;              // total tokens or -1
+  int64_t S_page, S_kv, S_tok, S_unit;  // pool strides, bytes
+  int R, maxp, P;
+  int U;                  // units per (token, plane)
+  int unit_chunks;        // VEC-byte chunks per unit
+  int planar;             // wire order
+  int overlap;            // 1: caller declared this launch independent of the kernels before it
+};
+
+// Programmatic dependent launch. Every copy kernel is launched with programmatic stream
+// serialisation, so its CTAs may become resident while the previous kernel of the stream
+// drains. By default a kernel waits for that previous kernel to finish (and its writes to be
+// visible) before it reads anything; a launch the caller declared independent skips the wait
+// and only holds one thread back at its end, so that kernels still COMPLETE in stream order.
+__device__ __forceinline__ void pdl_wait_prior_grid() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_release_next_grid() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_prologue(int overlap) {
+  if (!overlap) pdl_wait_prior_grid();
+  pdl_release_next_grid();
+}
+__device__ __forceinline__ void pdl_epilogue(int overlap) {
+  if (overlap && blockIdx.x == 0 && threadIdx.x == 0) pdl_wait_prior_grid();
+}
+
+// Launch with programmatic stream serialisation allowed (see pdl_prologue above).
+template <typename P>
+cudaError_t launch_pdl(void (*kernel)(const P), dim3 grid, dim3 block, size_t smem,
+                       cudaStream_t stream, const P& params) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, params);
+}
+
+}  // namespace topkv

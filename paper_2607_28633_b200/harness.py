@@ -4,7 +4,8 @@ per-layer calls through the C-ABI binding. No pack / unpack arithmetic happens h
 the CPU oracle is never imported."""
 from __future__ import annotations
 
-from dataclasses import dataclass
+import ctypes
+from dataclasses import dataclass, field
 
 import numpy as np
 import torch
@@ -28,20 +29,36 @@ class DeviceWorkload:
     cu: torch.Tensor            # int64 [R+1], filled by topkv_build_plan
     src_batch: tk.topkv_batch
     dst_batch: tk.topkv_batch
+    _overlap_batches: dict = field(default_factory=dict)
 
     @property
     def slab_bytes(self) -> int:
         return self.layout.pool_layer_stride
 
-    def pack(self, layer: int, stream=None, wire=None):
-        w = self.wire if wire is None else wire
-        return tk.check(tk.topkv_pack_layer(layer, self.src_pool, self.layout, self.src_batch, w,
-                                            w.numel(), stream))
+    def _flagged(self, batch: tk.topkv_batch, overlap: bool) -> tk.topkv_batch:
+        if not overlap:
+            return batch
+        key = id(batch)
+        if key not in self._overlap_batches:
+            b = tk.topkv_batch()
+            ctypes.memmove(ctypes.byref(b), ctypes.byref(batch), ctypes.sizeof(b))
+            b.flags = tk.TOPKV_FLAG_OVERLAP_PREVIOUS
+            self._overlap_batches[key] = b
+        return self._overlap_batches[key]
 
-    def unpack(self, layer: int, stream=None, wire=None):
+    def pack(self, layer: int, stream=None, wire=None, overlap: bool = False):
+        """overlap=True declares the call independent of the kernels enqueued just before it
+        (TOPKV_FLAG_OVERLAP_PREVIOUS): true for pack(l+1) after pack(l)."""
         w = self.wire if wire is None else wire
-        return tk.check(tk.topkv_unpack_layer(layer, self.dst_pool, self.layout, self.dst_batch, w,
-                                              w.numel(), stream))
+        return tk.check(tk.topkv_pack_layer(layer, self.src_pool, self.layout,
+                                            self._flagged(self.src_batch, overlap), w, w.numel(),
+                                            stream))
+
+    def unpack(self, layer: int, stream=None, wire=None, overlap: bool = False):
+        w = self.wire if wire is None else wire
+        return tk.check(tk.topkv_unpack_layer(layer, self.dst_pool, self.layout,
+                                              self._flagged(self.dst_batch, overlap), w, w.numel(),
+                                              stream))
 
     def pack_to_host(self, layer: int, h_pinned, staging=None, stream=None):
         return tk.check(tk.topkv_pack_layer_to_host(

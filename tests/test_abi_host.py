@@ -112,6 +112,8 @@ def test_argument_validation_without_gpu():
     assert P(0, pool, bad, b, wire, cap) == tk.TOPKV_ERR_ALIGNMENT
     bb = _batch(); bb.struct_size = 4
     assert P(0, pool, lo, bb, wire, cap) == tk.TOPKV_ERR_INVALID_ARG
+    bb = _batch(); bb.flags = 2                              # unknown flag bit
+    assert P(0, pool, lo, bb, wire, cap) == tk.TOPKV_ERR_INVALID_ARG
     bb = _batch(); bb.seq_lens = None
     assert P(0, pool, lo, bb, wire, cap) == tk.TOPKV_ERR_INVALID_ARG
     bb = _batch(R=tk.TOPKV_MAX_INLINE_R + 1, T=-1)          # no plan for a large batch

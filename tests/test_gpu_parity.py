@@ -23,6 +23,15 @@ def dev():
     return torch.device("cuda:0")
 
 
+@pytest.fixture(autouse=True, params=[0, 1], ids=["vec", "bulk"])
+def variant(request, dev):
+    """Every test runs once per kernel family (vectorised load/store, bulk-async ring)."""
+    prev = tk.topkv_set_kernel_variant(request.param)
+    yield request.param
+    tk.topkv_set_kernel_variant(prev)
+    assert tk.topkv_device_error_flags() == 0
+
+
 def _geom(spec, npages, L, wire_order, W_layer):
     return Geom(L=L, F=spec.F, h_kv=spec.H, d_h=spec.D, b_p=spec.E, P=spec.P, num_pages=npages,
                 wire_order=wire_order, W_layer=W_layer)
@@ -258,6 +267,36 @@ def test_cfg2_full_size_sampled_layers(dev):
                       + (i % s.P) * s.row_bytes)
                 wo = layer * w.n_layer + ((cu[r] + i) * s.F + c) * s.row_bytes
                 assert torch.equal(w.src_pool[po:po + s.row_bytes], w.wire[wo:wo + s.row_bytes])
+    del w
+    torch.cuda.empty_cache()
+
+
+def test_overlapped_launches_keep_results_and_order(dev):
+    """TOPKV_FLAG_OVERLAP_PREVIOUS on every layer after the first: results are unchanged, and
+    work enqueued after the chain (a copy on the same stream) sees all of it."""
+    spec = wl.with_layers(wl.CFG2, 6)
+    w = harness.setup(spec, dev)
+    b, s = w.batch, spec
+    g = _geom(s, b.num_pool_pages, 1, 0, 0)
+    stream = torch.cuda.Stream(dev)
+    host_wire = torch.empty(w.wire.numel(), dtype=torch.uint8).pin_memory()
+    host_dst = torch.empty(w.dst_pool.numel(), dtype=torch.uint8).pin_memory()
+    dst_before = [harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, l) for l in range(s.L)]
+    with torch.cuda.stream(stream):
+        for l in range(s.L):
+            w.pack(l, stream, overlap=l > 0)
+        host_wire.copy_(w.wire, non_blocking=True)          # right behind the chain
+        for l in range(s.L):
+            w.unpack(l, stream, overlap=l > 0)              # unpack(0) waits for the packs
+        host_dst.copy_(w.dst_pool, non_blocking=True)
+    stream.synchronize()
+    for l in range(s.L):
+        src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, l)
+        want = oracle.pack(g, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=8)
+        assert np.array_equal(host_wire[l * w.n_layer:(l + 1) * w.n_layer].numpy(), want), l
+        oracle.unpack(g, 0, dst_before[l], b.dst_block_table, b.seq_lens, want, impl="rows", threads=8)
+        assert np.array_equal(host_dst[l * w.slab_bytes:(l + 1) * w.slab_bytes].numpy(),
+                              dst_before[l]), l
     del w
     torch.cuda.empty_cache()
 
