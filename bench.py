@@ -32,10 +32,10 @@ METRIC = "kv_pack_unpack_GBps"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM traffic of one pack launch relative to its algorithmic bytes, from the ncu capture
-# summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over 2*N_layer).
-# None until a capture exists.
-NCU_TRAFFIC_RATIO = None
+# DRAM traffic of one pack launch relative to its algorithmic bytes, from the steady-state ncu
+# capture summarised in profiles/page_copy_kernel_pack_cfg2_4layers.md
+# ((dram__bytes_read.sum + dram__bytes_write.sum) / (2*N_layer), same per-launch size as here).
+NCU_TRAFFIC_RATIO = 0.995
 
 
 def measured_peak_gbs():
