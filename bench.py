@@ -446,15 +446,13 @@ def main():
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if rank == 0:
         entry.build()
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        torch.cuda.set_device(local)
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-        dist.barrier()
-    tk.lib()
+    from paper_2607_28633_b200 import dist_util
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
+    dist = dist_util.init("nccl", dev)
+    if dist is not None:
+        dist.barrier()
+    tk.lib()
     if args.variant is not None:
         tk.check(tk.topkv_set_kernel_variant(args.variant))
 
@@ -464,18 +462,10 @@ def main():
         torch.cuda.synchronize(dev)
 
     def max_over_ranks(x: float) -> float:
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return dist_util.max_over_ranks(dist, x, dev)
 
     def sum_over_ranks(x: float) -> float:
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.SUM)
-        return float(t.item())
+        return dist_util.sum_over_ranks(dist, x, dev)
 
     peak, peak_src = measured_peak_gbs()
     spec = wl.CFG2 if args.layers is None else wl.with_layers(wl.CFG2, args.layers)

@@ -358,6 +358,34 @@ def test_host_leg_cfg3_shape_two_layers(dev):
     torch.cuda.empty_cache()
 
 
+def test_side_stream_overlap_run_is_bit_exact(dev, variant):
+    """The layer-by-layer side-stream issue under the GEMM stand-in (reduced: 6 layers, ring of
+    4 pinned slots): what lands in pinned memory is the oracle's wire slab of that layer."""
+    if variant == 1:
+        pytest.skip("the overlap driver is kernel-family agnostic; run once")
+    from paper_2607_28633_b200 import overlap
+    spec = wl.with_layers(wl.CFG5, 6)
+    w = harness.setup(spec, dev, need_dst=False, need_wire=False)
+    b, s = w.batch, spec
+    g = _geom(s, b.num_pool_pages, 1, 0, 0)
+    slots = 4
+    pre = overlap.PrefillStandIn(dev, 7, tokens=1024, hidden=2048, ffn=4096)
+    staging = torch.zeros(w.n_layer, dtype=torch.uint8, device=dev)
+    for st in (staging, None):
+        pinned = torch.zeros(slots * w.n_layer, dtype=torch.uint8).pin_memory()
+        r = overlap.run_overlap(w, pinned, st, pre, slots=slots, warmup_layers=1)
+        assert r.layers == 6 and r.t_xfer_serial_ms > 0 and 0.0 <= r.hidden <= 1.0
+        assert r.hidden_upper_bound == pytest.approx(1 - 1 / 6)
+        # the ring holds the last `slots` layers: 2, 3 in slots 2, 3 and 4, 5 in slots 0, 1
+        for layer in (2, 3, 4, 5):
+            src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, layer)
+            want = oracle.pack(g, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=8)
+            slot = layer % slots
+            assert np.array_equal(pinned[slot * w.n_layer:(slot + 1) * w.n_layer].numpy(), want)
+    del w
+    torch.cuda.empty_cache()
+
+
 def test_smoke_entry(dev):
     import __graft_entry__ as entry
     entry.smoke()
