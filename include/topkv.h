@@ -231,10 +231,18 @@ const char* topkv_strerror(int status);
 int topkv_version(void);
 /* cudaError_t of the most recent failing CUDA call made by this library on this thread. */
 int topkv_last_cuda_error(void);
-/* Synchronises the device and returns the error bits kernels of this library have raised on
- * the current device since the library was loaded (0 = none; bit 0 = a bounded wait inside a
- * kernel ran out, its output is incomplete), or a negative topkv_status. */
+/* Device-side checks. Kernels never trap; when a device table is unusable they skip the
+ * affected work and raise a bit in a per-device status word:
+ *   1  a bounded wait inside a kernel ran out (output incomplete)
+ *   2  a page id lay outside [0, num_pool_pages) or a length exceeded its block-table row:
+ *      those pages were skipped, nothing outside the pool was touched
+ *   4  the lengths found on the device did not fit the wire slab (N_layer when total_tokens is
+ *      known, else the capacity passed): that work was skipped, nothing outside was touched
+ * topkv_device_error_flags() synchronises the device and returns the bits raised on the current
+ * device since the library was loaded or the flags were last reset (0 = none), or a negative
+ * topkv_status; topkv_reset_device_error_flags() clears them. */
 int topkv_device_error_flags(void);
+int topkv_reset_device_error_flags(void);
 /* Number of kernels this library has launched in this process (all threads). */
 int64_t topkv_kernel_launch_count(void);
 /* Selects the kernel family used by the four hot calls: 0 = vectorised load/store,

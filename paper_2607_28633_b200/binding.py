@@ -37,6 +37,7 @@ EXPORTS = (
     "topkv_model_transfer_s", "topkv_model_t_eff_s", "topkv_model_hidden_fraction",
     "topkv_strerror", "topkv_version", "topkv_last_cuda_error", "topkv_kernel_launch_count",
     "topkv_set_kernel_variant", "topkv_pack_layer_to_host_noalloc", "topkv_device_error_flags",
+    "topkv_reset_device_error_flags",
 )
 
 
@@ -154,8 +155,8 @@ def make_layout(L: int, F: int, H: int, D: int, E: int, P: int, num_pool_pages: 
 
 def make_batch(block_table, seq_lens, total_tokens: int = -1, cu_seq_lens=None,
                flags: int = 0) -> topkv_batch:
-    """block_table: device int32 [R][maxp]; seq_lens: device int32 [R]. The caller keeps the
-    tensors alive for as long as the descriptor is in use."""
+    """block_table: device int32 [R][maxp]; seq_lens: device int32 [R]. The descriptor keeps a
+    reference to the tensors it was built from."""
     b = topkv_batch()
     b.struct_size = ctypes.sizeof(topkv_batch)
     b.num_requests = int(block_table.shape[0])
@@ -165,6 +166,9 @@ def make_batch(block_table, seq_lens, total_tokens: int = -1, cu_seq_lens=None,
     b.cu_seq_lens = _ptr(cu_seq_lens)
     b.total_tokens = total_tokens
     b.flags = flags
+    # The struct only holds addresses: keep the tensors alive with it, so that a temporary
+    # passed here cannot be freed (and its memory reused) while the descriptor is in use.
+    b._keepalive = (block_table, seq_lens, cu_seq_lens)
     return b
 
 
@@ -254,6 +258,10 @@ def topkv_last_cuda_error():
 
 def topkv_device_error_flags():
     return lib().topkv_device_error_flags()
+
+
+def topkv_reset_device_error_flags():
+    return lib().topkv_reset_device_error_flags()
 
 
 def topkv_kernel_launch_count():

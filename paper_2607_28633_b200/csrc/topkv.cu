@@ -22,6 +22,9 @@ namespace {
 using namespace topkv;
 
 constexpr int kThreads = 256;
+constexpr int kMinCtasPerSm = 3;  // register cap: 3 x 256 threads resident per SM
+constexpr int kMaxPagesPerCta = 64;
+constexpr int64_t kSpanTargetBytes = 64 * 1024;  // bytes one CTA of the vectorised family moves
 constexpr int kUnroll16 = 8;  // vectors in flight per thread, 16-byte vectors
 constexpr int kUnroll32 = 4;  // and 32-byte vectors
 
@@ -95,15 +98,24 @@ __device__ __forceinline__ int64_t block_prefix(const int32_t* __restrict__ sl, 
 // One CTA per (request, page column). F: planes per token; PACK: pool -> wire, else
 // wire -> pool; MERGED: the valid tokens of a page form one contiguous run per plane on
 // both sides (MLA rows, or PLANAR wire with a token-contiguous pool).
-template <int F, bool PACK, bool MERGED, int VEC>
-__device__ __forceinline__ void copy_page(const KParams& p) {
+template <int F, bool PACK, bool MERGED, int VEC, bool MULTI>
+__device__ __forceinline__ void copy_span(const KParams& p) {
+  // A span = `ppc` consecutive page columns of one request (one page when pages are large;
+  // several small pages, so that every CTA moves a few tens of KiB).
+  __shared__ int32_t s_pages[kMaxPagesPerCta];
   const int slot = blockIdx.x;
-  const int r = slot / p.maxp;
-  const int j = slot - r * p.maxp;
+  const int r = slot / p.spr;
+  const int j0 = (slot - r * p.spr) * p.ppc;
   const int s_r = p.sl[r];
-  const int first = j * p.P;
+  const int first = j0 * p.P;
   if (first >= s_r) return;
-  const int v = min(p.P, s_r - first);  // valid tokens in this page
+  int v = min(p.ppc * p.P, s_r - first);  // valid tokens in this span
+  const int tid = threadIdx.x;
+  if (s_r > p.maxp * p.P) {  // length longer than its block-table row: copy what the row holds
+    v = min(v, (p.maxp - j0) * p.P);
+    if (tid == 0) raise_error(kErrTable);
+  }
+  const int npages = (v + p.P - 1) / p.P;
 
   int64_t cu_r, T = p.T;
   if (p.cu != nullptr) {
@@ -114,89 +126,123 @@ __device__ __forceinline__ void copy_page(const KParams& p) {
     cu_r = block_prefix(p.sl, (p.planar && T < 0) ? p.R : r, r, &total);
     if (p.planar && T < 0) T = total;
   }
-  const int64_t page = p.bt[(int64_t)r * p.maxp + j];
-  uint8_t* pool_page = p.pool + page * p.S_page;
-  const int64_t n0 = cu_r + first;  // global index of the page's first token
+  if (tid < npages) {
+    int pg = p.bt[(int64_t)r * p.maxp + j0 + tid];
+    if (pg < 0 || pg >= p.num_pages) {  // unusable entry: the page is skipped, nothing is touched
+      pg = -1;
+      raise_error(kErrTable);
+    }
+    s_pages[tid] = pg;
+  }
+  __syncthreads();
+  const int64_t n0 = cu_r + first;  // global index of the span's first token
   const int64_t unit_bytes = (int64_t)p.unit_chunks * VEC;
+  {  // the span must lie inside the wire slab, whatever lengths the device tables hold
+    const int64_t row = unit_bytes * p.U;
+    const bool fits = p.planar ? (n0 >= 0 && n0 + v <= T && T * F * row <= p.wire_limit)
+                               : (n0 >= 0 && (n0 + v) * F * row <= p.wire_limit);
+    if (!fits) {
+      if (tid == 0) raise_error(kErrWire);
+      return;
+    }
+  }
   constexpr int kUnroll = VEC == 32 ? kUnroll32 : kUnroll16;
-  const int tid = threadIdx.x;
 
   if (MERGED) {
-    // F runs of v * row bytes each (U == 1 here).
-    const int n = v * p.unit_chunks;
+    // per page, F runs of (valid tokens) * row bytes each (U == 1 here)
+    for (int jj = 0; jj < npages; ++jj) {
+      if (s_pages[jj] < 0) continue;
+      const int vj = min(p.P, v - jj * p.P);
+      const int n = vj * p.unit_chunks;
+      uint8_t* pool_page = p.pool + (int64_t)s_pages[jj] * p.S_page;
 #pragma unroll
-    for (int c = 0; c < F; ++c) {
-      uint8_t* a = pool_page + c * p.S_kv;
-      uint8_t* b = p.wire + ((p.planar ? c * T : 0) + n0) * unit_bytes;  // not planar => F == 1
-      const uint8_t* src = PACK ? a : b;
-      uint8_t* dst = PACK ? b : a;
-      for (int w0 = tid; w0 < n; w0 += kThreads * kUnroll) {
-        Vec<VEC> buf[kUnroll];
+      for (int c = 0; c < F; ++c) {
+        uint8_t* a = pool_page + c * p.S_kv;
+        // not planar => F == 1
+        uint8_t* b = p.wire + ((p.planar ? c * T : 0) + n0 + (int64_t)jj * p.P) * unit_bytes;
+        const uint8_t* src = PACK ? a : b;
+        uint8_t* dst = PACK ? b : a;
+        for (int w0 = tid; w0 < n; w0 += kThreads * kUnroll) {
+          Vec<VEC> buf[kUnroll];
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-          const int w = w0 + u * kThreads;
-          if (w < n) buf[u].load(src + (int64_t)w * VEC);
-        }
+          for (int u = 0; u < kUnroll; ++u) {
+            const int w = w0 + u * kThreads;
+            if (w < n) buf[u].load(src + (int64_t)w * VEC);
+          }
 #pragma unroll
-        for (int u = 0; u < kUnroll; ++u) {
-          const int w = w0 + u * kThreads;
-          if (w < n) buf[u].store(dst + (int64_t)w * VEC);
+          for (int u = 0; u < kUnroll; ++u) {
+            const int w = w0 + u * kThreads;
+            if (w < n) buf[u].store(dst + (int64_t)w * VEC);
+          }
         }
       }
     }
     return;
   }
 
-  // Units of this page in wire order: q = (t*F + c)*U + h  (TOKEN_KV), or
-  // q = (c*v + t)*U + h (PLANAR). `tpu` threads cooperate on one unit.
+  // Units of the span in wire order: q = (ts*F + c)*U + h (TOKEN_KV) or q = (c*v + ts)*U + h
+  // (PLANAR), ts = token index inside the span. `tpu` threads cooperate on one unit.
   const int nunits = v * F * p.U;
   const int tpu = min(p.unit_chunks, kThreads);
   const int groups = kThreads / tpu;
   const int my_g = tid / tpu;
   const int my_w = tid - my_g * tpu;
   if (my_g >= groups) return;
-  uint8_t* wire_page = p.wire + n0 * F * p.U * unit_bytes;  // TOKEN_KV: the page is one run
+  uint8_t* wire_span = p.wire + n0 * F * p.U * unit_bytes;  // TOKEN_KV: the span is one run
+  if (!MULTI && s_pages[0] < 0) return;                     // single page, unusable: skip it
+  uint8_t* page0 = p.pool + (int64_t)s_pages[0] * p.S_page;
 
   for (int q0 = my_g; q0 < nunits; q0 += groups * kUnroll) {
     for (int w = my_w; w < p.unit_chunks; w += tpu) {
       Vec<VEC> buf[kUnroll];
-      uint8_t* a[kUnroll];
-      uint8_t* b[kUnroll];
+      uint8_t* dstp[kUnroll];  // only the store side is kept across the batch of loads
+      bool ok[kUnroll];
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
-        const int q = q0 + u * groups;
+        const int q = min(q0 + u * groups, nunits - 1);  // clamped: addresses stay valid
         int h = 0, tc = q;
         if (p.U > 1) {
           tc = q / p.U;
           h = q - tc * p.U;
         }
-        int c, t;
+        int c, ts;
+        uint8_t *a, *b;
         if (p.planar) {
           c = (F > 1 && tc >= v) ? 1 : 0;
-          t = tc - c * v;
-          b[u] = p.wire + (((int64_t)c * T + n0 + t) * p.U + h) * unit_bytes + (int64_t)w * VEC;
+          ts = tc - c * v;
+          b = p.wire + (((int64_t)c * T + n0 + ts) * p.U + h) * unit_bytes + (int64_t)w * VEC;
         } else {
-          t = tc / F;
-          c = tc - t * F;
-          b[u] = wire_page + (int64_t)q * unit_bytes + (int64_t)w * VEC;
+          ts = tc / F;
+          c = tc - ts * F;
+          b = wire_span + (int64_t)q * unit_bytes + (int64_t)w * VEC;
         }
-        a[u] = pool_page + c * p.S_kv + t * p.S_tok + h * p.S_unit + (int64_t)w * VEC;
-        if (q < nunits) buf[u].load(PACK ? a[u] : b[u]);
+        if (MULTI) {  // several pages per span: look the token's page up
+          const int jj = ts / p.P;
+          const int t = ts - jj * p.P;
+          const int pg = s_pages[jj];
+          a = p.pool + (int64_t)pg * p.S_page + c * p.S_kv + t * p.S_tok + h * p.S_unit +
+              (int64_t)w * VEC;
+          ok[u] = q0 + u * groups < nunits && pg >= 0;
+        } else {
+          a = page0 + c * p.S_kv + ts * p.S_tok + h * p.S_unit + (int64_t)w * VEC;
+          ok[u] = q0 + u * groups < nunits;
+        }
+        dstp[u] = PACK ? b : a;
+        if (ok[u]) buf[u].load(PACK ? a : b);
       }
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u) {
-        const int q = q0 + u * groups;
-        if (q < nunits) buf[u].store(PACK ? b[u] : a[u]);
+        if (ok[u]) buf[u].store(dstp[u]);
       }
     }
   }
 }
 
-template <int F, bool PACK, bool MERGED, int VEC>
-__global__ void __launch_bounds__(kThreads)
+template <int F, bool PACK, bool MERGED, int VEC, bool MULTI>
+__global__ void __launch_bounds__(kThreads, kMinCtasPerSm)
 topkv_page_copy_kernel(const KParams p) {
   pdl_prologue(p.overlap);
-  copy_page<F, PACK, MERGED, VEC>(p);
+  copy_span<F, PACK, MERGED, VEC, MULTI>(p);
   pdl_epilogue(p.overlap);
 }
 
@@ -335,19 +381,29 @@ int prepare(int layer, const void* pool, const topkv_layout* lo, const topkv_bat
   kp->unit_chunks = (int)(rs->unit_bytes / 16);
   kp->planar = lo->wire_order == TOPKV_WIRE_PLANAR;
   kp->overlap = (b->flags & TOPKV_FLAG_OVERLAP_PREVIOUS) ? 1 : 0;
+  kp->ppc = 1;
+  kp->spr = kp->maxp;
+  kp->num_pages = lo->num_pool_pages;
+  kp->wire_limit = n_layer >= 0 ? n_layer : capacity - (int64_t)layer * wire_layer_stride;
   return TOPKV_OK;
+}
+
+template <bool PACK, int VEC, bool MULTI>
+void launch_vec2(const KParams& kp, bool merged, int F, dim3 grid, cudaStream_t stream) {
+  const dim3 block(kThreads);
+  if (merged) {
+    if (F == 1) launch_pdl(topkv_page_copy_kernel<1, PACK, true, VEC, MULTI>, grid, block, 0, stream, kp);
+    else launch_pdl(topkv_page_copy_kernel<2, PACK, true, VEC, MULTI>, grid, block, 0, stream, kp);
+  } else {
+    if (F == 1) launch_pdl(topkv_page_copy_kernel<1, PACK, false, VEC, MULTI>, grid, block, 0, stream, kp);
+    else launch_pdl(topkv_page_copy_kernel<2, PACK, false, VEC, MULTI>, grid, block, 0, stream, kp);
+  }
 }
 
 template <bool PACK, int VEC>
 void launch_vec(const KParams& kp, bool merged, int F, dim3 grid, cudaStream_t stream) {
-  const dim3 block(kThreads);
-  if (merged) {
-    if (F == 1) launch_pdl(topkv_page_copy_kernel<1, PACK, true, VEC>, grid, block, 0, stream, kp);
-    else launch_pdl(topkv_page_copy_kernel<2, PACK, true, VEC>, grid, block, 0, stream, kp);
-  } else {
-    if (F == 1) launch_pdl(topkv_page_copy_kernel<1, PACK, false, VEC>, grid, block, 0, stream, kp);
-    else launch_pdl(topkv_page_copy_kernel<2, PACK, false, VEC>, grid, block, 0, stream, kp);
-  }
+  if (kp.ppc > 1) launch_vec2<PACK, VEC, true>(kp, merged, F, grid, stream);
+  else launch_vec2<PACK, VEC, false>(kp, merged, F, grid, stream);
 }
 
 // ---- bulk-async family -------------------------------------------------------------------
@@ -392,6 +448,7 @@ int launch_bulk(const KParams& kp0, const Resolved& rs, int F, cudaStream_t stre
   if (kp0.R > kBulkMaxR) return TOPKV_OK;
   const int64_t tok_bytes = (int64_t)F * rs.row_bytes;
   if (tok_bytes > kStageTarget || rs.unit_bytes > 0x7fffffff) return TOPKV_OK;
+  if (!rs.merged && rs.unit_bytes < 1024) return TOPKV_OK;  // per-copy cost dominates small units
   BulkParams bp;
   bp.k = kp0;
   bp.k.unit_chunks = (int)(rs.unit_bytes / 16);
@@ -425,7 +482,11 @@ int launch_copy(KParams kp, const Resolved& rs, int F, cudaStream_t stream) {
     if (st != TOPKV_OK) return st;
   }
   if (!handled) {
-    const dim3 grid((unsigned)slots);
+    const int64_t page_bytes = (int64_t)kp.P * F * rs.row_bytes;
+    kp.ppc = (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(kMaxPagesPerCta, kp.maxp),
+                                                        kSpanTargetBytes / page_bytes));
+    kp.spr = (kp.maxp + kp.ppc - 1) / kp.ppc;
+    const dim3 grid((unsigned)((int64_t)kp.R * kp.spr));
     // 32-byte vectors when every address the kernel can form is 32-byte aligned
     const bool wide = ((reinterpret_cast<uintptr_t>(kp.pool) | reinterpret_cast<uintptr_t>(kp.wire) |
                         (uintptr_t)kp.S_page | (uintptr_t)kp.S_kv | (uintptr_t)kp.S_tok |
@@ -627,6 +688,13 @@ int topkv_build_plan(const topkv_batch* batch, int64_t* d_cu_seq_lens, topkv_str
 }
 
 int topkv_last_cuda_error(void) { return g_last_cuda_error; }
+
+int topkv_reset_device_error_flags(void) {
+  const int zero = 0;
+  const cudaError_t e = cudaMemcpyToSymbol(g_device_error_flags, &zero, sizeof(int));
+  if (e != cudaSuccess) return cuda_fail(e);
+  return TOPKV_OK;
+}
 
 int topkv_device_error_flags(void) {
   int flags = 0;

@@ -21,9 +21,6 @@ constexpr int kBulkMaxStages = 8;
 constexpr int kBulkMaxR = TOPKV_MAX_INLINE_R;
 constexpr uint32_t kWaitPollLimit = 1u << 22;  // bounded mbarrier wait (each poll may suspend)
 
-// Set when a bounded wait gave up. Read back by topkv_device_error_flags().
-__device__ int g_device_error_flags = 0;
-
 struct BulkParams {
   KParams k;
   int tpc;          // tokens per work item
@@ -97,7 +94,12 @@ __global__ void __launch_bounds__(kBulkThreads, 1) topkv_bulk_kernel(const BulkP
 
   // ---- per-CTA plan: token and page prefix sums in shared memory (R <= kBulkMaxR) ----------
   for (int q = threadIdx.x; q < p.R; q += kBulkThreads) {
-    const int s = p.sl[q];
+    int s = p.sl[q];
+    const int64_t row_tokens = (int64_t)p.maxp * p.P;  // what one block-table row can describe
+    if (s < 0 || s > row_tokens) {
+      raise_error(kErrTable);
+      s = s < 0 ? 0 : (int)row_tokens;
+    }
     s_cu[q + 1] = s;
     s_pc[q + 1] = (s + p.P - 1) / p.P;
   }
@@ -132,6 +134,12 @@ __global__ void __launch_bounds__(kBulkThreads, 1) topkv_bulk_kernel(const BulkP
   __syncthreads();
 
   const int64_t T = (p.T >= 0) ? p.T : (int64_t)s_cu[p.R];
+  if (T < (int64_t)s_cu[p.R] ||
+      T * F * p.U * ((int64_t)p.unit_chunks * 16) > p.wire_limit) {  // uniform over the grid
+    if (threadIdx.x == 0) raise_error(kErrWire);
+    pdl_epilogue(p.overlap);
+    return;
+  }
   const int64_t unit_bytes = (int64_t)p.unit_chunks * 16;
   const int64_t total_items = (int64_t)s_pc[p.R] * bp.cpp;
   const int64_t gw = (int64_t)blockIdx.x * kBulkWarps + warp;
@@ -158,7 +166,12 @@ __global__ void __launch_bounds__(kBulkThreads, 1) topkv_bulk_kernel(const BulkP
       d.t0 = k * bp.tpc;
       d.nt = min(min(bp.tpc, p.P - d.t0), s_r - first);
       d.n_first = (int64_t)s_cu[r] + first;
-      d.pool_page = p.pool + (int64_t)p.bt[(int64_t)r * p.maxp + j] * p.S_page;
+      const int64_t page = p.bt[(int64_t)r * p.maxp + j];
+      if (page < 0 || page >= p.num_pages) {
+        raise_error(kErrTable);
+        continue;
+      }
+      d.pool_page = p.pool + page * p.S_page;
       return true;
     }
     return false;
@@ -263,7 +276,7 @@ __global__ void __launch_bounds__(kBulkThreads, 1) topkv_bulk_kernel(const BulkP
       ++issued;
     }
   }
-  if (failed && lane == 0) atomicOr(&g_device_error_flags, 1);
+  if (failed && lane == 0) raise_error(kErrWait);
   bulk_wait_all();
   pdl_epilogue(p.overlap);
 }

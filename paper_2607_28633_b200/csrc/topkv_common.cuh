@@ -26,8 +26,22 @@ struct KParams {
   int U;                  // units per (token, plane)
   int unit_chunks;        // VEC-byte chunks per unit
   int planar;             // wire order
+  int ppc, spr;           // vectorised family: page columns per CTA, CTAs per request
+  int64_t num_pages;      // pages per pool slab: every page id is checked against it
+  int64_t wire_limit;     // bytes that may be touched behind `wire` (this layer's slab)
   int overlap;            // 1: caller declared this launch independent of the kernels before it
 };
+
+// Error bits raised by kernels (never a trap): read back with topkv_device_error_flags().
+//   1  a bounded wait inside a kernel ran out
+//   2  a table entry was unusable (page id outside the pool, or a length longer than its
+//      block-table row): the affected pages were skipped
+//   4  the lengths found on the device do not fit the wire slab: the affected work was skipped
+__device__ int g_device_error_flags = 0;
+constexpr int kErrWait = 1, kErrTable = 2, kErrWire = 4;
+__device__ __forceinline__ void raise_error(int bit) {
+  if ((*(volatile int*)&g_device_error_flags & bit) == 0) atomicOr(&g_device_error_flags, bit);
+}
 
 // Programmatic dependent launch. Every copy kernel is launched with programmatic stream
 // serialisation, so its CTAs may become resident while the previous kernel of the stream

@@ -42,6 +42,7 @@ class DeviceWorkload:
         if key not in self._overlap_batches:
             b = tk.topkv_batch()
             ctypes.memmove(ctypes.byref(b), ctypes.byref(batch), ctypes.sizeof(b))
+            b._keepalive = getattr(batch, "_keepalive", None)
             b.flags = tk.TOPKV_FLAG_OVERLAP_PREVIOUS
             self._overlap_batches[key] = b
         return self._overlap_batches[key]

@@ -27,6 +27,7 @@ def dev():
 def variant(request, dev):
     """Every test runs once per kernel family (vectorised load/store, bulk-async ring)."""
     prev = tk.topkv_set_kernel_variant(request.param)
+    tk.check(tk.topkv_reset_device_error_flags())
     yield request.param
     tk.topkv_set_kernel_variant(prev)
     assert tk.topkv_device_error_flags() == 0
@@ -211,6 +212,101 @@ def test_many_short_requests_inline_and_planned(dev):
     # without a plan a batch beyond the inline limit is refused, nothing is launched
     b = tk.make_batch(d_bt, d_sl, -1, None)
     assert tk.topkv_pack_layer(0, src, lo, b, wire, wire.numel()) == tk.TOPKV_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("P,H,D", [(1, 1, 8), (2, 1, 64), (4, 2, 128), (16, 1, 128)])
+def test_small_pages_many_per_cta(dev, P, H, D):
+    """Pages far smaller than a CTA's span: long block-table rows are cut into several spans
+    of up to 64 pages, with ragged ends in the middle of a span and of a page."""
+    rng = np.random.default_rng(P * 1000 + D)
+    R = 5
+    sl = np.array([300 * P + 1, 0, 64 * P, 129 * P - 1, 7], dtype=np.int32)
+    pages = (sl + P - 1) // P
+    maxp = int(pages.max()) + 2
+    npages = int(pages.sum()) + 9
+    for order in (0, 1):
+        for F in (1, 2):
+            g = Geom(L=2, F=F, h_kv=H, d_h=D, b_p=2, P=P, num_pages=npages, wire_order=order)
+            T = int(sl.sum())
+            g.W_layer = g.wire_layer_bytes(T)
+            bt_s = np.full((R, maxp), -1, dtype=np.int32)
+            bt_d = np.full((R, maxp), -1, dtype=np.int32)
+            ps, pd, pos = rng.permutation(npages), rng.permutation(npages), 0
+            for r in range(R):
+                bt_s[r, :pages[r]] = ps[pos:pos + pages[r]]
+                bt_d[r, :pages[r]] = pd[pos:pos + pages[r]]
+                pos += pages[r]
+            lo = _layout_from_geom(g)
+            src_h = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
+            dst_h = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
+            src, dst = torch.from_numpy(src_h).to(dev), torch.from_numpy(dst_h).to(dev)
+            wire = torch.zeros(2 * g.W_layer, dtype=torch.uint8, device=dev)
+            d_sl = torch.from_numpy(sl).to(dev)
+            d_bs, d_bd = torch.from_numpy(bt_s).to(dev), torch.from_numpy(bt_d).to(dev)
+            bs = tk.make_batch(d_bs, d_sl, T)
+            bd = tk.make_batch(d_bd, d_sl, T)
+            want_wire = np.zeros(2 * g.W_layer, dtype=np.uint8)
+            for layer in range(2):
+                tk.check(tk.topkv_pack_layer(layer, src, lo, bs, wire, wire.numel()))
+                tk.check(tk.topkv_unpack_layer(layer, dst, lo, bd, wire, wire.numel()))
+                oracle.pack(g, layer, src_h, bt_s, sl, wire=want_wire, impl="rows")
+                oracle.unpack(g, layer, dst_h, bt_d, sl, want_wire, impl="rows")
+            torch.cuda.synchronize()
+            assert np.array_equal(wire.cpu().numpy(), want_wire), (order, F)
+            assert np.array_equal(dst.cpu().numpy(), dst_h), (order, F)
+
+
+def test_unusable_tables_are_skipped_not_followed(dev):
+    """Device-side checks: a page id outside the pool, a length longer than its table row and
+    lengths that overflow the wire slab raise status bits; the affected work is skipped, the
+    rest is copied, and nothing outside the buffers is touched (guard bands, untouched pool)."""
+    rng = np.random.default_rng(77)
+    g = Geom(L=1, F=2, h_kv=2, d_h=64, b_p=2, P=16, num_pages=40)
+    sl = np.array([40, 16, 33], dtype=np.int32)
+    bt = np.array([[3, 9, 12, -1], [7, -1, -1, -1], [1, 2, 5, -1]], dtype=np.int32)
+    T = int(sl.sum())
+    lo = _layout_from_geom(g)
+    src_h = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
+    src = torch.from_numpy(src_h).to(dev)
+    guard = 4096
+    n = g.wire_layer_bytes(T)
+
+    def run(bt_dev, sl_dev, total, cap):
+        buf = torch.full((guard + n + guard,), 0xC3, dtype=torch.uint8, device=dev)
+        d_bt, d_sl = torch.from_numpy(bt_dev).to(dev), torch.from_numpy(sl_dev).to(dev)
+        b = tk.make_batch(d_bt, d_sl, total)
+        tk.check(tk.topkv_reset_device_error_flags())
+        tk.check(tk.topkv_pack_layer(0, src, lo, b, buf[guard:], cap))
+        flags = tk.topkv_device_error_flags()
+        out = buf.cpu().numpy()
+        assert (out[:guard] == 0xC3).all() and (out[guard + n:] == 0xC3).all()
+        return flags, out[guard:guard + n]
+
+    want = oracle.pack(g, 0, src_h, bt, sl)
+    flags, got = run(bt, sl, T, n)
+    assert flags == 0 and np.array_equal(got, want)
+    # (a) a page id outside the pool: that page's 16 tokens are skipped, all others copied
+    bad = bt.copy(); bad[0, 1] = 40
+    flags, got = run(bad, sl, T, n)
+    assert flags == 2
+    lo_b, hi_b = 16 * g.F * g.row_bytes, 32 * g.F * g.row_bytes     # tokens 16..31 of request 0
+    assert np.array_equal(got[:lo_b], want[:lo_b]) and np.array_equal(got[hi_b:], want[hi_b:])
+    assert (got[lo_b:hi_b] == 0xC3).all()
+    bad = bt.copy(); bad[2, 0] = -5
+    flags, _ = run(bad, sl, T, n)
+    assert flags == 2
+    # (b) a length longer than its block-table row (4 columns = 64 tokens)
+    long = sl.copy(); long[1] = 65
+    flags, _ = run(bt, long, T, n)
+    assert flags & 2
+    # (c) device lengths that need more wire than the slab has
+    more = sl.copy(); more[2] = 48
+    bt48 = bt.copy(); bt48[2, 2] = 5
+    flags, _ = run(bt48, more, T, n)
+    assert flags & 4
+    flags, _ = run(bt48, more, -1, n)                               # unknown T: capacity rules
+    assert flags & 4
+    tk.check(tk.topkv_reset_device_error_flags())
 
 
 # -------------------------------------------------------------------- benchmark shapes
