@@ -302,6 +302,27 @@ def bench_host_leg(w, stream, pinned, staging, steps, warmup, barrier, slots):
     return total, to_host, from_host
 
 
+def bench_repage(w, stream, steps):
+    """Direct pool -> pool re-paging of every layer (topkv_repage_layer); GB/s of read + write."""
+    import torch
+    from paper_2607_28633_b200 import binding as tk
+
+    def run():
+        for l in range(w.layers):
+            ov = l > 0
+            tk.check(tk.topkv_repage_layer(l, w.src_pool, w.layout, w._flagged(w.src_batch, ov),
+                                           w.dst_pool, w.layout, w._flagged(w.dst_batch, ov), stream))
+    run()
+    stream.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(steps):
+        run()
+    b.record(stream)
+    stream.synchronize()
+    return 2.0 * w.n_layer * w.layers * steps / (a.elapsed_time(b) * 1e-3) / 1e9
+
+
 def pinned_copy_baseline(dev, stream, nbytes, reps=5):
     """cudaMemcpyAsync of one slab between pinned host and device memory (torch copy_), GB/s."""
     import torch
@@ -511,6 +532,7 @@ def main():
     extra = {}
     if rank == 0 and world == 1:
         extra["device_copy_GBps_same_bytes"] = round(device_copy_baseline(dev, stream, n_layer), 1)
+        extra["repage_GBps"] = round(bench_repage(w, stream, max(1, min(args.steps, 5))), 1)
     batch = w.batch
     del w
     torch.cuda.empty_cache()

@@ -156,6 +156,23 @@ int topkv_unpack_layer_from_host(int layer, void* dst_pool, const topkv_layout* 
                                  int64_t host_bytes, void* d_staging,
                                  int64_t staging_capacity_bytes, topkv_stream_t stream);
 
+/* ---- direct re-paging (no wire slab) -------------------------------------------------------- */
+
+/* Moves layer `layer` of the batch from one paged pool straight into another paged pool with
+ * its own block table, page size and strides: the same bytes end up in `dst_pool` as after
+ * topkv_pack_layer followed by topkv_unpack_layer, at half the memory traffic and with no
+ * wire buffer. This is the same-GPU case of handing a cache over, e.g. when a worker changes
+ * role (§3.5) and the cache must move into the other role's pool.
+ * The two layouts must agree in kv_factor, num_kv_heads, head_dim and elem_bytes; everything
+ * else may differ. Lengths are read from src_batch->seq_lens (dst_batch->seq_lens must hold
+ * the same values); cu_seq_lens and total_tokens are not used. The launch overlaps the
+ * previous kernel only if BOTH batches carry TOPKV_FLAG_OVERLAP_PREVIOUS. Preconditions as for
+ * unpack: no two requests share a destination page; the pools do not overlap. */
+int topkv_repage_layer(int layer, const void* src_pool, const topkv_layout* src_layout,
+                       const topkv_batch* src_batch, void* dst_pool,
+                       const topkv_layout* dst_layout, const topkv_batch* dst_batch,
+                       topkv_stream_t stream);
+
 /* ---- allocation-free host leg -------------------------------------------------------------- */
 
 /* Size of the library's built-in staging slab (bytes). Every GPU that loads the library

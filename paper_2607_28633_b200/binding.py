@@ -37,7 +37,7 @@ EXPORTS = (
     "topkv_model_transfer_s", "topkv_model_t_eff_s", "topkv_model_hidden_fraction",
     "topkv_strerror", "topkv_version", "topkv_last_cuda_error", "topkv_kernel_launch_count",
     "topkv_set_kernel_variant", "topkv_pack_layer_to_host_noalloc", "topkv_device_error_flags",
-    "topkv_reset_device_error_flags",
+    "topkv_reset_device_error_flags", "topkv_repage_layer",
 )
 
 
@@ -87,6 +87,7 @@ def lib() -> ctypes.CDLL:
         L.topkv_unpack_layer_from_host.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64,
                                                    c_void_p, c_int64, c_void_p]
         L.topkv_build_plan.argtypes = [bp, c_void_p, c_void_p]
+        L.topkv_repage_layer.argtypes = [c_int, c_void_p, lp, bp, c_void_p, lp, bp, c_void_p]
         L.topkv_pack_layer_to_host_noalloc.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64,
                                                        c_void_p]
         L.topkv_validate_batch_host.argtypes = [lp, c_int32, c_int32, c_void_p, c_void_p, c_int]
@@ -207,6 +208,14 @@ def topkv_pack_layer_to_host_noalloc(layer, src_pool, layout, batch, h_pinned,
     return lib().topkv_pack_layer_to_host_noalloc(
         layer, _ptr(src_pool), ctypes.byref(layout), ctypes.byref(batch), _ptr(h_pinned),
         host_capacity_bytes, _stream(stream))
+
+
+def topkv_repage_layer(layer, src_pool, src_layout, src_batch, dst_pool, dst_layout, dst_batch,
+                       stream=None):
+    return lib().topkv_repage_layer(layer, _ptr(src_pool), ctypes.byref(src_layout),
+                                    ctypes.byref(src_batch), _ptr(dst_pool),
+                                    ctypes.byref(dst_layout), ctypes.byref(dst_batch),
+                                    _stream(stream))
 
 
 def topkv_build_plan(batch, d_cu_seq_lens, stream=None):

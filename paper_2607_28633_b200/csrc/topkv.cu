@@ -10,6 +10,7 @@
 
 #include "topkv_bulk.cuh"
 #include "topkv_common.cuh"
+#include "topkv_repage.cuh"
 
 #include <algorithm>
 #include <atomic>
@@ -671,6 +672,86 @@ int topkv_pack_layer_to_host_noalloc(int layer, const void* src_pool, const topk
     const cudaError_t e = cudaMemcpyAsync(host_slab, staging, (size_t)n_layer, cudaMemcpyDeviceToHost, s);
     if (e != cudaSuccess) return cuda_fail(e);
   }
+  return TOPKV_OK;
+}
+
+int topkv_repage_layer(int layer, const void* src_pool, const topkv_layout* src_layout,
+                       const topkv_batch* src_batch, void* dst_pool,
+                       const topkv_layout* dst_layout, const topkv_batch* dst_batch,
+                       topkv_stream_t stream) {
+  Resolved rs_s, rs_d;
+  int st = check_layout(src_layout, &rs_s);
+  if (st != TOPKV_OK) return st;
+  st = check_layout(dst_layout, &rs_d);
+  if (st != TOPKV_OK) return st;
+  st = check_batch(src_layout, src_batch);
+  if (st != TOPKV_OK) return st;
+  st = check_batch(dst_layout, dst_batch);
+  if (st != TOPKV_OK) return st;
+  const topkv_layout *ls = src_layout, *ld = dst_layout;
+  if (ls->kv_factor != ld->kv_factor || ls->num_kv_heads != ld->num_kv_heads ||
+      ls->head_dim != ld->head_dim || ls->elem_bytes != ld->elem_bytes)
+    return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  if (src_batch->num_requests != dst_batch->num_requests) return TOPKV_ERR_INVALID_ARG;
+  if (layer < 0 || (uint32_t)layer >= ls->num_layers || (uint32_t)layer >= ld->num_layers)
+    return TOPKV_ERR_LAYER_RANGE;
+  if (src_pool == nullptr || dst_pool == nullptr) return TOPKV_ERR_INVALID_ARG;
+  if (!mult16p(src_pool) || !mult16p(dst_pool)) return TOPKV_ERR_ALIGNMENT;
+  if (src_batch->num_requests == 0 || src_batch->max_pages_per_req == 0 ||
+      dst_batch->max_pages_per_req == 0)
+    return TOPKV_OK;
+  const int F = (int)ls->kv_factor;
+  const int64_t head_bytes = (int64_t)ls->head_dim * ls->elem_bytes;
+  const bool rows = rs_s.U == 1 && rs_d.U == 1;  // whole rows contiguous in both pools
+  RepageParams p;
+  p.src = const_cast<uint8_t*>(static_cast<const uint8_t*>(src_pool)) + (int64_t)layer * ls->pool_layer_stride;
+  p.dst = static_cast<uint8_t*>(dst_pool) + (int64_t)layer * ld->pool_layer_stride;
+  p.bt_s = src_batch->block_table;
+  p.bt_d = dst_batch->block_table;
+  p.sl = src_batch->seq_lens;
+  p.Ss_page = ls->pool_page_stride;
+  p.Ss_kv = F > 1 ? ls->pool_kv_stride : 0;
+  p.Ss_tok = ls->pool_token_stride;
+  p.Ss_unit = rows ? 0 : (rs_s.U == 1 ? head_bytes : ls->pool_head_stride);
+  p.Sd_page = ld->pool_page_stride;
+  p.Sd_kv = F > 1 ? ld->pool_kv_stride : 0;
+  p.Sd_tok = ld->pool_token_stride;
+  p.Sd_unit = rows ? 0 : (rs_d.U == 1 ? head_bytes : ld->pool_head_stride);
+  p.ns_pages = ls->num_pool_pages;
+  p.nd_pages = ld->num_pool_pages;
+  p.R = src_batch->num_requests;
+  p.maxp_s = src_batch->max_pages_per_req;
+  p.maxp_d = dst_batch->max_pages_per_req;
+  p.Ps = (int)ls->page_tokens;
+  p.Pd = (int)ld->page_tokens;
+  p.U = rows ? 1 : (int)ls->num_kv_heads;
+  const int64_t unit_bytes = rows ? rs_s.row_bytes : head_bytes;
+  const int64_t tok_bytes = (int64_t)F * rs_s.row_bytes;
+  const int pmin = std::min(p.Ps, p.Pd);
+  p.span_tokens = (int)std::max<int64_t>(
+      1, std::min<int64_t>(kSpanTargetBytes / tok_bytes, (int64_t)(kRepageMaxPages - 1) * pmin));
+  const int64_t row_tokens = std::min((int64_t)p.maxp_s * p.Ps, (int64_t)p.maxp_d * p.Pd);
+  p.spr = (int)((row_tokens + p.span_tokens - 1) / p.span_tokens);
+  if ((int64_t)p.R * p.spr > 0x7fffffffll) return TOPKV_ERR_INVALID_ARG;
+  p.overlap = ((src_batch->flags & dst_batch->flags) & TOPKV_FLAG_OVERLAP_PREVIOUS) ? 1 : 0;
+  const bool wide = ((reinterpret_cast<uintptr_t>(p.src) | reinterpret_cast<uintptr_t>(p.dst) |
+                      (uintptr_t)p.Ss_page | (uintptr_t)p.Ss_kv | (uintptr_t)p.Ss_tok |
+                      (uintptr_t)p.Ss_unit | (uintptr_t)p.Sd_page | (uintptr_t)p.Sd_kv |
+                      (uintptr_t)p.Sd_tok | (uintptr_t)p.Sd_unit | (uintptr_t)unit_bytes) & 31) == 0;
+  const dim3 grid((unsigned)((int64_t)p.R * p.spr)), block(kRepageThreads);
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  if (wide) {
+    p.unit_chunks = (int)(unit_bytes / 32);
+    if (F == 1) launch_pdl(topkv_repage_kernel<1, 32>, grid, block, 0, s, p);
+    else launch_pdl(topkv_repage_kernel<2, 32>, grid, block, 0, s, p);
+  } else {
+    p.unit_chunks = (int)(unit_bytes / 16);
+    if (F == 1) launch_pdl(topkv_repage_kernel<1, 16>, grid, block, 0, s, p);
+    else launch_pdl(topkv_repage_kernel<2, 16>, grid, block, 0, s, p);
+  }
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
   return TOPKV_OK;
 }
 

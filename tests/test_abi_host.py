@@ -132,6 +132,24 @@ def test_argument_validation_without_gpu():
     assert tk.topkv_set_kernel_variant(99) == tk.TOPKV_ERR_INVALID_ARG
 
 
+def test_repage_argument_validation_without_gpu():
+    lo_s, lo_d, b = _gqa(), _gqa(pages=128), _batch()
+    RP = tk.topkv_repage_layer
+    src, dst = 0x7000000, 0x9000000
+    assert RP(4, src, lo_s, b, dst, lo_d, b) == tk.TOPKV_ERR_LAYER_RANGE
+    assert RP(0, None, lo_s, b, dst, lo_d, b) == tk.TOPKV_ERR_INVALID_ARG
+    assert RP(0, src, lo_s, b, dst + 8, lo_d, b) == tk.TOPKV_ERR_ALIGNMENT
+    other = tk.make_layout(4, 2, 8, 64, 2, 16, 64)                      # head_dim differs
+    assert RP(0, src, lo_s, b, dst, other, b) == tk.TOPKV_ERR_UNSUPPORTED_LAYOUT
+    mla = tk.make_layout(4, 1, 1, 576, 2, 64, 64)
+    assert RP(0, src, lo_s, b, dst, mla, b) == tk.TOPKV_ERR_UNSUPPORTED_LAYOUT
+    assert RP(0, src, lo_s, b, dst, lo_d, _batch(R=5)) == tk.TOPKV_ERR_INVALID_ARG
+    p32 = tk.make_layout(4, 2, 8, 128, 2, 32, 64)                       # other page size: fine
+    import torch
+    if not torch.cuda.is_available():
+        assert RP(0, src, lo_s, b, dst, p32, _batch(maxp=8)) == tk.TOPKV_ERR_CUDA
+
+
 def test_empty_batches_launch_nothing():
     lo = _gqa(wire_layer_stride=0)
     before = tk.topkv_kernel_launch_count()

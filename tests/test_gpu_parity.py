@@ -397,6 +397,88 @@ def test_overlapped_launches_keep_results_and_order(dev):
     torch.cuda.empty_cache()
 
 
+# -------------------------------------------------------------------- direct re-paging
+
+def _repage_case(seed):
+    """Two pools with different page sizes and strides, the same requests."""
+    rng = np.random.default_rng(1000 + seed)
+    F = int(rng.integers(1, 3))
+    H = int(rng.choice([1, 2, 8]))
+    D = int(rng.choice([8, 64, 128]))
+    Ps, Pd = int(rng.choice([1, 3, 16, 64])), int(rng.choice([1, 4, 16, 32]))
+    R = int(rng.integers(1, 6))
+    sl = rng.integers(0, 5 * max(Ps, Pd) + 3, size=R).astype(np.int32)
+    if seed % 4 == 0:
+        sl[rng.integers(0, R)] = 0
+    geoms, tables = [], []
+    for P, style in ((Ps, seed % 3), (Pd, (seed // 3) % 3)):
+        pages = (sl + P - 1) // P
+        npages = int(pages.sum()) + 3
+        g = Geom(L=2, F=F, h_kv=H, d_h=D, b_p=2, P=P, num_pages=npages)
+        if style == 1:      # head-major inside the page
+            g.S_tok = D * 2
+            g.S_head = P * g.S_tok
+            g.S_kv = H * g.S_head
+            g.S_page = F * g.S_kv
+            g.S_layer = npages * g.S_page
+        elif style == 2:    # padded tokens, plane-major pool
+            g.S_tok = H * D * 2 + 16
+            g.S_page = P * g.S_tok
+            g.S_kv = npages * g.S_page
+            g.S_layer = F * g.S_kv + 48
+        maxp = max(int(pages.max()), 1) + int(rng.integers(0, 2))
+        bt = np.full((R, maxp), -1, dtype=np.int32)
+        perm, pos = rng.permutation(npages), 0
+        for r in range(R):
+            bt[r, :pages[r]] = perm[pos:pos + pages[r]]
+            pos += pages[r]
+        geoms.append(g)
+        tables.append(bt)
+    return geoms, tables, sl, rng
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_repage_equals_unpack_of_pack(dev, seed, variant):
+    if variant == 1:
+        pytest.skip("re-paging has one kernel family")
+    (gs, gd), (bt_s, bt_d), sl, rng = _repage_case(seed)
+    T = int(sl.sum())
+    src_h = rng.integers(0, 256, gs.pool_bytes(), dtype=np.uint8)
+    dst_h = rng.integers(0, 256, gd.pool_bytes(), dtype=np.uint8)
+    src, dst = torch.from_numpy(src_h).to(dev), torch.from_numpy(dst_h).to(dev)
+    d_sl = torch.from_numpy(sl).to(dev)
+    d_bs, d_bd = torch.from_numpy(bt_s).to(dev), torch.from_numpy(bt_d).to(dev)
+    los, lod = _layout_from_geom(gs), _layout_from_geom(gd)
+    for layer in range(2):
+        tk.check(tk.topkv_repage_layer(layer, src, los, tk.make_batch(d_bs, d_sl, T), dst, lod,
+                                       tk.make_batch(d_bd, d_sl, T)))
+        wire = oracle.pack(gs, layer, src_h, bt_s, sl)
+        gd.W_layer = gs.W_layer
+        oracle.unpack(gd, layer, dst_h, bt_d, sl, wire)
+    torch.cuda.synchronize()
+    assert np.array_equal(dst.cpu().numpy(), dst_h)
+    assert np.array_equal(src.cpu().numpy(), src_h)
+
+
+def test_repage_bench_shape(dev, variant):
+    if variant == 1:
+        pytest.skip("re-paging has one kernel family")
+    w = harness.setup(wl.CFG2, dev, layers=2)
+    b, s = w.batch, wl.CFG2
+    g = _geom(s, b.num_pool_pages, 1, 0, 0)
+    for layer in range(2):
+        dst_h = harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, layer)
+        src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, layer)
+        tk.check(tk.topkv_repage_layer(layer, w.src_pool, w.layout, w.src_batch, w.dst_pool,
+                                       w.layout, w.dst_batch))
+        torch.cuda.synchronize()
+        wire = oracle.pack(g, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=8)
+        oracle.unpack(g, 0, dst_h, b.dst_block_table, b.seq_lens, wire, impl="rows", threads=8)
+        assert np.array_equal(harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, layer), dst_h)
+    del w
+    torch.cuda.empty_cache()
+
+
 # -------------------------------------------------------------------- host leg
 
 @pytest.mark.parametrize("staged", [True, False])
