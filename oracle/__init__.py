@@ -41,7 +41,7 @@ def build(force: bool = False) -> str:
 class _Geom(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int64) for n in (
         "L", "F", "h_kv", "d_h", "b_p", "P", "S_layer", "S_page", "S_kv", "S_tok", "S_head",
-        "W_layer", "wire_order")]
+        "W_layer", "wire_order", "window")]
 
 
 _lib = None
@@ -54,6 +54,8 @@ def _load():
         i64, f64, vp = ctypes.c_int64, ctypes.c_double, ctypes.c_void_p
         lib.oracle_kv_bytes.restype = i64
         lib.oracle_kv_bytes.argtypes = [i64] * 6
+        lib.oracle_kv_bytes_layered.restype = i64
+        lib.oracle_kv_bytes_layered.argtypes = [i64] * 6 + [vp, vp]
         lib.oracle_transfer_s.restype = f64
         lib.oracle_transfer_s.argtypes = [f64] * 3
         lib.oracle_t_eff.restype = f64
@@ -90,6 +92,7 @@ class Geom:
     S_tok: int = 0
     S_head: int = 0
     W_layer: int = 0
+    window: int = 0          # 0: every token; W > 0: the layer keeps only the last min(s, W)
 
     def __post_init__(self):
         if self.S_page == 0:  # default pool: pool[l][page][c][t][h][d], dim contiguous
@@ -113,12 +116,28 @@ class Geom:
     def _c(self) -> _Geom:
         return _Geom(self.L, self.F, self.h_kv, self.d_h, self.b_p, self.P, self.S_layer,
                      self.S_page, self.S_kv, self.S_tok, self.S_head, self.W_layer,
-                     self.wire_order)
+                     self.wire_order, self.window)
+
+    def kept_tokens(self, sl) -> int:
+        """Tokens of a batch that this layer keeps: sum of min(s, window) (all, if no window)."""
+        sl = np.asarray(sl, dtype=np.int64)
+        return int(sl.sum() if self.window <= 0 else np.minimum(sl, self.window).sum())
 
 
 def kv_bytes(L: int, h_kv: int, d_h: int, s: int, b_p: int = 2, F: int = 2) -> int:
     """Eq. 1 (F = 2), or the MLA form without the K/V factor (F = 1, §5.3)."""
     return int(_load().oracle_kv_bytes(F, L, h_kv, d_h, s, b_p))
+
+
+def kv_bytes_layered(h_kv: int, d_h: int, s: int, kinds, b_p: int = 2, F: int = 2) -> int:
+    """Eq. 1 extended per layer kind (§2.2). ``kinds`` is one entry per layer: ("full",),
+    ("window", W) or ("state", nbytes)."""
+    code = {"full": 0, "window": 1, "state": 2}
+    k = np.array([code[x[0]] for x in kinds], dtype=np.int64)
+    prm = np.array([x[1] if len(x) > 1 else 0 for x in kinds], dtype=np.int64)
+    lib = _load()
+    return int(lib.oracle_kv_bytes_layered(F, h_kv, d_h, s, b_p, len(kinds), k.ctypes.data,
+                                           prm.ctypes.data))
 
 
 def transfer_s(S_bytes: float, B_bytes_per_s: float, L_m_s: float = 0.0) -> float:
@@ -152,15 +171,16 @@ def _tables(bt: np.ndarray, sl: np.ndarray):
 
 def _check_extent(g: Geom, layer: int, pool: np.ndarray, bt, sl, wire: np.ndarray):
     """Guards the C loops: every offset they will form must lie inside the arrays."""
-    T = int(sl.sum())
+    T = g.kept_tokens(sl)
     need_wire = layer * g.W_layer + g.wire_layer_bytes(T)
     assert wire.size >= need_wire, (wire.size, need_wire)
     assert 0 <= layer < g.L
     for r in range(sl.shape[0]):
         n = -(-int(sl[r]) // g.P)
         assert n <= bt.shape[1]
+        lo = 0 if g.window <= 0 or sl[r] <= g.window else (int(sl[r]) - g.window) // g.P
         if n:
-            used = bt[r, :n]
+            used = bt[r, lo:n]              # pages before the window are never touched
             assert used.min() >= 0
             last = (layer * g.S_layer + int(used.max()) * g.S_page + (g.F - 1) * g.S_kv
                     + (g.P - 1) * g.S_tok + (g.h_kv - 1) * g.S_head + g.d_h * g.b_p)
@@ -172,7 +192,7 @@ def pack(g: Geom, layer: int, pool: np.ndarray, bt: np.ndarray, sl: np.ndarray,
     """wire <- pool through the block table. ``pool`` is the uint8 view from layer 0's base,
     ``wire`` the uint8 view from layer 0's slab (allocated, zero-filled, if None)."""
     bt, sl = _tables(bt, sl)
-    T = int(sl.sum())
+    T = g.kept_tokens(sl)
     if wire is None:
         wire = np.zeros(layer * g.W_layer + g.wire_layer_bytes(T), dtype=np.uint8)
     _u8(pool, False), _u8(wire, True)

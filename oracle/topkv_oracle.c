@@ -16,6 +16,21 @@ int64_t oracle_kv_bytes(int64_t F, int64_t L, int64_t h_kv, int64_t d_h, int64_t
   return F * L * h_kv * d_h * s * b_p; /* Eq. 1 with the leading 2 generalised to F (§5.3) */
 }
 
+int64_t oracle_kv_bytes_layered(int64_t F, int64_t h_kv, int64_t d_h, int64_t s, int64_t b_p,
+                                int64_t L, const int64_t* kind, const int64_t* param) {
+  int64_t total = 0;
+  for (int64_t l = 0; l < L; ++l) {
+    if (kind[l] == 2) {
+      total += param[l]; /* fixed state, independent of s */
+    } else {
+      int64_t tokens = s;
+      if (kind[l] == 1 && param[l] < s) tokens = param[l]; /* capped at the window */
+      total += F * h_kv * d_h * tokens * b_p;
+    }
+  }
+  return total;
+}
+
 double oracle_transfer_s(double S_bytes, double B, double L_m) { return S_bytes / B + L_m; } /* Eq. 2 */
 
 double oracle_t_eff(double T_last, double T_xfer, double T_rem) { /* Eq. 3 */
@@ -44,45 +59,52 @@ static int64_t woff(const oracle_geom* g, int64_t l, int64_t n, int64_t T, int64
   return l * g->W_layer + row * row_bytes + (h * g->d_h + d) * g->b_p + b;
 }
 
-static int64_t total_tokens(int64_t R, const int32_t* sl) {
+/* First token a layer keeps for a sequence of s tokens: 0, or s - window for a windowed layer. */
+static int64_t first_kept(const oracle_geom* g, int64_t s) {
+  return (g->window > 0 && s > g->window) ? s - g->window : 0;
+}
+
+static int64_t total_tokens(const oracle_geom* g, int64_t R, const int32_t* sl) {
   int64_t T = 0;
-  for (int64_t r = 0; r < R; ++r) T += sl[r];
+  for (int64_t r = 0; r < R; ++r) T += sl[r] - first_kept(g, sl[r]);
   return T;
 }
 
 void oracle_pack_ref(const oracle_geom* g, int64_t layer, const uint8_t* pool, int64_t R,
                      int64_t maxp, const int32_t* bt, const int32_t* sl, uint8_t* wire) {
-  int64_t T = total_tokens(R, sl);
+  int64_t T = total_tokens(g, R, sl);
   int64_t cu = 0;
   for (int64_t r = 0; r < R; ++r) {
-    for (int64_t i = 0; i < sl[r]; ++i) {
+    int64_t i0 = first_kept(g, sl[r]);
+    for (int64_t i = i0; i < sl[r]; ++i) {
       int64_t page = bt[r * maxp + i / g->P];
       int64_t t = i % g->P;
       for (int64_t c = 0; c < g->F; ++c)
         for (int64_t h = 0; h < g->h_kv; ++h)
           for (int64_t d = 0; d < g->d_h; ++d)
             for (int64_t b = 0; b < g->b_p; ++b)
-              wire[woff(g, layer, cu + i, T, c, h, d, b)] = pool[poff(g, layer, page, c, t, h, d, b)];
+              wire[woff(g, layer, cu + i - i0, T, c, h, d, b)] = pool[poff(g, layer, page, c, t, h, d, b)];
     }
-    cu += sl[r];
+    cu += sl[r] - i0;
   }
 }
 
 void oracle_unpack_ref(const oracle_geom* g, int64_t layer, uint8_t* pool, int64_t R,
                        int64_t maxp, const int32_t* bt, const int32_t* sl, const uint8_t* wire) {
-  int64_t T = total_tokens(R, sl);
+  int64_t T = total_tokens(g, R, sl);
   int64_t cu = 0;
   for (int64_t r = 0; r < R; ++r) {
-    for (int64_t i = 0; i < sl[r]; ++i) {
+    int64_t i0 = first_kept(g, sl[r]);
+    for (int64_t i = i0; i < sl[r]; ++i) {
       int64_t page = bt[r * maxp + i / g->P];
       int64_t t = i % g->P;
       for (int64_t c = 0; c < g->F; ++c)
         for (int64_t h = 0; h < g->h_kv; ++h)
           for (int64_t d = 0; d < g->d_h; ++d)
             for (int64_t b = 0; b < g->b_p; ++b)
-              pool[poff(g, layer, page, c, t, h, d, b)] = wire[woff(g, layer, cu + i, T, c, h, d, b)];
+              pool[poff(g, layer, page, c, t, h, d, b)] = wire[woff(g, layer, cu + i - i0, T, c, h, d, b)];
     }
-    cu += sl[r];
+    cu += sl[r] - i0;
   }
 }
 
@@ -104,13 +126,14 @@ static void* run_job(void* arg) {
   const oracle_geom* g = j->g;
   size_t head_bytes = (size_t)(g->d_h * g->b_p);
   for (int64_t r = j->r_begin; r < j->r_end; ++r) {
-    for (int64_t i = 0; i < j->sl[r]; ++i) {
+    int64_t i0 = first_kept(g, j->sl[r]);
+    for (int64_t i = i0; i < j->sl[r]; ++i) {
       int64_t page = j->bt[r * j->maxp + i / g->P];
       int64_t t = i % g->P;
       for (int64_t c = 0; c < g->F; ++c)
         for (int64_t h = 0; h < g->h_kv; ++h) {
           uint8_t* p = j->pool + poff(g, j->layer, page, c, t, h, 0, 0);
-          uint8_t* w = j->wire + woff(g, j->layer, j->cu[r] + i, j->T, c, h, 0, 0);
+          uint8_t* w = j->wire + woff(g, j->layer, j->cu[r] + i - i0, j->T, c, h, 0, 0);
           if (j->pack) memcpy(w, p, head_bytes);
           else memcpy(p, w, head_bytes);
         }
@@ -126,7 +149,7 @@ static void run_rows(const oracle_geom* g, int64_t layer, uint8_t* pool, int64_t
   if (R < threads) threads = R > 0 ? (int)R : 1;
   int64_t* cu = (int64_t*)malloc(sizeof(int64_t) * (size_t)(R + 1));
   cu[0] = 0;
-  for (int64_t r = 0; r < R; ++r) cu[r + 1] = cu[r] + sl[r];
+  for (int64_t r = 0; r < R; ++r) cu[r + 1] = cu[r] + sl[r] - first_kept(g, sl[r]);
   job jobs[256];
   pthread_t tid[256];
   for (int k = 0; k < threads; ++k) {

@@ -21,10 +21,18 @@ typedef struct oracle_geom {
   int64_t S_layer, S_page, S_kv, S_tok, S_head; /* pool strides, bytes            */
   int64_t W_layer;              /* bytes between wire slabs of consecutive layers */
   int64_t wire_order;           /* ORACLE_WIRE_*                                  */
+  int64_t window;               /* 0: all tokens; W > 0: a windowed layer keeps   */
+                                /* (and sends) only the last min(s, W) tokens     */
 } oracle_geom;
 
 /* Eq. 1 (F = 2) and its MLA form (F = 1, §5.3): F * L * h_kv * d_h * s * b_p. */
 int64_t oracle_kv_bytes(int64_t F, int64_t L, int64_t h_kv, int64_t d_h, int64_t s, int64_t b_p);
+
+/* Eq. 1 extended per layer kind (§2.2): a full layer counts s tokens, a windowed layer
+ * min(s, window) tokens, a constant-state layer a fixed number of bytes. kind[l] is
+ * 0 = full, 1 = windowed (param = window in tokens), 2 = constant state (param = bytes). */
+int64_t oracle_kv_bytes_layered(int64_t F, int64_t h_kv, int64_t d_h, int64_t s, int64_t b_p,
+                                int64_t L, const int64_t* kind, const int64_t* param);
 
 /* Eq. 2. */
 double oracle_transfer_s(double S_bytes, double B_bytes_per_s, double L_m_s);

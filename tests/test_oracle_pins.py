@@ -370,3 +370,86 @@ def test_rows_impl_threads_agree_with_ref_on_cfg1():
         oracle.unpack(g, 1, dst_a, b.dst_block_table, b.seq_lens, ref)
         oracle.unpack(g, 1, dst_b, b.dst_block_table, b.seq_lens, ref, impl="rows", threads=3)
         assert np.array_equal(dst_a, dst_b)
+
+
+# ---------------------------------------------------------------- per-layer kinds (§2.2)
+
+def test_layered_sizes(golden):
+    g = golden("paper_values.txt")
+    s = int(g["seq_len"])
+    # all layers full == Eq. 1; a window at least as long as the sequence changes nothing
+    assert oracle.kv_bytes_layered(8, 128, s, [("full",)] * 80) == oracle.kv_bytes(80, 8, 128, s)
+    assert oracle.kv_bytes_layered(8, 128, s, [("window", s)] * 80) == oracle.kv_bytes(80, 8, 128, s)
+    assert oracle.kv_bytes_layered(8, 128, s, [("window", 2 * s)] * 3) == oracle.kv_bytes(3, 8, 128, s)
+    # a capped layer counts its window, a state layer a constant
+    assert oracle.kv_bytes_layered(8, 128, s, [("window", 128)]) == oracle.kv_bytes(1, 8, 128, 128)
+    assert oracle.kv_bytes_layered(8, 128, s, [("state", 12345), ("state", 5)]) == 12350
+    assert oracle.kv_bytes_layered(8, 128, 10 * s, [("state", 12345)]) == 12345
+    # Kimi K2 class: the DeepSeek-V3 latent on 61 layers
+    kimi = oracle.kv_bytes_layered(1, 576, s, [("full",)] * 61, F=1)
+    assert round(kimi / 2**30, 2) == float(g["layered.kimi_k2.gb"])
+    # gpt-oss-120b: the paper gives 36 layers, 18 of them window-capped, 0.15 GB. Heads, head
+    # dim and window are the model's published configuration (8 KV heads of 64, window 128).
+    L, nw = int(g["layered.gpt_oss_120b.layers"]), int(g["layered.gpt_oss_120b.windowed"])
+    kinds = [("window", 128) if l % 2 == 0 else ("full",) for l in range(L)]
+    assert sum(k[0] == "window" for k in kinds) == nw
+    oss = oracle.kv_bytes_layered(8, 64, s, kinds)
+    assert oss == 18 * 2 * 8 * 64 * 2 * (4096 + 128)
+    assert round(oss / 2**30, 2) == float(g["layered.gpt_oss_120b.gb"])     # binary GB, as Table 1
+    # Qwen3.5-397B: 60 layers, 45 carry constant state (size not given), 15 full layers of
+    # 2 KV heads x 256 dims (the published configuration of that family)
+    L, ns = int(g["layered.qwen35_397b.layers"]), int(g["layered.qwen35_397b.state_layers"])
+    kinds = [("full",) if l % 4 == 3 else ("state", 0) for l in range(L)]
+    assert sum(k[0] == "state" for k in kinds) == ns
+    assert round(oracle.kv_bytes_layered(2, 256, s, kinds) / 2**30, 2) == float(g["layered.qwen35_397b.gb"])
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_windowed_pack_is_a_slice_of_the_full_pack(seed):
+    g, pool, bt, sl = _random_case(300 + seed, 2, 2, 8, 4, strided=seed % 2 == 1)
+    g.W_layer = 0
+    cu = np.concatenate([[0], np.cumsum(sl.astype(np.int64))])
+    T = int(cu[-1])
+    for W in (1, 3, 4, 7, 100):
+        for order in (WIRE_TOKEN_KV, WIRE_PLANAR):
+            g.wire_order, g.window = order, 0
+            full = oracle.pack(g, 1, pool, bt, sl)
+            g.window = W
+            for impl in ("ref", "rows"):
+                got = oracle.pack(g, 1, pool, bt, sl, impl=impl, threads=2)
+                rb = g.row_bytes
+                if order == WIRE_TOKEN_KV:
+                    rows = full.reshape(T, g.F * rb)
+                    want = np.concatenate([rows[cu[r] + max(0, sl[r] - W):cu[r + 1]]
+                                           for r in range(len(sl))]).reshape(-1)
+                else:
+                    planes = full.reshape(g.F, T, rb)
+                    want = np.concatenate(
+                        [np.concatenate([planes[c, cu[r] + max(0, sl[r] - W):cu[r + 1]]
+                                         for r in range(len(sl))]).reshape(-1) for c in range(g.F)])
+                assert got.size == g.wire_layer_bytes(g.kept_tokens(sl))
+                assert np.array_equal(got, want), (W, order, impl)
+    g.window = 0
+
+
+def test_windowed_layer_never_touches_pages_before_the_window():
+    g = Geom(L=1, F=2, h_kv=1, d_h=8, b_p=2, P=4, num_pages=12, window=6)
+    rng = np.random.default_rng(4)
+    pool = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
+    sl = np.array([14, 5, 9], dtype=np.int32)        # windows start at tokens 8, 0, 3
+    bt = np.array([[-1, -1, 3, 7], [9, 1, -1, -1], [4, 2, 0, -1]], dtype=np.int32)
+    wire = oracle.pack(g, 0, pool, bt, sl)
+    assert wire.size == (6 + 5 + 6) * 32
+    # request 0 starts at token 8 = page column 2, token 0 of page 3
+    assert np.array_equal(wire[:16], pool[3 * g.S_page:3 * g.S_page + 16])
+    # request 2 starts at token 3 = last token of page 4: K row then V row
+    o = (6 + 5) * 32
+    assert np.array_equal(wire[o:o + 16], pool[4 * g.S_page + 3 * 16:4 * g.S_page + 4 * 16])
+    assert np.array_equal(wire[o + 16:o + 32],
+                          pool[4 * g.S_page + g.S_kv + 3 * 16:4 * g.S_page + g.S_kv + 4 * 16])
+    dst = np.full(g.pool_bytes(), 0x77, dtype=np.uint8)
+    oracle.unpack(g, 0, dst, bt, sl, wire)
+    assert np.array_equal(oracle.pack(g, 0, dst, bt, sl), wire)
+    assert (dst != 0x77).sum() <= wire.size
+    # tokens 0..2 of request 2 (page 4, first three rows of each plane) stay untouched
+    assert (dst[4 * g.S_page:4 * g.S_page + 48] == 0x77).all()
