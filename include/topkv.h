@@ -104,6 +104,12 @@ typedef struct topkv_batch {
                                  /* each CTA derives it (allowed for R <= TOPKV_MAX_INLINE_R)*/
   int64_t total_tokens;          /* T if the host knows it, else -1. When -1 the capacity   */
                                  /* checks are skipped and the caller guarantees them.      */
+  int32_t window_tokens;         /* 0 = every token. W > 0 = a windowed layer (§2.2): only  */
+                                 /* the last min(s_r, W) tokens of each request are kept,   */
+                                 /* so only they are packed / unpacked; T, cu_seq_lens and  */
+                                 /* N_layer then count min(s_r, W) per request, and table   */
+                                 /* columns before the window are ignored.                  */
+  int32_t reserved;              /* must be 0                                               */
 } topkv_batch;
 
 /* topkv_batch.flags. Every copy kernel is launched so that it may become resident while the
@@ -229,6 +235,18 @@ int64_t topkv_wire_layer_bytes(const topkv_layout* layout, int64_t total_tokens)
 
 /* Eq. 1 with the §5.3 MLA rule: F * L * H * D * seq_len * E bytes for one sequence. */
 int64_t topkv_kv_bytes(const topkv_layout* layout, int64_t seq_len);
+
+/* Eq. 1 extended per layer kind (§2.2): a full layer counts seq_len tokens, a windowed layer
+ * min(seq_len, window) tokens, a constant-state layer (linear attention) a fixed byte count. */
+enum { TOPKV_LAYER_FULL = 0, TOPKV_LAYER_WINDOW = 1, TOPKV_LAYER_STATE = 2 };
+typedef struct topkv_layer_spec {
+  uint32_t kind;     /* TOPKV_LAYER_*                                               */
+  uint32_t reserved; /* must be 0                                                   */
+  int64_t param;     /* WINDOW: window in tokens; STATE: bytes; FULL: ignored       */
+} topkv_layer_spec;
+/* specs: HOST array [layout->num_layers]. Returns bytes or a negative topkv_status. */
+int64_t topkv_kv_bytes_layered(const topkv_layout* layout, const topkv_layer_spec* specs,
+                               int64_t seq_len);
 
 /* ---- CPU-side analytic helpers (context only; no GPU work) ------------------------------- */
 

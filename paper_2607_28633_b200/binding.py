@@ -37,7 +37,7 @@ EXPORTS = (
     "topkv_model_transfer_s", "topkv_model_t_eff_s", "topkv_model_hidden_fraction",
     "topkv_strerror", "topkv_version", "topkv_last_cuda_error", "topkv_kernel_launch_count",
     "topkv_set_kernel_variant", "topkv_pack_layer_to_host_noalloc", "topkv_device_error_flags",
-    "topkv_reset_device_error_flags", "topkv_repage_layer",
+    "topkv_reset_device_error_flags", "topkv_repage_layer", "topkv_kv_bytes_layered",
 )
 
 
@@ -57,8 +57,16 @@ class topkv_batch(ctypes.Structure):
     _fields_ = [
         ("struct_size", c_uint32), ("num_requests", c_int32), ("max_pages_per_req", c_int32),
         ("flags", c_uint32), ("block_table", c_void_p), ("seq_lens", c_void_p),
-        ("cu_seq_lens", c_void_p), ("total_tokens", c_int64),
+        ("cu_seq_lens", c_void_p), ("total_tokens", c_int64), ("window_tokens", c_int32),
+        ("reserved", c_int32),
     ]
+
+
+class topkv_layer_spec(ctypes.Structure):
+    _fields_ = [("kind", c_uint32), ("reserved", c_uint32), ("param", c_int64)]
+
+
+TOPKV_LAYER_FULL, TOPKV_LAYER_WINDOW, TOPKV_LAYER_STATE = 0, 1, 2
 
 
 class TopkvError(RuntimeError):
@@ -96,6 +104,8 @@ def lib() -> ctypes.CDLL:
         L.topkv_wire_layer_bytes.restype = c_int64
         L.topkv_kv_bytes.argtypes = [lp, c_int64]
         L.topkv_kv_bytes.restype = c_int64
+        L.topkv_kv_bytes_layered.argtypes = [lp, c_void_p, c_int64]
+        L.topkv_kv_bytes_layered.restype = c_int64
         L.topkv_model_transfer_s.argtypes = [c_double] * 3
         L.topkv_model_transfer_s.restype = c_double
         L.topkv_model_t_eff_s.argtypes = [c_double] * 3
@@ -155,7 +165,7 @@ def make_layout(L: int, F: int, H: int, D: int, E: int, P: int, num_pool_pages: 
 
 
 def make_batch(block_table, seq_lens, total_tokens: int = -1, cu_seq_lens=None,
-               flags: int = 0) -> topkv_batch:
+               flags: int = 0, window_tokens: int = 0) -> topkv_batch:
     """block_table: device int32 [R][maxp]; seq_lens: device int32 [R]. The descriptor keeps a
     reference to the tensors it was built from."""
     b = topkv_batch()
@@ -167,6 +177,7 @@ def make_batch(block_table, seq_lens, total_tokens: int = -1, cu_seq_lens=None,
     b.cu_seq_lens = _ptr(cu_seq_lens)
     b.total_tokens = total_tokens
     b.flags = flags
+    b.window_tokens = window_tokens
     # The struct only holds addresses: keep the tensors alive with it, so that a temporary
     # passed here cannot be freed (and its memory reused) while the descriptor is in use.
     b._keepalive = (block_table, seq_lens, cu_seq_lens)
@@ -239,6 +250,17 @@ def topkv_wire_layer_bytes(layout, total_tokens):
 
 def topkv_kv_bytes(layout, seq_len):
     return lib().topkv_kv_bytes(ctypes.byref(layout), seq_len)
+
+
+def topkv_kv_bytes_layered(layout, specs, seq_len):
+    """specs: sequence of (kind, param) pairs, one per layer, or a ctypes array of
+    topkv_layer_spec."""
+    if not isinstance(specs, ctypes.Array):
+        arr = (topkv_layer_spec * len(specs))()
+        for i, (kind, param) in enumerate(specs):
+            arr[i].kind, arr[i].param = kind, param
+        specs = arr
+    return lib().topkv_kv_bytes_layered(ctypes.byref(layout), ctypes.addressof(specs), seq_len)
 
 
 def topkv_model_transfer_s(nbytes, bandwidth_bytes_per_s, setup_s=0.0):

@@ -67,12 +67,13 @@ struct Vec<32> {
 
 // Sum of sl[0..n) over the CTA, result broadcast to all threads. n <= TOPKV_MAX_INLINE_R.
 __device__ __forceinline__ int64_t block_prefix(const int32_t* __restrict__ sl, int n, int r_split,
-                                                int64_t* total_out) {
+                                                int window, int64_t* total_out) {
   // returns sum_{q < r_split} sl[q]; *total_out = sum_{q < n} sl[q]
   __shared__ int64_t s_part[2][kThreads / 32];
   int64_t below = 0, all = 0;
   for (int q = threadIdx.x; q < n; q += kThreads) {
     int64_t v = sl[q];
+    if (window > 0 && v > window) v = window;  // a windowed layer keeps min(s, W) tokens
     all += v;
     if (q < r_split) below += v;
   }
@@ -108,15 +109,20 @@ __device__ __forceinline__ void copy_span(const KParams& p) {
   const int r = slot / p.spr;
   const int j0 = (slot - r * p.spr) * p.ppc;
   const int s_r = p.sl[r];
-  const int first = j0 * p.P;
-  if (first >= s_r) return;
-  int v = min(p.ppc * p.P, s_r - first);  // valid tokens in this span
+  // first token this layer keeps: 0, or s_r - window for a windowed layer (§2.2)
+  const int b_r = (p.window > 0 && s_r > p.window) ? s_r - p.window : 0;
+  const int first = j0 * p.P;  // first token of the span's page columns
   const int tid = threadIdx.x;
+  int hi = min(first + p.ppc * p.P, s_r);
   if (s_r > p.maxp * p.P) {  // length longer than its block-table row: copy what the row holds
-    v = min(v, (p.maxp - j0) * p.P);
-    if (tid == 0) raise_error(kErrTable);
+    hi = min(hi, p.maxp * p.P);
+    if (tid == 0 && j0 == 0) raise_error(kErrTable);
   }
-  const int npages = (v + p.P - 1) / p.P;
+  const int lo = max(first, b_r);
+  if (lo >= hi) return;
+  const int v = hi - lo;       // kept tokens in this span
+  const int ts0 = lo - first;  // where they start inside the span
+  const int jlo = ts0 / p.P, jhi = (ts0 + v - 1) / p.P;  // page columns (relative) they touch
 
   int64_t cu_r, T = p.T;
   if (p.cu != nullptr) {
@@ -124,10 +130,10 @@ __device__ __forceinline__ void copy_span(const KParams& p) {
     if (p.planar && T < 0) T = p.cu[p.R];
   } else {
     int64_t total;
-    cu_r = block_prefix(p.sl, (p.planar && T < 0) ? p.R : r, r, &total);
+    cu_r = block_prefix(p.sl, (p.planar && T < 0) ? p.R : r, r, p.window, &total);
     if (p.planar && T < 0) T = total;
   }
-  if (tid < npages) {
+  if (tid >= jlo && tid <= jhi) {
     int pg = p.bt[(int64_t)r * p.maxp + j0 + tid];
     if (pg < 0 || pg >= p.num_pages) {  // unusable entry: the page is skipped, nothing is touched
       pg = -1;
@@ -136,7 +142,7 @@ __device__ __forceinline__ void copy_span(const KParams& p) {
     s_pages[tid] = pg;
   }
   __syncthreads();
-  const int64_t n0 = cu_r + first;  // global index of the span's first token
+  const int64_t n0 = cu_r + (lo - b_r);  // wire index of the span's first kept token
   const int64_t unit_bytes = (int64_t)p.unit_chunks * VEC;
   {  // the span must lie inside the wire slab, whatever lengths the device tables hold
     const int64_t row = unit_bytes * p.U;
@@ -151,16 +157,17 @@ __device__ __forceinline__ void copy_span(const KParams& p) {
 
   if (MERGED) {
     // per page, F runs of (valid tokens) * row bytes each (U == 1 here)
-    for (int jj = 0; jj < npages; ++jj) {
+    for (int jj = jlo; jj <= jhi; ++jj) {
       if (s_pages[jj] < 0) continue;
-      const int vj = min(p.P, v - jj * p.P);
-      const int n = vj * p.unit_chunks;
-      uint8_t* pool_page = p.pool + (int64_t)s_pages[jj] * p.S_page;
+      const int t_lo = max(0, ts0 - jj * p.P), t_hi = min(p.P, ts0 + v - jj * p.P);
+      const int n = (t_hi - t_lo) * p.unit_chunks;
+      uint8_t* pool_page = p.pool + (int64_t)s_pages[jj] * p.S_page + (int64_t)t_lo * p.S_tok;
 #pragma unroll
       for (int c = 0; c < F; ++c) {
         uint8_t* a = pool_page + c * p.S_kv;
         // not planar => F == 1
-        uint8_t* b = p.wire + ((p.planar ? c * T : 0) + n0 + (int64_t)jj * p.P) * unit_bytes;
+        uint8_t* b = p.wire +
+                     ((p.planar ? c * T : 0) + n0 + (int64_t)(jj * p.P + t_lo - ts0)) * unit_bytes;
         const uint8_t* src = PACK ? a : b;
         uint8_t* dst = PACK ? b : a;
         for (int w0 = tid; w0 < n; w0 += kThreads * kUnroll) {
@@ -191,7 +198,7 @@ __device__ __forceinline__ void copy_span(const KParams& p) {
   if (my_g >= groups) return;
   uint8_t* wire_span = p.wire + n0 * F * p.U * unit_bytes;  // TOKEN_KV: the span is one run
   if (!MULTI && s_pages[0] < 0) return;                     // single page, unusable: skip it
-  uint8_t* page0 = p.pool + (int64_t)s_pages[0] * p.S_page;
+  uint8_t* page0 = p.pool + (int64_t)s_pages[0] * p.S_page + (int64_t)ts0 * p.S_tok;
 
   for (int q0 = my_g; q0 < nunits; q0 += groups * kUnroll) {
     for (int w = my_w; w < p.unit_chunks; w += tpu) {
@@ -218,8 +225,8 @@ __device__ __forceinline__ void copy_span(const KParams& p) {
           b = wire_span + (int64_t)q * unit_bytes + (int64_t)w * VEC;
         }
         if (MULTI) {  // several pages per span: look the token's page up
-          const int jj = ts / p.P;
-          const int t = ts - jj * p.P;
+          const int jj = (ts0 + ts) / p.P;
+          const int t = ts0 + ts - jj * p.P;
           const int pg = s_pages[jj];
           a = p.pool + (int64_t)pg * p.S_page + c * p.S_kv + t * p.S_tok + h * p.S_unit +
               (int64_t)w * VEC;
@@ -249,7 +256,7 @@ topkv_page_copy_kernel(const KParams p) {
 
 // Exclusive prefix sum of seq_lens into int64 [R+1]; one CTA, any R.
 __global__ void __launch_bounds__(kThreads)
-topkv_plan_kernel(const int32_t* __restrict__ sl, int R, int64_t* __restrict__ cu) {
+topkv_plan_kernel(const int32_t* __restrict__ sl, int R, int window, int64_t* __restrict__ cu) {
   __shared__ int64_t s_warp[kThreads / 32];
   __shared__ int64_t s_carry;
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
@@ -257,7 +264,8 @@ topkv_plan_kernel(const int32_t* __restrict__ sl, int R, int64_t* __restrict__ c
   __syncthreads();
   for (int base = 0; base < R; base += kThreads) {
     const int q = base + tid;
-    const int64_t x = q < R ? (int64_t)sl[q] : 0;
+    int64_t x = q < R ? (int64_t)sl[q] : 0;
+    if (window > 0 && x > window) x = window;
     int64_t inc = x;  // inclusive scan inside the warp
     for (int o = 1; o < 32; o <<= 1) {
       const int64_t y = __shfl_up_sync(0xffffffffu, inc, o);
@@ -334,7 +342,8 @@ int check_batch(const topkv_layout* lo, const topkv_batch* b) {
   if (b == nullptr || b->struct_size != sizeof(topkv_batch) ||
       (b->flags & ~(uint32_t)TOPKV_FLAG_OVERLAP_PREVIOUS) != 0)
     return TOPKV_ERR_INVALID_ARG;
-  if (b->num_requests < 0 || b->max_pages_per_req < 0 || b->total_tokens < -1)
+  if (b->num_requests < 0 || b->max_pages_per_req < 0 || b->total_tokens < -1 ||
+      b->window_tokens < 0 || b->reserved != 0)
     return TOPKV_ERR_INVALID_ARG;
   if (b->num_requests > 0 && b->max_pages_per_req > 0) {
     if (b->block_table == nullptr || b->seq_lens == nullptr) return TOPKV_ERR_INVALID_ARG;
@@ -384,6 +393,7 @@ int prepare(int layer, const void* pool, const topkv_layout* lo, const topkv_bat
   kp->overlap = (b->flags & TOPKV_FLAG_OVERLAP_PREVIOUS) ? 1 : 0;
   kp->ppc = 1;
   kp->spr = kp->maxp;
+  kp->window = b->window_tokens;
   kp->num_pages = lo->num_pool_pages;
   kp->wire_limit = n_layer >= 0 ? n_layer : capacity - (int64_t)layer * wire_layer_stride;
   return TOPKV_OK;
@@ -446,7 +456,7 @@ int bulk_prepare_device(int* sms_out) {
 template <bool PACK>
 int launch_bulk(const KParams& kp0, const Resolved& rs, int F, cudaStream_t stream, bool* handled) {
   *handled = false;
-  if (kp0.R > kBulkMaxR) return TOPKV_OK;
+  if (kp0.R > kBulkMaxR || kp0.window > 0) return TOPKV_OK;
   const int64_t tok_bytes = (int64_t)F * rs.row_bytes;
   if (tok_bytes > kStageTarget || rs.unit_bytes > 0x7fffffff) return TOPKV_OK;
   if (!rs.merged && rs.unit_bytes < 1024) return TOPKV_OK;  // per-copy cost dominates small units
@@ -693,6 +703,7 @@ int topkv_repage_layer(int layer, const void* src_pool, const topkv_layout* src_
       ls->head_dim != ld->head_dim || ls->elem_bytes != ld->elem_bytes)
     return TOPKV_ERR_UNSUPPORTED_LAYOUT;
   if (src_batch->num_requests != dst_batch->num_requests) return TOPKV_ERR_INVALID_ARG;
+  if (src_batch->window_tokens != 0 || dst_batch->window_tokens != 0) return TOPKV_ERR_INVALID_ARG;
   if (layer < 0 || (uint32_t)layer >= ls->num_layers || (uint32_t)layer >= ld->num_layers)
     return TOPKV_ERR_LAYER_RANGE;
   if (src_pool == nullptr || dst_pool == nullptr) return TOPKV_ERR_INVALID_ARG;
@@ -758,10 +769,11 @@ int topkv_repage_layer(int layer, const void* src_pool, const topkv_layout* src_
 int topkv_build_plan(const topkv_batch* batch, int64_t* d_cu_seq_lens, topkv_stream_t stream) {
   if (batch == nullptr || batch->struct_size != sizeof(topkv_batch) || d_cu_seq_lens == nullptr)
     return TOPKV_ERR_INVALID_ARG;
-  if (batch->num_requests < 0 || (batch->num_requests > 0 && batch->seq_lens == nullptr))
+  if (batch->num_requests < 0 || (batch->num_requests > 0 && batch->seq_lens == nullptr) ||
+      batch->window_tokens < 0)
     return TOPKV_ERR_INVALID_ARG;
   topkv_plan_kernel<<<1, kThreads, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
-      batch->seq_lens, batch->num_requests, d_cu_seq_lens);
+      batch->seq_lens, batch->num_requests, batch->window_tokens, d_cu_seq_lens);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   g_launches.fetch_add(1, std::memory_order_relaxed);

@@ -39,6 +39,24 @@ int64_t topkv_kv_bytes(const topkv_layout* lo, int64_t seq_len) {
          lo->elem_bytes;
 }
 
+int64_t topkv_kv_bytes_layered(const topkv_layout* lo, const topkv_layer_spec* specs,
+                               int64_t seq_len) {
+  if (!layout_header_ok(lo) || specs == nullptr || seq_len < 0) return TOPKV_ERR_INVALID_ARG;
+  const int64_t tok_bytes = (int64_t)lo->kv_factor * lo->num_kv_heads * lo->head_dim * lo->elem_bytes;
+  int64_t total = 0;
+  for (uint32_t l = 0; l < lo->num_layers; ++l) {
+    const topkv_layer_spec& sp = specs[l];
+    if (sp.reserved != 0 || sp.param < 0) return TOPKV_ERR_INVALID_ARG;
+    switch (sp.kind) {
+      case TOPKV_LAYER_FULL: total += tok_bytes * seq_len; break;
+      case TOPKV_LAYER_WINDOW: total += tok_bytes * (sp.param < seq_len ? sp.param : seq_len); break;
+      case TOPKV_LAYER_STATE: total += sp.param; break;
+      default: return TOPKV_ERR_INVALID_ARG;
+    }
+  }
+  return total;
+}
+
 double topkv_model_transfer_s(double bytes, double bandwidth_bytes_per_s, double setup_s) {
   return bytes / bandwidth_bytes_per_s + setup_s;
 }

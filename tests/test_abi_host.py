@@ -38,7 +38,8 @@ def test_exports_every_declared_symbol():
 def test_struct_sizes_match_header():
     # natural alignment of the C structs: 10 x u32 + 7 x i64, and 4 x 32-bit + 3 ptr + i64
     assert ctypes.sizeof(tk.topkv_layout) == 96
-    assert ctypes.sizeof(tk.topkv_batch) == 48
+    assert ctypes.sizeof(tk.topkv_batch) == 56
+    assert ctypes.sizeof(tk.topkv_layer_spec) == 16
 
 
 def _gqa(L=4, pages=64, **kw):
@@ -60,6 +61,24 @@ def test_default_strides_and_sizes(golden):
     assert tk.topkv_kv_bytes(tk.make_layout(56, 2, 8, 128, 2, 16, 1), s) == 939_524_096
     assert tk.topkv_wire_layer_bytes(l70, s) * 80 == tk.topkv_kv_bytes(l70, s)
     assert tk.topkv_wire_layer_bytes(l70, -1) == tk.TOPKV_ERR_INVALID_ARG
+
+
+def test_layered_sizes(golden):
+    g = golden("paper_values.txt")
+    s = int(g["seq_len"])
+    F, W, S = tk.TOPKV_LAYER_FULL, tk.TOPKV_LAYER_WINDOW, tk.TOPKV_LAYER_STATE
+    oss = tk.make_layout(36, 2, 8, 64, 2, 16, 1)
+    specs = [(W, 128) if l % 2 == 0 else (F, 0) for l in range(36)]
+    got = tk.topkv_kv_bytes_layered(oss, specs, s)
+    assert got == 18 * 2 * 8 * 64 * 2 * (4096 + 128)
+    assert round(got / 2**30, 2) == float(g["layered.gpt_oss_120b.gb"])
+    l70 = tk.make_layout(80, 2, 8, 128, 2, 16, 1)
+    assert tk.topkv_kv_bytes_layered(l70, [(F, 0)] * 80, s) == tk.topkv_kv_bytes(l70, s)
+    assert tk.topkv_kv_bytes_layered(l70, [(W, 2 * s)] * 80, s) == tk.topkv_kv_bytes(l70, s)
+    two = tk.make_layout(2, 2, 8, 128, 2, 16, 1)
+    assert tk.topkv_kv_bytes_layered(two, [(S, 1000), (S, 24)], s) == 1024
+    assert tk.topkv_kv_bytes_layered(two, [(7, 0), (F, 0)], s) == tk.TOPKV_ERR_INVALID_ARG
+    assert tk.topkv_kv_bytes_layered(two, [(W, -1), (F, 0)], s) == tk.TOPKV_ERR_INVALID_ARG
 
 
 def test_model_helpers(golden):
@@ -111,6 +130,8 @@ def test_argument_validation_without_gpu():
     bad = tk.make_layout(2, 2, 1, 4, 2, 16, 8)               # 8-byte rows
     assert P(0, pool, bad, b, wire, cap) == tk.TOPKV_ERR_ALIGNMENT
     bb = _batch(); bb.struct_size = 4
+    assert P(0, pool, lo, bb, wire, cap) == tk.TOPKV_ERR_INVALID_ARG
+    bb = _batch(); bb.window_tokens = -1
     assert P(0, pool, lo, bb, wire, cap) == tk.TOPKV_ERR_INVALID_ARG
     bb = _batch(); bb.flags = 2                              # unknown flag bit
     assert P(0, pool, lo, bb, wire, cap) == tk.TOPKV_ERR_INVALID_ARG

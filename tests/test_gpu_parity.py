@@ -397,6 +397,74 @@ def test_overlapped_launches_keep_results_and_order(dev):
     torch.cuda.empty_cache()
 
 
+# -------------------------------------------------------------------- windowed layers (§2.2)
+
+@pytest.mark.parametrize("seed", range(16))
+def test_windowed_layers(dev, seed):
+    """A windowed layer keeps (and ships) only the last min(s, W) tokens of each request;
+    block-table columns before the window are stale (-1 here) and must never be followed."""
+    g, sl, bt_s, bt_d, rng = _case(seed)
+    W = int(rng.choice([1, 2, g.P, g.P + 1, 3 * g.P - 1, 1000]))
+    g.window = W
+    for bt in (bt_s, bt_d):                               # free the pages before the window
+        for r in range(len(sl)):
+            bt[r, :max(0, int(sl[r]) - W) // g.P] = -1
+    T = g.kept_tokens(sl)
+    g.W_layer = g.wire_layer_bytes(T) + 32
+    lo = _layout_from_geom(g)
+    src_h = rng.integers(0, 256, g.L * g.S_layer, dtype=np.uint8)
+    dst_h = rng.integers(0, 256, g.L * g.S_layer, dtype=np.uint8)
+    src, dst = torch.from_numpy(src_h).to(dev), torch.from_numpy(dst_h).to(dev)
+    wire = torch.full((g.L * g.W_layer + 64,), 0x3C, dtype=torch.uint8, device=dev)
+    d_sl = torch.from_numpy(sl).to(dev)
+    d_bs, d_bd = torch.from_numpy(bt_s).to(dev), torch.from_numpy(bt_d).to(dev)
+    cu = None
+    if seed % 2:
+        cu = torch.zeros(len(sl) + 1, dtype=torch.int64, device=dev)
+        tk.check(tk.topkv_build_plan(tk.make_batch(d_bs, d_sl, window_tokens=W), cu))
+        want_cu = np.concatenate([[0], np.cumsum(np.minimum(sl, W).astype(np.int64))])
+        assert np.array_equal(cu.cpu().numpy(), want_cu)
+    bs = tk.make_batch(d_bs, d_sl, T if seed % 3 else -1, cu, window_tokens=W)
+    bd = tk.make_batch(d_bd, d_sl, T if seed % 3 else -1, cu, window_tokens=W)
+    want_wire = np.full(g.L * g.W_layer + 64, 0x3C, dtype=np.uint8)
+    for layer in range(g.L):
+        tk.check(tk.topkv_pack_layer(layer, src, lo, bs, wire, wire.numel()))
+        tk.check(tk.topkv_unpack_layer(layer, dst, lo, bd, wire, wire.numel()))
+        oracle.pack(g, layer, src_h, bt_s, sl, wire=want_wire)
+        oracle.unpack(g, layer, dst_h, bt_d, sl, want_wire)
+    torch.cuda.synchronize()
+    assert np.array_equal(wire.cpu().numpy(), want_wire)
+    assert np.array_equal(dst.cpu().numpy(), dst_h)
+
+
+def test_windowed_layer_bench_shape(dev):
+    """gpt-oss-like windowed layer on the 8B batch: window 128 of up to 4096 tokens."""
+    w = harness.setup(wl.CFG2, dev, layers=2)
+    b, s = w.batch, wl.CFG2
+    W = 128
+    g = _geom(s, b.num_pool_pages, 1, 0, 0)
+    g.window = W
+    T = g.kept_tokens(b.seq_lens)
+    assert T == 16 * 128
+    bs = tk.make_batch(w.src_bt, w.seq_lens, T, None, window_tokens=W)
+    bd = tk.make_batch(w.dst_bt, w.seq_lens, T, None, window_tokens=W)
+    n = g.wire_layer_bytes(T)
+    wire = torch.zeros(n, dtype=torch.uint8, device=dev)
+    lo = tk.make_layout(2, s.F, s.H, s.D, s.E, s.P, b.num_pool_pages, wire_layer_stride=0)
+    for layer in range(2):
+        src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, layer)
+        dst_h = harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, layer)
+        tk.check(tk.topkv_pack_layer(layer, w.src_pool, lo, bs, wire, n))
+        tk.check(tk.topkv_unpack_layer(layer, w.dst_pool, lo, bd, wire, n))
+        torch.cuda.synchronize()
+        want = oracle.pack(g, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=8)
+        assert np.array_equal(wire.cpu().numpy(), want)
+        oracle.unpack(g, 0, dst_h, b.dst_block_table, b.seq_lens, want, impl="rows", threads=8)
+        assert np.array_equal(harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, layer), dst_h)
+    del w
+    torch.cuda.empty_cache()
+
+
 # -------------------------------------------------------------------- direct re-paging
 
 def _repage_case(seed):
