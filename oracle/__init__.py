@@ -71,6 +71,13 @@ def _load():
             fn = getattr(lib, name)
             fn.restype = None
             fn.argtypes = [gp, i64, vp, i64, i64, vp, vp, vp, ctypes.c_int]
+        u64 = ctypes.c_uint64
+        lib.oracle_crc64.restype = u64
+        lib.oracle_crc64.argtypes = [vp, i64, u64]
+        lib.oracle_crc64_iso.restype = u64
+        lib.oracle_crc64_iso.argtypes = [vp, i64]
+        lib.oracle_kv_plane_crc.restype = u64
+        lib.oracle_kv_plane_crc.argtypes = [gp, vp, i64, i64, vp, vp, i64, i64]
         _lib = lib
     return _lib
 
@@ -225,3 +232,42 @@ def unpack(g: Geom, layer: int, pool: np.ndarray, bt: np.ndarray, sl: np.ndarray
     else:
         raise ValueError(impl)
     return pool
+
+
+# ---- integrity check and header of the serialised cache (§3.4) --------------------------------
+
+POLY_ISO_REFLECTED = 0xD800000000000000    # x^64 + x^4 + x^3 + x + 1 (CRC-64/GO-ISO), the reading taken
+POLY_ECMA_REFLECTED = 0xC96C5795D7870F42   # ECMA-182 (CRC-64/XZ), used only to check the routine
+HEADER_BYTES = 128
+HEADER_MAGIC = b"KVCACHE1"
+
+
+def crc64(data, poly_reflected: int = POLY_ISO_REFLECTED) -> int:
+    """Reflected CRC-64, all-ones initial value, final inversion, bit by bit."""
+    a = np.frombuffer(bytes(data), dtype=np.uint8) if not isinstance(data, np.ndarray) else data
+    a = np.ascontiguousarray(a, dtype=np.uint8)
+    return int(_load().oracle_crc64(a.ctypes.data, a.size, poly_reflected))
+
+
+def kv_plane_crc(g: Geom, pool: np.ndarray, bt: np.ndarray, sl: np.ndarray, r: int, c: int) -> int:
+    """CRC-64 of the K (c = 0) or V (c = 1) tensor of request r in the order
+    [layers][seq_len][kv_heads][head_dim], gathered from the paged pool."""
+    bt, sl = _tables(bt, sl)
+    _u8(pool, False)
+    cg = g._c()
+    return int(_load().oracle_kv_plane_crc(ctypes.byref(cg), pool.ctypes.data, sl.shape[0],
+                                           bt.shape[1], bt.ctypes.data, sl.ctypes.data, r, c))
+
+
+def build_header(request_id: int, model_id: int, seq_len: int, g: Geom, crc_k: int, crc_v: int) -> bytes:
+    """The fixed 128-byte header of §3.4: magic, request ID, model ID, tensor dimensions
+    (sequence length, layers, KV heads, head dimension), tensor sizes, the two checksums.
+    The paper fixes the content and the total size, not the field order or widths; the order
+    below follows the order in which §3.4 lists the fields, little-endian, zero padded."""
+    import struct
+    plane = g.L * seq_len * g.h_kv * g.d_h * g.b_p
+    body = struct.pack("<8sQQIIIIIIQQQQ", HEADER_MAGIC, request_id, model_id, seq_len, g.L, g.h_kv,
+                       g.d_h, g.b_p, g.F, plane, plane if g.F == 2 else 0, crc_k,
+                       crc_v if g.F == 2 else 0)
+    assert len(body) == 80
+    return body + bytes(HEADER_BYTES - len(body))

@@ -176,3 +176,40 @@ void oracle_unpack_rows(const oracle_geom* g, int64_t layer, uint8_t* pool, int6
                         int threads) {
   run_rows(g, layer, pool, R, maxp, bt, sl, (uint8_t*)wire, threads, 0);
 }
+
+/* ---- CRC-64 (§3.4) -------------------------------------------------------------------- */
+
+/* One step of the reflected shift register: feed the byte, then shift eight times. */
+static uint64_t crc64_byte(uint64_t crc, uint8_t b, uint64_t poly_reflected) {
+  crc ^= b;
+  for (int k = 0; k < 8; ++k) crc = (crc & 1) ? (crc >> 1) ^ poly_reflected : (crc >> 1);
+  return crc;
+}
+
+uint64_t oracle_crc64(const uint8_t* data, int64_t n, uint64_t poly_reflected) {
+  uint64_t crc = ~(uint64_t)0; /* initial value: all ones */
+  for (int64_t i = 0; i < n; ++i) crc = crc64_byte(crc, data[i], poly_reflected);
+  return ~crc; /* final inversion */
+}
+
+#define ORACLE_POLY_ISO_REFLECTED 0xD800000000000000ull /* x^64 + x^4 + x^3 + x + 1 */
+
+uint64_t oracle_crc64_iso(const uint8_t* data, int64_t n) {
+  return oracle_crc64(data, n, ORACLE_POLY_ISO_REFLECTED);
+}
+
+uint64_t oracle_kv_plane_crc(const oracle_geom* g, const uint8_t* pool, int64_t R, int64_t maxp,
+                             const int32_t* bt, const int32_t* sl, int64_t r, int64_t c) {
+  (void)R;
+  uint64_t crc = ~(uint64_t)0;
+  for (int64_t l = 0; l < g->L; ++l)
+    for (int64_t i = first_kept(g, sl[r]); i < sl[r]; ++i) {
+      int64_t page = bt[r * maxp + i / g->P];
+      int64_t t = i % g->P;
+      for (int64_t h = 0; h < g->h_kv; ++h)
+        for (int64_t d = 0; d < g->d_h; ++d)
+          for (int64_t b = 0; b < g->b_p; ++b)
+            crc = crc64_byte(crc, pool[poff(g, l, page, c, t, h, d, b)], ORACLE_POLY_ISO_REFLECTED);
+    }
+  return ~crc;
+}

@@ -56,4 +56,20 @@ void oracle_pack_rows(const oracle_geom* g, int64_t layer, const uint8_t* pool, 
 void oracle_unpack_rows(const oracle_geom* g, int64_t layer, uint8_t* pool, int64_t R,
                         int64_t maxp, const int32_t* bt, const int32_t* sl, const uint8_t* wire,
                         int threads);
+
+/* ---- integrity check of the serialised tensors (§3.4) -----------------------------------
+ * The paper's header carries "CRC-64 checksums for both key and value tensors" and does not
+ * name the polynomial. Reading taken: the reflected CRC-64 with all-ones initial value and
+ * final inversion, on the ISO 3309 polynomial x^64 + x^4 + x^3 + x + 1 (catalogue name
+ * CRC-64/GO-ISO). oracle_crc64 is the textbook bit-by-bit shift register for any reflected
+ * polynomial, so that the same routine can be checked against a library on the ECMA-182
+ * polynomial; oracle_crc64_iso fixes the ISO one. */
+uint64_t oracle_crc64(const uint8_t* data, int64_t n, uint64_t poly_reflected);
+uint64_t oracle_crc64_iso(const uint8_t* data, int64_t n);
+
+/* CRC of plane c (0 = K, 1 = V) of request r, over the tensor in the paper's order
+ * [layers][seq_len][kv_heads][head_dim] (§3.4), read from the paged pool through the block
+ * table. A windowed geometry contributes only the tokens it keeps. */
+uint64_t oracle_kv_plane_crc(const oracle_geom* g, const uint8_t* pool, int64_t R, int64_t maxp,
+                             const int32_t* bt, const int32_t* sl, int64_t r, int64_t c);
 #endif

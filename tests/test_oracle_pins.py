@@ -453,3 +453,81 @@ def test_windowed_layer_never_touches_pages_before_the_window():
     assert (dst != 0x77).sum() <= wire.size
     # tokens 0..2 of request 2 (page 4, first three rows of each plane) stay untouched
     assert (dst[4 * g.S_page:4 * g.S_page + 48] == 0x77).all()
+
+
+# ---------------------------------------------------------------- CRC-64 (§3.4)
+
+def _xz_crc64(data: bytes) -> int:
+    """CRC-64/XZ of data as liblzma computes it: compress with an integrity check of type
+    CRC64 and read the 8-byte check field that precedes the stream index."""
+    import lzma
+    import struct
+    blob = lzma.compress(data, format=lzma.FORMAT_XZ, check=lzma.CHECK_CRC64)
+    backward = struct.unpack("<I", blob[-8:-4])[0]           # stream footer: stored backward size
+    index_size = (backward + 1) * 4
+    end = len(blob) - 12 - index_size
+    return struct.unpack("<Q", blob[end - 8:end])[0]
+
+
+def _crc64_as_polynomial_remainder(data: bytes, poly_normal: int) -> int:
+    """Third derivation, from the definition: with the message as a polynomial M (first bit =
+    highest power, n bytes), the check is (ones * x^(8n) + M * x^64) mod P, inverted; the bits
+    of every byte and of the result are reflected. Python integers, no shift register."""
+    n = len(data)
+    M = 0
+    for b in data:
+        M = (M << 8) | int(f"{b:08b}"[::-1], 2)
+    val = (((1 << 64) - 1) << (8 * n)) ^ (M << 64)
+    P = (1 << 64) | poly_normal
+    while val.bit_length() > 64:
+        val ^= P << (val.bit_length() - 65)
+    val ^= (1 << 64) - 1
+    return int(f"{val:064b}"[::-1], 2)
+
+
+def test_crc64_routine_against_library_and_catalogue():
+    rng = np.random.default_rng(11)
+    # the generic routine on the ECMA-182 polynomial is what liblzma computes ...
+    for n in (1, 2, 7, 8, 9, 64, 1000, 4099):     # (an empty stream has no block to carry a check)
+        data = rng.integers(0, 256, n, dtype=np.uint8).tobytes()
+        assert oracle.crc64(data, oracle.POLY_ECMA_REFLECTED) == _xz_crc64(data), n
+    # ... and gives the catalogue check values of both parameter sets
+    assert oracle.crc64(b"123456789", oracle.POLY_ECMA_REFLECTED) == 0x995DC9BBDF1939FA  # CRC-64/XZ
+    assert oracle.crc64(b"123456789") == 0xB90956C775A41001                              # CRC-64/GO-ISO
+    assert oracle.crc64(b"") == 0
+    # the polynomial-remainder definition agrees on both polynomials
+    for n in (0, 3, 8, 31, 257):
+        data = rng.integers(0, 256, n, dtype=np.uint8).tobytes()
+        assert oracle.crc64(data) == _crc64_as_polynomial_remainder(data, 0x1B), n
+        assert oracle.crc64(data, oracle.POLY_ECMA_REFLECTED) == \
+            _crc64_as_polynomial_remainder(data, 0x42F0E1EBA9EA3693), n
+
+
+def test_kv_plane_crc_is_the_crc_of_the_paper_payload_order():
+    # K tensor of a request = [layers][seq_len][kv_heads][head_dim]: build it with numpy from
+    # the PLANAR pack of each layer (already pinned) and checksum the bytes
+    g, pool, bt, sl = _random_case(21, 2, 2, 8, 4, strided=True)
+    g.W_layer = 0
+    g.wire_order = WIRE_PLANAR
+    cu = np.concatenate([[0], np.cumsum(sl.astype(np.int64))])
+    T = int(cu[-1])
+    planes = [oracle.pack(g, l, pool, bt, sl).reshape(g.F, T, g.row_bytes) for l in range(g.L)]
+    for r in range(len(sl)):
+        for c in range(g.F):
+            tensor = np.concatenate([planes[l][c, cu[r]:cu[r + 1]].reshape(-1) for l in range(g.L)])
+            assert oracle.kv_plane_crc(g, pool, bt, sl, r, c) == oracle.crc64(tensor.tobytes())
+    g.wire_order = WIRE_TOKEN_KV
+
+
+def test_header_layout():
+    g = Geom(L=80, F=2, h_kv=8, d_h=128, b_p=2, P=16, num_pages=1)
+    h = oracle.build_header(7, 0xABCDEF, 4096, g, 0x1122334455667788, 0x99AABBCCDDEEFF00)
+    assert len(h) == 128 and h[:8] == b"KVCACHE1"                  # §3.4: 128 bytes, 8-byte magic
+    assert int.from_bytes(h[8:16], "little") == 7 and int.from_bytes(h[16:24], "little") == 0xABCDEF
+    dims = [int.from_bytes(h[24 + 4 * k:28 + 4 * k], "little") for k in range(6)]
+    assert dims == [4096, 80, 8, 128, 2, 2]
+    assert int.from_bytes(h[48:56], "little") == 80 * 4096 * 8 * 128 * 2 == 671_088_640
+    assert 2 * 671_088_640 == oracle.kv_bytes(80, 8, 128, 4096)     # K + V sizes add up to Eq. 1
+    assert int.from_bytes(h[64:72], "little") == 0x1122334455667788
+    assert int.from_bytes(h[72:80], "little") == 0x99AABBCCDDEEFF00
+    assert h[80:] == bytes(48)
