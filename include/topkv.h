@@ -62,7 +62,8 @@ typedef enum topkv_status {
   TOPKV_ERR_ALIGNMENT = -3,          /* a base, stride or row_bytes is not a multiple of 16 B */
   TOPKV_ERR_CAPACITY = -4,           /* wire / host / staging buffer smaller than N_layer     */
   TOPKV_ERR_UNSUPPORTED_LAYOUT = -5, /* descriptor is self-inconsistent or not supported      */
-  TOPKV_ERR_CUDA = -6                /* a CUDA call failed; see topkv_last_cuda_error()       */
+  TOPKV_ERR_CUDA = -6,               /* a CUDA call failed; see topkv_last_cuda_error()       */
+  TOPKV_ERR_CHECKSUM = -7            /* header magic, dimensions or a CRC-64 do not match      */
 } topkv_status;
 
 enum { TOPKV_KIND_GQA = 0, TOPKV_KIND_MLA = 1 };
@@ -178,6 +179,66 @@ int topkv_repage_layer(int layer, const void* src_pool, const topkv_layout* src_
                        const topkv_batch* src_batch, void* dst_pool,
                        const topkv_layout* dst_layout, const topkv_batch* dst_batch,
                        topkv_stream_t stream);
+
+/* ---- integrity: wire header and CRC-64 (§3.4) ------------------------------------------------ */
+
+/* The fixed 128-byte header of §3.4, one per request: magic, request ID, model ID, tensor
+ * dimensions (sequence length, layers, KV heads, head dimension), tensor sizes, CRC-64 of the
+ * key tensor and of the value tensor. The paper fixes the content and the size; field order
+ * and widths below are this library's reading (the order in which the paper lists them,
+ * little-endian, zero padded). For an MLA cache (kv_factor 1) v_bytes and crc_v are 0. */
+typedef struct topkv_wire_header {
+  char magic[8];          /* "KVCACHE1"                                                    */
+  uint64_t request_id;
+  uint64_t model_id;
+  uint32_t seq_len, num_layers, num_kv_heads, head_dim, elem_bytes, kv_factor;
+  uint64_t k_bytes, v_bytes; /* L * seq_len * H * D * E each                                */
+  uint64_t crc_k, crc_v;
+  uint8_t reserved[48];   /* zero                                                           */
+} topkv_wire_header;
+
+int topkv_header_fill(topkv_wire_header* header, uint64_t request_id, uint64_t model_id,
+                      const topkv_layout* layout, int64_t seq_len, uint64_t crc_k, uint64_t crc_v);
+/* TOPKV_OK, or TOPKV_ERR_CHECKSUM when the magic, a dimension, a size or a checksum differs
+ * from what the receiver expects / has computed. */
+int topkv_header_check(const topkv_wire_header* header, const topkv_layout* layout,
+                       int64_t seq_len, uint64_t crc_k, uint64_t crc_v);
+
+/* The checksum: reflected CRC-64, all-ones initial value, final inversion, ISO 3309
+ * polynomial x^64 + x^4 + x^3 + x + 1 (the paper names no polynomial). The
+ * K (V) checksum of a request covers its K (V) tensor in the order
+ * [layers][seq_len][kv_heads][head_dim]. topkv_crc64 is the plain HOST routine. */
+uint64_t topkv_crc64(const void* h_data, int64_t nbytes);
+
+/* Device-side checksumming, fused into pack / unpack. Usage, per batch:
+ *   topkv_crc_begin(...)                      once: tables + running states (all on `stream`)
+ *   topkv_pack_layer_crc(l, ...)              for l = 0 .. L-1 IN ORDER (or unpack on the receiver)
+ *   topkv_crc_finish(...)                     d_crc_out[r*F + c] = checksum of request r, plane c
+ * d_crc_state: DEVICE uint64 [R*F]; d_workspace: DEVICE scratch of at least
+ * topkv_crc_workspace_bytes(...) bytes, 16-byte aligned, owned by the caller and reserved for
+ * this batch between begin and finish. Requirements: heads contiguous in the pool,
+ * batch->cu_seq_lens given, window_tokens 0, kv_factor * page_tokens * (runs per row) <= 1024
+ * (else TOPKV_ERR_UNSUPPORTED_LAYOUT). TOPKV_FLAG_OVERLAP_PREVIOUS is ignored by these calls.
+ * The copy itself is identical to topkv_pack_layer / topkv_unpack_layer. */
+int64_t topkv_crc_workspace_bytes(const topkv_layout* layout, int32_t num_requests,
+                                  int32_t max_pages_per_req);
+int topkv_crc_begin(const topkv_layout* layout, const topkv_batch* batch, uint64_t* d_crc_state,
+                    void* d_workspace, int64_t workspace_bytes, topkv_stream_t stream);
+int topkv_pack_layer_crc(int layer, const void* src_pool, const topkv_layout* layout,
+                         const topkv_batch* batch, void* d_wire, int64_t wire_capacity_bytes,
+                         uint64_t* d_crc_state, void* d_workspace, int64_t workspace_bytes,
+                         topkv_stream_t stream);
+int topkv_unpack_layer_crc(int layer, void* dst_pool, const topkv_layout* layout,
+                           const topkv_batch* batch, const void* d_wire, int64_t wire_bytes,
+                           uint64_t* d_crc_state, void* d_workspace, int64_t workspace_bytes,
+                           topkv_stream_t stream);
+int topkv_crc_finish(const topkv_layout* layout, const topkv_batch* batch,
+                     const uint64_t* d_crc_state, uint64_t* d_crc_out, topkv_stream_t stream);
+
+/* Host-side retry policy of the transfer orchestrator (§3.1: 2 retries, 100 ms exponential
+ * backoff): calls attempt(ctx) until it returns TOPKV_OK, at most 1 + retries times, sleeping
+ * backoff_ms, 2*backoff_ms, ... between attempts. Returns the last status. */
+int topkv_retry(int (*attempt)(void* ctx), void* ctx, int retries, int backoff_ms);
 
 /* ---- allocation-free host leg -------------------------------------------------------------- */
 

@@ -22,6 +22,7 @@ TOPKV_ERR_ALIGNMENT = -3
 TOPKV_ERR_CAPACITY = -4
 TOPKV_ERR_UNSUPPORTED_LAYOUT = -5
 TOPKV_ERR_CUDA = -6
+TOPKV_ERR_CHECKSUM = -7
 
 TOPKV_KIND_GQA, TOPKV_KIND_MLA = 0, 1
 TOPKV_WIRE_TOKEN_KV, TOPKV_WIRE_PLANAR = 0, 1
@@ -38,6 +39,9 @@ EXPORTS = (
     "topkv_strerror", "topkv_version", "topkv_last_cuda_error", "topkv_kernel_launch_count",
     "topkv_set_kernel_variant", "topkv_pack_layer_to_host_noalloc", "topkv_device_error_flags",
     "topkv_reset_device_error_flags", "topkv_repage_layer", "topkv_kv_bytes_layered",
+    "topkv_header_fill", "topkv_header_check", "topkv_crc64", "topkv_crc_workspace_bytes",
+    "topkv_crc_begin", "topkv_pack_layer_crc", "topkv_unpack_layer_crc", "topkv_crc_finish",
+    "topkv_retry",
 )
 
 
@@ -69,6 +73,19 @@ class topkv_layer_spec(ctypes.Structure):
 TOPKV_LAYER_FULL, TOPKV_LAYER_WINDOW, TOPKV_LAYER_STATE = 0, 1, 2
 
 
+class topkv_wire_header(ctypes.Structure):
+    _fields_ = [
+        ("magic", ctypes.c_char * 8), ("request_id", ctypes.c_uint64), ("model_id", ctypes.c_uint64),
+        ("seq_len", c_uint32), ("num_layers", c_uint32), ("num_kv_heads", c_uint32),
+        ("head_dim", c_uint32), ("elem_bytes", c_uint32), ("kv_factor", c_uint32),
+        ("k_bytes", ctypes.c_uint64), ("v_bytes", ctypes.c_uint64), ("crc_k", ctypes.c_uint64),
+        ("crc_v", ctypes.c_uint64), ("reserved", ctypes.c_uint8 * 48),
+    ]
+
+
+RETRY_ATTEMPT = ctypes.CFUNCTYPE(c_int, c_void_p)
+
+
 class TopkvError(RuntimeError):
     def __init__(self, status: int):
         self.status = status
@@ -95,6 +112,21 @@ def lib() -> ctypes.CDLL:
         L.topkv_unpack_layer_from_host.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64,
                                                    c_void_p, c_int64, c_void_p]
         L.topkv_build_plan.argtypes = [bp, c_void_p, c_void_p]
+        u64 = ctypes.c_uint64
+        hp = ctypes.POINTER(topkv_wire_header)
+        L.topkv_header_fill.argtypes = [hp, u64, u64, lp, c_int64, u64, u64]
+        L.topkv_header_check.argtypes = [hp, lp, c_int64, u64, u64]
+        L.topkv_crc64.argtypes = [c_void_p, c_int64]
+        L.topkv_crc64.restype = u64
+        L.topkv_crc_workspace_bytes.argtypes = [lp, c_int32, c_int32]
+        L.topkv_crc_workspace_bytes.restype = c_int64
+        L.topkv_crc_begin.argtypes = [lp, bp, c_void_p, c_void_p, c_int64, c_void_p]
+        L.topkv_pack_layer_crc.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p,
+                                           c_void_p, c_int64, c_void_p]
+        L.topkv_unpack_layer_crc.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p,
+                                             c_void_p, c_int64, c_void_p]
+        L.topkv_crc_finish.argtypes = [lp, bp, c_void_p, c_void_p, c_void_p]
+        L.topkv_retry.argtypes = [RETRY_ATTEMPT, c_void_p, c_int, c_int]
         L.topkv_repage_layer.argtypes = [c_int, c_void_p, lp, bp, c_void_p, lp, bp, c_void_p]
         L.topkv_pack_layer_to_host_noalloc.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64,
                                                        c_void_p]
@@ -227,6 +259,60 @@ def topkv_repage_layer(layer, src_pool, src_layout, src_batch, dst_pool, dst_lay
                                     ctypes.byref(src_batch), _ptr(dst_pool),
                                     ctypes.byref(dst_layout), ctypes.byref(dst_batch),
                                     _stream(stream))
+
+
+def topkv_header_fill(header, request_id, model_id, layout, seq_len, crc_k, crc_v):
+    return lib().topkv_header_fill(ctypes.byref(header), request_id, model_id, ctypes.byref(layout),
+                                   seq_len, crc_k, crc_v)
+
+
+def topkv_header_check(header, layout, seq_len, crc_k, crc_v):
+    return lib().topkv_header_check(ctypes.byref(header), ctypes.byref(layout), seq_len, crc_k,
+                                    crc_v)
+
+
+def topkv_crc64(h_data, nbytes=None):
+    """Host CRC-64 of a bytes object or a numpy array."""
+    if isinstance(h_data, (bytes, bytearray)):
+        buf = (ctypes.c_char * len(h_data)).from_buffer_copy(h_data)
+        return lib().topkv_crc64(ctypes.addressof(buf), len(h_data))
+    return lib().topkv_crc64(_ptr(h_data), h_data.nbytes if nbytes is None else nbytes)
+
+
+def topkv_crc_workspace_bytes(layout, num_requests, max_pages_per_req):
+    return lib().topkv_crc_workspace_bytes(ctypes.byref(layout), num_requests, max_pages_per_req)
+
+
+def topkv_crc_begin(layout, batch, d_crc_state, d_workspace, workspace_bytes, stream=None):
+    return lib().topkv_crc_begin(ctypes.byref(layout), ctypes.byref(batch), _ptr(d_crc_state),
+                                 _ptr(d_workspace), workspace_bytes, _stream(stream))
+
+
+def topkv_pack_layer_crc(layer, src_pool, layout, batch, d_wire, wire_capacity_bytes, d_crc_state,
+                         d_workspace, workspace_bytes, stream=None):
+    return lib().topkv_pack_layer_crc(layer, _ptr(src_pool), ctypes.byref(layout),
+                                      ctypes.byref(batch), _ptr(d_wire), wire_capacity_bytes,
+                                      _ptr(d_crc_state), _ptr(d_workspace), workspace_bytes,
+                                      _stream(stream))
+
+
+def topkv_unpack_layer_crc(layer, dst_pool, layout, batch, d_wire, wire_bytes, d_crc_state,
+                           d_workspace, workspace_bytes, stream=None):
+    return lib().topkv_unpack_layer_crc(layer, _ptr(dst_pool), ctypes.byref(layout),
+                                        ctypes.byref(batch), _ptr(d_wire), wire_bytes,
+                                        _ptr(d_crc_state), _ptr(d_workspace), workspace_bytes,
+                                        _stream(stream))
+
+
+def topkv_crc_finish(layout, batch, d_crc_state, d_crc_out, stream=None):
+    return lib().topkv_crc_finish(ctypes.byref(layout), ctypes.byref(batch), _ptr(d_crc_state),
+                                  _ptr(d_crc_out), _stream(stream))
+
+
+def topkv_retry(attempt, retries=2, backoff_ms=100):
+    """attempt: a Python callable returning a topkv status; §3.1's policy by default."""
+    cb = RETRY_ATTEMPT(lambda _ctx: int(attempt()))
+    return lib().topkv_retry(cb, None, retries, backoff_ms)
 
 
 def topkv_build_plan(batch, d_cu_seq_lens, stream=None):

@@ -10,6 +10,7 @@
 
 #include "topkv_bulk.cuh"
 #include "topkv_common.cuh"
+#include "topkv_crc.cuh"
 #include "topkv_repage.cuh"
 
 #include <algorithm>
@@ -560,6 +561,66 @@ int noalloc_staging_address(void** out) {
   return TOPKV_OK;
 }
 
+// ---- CRC-64 fused into pack / unpack ------------------------------------------------------------
+// Cuts a token row into runs of at most 1 KiB (one per thread); fails when a page and plane
+// would need more threads than a CTA has.
+int crc_geometry(const topkv_layout* lo, const Resolved& rs, CrcGeom* g) {
+  if (rs.U != 1) return TOPKV_ERR_UNSUPPORTED_LAYOUT;  // heads must be contiguous
+  int rpr = 0;
+  for (int k = 1; k <= 4096; ++k) {
+    if (rs.row_bytes % k) continue;
+    const int64_t run = rs.row_bytes / k;
+    if (run % 16) continue;
+    if (run <= 1024) {
+      rpr = k;
+      break;
+    }
+  }
+  if (rpr == 0) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  g->rpr = rpr;
+  g->run_bytes = (int)(rs.row_bytes / rpr);
+  g->RB = (int)lo->page_tokens * rpr;
+  if ((int64_t)lo->kv_factor * g->RB > 1024) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  return TOPKV_OK;
+}
+
+int64_t crc_workspace_words(const CrcGeom& g, int R, int maxp, int F) {
+  return (int64_t)g.RB + (maxp + 1) + 2 * (int64_t)R + (int64_t)R * maxp * F;
+}
+
+template <bool PACK>
+int crc_copy(int layer, const void* pool, const topkv_layout* lo, const topkv_batch* b,
+             const void* wire, int64_t cap, uint64_t* state, void* ws, int64_t ws_bytes,
+             cudaStream_t stream) {
+  CrcCopyParams cp;
+  Resolved rs;
+  int64_t n_layer;
+  int st = prepare(layer, pool, lo, b, wire, cap, lo ? lo->wire_layer_stride : 0, &cp.k, &rs, &n_layer);
+  if (st != TOPKV_OK) return st;
+  if (state == nullptr || ws == nullptr || !mult16p(ws)) return TOPKV_ERR_INVALID_ARG;
+  if (b->cu_seq_lens == nullptr || b->window_tokens != 0) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  st = crc_geometry(lo, rs, &cp.g);
+  if (st != TOPKV_OK) return st;
+  const int F = (int)lo->kv_factor, R = b->num_requests, maxp = b->max_pages_per_req;
+  if (ws_bytes < 8 * crc_workspace_words(cp.g, R, maxp, F)) return TOPKV_ERR_CAPACITY;
+  if (R == 0 || maxp == 0) return TOPKV_OK;
+  const CrcWorkspace w = crc_carve(ws, cp.g.RB, maxp, R);
+  cp.c_run = w.c_run;
+  cp.page_rem = w.page_rem;
+  cp.k.overlap = 0;  // the page remainders are shared with the fold kernel of the previous layer
+  const dim3 grid((unsigned)((int64_t)R * maxp)), block((unsigned)((F * cp.g.RB + 31) / 32 * 32));
+  if (F == 1) launch_pdl(topkv_crc_copy_kernel<1, PACK>, grid, block, 0, stream, cp);
+  else launch_pdl(topkv_crc_copy_kernel<2, PACK>, grid, block, 0, stream, cp);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  topkv_crc_fold_kernel<<<(unsigned)(R * F), 256, 0, stream>>>(w, b->seq_lens, maxp, (int)lo->page_tokens,
+                                                              F, state);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_launches.fetch_add(2, std::memory_order_relaxed);
+  return TOPKV_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -760,6 +821,77 @@ int topkv_repage_layer(int layer, const void* src_pool, const topkv_layout* src_
     if (F == 1) launch_pdl(topkv_repage_kernel<1, 16>, grid, block, 0, s, p);
     else launch_pdl(topkv_repage_kernel<2, 16>, grid, block, 0, s, p);
   }
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return TOPKV_OK;
+}
+
+int64_t topkv_crc_workspace_bytes(const topkv_layout* layout, int32_t num_requests,
+                                  int32_t max_pages_per_req) {
+  Resolved rs;
+  int st = check_layout(layout, &rs);
+  if (st != TOPKV_OK) return st;
+  if (num_requests < 0 || max_pages_per_req < 0) return TOPKV_ERR_INVALID_ARG;
+  CrcGeom g;
+  st = crc_geometry(layout, rs, &g);
+  if (st != TOPKV_OK) return st;
+  return 8 * crc_workspace_words(g, num_requests, max_pages_per_req, (int)layout->kv_factor);
+}
+
+int topkv_crc_begin(const topkv_layout* layout, const topkv_batch* batch, uint64_t* d_crc_state,
+                    void* d_workspace, int64_t workspace_bytes, topkv_stream_t stream) {
+  Resolved rs;
+  int st = check_layout(layout, &rs);
+  if (st != TOPKV_OK) return st;
+  st = check_batch(layout, batch);
+  if (st != TOPKV_OK) return st;
+  if (d_crc_state == nullptr || d_workspace == nullptr || !mult16p(d_workspace))
+    return TOPKV_ERR_INVALID_ARG;
+  if (batch->window_tokens != 0) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  CrcGeom g;
+  st = crc_geometry(layout, rs, &g);
+  if (st != TOPKV_OK) return st;
+  const int F = (int)layout->kv_factor, R = batch->num_requests, maxp = batch->max_pages_per_req;
+  if (workspace_bytes < 8 * crc_workspace_words(g, R, maxp, F)) return TOPKV_ERR_CAPACITY;
+  if (R == 0) return TOPKV_OK;
+  const CrcWorkspace w = crc_carve(d_workspace, g.RB, maxp, R);
+  const int64_t total = (int64_t)g.RB + maxp + 1 + 2 * (int64_t)R + (int64_t)R * F;
+  const unsigned blocks = (unsigned)std::min<int64_t>((total + 255) / 256, 1024);
+  topkv_crc_begin_kernel<<<blocks, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+      w, g, batch->seq_lens, R, maxp, (int)layout->page_tokens, rs.row_bytes, F, d_crc_state);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  return TOPKV_OK;
+}
+
+int topkv_pack_layer_crc(int layer, const void* src_pool, const topkv_layout* layout,
+                         const topkv_batch* batch, void* d_wire, int64_t wire_capacity_bytes,
+                         uint64_t* d_crc_state, void* d_workspace, int64_t workspace_bytes,
+                         topkv_stream_t stream) {
+  return crc_copy<true>(layer, src_pool, layout, batch, d_wire, wire_capacity_bytes, d_crc_state,
+                        d_workspace, workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int topkv_unpack_layer_crc(int layer, void* dst_pool, const topkv_layout* layout,
+                           const topkv_batch* batch, const void* d_wire, int64_t wire_bytes,
+                           uint64_t* d_crc_state, void* d_workspace, int64_t workspace_bytes,
+                           topkv_stream_t stream) {
+  return crc_copy<false>(layer, dst_pool, layout, batch, d_wire, wire_bytes, d_crc_state,
+                         d_workspace, workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int topkv_crc_finish(const topkv_layout* layout, const topkv_batch* batch,
+                     const uint64_t* d_crc_state, uint64_t* d_crc_out, topkv_stream_t stream) {
+  if (layout == nullptr || layout->struct_size != sizeof(topkv_layout) || batch == nullptr ||
+      batch->struct_size != sizeof(topkv_batch) || d_crc_state == nullptr || d_crc_out == nullptr ||
+      batch->num_requests < 0)
+    return TOPKV_ERR_INVALID_ARG;
+  const int n = batch->num_requests * (int)layout->kv_factor;
+  if (n == 0) return TOPKV_OK;
+  topkv_crc_finish_kernel<<<(n + 255) / 256, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+      d_crc_state, n, d_crc_out);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   g_launches.fetch_add(1, std::memory_order_relaxed);

@@ -2,7 +2,11 @@
 // (Eq. 2, Eq. 3), the host-side batch validator and diagnostics. No CUDA calls here.
 #include "topkv.h"
 
+#include <chrono>
 #include <cstdint>
+#include <cstring>
+#include <mutex>
+#include <thread>
 #include <vector>
 
 namespace {
@@ -96,6 +100,73 @@ int topkv_validate_batch_host(const topkv_layout* lo, int32_t R, int32_t maxp,
   return TOPKV_OK;
 }
 
+// ---- CRC-64 (host), header, retry --------------------------------------------------------------
+namespace {
+uint64_t g_crc_table[256];
+std::once_flag g_crc_once;
+void build_crc_table() {
+  const uint64_t poly = 0xD800000000000000ull;  // x^64 + x^4 + x^3 + x + 1, reflected
+  for (int b = 0; b < 256; ++b) {
+    uint64_t v = (uint64_t)b;
+    for (int k = 0; k < 8; ++k) v = (v & 1) ? (v >> 1) ^ poly : (v >> 1);
+    g_crc_table[b] = v;
+  }
+}
+}  // namespace
+
+uint64_t topkv_crc64(const void* h_data, int64_t nbytes) {
+  std::call_once(g_crc_once, build_crc_table);
+  const uint8_t* p = static_cast<const uint8_t*>(h_data);
+  uint64_t crc = ~0ull;
+  for (int64_t i = 0; i < nbytes; ++i) crc = g_crc_table[(crc ^ p[i]) & 0xff] ^ (crc >> 8);
+  return ~crc;
+}
+
+int topkv_header_fill(topkv_wire_header* h, uint64_t request_id, uint64_t model_id,
+                      const topkv_layout* lo, int64_t seq_len, uint64_t crc_k, uint64_t crc_v) {
+  if (h == nullptr || !layout_header_ok(lo) || seq_len < 0 || seq_len > 0xffffffffll)
+    return TOPKV_ERR_INVALID_ARG;
+  static_assert(sizeof(topkv_wire_header) == 128, "the header is 128 bytes");
+  std::memset(h, 0, sizeof(*h));
+  std::memcpy(h->magic, "KVCACHE1", 8);
+  h->request_id = request_id;
+  h->model_id = model_id;
+  h->seq_len = (uint32_t)seq_len;
+  h->num_layers = lo->num_layers;
+  h->num_kv_heads = lo->num_kv_heads;
+  h->head_dim = lo->head_dim;
+  h->elem_bytes = lo->elem_bytes;
+  h->kv_factor = lo->kv_factor;
+  const uint64_t plane = (uint64_t)lo->num_layers * (uint64_t)seq_len * lo->num_kv_heads *
+                         lo->head_dim * lo->elem_bytes;
+  h->k_bytes = plane;
+  h->v_bytes = lo->kv_factor == 2 ? plane : 0;
+  h->crc_k = crc_k;
+  h->crc_v = lo->kv_factor == 2 ? crc_v : 0;
+  return TOPKV_OK;
+}
+
+int topkv_header_check(const topkv_wire_header* h, const topkv_layout* lo, int64_t seq_len,
+                       uint64_t crc_k, uint64_t crc_v) {
+  if (h == nullptr || !layout_header_ok(lo) || seq_len < 0) return TOPKV_ERR_INVALID_ARG;
+  topkv_wire_header want;
+  const int st = topkv_header_fill(&want, h->request_id, h->model_id, lo, seq_len, crc_k, crc_v);
+  if (st != TOPKV_OK) return st;
+  return std::memcmp(&want, h, sizeof(want)) == 0 ? TOPKV_OK : TOPKV_ERR_CHECKSUM;
+}
+
+int topkv_retry(int (*attempt)(void* ctx), void* ctx, int retries, int backoff_ms) {
+  if (attempt == nullptr || retries < 0 || backoff_ms < 0) return TOPKV_ERR_INVALID_ARG;
+  int status = attempt(ctx);
+  int64_t wait_ms = backoff_ms;
+  for (int k = 0; k < retries && status != TOPKV_OK; ++k) {
+    std::this_thread::sleep_for(std::chrono::milliseconds(wait_ms));
+    wait_ms *= 2;
+    status = attempt(ctx);
+  }
+  return status;
+}
+
 const char* topkv_strerror(int status) {
   switch (status) {
     case TOPKV_OK: return "ok";
@@ -105,6 +176,7 @@ const char* topkv_strerror(int status) {
     case TOPKV_ERR_CAPACITY: return "buffer too small for this layer's wire slab";
     case TOPKV_ERR_UNSUPPORTED_LAYOUT: return "unsupported or inconsistent layout descriptor";
     case TOPKV_ERR_CUDA: return "CUDA call failed (see topkv_last_cuda_error)";
+    case TOPKV_ERR_CHECKSUM: return "header or CRC-64 mismatch";
     default: return "unknown status";
   }
 }

@@ -171,6 +171,53 @@ def test_repage_argument_validation_without_gpu():
         assert RP(0, src, lo_s, b, dst, p32, _batch(maxp=8)) == tk.TOPKV_ERR_CUDA
 
 
+def test_host_crc64_header_and_retry():
+    import time
+    import oracle
+    rng = np.random.default_rng(5)
+    assert tk.topkv_crc64(b"123456789") == 0xB90956C775A41001        # CRC-64/GO-ISO check value
+    assert tk.topkv_crc64(b"") == 0
+    for n in (1, 7, 8, 9, 1000, 65537):
+        data = rng.integers(0, 256, n, dtype=np.uint8)
+        assert tk.topkv_crc64(data) == oracle.crc64(data), n
+    # header: byte-identical to the oracle's reading of the 128-byte layout
+    assert ctypes.sizeof(tk.topkv_wire_header) == 128
+    lo = tk.make_layout(80, 2, 8, 128, 2, 16, 1)
+    h = tk.topkv_wire_header()
+    assert tk.topkv_header_fill(h, 7, 0xABCDEF, lo, 4096, 0x1122334455667788, 0x99AABBCCDDEEFF00) == 0
+    g = oracle.Geom(L=80, F=2, h_kv=8, d_h=128, b_p=2, P=16, num_pages=1)
+    assert bytes(h) == oracle.build_header(7, 0xABCDEF, 4096, g, 0x1122334455667788, 0x99AABBCCDDEEFF00)
+    assert h.k_bytes + h.v_bytes == tk.topkv_kv_bytes(lo, 4096)       # Eq. 1
+    mla = tk.make_layout(61, 1, 1, 576, 2, 64, 1)
+    hm = tk.topkv_wire_header()
+    assert tk.topkv_header_fill(hm, 1, 2, mla, 4096, 5, 6) == 0
+    gm = oracle.Geom(L=61, F=1, h_kv=1, d_h=576, b_p=2, P=64, num_pages=1)
+    assert bytes(hm) == oracle.build_header(1, 2, 4096, gm, 5, 6) and hm.crc_v == 0 and hm.v_bytes == 0
+    # check: equal -> OK; any differing field or checksum -> TOPKV_ERR_CHECKSUM
+    C = tk.topkv_header_check
+    assert C(h, lo, 4096, 0x1122334455667788, 0x99AABBCCDDEEFF00) == tk.TOPKV_OK
+    assert C(h, lo, 4096, 0x1122334455667789, 0x99AABBCCDDEEFF00) == tk.TOPKV_ERR_CHECKSUM
+    assert C(h, lo, 4095, 0x1122334455667788, 0x99AABBCCDDEEFF00) == tk.TOPKV_ERR_CHECKSUM
+    bad = tk.topkv_wire_header.from_buffer_copy(bytes(h)); bad.magic = b"KVCACHE2"
+    assert C(bad, lo, 4096, 0x1122334455667788, 0x99AABBCCDDEEFF00) == tk.TOPKV_ERR_CHECKSUM
+    # retry policy (§3.1: 2 retries, exponential backoff): fails twice, then succeeds
+    calls = []
+    def attempt():
+        calls.append(time.perf_counter())
+        return tk.TOPKV_OK if len(calls) == 3 else tk.TOPKV_ERR_CHECKSUM
+    assert tk.topkv_retry(attempt, retries=2, backoff_ms=20) == tk.TOPKV_OK
+    assert len(calls) == 3
+    assert calls[1] - calls[0] >= 0.019 and calls[2] - calls[1] >= 0.039   # 20 ms, then 40 ms
+    calls.clear()
+    assert tk.topkv_retry(lambda: (calls.append(0), tk.TOPKV_ERR_CHECKSUM)[1], 2, 1) \
+        == tk.TOPKV_ERR_CHECKSUM and len(calls) == 3                     # gives up after 1 + 2
+    # workspace sizing and unsupported shapes
+    assert tk.topkv_crc_workspace_bytes(lo, 8, 256) == 8 * (32 + 257 + 16 + 8 * 256 * 2)
+    assert tk.topkv_crc_workspace_bytes(mla, 32, 128) == 8 * (128 + 129 + 64 + 32 * 128)
+    big = tk.make_layout(2, 2, 8, 128, 2, 512, 4)                    # 2 * 512 * 2 runs > 1024 threads
+    assert tk.topkv_crc_workspace_bytes(big, 1, 1) == tk.TOPKV_ERR_UNSUPPORTED_LAYOUT
+
+
 def test_empty_batches_launch_nothing():
     lo = _gqa(wire_layer_stride=0)
     before = tk.topkv_kernel_launch_count()

@@ -465,6 +465,128 @@ def test_windowed_layer_bench_shape(dev):
     torch.cuda.empty_cache()
 
 
+# -------------------------------------------------------------------- header + CRC-64 (§3.4)
+
+def _crc_run(dev, g, sl, bt_s, bt_d, src_h, dst_h, corrupt=None):
+    """Sender: pack every layer with checksums. Receiver: unpack with checksums from the
+    (optionally corrupted) wire. Returns wire, destination pool and both checksum arrays."""
+    lo = _layout_from_geom(g)
+    R, F = len(sl), g.F
+    T = int(sl.sum())
+    src, dst = torch.from_numpy(src_h).to(dev), torch.from_numpy(dst_h.copy()).to(dev)
+    wire = torch.zeros(max(g.L * g.W_layer, 16), dtype=torch.uint8, device=dev)
+    d_sl = torch.from_numpy(sl).to(dev)
+    d_bs, d_bd = torch.from_numpy(bt_s).to(dev), torch.from_numpy(bt_d).to(dev)
+    cu = torch.zeros(R + 1, dtype=torch.int64, device=dev)
+    tk.check(tk.topkv_build_plan(tk.make_batch(d_bs, d_sl), cu))
+    bs, bd = tk.make_batch(d_bs, d_sl, T, cu), tk.make_batch(d_bd, d_sl, T, cu)
+    nws = tk.topkv_crc_workspace_bytes(lo, R, bt_s.shape[1])
+    assert nws > 0
+    out = []
+    for side, (pool, batch, fn) in enumerate(((src, bs, tk.topkv_pack_layer_crc),
+                                              (dst, bd, tk.topkv_unpack_layer_crc))):
+        ws = torch.zeros(nws, dtype=torch.uint8, device=dev)
+        state = torch.zeros(R * F, dtype=torch.int64, device=dev)
+        crc = torch.zeros(R * F, dtype=torch.int64, device=dev)
+        tk.check(tk.topkv_crc_begin(lo, batch, state, ws, nws))
+        for layer in range(g.L):
+            tk.check(fn(layer, pool, lo, batch, wire, wire.numel(), state, ws, nws))
+        tk.check(tk.topkv_crc_finish(lo, batch, state, crc))
+        torch.cuda.synchronize()
+        out.append(crc.cpu().numpy().view(np.uint64).reshape(R, F))
+        if side == 0 and corrupt is not None:
+            wire[corrupt] ^= 0x10                      # one flipped bit on the way
+    return wire.cpu().numpy(), dst.cpu().numpy(), out[0], out[1]
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_crc_fused_pack_unpack(dev, seed, variant):
+    if variant == 1:
+        pytest.skip("the checksumming copy has one kernel family")
+    rng = np.random.default_rng(500 + seed)
+    F = int(rng.integers(1, 3))
+    H, D = [(8, 128), (1, 576), (1, 128), (2, 8), (4, 64), (8, 256)][seed % 6]
+    P = int(rng.choice([1, 4, 16]))
+    R = int(rng.integers(1, 5))
+    sl = rng.integers(0, 4 * P + 2, size=R).astype(np.int32)
+    if seed % 4 == 1:
+        sl[rng.integers(0, R)] = 0
+    pages = (sl + P - 1) // P
+    maxp = max(int(pages.max()), 1) + 1
+    npages = int(pages.sum()) + 2
+    g = Geom(L=3, F=F, h_kv=H, d_h=D, b_p=2, P=P, num_pages=npages,
+             wire_order=int(rng.integers(0, 2)))
+    if seed % 3 == 2:                                  # plane-major pool with padded tokens
+        g.S_tok = H * D * 2 + 32
+        g.S_page = P * g.S_tok
+        g.S_kv = npages * g.S_page
+        g.S_layer = F * g.S_kv
+    T = int(sl.sum())
+    g.W_layer = g.wire_layer_bytes(T)
+    bt_s = np.full((R, maxp), -1, dtype=np.int32)
+    bt_d = np.full((R, maxp), -1, dtype=np.int32)
+    ps, pd, pos = rng.permutation(npages), rng.permutation(npages), 0
+    for r in range(R):
+        bt_s[r, :pages[r]] = ps[pos:pos + pages[r]]
+        bt_d[r, :pages[r]] = pd[pos:pos + pages[r]]
+        pos += pages[r]
+    src_h = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
+    dst_h = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
+    wire, dst, crc_tx, crc_rx = _crc_run(dev, g, sl, bt_s, bt_d, src_h, dst_h)
+    want_wire = np.zeros(max(g.L * g.W_layer, 16), dtype=np.uint8)
+    want_dst = dst_h.copy()
+    for layer in range(g.L):
+        oracle.pack(g, layer, src_h, bt_s, sl, wire=want_wire)
+        oracle.unpack(g, layer, want_dst, bt_d, sl, want_wire)
+    assert np.array_equal(wire, want_wire) and np.array_equal(dst, want_dst)
+    for r in range(R):
+        for c in range(F):
+            want = oracle.kv_plane_crc(g, src_h, bt_s, sl, r, c)
+            assert int(crc_tx[r, c]) == want, (r, c, hex(int(crc_tx[r, c])), hex(want))
+            assert int(crc_rx[r, c]) == want
+
+
+def test_crc_cfg1_header_round_trip_and_corruption(dev, variant):
+    """cfg1 end to end: the sender's headers verify on the receiver; one flipped wire bit makes
+    exactly the affected request fail with TOPKV_ERR_CHECKSUM, and the retry policy of §3.1
+    (re-send, then verify again) recovers."""
+    if variant == 1:
+        pytest.skip("the checksumming copy has one kernel family")
+    b = wl.make_batch(wl.CFG1)
+    s = b.spec
+    g = _geom(s, b.num_pool_pages, s.L, 0, b.total_tokens * s.tok_bytes)
+    src_h = wl.fill_numpy(g.pool_bytes(), b.seeds["data"])
+    dst_h = wl.fill_numpy(g.pool_bytes(), b.seeds["dst_fill"])
+    lo = _layout_from_geom(g)
+    _, _, tx, rx = _crc_run(dev, g, b.seq_lens, b.src_block_table, b.dst_block_table, src_h, dst_h)
+    headers = []
+    for r in range(s.R):
+        assert int(tx[r, 0]) == oracle.kv_plane_crc(g, src_h, b.src_block_table, b.seq_lens, r, 0)
+        assert int(tx[r, 1]) == oracle.kv_plane_crc(g, src_h, b.src_block_table, b.seq_lens, r, 1)
+        h = tk.topkv_wire_header()
+        tk.check(tk.topkv_header_fill(h, 1000 + r, 42, lo, int(b.seq_lens[r]), int(tx[r, 0]), int(tx[r, 1])))
+        headers.append(h)
+        assert tk.topkv_header_check(h, lo, int(b.seq_lens[r]), int(rx[r, 0]), int(rx[r, 1])) == 0
+    # flip one bit inside request 2's V row of token 5, layer 1
+    cu = np.concatenate([[0], np.cumsum(b.seq_lens)])
+    off = 1 * g.W_layer + ((int(cu[2]) + 5) * 2 + 1) * g.row_bytes + 77
+    attempts = []
+
+    def transfer():
+        bad = off if not attempts else None           # the first attempt is corrupted in flight
+        attempts.append(1)
+        _, _, _, rx2 = _crc_run(dev, g, b.seq_lens, b.src_block_table, b.dst_block_table, src_h,
+                                dst_h, corrupt=bad)
+        status = [tk.topkv_header_check(headers[r], lo, int(b.seq_lens[r]), int(rx2[r, 0]),
+                                        int(rx2[r, 1])) for r in range(s.R)]
+        if len(attempts) == 1:
+            assert status == [0, 0, tk.TOPKV_ERR_CHECKSUM, 0]
+        return min(status)
+
+    assert tk.topkv_retry(transfer, retries=2, backoff_ms=1) == tk.TOPKV_OK
+    assert len(attempts) == 2
+
+
 # -------------------------------------------------------------------- direct re-paging
 
 def _repage_case(seed):
