@@ -211,29 +211,28 @@ int topkv_header_check(const topkv_wire_header* header, const topkv_layout* layo
 uint64_t topkv_crc64(const void* h_data, int64_t nbytes);
 
 /* Device-side checksumming, fused into pack / unpack. Usage, per batch:
- *   topkv_crc_begin(...)                      once: tables + running states (all on `stream`)
- *   topkv_pack_layer_crc(l, ...)              for l = 0 .. L-1 IN ORDER (or unpack on the receiver)
- *   topkv_crc_finish(...)                     d_crc_out[r*F + c] = checksum of request r, plane c
- * d_crc_state: DEVICE uint64 [R*F]; d_workspace: DEVICE scratch of at least
- * topkv_crc_workspace_bytes(...) bytes, 16-byte aligned, owned by the caller and reserved for
- * this batch between begin and finish. Requirements: heads contiguous in the pool,
- * batch->cu_seq_lens given, window_tokens 0, kv_factor * page_tokens * (runs per row) <= 1024
- * (else TOPKV_ERR_UNSUPPORTED_LAYOUT). TOPKV_FLAG_OVERLAP_PREVIOUS is ignored by these calls.
- * The copy itself is identical to topkv_pack_layer / topkv_unpack_layer. */
+ *   topkv_crc_begin(...)                 once: constant tables and counters (on `stream`)
+ *   topkv_pack_layer_crc(l, ...)         every layer l of the layout exactly once, in any order
+ *                                        (topkv_unpack_layer_crc on the receiving side)
+ *   topkv_crc_finish(...)                d_crc_out[r*F + c] = checksum of request r, plane c
+ * d_workspace: DEVICE scratch of at least topkv_crc_workspace_bytes(...) bytes, 16-byte
+ * aligned, owned by the caller and reserved for this batch from begin to finish (it holds the
+ * per-layer remainders). d_crc_out: DEVICE uint64 [R*F]. Requirements: heads contiguous in the
+ * pool, batch->cu_seq_lens given, window_tokens 0, kv_factor * page_tokens * (runs per row)
+ * <= 1024 (else TOPKV_ERR_UNSUPPORTED_LAYOUT). TOPKV_FLAG_OVERLAP_PREVIOUS may be set as for
+ * the plain calls. The copy itself is identical to topkv_pack_layer / topkv_unpack_layer. */
 int64_t topkv_crc_workspace_bytes(const topkv_layout* layout, int32_t num_requests,
                                   int32_t max_pages_per_req);
-int topkv_crc_begin(const topkv_layout* layout, const topkv_batch* batch, uint64_t* d_crc_state,
-                    void* d_workspace, int64_t workspace_bytes, topkv_stream_t stream);
+int topkv_crc_begin(const topkv_layout* layout, const topkv_batch* batch, void* d_workspace,
+                    int64_t workspace_bytes, topkv_stream_t stream);
 int topkv_pack_layer_crc(int layer, const void* src_pool, const topkv_layout* layout,
                          const topkv_batch* batch, void* d_wire, int64_t wire_capacity_bytes,
-                         uint64_t* d_crc_state, void* d_workspace, int64_t workspace_bytes,
-                         topkv_stream_t stream);
+                         void* d_workspace, int64_t workspace_bytes, topkv_stream_t stream);
 int topkv_unpack_layer_crc(int layer, void* dst_pool, const topkv_layout* layout,
                            const topkv_batch* batch, const void* d_wire, int64_t wire_bytes,
-                           uint64_t* d_crc_state, void* d_workspace, int64_t workspace_bytes,
-                           topkv_stream_t stream);
-int topkv_crc_finish(const topkv_layout* layout, const topkv_batch* batch,
-                     const uint64_t* d_crc_state, uint64_t* d_crc_out, topkv_stream_t stream);
+                           void* d_workspace, int64_t workspace_bytes, topkv_stream_t stream);
+int topkv_crc_finish(const topkv_layout* layout, const topkv_batch* batch, void* d_workspace,
+                     int64_t workspace_bytes, uint64_t* d_crc_out, topkv_stream_t stream);
 
 /* Host-side retry policy of the transfer orchestrator (§3.1: 2 retries, 100 ms exponential
  * backoff): calls attempt(ctx) until it returns TOPKV_OK, at most 1 + retries times, sleeping

@@ -120,12 +120,12 @@ def lib() -> ctypes.CDLL:
         L.topkv_crc64.restype = u64
         L.topkv_crc_workspace_bytes.argtypes = [lp, c_int32, c_int32]
         L.topkv_crc_workspace_bytes.restype = c_int64
-        L.topkv_crc_begin.argtypes = [lp, bp, c_void_p, c_void_p, c_int64, c_void_p]
+        L.topkv_crc_begin.argtypes = [lp, bp, c_void_p, c_int64, c_void_p]
         L.topkv_pack_layer_crc.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p,
-                                           c_void_p, c_int64, c_void_p]
+                                           c_int64, c_void_p]
         L.topkv_unpack_layer_crc.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p,
-                                             c_void_p, c_int64, c_void_p]
-        L.topkv_crc_finish.argtypes = [lp, bp, c_void_p, c_void_p, c_void_p]
+                                             c_int64, c_void_p]
+        L.topkv_crc_finish.argtypes = [lp, bp, c_void_p, c_int64, c_void_p, c_void_p]
         L.topkv_retry.argtypes = [RETRY_ATTEMPT, c_void_p, c_int, c_int]
         L.topkv_repage_layer.argtypes = [c_int, c_void_p, lp, bp, c_void_p, lp, bp, c_void_p]
         L.topkv_pack_layer_to_host_noalloc.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64,
@@ -283,30 +283,28 @@ def topkv_crc_workspace_bytes(layout, num_requests, max_pages_per_req):
     return lib().topkv_crc_workspace_bytes(ctypes.byref(layout), num_requests, max_pages_per_req)
 
 
-def topkv_crc_begin(layout, batch, d_crc_state, d_workspace, workspace_bytes, stream=None):
-    return lib().topkv_crc_begin(ctypes.byref(layout), ctypes.byref(batch), _ptr(d_crc_state),
-                                 _ptr(d_workspace), workspace_bytes, _stream(stream))
+def topkv_crc_begin(layout, batch, d_workspace, workspace_bytes, stream=None):
+    return lib().topkv_crc_begin(ctypes.byref(layout), ctypes.byref(batch), _ptr(d_workspace),
+                                 workspace_bytes, _stream(stream))
 
 
-def topkv_pack_layer_crc(layer, src_pool, layout, batch, d_wire, wire_capacity_bytes, d_crc_state,
-                         d_workspace, workspace_bytes, stream=None):
+def topkv_pack_layer_crc(layer, src_pool, layout, batch, d_wire, wire_capacity_bytes, d_workspace,
+                         workspace_bytes, stream=None):
     return lib().topkv_pack_layer_crc(layer, _ptr(src_pool), ctypes.byref(layout),
                                       ctypes.byref(batch), _ptr(d_wire), wire_capacity_bytes,
-                                      _ptr(d_crc_state), _ptr(d_workspace), workspace_bytes,
-                                      _stream(stream))
+                                      _ptr(d_workspace), workspace_bytes, _stream(stream))
 
 
-def topkv_unpack_layer_crc(layer, dst_pool, layout, batch, d_wire, wire_bytes, d_crc_state,
-                           d_workspace, workspace_bytes, stream=None):
+def topkv_unpack_layer_crc(layer, dst_pool, layout, batch, d_wire, wire_bytes, d_workspace,
+                           workspace_bytes, stream=None):
     return lib().topkv_unpack_layer_crc(layer, _ptr(dst_pool), ctypes.byref(layout),
                                         ctypes.byref(batch), _ptr(d_wire), wire_bytes,
-                                        _ptr(d_crc_state), _ptr(d_workspace), workspace_bytes,
-                                        _stream(stream))
+                                        _ptr(d_workspace), workspace_bytes, _stream(stream))
 
 
-def topkv_crc_finish(layout, batch, d_crc_state, d_crc_out, stream=None):
-    return lib().topkv_crc_finish(ctypes.byref(layout), ctypes.byref(batch), _ptr(d_crc_state),
-                                  _ptr(d_crc_out), _stream(stream))
+def topkv_crc_finish(layout, batch, d_workspace, workspace_bytes, d_crc_out, stream=None):
+    return lib().topkv_crc_finish(ctypes.byref(layout), ctypes.byref(batch), _ptr(d_workspace),
+                                  workspace_bytes, _ptr(d_crc_out), _stream(stream))
 
 
 def topkv_retry(attempt, retries=2, backoff_ms=100):

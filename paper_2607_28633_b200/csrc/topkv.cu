@@ -584,40 +584,49 @@ int crc_geometry(const topkv_layout* lo, const Resolved& rs, CrcGeom* g) {
   return TOPKV_OK;
 }
 
-int64_t crc_workspace_words(const CrcGeom& g, int R, int maxp, int F) {
-  return (int64_t)g.RB + (maxp + 1) + 2 * (int64_t)R + (int64_t)R * maxp * F;
-}
-
 template <bool PACK>
 int crc_copy(int layer, const void* pool, const topkv_layout* lo, const topkv_batch* b,
-             const void* wire, int64_t cap, uint64_t* state, void* ws, int64_t ws_bytes,
-             cudaStream_t stream) {
+             const void* wire, int64_t cap, void* ws, int64_t ws_bytes, cudaStream_t stream) {
   CrcCopyParams cp;
   Resolved rs;
   int64_t n_layer;
   int st = prepare(layer, pool, lo, b, wire, cap, lo ? lo->wire_layer_stride : 0, &cp.k, &rs, &n_layer);
   if (st != TOPKV_OK) return st;
-  if (state == nullptr || ws == nullptr || !mult16p(ws)) return TOPKV_ERR_INVALID_ARG;
+  if (ws == nullptr || !mult16p(ws)) return TOPKV_ERR_INVALID_ARG;
   if (b->cu_seq_lens == nullptr || b->window_tokens != 0) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
   st = crc_geometry(lo, rs, &cp.g);
   if (st != TOPKV_OK) return st;
   const int F = (int)lo->kv_factor, R = b->num_requests, maxp = b->max_pages_per_req;
-  if (ws_bytes < 8 * crc_workspace_words(cp.g, R, maxp, F)) return TOPKV_ERR_CAPACITY;
+  const int L = (int)lo->num_layers;
+  if (ws_bytes < 8 * crc_workspace_words(cp.g.RB, L, R, maxp, F)) return TOPKV_ERR_CAPACITY;
   if (R == 0 || maxp == 0) return TOPKV_OK;
-  const CrcWorkspace w = crc_carve(ws, cp.g.RB, maxp, R);
-  cp.c_run = w.c_run;
-  cp.page_rem = w.page_rem;
-  cp.k.overlap = 0;  // the page remainders are shared with the fold kernel of the previous layer
-  const dim3 grid((unsigned)((int64_t)R * maxp)), block((unsigned)((F * cp.g.RB + 31) / 32 * 32));
-  if (F == 1) launch_pdl(topkv_crc_copy_kernel<1, PACK>, grid, block, 0, stream, cp);
-  else launch_pdl(topkv_crc_copy_kernel<2, PACK>, grid, block, 0, stream, cp);
-  cudaError_t e = cudaGetLastError();
+  cp.w = crc_carve(ws, cp.g.RB, L, R, maxp, F);
+  cp.layer = layer;
+  cp.F = F;
+  const int threads = (F * cp.g.RB + 31) / 32 * 32;
+  const dim3 grid((unsigned)((int64_t)R * maxp)), block((unsigned)threads);
+  const size_t smem = (size_t)(threads / 32) * kCrcTileBytes;
+  // 32-byte pieces when every address the kernel can form is 32-byte aligned
+  const bool wide = ((reinterpret_cast<uintptr_t>(cp.k.pool) | reinterpret_cast<uintptr_t>(cp.k.wire) |
+                      (uintptr_t)cp.k.S_page | (uintptr_t)cp.k.S_kv | (uintptr_t)cp.k.S_tok |
+                      (uintptr_t)cp.g.run_bytes) & 31) == 0;
+  cudaError_t e = cudaSuccess;
+  auto go = [&](auto kernel) {
+    if (smem > 48 * 1024)
+      e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32 * kCrcTileBytes);
+    if (e == cudaSuccess) e = launch_pdl(kernel, grid, block, smem, stream, cp);
+  };
+  if (threads <= 128) {
+    if (wide) { if (F == 1) go(topkv_crc_copy_kernel<1, PACK, 32, 128>); else go(topkv_crc_copy_kernel<2, PACK, 32, 128>); }
+    else { if (F == 1) go(topkv_crc_copy_kernel<1, PACK, 16, 128>); else go(topkv_crc_copy_kernel<2, PACK, 16, 128>); }
+  } else {
+    if (wide) { if (F == 1) go(topkv_crc_copy_kernel<1, PACK, 32, 1024>); else go(topkv_crc_copy_kernel<2, PACK, 32, 1024>); }
+    else { if (F == 1) go(topkv_crc_copy_kernel<1, PACK, 16, 1024>); else go(topkv_crc_copy_kernel<2, PACK, 16, 1024>); }
+  }
   if (e != cudaSuccess) return cuda_fail(e);
-  topkv_crc_fold_kernel<<<(unsigned)(R * F), 256, 0, stream>>>(w, b->seq_lens, maxp, (int)lo->page_tokens,
-                                                              F, state);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
-  g_launches.fetch_add(2, std::memory_order_relaxed);
+  g_launches.fetch_add(1, std::memory_order_relaxed);
   return TOPKV_OK;
 }
 
@@ -836,30 +845,31 @@ int64_t topkv_crc_workspace_bytes(const topkv_layout* layout, int32_t num_reques
   CrcGeom g;
   st = crc_geometry(layout, rs, &g);
   if (st != TOPKV_OK) return st;
-  return 8 * crc_workspace_words(g, num_requests, max_pages_per_req, (int)layout->kv_factor);
+  return 8 * crc_workspace_words(g.RB, (int)layout->num_layers, num_requests, max_pages_per_req,
+                                 (int)layout->kv_factor);
 }
 
-int topkv_crc_begin(const topkv_layout* layout, const topkv_batch* batch, uint64_t* d_crc_state,
-                    void* d_workspace, int64_t workspace_bytes, topkv_stream_t stream) {
+int topkv_crc_begin(const topkv_layout* layout, const topkv_batch* batch, void* d_workspace,
+                    int64_t workspace_bytes, topkv_stream_t stream) {
   Resolved rs;
   int st = check_layout(layout, &rs);
   if (st != TOPKV_OK) return st;
   st = check_batch(layout, batch);
   if (st != TOPKV_OK) return st;
-  if (d_crc_state == nullptr || d_workspace == nullptr || !mult16p(d_workspace))
-    return TOPKV_ERR_INVALID_ARG;
+  if (d_workspace == nullptr || !mult16p(d_workspace)) return TOPKV_ERR_INVALID_ARG;
   if (batch->window_tokens != 0) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
   CrcGeom g;
   st = crc_geometry(layout, rs, &g);
   if (st != TOPKV_OK) return st;
   const int F = (int)layout->kv_factor, R = batch->num_requests, maxp = batch->max_pages_per_req;
-  if (workspace_bytes < 8 * crc_workspace_words(g, R, maxp, F)) return TOPKV_ERR_CAPACITY;
+  const int L = (int)layout->num_layers;
+  if (workspace_bytes < 8 * crc_workspace_words(g.RB, L, R, maxp, F)) return TOPKV_ERR_CAPACITY;
   if (R == 0) return TOPKV_OK;
-  const CrcWorkspace w = crc_carve(d_workspace, g.RB, maxp, R);
-  const int64_t total = (int64_t)g.RB + maxp + 1 + 2 * (int64_t)R + (int64_t)R * F;
+  const CrcWorkspace w = crc_carve(d_workspace, g.RB, L, R, maxp, F);
+  const int64_t total = (int64_t)g.RB + maxp + 1 + 2 * (int64_t)R + (int64_t)L * R;
   const unsigned blocks = (unsigned)std::min<int64_t>((total + 255) / 256, 1024);
   topkv_crc_begin_kernel<<<blocks, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
-      w, g, batch->seq_lens, R, maxp, (int)layout->page_tokens, rs.row_bytes, F, d_crc_state);
+      w, g, batch->seq_lens, L, R, maxp, (int)layout->page_tokens, rs.row_bytes);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -868,30 +878,37 @@ int topkv_crc_begin(const topkv_layout* layout, const topkv_batch* batch, uint64
 
 int topkv_pack_layer_crc(int layer, const void* src_pool, const topkv_layout* layout,
                          const topkv_batch* batch, void* d_wire, int64_t wire_capacity_bytes,
-                         uint64_t* d_crc_state, void* d_workspace, int64_t workspace_bytes,
-                         topkv_stream_t stream) {
-  return crc_copy<true>(layer, src_pool, layout, batch, d_wire, wire_capacity_bytes, d_crc_state,
-                        d_workspace, workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
+                         void* d_workspace, int64_t workspace_bytes, topkv_stream_t stream) {
+  return crc_copy<true>(layer, src_pool, layout, batch, d_wire, wire_capacity_bytes, d_workspace,
+                        workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
 }
 
 int topkv_unpack_layer_crc(int layer, void* dst_pool, const topkv_layout* layout,
                            const topkv_batch* batch, const void* d_wire, int64_t wire_bytes,
-                           uint64_t* d_crc_state, void* d_workspace, int64_t workspace_bytes,
-                           topkv_stream_t stream) {
-  return crc_copy<false>(layer, dst_pool, layout, batch, d_wire, wire_bytes, d_crc_state,
-                         d_workspace, workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
+                           void* d_workspace, int64_t workspace_bytes, topkv_stream_t stream) {
+  return crc_copy<false>(layer, dst_pool, layout, batch, d_wire, wire_bytes, d_workspace,
+                         workspace_bytes, reinterpret_cast<cudaStream_t>(stream));
 }
 
-int topkv_crc_finish(const topkv_layout* layout, const topkv_batch* batch,
-                     const uint64_t* d_crc_state, uint64_t* d_crc_out, topkv_stream_t stream) {
-  if (layout == nullptr || layout->struct_size != sizeof(topkv_layout) || batch == nullptr ||
-      batch->struct_size != sizeof(topkv_batch) || d_crc_state == nullptr || d_crc_out == nullptr ||
-      batch->num_requests < 0)
+int topkv_crc_finish(const topkv_layout* layout, const topkv_batch* batch, void* d_workspace,
+                     int64_t workspace_bytes, uint64_t* d_crc_out, topkv_stream_t stream) {
+  Resolved rs;
+  int st = check_layout(layout, &rs);
+  if (st != TOPKV_OK) return st;
+  st = check_batch(layout, batch);
+  if (st != TOPKV_OK) return st;
+  if (d_workspace == nullptr || !mult16p(d_workspace) || d_crc_out == nullptr)
     return TOPKV_ERR_INVALID_ARG;
-  const int n = batch->num_requests * (int)layout->kv_factor;
-  if (n == 0) return TOPKV_OK;
-  topkv_crc_finish_kernel<<<(n + 255) / 256, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
-      d_crc_state, n, d_crc_out);
+  CrcGeom g;
+  st = crc_geometry(layout, rs, &g);
+  if (st != TOPKV_OK) return st;
+  const int F = (int)layout->kv_factor, R = batch->num_requests, maxp = batch->max_pages_per_req;
+  const int L = (int)layout->num_layers;
+  if (workspace_bytes < 8 * crc_workspace_words(g.RB, L, R, maxp, F)) return TOPKV_ERR_CAPACITY;
+  if (R == 0) return TOPKV_OK;
+  const CrcWorkspace w = crc_carve(d_workspace, g.RB, L, R, maxp, F);
+  topkv_crc_finish_kernel<<<(R * F + 127) / 128, 128, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+      w, batch->seq_lens, L, R, F, d_crc_out);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   g_launches.fetch_add(1, std::memory_order_relaxed);

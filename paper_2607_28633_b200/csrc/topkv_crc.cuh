@@ -5,12 +5,13 @@
 // Everything is linear over GF(2). With rem(M) = M(x) * x^64 mod P (no initial value, no
 // inversion) and "||" concatenation:   rem(A || B) = rem(A) * x^(8|B|) + rem(B)   (mod P).
 // The tensor of one request and one plane, [layers][seq_len][kv_heads][head_dim], is cut
-// into runs (a fraction of a token row); every thread streams one run through its registers on
-// the way from source to destination and folds it into a 64-bit remainder, multiplies that by
+// into runs (a fraction of a token row); every thread owns one run: while the warp moves the
+// data from source to destination it folds its run into a 64-bit remainder, multiplies that by
 // x^(8 * bytes that follow the run inside its page), and the page's threads XOR their results.
-// A second, tiny kernel aligns the page remainders inside the request and chains the layers:
-//   state' = state * x^(8 * bytes of this layer's plane) + rem(layer's plane),  state_0 = ~0,
-// so that after the last layer the checksum is ~state.
+// The CTA that finishes the last page of a request aligns the page remainders inside the
+// request's plane and stores the layer's remainder; topkv_crc_finish chains the layers:
+//   state_0 = ~0,  state_l+1 = state_l * x^(8 * bytes of the plane in one layer) + rem_l,
+// and the checksum is ~state_L.
 //
 // Register convention (reflected): bit i of a 64-bit value is the coefficient of x^(63 - i);
 // multiplying by x is a right shift. A little-endian 64-bit load of eight message bytes is
@@ -34,13 +35,25 @@ __host__ __device__ __forceinline__ uint64_t gf_mulx(uint64_t v) {
   return (v >> 1) ^ ((v & 1) ? kCrcPoly : 0ull);
 }
 
-// v * x^64 mod P = v * (x^4 + x^3 + x + 1) mod P.
+// v * x^64 mod P. x^64 = x^4 + x^3 + x + 1 = (1 + x)(1 + x^3) (mod P), so two cheap steps:
+// u = v + v*x, then u + u*x^3, each reduced at once. Only the top byte of the generator is
+// populated, so every reduction touches the high 32-bit half only.
 __host__ __device__ __forceinline__ uint64_t gf_mulx64(uint64_t v) {
-  const uint64_t a = v ^ (v >> 1) ^ (v >> 3) ^ (v >> 4);
-  // the bits shifted out have degree >= 64: q = their quotient by x^64 (degree < 4, top bits),
-  // and q * x^64 = q * (x^4 + x^3 + x + 1) again, now without overflow
-  const uint64_t q = (v << 63) ^ (v << 61) ^ (v << 60);
-  return a ^ q ^ (q >> 1) ^ (q >> 3) ^ (q >> 4);
+  // u = v * (1 + x): the bit shifted out (degree 64) comes back as x^4 + x^3 + x + 1
+  const uint64_t u = v ^ (v >> 1) ^ ((0ull - (v & 1)) & kCrcPoly);
+  // u * (1 + x^3): three bits are shifted out, q = their polynomial (degree < 3, top bits);
+  // q * x^64 = q * (x^4 + x^3 + x + 1) has degree < 7 and needs no further reduction
+  const uint64_t q = u << 61;
+  return u ^ (u >> 3) ^ q ^ (q >> 1) ^ (q >> 3) ^ (q >> 4);
+}
+
+// v * x^256 mod P: x^256 = (x^64)^4 = (1 + x^4)(1 + x^12) (mod P; squaring is linear over GF(2)).
+// Same cost as gf_mulx64; it lets four interleaved Horner chains run side by side.
+__host__ __device__ __forceinline__ uint64_t gf_mulx256(uint64_t v) {
+  const uint64_t q1 = v << 60;  // the 4 bits shifted out by v * x^4, as a polynomial in the top bits
+  const uint64_t u = v ^ (v >> 4) ^ q1 ^ (q1 >> 1) ^ (q1 >> 3) ^ (q1 >> 4);
+  const uint64_t q2 = u << 52;  // the 12 bits shifted out by u * x^12
+  return u ^ (u >> 12) ^ q2 ^ (q2 >> 1) ^ (q2 >> 3) ^ (q2 >> 4);
 }
 
 // a * b mod P, Horner over the coefficients of a from the highest power down.
@@ -64,18 +77,23 @@ __host__ __device__ inline uint64_t gf_powx(uint64_t n) {
   return result;
 }
 
-// ---- workspace (device memory owned by the caller) ---------------------------------------------
-// [0]                 c_run  [max_runs]      x^(8 * run_bytes * m)
-// [max_runs]          c_page [max_pages + 1] x^(8 * P * row_bytes * k)
-// [.. + max_pages+1]  x_req  [R]             x^(8 * s_r * row_bytes)        (per batch)
-// [.. + R]            x_last [R]             x^(8 * v_last(r) * row_bytes)  (per batch)
-// [.. + R]            page_rem [R * maxp * F]
+// ---- workspace (device memory owned by the caller), in 8-byte words ------------------------------
+// c_run    [RB]            x^(8 * run_bytes * m)
+// c_page   [maxp + 1]      x^(8 * P * row_bytes * k)
+// x_req    [R]             x^(8 * s_r * row_bytes)        (per batch)
+// x_last   [R]             x^(8 * v_last(r) * row_bytes)  (per batch)
+// layer_rem[L * R * F]     remainder of request r, plane c, layer l (written by the last CTA
+//                          of that request and layer)
+// page_rem [L * R * maxp * F]  remainder of every page and plane, per layer
+// done     [L * R] (int32) pages of request r finished in layer l
 struct CrcWorkspace {
   uint64_t* c_run;
   uint64_t* c_page;
   uint64_t* x_req;
   uint64_t* x_last;
+  uint64_t* layer_rem;
   uint64_t* page_rem;
+  int32_t* done;
 };
 
 struct CrcGeom {
@@ -84,23 +102,30 @@ struct CrcGeom {
   int RB;         // runs per page and plane = P * rpr
 };
 
-__host__ __device__ inline CrcWorkspace crc_carve(void* base, int max_runs, int max_pages, int R) {
+__host__ __device__ inline int64_t crc_workspace_words(int RB, int L, int R, int maxp, int F) {
+  return (int64_t)RB + (maxp + 1) + 2 * (int64_t)R + (int64_t)L * R * F +
+         (int64_t)L * R * maxp * F + ((int64_t)L * R + 1) / 2;
+}
+
+__host__ __device__ inline CrcWorkspace crc_carve(void* base, int RB, int L, int R, int maxp, int F) {
   CrcWorkspace w;
   w.c_run = static_cast<uint64_t*>(base);
-  w.c_page = w.c_run + max_runs;
-  w.x_req = w.c_page + (max_pages + 1);
+  w.c_page = w.c_run + RB;
+  w.x_req = w.c_page + (maxp + 1);
   w.x_last = w.x_req + R;
-  w.page_rem = w.x_last + R;
+  w.layer_rem = w.x_last + R;
+  w.page_rem = w.layer_rem + (int64_t)L * R * F;
+  w.done = reinterpret_cast<int32_t*>(w.page_rem + (int64_t)L * R * maxp * F);
   return w;
 }
 
-// Builds the constant tables for this batch and sets every running state to ~0.
+// Builds the constant tables for this batch and clears the per-layer page counters.
 __global__ void __launch_bounds__(256)
-topkv_crc_begin_kernel(CrcWorkspace w, CrcGeom g, const int32_t* __restrict__ sl, int R, int maxp,
-                       int P, int64_t row_bytes, int F, uint64_t* __restrict__ state) {
+topkv_crc_begin_kernel(CrcWorkspace w, CrcGeom g, const int32_t* __restrict__ sl, int L, int R,
+                       int maxp, int P, int64_t row_bytes) {
   pdl_prologue(0);
   const int64_t n_run = g.RB, n_page = maxp + 1;
-  const int64_t total = n_run + n_page + 2 * (int64_t)R + (int64_t)R * F;
+  const int64_t total = n_run + n_page + 2 * (int64_t)R + (int64_t)L * R;
   for (int64_t k = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; k < total;
        k += (int64_t)gridDim.x * blockDim.x) {
     if (k < n_run) {
@@ -117,7 +142,7 @@ topkv_crc_begin_kernel(CrcWorkspace w, CrcGeom g, const int32_t* __restrict__ sl
       if (q & 1) w.x_last[r] = gf_powx(8ull * (uint64_t)v_last * row_bytes);
       else w.x_req[r] = gf_powx(8ull * (uint64_t)s * row_bytes);
     } else {
-      state[k - n_run - n_page - 2 * (int64_t)R] = ~0ull;
+      w.done[k - n_run - n_page - 2 * (int64_t)R] = 0;
     }
   }
 }
@@ -125,17 +150,57 @@ topkv_crc_begin_kernel(CrcWorkspace w, CrcGeom g, const int32_t* __restrict__ sl
 struct CrcCopyParams {
   KParams k;
   CrcGeom g;
-  const uint64_t* c_run;
-  uint64_t* page_rem;
+  CrcWorkspace w;
+  int layer;
+  int F;
 };
 
-// One CTA per (request, page column); one thread per run of one plane. F * RB threads work.
-template <int F, bool PACK>
-__global__ void __launch_bounds__(1024, 1) topkv_crc_copy_kernel(const CrcCopyParams cp) {
+constexpr int kCrcPitch = 144;          // bytes per run in the exchange tile: 128 + 16 of padding
+constexpr int kCrcTileBytes = 32 * kCrcPitch;  // one tile per warp
+
+template <int VEC>
+struct Piece;
+template <>
+struct Piece<16> {
+  uint4 a;
+  __device__ __forceinline__ void load(const uint8_t* p) { a = *reinterpret_cast<const uint4*>(p); }
+  __device__ __forceinline__ void store(uint8_t* p) const { *reinterpret_cast<uint4*>(p) = a; }
+  __device__ __forceinline__ void to_tile(uint8_t* p) const { *reinterpret_cast<uint4*>(p) = a; }
+};
+template <>
+struct Piece<32> {
+  uint4 a, b;
+  __device__ __forceinline__ void load(const uint8_t* p) {
+    asm volatile("ld.global.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w), "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w)
+                 : "l"(p));
+  }
+  __device__ __forceinline__ void store(uint8_t* p) const {
+    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(a.x), "r"(a.y),
+                 "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w)
+                 : "memory");
+  }
+  __device__ __forceinline__ void to_tile(uint8_t* p) const {
+    *reinterpret_cast<uint4*>(p) = a;
+    *reinterpret_cast<uint4*>(p + 16) = b;
+  }
+};
+
+// One CTA per (request, page column); one thread owns one run of one plane (F * RB threads
+// work). Global memory is accessed warp-coalesced: in every step the warp moves 128 bytes of
+// each of several of its runs, 128 / VEC lanes per run, straight from source to destination;
+// the same registers are also dropped into a padded shared-memory tile from which every lane
+// picks up the 128 bytes of its OWN run, in order, for the checksum. The next batch's loads are
+// issued before the current batch is folded, so that they are in flight during the ALU work.
+template <int F, bool PACK, int VEC, int MAXT>
+__global__ void __launch_bounds__(MAXT, 1) topkv_crc_copy_kernel(const CrcCopyParams cp) {
+  extern __shared__ __align__(16) uint8_t s_tiles[];
   __shared__ unsigned long long s_rem[2];
+  constexpr int kPieces = 128 / VEC;      // pieces of one run in a batch = steps per batch
+  constexpr int kRunsPerStep = 32 / kPieces;
   const KParams& p = cp.k;
   pdl_prologue(p.overlap);
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31;
   const int slot = blockIdx.x;
   const int r = slot / p.maxp;
   const int j = slot - r * p.maxp;
@@ -161,79 +226,143 @@ __global__ void __launch_bounds__(1024, 1) topkv_crc_copy_kernel(const CrcCopyPa
     const int c = tid / cp.g.RB;
     const int idx = tid - c * cp.g.RB;
     const int nruns = v * cp.g.rpr;
-    if (page_ok && fits && c < F && idx < nruns) {
+    const bool mine = page_ok && fits && c < F && idx < nruns;  // this lane owns a run
+    // source and destination of this lane's run (null when it owns none)
+    const uint8_t* src_run = nullptr;
+    uint8_t* dst_run = nullptr;
+    if (mine) {
       const int t = idx / cp.g.rpr;
       const int seg = idx - t * cp.g.rpr;
       uint8_t* a = p.pool + page * p.S_page + c * p.S_kv + (int64_t)t * p.S_tok +
                    (int64_t)seg * cp.g.run_bytes;
       const int64_t wrow = p.planar ? ((int64_t)c * T + n0 + t) : ((n0 + t) * F + c);
       uint8_t* b = p.wire + wrow * row + (int64_t)seg * cp.g.run_bytes;
-      const uint4* src = reinterpret_cast<const uint4*>(PACK ? a : b);
-      uint4* dst = reinterpret_cast<uint4*>(PACK ? b : a);
-      const int nvec = cp.g.run_bytes / 16;
-      uint64_t rem = 0;
-      constexpr int kBatch = 8;  // 128 bytes in flight per thread
-      for (int k0 = 0; k0 < nvec; k0 += kBatch) {
-        uint4 buf[kBatch];
+      src_run = PACK ? a : b;
+      dst_run = PACK ? b : a;
+    }
+    uint8_t* tile = s_tiles + (size_t)(tid >> 5) * kCrcTileBytes;
+    const int sub = lane / kPieces, piece = lane % kPieces;
+    uint64_t rem = 0;
+    if (__any_sync(0xffffffffu, mine)) {
+      // In step m this lane moves piece `piece` of the run owned by lane kRunsPerStep*m + sub.
+      const uint8_t* sp[kPieces];
+      uint8_t* dp[kPieces];
 #pragma unroll
-        for (int u = 0; u < kBatch; ++u)
-          if (k0 + u < nvec) buf[u] = src[k0 + u];
-#pragma unroll
-        for (int u = 0; u < kBatch; ++u)
-          if (k0 + u < nvec) {
-            dst[k0 + u] = buf[u];
-            const uint64_t w0 = (uint64_t)buf[u].x | ((uint64_t)buf[u].y << 32);
-            const uint64_t w1 = (uint64_t)buf[u].z | ((uint64_t)buf[u].w << 32);
-            rem = gf_mulx64(rem ^ w0);
-            rem = gf_mulx64(rem ^ w1);
-          }
+      for (int m = 0; m < kPieces; ++m) {
+        const int owner = kRunsPerStep * m + sub;
+        const uint64_t s0 = __shfl_sync(0xffffffffu, (uint64_t)src_run, owner);
+        const uint64_t d0 = __shfl_sync(0xffffffffu, (uint64_t)dst_run, owner);
+        sp[m] = s0 ? reinterpret_cast<const uint8_t*>(s0) + piece * VEC : nullptr;
+        dp[m] = reinterpret_cast<uint8_t*>(d0) + piece * VEC;
       }
+      uint8_t* my_tile_out = tile + sub * kCrcPitch + piece * VEC;  // + m * kRunsPerStep * pitch
+      const uint8_t* my_tile_in = tile + lane * kCrcPitch;
+      Piece<VEC> x[kPieces];
+      auto fetch = [&](int off) {
+        const int left = cp.g.run_bytes - off;  // bytes of every run still to move
+#pragma unroll
+        for (int m = 0; m < kPieces; ++m)
+          if (sp[m] != nullptr && piece * VEC < left) x[m].load(sp[m] + off);
+      };
+      fetch(0);
+      for (int off = 0; off < cp.g.run_bytes; off += 128) {
+        const int left = cp.g.run_bytes - off;
+#pragma unroll
+        for (int m = 0; m < kPieces; ++m)
+          if (sp[m] != nullptr && piece * VEC < left) {
+            x[m].store(dp[m] + off);
+            x[m].to_tile(my_tile_out + m * kRunsPerStep * kCrcPitch);
+          }
+        __syncwarp();
+        if (off + 128 < cp.g.run_bytes) fetch(off + 128);  // in flight while this batch is folded
+        if (mine) {
+          if (left >= 128) {
+            // 16 words w0..w15. Four independent chains, chain c over w_c, w_c+4, w_c+8, w_c+12
+            // with step x^256; the running remainder rides on w0. Then the chains are joined:
+            // rem = (((S0*x^64 + S1)*x^64 + S2)*x^64 + S3)*x^64.
+            uint64_t s0 = rem, s1 = 0, s2 = 0, s3 = 0;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const uint4 ya = *reinterpret_cast<const uint4*>(my_tile_in + k * 32);
+              const uint4 yb = *reinterpret_cast<const uint4*>(my_tile_in + k * 32 + 16);
+              s0 ^= (uint64_t)ya.x | ((uint64_t)ya.y << 32);
+              s1 ^= (uint64_t)ya.z | ((uint64_t)ya.w << 32);
+              s2 ^= (uint64_t)yb.x | ((uint64_t)yb.y << 32);
+              s3 ^= (uint64_t)yb.z | ((uint64_t)yb.w << 32);
+              if (k < 3) {
+                s0 = gf_mulx256(s0);
+                s1 = gf_mulx256(s1);
+                s2 = gf_mulx256(s2);
+                s3 = gf_mulx256(s3);
+              }
+            }
+            rem = gf_mulx64(gf_mulx64(gf_mulx64(gf_mulx64(s0) ^ s1) ^ s2) ^ s3);
+          } else {  // ragged last batch of a run that is not a multiple of 128 bytes
+            const int words16 = left >> 4;
+            for (int k = 0; k < words16; ++k) {
+              const uint4 y = *reinterpret_cast<const uint4*>(my_tile_in + k * 16);
+              rem = gf_mulx64(rem ^ ((uint64_t)y.x | ((uint64_t)y.y << 32)));
+              rem = gf_mulx64(rem ^ ((uint64_t)y.z | ((uint64_t)y.w << 32)));
+            }
+          }
+        }
+        __syncwarp();
+      }
+    }
+    if (mine) {
       // align to the end of this page's plane: (nruns - 1 - idx) runs follow
-      rem = gf_mulmod(rem, cp.c_run[nruns - 1 - idx]);
+      rem = gf_mulmod(rem, cp.w.c_run[nruns - 1 - idx]);
       atomicXor(&s_rem[c], (unsigned long long)rem);
     }
     __syncthreads();
-    if (tid < F) cp.page_rem[((int64_t)r * p.maxp + j) * F + tid] = page_ok && fits ? s_rem[tid] : 0ull;
+    // Publish this page's remainders; the CTA that finishes the request's last page folds them.
+    uint64_t* page_rem = cp.w.page_rem + ((int64_t)cp.layer * p.R + r) * p.maxp * F;
+    const int n_r = (s_r + p.P - 1) / p.P;
+    if (tid < F) page_rem[(int64_t)j * F + tid] = page_ok && fits ? s_rem[tid] : 0ull;
+    __threadfence();
+    __syncthreads();
+    __shared__ int s_last;
+    if (tid == 0) s_last = atomicAdd(&cp.w.done[(int64_t)cp.layer * p.R + r], 1) == n_r - 1;
+    __syncthreads();
+    if (s_last) {
+      __threadfence();
+      if (tid < 2) s_rem[tid] = 0ull;
+      __syncthreads();
+      const uint64_t x_last = cp.w.x_last[r];
+      for (int k = tid; k < n_r * F; k += blockDim.x) {
+        const int jj = k / F, cc = k - jj * F;
+        uint64_t v2 = __ldcg(&page_rem[(int64_t)jj * F + cc]);
+        if (jj < n_r - 1) {  // followed by n_r - 2 - jj full pages and the last, possibly partial, page
+          v2 = gf_mulmod(v2, cp.w.c_page[n_r - 2 - jj]);
+          v2 = gf_mulmod(v2, x_last);
+        }
+        atomicXor(&s_rem[cc], (unsigned long long)v2);
+      }
+      __syncthreads();
+      if (tid < F) cp.w.layer_rem[((int64_t)cp.layer * p.R + r) * F + tid] = s_rem[tid];
+    }
   }
   pdl_epilogue(p.overlap);
 }
 
-// One CTA per (request, plane): aligns the page remainders of this layer inside the request's
-// plane, XORs them, and chains the result onto the running state.
-__global__ void __launch_bounds__(256)
-topkv_crc_fold_kernel(CrcWorkspace w, const int32_t* __restrict__ sl, int maxp, int P, int F,
-                      uint64_t* __restrict__ state) {
-  __shared__ unsigned long long s_acc;
-  pdl_prologue(0);
-  const int r = blockIdx.x / F, c = blockIdx.x - r * F;
-  int s = sl[r];
-  s = max(0, min(s, maxp * P));
-  const int n_r = (s + P - 1) / P;
-  if (threadIdx.x == 0) s_acc = 0ull;
-  __syncthreads();
-  uint64_t acc = 0;
-  for (int jj = threadIdx.x; jj < n_r; jj += blockDim.x) {
-    uint64_t rem = w.page_rem[((int64_t)r * maxp + jj) * F + c];
-    if (jj < n_r - 1) {  // followed by n_r - 2 - jj full pages and the last, possibly partial, page
-      rem = gf_mulmod(rem, w.c_page[n_r - 2 - jj]);
-      rem = gf_mulmod(rem, w.x_last[r]);
-    }
-    acc ^= rem;
-  }
-  for (int o = 16; o > 0; o >>= 1) acc ^= __shfl_xor_sync(0xffffffffu, acc, o);
-  if ((threadIdx.x & 31) == 0 && acc) atomicXor(&s_acc, (unsigned long long)acc);
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    const int64_t k = (int64_t)r * F + c;
-    state[k] = gf_mulmod(state[k], w.x_req[r]) ^ s_acc;
-  }
-}
-
-__global__ void topkv_crc_finish_kernel(const uint64_t* __restrict__ state, int n,
-                                        uint64_t* __restrict__ out) {
+// One thread per (request, plane): chains the layers,
+//   state_0 = ~0,  state_l+1 = state_l * x^(8 * bytes of the plane in one layer) + rem_l,
+// and inverts. A request without tokens has remainder 0 in every layer.
+__global__ void __launch_bounds__(128)
+topkv_crc_finish_kernel(CrcWorkspace w, const int32_t* __restrict__ sl, int L, int R, int F,
+                        uint64_t* __restrict__ out) {
   pdl_prologue(0);
   const int k = blockIdx.x * blockDim.x + threadIdx.x;
-  if (k < n) out[k] = ~state[k];
+  if (k >= R * F) return;
+  const int r = k / F, c = k - r * F;
+  const bool empty = sl[r] <= 0;
+  const uint64_t x_req = w.x_req[r];
+  uint64_t state = ~0ull;
+  for (int l = 0; l < L; ++l) {
+    const uint64_t rem = empty ? 0ull : w.layer_rem[((int64_t)l * R + r) * F + c];
+    state = gf_mulmod(state, x_req) ^ rem;
+  }
+  out[k] = ~state;
 }
 
 }  // namespace topkv

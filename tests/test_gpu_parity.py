@@ -480,18 +480,20 @@ def _crc_run(dev, g, sl, bt_s, bt_d, src_h, dst_h, corrupt=None):
     cu = torch.zeros(R + 1, dtype=torch.int64, device=dev)
     tk.check(tk.topkv_build_plan(tk.make_batch(d_bs, d_sl), cu))
     bs, bd = tk.make_batch(d_bs, d_sl, T, cu), tk.make_batch(d_bd, d_sl, T, cu)
+    ov = tk.TOPKV_FLAG_OVERLAP_PREVIOUS                 # layers after the first may overlap
+    bs_ov, bd_ov = tk.make_batch(d_bs, d_sl, T, cu, ov), tk.make_batch(d_bd, d_sl, T, cu, ov)
     nws = tk.topkv_crc_workspace_bytes(lo, R, bt_s.shape[1])
     assert nws > 0
     out = []
-    for side, (pool, batch, fn) in enumerate(((src, bs, tk.topkv_pack_layer_crc),
-                                              (dst, bd, tk.topkv_unpack_layer_crc))):
-        ws = torch.zeros(nws, dtype=torch.uint8, device=dev)
-        state = torch.zeros(R * F, dtype=torch.int64, device=dev)
+    for side, (pool, batch, batch_ov, fn) in enumerate(((src, bs, bs_ov, tk.topkv_pack_layer_crc),
+                                                        (dst, bd, bd_ov, tk.topkv_unpack_layer_crc))):
+        ws = torch.full((nws,), 0xEE, dtype=torch.uint8, device=dev)   # scratch starts dirty
         crc = torch.zeros(R * F, dtype=torch.int64, device=dev)
-        tk.check(tk.topkv_crc_begin(lo, batch, state, ws, nws))
-        for layer in range(g.L):
-            tk.check(fn(layer, pool, lo, batch, wire, wire.numel(), state, ws, nws))
-        tk.check(tk.topkv_crc_finish(lo, batch, state, crc))
+        tk.check(tk.topkv_crc_begin(lo, batch, ws, nws))
+        order = list(range(g.L)) if side == 0 else list(reversed(range(g.L)))  # any layer order
+        for k, layer in enumerate(order):
+            tk.check(fn(layer, pool, lo, batch_ov if k else batch, wire, wire.numel(), ws, nws))
+        tk.check(tk.topkv_crc_finish(lo, batch, ws, nws, crc))
         torch.cuda.synchronize()
         out.append(crc.cpu().numpy().view(np.uint64).reshape(R, F))
         if side == 0 and corrupt is not None:
