@@ -323,6 +323,39 @@ def bench_repage(w, stream, steps):
     return 2.0 * w.n_layer * w.layers * steps / (a.elapsed_time(b) * 1e-3) / 1e9
 
 
+def bench_crc(w, stream, steps):
+    """pack and unpack with the CRC-64 of every request's K and V tensors fused in
+    (topkv_pack_layer_crc / topkv_unpack_layer_crc); GB/s of read + write traffic."""
+    import torch
+    from paper_2607_28633_b200 import binding as tk
+    spec = w.batch.spec
+    nws = tk.topkv_crc_workspace_bytes(w.layout, spec.R, w.batch.max_pages_per_req)
+    ws = torch.empty(nws, dtype=torch.uint8, device=w.src_pool.device)
+    crc = torch.empty(spec.R * spec.F, dtype=torch.int64, device=w.src_pool.device)
+    out = {}
+    for name, fn, pool, batch in (("pack_crc", tk.topkv_pack_layer_crc, w.src_pool, w.src_batch),
+                                  ("unpack_crc", tk.topkv_unpack_layer_crc, w.dst_pool, w.dst_batch)):
+        def run():
+            tk.check(tk.topkv_crc_begin(w.layout, batch, ws, nws, stream))
+            for l in range(w.layers):
+                tk.check(fn(l, pool, w.layout, w._flagged(batch, l > 0), w.wire, w.wire.numel(), ws,
+                            nws, stream))
+            tk.check(tk.topkv_crc_finish(w.layout, batch, ws, nws, crc, stream))
+        run()
+        stream.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(steps):
+            run()
+        b.record(stream)
+        stream.synchronize()
+        ms = a.elapsed_time(b) / steps
+        out[name + "_GBps"] = round(2.0 * w.n_layer * w.layers / (ms * 1e-3) / 1e9, 1)
+        out[name + "_us_per_layer"] = round(ms / w.layers * 1e3, 2)
+    out["checksummed_payload_GBps"] = round(out["pack_crc_GBps"] / 2, 1)
+    return out
+
+
 def pinned_copy_baseline(dev, stream, nbytes, reps=5):
     """cudaMemcpyAsync of one slab between pinned host and device memory (torch copy_), GB/s."""
     import torch
@@ -369,9 +402,18 @@ def run_extra(name, dev, stream, args, peak):
     import torch
     from paper_2607_28633_b200 import harness, overlap
     from paper_2607_28633_b200 import workloads as wl
-    spec = wl.ALL[name]
     nobar = lambda: None
-    out = {"workload": spec.name}
+    spec = wl.ALL[name] if name in wl.ALL else None
+    out = {"workload": spec.name if spec else name}
+    if name == "crc":
+        spec = wl.CFG2 if args.layers is None else wl.with_layers(wl.CFG2, args.layers)
+        w = harness.setup(spec, dev, fill_dst=False)
+        out = {"workload": spec.name}
+        out.update(bench_crc(w, stream, max(1, min(args.steps, 5))))
+        out["frac_of_hbm_peak"] = round(out["pack_crc_GBps"] / peak, 4)
+        del w
+        torch.cuda.empty_cache()
+        return out
     if name in ("cfg3", "cfg4"):
         w = harness.setup(spec, dev, fill_dst=False)
         ms, pack_ms, unpack_ms, _ = bench_d2d(w, stream, args.steps, args.warmup, nobar)
@@ -441,7 +483,7 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="topkv", choices=["topkv", "reference"])
-    ap.add_argument("--extras", default="cfg5,cfg3,cfg4",
+    ap.add_argument("--extras", default="cfg5,cfg3,cfg4,crc",
                     help="comma list of extra workloads measured at one GPU ('' for none)")
     ap.add_argument("--variant", type=int, default=None, help="kernel family (see topkv.h)")
     ap.add_argument("--layers", type=int, default=None, help="fewer layers (profiling only)")

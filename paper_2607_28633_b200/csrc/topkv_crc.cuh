@@ -155,6 +155,10 @@ struct CrcCopyParams {
   int F;
 };
 
+#ifndef TOPKV_CRC_FOUR_CHAINS
+#define TOPKV_CRC_FOUR_CHAINS 0
+#endif
+constexpr bool kCrcFourChains = TOPKV_CRC_FOUR_CHAINS != 0;
 constexpr int kCrcPitch = 144;          // bytes per run in the exchange tile: 128 + 16 of padding
 constexpr int kCrcTileBytes = 32 * kCrcPitch;  // one tile per warp
 
@@ -276,7 +280,7 @@ __global__ void __launch_bounds__(MAXT, 1) topkv_crc_copy_kernel(const CrcCopyPa
         __syncwarp();
         if (off + 128 < cp.g.run_bytes) fetch(off + 128);  // in flight while this batch is folded
         if (mine) {
-          if (left >= 128) {
+          if (kCrcFourChains && left >= 128) {
             // 16 words w0..w15. Four independent chains, chain c over w_c, w_c+4, w_c+8, w_c+12
             // with step x^256; the running remainder rides on w0. Then the chains are joined:
             // rem = (((S0*x^64 + S1)*x^64 + S2)*x^64 + S3)*x^64.
@@ -297,8 +301,8 @@ __global__ void __launch_bounds__(MAXT, 1) topkv_crc_copy_kernel(const CrcCopyPa
               }
             }
             rem = gf_mulx64(gf_mulx64(gf_mulx64(gf_mulx64(s0) ^ s1) ^ s2) ^ s3);
-          } else {  // ragged last batch of a run that is not a multiple of 128 bytes
-            const int words16 = left >> 4;
+          } else {  // one chain (also the ragged last batch of a run that is no multiple of 128 B)
+            const int words16 = min(8, left >> 4);  // never past this lane's 128 bytes of the tile
             for (int k = 0; k < words16; ++k) {
               const uint4 y = *reinterpret_cast<const uint4*>(my_tile_in + k * 16);
               rem = gf_mulx64(rem ^ ((uint64_t)y.x | ((uint64_t)y.y << 32)));
