@@ -4,7 +4,11 @@
  * Pinned by tests/test_oracle_*.py against: the values of Table 1 and Table 4, the §5.2
  * worked example, a hand-derived miniature, an independently derived inverse index map,
  * memcpy / row-gather special cases, and round-trip and permutation invariants.
- * Unpinned parts: none in this file.
+ * The CRC routine is pinned against liblzma (ECMA-182 polynomial), both catalogue check values
+ * and a polynomial-remainder derivation.
+ * parity unpinned: WHICH CRC-64 the paper means (it names no polynomial; the ISO 3309 one is
+ * this build's reading) and the header's field order and widths (the paper lists the fields
+ * and the 128-byte size only). Everything else in this file is pinned.
  */
 #include "topkv_oracle.h"
 

@@ -47,15 +47,6 @@ __host__ __device__ __forceinline__ uint64_t gf_mulx64(uint64_t v) {
   return u ^ (u >> 3) ^ q ^ (q >> 1) ^ (q >> 3) ^ (q >> 4);
 }
 
-// v * x^256 mod P: x^256 = (x^64)^4 = (1 + x^4)(1 + x^12) (mod P; squaring is linear over GF(2)).
-// Same cost as gf_mulx64; it lets four interleaved Horner chains run side by side.
-__host__ __device__ __forceinline__ uint64_t gf_mulx256(uint64_t v) {
-  const uint64_t q1 = v << 60;  // the 4 bits shifted out by v * x^4, as a polynomial in the top bits
-  const uint64_t u = v ^ (v >> 4) ^ q1 ^ (q1 >> 1) ^ (q1 >> 3) ^ (q1 >> 4);
-  const uint64_t q2 = u << 52;  // the 12 bits shifted out by u * x^12
-  return u ^ (u >> 12) ^ q2 ^ (q2 >> 1) ^ (q2 >> 3) ^ (q2 >> 4);
-}
-
 // a * b mod P, Horner over the coefficients of a from the highest power down.
 __host__ __device__ __forceinline__ uint64_t gf_mulmod(uint64_t a, uint64_t b) {
   uint64_t res = 0;
@@ -155,10 +146,6 @@ struct CrcCopyParams {
   int F;
 };
 
-#ifndef TOPKV_CRC_FOUR_CHAINS
-#define TOPKV_CRC_FOUR_CHAINS 0
-#endif
-constexpr bool kCrcFourChains = TOPKV_CRC_FOUR_CHAINS != 0;
 constexpr int kCrcPitch = 144;          // bytes per run in the exchange tile: 128 + 16 of padding
 constexpr int kCrcTileBytes = 32 * kCrcPitch;  // one tile per warp
 
@@ -280,30 +267,10 @@ __global__ void __launch_bounds__(MAXT, 1) topkv_crc_copy_kernel(const CrcCopyPa
         __syncwarp();
         if (off + 128 < cp.g.run_bytes) fetch(off + 128);  // in flight while this batch is folded
         if (mine) {
-          if (kCrcFourChains && left >= 128) {
-            // 16 words w0..w15. Four independent chains, chain c over w_c, w_c+4, w_c+8, w_c+12
-            // with step x^256; the running remainder rides on w0. Then the chains are joined:
-            // rem = (((S0*x^64 + S1)*x^64 + S2)*x^64 + S3)*x^64.
-            uint64_t s0 = rem, s1 = 0, s2 = 0, s3 = 0;
+          const int words16 = min(8, left >> 4);  // never past this lane's 128 bytes of the tile
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              const uint4 ya = *reinterpret_cast<const uint4*>(my_tile_in + k * 32);
-              const uint4 yb = *reinterpret_cast<const uint4*>(my_tile_in + k * 32 + 16);
-              s0 ^= (uint64_t)ya.x | ((uint64_t)ya.y << 32);
-              s1 ^= (uint64_t)ya.z | ((uint64_t)ya.w << 32);
-              s2 ^= (uint64_t)yb.x | ((uint64_t)yb.y << 32);
-              s3 ^= (uint64_t)yb.z | ((uint64_t)yb.w << 32);
-              if (k < 3) {
-                s0 = gf_mulx256(s0);
-                s1 = gf_mulx256(s1);
-                s2 = gf_mulx256(s2);
-                s3 = gf_mulx256(s3);
-              }
-            }
-            rem = gf_mulx64(gf_mulx64(gf_mulx64(gf_mulx64(s0) ^ s1) ^ s2) ^ s3);
-          } else {  // one chain (also the ragged last batch of a run that is no multiple of 128 B)
-            const int words16 = min(8, left >> 4);  // never past this lane's 128 bytes of the tile
-            for (int k = 0; k < words16; ++k) {
+          for (int k = 0; k < 8; ++k) {
+            if (k < words16) {
               const uint4 y = *reinterpret_cast<const uint4*>(my_tile_in + k * 16);
               rem = gf_mulx64(rem ^ ((uint64_t)y.x | ((uint64_t)y.y << 32)));
               rem = gf_mulx64(rem ^ ((uint64_t)y.z | ((uint64_t)y.w << 32)));
