@@ -340,29 +340,52 @@ def test_bench_shapes_reduced_layers(dev, name):
     torch.cuda.empty_cache()
 
 
-def test_cfg2_full_size_sampled_layers(dev):
-    """The launch configuration bench.py times (all 32 layers resident), three layers checked
-    in full against the oracle and every other layer's wire by a sampled-row comparison."""
-    spec = wl.CFG2
+def _oracle_token(spec, page_host, t):
+    """The wire bytes of token t of one page, computed by the oracle on a one-page problem."""
+    g = Geom(L=1, F=spec.F, h_kv=spec.H, d_h=spec.D, b_p=spec.E, P=spec.P, num_pages=1)
+    wire = oracle.pack(g, 0, page_host, np.zeros((1, 1), dtype=np.int32),
+                       np.array([t + 1], dtype=np.int32))
+    return wire[t * spec.tok_bytes:(t + 1) * spec.tok_bytes]
+
+
+@pytest.mark.parametrize("name,full_layers", [("cfg2", (0, 17, 31)), ("cfg3", (0, 79)), ("cfg4", (0, 60))])
+def test_full_size_in_the_bench_launch_configuration(dev, name, full_layers):
+    """The workloads at full size, all layers resident, issued as bench.py issues them (one
+    stream, TOPKV_FLAG_OVERLAP_PREVIOUS after the first layer of each phase). A few layers are
+    compared in full with the oracle; in every layer sampled tokens are compared with what the
+    oracle computes for them one by one, on the wire and in the destination pool."""
+    spec = wl.ALL[name]
     w = harness.setup(spec, dev)
-    _check_layers(w, [0, 17, spec.L - 1], dev)
     b, s = w.batch, spec
+    stream = torch.cuda.Stream(dev)
+    g1 = _geom(s, b.num_pool_pages, 1, 0, 0)
+    dst_before = {l: harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, l) for l in full_layers}
+    for layer in range(s.L):
+        w.pack(layer, stream, overlap=layer > 0)
+    for layer in range(s.L):
+        w.unpack(layer, stream, overlap=layer > 0)
+    stream.synchronize()
+    for layer in full_layers:
+        src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, layer)
+        want = oracle.pack(g1, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=8)
+        got = w.wire[layer * w.n_layer:(layer + 1) * w.n_layer].cpu().numpy()
+        assert np.array_equal(got, want), f"pack layer {layer}"
+        dst_h = dst_before[layer]
+        oracle.unpack(g1, 0, dst_h, b.dst_block_table, b.seq_lens, want, impl="rows", threads=8)
+        assert np.array_equal(harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, layer), dst_h), \
+            f"unpack layer {layer}"
     rng = np.random.default_rng(7)
     cu = np.concatenate([[0], np.cumsum(b.seq_lens.astype(np.int64))])
-    for layer in range(spec.L):
-        w.pack(layer)
-    torch.cuda.synchronize()
-    for layer in range(spec.L):
-        # sampled tokens, each computed one by one from the definition
-        for _ in range(16):
+    for layer in range(s.L):
+        for _ in range(4):
             r = int(rng.integers(0, s.R))
             i = int(rng.integers(0, b.seq_lens[r]))
-            page = int(b.src_block_table[r, i // s.P])
-            for c in range(s.F):
-                po = (layer * w.slab_bytes + page * s.page_bytes + c * s.P * s.row_bytes
-                      + (i % s.P) * s.row_bytes)
-                wo = layer * w.n_layer + ((cu[r] + i) * s.F + c) * s.row_bytes
-                assert torch.equal(w.src_pool[po:po + s.row_bytes], w.wire[wo:wo + s.row_bytes])
+            wo = layer * w.n_layer + (int(cu[r]) + i) * s.tok_bytes
+            got_wire = w.wire[wo:wo + s.tok_bytes].cpu().numpy()
+            for pool, table in ((w.src_pool, b.src_block_table), (w.dst_pool, b.dst_block_table)):
+                po = layer * w.slab_bytes + int(table[r, i // s.P]) * s.page_bytes
+                page_h = pool[po:po + s.page_bytes].cpu().numpy()
+                assert np.array_equal(_oracle_token(s, page_h, i % s.P), got_wire), (layer, r, i)
     del w
     torch.cuda.empty_cache()
 
