@@ -32,9 +32,9 @@ METRIC = "kv_pack_unpack_GBps"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM traffic of one pack launch relative to its algorithmic bytes, from the steady-state ncu
-# capture summarised in profiles/page_copy_kernel_pack_cfg2_4layers.md
-# ((dram__bytes_read.sum + dram__bytes_write.sum) / (2*N_layer), same per-launch size as here).
+# DRAM traffic of one pack launch relative to its algorithmic bytes, from a steady-state ncu
+# capture of this kernel at the same per-launch size (--cache-control none, six launches):
+# (dram__bytes_read.sum + dram__bytes_write.sum) / (2*N_layer).
 NCU_TRAFFIC_RATIO = 0.995
 
 

@@ -205,8 +205,9 @@ int topkv_header_check(const topkv_wire_header* header, const topkv_layout* layo
                        int64_t seq_len, uint64_t crc_k, uint64_t crc_v);
 
 /* The checksum: reflected CRC-64, all-ones initial value, final inversion, ISO 3309
- * polynomial x^64 + x^4 + x^3 + x + 1 (the paper names no polynomial). The
- * K (V) checksum of a request covers its K (V) tensor in the order
+ * polynomial x^64 + x^4 + x^3 + x + 1 (the paper names no polynomial: this is the
+ * generator of Go's crc64.ISO table, catalogue name CRC-64/GO-ISO, check value of "123456789"
+ * 0xB90956C775A41001). The K (V) checksum of a request covers its K (V) tensor in the order
  * [layers][seq_len][kv_heads][head_dim]. topkv_crc64 is the plain HOST routine. */
 uint64_t topkv_crc64(const void* h_data, int64_t nbytes);
 
