@@ -208,15 +208,6 @@ def workload_config(spec, batch):
                   "precede all unpacks, so no slab is re-read from L2"}
 
 
-def time_phase(stream, fn):
-    import torch
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record(stream)
-    fn()
-    b.record(stream)
-    return a, b
-
-
 def bench_d2d(w, stream, steps, warmup, barrier):
     """Times K steps of plan + pack(all layers) + unpack(all layers). Returns per-step ms
     (whole region / K), and the summed pack-phase and unpack-phase ms."""

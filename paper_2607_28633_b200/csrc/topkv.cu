@@ -351,6 +351,8 @@ int check_batch(const topkv_layout* lo, const topkv_batch* b) {
     if (b->cu_seq_lens == nullptr && b->num_requests > TOPKV_MAX_INLINE_R)
       return TOPKV_ERR_INVALID_ARG;
     if ((int64_t)b->num_requests * b->max_pages_per_req > 0x7fffffffll) return TOPKV_ERR_INVALID_ARG;
+    // a block-table row must not describe more tokens than an int32 length can hold
+    if ((int64_t)b->max_pages_per_req * lo->page_tokens > 0x7fffffffll) return TOPKV_ERR_INVALID_ARG;
     if (b->total_tokens > (int64_t)b->num_requests * b->max_pages_per_req * lo->page_tokens)
       return TOPKV_ERR_INVALID_ARG;
   }
@@ -458,6 +460,7 @@ template <bool PACK>
 int launch_bulk(const KParams& kp0, const Resolved& rs, int F, cudaStream_t stream, bool* handled) {
   *handled = false;
   if (kp0.R > kBulkMaxR || kp0.window > 0) return TOPKV_OK;
+  if ((int64_t)kp0.R * kp0.maxp * kp0.P > 0x7fffffffll) return TOPKV_OK;  // its prefix sums are int32
   const int64_t tok_bytes = (int64_t)F * rs.row_bytes;
   if (tok_bytes > kStageTarget || rs.unit_bytes > 0x7fffffff) return TOPKV_OK;
   if (!rs.merged && rs.unit_bytes < 1024) return TOPKV_OK;  // per-copy cost dominates small units

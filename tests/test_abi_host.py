@@ -131,6 +131,8 @@ def test_argument_validation_without_gpu():
     assert P(0, pool, bad, b, wire, cap) == tk.TOPKV_ERR_ALIGNMENT
     bb = _batch(); bb.struct_size = 4
     assert P(0, pool, lo, bb, wire, cap) == tk.TOPKV_ERR_INVALID_ARG
+    huge = tk.make_layout(4, 2, 8, 128, 2, 1 << 20, 64)      # 2^20-token pages x 4096 columns
+    assert P(0, pool, huge, _batch(R=1, maxp=4096, T=-1), wire, cap) == tk.TOPKV_ERR_INVALID_ARG
     bb = _batch(); bb.window_tokens = -1
     assert P(0, pool, lo, bb, wire, cap) == tk.TOPKV_ERR_INVALID_ARG
     bb = _batch(); bb.flags = 2                              # unknown flag bit
