@@ -396,6 +396,41 @@ def run_extra(name, dev, stream, args, peak):
     nobar = lambda: None
     spec = wl.ALL[name] if name in wl.ALL else None
     out = {"workload": spec.name if spec else name}
+    if name == "cfg1":
+        # the tiny, launch-bound case: eager issue against one CUDA graph of the whole step
+        w = harness.setup(wl.CFG1, dev, fill_dst=False)
+
+        def step():
+            for l in range(w.layers):
+                w.pack(l, stream, overlap=l > 0)
+            for l in range(w.layers):
+                w.unpack(l, stream, overlap=l > 0)
+
+        def timed(fn, reps=200):
+            for _ in range(10):
+                fn()
+            stream.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(reps):
+                fn()
+            b.record(stream)
+            stream.synchronize()
+            return a.elapsed_time(b) / reps * 1e3
+
+        with torch.cuda.stream(stream):
+            eager_us = timed(step)
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                step()
+            graph_us = timed(graph.replay)
+        out = {"workload": wl.CFG1.name, "kernels_per_step": 2 * w.layers,
+               "eager_us_per_step": round(eager_us, 2), "cuda_graph_us_per_step": round(graph_us, 2),
+               "bytes_moved_per_step": 4 * w.n_layer * w.layers,
+               "note": "1.8 MB per layer: L2-resident and launch-bound, no roofline claim"}
+        del w, graph
+        torch.cuda.empty_cache()
+        return out
     if name == "crc":
         spec = wl.CFG2 if args.layers is None else wl.with_layers(wl.CFG2, args.layers)
         w = harness.setup(spec, dev, fill_dst=False)
@@ -474,7 +509,7 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="topkv", choices=["topkv", "reference"])
-    ap.add_argument("--extras", default="cfg5,cfg3,cfg4,crc",
+    ap.add_argument("--extras", default="cfg5,cfg3,cfg4,crc,cfg1",
                     help="comma list of extra workloads measured at one GPU ('' for none)")
     ap.add_argument("--variant", type=int, default=None, help="kernel family (see topkv.h)")
     ap.add_argument("--layers", type=int, default=None, help="fewer layers (profiling only)")

@@ -39,6 +39,11 @@
  * once the caller has synchronised with the stream. All `const void*`/`void*`
  * arguments are DEVICE pointers unless their name starts with `h_`.
  *
+ * Stream capture: topkv_pack_layer, topkv_unpack_layer, the two host-leg calls,
+ * topkv_repage_layer, topkv_build_plan and the checksummed copies only enqueue kernels and
+ * copies, so they may be issued while `stream` is being captured into a CUDA graph (the
+ * descriptors are read at call time; the buffers they point to at replay time).
+ *
  * Errors: every int-returning function returns TOPKV_OK (0) or a negative
  * topkv_status. When an error is returned nothing has been launched.
  */

@@ -420,6 +420,67 @@ def test_overlapped_launches_keep_results_and_order(dev):
     torch.cuda.empty_cache()
 
 
+def test_cuda_graph_capture_and_replay(dev):
+    """The hot calls only enqueue work, so a whole layer loop can be captured in a CUDA graph
+    and replayed (the launch-bound tiny case is where that pays)."""
+    w = harness.setup(wl.CFG1, dev)
+    b, s = w.batch, wl.CFG1
+    g = _geom(s, b.num_pool_pages, s.L, 0, w.n_layer)
+    src_h, dst_h = w.src_pool.cpu().numpy(), w.dst_pool.cpu().numpy()
+    stream = torch.cuda.Stream(dev)
+    with torch.cuda.stream(stream):                      # warm up outside the capture
+        for layer in range(s.L):
+            w.pack(layer, stream)
+            w.unpack(layer, stream)
+    stream.synchronize()
+    w.wire.zero_()
+    w.dst_pool.copy_(torch.from_numpy(dst_h))
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        for layer in range(s.L):
+            w.pack(layer, stream, overlap=layer > 0)
+        for layer in range(s.L):
+            w.unpack(layer, stream, overlap=layer > 0)
+    assert not w.wire.any()                              # capturing executed nothing
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    want_wire = np.zeros(s.L * w.n_layer, dtype=np.uint8)
+    for layer in range(s.L):
+        oracle.pack(g, layer, src_h, b.src_block_table, b.seq_lens, wire=want_wire)
+        oracle.unpack(g, layer, dst_h, b.dst_block_table, b.seq_lens, want_wire)
+    assert np.array_equal(w.wire.cpu().numpy(), want_wire)
+    assert np.array_equal(w.dst_pool.cpu().numpy(), dst_h)
+
+
+def test_two_batches_on_two_streams(dev):
+    """Independent batches issued concurrently on two streams do not disturb each other (the
+    library keeps no per-call state)."""
+    specs = [wl.with_layers(wl.CFG2, 3), wl.with_layers(wl.CFG4, 3)]
+    ws = [harness.setup(sp, dev) for sp in specs]
+    streams = [torch.cuda.Stream(dev) for _ in ws]
+    before = [[harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, l) for l in range(3)] for w in ws]
+    for layer in range(3):
+        for w, st in zip(ws, streams):
+            w.pack(layer, st, overlap=layer > 0)
+    for layer in range(3):
+        for w, st in zip(ws, streams):
+            w.unpack(layer, st, overlap=layer > 0)
+    torch.cuda.synchronize()
+    for w, sp, dst0 in zip(ws, specs, before):
+        g = _geom(sp, w.batch.num_pool_pages, 1, 0, 0)
+        for layer in range(3):
+            src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, layer)
+            want = oracle.pack(g, 0, src_h, w.batch.src_block_table, w.batch.seq_lens, impl="rows", threads=8)
+            assert np.array_equal(w.wire[layer * w.n_layer:(layer + 1) * w.n_layer].cpu().numpy(), want)
+            oracle.unpack(g, 0, dst0[layer], w.batch.dst_block_table, w.batch.seq_lens, want,
+                          impl="rows", threads=8)
+            assert np.array_equal(harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, layer), dst0[layer])
+    del ws
+    torch.cuda.empty_cache()
+
+
 # -------------------------------------------------------------------- windowed layers (§2.2)
 
 @pytest.mark.parametrize("seed", range(16))
