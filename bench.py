@@ -139,13 +139,14 @@ def host_cores():
     return len(os.sched_getaffinity(0))
 
 
-def oracle_sample(spec, batch, seconds_target=12.0):
-    """Times the CPU oracle (row-memcpy form, all cores) on whole layers of this workload until
-    about ``seconds_target`` of wall time has passed. Returns (GB/s, layers timed, cores)."""
+def oracle_sample(spec, batch, seconds_target=12.0, threads=None, impl="rows"):
+    """Times the CPU oracle (row-memcpy form on all cores unless told otherwise) on whole layers
+    of this workload until about ``seconds_target`` of wall time has passed. Returns
+    (GB/s, layers timed, threads, seconds)."""
     import numpy as np
     import oracle
     from paper_2607_28633_b200 import workloads as wl
-    cores = host_cores()
+    cores = host_cores() if threads is None else threads
     g = oracle.Geom(L=1, F=spec.F, h_kv=spec.H, d_h=spec.D, b_p=spec.E, P=spec.P,
                     num_pages=batch.num_pool_pages)
     src = wl.fill_numpy(g.pool_bytes(), batch.seeds["data"], raw_bits=True)
@@ -157,9 +158,9 @@ def oracle_sample(spec, batch, seconds_target=12.0):
     oracle.unpack(g, 0, dst, batch.dst_block_table, batch.seq_lens, wire, impl="rows", threads=cores)
     t0, n = time.perf_counter(), 0
     while True:
-        oracle.pack(g, 0, src, batch.src_block_table, batch.seq_lens, wire=wire, impl="rows",
+        oracle.pack(g, 0, src, batch.src_block_table, batch.seq_lens, wire=wire, impl=impl,
                     threads=cores)
-        oracle.unpack(g, 0, dst, batch.dst_block_table, batch.seq_lens, wire, impl="rows",
+        oracle.unpack(g, 0, dst, batch.dst_block_table, batch.seq_lens, wire, impl=impl,
                       threads=cores)
         n += 1
         dt = time.perf_counter() - t0
@@ -618,6 +619,12 @@ def main():
         cpu = {"value": round(v, 3), "unit": UNIT, "cores": cores, "kind": "oracle",
                "sample": f"{n} layer(s) of {wl.CFG2.L} of this workload, pack+unpack, "
                          f"rows-memcpy oracle, {dt:.1f} s"}
+        # for context: the same oracle on one thread, and the byte-by-byte definition on cfg1
+        v1, n1, _, dt1 = oracle_sample(wl.CFG2, wl.make_batch(wl.CFG2), seconds_target=4.0, threads=1)
+        vr, nr, _, dtr = oracle_sample(wl.CFG1, wl.make_batch(wl.CFG1), seconds_target=3.0, threads=1,
+                                       impl="ref")
+        cpu["one_thread_GBps"] = round(v1, 3)
+        cpu["byte_loop_definition_cfg1_GBps"] = round(vr, 4)
 
     if rank == 0:
         line = {

@@ -63,6 +63,42 @@ __device__ __forceinline__ void pdl_epilogue(int overlap) {
   if (overlap && blockIdx.x == 0 && threadIdx.x == 0) pdl_wait_prior_grid();
 }
 
+// Streaming vector accesses: every byte is touched exactly once, so neither side should
+// displace anything useful from L1 / L2. Vec<32> uses the 256-bit global accesses of sm_100.
+template <int VEC>
+struct Vec;
+template <>
+struct Vec<16> {
+  uint32_t v[4];
+  __device__ __forceinline__ void load(const uint8_t* p) {
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3])
+                 : "l"(p));
+  }
+  __device__ __forceinline__ void store(uint8_t* p) const {
+    asm volatile("st.global.L1::no_allocate.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v[0]),
+                 "r"(v[1]), "r"(v[2]), "r"(v[3])
+                 : "memory");
+  }
+};
+template <>
+struct Vec<32> {
+  uint32_t v[8];
+  __device__ __forceinline__ void load(const uint8_t* p) {
+    asm volatile(
+        "ld.global.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+          "=r"(v[7])
+        : "l"(p));
+  }
+  __device__ __forceinline__ void store(uint8_t* p) const {
+    asm volatile(
+        "st.global.L1::no_allocate.L2::evict_first.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p),
+        "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+        : "memory");
+  }
+};
+
 // Launch with programmatic stream serialisation allowed (see pdl_prologue above).
 template <typename P>
 cudaError_t launch_pdl(void (*kernel)(const P), dim3 grid, dim3 block, size_t smem,

@@ -30,40 +30,6 @@ struct RepageParams {
   int overlap;
 };
 
-template <int VEC>
-struct RVec;
-template <>
-struct RVec<16> {
-  uint32_t v[4];
-  __device__ __forceinline__ void load(const uint8_t* p) {
-    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3])
-                 : "l"(p));
-  }
-  __device__ __forceinline__ void store(uint8_t* p) const {
-    asm volatile("st.global.L1::no_allocate.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v[0]),
-                 "r"(v[1]), "r"(v[2]), "r"(v[3])
-                 : "memory");
-  }
-};
-template <>
-struct RVec<32> {
-  uint32_t v[8];
-  __device__ __forceinline__ void load(const uint8_t* p) {
-    asm volatile(
-        "ld.global.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
-          "=r"(v[7])
-        : "l"(p));
-  }
-  __device__ __forceinline__ void store(uint8_t* p) const {
-    asm volatile(
-        "st.global.L1::no_allocate.L2::evict_first.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p),
-        "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
-        : "memory");
-  }
-};
-
 template <int F, int VEC>
 __global__ void __launch_bounds__(kRepageThreads, 3) topkv_repage_kernel(const RepageParams p) {
   __shared__ int32_t s_pg_s[kRepageMaxPages];
@@ -110,7 +76,7 @@ __global__ void __launch_bounds__(kRepageThreads, 3) topkv_repage_kernel(const R
     if (my_g < groups) {
       for (int q0 = my_g; q0 < nunits; q0 += groups * kUnroll) {
         for (int w = my_w; w < p.unit_chunks; w += tpu) {
-          RVec<VEC> buf[kUnroll];
+          Vec<VEC> buf[kUnroll];
           uint8_t* dstp[kUnroll];
           bool ok[kUnroll];
 #pragma unroll
