@@ -41,7 +41,7 @@ def build(force: bool = False) -> str:
 class _Geom(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int64) for n in (
         "L", "F", "h_kv", "d_h", "b_p", "P", "S_layer", "S_page", "S_kv", "S_tok", "S_head",
-        "W_layer", "wire_order", "window")]
+        "W_layer", "wire_order", "W_plane", "window")]
 
 
 _lib = None
@@ -99,6 +99,7 @@ class Geom:
     S_tok: int = 0
     S_head: int = 0
     W_layer: int = 0
+    W_plane: int = 0         # PLANAR: bytes between the planes of a slab (0 = adjacent)
     window: int = 0          # 0: every token; W > 0: the layer keeps only the last min(s, W)
 
     def __post_init__(self):
@@ -123,7 +124,7 @@ class Geom:
     def _c(self) -> _Geom:
         return _Geom(self.L, self.F, self.h_kv, self.d_h, self.b_p, self.P, self.S_layer,
                      self.S_page, self.S_kv, self.S_tok, self.S_head, self.W_layer,
-                     self.wire_order, self.window)
+                     self.wire_order, self.W_plane, self.window)
 
     def kept_tokens(self, sl) -> int:
         """Tokens of a batch that this layer keeps: sum of min(s, window) (all, if no window)."""
@@ -180,6 +181,8 @@ def _check_extent(g: Geom, layer: int, pool: np.ndarray, bt, sl, wire: np.ndarra
     """Guards the C loops: every offset they will form must lie inside the arrays."""
     T = g.kept_tokens(sl)
     need_wire = layer * g.W_layer + g.wire_layer_bytes(T)
+    if g.W_plane > 0 and g.wire_order == WIRE_PLANAR:
+        need_wire = layer * g.W_layer + (g.F - 1) * g.W_plane + T * g.row_bytes
     assert wire.size >= need_wire, (wire.size, need_wire)
     assert 0 <= layer < g.L
     for r in range(sl.shape[0]):
@@ -201,6 +204,7 @@ def pack(g: Geom, layer: int, pool: np.ndarray, bt: np.ndarray, sl: np.ndarray,
     bt, sl = _tables(bt, sl)
     T = g.kept_tokens(sl)
     if wire is None:
+        assert g.W_plane == 0, "spread planes need a caller-sized wire"
         wire = np.zeros(layer * g.W_layer + g.wire_layer_bytes(T), dtype=np.uint8)
     _u8(pool, False), _u8(wire, True)
     _check_extent(g, layer, pool, bt, sl, wire)

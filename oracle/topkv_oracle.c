@@ -59,7 +59,10 @@ static int64_t poff(const oracle_geom* g, int64_t l, int64_t page, int64_t c, in
 static int64_t woff(const oracle_geom* g, int64_t l, int64_t n, int64_t T, int64_t c, int64_t h,
                     int64_t d, int64_t b) {
   int64_t row_bytes = g->h_kv * g->d_h * g->b_p;
-  int64_t row = (g->wire_order == ORACLE_WIRE_PLANAR) ? (c * T + n) : (n * g->F + c);
+  /* PLANAR: plane c starts c*T rows into the slab, or c*W_plane bytes when the caller spreads
+   * the planes (e.g. K of all layers, then V of all layers, as in the paper's payload, §3.4) */
+  int64_t plane_rows = g->W_plane > 0 ? g->W_plane / row_bytes : T;
+  int64_t row = (g->wire_order == ORACLE_WIRE_PLANAR) ? (c * plane_rows + n) : (n * g->F + c);
   return l * g->W_layer + row * row_bytes + (h * g->d_h + d) * g->b_p + b;
 }
 

@@ -21,6 +21,8 @@ typedef struct oracle_geom {
   int64_t S_layer, S_page, S_kv, S_tok, S_head; /* pool strides, bytes            */
   int64_t W_layer;              /* bytes between wire slabs of consecutive layers */
   int64_t wire_order;           /* ORACLE_WIRE_*                                  */
+  int64_t W_plane;              /* PLANAR only: bytes between the K and the V     */
+                                /* plane of a slab; 0 = they are adjacent (T rows) */
   int64_t window;               /* 0: all tokens; W > 0: a windowed layer keeps   */
                                 /* (and sends) only the last min(s, W) tokens     */
 } oracle_geom;

@@ -531,3 +531,28 @@ def test_header_layout():
     assert int.from_bytes(h[64:72], "little") == 0x1122334455667788
     assert int.from_bytes(h[72:80], "little") == 0x99AABBCCDDEEFF00
     assert h[80:] == bytes(48)
+
+
+def test_paper_payload_layout_k_tensor_then_v_tensor():
+    """§3.4: header, then the K tensor [layers][seq_len][kv_heads][head_dim], then the V tensor.
+    With one request, PLANAR order, a layer stride of one plane and a plane stride of L planes
+    the per-layer packs assemble exactly that payload."""
+    g, pool, bt, sl = _random_case(33, 2, 2, 8, 4, strided=False)
+    r = int(np.argmax(sl))
+    bt1, sl1 = bt[r:r + 1], sl[r:r + 1]
+    s = int(sl1[0])
+    assert s > 0
+    plane = s * g.row_bytes                       # one layer of one plane
+    g.wire_order, g.W_layer, g.W_plane = WIRE_PLANAR, plane, g.L * plane
+    payload = np.zeros(2 * g.L * plane, dtype=np.uint8)
+    for layer in range(g.L):
+        oracle.pack(g, layer, pool, bt1, sl1, wire=payload)
+    # the same tensors from the adjacent-plane PLANAR pack pinned above
+    g.W_layer = g.W_plane = 0
+    per_layer = [oracle.pack(g, l, pool, bt1, sl1).reshape(2, s * g.row_bytes) for l in range(g.L)]
+    k_tensor = np.concatenate([x[0] for x in per_layer])
+    v_tensor = np.concatenate([x[1] for x in per_layer])
+    assert np.array_equal(payload, np.concatenate([k_tensor, v_tensor]))
+    assert oracle.crc64(k_tensor) == oracle.kv_plane_crc(g, pool, bt1, sl1, 0, 0)
+    assert oracle.crc64(v_tensor) == oracle.kv_plane_crc(g, pool, bt1, sl1, 0, 1)
+    g.wire_order = WIRE_TOKEN_KV
