@@ -94,6 +94,13 @@ typedef struct topkv_layout {
   int64_t pool_token_stride;
   int64_t pool_head_stride; /* ignored when H == 1                                        */
   int64_t wire_layer_stride;/* bytes between wire slabs; 0 = caller passes layer's slab   */
+  int64_t wire_plane_stride;/* PLANAR only: bytes from the K plane to the V plane of a    */
+                            /* slab; 0 = adjacent (T*row_bytes). With one request, a      */
+                            /* layer stride of s*row_bytes and a plane stride of          */
+                            /* L*s*row_bytes the layers assemble the paper's payload: the */
+                            /* K tensor [layers][seq_len][heads][dim], then the V tensor  */
+                            /* (§3.4). Must be a multiple of row_bytes; not accepted by   */
+                            /* the staged host-leg calls (they copy one contiguous slab). */
 } topkv_layout;
 
 /* One batch of requests. block_table and seq_lens do not depend on the layer

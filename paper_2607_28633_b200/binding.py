@@ -53,7 +53,7 @@ class topkv_layout(ctypes.Structure):
         ("reserved", c_uint32), ("num_pool_pages", c_int64), ("pool_layer_stride", c_int64),
         ("pool_page_stride", c_int64), ("pool_kv_stride", c_int64),
         ("pool_token_stride", c_int64), ("pool_head_stride", c_int64),
-        ("wire_layer_stride", c_int64),
+        ("wire_layer_stride", c_int64), ("wire_plane_stride", c_int64),
     ]
 
 

@@ -68,7 +68,9 @@ int check_layout(const topkv_layout* lo, Resolved* out) {
   if (lo->pool_page_stride <= 0 || lo->pool_layer_stride <= 0 ||
       (lo->page_tokens > 1 && lo->pool_token_stride < unit) ||
       (lo->kv_factor > 1 && lo->pool_kv_stride <= 0) ||
-      (!heads_contig && lo->pool_head_stride < head_bytes) || lo->wire_layer_stride < 0)
+      (!heads_contig && lo->pool_head_stride < head_bytes) || lo->wire_layer_stride < 0 ||
+      lo->wire_plane_stride < 0 || lo->wire_plane_stride % row_bytes != 0 ||
+      (lo->wire_plane_stride != 0 && lo->wire_order != TOPKV_WIRE_PLANAR))
     return TOPKV_ERR_UNSUPPORTED_LAYOUT;
   if (!mult16(unit) || !mult16(lo->pool_page_stride) || !mult16(lo->pool_token_stride) ||
       !mult16(lo->pool_layer_stride) || (lo->kv_factor > 1 && !mult16(lo->pool_kv_stride)) ||
@@ -115,9 +117,12 @@ int prepare(int layer, const void* pool, const topkv_layout* lo, const topkv_bat
   if (pool == nullptr || wire_base == nullptr || capacity < 0) return TOPKV_ERR_INVALID_ARG;
   if (!mult16p(pool) || !mult16p(wire_base)) return TOPKV_ERR_ALIGNMENT;
   int64_t n_layer = -1;
+  const bool spread = lo->wire_plane_stride > 0;  // planes of a slab are not adjacent
   if (b->total_tokens >= 0) {
     n_layer = b->total_tokens * lo->kv_factor * rs->row_bytes;
-    if ((int64_t)layer * wire_layer_stride + n_layer > capacity) return TOPKV_ERR_CAPACITY;
+    const int64_t extent = spread ? (lo->kv_factor - 1) * lo->wire_plane_stride + b->total_tokens * rs->row_bytes
+                                  : n_layer;  // bytes from the slab's base to its last byte
+    if ((int64_t)layer * wire_layer_stride + extent > capacity) return TOPKV_ERR_CAPACITY;
   }
   *n_layer_out = n_layer;
   kp->pool = const_cast<uint8_t*>(static_cast<const uint8_t*>(pool)) + (int64_t)layer * lo->pool_layer_stride;
@@ -141,7 +146,8 @@ int prepare(int layer, const void* pool, const topkv_layout* lo, const topkv_bat
   kp->spr = kp->maxp;
   kp->window = b->window_tokens;
   kp->num_pages = lo->num_pool_pages;
-  kp->wire_limit = n_layer >= 0 ? n_layer : capacity - (int64_t)layer * wire_layer_stride;
+  kp->wire_limit = (n_layer >= 0 && !spread) ? n_layer : capacity - (int64_t)layer * wire_layer_stride;
+  kp->plane_rows = spread ? lo->wire_plane_stride / rs->row_bytes : -1;
   return TOPKV_OK;
 }
 
@@ -428,6 +434,7 @@ int topkv_pack_layer_to_host(int layer, const void* src_pool, const topkv_layout
   int st = prepare(layer, src_pool, layout, batch, h_pinned, host_capacity_bytes,
                    layout ? layout->wire_layer_stride : 0, &kp, &rs, &n_layer);
   if (st != TOPKV_OK) return st;
+  if (layout->wire_plane_stride != 0) return TOPKV_ERR_UNSUPPORTED_LAYOUT;  // one contiguous copy
   if (!mult16p(d_staging)) return TOPKV_ERR_ALIGNMENT;
   if (staging_capacity_bytes < n_layer) return TOPKV_ERR_CAPACITY;
   uint8_t* host_slab = kp.wire;
@@ -464,6 +471,7 @@ int topkv_unpack_layer_from_host(int layer, void* dst_pool, const topkv_layout* 
   int st = prepare(layer, dst_pool, layout, batch, h_pinned, host_bytes,
                    layout ? layout->wire_layer_stride : 0, &kp, &rs, &n_layer);
   if (st != TOPKV_OK) return st;
+  if (layout->wire_plane_stride != 0) return TOPKV_ERR_UNSUPPORTED_LAYOUT;  // one contiguous copy
   if (!mult16p(d_staging)) return TOPKV_ERR_ALIGNMENT;
   if (staging_capacity_bytes < n_layer) return TOPKV_ERR_CAPACITY;
   if (n_layer > 0) {
@@ -486,6 +494,7 @@ int topkv_pack_layer_to_host_noalloc(int layer, const void* src_pool, const topk
   int st = prepare(layer, src_pool, layout, batch, h_pinned, host_capacity_bytes,
                    layout ? layout->wire_layer_stride : 0, &kp, &rs, &n_layer);
   if (st != TOPKV_OK) return st;
+  if (layout->wire_plane_stride != 0) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
   if (n_layer > (int64_t)TOPKV_NOALLOC_STAGING_BYTES) return TOPKV_ERR_CAPACITY;
   void* staging = nullptr;
   st = noalloc_staging_address(&staging);  // first call on this device: symbol lookup

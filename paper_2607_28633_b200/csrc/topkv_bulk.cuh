@@ -133,12 +133,16 @@ __global__ void __launch_bounds__(kBulkThreads, 1) topkv_bulk_kernel(const BulkP
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   __syncthreads();
 
-  const int64_t T = (p.T >= 0) ? p.T : (int64_t)s_cu[p.R];
-  if (T < (int64_t)s_cu[p.R] ||
-      T * F * p.U * ((int64_t)p.unit_chunks * 16) > p.wire_limit) {  // uniform over the grid
-    if (threadIdx.x == 0) raise_error(kErrWire);
-    pdl_epilogue(p.overlap);
-    return;
+  // rows from the K plane to the V plane of a PLANAR slab
+  const int64_t T = p.plane_rows >= 0 ? p.plane_rows : ((p.T >= 0) ? p.T : (int64_t)s_cu[p.R]);
+  {
+    const int64_t row = (int64_t)p.U * p.unit_chunks * 16, S = s_cu[p.R];  // uniform over the grid
+    const bool fits = p.planar ? ((F - 1) * T + S) * row <= p.wire_limit : S * F * row <= p.wire_limit;
+    if (!fits) {
+      if (threadIdx.x == 0) raise_error(kErrWire);
+      pdl_epilogue(p.overlap);
+      return;
+    }
   }
   const int64_t unit_bytes = (int64_t)p.unit_chunks * 16;
   const int64_t total_items = (int64_t)s_pc[p.R] * bp.cpp;

@@ -26,6 +26,7 @@ struct KParams {
   int U;                  // units per (token, plane)
   int unit_chunks;        // VEC-byte chunks per unit
   int planar;             // wire order
+  int64_t plane_rows;     // PLANAR: rows between the planes of a slab, or -1 = total tokens T
   int window;             // 0, or the layer keeps only the last min(s, window) tokens
   int ppc, spr;           // vectorised family: page columns per CTA, CTAs per request
   int64_t num_pages;      // pages per pool slab: every page id is checked against it

@@ -204,11 +204,11 @@ __global__ void __launch_bounds__(MAXT, 1) topkv_crc_copy_kernel(const CrcCopyPa
   if (first < s_r) {
     const int v = min(p.P, s_r - first);
     const int64_t n0 = p.cu[r] + first;
-    const int64_t T = p.T >= 0 ? p.T : p.cu[p.R];
+    const int64_t T = p.plane_rows >= 0 ? p.plane_rows : (p.T >= 0 ? p.T : p.cu[p.R]);  // plane rows
     const int64_t row = (int64_t)cp.g.run_bytes * cp.g.rpr;
     const int64_t page = p.bt[(int64_t)r * p.maxp + j];
     const bool page_ok = page >= 0 && page < p.num_pages;
-    const bool fits = p.planar ? (n0 >= 0 && n0 + v <= T && T * F * row <= p.wire_limit)
+    const bool fits = p.planar ? (n0 >= 0 && ((F - 1) * T + n0 + v) * row <= p.wire_limit)
                                : (n0 >= 0 && (n0 + v) * F * row <= p.wire_limit);
     if (tid == 0 && !page_ok) raise_error(kErrTable);
     if (tid == 0 && !fits) raise_error(kErrWire);

@@ -81,12 +81,14 @@ __device__ __forceinline__ void copy_span(const KParams& p) {
   int64_t cu_r, T = p.T;
   if (p.cu != nullptr) {
     cu_r = p.cu[r];
-    if (p.planar && T < 0) T = p.cu[p.R];
+    if (p.planar && p.plane_rows < 0 && T < 0) T = p.cu[p.R];
   } else {
     int64_t total;
-    cu_r = block_prefix(p.sl, (p.planar && T < 0) ? p.R : r, r, p.window, &total);
-    if (p.planar && T < 0) T = total;
+    const bool need_T = p.planar && p.plane_rows < 0 && T < 0;
+    cu_r = block_prefix(p.sl, need_T ? p.R : r, r, p.window, &total);
+    if (need_T) T = total;
   }
+  const int64_t PR = p.plane_rows >= 0 ? p.plane_rows : T;  // rows from the K to the V plane
   if (tid >= jlo && tid <= jhi) {
     int pg = p.bt[(int64_t)r * p.maxp + j0 + tid];
     if (pg < 0 || pg >= p.num_pages) {  // unusable entry: the page is skipped, nothing is touched
@@ -100,7 +102,7 @@ __device__ __forceinline__ void copy_span(const KParams& p) {
   const int64_t unit_bytes = (int64_t)p.unit_chunks * VEC;
   {  // the span must lie inside the wire slab, whatever lengths the device tables hold
     const int64_t row = unit_bytes * p.U;
-    const bool fits = p.planar ? (n0 >= 0 && n0 + v <= T && T * F * row <= p.wire_limit)
+    const bool fits = p.planar ? (n0 >= 0 && ((F - 1) * PR + n0 + v) * row <= p.wire_limit)
                                : (n0 >= 0 && (n0 + v) * F * row <= p.wire_limit);
     if (!fits) {
       if (tid == 0) raise_error(kErrWire);
@@ -121,7 +123,7 @@ __device__ __forceinline__ void copy_span(const KParams& p) {
         uint8_t* a = pool_page + c * p.S_kv;
         // not planar => F == 1
         uint8_t* b = p.wire +
-                     ((p.planar ? c * T : 0) + n0 + (int64_t)(jj * p.P + t_lo - ts0)) * unit_bytes;
+                     ((p.planar ? c * PR : 0) + n0 + (int64_t)(jj * p.P + t_lo - ts0)) * unit_bytes;
         const uint8_t* src = PACK ? a : b;
         uint8_t* dst = PACK ? b : a;
         for (int w0 = tid; w0 < n; w0 += kThreads * kUnroll) {
@@ -172,7 +174,7 @@ __device__ __forceinline__ void copy_span(const KParams& p) {
         if (p.planar) {
           c = (F > 1 && tc >= v) ? 1 : 0;
           ts = tc - c * v;
-          b = p.wire + (((int64_t)c * T + n0 + ts) * p.U + h) * unit_bytes + (int64_t)w * VEC;
+          b = p.wire + (((int64_t)c * PR + n0 + ts) * p.U + h) * unit_bytes + (int64_t)w * VEC;
         } else {
           ts = tc / F;
           c = tc - ts * F;

@@ -36,8 +36,8 @@ def test_exports_every_declared_symbol():
 
 
 def test_struct_sizes_match_header():
-    # natural alignment of the C structs: 10 x u32 + 7 x i64, and 4 x 32-bit + 3 ptr + i64
-    assert ctypes.sizeof(tk.topkv_layout) == 96
+    # natural alignment of the C structs: 10 x u32 + 8 x i64, and 4 x 32-bit + 3 ptr + i64 + 2 x i32
+    assert ctypes.sizeof(tk.topkv_layout) == 104
     assert ctypes.sizeof(tk.topkv_batch) == 56
     assert ctypes.sizeof(tk.topkv_layer_spec) == 16
 
@@ -125,6 +125,14 @@ def test_argument_validation_without_gpu():
     assert P(0, pool, bad, b, wire, cap) == tk.TOPKV_ERR_UNSUPPORTED_LAYOUT
     bad = _gqa(); bad.wire_order = 7
     assert P(0, pool, bad, b, wire, cap) == tk.TOPKV_ERR_UNSUPPORTED_LAYOUT
+    bad = _gqa(); bad.wire_plane_stride = 4096               # spread planes need the PLANAR order
+    assert P(0, pool, bad, b, wire, cap) == tk.TOPKV_ERR_UNSUPPORTED_LAYOUT
+    bad = _gqa(wire_order=tk.TOPKV_WIRE_PLANAR); bad.wire_plane_stride = 2048 * 436 + 16
+    assert P(0, pool, bad, b, wire, cap) == tk.TOPKV_ERR_UNSUPPORTED_LAYOUT   # not whole rows
+    bad = _gqa(wire_order=tk.TOPKV_WIRE_PLANAR); bad.wire_plane_stride = 2048 * 1000
+    assert P(0, pool, bad, b, wire, 2048 * 1000 + 436 * 2048 - 1) == tk.TOPKV_ERR_CAPACITY
+    assert tk.topkv_pack_layer_to_host(0, pool, bad, b, wire, 1 << 40, 0xA000000, 1 << 40) \
+        == tk.TOPKV_ERR_UNSUPPORTED_LAYOUT
     bad = _gqa(); bad.pool_token_stride = 2048 + 8
     assert P(0, pool, bad, b, wire, cap) == tk.TOPKV_ERR_ALIGNMENT
     bad = tk.make_layout(2, 2, 1, 4, 2, 16, 8)               # 8-byte rows

@@ -137,6 +137,7 @@ def _layout_from_geom(g: Geom):
                         kind=tk.TOPKV_KIND_GQA)
     lo.pool_layer_stride, lo.pool_page_stride, lo.pool_kv_stride = g.S_layer, g.S_page, g.S_kv
     lo.pool_token_stride, lo.pool_head_stride = g.S_tok, g.S_head
+    lo.wire_plane_stride = g.W_plane
     return lo
 
 
@@ -671,6 +672,61 @@ def test_crc_cfg1_header_round_trip_and_corruption(dev, variant):
 
     assert tk.topkv_retry(transfer, retries=2, backoff_ms=1) == tk.TOPKV_OK
     assert len(attempts) == 2
+
+
+def test_paper_payload_one_request_end_to_end(dev, variant):
+    """§3.4 end to end for one request: 128-byte header, then the K tensor
+    [layers][seq_len][kv_heads][head_dim], then the V tensor, assembled by per-layer PLANAR
+    packs (layer stride = one plane, plane stride = L planes); the header's checksums come from
+    the checksummed copy and equal the host CRC-64 of the payload's two halves."""
+    rng = np.random.default_rng(91)
+    L, H, D, P, s_len = 5, 8, 128, 16, 333
+    npages = 40
+    g = Geom(L=L, F=2, h_kv=H, d_h=D, b_p=2, P=P, num_pages=npages, wire_order=1)
+    plane = s_len * g.row_bytes
+    g.W_layer, g.W_plane = plane, L * plane
+    sl = np.array([s_len], dtype=np.int32)
+    bt = rng.permutation(npages)[:21].astype(np.int32).reshape(1, 21)
+    lo = _layout_from_geom(g)
+    src_h = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
+    src = torch.from_numpy(src_h).to(dev)
+    d_sl, d_bt = torch.from_numpy(sl).to(dev), torch.from_numpy(bt).to(dev)
+    cu = torch.zeros(2, dtype=torch.int64, device=dev)
+    tk.check(tk.topkv_build_plan(tk.make_batch(d_bt, d_sl), cu))
+    batch = tk.make_batch(d_bt, d_sl, s_len, cu)
+    message = torch.zeros(128 + 2 * L * plane, dtype=torch.uint8, device=dev)
+    payload = message[128:]
+    want = np.zeros(2 * L * plane, dtype=np.uint8)
+    for layer in range(L):
+        oracle.pack(g, layer, src_h, bt, sl, wire=want)
+    # plain pack (both kernel families)
+    for layer in range(L):
+        tk.check(tk.topkv_pack_layer(layer, src, lo, batch, payload, payload.numel()))
+    torch.cuda.synchronize()
+    assert np.array_equal(payload.cpu().numpy(), want)
+    # checksummed pack into a fresh message, header built from the device checksums
+    payload.zero_()
+    nws = tk.topkv_crc_workspace_bytes(lo, 1, 21)
+    ws = torch.zeros(nws, dtype=torch.uint8, device=dev)
+    crc = torch.zeros(2, dtype=torch.int64, device=dev)
+    tk.check(tk.topkv_crc_begin(lo, batch, ws, nws))
+    for layer in range(L):
+        tk.check(tk.topkv_pack_layer_crc(layer, src, lo, batch, payload, payload.numel(), ws, nws))
+    tk.check(tk.topkv_crc_finish(lo, batch, ws, nws, crc))
+    torch.cuda.synchronize()
+    crc_k, crc_v = (int(x) for x in crc.cpu().numpy().view(np.uint64))
+    h = tk.topkv_wire_header()
+    tk.check(tk.topkv_header_fill(h, 77, 5, lo, s_len, crc_k, crc_v))
+    message[:128] = torch.frombuffer(bytearray(bytes(h)), dtype=torch.uint8).to(dev)
+    msg = message.cpu().numpy()
+    assert bytes(msg[:8]) == b"KVCACHE1" and np.array_equal(msg[128:], want)
+    k_bytes = L * plane
+    assert tk.topkv_crc64(np.ascontiguousarray(msg[128:128 + k_bytes])) == crc_k
+    assert tk.topkv_crc64(np.ascontiguousarray(msg[128 + k_bytes:])) == crc_v
+    assert crc_k == oracle.kv_plane_crc(g, src_h, bt, sl, 0, 0) == oracle.crc64(want[:k_bytes])
+    assert crc_v == oracle.kv_plane_crc(g, src_h, bt, sl, 0, 1) == oracle.crc64(want[k_bytes:])
+    assert bytes(msg[:128]) == oracle.build_header(77, 5, s_len, g, crc_k, crc_v)
+    assert h.k_bytes == k_bytes
 
 
 # -------------------------------------------------------------------- direct re-paging
