@@ -621,10 +621,10 @@ int topkv_crc_begin(const topkv_layout* layout, const topkv_batch* batch, void* 
   if (workspace_bytes < 8 * crc_workspace_words(g.RB, L, R, maxp, F)) return TOPKV_ERR_CAPACITY;
   if (R == 0) return TOPKV_OK;
   const CrcWorkspace w = crc_carve(d_workspace, g.RB, L, R, maxp, F);
-  const int64_t total = (int64_t)g.RB + maxp + 1 + 2 * (int64_t)R + (int64_t)L * R;
+  const int64_t total = (int64_t)g.RB + maxp + 1 + 2 * (int64_t)R + (int64_t)L * R * F;
   const unsigned blocks = (unsigned)std::min<int64_t>((total + 255) / 256, 1024);
   topkv_crc_begin_kernel<<<blocks, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
-      w, g, batch->seq_lens, L, R, maxp, (int)layout->page_tokens, rs.row_bytes);
+      w, g, batch->seq_lens, L, R, maxp, (int)layout->page_tokens, rs.row_bytes, F);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   g_launches.fetch_add(1, std::memory_order_relaxed);

@@ -8,8 +8,8 @@
 // into runs (a fraction of a token row); every thread owns one run: while the warp moves the
 // data from source to destination it folds its run into a 64-bit remainder, multiplies that by
 // x^(8 * bytes that follow the run inside its page), and the page's threads XOR their results.
-// The CTA that finishes the last page of a request aligns the page remainders inside the
-// request's plane and stores the layer's remainder; topkv_crc_finish chains the layers:
+// Each page then aligns its remainder inside the request's plane and XORs it into the layer's
+// remainder (one atomic per page and plane); topkv_crc_finish chains the layers:
 //   state_0 = ~0,  state_l+1 = state_l * x^(8 * bytes of the plane in one layer) + rem_l,
 // and the checksum is ~state_L.
 //
@@ -73,18 +73,14 @@ __host__ __device__ inline uint64_t gf_powx(uint64_t n) {
 // c_page   [maxp + 1]      x^(8 * P * row_bytes * k)
 // x_req    [R]             x^(8 * s_r * row_bytes)        (per batch)
 // x_last   [R]             x^(8 * v_last(r) * row_bytes)  (per batch)
-// layer_rem[L * R * F]     remainder of request r, plane c, layer l (written by the last CTA
-//                          of that request and layer)
-// page_rem [L * R * maxp * F]  remainder of every page and plane, per layer
-// done     [L * R] (int32) pages of request r finished in layer l
+// layer_rem[L * R * F]     remainder of request r, plane c in layer l: every page's CTA XORs its
+//                          aligned page remainder in (atomicXor), so it starts at zero
 struct CrcWorkspace {
   uint64_t* c_run;
   uint64_t* c_page;
   uint64_t* x_req;
   uint64_t* x_last;
-  uint64_t* layer_rem;
-  uint64_t* page_rem;
-  int32_t* done;
+  unsigned long long* layer_rem;
 };
 
 struct CrcGeom {
@@ -94,29 +90,28 @@ struct CrcGeom {
 };
 
 __host__ __device__ inline int64_t crc_workspace_words(int RB, int L, int R, int maxp, int F) {
-  return (int64_t)RB + (maxp + 1) + 2 * (int64_t)R + (int64_t)L * R * F +
-         (int64_t)L * R * maxp * F + ((int64_t)L * R + 1) / 2;
+  return (int64_t)RB + (maxp + 1) + 2 * (int64_t)R + (int64_t)L * R * F;
 }
 
 __host__ __device__ inline CrcWorkspace crc_carve(void* base, int RB, int L, int R, int maxp, int F) {
+  (void)L;
+  (void)F;
   CrcWorkspace w;
   w.c_run = static_cast<uint64_t*>(base);
   w.c_page = w.c_run + RB;
   w.x_req = w.c_page + (maxp + 1);
   w.x_last = w.x_req + R;
-  w.layer_rem = w.x_last + R;
-  w.page_rem = w.layer_rem + (int64_t)L * R * F;
-  w.done = reinterpret_cast<int32_t*>(w.page_rem + (int64_t)L * R * maxp * F);
+  w.layer_rem = reinterpret_cast<unsigned long long*>(w.x_last + R);
   return w;
 }
 
-// Builds the constant tables for this batch and clears the per-layer page counters.
+// Builds the constant tables for this batch and clears the per-layer remainders.
 __global__ void __launch_bounds__(256)
 topkv_crc_begin_kernel(CrcWorkspace w, CrcGeom g, const int32_t* __restrict__ sl, int L, int R,
-                       int maxp, int P, int64_t row_bytes) {
+                       int maxp, int P, int64_t row_bytes, int F) {
   pdl_prologue(0);
   const int64_t n_run = g.RB, n_page = maxp + 1;
-  const int64_t total = n_run + n_page + 2 * (int64_t)R + (int64_t)L * R;
+  const int64_t total = n_run + n_page + 2 * (int64_t)R + (int64_t)L * R * F;
   for (int64_t k = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; k < total;
        k += (int64_t)gridDim.x * blockDim.x) {
     if (k < n_run) {
@@ -133,7 +128,7 @@ topkv_crc_begin_kernel(CrcWorkspace w, CrcGeom g, const int32_t* __restrict__ sl
       if (q & 1) w.x_last[r] = gf_powx(8ull * (uint64_t)v_last * row_bytes);
       else w.x_req[r] = gf_powx(8ull * (uint64_t)s * row_bytes);
     } else {
-      w.done[k - n_run - n_page - 2 * (int64_t)R] = 0;
+      w.layer_rem[k - n_run - n_page - 2 * (int64_t)R] = 0ull;
     }
   }
 }
@@ -286,31 +281,16 @@ __global__ void __launch_bounds__(MAXT, 1) topkv_crc_copy_kernel(const CrcCopyPa
       atomicXor(&s_rem[c], (unsigned long long)rem);
     }
     __syncthreads();
-    // Publish this page's remainders; the CTA that finishes the request's last page folds them.
-    uint64_t* page_rem = cp.w.page_rem + ((int64_t)cp.layer * p.R + r) * p.maxp * F;
-    const int n_r = (s_r + p.P - 1) / p.P;
-    if (tid < F) page_rem[(int64_t)j * F + tid] = page_ok && fits ? s_rem[tid] : 0ull;
-    __threadfence();
-    __syncthreads();
-    __shared__ int s_last;
-    if (tid == 0) s_last = atomicAdd(&cp.w.done[(int64_t)cp.layer * p.R + r], 1) == n_r - 1;
-    __syncthreads();
-    if (s_last) {
-      __threadfence();
-      if (tid < 2) s_rem[tid] = 0ull;
-      __syncthreads();
-      const uint64_t x_last = cp.w.x_last[r];
-      for (int k = tid; k < n_r * F; k += blockDim.x) {
-        const int jj = k / F, cc = k - jj * F;
-        uint64_t v2 = __ldcg(&page_rem[(int64_t)jj * F + cc]);
-        if (jj < n_r - 1) {  // followed by n_r - 2 - jj full pages and the last, possibly partial, page
-          v2 = gf_mulmod(v2, cp.w.c_page[n_r - 2 - jj]);
-          v2 = gf_mulmod(v2, x_last);
-        }
-        atomicXor(&s_rem[cc], (unsigned long long)v2);
+    // Align this page's remainder inside the request's plane (n_r - 2 - j full pages and the
+    // last, possibly partial, page follow it) and add it to the layer's remainder.
+    if (tid < F && page_ok && fits) {
+      const int n_r = (s_r + p.P - 1) / p.P;
+      uint64_t v2 = s_rem[tid];
+      if (j < n_r - 1) {
+        v2 = gf_mulmod(v2, cp.w.c_page[n_r - 2 - j]);
+        v2 = gf_mulmod(v2, cp.w.x_last[r]);
       }
-      __syncthreads();
-      if (tid < F) cp.w.layer_rem[((int64_t)cp.layer * p.R + r) * F + tid] = s_rem[tid];
+      atomicXor(&cp.w.layer_rem[((int64_t)cp.layer * p.R + r) * F + tid], (unsigned long long)v2);
     }
   }
   pdl_epilogue(p.overlap);
@@ -330,7 +310,7 @@ topkv_crc_finish_kernel(CrcWorkspace w, const int32_t* __restrict__ sl, int L, i
   const uint64_t x_req = w.x_req[r];
   uint64_t state = ~0ull;
   for (int l = 0; l < L; ++l) {
-    const uint64_t rem = empty ? 0ull : w.layer_rem[((int64_t)l * R + r) * F + c];
+    const uint64_t rem = empty ? 0ull : (uint64_t)w.layer_rem[((int64_t)l * R + r) * F + c];
     state = gf_mulmod(state, x_req) ^ rem;
   }
   out[k] = ~state;

@@ -222,8 +222,8 @@ def test_host_crc64_header_and_retry():
     assert tk.topkv_retry(lambda: (calls.append(0), tk.TOPKV_ERR_CHECKSUM)[1], 2, 1) \
         == tk.TOPKV_ERR_CHECKSUM and len(calls) == 3                     # gives up after 1 + 2
     # workspace sizing and unsupported shapes
-    assert tk.topkv_crc_workspace_bytes(lo, 8, 256) == 8 * (32 + 257 + 16 + 80 * 8 * 2 + 80 * 8 * 256 * 2 + 80 * 8 // 2)
-    assert tk.topkv_crc_workspace_bytes(mla, 32, 128) == 8 * (128 + 129 + 64 + 61 * 32 + 61 * 32 * 128 + (61 * 32 + 1) // 2)
+    assert tk.topkv_crc_workspace_bytes(lo, 8, 256) == 8 * (32 + 257 + 16 + 80 * 8 * 2)
+    assert tk.topkv_crc_workspace_bytes(mla, 32, 128) == 8 * (128 + 129 + 64 + 61 * 32)
     big = tk.make_layout(2, 2, 8, 128, 2, 512, 4)                    # 2 * 512 * 2 runs > 1024 threads
     assert tk.topkv_crc_workspace_bytes(big, 1, 1) == tk.TOPKV_ERR_UNSUPPORTED_LAYOUT
 
