@@ -884,7 +884,9 @@ def test_side_stream_overlap_run_is_bit_exact(dev, variant):
     for st in (staging, None):
         pinned = torch.zeros(slots * w.n_layer, dtype=torch.uint8).pin_memory()
         r = overlap.run_overlap(w, pinned, st, pre, slots=slots, warmup_layers=1)
-        assert r.layers == 6 and r.t_xfer_serial_ms > 0 and 0.0 <= r.hidden <= 1.0
+        # timing figures are only sanity-checked: on a cold box the overlapped pass can be slower
+        # than the serial one, so the hidden fraction of this tiny case may even be negative
+        assert r.layers == 6 and r.t_xfer_serial_ms > 0 and r.exposed_ms >= 0 and r.hidden <= 1.0
         assert r.hidden_upper_bound == pytest.approx(1 - 1 / 6)
         # the ring holds the last `slots` layers: 2, 3 in slots 2, 3 and 4, 5 in slots 0, 1
         for layer in (2, 3, 4, 5):
