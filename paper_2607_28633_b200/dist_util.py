@@ -17,9 +17,11 @@ def env_rank_world():
 
 def init(backend: str, device=None):
     """Initialises the default process group from the torchrun environment (MASTER_ADDR /
-    MASTER_PORT / RANK / WORLD_SIZE); returns the module, or None for a single process."""
+    MASTER_PORT / RANK / WORLD_SIZE), also for a world of one, so that the N = 1 leg of a
+    scaling run goes through the same calls; returns the module, or None for a plain process."""
     rank, world, _ = env_rank_world()
-    if world <= 1:
+    launched = "RANK" in os.environ and "MASTER_ADDR" in os.environ   # under torchrun
+    if world <= 1 and not launched:
         return None
     import torch.distributed as dist
     if not dist.is_initialized():
