@@ -898,6 +898,35 @@ def test_side_stream_overlap_run_is_bit_exact(dev, variant):
     torch.cuda.empty_cache()
 
 
+def test_relay_through_host_on_two_streams(dev):
+    """pack_to_host on one stream, unpack_from_host on another, gated per layer by an event:
+    the destination pool ends up as the oracle's unpack of the oracle's pack."""
+    spec = wl.with_layers(wl.CFG2, 3)
+    w = harness.setup(spec, dev)
+    b = w.batch
+    g = _geom(spec, b.num_pool_pages, 1, 0, 0)
+    tx, rx = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    pinned = torch.zeros(3 * w.n_layer, dtype=torch.uint8).pin_memory()
+    st_tx = torch.zeros(w.n_layer, dtype=torch.uint8, device=dev)
+    st_rx = torch.zeros(w.n_layer, dtype=torch.uint8, device=dev)
+    before = [harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, l) for l in range(3)]
+    for layer in range(3):
+        w.pack_to_host(layer, pinned, st_tx, tx)
+        ev = torch.cuda.Event()
+        ev.record(tx)
+        rx.wait_event(ev)
+        w.unpack_from_host(layer, pinned, st_rx, rx)
+    torch.cuda.synchronize()
+    for layer in range(3):
+        src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, layer)
+        want = oracle.pack(g, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=8)
+        assert np.array_equal(pinned[layer * w.n_layer:(layer + 1) * w.n_layer].numpy(), want)
+        oracle.unpack(g, 0, before[layer], b.dst_block_table, b.seq_lens, want, impl="rows", threads=8)
+        assert np.array_equal(harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, layer), before[layer])
+    del w
+    torch.cuda.empty_cache()
+
+
 def test_smoke_entry(dev):
     import __graft_entry__ as entry
     entry.smoke()
