@@ -16,8 +16,8 @@
 // Register convention (reflected): bit i of a 64-bit value is the coefficient of x^(63 - i);
 // multiplying by x is a right shift. A little-endian 64-bit load of eight message bytes is
 // their polynomial in this convention. Because the generator is sparse, x^64 = x^4+x^3+x+1
-// (mod P) and a multiplication by x^64 costs a handful of shifts and XORs: no table, no
-// shared memory, pure integer ALU work (B200 has no carry-less multiply).
+// (mod P) and a multiplication by x^64 costs a handful of shifts and XORs: no lookup table,
+// pure integer ALU work (B200 has no carry-less multiply).
 #pragma once
 #include <cuda_runtime.h>
 
