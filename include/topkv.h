@@ -246,6 +246,18 @@ int topkv_unpack_layer_crc(int layer, void* dst_pool, const topkv_layout* layout
                            void* d_workspace, int64_t workspace_bytes, topkv_stream_t stream);
 int topkv_crc_finish(const topkv_layout* layout, const topkv_batch* batch, void* d_workspace,
                      int64_t workspace_bytes, uint64_t* d_crc_out, topkv_stream_t stream);
+/* The host leg with checksums: topkv_pack_layer_to_host / topkv_unpack_layer_from_host with the
+ * checksummed copy as their kernel (same staged and direct forms, same rules), so that the
+ * sender checksums while it ships a layer and the receiver while it places it. */
+int topkv_pack_layer_to_host_crc(int layer, const void* src_pool, const topkv_layout* layout,
+                                 const topkv_batch* batch, void* h_pinned, int64_t host_capacity_bytes,
+                                 void* d_staging, int64_t staging_capacity_bytes, void* d_workspace,
+                                 int64_t workspace_bytes, topkv_stream_t stream);
+int topkv_unpack_layer_from_host_crc(int layer, void* dst_pool, const topkv_layout* layout,
+                                     const topkv_batch* batch, const void* h_pinned, int64_t host_bytes,
+                                     void* d_staging, int64_t staging_capacity_bytes,
+                                     void* d_workspace, int64_t workspace_bytes,
+                                     topkv_stream_t stream);
 
 /* Host-side retry policy of the transfer orchestrator (§3.1: 2 retries, 100 ms exponential
  * backoff): calls attempt(ctx) until it returns TOPKV_OK, at most 1 + retries times, sleeping

@@ -41,7 +41,7 @@ EXPORTS = (
     "topkv_reset_device_error_flags", "topkv_repage_layer", "topkv_kv_bytes_layered",
     "topkv_header_fill", "topkv_header_check", "topkv_crc64", "topkv_crc_workspace_bytes",
     "topkv_crc_begin", "topkv_pack_layer_crc", "topkv_unpack_layer_crc", "topkv_crc_finish",
-    "topkv_retry",
+    "topkv_retry", "topkv_pack_layer_to_host_crc", "topkv_unpack_layer_from_host_crc",
 )
 
 
@@ -126,6 +126,9 @@ def lib() -> ctypes.CDLL:
         L.topkv_unpack_layer_crc.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p,
                                              c_int64, c_void_p]
         L.topkv_crc_finish.argtypes = [lp, bp, c_void_p, c_int64, c_void_p, c_void_p]
+        for fn in (L.topkv_pack_layer_to_host_crc, L.topkv_unpack_layer_from_host_crc):
+            fn.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p, c_int64, c_void_p,
+                           c_int64, c_void_p]
         L.topkv_retry.argtypes = [RETRY_ATTEMPT, c_void_p, c_int, c_int]
         L.topkv_repage_layer.argtypes = [c_int, c_void_p, lp, bp, c_void_p, lp, bp, c_void_p]
         L.topkv_pack_layer_to_host_noalloc.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64,
@@ -305,6 +308,23 @@ def topkv_unpack_layer_crc(layer, dst_pool, layout, batch, d_wire, wire_bytes, d
 def topkv_crc_finish(layout, batch, d_workspace, workspace_bytes, d_crc_out, stream=None):
     return lib().topkv_crc_finish(ctypes.byref(layout), ctypes.byref(batch), _ptr(d_workspace),
                                   workspace_bytes, _ptr(d_crc_out), _stream(stream))
+
+
+def topkv_pack_layer_to_host_crc(layer, src_pool, layout, batch, h_pinned, host_capacity_bytes,
+                                 d_staging, staging_capacity_bytes, d_workspace, workspace_bytes,
+                                 stream=None):
+    return lib().topkv_pack_layer_to_host_crc(
+        layer, _ptr(src_pool), ctypes.byref(layout), ctypes.byref(batch), _ptr(h_pinned),
+        host_capacity_bytes, _ptr(d_staging), staging_capacity_bytes, _ptr(d_workspace),
+        workspace_bytes, _stream(stream))
+
+
+def topkv_unpack_layer_from_host_crc(layer, dst_pool, layout, batch, h_pinned, host_bytes,
+                                     d_staging, staging_capacity_bytes, d_workspace,
+                                     workspace_bytes, stream=None):
+    return lib().topkv_unpack_layer_from_host_crc(
+        layer, _ptr(dst_pool), ctypes.byref(layout), ctypes.byref(batch), _ptr(h_pinned), host_bytes,
+        _ptr(d_staging), staging_capacity_bytes, _ptr(d_workspace), workspace_bytes, _stream(stream))
 
 
 def topkv_retry(attempt, retries=2, backoff_ms=100):

@@ -338,12 +338,17 @@ int crc_geometry(const topkv_layout* lo, const Resolved& rs, CrcGeom* g) {
 
 template <bool PACK>
 int crc_copy(int layer, const void* pool, const topkv_layout* lo, const topkv_batch* b,
-             const void* wire, int64_t cap, void* ws, int64_t ws_bytes, cudaStream_t stream) {
+             const void* wire, int64_t cap, void* ws, int64_t ws_bytes, cudaStream_t stream,
+             void* slab_override = nullptr, int64_t* n_layer_out = nullptr) {
+  // slab_override: device address to use for this layer's wire slab instead of
+  // wire + layer*stride (a staging slab, or the device view of a pinned host slab)
   CrcCopyParams cp;
   Resolved rs;
   int64_t n_layer;
   int st = prepare(layer, pool, lo, b, wire, cap, lo ? lo->wire_layer_stride : 0, &cp.k, &rs, &n_layer);
   if (st != TOPKV_OK) return st;
+  if (n_layer_out != nullptr) *n_layer_out = n_layer;
+  if (slab_override != nullptr) cp.k.wire = static_cast<uint8_t*>(slab_override);
   if (ws == nullptr || !mult16p(ws)) return TOPKV_ERR_INVALID_ARG;
   if (b->cu_seq_lens == nullptr || b->window_tokens != 0) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
   st = crc_geometry(lo, rs, &cp.g);
@@ -379,6 +384,44 @@ int crc_copy(int layer, const void* pool, const topkv_layout* lo, const topkv_ba
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   g_launches.fetch_add(1, std::memory_order_relaxed);
+  return TOPKV_OK;
+}
+
+// Host leg with checksums: the same two forms as the plain host-leg calls.
+template <bool PACK>
+int crc_host_leg(int layer, const void* pool, const topkv_layout* layout,
+                        const topkv_batch* batch, const void* h_pinned, int64_t host_bytes,
+                        void* d_staging, int64_t staging_capacity_bytes, void* ws, int64_t ws_bytes,
+                        cudaStream_t s) {
+  if (layout == nullptr || batch == nullptr || h_pinned == nullptr) return TOPKV_ERR_INVALID_ARG;
+  if (d_staging == nullptr) {  // direct: the kernel works on the mapped pinned slab
+    void* dev = nullptr;
+    int st = mapped_device_pointer(h_pinned, &dev);
+    if (st != TOPKV_OK) return st;
+    void* slab = static_cast<uint8_t*>(dev) + (int64_t)layer * layout->wire_layer_stride;
+    return crc_copy<PACK>(layer, pool, layout, batch, h_pinned, host_bytes, ws, ws_bytes, s, slab);
+  }
+  if (batch->struct_size == sizeof(topkv_batch) && batch->total_tokens < 0) return TOPKV_ERR_INVALID_ARG;
+  if (layout->struct_size == sizeof(topkv_layout) && layout->wire_plane_stride != 0)
+    return TOPKV_ERR_UNSUPPORTED_LAYOUT;  // one contiguous copy
+  if (!mult16p(d_staging)) return TOPKV_ERR_ALIGNMENT;
+  const uint8_t* host_slab = static_cast<const uint8_t*>(h_pinned) + (int64_t)layer * layout->wire_layer_stride;
+  const int64_t n_known = topkv_wire_layer_bytes(layout, batch->total_tokens);
+  if (n_known < 0) return TOPKV_ERR_INVALID_ARG;
+  if (staging_capacity_bytes < n_known) return TOPKV_ERR_CAPACITY;
+  if (!PACK && n_known > 0) {  // bring the slab in first
+    const cudaError_t e = cudaMemcpyAsync(d_staging, host_slab, (size_t)n_known, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  int64_t n_layer = -1;
+  const int st = crc_copy<PACK>(layer, pool, layout, batch, h_pinned, host_bytes, ws, ws_bytes, s,
+                                d_staging, &n_layer);
+  if (st != TOPKV_OK) return st;
+  if (PACK && n_layer > 0) {
+    const cudaError_t e = cudaMemcpyAsync(const_cast<uint8_t*>(host_slab), d_staging, (size_t)n_layer,
+                                          cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
   return TOPKV_OK;
 }
 
@@ -589,6 +632,25 @@ int topkv_repage_layer(int layer, const void* src_pool, const topkv_layout* src_
   if (e != cudaSuccess) return cuda_fail(e);
   g_launches.fetch_add(1, std::memory_order_relaxed);
   return TOPKV_OK;
+}
+
+int topkv_pack_layer_to_host_crc(int layer, const void* src_pool, const topkv_layout* layout,
+                                 const topkv_batch* batch, void* h_pinned, int64_t host_capacity_bytes,
+                                 void* d_staging, int64_t staging_capacity_bytes, void* d_workspace,
+                                 int64_t workspace_bytes, topkv_stream_t stream) {
+  return crc_host_leg<true>(layer, src_pool, layout, batch, h_pinned, host_capacity_bytes, d_staging,
+                            staging_capacity_bytes, d_workspace, workspace_bytes,
+                            reinterpret_cast<cudaStream_t>(stream));
+}
+
+int topkv_unpack_layer_from_host_crc(int layer, void* dst_pool, const topkv_layout* layout,
+                                     const topkv_batch* batch, const void* h_pinned, int64_t host_bytes,
+                                     void* d_staging, int64_t staging_capacity_bytes,
+                                     void* d_workspace, int64_t workspace_bytes,
+                                     topkv_stream_t stream) {
+  return crc_host_leg<false>(layer, dst_pool, layout, batch, h_pinned, host_bytes, d_staging,
+                             staging_capacity_bytes, d_workspace, workspace_bytes,
+                             reinterpret_cast<cudaStream_t>(stream));
 }
 
 int64_t topkv_crc_workspace_bytes(const topkv_layout* layout, int32_t num_requests,

@@ -64,9 +64,11 @@ class PrefillStandIn:
 
 def run_overlap(w: DeviceWorkload, h_pinned: torch.Tensor, staging, prefill: PrefillStandIn,
                 layers: int | None = None, slots: int | None = None,
-                warmup_layers: int = 3) -> OverlapResult:
+                warmup_layers: int = 3, crc_workspace=None) -> OverlapResult:
     """h_pinned holds ``slots`` wire slabs (a ring when slots < layers); w.layout must have
-    wire_layer_stride == n_layer. Returns the event-timed overlap figures."""
+    wire_layer_stride == n_layer. With ``crc_workspace`` (a device buffer prepared by
+    topkv_crc_begin) every transfer also checksums the layer (topkv_pack_layer_to_host_crc).
+    Returns the event-timed overlap figures."""
     dev = w.src_pool.device
     L = w.layers if layers is None else layers
     n = w.n_layer
@@ -85,8 +87,14 @@ def run_overlap(w: DeviceWorkload, h_pinned: torch.Tensor, staging, prefill: Pre
 
     def xfer(l, stream):
         slab = h_pinned[(l % slots) * n:(l % slots + 1) * n]
-        tk.check(tk.topkv_pack_layer_to_host(l, w.src_pool, lo, w.src_batch, slab, n, staging,
-                                             0 if staging is None else staging.numel(), stream))
+        cap = 0 if staging is None else staging.numel()
+        if crc_workspace is None:
+            tk.check(tk.topkv_pack_layer_to_host(l, w.src_pool, lo, w.src_batch, slab, n, staging,
+                                                 cap, stream))
+        else:
+            tk.check(tk.topkv_pack_layer_to_host_crc(l, w.src_pool, lo, w.src_batch, slab, n, staging,
+                                                     cap, crc_workspace, crc_workspace.numel(),
+                                                     stream))
 
     def ev():
         return torch.cuda.Event(enable_timing=True)

@@ -729,6 +729,43 @@ def test_paper_payload_one_request_end_to_end(dev, variant):
     assert h.k_bytes == k_bytes
 
 
+@pytest.mark.parametrize("staged", [True, False])
+def test_host_leg_with_checksums(dev, staged, variant):
+    """Sender: pack to pinned host memory with checksums; receiver: unpack from it with
+    checksums. Bytes and both sets of checksums equal the oracle's."""
+    if variant == 1:
+        pytest.skip("the checksumming copy has one kernel family")
+    w = harness.setup(wl.CFG1, dev)
+    b, s = w.batch, wl.CFG1
+    g = _geom(s, b.num_pool_pages, s.L, 0, w.n_layer)
+    src_h, dst_h = w.src_pool.cpu().numpy(), w.dst_pool.cpu().numpy()
+    pinned = torch.zeros(s.L * w.n_layer, dtype=torch.uint8).pin_memory()
+    staging = torch.zeros(w.n_layer, dtype=torch.uint8, device=dev) if staged else None
+    cap = w.n_layer if staged else 0
+    nws = tk.topkv_crc_workspace_bytes(w.layout, s.R, b.max_pages_per_req)
+    got = []
+    for fn, pool, batch in ((tk.topkv_pack_layer_to_host_crc, w.src_pool, w.src_batch),
+                            (tk.topkv_unpack_layer_from_host_crc, w.dst_pool, w.dst_batch)):
+        ws = torch.zeros(nws, dtype=torch.uint8, device=dev)
+        crc = torch.zeros(s.R * s.F, dtype=torch.int64, device=dev)
+        tk.check(tk.topkv_crc_begin(w.layout, batch, ws, nws))
+        for layer in range(s.L):
+            tk.check(fn(layer, pool, w.layout, batch, pinned, pinned.numel(), staging, cap, ws, nws))
+        tk.check(tk.topkv_crc_finish(w.layout, batch, ws, nws, crc))
+        torch.cuda.synchronize()
+        got.append(crc.cpu().numpy().view(np.uint64).reshape(s.R, s.F))
+    want_wire = np.zeros(s.L * w.n_layer, dtype=np.uint8)
+    for layer in range(s.L):
+        oracle.pack(g, layer, src_h, b.src_block_table, b.seq_lens, wire=want_wire)
+        oracle.unpack(g, layer, dst_h, b.dst_block_table, b.seq_lens, want_wire)
+    assert np.array_equal(pinned.numpy(), want_wire)
+    assert np.array_equal(w.dst_pool.cpu().numpy(), dst_h)
+    for r in range(s.R):
+        for c in range(s.F):
+            want = oracle.kv_plane_crc(g, src_h, b.src_block_table, b.seq_lens, r, c)
+            assert int(got[0][r, c]) == want and int(got[1][r, c]) == want
+
+
 # -------------------------------------------------------------------- direct re-paging
 
 def _repage_case(seed):
