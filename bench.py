@@ -591,9 +591,20 @@ def main():
     from paper_2607_28633_b200 import dist_util
     dev = torch.device("cuda", local)
     torch.cuda.set_device(dev)
-    dist = dist_util.init("nccl", dev)
-    if dist is not None:
-        dist.barrier()
+    # Keep stdout to the one JSON line: the communicator's set-up prints a version banner there,
+    # so file descriptor 1 points at stderr while the process group comes up.
+    sys.stdout.flush()
+    saved_stdout = os.dup(1)
+    os.dup2(2, 1)
+    try:
+        dist = dist_util.init("nccl", dev)
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize(dev)
+    finally:
+        sys.stdout.flush()
+        os.dup2(saved_stdout, 1)
+        os.close(saved_stdout)
     tk.lib()
     if args.variant is not None:
         tk.check(tk.topkv_set_kernel_variant(args.variant))
