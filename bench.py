@@ -527,8 +527,14 @@ def run_extra(name, dev, stream, args, peak):
         staging = torch.empty(w.n_layer, dtype=torch.uint8, device=dev)
         pre = overlap.PrefillStandIn(dev, w.batch.seeds["data"] + 50)
         best = None
-        for form, st in (("staged", staging), ("direct", None)):
+        # direct = mapped stores from a bounded grid (the library's default, 16 CTAs);
+        # direct_cta_per_span = the same stores from one CTA per page span, for contrast
+        for form, st, ctas in (("staged", staging, None), ("direct", None, None),
+                               ("direct_cta_per_span", None, 0)):
+            prev = tk.topkv_set_host_leg_ctas(ctas) if ctas is not None else None
             r = overlap.run_overlap(w, pinned, st, pre, slots=slots)
+            if prev is not None:
+                tk.topkv_set_host_leg_ctas(prev)
             d = r.as_dict()
             d["form"] = form
             d["hidden_model"] = round(min(1.0, (r.layers - 1) * r.t_layer_compute_ms

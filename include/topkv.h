@@ -369,6 +369,15 @@ int64_t topkv_kernel_launch_count(void);
  * 1 = bulk-async copies staged through shared memory. Returns the previous value, or
  * TOPKV_ERR_INVALID_ARG. Process-wide; intended for benchmarking, not for the hot path. */
 int topkv_set_kernel_variant(int variant);
+/* Grid of the DIRECT host leg (topkv_pack_layer_to_host / topkv_unpack_layer_from_host with
+ * d_staging == NULL), the PCIe transport of §3.3 / Table 4: n > 0 = at most n CTAs walk all
+ * spans of pages (default TOPKV_DEFAULT_HOST_LEG_CTAS); 0 = one CTA per span, as for a device
+ * wire. The PCIe link sets the pace of that leg, so a few CTAs keep it full while the rest of
+ * the GPU stays with the prefill that runs beside the transfer (§5.2). Returns the previous
+ * value, or TOPKV_ERR_INVALID_ARG for n < 0 or n > 65535. Process-wide; takes effect for calls
+ * made after it returns. The bytes moved are the same for every setting. */
+#define TOPKV_DEFAULT_HOST_LEG_CTAS 16
+int topkv_set_host_leg_ctas(int ctas);
 
 #ifdef __cplusplus
 }

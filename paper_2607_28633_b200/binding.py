@@ -42,6 +42,7 @@ EXPORTS = (
     "topkv_header_fill", "topkv_header_check", "topkv_crc64", "topkv_crc_workspace_bytes",
     "topkv_crc_begin", "topkv_pack_layer_crc", "topkv_unpack_layer_crc", "topkv_crc_finish",
     "topkv_retry", "topkv_pack_layer_to_host_crc", "topkv_unpack_layer_from_host_crc",
+    "topkv_set_host_leg_ctas",
 )
 
 
@@ -151,6 +152,7 @@ def lib() -> ctypes.CDLL:
         L.topkv_strerror.restype = ctypes.c_char_p
         L.topkv_kernel_launch_count.restype = c_int64
         L.topkv_set_kernel_variant.argtypes = [c_int]
+        L.topkv_set_host_leg_ctas.argtypes = [c_int]
         _lib = L
     return _lib
 
@@ -401,6 +403,10 @@ def topkv_reset_device_error_flags():
 
 def topkv_kernel_launch_count():
     return lib().topkv_kernel_launch_count()
+
+
+def topkv_set_host_leg_ctas(ctas):
+    return lib().topkv_set_host_leg_ctas(ctas)
 
 
 def topkv_set_kernel_variant(variant):

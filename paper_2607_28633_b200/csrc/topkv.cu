@@ -33,6 +33,10 @@ using namespace topkv;
 thread_local int g_last_cuda_error = 0;
 std::atomic<int64_t> g_launches{0};
 std::atomic<int> g_variant{0};
+// Direct host leg: 0 = one CTA per span, n = at most n CTAs walk the spans. 6 CTAs already keep
+// the link full in both directions; 16 leaves slack and still costs a concurrent GEMM nothing
+// measurable, where one CTA per span slowed it by 30 %.
+std::atomic<int> g_host_leg_ctas{TOPKV_DEFAULT_HOST_LEG_CTAS};
 
 inline bool mult16(int64_t x) { return (x & 15) == 0; }
 inline bool mult16p(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
@@ -152,8 +156,18 @@ int prepare(int layer, const void* pool, const topkv_layout* lo, const topkv_bat
 }
 
 template <bool PACK, int VEC, bool MULTI>
-void launch_vec2(const KParams& kp, bool merged, int F, dim3 grid, cudaStream_t stream) {
+void launch_vec2(const KParams& kp, bool merged, int F, dim3 grid, cudaStream_t stream, bool walk) {
   const dim3 block(kThreads);
+  if (walk) {  // bounded grid, every CTA walks several spans
+    if (merged) {
+      if (F == 1) launch_pdl(topkv_page_copy_walk_kernel<1, PACK, true, VEC, MULTI>, grid, block, 0, stream, kp);
+      else launch_pdl(topkv_page_copy_walk_kernel<2, PACK, true, VEC, MULTI>, grid, block, 0, stream, kp);
+    } else {
+      if (F == 1) launch_pdl(topkv_page_copy_walk_kernel<1, PACK, false, VEC, MULTI>, grid, block, 0, stream, kp);
+      else launch_pdl(topkv_page_copy_walk_kernel<2, PACK, false, VEC, MULTI>, grid, block, 0, stream, kp);
+    }
+    return;
+  }
   if (merged) {
     if (F == 1) launch_pdl(topkv_page_copy_kernel<1, PACK, true, VEC, MULTI>, grid, block, 0, stream, kp);
     else launch_pdl(topkv_page_copy_kernel<2, PACK, true, VEC, MULTI>, grid, block, 0, stream, kp);
@@ -164,9 +178,9 @@ void launch_vec2(const KParams& kp, bool merged, int F, dim3 grid, cudaStream_t 
 }
 
 template <bool PACK, int VEC>
-void launch_vec(const KParams& kp, bool merged, int F, dim3 grid, cudaStream_t stream) {
-  if (kp.ppc > 1) launch_vec2<PACK, VEC, true>(kp, merged, F, grid, stream);
-  else launch_vec2<PACK, VEC, false>(kp, merged, F, grid, stream);
+void launch_vec(const KParams& kp, bool merged, int F, dim3 grid, cudaStream_t stream, bool walk) {
+  if (kp.ppc > 1) launch_vec2<PACK, VEC, true>(kp, merged, F, grid, stream, walk);
+  else launch_vec2<PACK, VEC, false>(kp, merged, F, grid, stream, walk);
 }
 
 // ---- bulk-async family -------------------------------------------------------------------
@@ -236,12 +250,13 @@ int launch_bulk(const KParams& kp0, const Resolved& rs, int F, cudaStream_t stre
   return TOPKV_OK;
 }
 
+// max_ctas > 0: the wire is host memory behind PCIe; at most that many CTAs walk the spans.
 template <bool PACK>
-int launch_copy(KParams kp, const Resolved& rs, int F, cudaStream_t stream) {
+int launch_copy(KParams kp, const Resolved& rs, int F, cudaStream_t stream, int max_ctas = 0) {
   const int64_t slots = (int64_t)kp.R * kp.maxp;
   if (slots == 0) return TOPKV_OK;
   bool handled = false;
-  if (g_variant.load(std::memory_order_relaxed) == 1) {
+  if (max_ctas <= 0 && g_variant.load(std::memory_order_relaxed) == 1) {
     const int st = launch_bulk<PACK>(kp, rs, F, stream, &handled);
     if (st != TOPKV_OK) return st;
   }
@@ -250,17 +265,19 @@ int launch_copy(KParams kp, const Resolved& rs, int F, cudaStream_t stream) {
     kp.ppc = (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(kMaxPagesPerCta, kp.maxp),
                                                         kSpanTargetBytes / page_bytes));
     kp.spr = (kp.maxp + kp.ppc - 1) / kp.ppc;
-    const dim3 grid((unsigned)((int64_t)kp.R * kp.spr));
+    const int64_t spans = (int64_t)kp.R * kp.spr;
+    const bool walk = max_ctas > 0 && spans > max_ctas;
+    const dim3 grid((unsigned)(walk ? max_ctas : spans));
     // 32-byte vectors when every address the kernel can form is 32-byte aligned
     const bool wide = ((reinterpret_cast<uintptr_t>(kp.pool) | reinterpret_cast<uintptr_t>(kp.wire) |
                         (uintptr_t)kp.S_page | (uintptr_t)kp.S_kv | (uintptr_t)kp.S_tok |
                         (uintptr_t)kp.S_unit | (uintptr_t)rs.unit_bytes) & 31) == 0;
     if (wide) {
       kp.unit_chunks = (int)(rs.unit_bytes / 32);
-      launch_vec<PACK, 32>(kp, rs.merged, F, grid, stream);
+      launch_vec<PACK, 32>(kp, rs.merged, F, grid, stream, walk);
     } else {
       kp.unit_chunks = (int)(rs.unit_bytes / 16);
-      launch_vec<PACK, 16>(kp, rs.merged, F, grid, stream);
+      launch_vec<PACK, 16>(kp, rs.merged, F, grid, stream, walk);
     }
   }
   const cudaError_t e = cudaGetLastError();
@@ -469,7 +486,8 @@ int topkv_pack_layer_to_host(int layer, const void* src_pool, const topkv_layout
     st = mapped_device_pointer(h_pinned, &dev);
     if (st != TOPKV_OK) return st;
     kp.wire = static_cast<uint8_t*>(dev) + (int64_t)layer * layout->wire_layer_stride;
-    return launch_copy<true>(kp, rs, (int)layout->kv_factor, s);
+    return launch_copy<true>(kp, rs, (int)layout->kv_factor, s,
+                             g_host_leg_ctas.load(std::memory_order_relaxed));
   }
   // staged: pack this layer into the staging slab, then one copy-engine transfer
   if (batch != nullptr && batch->struct_size == sizeof(topkv_batch) && batch->total_tokens < 0)
@@ -507,7 +525,8 @@ int topkv_unpack_layer_from_host(int layer, void* dst_pool, const topkv_layout* 
     st = mapped_device_pointer(h_pinned, &dev);
     if (st != TOPKV_OK) return st;
     kp.wire = static_cast<uint8_t*>(dev) + (int64_t)layer * layout->wire_layer_stride;
-    return launch_copy<false>(kp, rs, (int)layout->kv_factor, s);
+    return launch_copy<false>(kp, rs, (int)layout->kv_factor, s,
+                              g_host_leg_ctas.load(std::memory_order_relaxed));
   }
   if (batch != nullptr && batch->struct_size == sizeof(topkv_batch) && batch->total_tokens < 0)
     return TOPKV_ERR_INVALID_ARG;
@@ -762,6 +781,11 @@ int topkv_device_error_flags(void) {
   return flags;
 }
 int64_t topkv_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int topkv_set_host_leg_ctas(int ctas) {
+  if (ctas < 0 || ctas > 65535) return TOPKV_ERR_INVALID_ARG;
+  return g_host_leg_ctas.exchange(ctas);
+}
 
 int topkv_set_kernel_variant(int variant) {
   if (variant < 0 || variant > 1) return TOPKV_ERR_INVALID_ARG;

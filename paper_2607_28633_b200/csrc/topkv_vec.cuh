@@ -55,11 +55,10 @@ __device__ __forceinline__ int64_t block_prefix(const int32_t* __restrict__ sl, 
 // wire -> pool; MERGED: the valid tokens of a page form one contiguous run per plane on
 // both sides (MLA rows, or PLANAR wire with a token-contiguous pool).
 template <int F, bool PACK, bool MERGED, int VEC, bool MULTI>
-__device__ __forceinline__ void copy_span(const KParams& p) {
+__device__ __forceinline__ void copy_span(const KParams& p, const int slot) {
   // A span = `ppc` consecutive page columns of one request (one page when pages are large;
   // several small pages, so that every CTA moves a few tens of KiB).
   __shared__ int32_t s_pages[kMaxPagesPerCta];
-  const int slot = blockIdx.x;
   const int r = slot / p.spr;
   const int j0 = (slot - r * p.spr) * p.ppc;
   const int s_r = p.sl[r];
@@ -206,7 +205,24 @@ template <int F, bool PACK, bool MERGED, int VEC, bool MULTI>
 __global__ void __launch_bounds__(kThreads, kMinCtasPerSm)
 topkv_page_copy_kernel(const KParams p) {
   pdl_prologue(p.overlap);
-  copy_span<F, PACK, MERGED, VEC, MULTI>(p);
+  copy_span<F, PACK, MERGED, VEC, MULTI>(p, blockIdx.x);
+  pdl_epilogue(p.overlap);
+}
+
+// The same copy with a bounded grid: gridDim.x CTAs walk all R * spr spans, CTA b taking spans
+// b, b + gridDim.x, ... Used when the wire is pinned host memory reached over PCIe (the direct
+// host leg): the link, not the SMs, sets the pace there, a few CTAs keep it full, and the rest
+// of the GPU stays with whatever else is running (the prefill). Neighbouring CTAs work on
+// neighbouring spans, so the host side is written (read) in roughly ascending order.
+template <int F, bool PACK, bool MERGED, int VEC, bool MULTI>
+__global__ void __launch_bounds__(kThreads, kMinCtasPerSm)
+topkv_page_copy_walk_kernel(const KParams p) {
+  pdl_prologue(p.overlap);
+  const int nslots = p.R * p.spr;
+  for (int slot = blockIdx.x; slot < nslots; slot += gridDim.x) {
+    copy_span<F, PACK, MERGED, VEC, MULTI>(p, slot);
+    __syncthreads();  // the span's page ids in shared memory are re-used by the next span
+  }
   pdl_epilogue(p.overlap);
 }
 

@@ -850,6 +850,79 @@ def test_repage_bench_shape(dev, variant):
 
 # -------------------------------------------------------------------- host leg
 
+@pytest.fixture
+def host_leg_ctas(request):
+    prev = tk.topkv_set_host_leg_ctas(request.param)
+    assert prev >= 0
+    yield request.param
+    tk.topkv_set_host_leg_ctas(prev)
+
+
+def test_host_leg_cta_bound_setter(dev):
+    assert tk.topkv_set_host_leg_ctas(-1) == tk.TOPKV_ERR_INVALID_ARG
+    assert tk.topkv_set_host_leg_ctas(1 << 16) == tk.TOPKV_ERR_INVALID_ARG
+    prev = tk.topkv_set_host_leg_ctas(5)
+    assert prev == 16                                  # the documented default
+    assert tk.topkv_set_host_leg_ctas(prev) == 5
+
+
+@pytest.mark.parametrize("host_leg_ctas", [0, 1, 3, 16, 1000], indirect=True)
+@pytest.mark.parametrize("seed", range(6))
+def test_direct_host_leg_walking_grid_random_geometries(dev, seed, host_leg_ctas, variant):
+    """The direct host leg with a bounded grid (every CTA walks several spans): pinned bytes
+    and destination pool equal the oracle's for strided pools, both wire orders, empty and
+    ragged requests, small pages grouped per CTA, more CTAs than spans."""
+    if variant == 1:
+        pytest.skip("the bounded grid belongs to the vectorised family")
+    rng = np.random.default_rng(7000 + seed)
+    F = int(rng.integers(1, 3))
+    H, D = [(8, 128), (1, 576), (2, 64), (4, 8), (8, 64), (1, 128)][seed]
+    P = int(rng.choice([1, 4, 16, 64]))
+    R = int(rng.integers(1, 7))
+    sl = rng.integers(0, 6 * P + 3, size=R).astype(np.int32)
+    if seed % 2:
+        sl[rng.integers(0, R)] = 0
+    pages = (sl + P - 1) // P
+    maxp = max(int(pages.max()), 1) + 1
+    npages = int(pages.sum()) + 3
+    g = Geom(L=2, F=F, h_kv=H, d_h=D, b_p=2, P=P, num_pages=npages, wire_order=seed % 2)
+    if seed % 3 == 1:                                  # head-major inside the page
+        g.S_tok = D * 2
+        g.S_head = P * g.S_tok
+        g.S_kv = H * g.S_head
+        g.S_page = F * g.S_kv
+        g.S_layer = npages * g.S_page
+    T = int(sl.sum())
+    g.W_layer = g.wire_layer_bytes(T) + 32
+    bt_s = np.full((R, maxp), -1, dtype=np.int32)
+    bt_d = np.full((R, maxp), -1, dtype=np.int32)
+    ps, pd, pos = rng.permutation(npages), rng.permutation(npages), 0
+    for r in range(R):
+        bt_s[r, :pages[r]] = ps[pos:pos + pages[r]]
+        bt_d[r, :pages[r]] = pd[pos:pos + pages[r]]
+        pos += pages[r]
+    src_h = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
+    dst_h = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
+    lo = _layout_from_geom(g)
+    src, dst = torch.from_numpy(src_h).to(dev), torch.from_numpy(dst_h.copy()).to(dev)
+    d_sl = torch.from_numpy(sl).to(dev)
+    d_bs, d_bd = torch.from_numpy(bt_s).to(dev), torch.from_numpy(bt_d).to(dev)
+    bs, bd = tk.make_batch(d_bs, d_sl, T), tk.make_batch(d_bd, d_sl, T)
+    pinned = torch.full((2 * g.W_layer,), 0xA5, dtype=torch.uint8).pin_memory()
+    want = np.full(2 * g.W_layer, 0xA5, dtype=np.uint8)
+    for layer in (1, 0):
+        tk.check(tk.topkv_pack_layer_to_host(layer, src, lo, bs, pinned, pinned.numel(), None, 0))
+        oracle.pack(g, layer, src_h, bt_s, sl, wire=want)
+    torch.cuda.synchronize()
+    assert np.array_equal(pinned.numpy(), want)       # gaps between slabs untouched as well
+    for layer in (0, 1):
+        tk.check(tk.topkv_unpack_layer_from_host(layer, dst, lo, bd, pinned, pinned.numel(), None, 0))
+        oracle.unpack(g, layer, dst_h, bt_d, sl, want)
+    torch.cuda.synchronize()
+    assert np.array_equal(dst.cpu().numpy(), dst_h)
+    assert np.array_equal(src.cpu().numpy(), src_h)
+
+
 @pytest.mark.parametrize("staged", [True, False])
 def test_host_leg_cfg1(dev, staged):
     w = harness.setup(wl.CFG1, dev)
