@@ -412,6 +412,36 @@ def pinned_copy_baseline(dev, stream, nbytes, reps=5):
     return out
 
 
+def pinned_copy_bidirectional_baseline(dev, nbytes, reps=8):
+    """cudaMemcpyAsync device->host and host->device at the same time on two streams (torch
+    copy_), ``reps`` slabs each way back to back: GB/s per direction with both busy."""
+    import torch
+    h_out = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
+    h_in = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
+    d_out = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    d_in = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    s1, s2 = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    best = 1e30
+    for it in range(3):
+        torch.cuda.synchronize(dev)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c, d = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(s1):
+            a.record(s1)
+            for _ in range(reps):
+                h_out.copy_(d_out, non_blocking=True)
+            b.record(s1)
+        with torch.cuda.stream(s2):
+            c.record(s2)
+            for _ in range(reps):
+                d_in.copy_(h_in, non_blocking=True)
+            d.record(s2)
+        torch.cuda.synchronize(dev)
+        if it:
+            best = min(best, max(a.elapsed_time(b), c.elapsed_time(d)))
+    return reps * nbytes / (best * 1e-3) / 1e9
+
+
 def device_copy_baseline(dev, stream, nbytes, reps=10):
     """Plain device-to-device copy of nbytes (torch copy_), read+write GB/s, best of reps."""
     import torch
@@ -676,6 +706,13 @@ def main():
                "to_host_link_GBps": round(n_layer * L / (th * 1e-3) / 1e9, 2),
                "from_host_link_GBps": round(n_layer * L / (fh * 1e-3) / 1e9, 2)}
         del pinned, staging
+        if rank == 0 and world == 1 and slots >= L:
+            # what the link gives each direction while both are busy: plain pinned copies
+            bidir = pinned_copy_bidirectional_baseline(dev, n_layer)
+            e2e["pinned_copy_both_directions_GBps_each"] = round(bidir, 2)
+            e2e["link_GBps_each_direction"] = round(n_layer * L / (ems_max * 1e-3) / 1e9, 2)
+            e2e["frac_of_pinned_copy_both_directions"] = round(
+                n_layer * L / (ems_max * 1e-3) / 1e9 / bidir, 4)
 
     extra = {}
     if rank == 0 and world == 1:

@@ -224,16 +224,21 @@ int topkv_header_check(const topkv_wire_header* header, const topkv_layout* layo
 uint64_t topkv_crc64(const void* h_data, int64_t nbytes);
 
 /* Device-side checksumming, fused into pack / unpack. Usage, per batch:
- *   topkv_crc_begin(...)                 once: constant tables and counters (on `stream`)
- *   topkv_pack_layer_crc(l, ...)         every layer l of the layout exactly once, in any order
- *                                        (topkv_unpack_layer_crc on the receiving side)
- *   topkv_crc_finish(...)                d_crc_out[r*F + c] = checksum of request r, plane c
+ *   topkv_crc_begin(...)                 once: constant tables, clears the remainders (on `stream`)
+ *   topkv_pack_layer_crc(l, ...)         every layer l of the layout, in any order
+ *                                        (topkv_unpack_layer_crc on the receiving side); doing a
+ *                                        layer again (a re-send) rewrites its remainders
+ *   topkv_crc_finish(...)                d_crc_out[r*F + c] = checksum of request r, plane c;
+ *                                        may be called again, changes nothing in the workspace
  * d_workspace: DEVICE scratch of at least topkv_crc_workspace_bytes(...) bytes, 16-byte
- * aligned, owned by the caller and reserved for this batch from begin to finish (it holds the
- * per-layer remainders). d_crc_out: DEVICE uint64 [R*F]. Requirements: heads contiguous in the
- * pool, batch->cu_seq_lens given, window_tokens 0, kv_factor * page_tokens * (runs per row)
- * <= 1024 (else TOPKV_ERR_UNSUPPORTED_LAYOUT). TOPKV_FLAG_OVERLAP_PREVIOUS may be set as for
- * the plain calls. The copy itself is identical to topkv_pack_layer / topkv_unpack_layer. */
+ * aligned, owned by the caller and reserved for this batch from begin to finish. It holds one
+ * 8-byte remainder per 32 runs (of at most 1 KiB) of every request, plane and layer, i.e.
+ * about N_layer * L / 4096 bytes (Llama-3-70B shape, 8 x 4096 tokens: 2.6 MB). d_crc_out:
+ * DEVICE uint64 [R*F]. batch->cu_seq_lens and total_tokens are optional (the kernel rebuilds
+ * the prefix sums from seq_lens), head-split pools are supported; window_tokens must be 0 and
+ * num_requests at most 8192 (else TOPKV_ERR_UNSUPPORTED_LAYOUT). TOPKV_FLAG_OVERLAP_PREVIOUS
+ * may be set as for the plain calls. The bytes moved are identical to topkv_pack_layer /
+ * topkv_unpack_layer. */
 int64_t topkv_crc_workspace_bytes(const topkv_layout* layout, int32_t num_requests,
                                   int32_t max_pages_per_req);
 int topkv_crc_begin(const topkv_layout* layout, const topkv_batch* batch, void* d_workspace,

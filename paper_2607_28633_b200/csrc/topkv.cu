@@ -331,34 +331,79 @@ int noalloc_staging_address(void** out) {
 }
 
 // ---- CRC-64 fused into pack / unpack ------------------------------------------------------------
-// Cuts a token row into runs of at most 1 KiB (one per thread); fails when a page and plane
-// would need more threads than a CTA has.
-int crc_geometry(const topkv_layout* lo, const Resolved& rs, CrcGeom* g) {
-  if (rs.U != 1) return TOPKV_ERR_UNSUPPORTED_LAYOUT;  // heads must be contiguous
-  int rpr = 0;
-  for (int k = 1; k <= 4096; ++k) {
-    if (rs.row_bytes % k) continue;
-    const int64_t run = rs.row_bytes / k;
+// Cuts the contiguous unit (a token row, or one head of a head-split pool) into runs of at most
+// kCrcRunMax bytes, one per lane; fails when no such cut exists or the tables would not fit.
+int crc_geometry(const topkv_layout* lo, const Resolved& rs, int maxp, CrcGeom* g) {
+  int rpu = 0;
+  for (int k = 1; k <= 65536; ++k) {
+    if (rs.unit_bytes % k) continue;
+    const int64_t run = rs.unit_bytes / k;
     if (run % 16) continue;
-    if (run <= 1024) {
-      rpr = k;
+    if (run <= kCrcRunMax) {
+      rpu = k;
       break;
     }
   }
-  if (rpr == 0) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
-  g->rpr = rpr;
-  g->run_bytes = (int)(rs.row_bytes / rpr);
-  g->RB = (int)lo->page_tokens * rpr;
-  if ((int64_t)lo->kv_factor * g->RB > 1024) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  if (rpu == 0) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  g->rpu = rpu;
+  g->run_bytes = (int)(rs.unit_bytes / rpu);
+  g->rpr = rs.U * rpu;
+  const int run16 = g->run_bytes / 16;
+  g->pitch = (run16 | 1) * 16;  // odd number of 16-byte slots: lanes' rows start in distinct banks
+  const int64_t runs = (int64_t)maxp * lo->page_tokens * g->rpr;  // of one block-table row
+  if (runs > 0x7fffff00ll) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  g->kmax = (int)std::max<int64_t>(1, (runs + kCrcRunsPerItem - 1) / kCrcRunsPerItem);
+  return TOPKV_OK;
+}
+
+constexpr int kCrcMaxR = 8192;  // the per-CTA plan (12 bytes per request) lives in shared memory
+
+// Warps per CTA and dynamic shared memory of the checksummed copy for this shape.
+int crc_launch_shape(const CrcGeom& g, int R, int stages, int* warps, size_t* smem) {
+  const size_t fixed = kCrcMaxWarps * kCrcMaxStages * sizeof(uint64_t) + (size_t)(R + 1) * 12 + 16;
+  const size_t per_warp = (size_t)stages * ((size_t)kCrcRunsPerItem * g.pitch + 32 * 8 + 8);
+  if (fixed + per_warp > (size_t)kSmemBudget) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  *warps = (int)std::min<size_t>(kCrcMaxWarps, ((size_t)kSmemBudget - fixed) / per_warp);
+  *smem = (size_t)*warps * per_warp + fixed;
+  return TOPKV_OK;
+}
+
+std::mutex g_crc_mutex;
+bool g_crc_attr_set[64][4] = {};
+
+template <int F, bool PACK>
+int crc_prepare_device(int* sms_out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (dev < 0 || dev >= 64) return TOPKV_ERR_INVALID_ARG;
+  {
+    std::lock_guard<std::mutex> lock(g_devinfo_mutex);
+    DeviceInfo& di = g_devinfo[dev];
+    if (di.sms == 0) {
+      e = cudaDeviceGetAttribute(&di.sms, cudaDevAttrMultiProcessorCount, dev);
+      if (e != cudaSuccess) return cuda_fail(e);
+    }
+    *sms_out = di.sms;
+  }
+  std::lock_guard<std::mutex> lock(g_crc_mutex);
+  const int idx = (F - 1) * 2 + (PACK ? 1 : 0);
+  if (!g_crc_attr_set[dev][idx]) {
+    e = cudaFuncSetAttribute(topkv_crc_copy_kernel<F, PACK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kSmemBudget);
+    if (e != cudaSuccess) return cuda_fail(e);
+    g_crc_attr_set[dev][idx] = true;
+  }
   return TOPKV_OK;
 }
 
 template <bool PACK>
 int crc_copy(int layer, const void* pool, const topkv_layout* lo, const topkv_batch* b,
              const void* wire, int64_t cap, void* ws, int64_t ws_bytes, cudaStream_t stream,
-             void* slab_override = nullptr, int64_t* n_layer_out = nullptr) {
+             void* slab_override = nullptr, int64_t* n_layer_out = nullptr, int max_ctas = 0) {
   // slab_override: device address to use for this layer's wire slab instead of
-  // wire + layer*stride (a staging slab, or the device view of a pinned host slab)
+  // wire + layer*stride (a staging slab, or the device view of a pinned host slab);
+  // max_ctas > 0: the wire is host memory behind PCIe, at most that many CTAs run
   CrcCopyParams cp;
   Resolved rs;
   int64_t n_layer;
@@ -367,36 +412,32 @@ int crc_copy(int layer, const void* pool, const topkv_layout* lo, const topkv_ba
   if (n_layer_out != nullptr) *n_layer_out = n_layer;
   if (slab_override != nullptr) cp.k.wire = static_cast<uint8_t*>(slab_override);
   if (ws == nullptr || !mult16p(ws)) return TOPKV_ERR_INVALID_ARG;
-  if (b->cu_seq_lens == nullptr || b->window_tokens != 0) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
-  st = crc_geometry(lo, rs, &cp.g);
-  if (st != TOPKV_OK) return st;
+  if (b->window_tokens != 0) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
   const int F = (int)lo->kv_factor, R = b->num_requests, maxp = b->max_pages_per_req;
   const int L = (int)lo->num_layers;
-  if (ws_bytes < 8 * crc_workspace_words(cp.g.RB, L, R, maxp, F)) return TOPKV_ERR_CAPACITY;
+  if (R > kCrcMaxR) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  st = crc_geometry(lo, rs, maxp, &cp.g);
+  if (st != TOPKV_OK) return st;
+  if (ws_bytes < 8 * crc_workspace_words(cp.g.kmax, L, R, F)) return TOPKV_ERR_CAPACITY;
   if (R == 0 || maxp == 0) return TOPKV_OK;
-  cp.w = crc_carve(ws, cp.g.RB, L, R, maxp, F);
+  if ((int64_t)R * cp.g.kmax * F > 0x7fffffffll) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  cp.w = crc_carve(ws, cp.g.kmax, L, R, F);
   cp.layer = layer;
-  cp.F = F;
-  const int threads = (F * cp.g.RB + 31) / 32 * 32;
-  const dim3 grid((unsigned)((int64_t)R * maxp)), block((unsigned)threads);
-  const size_t smem = (size_t)(threads / 32) * kCrcTileBytes;
-  // 32-byte pieces when every address the kernel can form is 32-byte aligned
-  const bool wide = ((reinterpret_cast<uintptr_t>(cp.k.pool) | reinterpret_cast<uintptr_t>(cp.k.wire) |
-                      (uintptr_t)cp.k.S_page | (uintptr_t)cp.k.S_kv | (uintptr_t)cp.k.S_tok |
-                      (uintptr_t)cp.g.run_bytes) & 31) == 0;
-  cudaError_t e = cudaSuccess;
-  auto go = [&](auto kernel) {
-    if (smem > 48 * 1024)
-      e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32 * kCrcTileBytes);
-    if (e == cudaSuccess) e = launch_pdl(kernel, grid, block, smem, stream, cp);
-  };
-  if (threads <= 128) {
-    if (wide) { if (F == 1) go(topkv_crc_copy_kernel<1, PACK, 32, 128>); else go(topkv_crc_copy_kernel<2, PACK, 32, 128>); }
-    else { if (F == 1) go(topkv_crc_copy_kernel<1, PACK, 16, 128>); else go(topkv_crc_copy_kernel<2, PACK, 16, 128>); }
-  } else {
-    if (wide) { if (F == 1) go(topkv_crc_copy_kernel<1, PACK, 32, 1024>); else go(topkv_crc_copy_kernel<2, PACK, 32, 1024>); }
-    else { if (F == 1) go(topkv_crc_copy_kernel<1, PACK, 16, 1024>); else go(topkv_crc_copy_kernel<2, PACK, 16, 1024>); }
-  }
+  cp.stages = TOPKV_CRC_STAGES;
+  int warps = 0, sms = 0;
+  size_t smem = 0;
+  st = crc_launch_shape(cp.g, R, cp.stages, &warps, &smem);
+  if (st != TOPKV_OK) return st;
+  st = (F == 1) ? crc_prepare_device<1, PACK>(&sms) : crc_prepare_device<2, PACK>(&sms);
+  if (st != TOPKV_OK) return st;
+  // persistent grid: one CTA per SM, fewer when there is less work or the wire is behind PCIe
+  const int64_t items = (int64_t)R * cp.g.kmax * F;  // upper bound
+  int64_t ctas = std::min<int64_t>(sms, (items + warps - 1) / warps);
+  if (max_ctas > 0) ctas = std::min<int64_t>(ctas, max_ctas);
+  const dim3 grid((unsigned)std::max<int64_t>(1, ctas)), block((unsigned)(warps * 32));
+  cudaError_t e;
+  if (F == 1) e = launch_pdl(topkv_crc_copy_kernel<1, PACK>, grid, block, smem, stream, cp);
+  else e = launch_pdl(topkv_crc_copy_kernel<2, PACK>, grid, block, smem, stream, cp);
   if (e != cudaSuccess) return cuda_fail(e);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
@@ -416,7 +457,8 @@ int crc_host_leg(int layer, const void* pool, const topkv_layout* layout,
     int st = mapped_device_pointer(h_pinned, &dev);
     if (st != TOPKV_OK) return st;
     void* slab = static_cast<uint8_t*>(dev) + (int64_t)layer * layout->wire_layer_stride;
-    return crc_copy<PACK>(layer, pool, layout, batch, h_pinned, host_bytes, ws, ws_bytes, s, slab);
+    return crc_copy<PACK>(layer, pool, layout, batch, h_pinned, host_bytes, ws, ws_bytes, s, slab, nullptr,
+                          g_host_leg_ctas.load(std::memory_order_relaxed));
   }
   if (batch->struct_size == sizeof(topkv_batch) && batch->total_tokens < 0) return TOPKV_ERR_INVALID_ARG;
   if (layout->struct_size == sizeof(topkv_layout) && layout->wire_plane_stride != 0)
@@ -679,10 +721,9 @@ int64_t topkv_crc_workspace_bytes(const topkv_layout* layout, int32_t num_reques
   if (st != TOPKV_OK) return st;
   if (num_requests < 0 || max_pages_per_req < 0) return TOPKV_ERR_INVALID_ARG;
   CrcGeom g;
-  st = crc_geometry(layout, rs, &g);
+  st = crc_geometry(layout, rs, max_pages_per_req, &g);
   if (st != TOPKV_OK) return st;
-  return 8 * crc_workspace_words(g.RB, (int)layout->num_layers, num_requests, max_pages_per_req,
-                                 (int)layout->kv_factor);
+  return 8 * crc_workspace_words(g.kmax, (int)layout->num_layers, num_requests, (int)layout->kv_factor);
 }
 
 int topkv_crc_begin(const topkv_layout* layout, const topkv_batch* batch, void* d_workspace,
@@ -694,15 +735,15 @@ int topkv_crc_begin(const topkv_layout* layout, const topkv_batch* batch, void* 
   if (st != TOPKV_OK) return st;
   if (d_workspace == nullptr || !mult16p(d_workspace)) return TOPKV_ERR_INVALID_ARG;
   if (batch->window_tokens != 0) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
-  CrcGeom g;
-  st = crc_geometry(layout, rs, &g);
-  if (st != TOPKV_OK) return st;
   const int F = (int)layout->kv_factor, R = batch->num_requests, maxp = batch->max_pages_per_req;
   const int L = (int)layout->num_layers;
-  if (workspace_bytes < 8 * crc_workspace_words(g.RB, L, R, maxp, F)) return TOPKV_ERR_CAPACITY;
+  CrcGeom g;
+  st = crc_geometry(layout, rs, maxp, &g);
+  if (st != TOPKV_OK) return st;
+  if (workspace_bytes < 8 * crc_workspace_words(g.kmax, L, R, F)) return TOPKV_ERR_CAPACITY;
   if (R == 0) return TOPKV_OK;
-  const CrcWorkspace w = crc_carve(d_workspace, g.RB, L, R, maxp, F);
-  const int64_t total = (int64_t)g.RB + maxp + 1 + 2 * (int64_t)R + (int64_t)L * R * F;
+  const CrcWorkspace w = crc_carve(d_workspace, g.kmax, L, R, F);
+  const int64_t total = crc_workspace_words(g.kmax, L, R, F) - (int64_t)L * R * F;
   const unsigned blocks = (unsigned)std::min<int64_t>((total + 255) / 256, 1024);
   topkv_crc_begin_kernel<<<blocks, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
       w, g, batch->seq_lens, L, R, maxp, (int)layout->page_tokens, rs.row_bytes, F);
@@ -735,19 +776,25 @@ int topkv_crc_finish(const topkv_layout* layout, const topkv_batch* batch, void*
   if (st != TOPKV_OK) return st;
   if (d_workspace == nullptr || !mult16p(d_workspace) || d_crc_out == nullptr)
     return TOPKV_ERR_INVALID_ARG;
-  CrcGeom g;
-  st = crc_geometry(layout, rs, &g);
-  if (st != TOPKV_OK) return st;
   const int F = (int)layout->kv_factor, R = batch->num_requests, maxp = batch->max_pages_per_req;
   const int L = (int)layout->num_layers;
-  if (workspace_bytes < 8 * crc_workspace_words(g.RB, L, R, maxp, F)) return TOPKV_ERR_CAPACITY;
+  CrcGeom g;
+  st = crc_geometry(layout, rs, maxp, &g);
+  if (st != TOPKV_OK) return st;
+  if (workspace_bytes < 8 * crc_workspace_words(g.kmax, L, R, F)) return TOPKV_ERR_CAPACITY;
   if (R == 0) return TOPKV_OK;
-  const CrcWorkspace w = crc_carve(d_workspace, g.RB, L, R, maxp, F);
-  topkv_crc_finish_kernel<<<(R * F + 127) / 128, 128, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
-      w, batch->seq_lens, L, R, F, d_crc_out);
-  const cudaError_t e = cudaGetLastError();
+  const CrcWorkspace w = crc_carve(d_workspace, g.kmax, L, R, F);
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  const int64_t warps = (int64_t)L * R * F;  // one per (layer, request, plane)
+  if ((warps + 3) / 4 > 0x7fffffffll) return TOPKV_ERR_INVALID_ARG;
+  topkv_crc_layer_kernel<<<(unsigned)((warps + 3) / 4), 128, 0, s>>>(w, g, batch->seq_lens, L, R, F, maxp,
+                                                                     (int)layout->page_tokens);
+  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
-  g_launches.fetch_add(1, std::memory_order_relaxed);
+  topkv_crc_finish_kernel<<<(R * F + 127) / 128, 128, 0, s>>>(w, batch->seq_lens, L, R, F, d_crc_out);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e);
+  g_launches.fetch_add(2, std::memory_order_relaxed);
   return TOPKV_OK;
 }
 

@@ -4,12 +4,20 @@
 //
 // Everything is linear over GF(2). With rem(M) = M(x) * x^64 mod P (no initial value, no
 // inversion) and "||" concatenation:   rem(A || B) = rem(A) * x^(8|B|) + rem(B)   (mod P).
-// The tensor of one request and one plane, [layers][seq_len][kv_heads][head_dim], is cut
-// into runs (a fraction of a token row); every thread owns one run: while the warp moves the
-// data from source to destination it folds its run into a 64-bit remainder, multiplies that by
-// x^(8 * bytes that follow the run inside its page), and the page's threads XOR their results.
-// Each page then aligns its remainder inside the request's plane and XORs it into the layer's
-// remainder (one atomic per page and plane); topkv_crc_finish chains the layers:
+// The tensor of one request and one plane, [layers][seq_len][kv_heads][head_dim], is cut,
+// layer by layer, into runs (a fraction of a token row, at most 512 bytes) and the runs into
+// items of 32 consecutive runs counted from the END of the request's plane, so that every item
+// but the first of a request is full and k full items follow item k. One warp takes one item,
+// one lane one run:
+//   - the lane brings its run into its own row of the warp's shared-memory stage with one
+//     bulk-async copy (cp.async.bulk, completion on the warp's mbarrier);
+//   - it folds the row, 8 bytes per step, rem = (rem ^ word) * x^64, and sends the row on to
+//     the destination with one bulk-async store, so no thread moves payload through registers
+//     except to checksum it;
+//   - it multiplies its remainder by x^(8 * run_bytes * (31 - lane)) (the runs that follow it
+//     inside the item), the warp XORs the 32 results, and lane 0 stores the item's remainder.
+// topkv_crc_finish multiplies item k's remainder by x^(8 * run_bytes * 32 * k), XORs the items
+// of a layer, and chains the layers:
 //   state_0 = ~0,  state_l+1 = state_l * x^(8 * bytes of the plane in one layer) + rem_l,
 // and the checksum is ~state_L.
 //
@@ -23,6 +31,7 @@
 
 #include <cstdint>
 
+#include "topkv_bulk.cuh"
 #include "topkv_common.cuh"
 
 namespace topkv {
@@ -57,6 +66,86 @@ __host__ __device__ __forceinline__ uint64_t gf_mulmod(uint64_t a, uint64_t b) {
   return res;
 }
 
+// Carry-less product of two 32-bit polynomials (bit i = coefficient of x^i here, plain order)
+// with integer multipliers: each operand is split into four "every fourth bit" parts, so that
+// in an integer product of two parts at most 8 terms meet in one bit position and their sum
+// (< 16) cannot carry into the next position of the same class; the lowest bit of each 4-bit
+// cell is then the XOR of the terms, the other three bits are masked away.
+__host__ __device__ __forceinline__ uint64_t gf_clmul32(uint32_t x, uint32_t y) {
+  const uint32_t x0 = x & 0x11111111u, x1 = x & 0x22222222u, x2 = x & 0x44444444u, x3 = x & 0x88888888u;
+  const uint32_t y0 = y & 0x11111111u, y1 = y & 0x22222222u, y2 = y & 0x44444444u, y3 = y & 0x88888888u;
+  auto m = [](uint32_t a, uint32_t b) { return (uint64_t)a * (uint64_t)b; };
+  const uint64_t z0 = m(x0, y0) ^ m(x1, y3) ^ m(x2, y2) ^ m(x3, y1);
+  const uint64_t z1 = m(x0, y1) ^ m(x1, y0) ^ m(x2, y3) ^ m(x3, y2);
+  const uint64_t z2 = m(x0, y2) ^ m(x1, y1) ^ m(x2, y0) ^ m(x3, y3);
+  const uint64_t z3 = m(x0, y3) ^ m(x1, y2) ^ m(x2, y1) ^ m(x3, y0);
+  return (z0 & 0x1111111111111111ull) | (z1 & 0x2222222222222222ull) | (z2 & 0x4444444444444444ull) |
+         (z3 & 0x8888888888888888ull);
+}
+
+// a * b mod P without a bit loop: a 64 x 64 carry-less product from three 32 x 32 ones
+// (Karatsuba), then the reduction, which is cheap because the generator is sparse. In the
+// reflected convention the plain-order product c of the two registers holds the coefficient of
+// x^d in bit 126 - d: degrees 0..63 sit in bits 63..126 and degrees 64..126 in bits 62..0, so the
+// low part is c >> 63, the high part (to be multiplied by x^64) is the low word shifted left once.
+__host__ __device__ __forceinline__ uint64_t gf_mulmod_clmul(uint64_t a, uint64_t b) {
+  const uint32_t a0 = (uint32_t)a, a1 = (uint32_t)(a >> 32), b0 = (uint32_t)b, b1 = (uint32_t)(b >> 32);
+  const uint64_t lo = gf_clmul32(a0, b0), hi = gf_clmul32(a1, b1);
+  const uint64_t mid = gf_clmul32(a0 ^ a1, b0 ^ b1) ^ lo ^ hi;
+  const uint64_t c_lo = lo ^ (mid << 32), c_hi = hi ^ (mid >> 32);  // the 128-bit product
+  return ((c_hi << 1) | (c_lo >> 63)) ^ gf_mulx64(c_lo << 1);
+}
+
+// ---- 64 message bytes per step, with the reduction put off to the end of the step -----------
+// Since x^64 = m(x) = (1 + x)(1 + x^3) (mod P), eight Horner steps over the words w0..w7 give
+//   new = (rem ^ w0) * m^8 + (w1 * m^6 + w2 * m^5 + ... + w6 * m + w7) * m          (mod P).
+// Nothing has to be reduced on the way: a 96-bit register (three 32-bit words h:l:e, bit 95 the
+// coefficient of x^0) holds every intermediate value, because each multiplication by m adds
+// only 4 to the degree (63 + 7 * 4 = 91) and m^8 = 1 + x^8 + x^24 + x^32 adds 32. A
+// multiplication by (1 + x^k) is "v ^= v >> k" over the three words. The 32 coefficients that
+// end up in e (degrees 64..95) are brought back once per step: e(x) * x^64 = e(x) * m(x).
+__host__ __device__ __forceinline__ uint32_t gf_fsr(uint32_t lo, uint32_t hi, int k) {
+#ifdef __CUDA_ARCH__
+  return __funnelshift_r(lo, hi, k);  // low word of (hi:lo) >> k, 0 < k < 32
+#else
+  return (lo >> k) | (hi << (32 - k));
+#endif
+}
+
+struct Gf96 {
+  uint32_t h, l, e;
+};
+
+// u * m(x) + w, unreduced (the caller keeps the degree below 96).
+__host__ __device__ __forceinline__ Gf96 gf96_mulm_add(Gf96 u, uint32_t w_hi, uint32_t w_lo) {
+  Gf96 a, b;  // a = u * (1 + x), b = a * (1 + x^3) + w
+  a.h = u.h ^ (u.h >> 1);
+  a.l = u.l ^ gf_fsr(u.l, u.h, 1);
+  a.e = u.e ^ gf_fsr(u.e, u.l, 1);
+  b.h = a.h ^ (a.h >> 3) ^ w_hi;
+  b.l = a.l ^ gf_fsr(a.l, a.h, 3) ^ w_lo;
+  b.e = a.e ^ gf_fsr(a.e, a.l, 3);
+  return b;
+}
+
+// Remainder after the eight words w[0..7] (w[2i] = low half, w[2i+1] = high half of word i, as
+// a little-endian load delivers them) have followed a message whose remainder was rem.
+__host__ __device__ __forceinline__ uint64_t gf_fold64(uint64_t rem, const uint32_t (&w)[16]) {
+  Gf96 u = {w[3], w[2], 0u};  // w1
+#pragma unroll
+  for (int i = 2; i < 8; ++i) u = gf96_mulm_add(u, w[2 * i + 1], w[2 * i]);
+  u = gf96_mulm_add(u, 0u, 0u);  // the last * m
+  const uint32_t vh = (uint32_t)(rem >> 32) ^ w[1], vl = (uint32_t)rem ^ w[0];  // rem ^ w0
+  // (rem ^ w0) * (1 + x^8 + x^24 + x^32): whole-byte shifts over h:l:e
+  const uint32_t h = u.h ^ vh ^ (vh >> 8) ^ (vh >> 24);
+  const uint32_t l = u.l ^ vl ^ gf_fsr(vl, vh, 8) ^ gf_fsr(vl, vh, 24) ^ vh;
+  const uint32_t e = u.e ^ (vl << 24) ^ (vl << 8) ^ vl;
+  // e holds the coefficients of x^64 .. x^95: e * x^64 = e * (1 + x + x^3 + x^4), degree < 36
+  const uint32_t rh = h ^ e ^ (e >> 1) ^ (e >> 3) ^ (e >> 4);
+  const uint32_t rl = l ^ (e << 31) ^ (e << 29) ^ (e << 28);
+  return ((uint64_t)rh << 32) | rl;
+}
+
 // x^n mod P by square and multiply.
 __host__ __device__ inline uint64_t gf_powx(uint64_t n) {
   uint64_t result = kGfOne, base = kGfX;
@@ -69,66 +158,76 @@ __host__ __device__ inline uint64_t gf_powx(uint64_t n) {
 }
 
 // ---- workspace (device memory owned by the caller), in 8-byte words ------------------------------
-// c_run    [RB]            x^(8 * run_bytes * m)
-// c_page   [maxp + 1]      x^(8 * P * row_bytes * k)
-// x_req    [R]             x^(8 * s_r * row_bytes)        (per batch)
-// x_last   [R]             x^(8 * v_last(r) * row_bytes)  (per batch)
-// layer_rem[L * R * F]     remainder of request r, plane c in layer l: every page's CTA XORs its
-//                          aligned page remainder in (atomicXor), so it starts at zero
+// c_run    [32]                 x^(8 * run_bytes * (31 - lane))
+// c_tail   [kmax + 1]           x^(8 * run_bytes * 32 * k)
+// x_req    [R]                  x^(8 * s_r * row_bytes)        (per batch)
+// item_rem [L * R * kmax * F]   remainder of item k (counted from the end) of request r, plane c,
+//                               layer l, aligned to the item's end; cleared by topkv_crc_begin,
+//                               stored (not accumulated) by the copy, so packing a layer again
+//                               just rewrites its entries
+// layer_rem[L * R * F]          written by topkv_crc_finish
 struct CrcWorkspace {
   uint64_t* c_run;
-  uint64_t* c_page;
+  uint64_t* c_tail;
   uint64_t* x_req;
-  uint64_t* x_last;
-  unsigned long long* layer_rem;
+  uint64_t* item_rem;
+  uint64_t* layer_rem;
 };
+
+constexpr int kCrcRunsPerItem = 32;  // one run per lane
+#ifndef TOPKV_CRC_RUN_MAX
+#define TOPKV_CRC_RUN_MAX 1024
+#endif
+constexpr int kCrcRunMax = TOPKV_CRC_RUN_MAX;  // bytes one lane streams per item, at most
+constexpr int kCrcMaxWarps = 16;
+constexpr int kCrcMaxStages = 4;  // shared-memory stages per warp, at most
+#ifndef TOPKV_CRC_STAGES
+#define TOPKV_CRC_STAGES 1
+#endif
 
 struct CrcGeom {
-  int run_bytes;  // bytes one thread streams (divides row_bytes, multiple of 16)
-  int rpr;        // runs per token row
-  int RB;         // runs per page and plane = P * rpr
+  int run_bytes;  // bytes one lane streams per item (divides the contiguous unit, multiple of 16)
+  int rpu;        // runs per contiguous unit (the whole row, or one head when heads are split)
+  int rpr;        // runs per token row = units per row * rpu
+  int pitch;      // bytes between the rows of a stage: odd multiple of 16 (conflict-free reads)
+  int kmax;       // items per request and plane that the tables cover: ceil(maxp * P * rpr / 32)
 };
 
-__host__ __device__ inline int64_t crc_workspace_words(int RB, int L, int R, int maxp, int F) {
-  return (int64_t)RB + (maxp + 1) + 2 * (int64_t)R + (int64_t)L * R * F;
+__host__ __device__ inline int64_t crc_workspace_words(int kmax, int L, int R, int F) {
+  return 32 + ((int64_t)kmax + 1) + (int64_t)R + (int64_t)L * R * kmax * F + (int64_t)L * R * F;
 }
 
-__host__ __device__ inline CrcWorkspace crc_carve(void* base, int RB, int L, int R, int maxp, int F) {
-  (void)L;
-  (void)F;
+__host__ __device__ inline CrcWorkspace crc_carve(void* base, int kmax, int L, int R, int F) {
   CrcWorkspace w;
   w.c_run = static_cast<uint64_t*>(base);
-  w.c_page = w.c_run + RB;
-  w.x_req = w.c_page + (maxp + 1);
-  w.x_last = w.x_req + R;
-  w.layer_rem = reinterpret_cast<unsigned long long*>(w.x_last + R);
+  w.c_tail = w.c_run + 32;
+  w.x_req = w.c_tail + (kmax + 1);
+  w.item_rem = w.x_req + R;
+  w.layer_rem = w.item_rem + (int64_t)L * R * kmax * F;
   return w;
 }
 
-// Builds the constant tables for this batch and clears the per-layer remainders.
+// Builds the constant tables for this batch and clears the item remainders.
 __global__ void __launch_bounds__(256)
 topkv_crc_begin_kernel(CrcWorkspace w, CrcGeom g, const int32_t* __restrict__ sl, int L, int R,
                        int maxp, int P, int64_t row_bytes, int F) {
   pdl_prologue(0);
-  const int64_t n_run = g.RB, n_page = maxp + 1;
-  const int64_t total = n_run + n_page + 2 * (int64_t)R + (int64_t)L * R * F;
+  const int64_t n_tail = (int64_t)g.kmax + 1;
+  const int64_t n_items = (int64_t)L * R * g.kmax * F;
+  const int64_t total = 32 + n_tail + R + n_items;
   for (int64_t k = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; k < total;
        k += (int64_t)gridDim.x * blockDim.x) {
-    if (k < n_run) {
-      w.c_run[k] = gf_powx(8ull * g.run_bytes * (uint64_t)k);
-    } else if (k < n_run + n_page) {
-      const int64_t j = k - n_run;
-      w.c_page[j] = gf_powx(8ull * (uint64_t)P * row_bytes * (uint64_t)j);
-    } else if (k < n_run + n_page + 2 * (int64_t)R) {
-      const int64_t q = k - n_run - n_page;
-      const int r = (int)(q >> 1);
-      int s = sl[r];
-      s = max(0, min(s, maxp * P));
-      const int v_last = s == 0 ? 0 : s - ((s - 1) / P) * P;
-      if (q & 1) w.x_last[r] = gf_powx(8ull * (uint64_t)v_last * row_bytes);
-      else w.x_req[r] = gf_powx(8ull * (uint64_t)s * row_bytes);
+    if (k < 32) {
+      w.c_run[k] = gf_powx(8ull * g.run_bytes * (uint64_t)(31 - k));
+    } else if (k < 32 + n_tail) {
+      w.c_tail[k - 32] = gf_powx(8ull * g.run_bytes * 32ull * (uint64_t)(k - 32));
+    } else if (k < 32 + n_tail + R) {
+      const int r = (int)(k - 32 - n_tail);
+      int64_t s = sl[r];
+      s = s < 0 ? 0 : (s > (int64_t)maxp * P ? (int64_t)maxp * P : s);
+      w.x_req[r] = gf_powx(8ull * (uint64_t)s * (uint64_t)row_bytes);
     } else {
-      w.layer_rem[k - n_run - n_page - 2 * (int64_t)R] = 0ull;
+      w.item_rem[k - 32 - n_tail - R] = 0ull;
     }
   }
 }
@@ -138,162 +237,273 @@ struct CrcCopyParams {
   CrcGeom g;
   CrcWorkspace w;
   int layer;
-  int F;
+  int stages;  // shared-memory stages per warp (1 .. kCrcMaxStages)
 };
 
-constexpr int kCrcPitch = 144;          // bytes per run in the exchange tile: 128 + 16 of padding
-constexpr int kCrcTileBytes = 32 * kCrcPitch;  // one tile per warp
-
-template <int VEC>
-struct Piece;
-template <>
-struct Piece<16> {
-  uint4 a;
-  __device__ __forceinline__ void load(const uint8_t* p) { a = *reinterpret_cast<const uint4*>(p); }
-  __device__ __forceinline__ void store(uint8_t* p) const { *reinterpret_cast<uint4*>(p) = a; }
-  __device__ __forceinline__ void to_tile(uint8_t* p) const { *reinterpret_cast<uint4*>(p) = a; }
-};
-template <>
-struct Piece<32> {
-  uint4 a, b;
-  __device__ __forceinline__ void load(const uint8_t* p) {
-    asm volatile("ld.global.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                 : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w), "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w)
-                 : "l"(p));
-  }
-  __device__ __forceinline__ void store(uint8_t* p) const {
-    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(a.x), "r"(a.y),
-                 "r"(a.z), "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w)
-                 : "memory");
-  }
-  __device__ __forceinline__ void to_tile(uint8_t* p) const {
-    *reinterpret_cast<uint4*>(p) = a;
-    *reinterpret_cast<uint4*>(p + 16) = b;
-  }
-};
-
-// One CTA per (request, page column); one thread owns one run of one plane (F * RB threads
-// work). Global memory is accessed warp-coalesced: in every step the warp moves 128 bytes of
-// each of several of its runs, 128 / VEC lanes per run, straight from source to destination;
-// the same registers are also dropped into a padded shared-memory tile from which every lane
-// picks up the 128 bytes of its OWN run, in order, for the checksum. The next batch's loads are
-// issued before the current batch is folded, so that they are in flight during the ALU work.
-template <int F, bool PACK, int VEC, int MAXT>
-__global__ void __launch_bounds__(MAXT, 1) topkv_crc_copy_kernel(const CrcCopyParams cp) {
-  extern __shared__ __align__(16) uint8_t s_tiles[];
-  __shared__ unsigned long long s_rem[2];
-  constexpr int kPieces = 128 / VEC;      // pieces of one run in a batch = steps per batch
-  constexpr int kRunsPerStep = 32 / kPieces;
+// Persistent grid; every warp runs its own pipeline of `stages` stages over the items gw,
+// gw + GW, ... (gw = global warp index), so neighbouring warps work on neighbouring runs.
+// Shared memory: [warps][stages] stages of 32 rows of `pitch` bytes, the mbarriers, where every
+// staged run goes and which item it belongs to, the per-CTA plan
+// (token prefix sums int64 [R+1] and item prefix sums int32 [R+1], rebuilt from seq_lens).
+template <int F, bool PACK>
+__global__ void __launch_bounds__(kCrcMaxWarps * 32, 1) topkv_crc_copy_kernel(const CrcCopyParams cp) {
+  extern __shared__ __align__(128) uint8_t smem[];
   const KParams& p = cp.k;
   pdl_prologue(p.overlap);
-  const int tid = threadIdx.x, lane = tid & 31;
-  const int slot = blockIdx.x;
-  const int r = slot / p.maxp;
-  const int j = slot - r * p.maxp;
-  int s_r = p.sl[r];
-  if (s_r > p.maxp * p.P) {
-    s_r = p.maxp * p.P;
-    if (tid == 0 && j == 0) raise_error(kErrTable);
-  }
-  const int first = j * p.P;
-  if (first < s_r) {
-    const int v = min(p.P, s_r - first);
-    const int64_t n0 = p.cu[r] + first;
-    const int64_t T = p.plane_rows >= 0 ? p.plane_rows : (p.T >= 0 ? p.T : p.cu[p.R]);  // plane rows
-    const int64_t row = (int64_t)cp.g.run_bytes * cp.g.rpr;
-    const int64_t page = p.bt[(int64_t)r * p.maxp + j];
-    const bool page_ok = page >= 0 && page < p.num_pages;
-    const bool fits = p.planar ? (n0 >= 0 && ((F - 1) * T + n0 + v) * row <= p.wire_limit)
-                               : (n0 >= 0 && (n0 + v) * F * row <= p.wire_limit);
-    if (tid == 0 && !page_ok) raise_error(kErrTable);
-    if (tid == 0 && !fits) raise_error(kErrWire);
-    if (tid < 2) s_rem[tid] = 0ull;
-    __syncthreads();
-    const int c = tid / cp.g.RB;
-    const int idx = tid - c * cp.g.RB;
-    const int nruns = v * cp.g.rpr;
-    const bool mine = page_ok && fits && c < F && idx < nruns;  // this lane owns a run
-    // source and destination of this lane's run (null when it owns none)
-    const uint8_t* src_run = nullptr;
-    uint8_t* dst_run = nullptr;
-    if (mine) {
-      const int t = idx / cp.g.rpr;
-      const int seg = idx - t * cp.g.rpr;
-      uint8_t* a = p.pool + page * p.S_page + c * p.S_kv + (int64_t)t * p.S_tok +
-                   (int64_t)seg * cp.g.run_bytes;
-      const int64_t wrow = p.planar ? ((int64_t)c * T + n0 + t) : ((n0 + t) * F + c);
-      uint8_t* b = p.wire + wrow * row + (int64_t)seg * cp.g.run_bytes;
-      src_run = PACK ? a : b;
-      dst_run = PACK ? b : a;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int W = blockDim.x >> 5;
+  const int run_bytes = cp.g.run_bytes, rpr = cp.g.rpr;
+  const int stage_bytes = kCrcRunsPerItem * cp.g.pitch;
+
+  const int S = cp.stages;
+  uint8_t* my_row = smem + (size_t)warp * S * stage_bytes + (size_t)lane * cp.g.pitch;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)W * S * stage_bytes);
+  uint8_t** s_dst = reinterpret_cast<uint8_t**>(bars + kCrcMaxWarps * kCrcMaxStages);
+  int64_t* s_idx = reinterpret_cast<int64_t*>(s_dst + (size_t)W * S * 32);
+  int64_t* s_cu = s_idx + (size_t)W * S;  // [R+1] tokens
+  uint8_t** my_dst = s_dst + (size_t)warp * S * 32 + lane;  // [slot * 32]: where this lane's run goes
+  int64_t* my_idx = s_idx + (size_t)warp * S;              // [slot]: the item's place in item_rem
+  int32_t* s_ic = reinterpret_cast<int32_t*>(s_cu + (p.R + 1));     // [R+1] items per plane
+
+  // ---- per-CTA plan ------------------------------------------------------------------------
+  const int64_t row_tokens = (int64_t)p.maxp * p.P;  // what one block-table row can describe
+  for (int q = threadIdx.x; q < p.R; q += blockDim.x) {
+    int64_t s = p.sl[q];
+    if (s < 0 || s > row_tokens) {
+      raise_error(kErrTable);
+      s = s < 0 ? 0 : row_tokens;
     }
-    uint8_t* tile = s_tiles + (size_t)(tid >> 5) * kCrcTileBytes;
-    const int sub = lane / kPieces, piece = lane % kPieces;
-    uint64_t rem = 0;
-    if (__any_sync(0xffffffffu, mine)) {
-      // In step m this lane moves piece `piece` of the run owned by lane kRunsPerStep*m + sub.
-      const uint8_t* sp[kPieces];
-      uint8_t* dp[kPieces];
-#pragma unroll
-      for (int m = 0; m < kPieces; ++m) {
-        const int owner = kRunsPerStep * m + sub;
-        const uint64_t s0 = __shfl_sync(0xffffffffu, (uint64_t)src_run, owner);
-        const uint64_t d0 = __shfl_sync(0xffffffffu, (uint64_t)dst_run, owner);
-        sp[m] = s0 ? reinterpret_cast<const uint8_t*>(s0) + piece * VEC : nullptr;
-        dp[m] = reinterpret_cast<uint8_t*>(d0) + piece * VEC;
-      }
-      uint8_t* my_tile_out = tile + sub * kCrcPitch + piece * VEC;  // + m * kRunsPerStep * pitch
-      const uint8_t* my_tile_in = tile + lane * kCrcPitch;
-      Piece<VEC> x[kPieces];
-      auto fetch = [&](int off) {
-        const int left = cp.g.run_bytes - off;  // bytes of every run still to move
-#pragma unroll
-        for (int m = 0; m < kPieces; ++m)
-          if (sp[m] != nullptr && piece * VEC < left) x[m].load(sp[m] + off);
-      };
-      fetch(0);
-      for (int off = 0; off < cp.g.run_bytes; off += 128) {
-        const int left = cp.g.run_bytes - off;
-#pragma unroll
-        for (int m = 0; m < kPieces; ++m)
-          if (sp[m] != nullptr && piece * VEC < left) {
-            x[m].store(dp[m] + off);
-            x[m].to_tile(my_tile_out + m * kRunsPerStep * kCrcPitch);
-          }
-        __syncwarp();
-        if (off + 128 < cp.g.run_bytes) fetch(off + 128);  // in flight while this batch is folded
-        if (mine) {
-          const int words16 = min(8, left >> 4);  // never past this lane's 128 bytes of the tile
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            if (k < words16) {
-              const uint4 y = *reinterpret_cast<const uint4*>(my_tile_in + k * 16);
-              rem = gf_mulx64(rem ^ ((uint64_t)y.x | ((uint64_t)y.y << 32)));
-              rem = gf_mulx64(rem ^ ((uint64_t)y.z | ((uint64_t)y.w << 32)));
-            }
-          }
+    s_cu[q + 1] = s;
+    s_ic[q + 1] = (int32_t)((s * rpr + kCrcRunsPerItem - 1) / kCrcRunsPerItem);
+  }
+  if (threadIdx.x == 0) {
+    s_cu[0] = 0;
+    s_ic[0] = 0;
+  }
+  if (lane == 0)
+    for (int q = 0; q < S; ++q) mbar_init(smem_addr(&bars[warp * kCrcMaxStages + q]), 1);
+  __syncthreads();
+  if (warp == 0) {  // inclusive scans, 32 entries per round
+    int64_t carry_c = 0;
+    int carry_i = 0;
+    for (int base = 1; base <= p.R; base += 32) {
+      const int q = base + lane;
+      int64_t c = q <= p.R ? s_cu[q] : 0;
+      int g = q <= p.R ? s_ic[q] : 0;
+      for (int o = 1; o < 32; o <<= 1) {
+        const int64_t c2 = __shfl_up_sync(0xffffffffu, c, o);
+        const int g2 = __shfl_up_sync(0xffffffffu, g, o);
+        if (lane >= o) {
+          c += c2;
+          g += g2;
         }
+      }
+      if (q <= p.R) {
+        s_cu[q] = c + carry_c;
+        s_ic[q] = g + carry_i;
+      }
+      carry_c += __shfl_sync(0xffffffffu, c, 31);
+      carry_i += __shfl_sync(0xffffffffu, g, 31);
+    }
+  }
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  __syncthreads();
+
+  const int64_t row = (int64_t)run_bytes * rpr;  // bytes of one [head][dim] row
+  // rows from the K plane to the V plane of a PLANAR slab
+  const int64_t PR = p.plane_rows >= 0 ? p.plane_rows : (p.T >= 0 ? p.T : s_cu[p.R]);
+  {
+    const int64_t S = s_cu[p.R];  // uniform over the grid
+    const bool fits = p.planar ? ((F - 1) * PR + S) * row <= p.wire_limit : S * F * row <= p.wire_limit;
+    if (!fits) {
+      if (threadIdx.x == 0) raise_error(kErrWire);
+      pdl_epilogue(p.overlap);
+      return;
+    }
+  }
+
+  const int64_t total_items = (int64_t)s_ic[p.R] * F;
+  const int64_t GW = (int64_t)gridDim.x * W;
+  const uint64_t c_lane = cp.w.c_run[lane];
+  int64_t next_item = (int64_t)blockIdx.x * W + warp;
+  bool failed = false;
+
+  // Finds this warp's next item with anything to move and starts its loads into stage `slot`
+  // (every lane brings its own run). Returns false when the items are used up; otherwise *dst
+  // is where this lane's run goes (null when the lane has none) and *idx the item's place in
+  // item_rem. Uniform across the warp.
+  auto issue_next = [&](int slot, uint8_t** dst_out, int64_t* idx_out) -> bool {
+    while (next_item < total_items) {
+      const int64_t it = next_item;
+      next_item += GW;
+      const int m = (int)(it / F);
+      const int c = (int)(it - (int64_t)m * F);
+      int lo = 0, hi = p.R;  // largest r with s_ic[r] <= m
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (s_ic[mid] <= m) lo = mid;
+        else hi = mid;
+      }
+      const int r = lo;
+      const int64_t cu_r = s_cu[r];
+      const int64_t n_r = (s_cu[r + 1] - cu_r) * rpr;  // runs of this request's plane
+      const int k = s_ic[r + 1] - 1 - m;                // full items that follow this one
+      const int g = (int)(n_r - (int64_t)kCrcRunsPerItem * (k + 1)) + lane;  // this lane's run
+      bool active = g >= 0;
+      const uint8_t* src = nullptr;
+      uint8_t* dst = nullptr;
+      if (active) {
+        const int t = g / rpr;                               // token inside the request
+        const int u = g - t * rpr;                           // run inside the row
+        const int h = u / cp.g.rpu, seg = u - h * cp.g.rpu;  // unit (head) and run inside it
+        const int j = t / p.P, tt = t - j * p.P;
+        const int64_t page = p.bt[(int64_t)r * p.maxp + j];
+        if (page < 0 || page >= p.num_pages) {  // unusable entry: the run is skipped
+          raise_error(kErrTable);
+          active = false;
+        } else {
+          uint8_t* a = p.pool + page * p.S_page + c * p.S_kv + (int64_t)tt * p.S_tok +
+                       (int64_t)h * p.S_unit + (int64_t)seg * run_bytes;
+          const int64_t wrow = p.planar ? ((int64_t)c * PR + cu_r + t) : ((cu_r + t) * F + c);
+          uint8_t* b = p.wire + wrow * row + (int64_t)u * run_bytes;
+          src = PACK ? a : b;
+          dst = PACK ? b : a;
+        }
+      }
+      const unsigned mask = __ballot_sync(0xffffffffu, active);
+      if (mask == 0) continue;
+      const uint32_t bar = smem_addr(&bars[warp * kCrcMaxStages + slot]);
+      if (lane == 0) mbar_expect_tx(bar, (uint32_t)(__popc(mask) * run_bytes));
+      __syncwarp();
+      if (active) bulk_g2s(smem_addr(my_row + (size_t)slot * stage_bytes), src, (uint32_t)run_bytes, bar);
+      *dst_out = active ? dst : nullptr;
+      *idx_out = (((int64_t)cp.layer * p.R + r) * cp.g.kmax + k) * F + c;
+      return true;
+    }
+    return false;
+  };
+
+  // Folds this lane's row of stage `slot`, sends the row on to `dst`, aligns the remainder to the
+  // item's end, combines the lanes and stores the item's remainder.
+  auto fold_and_store = [&](int slot, uint8_t* dst, int64_t idx) {
+    uint8_t* row_g = my_row + (size_t)slot * stage_bytes;
+    uint64_t rem = 0;
+    if (dst != nullptr) {
+      int off = 0;
+#pragma unroll 2
+      for (; off + 64 <= run_bytes; off += 64) {  // 64 bytes per step, one reduction per step
+        const uint4 y0 = *reinterpret_cast<const uint4*>(row_g + off);
+        const uint4 y1 = *reinterpret_cast<const uint4*>(row_g + off + 16);
+        const uint4 y2 = *reinterpret_cast<const uint4*>(row_g + off + 32);
+        const uint4 y3 = *reinterpret_cast<const uint4*>(row_g + off + 48);
+        const uint32_t w[16] = {y0.x, y0.y, y0.z, y0.w, y1.x, y1.y, y1.z, y1.w,
+                                y2.x, y2.y, y2.z, y2.w, y3.x, y3.y, y3.z, y3.w};
+        rem = gf_fold64(rem, w);
+      }
+      for (; off < run_bytes; off += 16) {  // what is left of a run that is no multiple of 64
+        const uint4 y = *reinterpret_cast<const uint4*>(row_g + off);
+        rem = gf_mulx64(rem ^ ((uint64_t)y.x | ((uint64_t)y.y << 32)));
+        rem = gf_mulx64(rem ^ ((uint64_t)y.z | ((uint64_t)y.w << 32)));
+      }
+      rem = gf_mulmod_clmul(rem, c_lane);  // 31 - lane runs follow inside the item
+      bulk_s2g(dst, smem_addr(row_g), (uint32_t)run_bytes);
+    }
+    bulk_commit();
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) rem ^= __shfl_xor_sync(0xffffffffu, rem, o);
+    if (lane == 0) cp.w.item_rem[idx] = rem;
+  };
+  auto wait_loaded = [&](int slot, uint32_t parity) -> bool {
+    const uint32_t bar = smem_addr(&bars[warp * kCrcMaxStages + slot]);
+    uint32_t polls = 0;
+    while (!mbar_try_wait(bar, parity)) {
+      if (++polls > kWaitPollLimit) return false;
+    }
+    return true;
+  };
+
+  if (S == 1) {
+    // One stage per warp: load, fold, store, wait for the store to have read the rows, next item.
+    // The overlap of transfers and arithmetic comes from the other warps of the SM.
+    uint8_t* d;
+    int64_t ix;
+    uint32_t parity = 0u;
+    while (issue_next(0, &d, &ix)) {
+      if (!wait_loaded(0, parity)) {
+        failed = true;
+        break;
+      }
+      parity ^= 1u;
+      fold_and_store(0, d, ix);
+      bulk_wait_read<0>();
+      __syncwarp();
+    }
+  } else {
+    // S stages per warp. Loads run up to S - 1 items ahead. After the store of item i has been
+    // issued, the stage of item i - 1 is re-filled: its store was issued one item earlier and
+    // has had the whole folding of item i to read its rows out of shared memory.
+    int issued = 0, consumed = 0;
+    uint32_t parity_bits = 0u;  // bit q: phase parity of stage q's mbarrier
+    {
+      uint8_t* d;
+      int64_t ix;
+      while (issued < S - 1 && issue_next(issued, &d, &ix)) {
+        my_dst[issued * 32] = d;
+        if (lane == 0) my_idx[issued] = ix;
+        ++issued;
+      }
+    }
+    __syncwarp();
+    while (consumed < issued) {
+      const int cur = consumed % S;
+      if (!wait_loaded(cur, (parity_bits >> cur) & 1u)) {
+        failed = true;
+        break;
+      }
+      parity_bits ^= 1u << cur;
+      fold_and_store(cur, my_dst[cur * 32], my_idx[cur]);
+      ++consumed;
+      bulk_wait_read<1>();  // the store before the one just issued has read its rows
+      __syncwarp();
+      const int slot = issued % S;
+      uint8_t* d;
+      int64_t ix;
+      if (issue_next(slot, &d, &ix)) {
+        my_dst[slot * 32] = d;
+        if (lane == 0) my_idx[slot] = ix;
+        ++issued;
         __syncwarp();
       }
     }
-    if (mine) {
-      // align to the end of this page's plane: (nruns - 1 - idx) runs follow
-      rem = gf_mulmod(rem, cp.w.c_run[nruns - 1 - idx]);
-      atomicXor(&s_rem[c], (unsigned long long)rem);
-    }
-    __syncthreads();
-    // Align this page's remainder inside the request's plane (n_r - 2 - j full pages and the
-    // last, possibly partial, page follow it) and add it to the layer's remainder.
-    if (tid < F && page_ok && fits) {
-      const int n_r = (s_r + p.P - 1) / p.P;
-      uint64_t v2 = s_rem[tid];
-      if (j < n_r - 1) {
-        v2 = gf_mulmod(v2, cp.w.c_page[n_r - 2 - j]);
-        v2 = gf_mulmod(v2, cp.w.x_last[r]);
-      }
-      atomicXor(&cp.w.layer_rem[((int64_t)cp.layer * p.R + r) * F + tid], (unsigned long long)v2);
-    }
   }
+  if (failed && lane == 0) raise_error(kErrWait);
+  bulk_wait_all();
   pdl_epilogue(p.overlap);
+}
+
+// One warp per (layer, request, plane): rem_l = XOR over the items k of item_rem * x^(8 * bytes
+// that follow item k in the request's plane) = item_rem * c_tail[k].
+__global__ void __launch_bounds__(128)
+topkv_crc_layer_kernel(CrcWorkspace w, CrcGeom g, const int32_t* __restrict__ sl, int L, int R,
+                       int F, int maxp, int P) {
+  pdl_prologue(0);
+  const int lane = threadIdx.x & 31;
+  const int64_t q = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (q >= (int64_t)L * R * F) return;
+  const int c = (int)(q % F);
+  const int r = (int)((q / F) % R);
+  const int l = (int)(q / ((int64_t)F * R));
+  int64_t s = sl[r];
+  s = s < 0 ? 0 : (s > (int64_t)maxp * P ? (int64_t)maxp * P : s);
+  const int K = (int)((s * g.rpr + kCrcRunsPerItem - 1) / kCrcRunsPerItem);
+  uint64_t acc = 0;
+  for (int k = lane; k < K; k += 32) {
+    const uint64_t v = w.item_rem[(((int64_t)l * R + r) * g.kmax + k) * F + c];
+    acc ^= k == 0 ? v : gf_mulmod_clmul(v, w.c_tail[k]);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc ^= __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) w.layer_rem[((int64_t)l * R + r) * F + c] = acc;
 }
 
 // One thread per (request, plane): chains the layers,
@@ -310,8 +520,8 @@ topkv_crc_finish_kernel(CrcWorkspace w, const int32_t* __restrict__ sl, int L, i
   const uint64_t x_req = w.x_req[r];
   uint64_t state = ~0ull;
   for (int l = 0; l < L; ++l) {
-    const uint64_t rem = empty ? 0ull : (uint64_t)w.layer_rem[((int64_t)l * R + r) * F + c];
-    state = gf_mulmod(state, x_req) ^ rem;
+    const uint64_t rem = empty ? 0ull : w.layer_rem[((int64_t)l * R + r) * F + c];
+    state = gf_mulmod_clmul(state, x_req) ^ rem;
   }
   out[k] = ~state;
 }

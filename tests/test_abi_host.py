@@ -222,10 +222,16 @@ def test_host_crc64_header_and_retry():
     assert tk.topkv_retry(lambda: (calls.append(0), tk.TOPKV_ERR_CHECKSUM)[1], 2, 1) \
         == tk.TOPKV_ERR_CHECKSUM and len(calls) == 3                     # gives up after 1 + 2
     # workspace sizing and unsupported shapes
-    assert tk.topkv_crc_workspace_bytes(lo, 8, 256) == 8 * (32 + 257 + 16 + 80 * 8 * 2)
-    assert tk.topkv_crc_workspace_bytes(mla, 32, 128) == 8 * (128 + 129 + 64 + 61 * 32)
-    big = tk.make_layout(2, 2, 8, 128, 2, 512, 4)                    # 2 * 512 * 2 runs > 1024 threads
-    assert tk.topkv_crc_workspace_bytes(big, 1, 1) == tk.TOPKV_ERR_UNSUPPORTED_LAYOUT
+    # workspace sizing: 32 lane constants, kmax + 1 item constants, R request constants,
+    # L*R*kmax*F item remainders, L*R*F layer remainders, 8 bytes each; kmax = items of 32 runs
+    # (<= 1 KiB each) that one block-table row can hold
+    kmax = 256 * 16 * (2048 // 1024) // 32
+    assert tk.topkv_crc_workspace_bytes(lo, 8, 256) == \
+        8 * (32 + kmax + 1 + 8 + 80 * 8 * kmax * 2 + 80 * 8 * 2)
+    kmax = 128 * 64 * (1152 // 576) // 32                          # 1152-byte rows: 2 runs of 576
+    assert tk.topkv_crc_workspace_bytes(mla, 32, 128) == \
+        8 * (32 + kmax + 1 + 32 + 61 * 32 * kmax + 61 * 32)
+    assert tk.topkv_crc_workspace_bytes(lo, -1, 4) == tk.TOPKV_ERR_INVALID_ARG
 
 
 def test_empty_batches_launch_nothing():

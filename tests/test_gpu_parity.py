@@ -552,7 +552,7 @@ def test_windowed_layer_bench_shape(dev):
 
 # -------------------------------------------------------------------- header + CRC-64 (§3.4)
 
-def _crc_run(dev, g, sl, bt_s, bt_d, src_h, dst_h, corrupt=None):
+def _crc_run(dev, g, sl, bt_s, bt_d, src_h, dst_h, corrupt=None, use_plan=True, repeat_layer=None):
     """Sender: pack every layer with checksums. Receiver: unpack with checksums from the
     (optionally corrupted) wire. Returns wire, destination pool and both checksum arrays."""
     lo = _layout_from_geom(g)
@@ -562,11 +562,14 @@ def _crc_run(dev, g, sl, bt_s, bt_d, src_h, dst_h, corrupt=None):
     wire = torch.zeros(max(g.L * g.W_layer, 16), dtype=torch.uint8, device=dev)
     d_sl = torch.from_numpy(sl).to(dev)
     d_bs, d_bd = torch.from_numpy(bt_s).to(dev), torch.from_numpy(bt_d).to(dev)
-    cu = torch.zeros(R + 1, dtype=torch.int64, device=dev)
-    tk.check(tk.topkv_build_plan(tk.make_batch(d_bs, d_sl), cu))
-    bs, bd = tk.make_batch(d_bs, d_sl, T, cu), tk.make_batch(d_bd, d_sl, T, cu)
+    cu = None
+    if use_plan:
+        cu = torch.zeros(R + 1, dtype=torch.int64, device=dev)
+        tk.check(tk.topkv_build_plan(tk.make_batch(d_bs, d_sl), cu))
+    Tk = T if use_plan else -1                          # without a plan: total unknown as well
+    bs, bd = tk.make_batch(d_bs, d_sl, Tk, cu), tk.make_batch(d_bd, d_sl, Tk, cu)
     ov = tk.TOPKV_FLAG_OVERLAP_PREVIOUS                 # layers after the first may overlap
-    bs_ov, bd_ov = tk.make_batch(d_bs, d_sl, T, cu, ov), tk.make_batch(d_bd, d_sl, T, cu, ov)
+    bs_ov, bd_ov = tk.make_batch(d_bs, d_sl, Tk, cu, ov), tk.make_batch(d_bd, d_sl, Tk, cu, ov)
     nws = tk.topkv_crc_workspace_bytes(lo, R, bt_s.shape[1])
     assert nws > 0
     out = []
@@ -578,7 +581,10 @@ def _crc_run(dev, g, sl, bt_s, bt_d, src_h, dst_h, corrupt=None):
         order = list(range(g.L)) if side == 0 else list(reversed(range(g.L)))  # any layer order
         for k, layer in enumerate(order):
             tk.check(fn(layer, pool, lo, batch_ov if k else batch, wire, wire.numel(), ws, nws))
+        if repeat_layer is not None:                    # doing a layer again changes nothing
+            tk.check(fn(repeat_layer, pool, lo, batch, wire, wire.numel(), ws, nws))
         tk.check(tk.topkv_crc_finish(lo, batch, ws, nws, crc))
+        tk.check(tk.topkv_crc_finish(lo, batch, ws, nws, crc))   # and so does finishing twice
         torch.cuda.synchronize()
         out.append(crc.cpu().numpy().view(np.uint64).reshape(R, F))
         if side == 0 and corrupt is not None:
@@ -586,7 +592,7 @@ def _crc_run(dev, g, sl, bt_s, bt_d, src_h, dst_h, corrupt=None):
     return wire.cpu().numpy(), dst.cpu().numpy(), out[0], out[1]
 
 
-@pytest.mark.parametrize("seed", range(12))
+@pytest.mark.parametrize("seed", range(24))
 def test_crc_fused_pack_unpack(dev, seed, variant):
     if variant == 1:
         pytest.skip("the checksumming copy has one kernel family")
@@ -596,6 +602,8 @@ def test_crc_fused_pack_unpack(dev, seed, variant):
     P = int(rng.choice([1, 4, 16]))
     R = int(rng.integers(1, 5))
     sl = rng.integers(0, 4 * P + 2, size=R).astype(np.int32)
+    if seed >= 12:                                     # long requests: many items per plane
+        sl = rng.integers(0, 40 * P + 2, size=R).astype(np.int32)
     if seed % 4 == 1:
         sl[rng.integers(0, R)] = 0
     pages = (sl + P - 1) // P
@@ -608,6 +616,12 @@ def test_crc_fused_pack_unpack(dev, seed, variant):
         g.S_page = P * g.S_tok
         g.S_kv = npages * g.S_page
         g.S_layer = F * g.S_kv
+    elif seed % 3 == 1 and H > 1:                      # head-major inside the page
+        g.S_tok = D * 2
+        g.S_head = P * g.S_tok
+        g.S_kv = H * g.S_head
+        g.S_page = F * g.S_kv
+        g.S_layer = npages * g.S_page
     T = int(sl.sum())
     g.W_layer = g.wire_layer_bytes(T)
     bt_s = np.full((R, maxp), -1, dtype=np.int32)
@@ -619,7 +633,8 @@ def test_crc_fused_pack_unpack(dev, seed, variant):
         pos += pages[r]
     src_h = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
     dst_h = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
-    wire, dst, crc_tx, crc_rx = _crc_run(dev, g, sl, bt_s, bt_d, src_h, dst_h)
+    wire, dst, crc_tx, crc_rx = _crc_run(dev, g, sl, bt_s, bt_d, src_h, dst_h,
+                                         use_plan=seed % 2 == 0, repeat_layer=seed % g.L)
     want_wire = np.zeros(max(g.L * g.W_layer, 16), dtype=np.uint8)
     want_dst = dst_h.copy()
     for layer in range(g.L):
