@@ -328,11 +328,10 @@ __global__ void __launch_bounds__(kCrcMaxWarps * 32, 1) topkv_crc_copy_kernel(co
   int64_t next_item = (int64_t)blockIdx.x * W + warp;
   bool failed = false;
 
-  // Finds this warp's next item with anything to move and starts its loads into stage `slot`
-  // (every lane brings its own run). Returns false when the items are used up; otherwise *dst
-  // is where this lane's run goes (null when the lane has none) and *idx the item's place in
-  // item_rem. Uniform across the warp.
-  auto issue_next = [&](int slot, uint8_t** dst_out, int64_t* idx_out) -> bool {
+  // Finds this warp's next item with anything to move. Returns false when the items are used
+  // up; otherwise *src / *dst are where this lane's run comes from and goes to (null when the
+  // lane has none) and *idx is the item's place in item_rem. Uniform across the warp.
+  auto prepare_next = [&](const uint8_t** src_out, uint8_t** dst_out, int64_t* idx_out) -> bool {
     while (next_item < total_items) {
       const int64_t it = next_item;
       next_item += GW;
@@ -370,24 +369,37 @@ __global__ void __launch_bounds__(kCrcMaxWarps * 32, 1) topkv_crc_copy_kernel(co
           dst = PACK ? b : a;
         }
       }
-      const unsigned mask = __ballot_sync(0xffffffffu, active);
-      if (mask == 0) continue;
-      const uint32_t bar = smem_addr(&bars[warp * kCrcMaxStages + slot]);
-      if (lane == 0) mbar_expect_tx(bar, (uint32_t)(__popc(mask) * run_bytes));
-      __syncwarp();
-      if (active) bulk_g2s(smem_addr(my_row + (size_t)slot * stage_bytes), src, (uint32_t)run_bytes, bar);
+      if (__ballot_sync(0xffffffffu, active) == 0) continue;
+      *src_out = active ? src : nullptr;
       *dst_out = active ? dst : nullptr;
       *idx_out = (((int64_t)cp.layer * p.R + r) * cp.g.kmax + k) * F + c;
       return true;
     }
     return false;
   };
+  // Starts the loads of a prepared item into stage `slot`: every lane brings its own run.
+  auto launch_loads = [&](int slot, const uint8_t* src) {
+    const unsigned mask = __ballot_sync(0xffffffffu, src != nullptr);
+    const uint32_t bar = smem_addr(&bars[warp * kCrcMaxStages + slot]);
+    if (lane == 0) mbar_expect_tx(bar, (uint32_t)(__popc(mask) * run_bytes));
+    __syncwarp();
+    if (src != nullptr)
+      bulk_g2s(smem_addr(my_row + (size_t)slot * stage_bytes), src, (uint32_t)run_bytes, bar);
+  };
+  auto issue_next = [&](int slot, uint8_t** dst_out, int64_t* idx_out) -> bool {
+    const uint8_t* src;
+    if (!prepare_next(&src, dst_out, idx_out)) return false;
+    launch_loads(slot, src);
+    return true;
+  };
 
-  // Folds this lane's row of stage `slot`, sends the row on to `dst`, aligns the remainder to the
-  // item's end, combines the lanes and stores the item's remainder.
+  // Sends this lane's row of stage `slot` on to `dst` and, while the store reads the row, folds
+  // it; aligns the remainder to the item's end, combines the lanes, stores the item's remainder.
   auto fold_and_store = [&](int slot, uint8_t* dst, int64_t idx) {
     uint8_t* row_g = my_row + (size_t)slot * stage_bytes;
     uint64_t rem = 0;
+    if (dst != nullptr) bulk_s2g(dst, smem_addr(row_g), (uint32_t)run_bytes);
+    bulk_commit();
     if (dst != nullptr) {
       int off = 0;
 #pragma unroll 2
@@ -406,9 +418,7 @@ __global__ void __launch_bounds__(kCrcMaxWarps * 32, 1) topkv_crc_copy_kernel(co
         rem = gf_mulx64(rem ^ ((uint64_t)y.z | ((uint64_t)y.w << 32)));
       }
       rem = gf_mulmod_clmul(rem, c_lane);  // 31 - lane runs follow inside the item
-      bulk_s2g(dst, smem_addr(row_g), (uint32_t)run_bytes);
     }
-    bulk_commit();
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) rem ^= __shfl_xor_sync(0xffffffffu, rem, o);
     if (lane == 0) cp.w.item_rem[idx] = rem;
@@ -425,16 +435,22 @@ __global__ void __launch_bounds__(kCrcMaxWarps * 32, 1) topkv_crc_copy_kernel(co
   if (S == 1) {
     // One stage per warp: load, fold, store, wait for the store to have read the rows, next item.
     // The overlap of transfers and arithmetic comes from the other warps of the SM.
-    uint8_t* d;
-    int64_t ix;
+    const uint8_t* src;
+    uint8_t* dst;
+    int64_t idx;
     uint32_t parity = 0u;
-    while (issue_next(0, &d, &ix)) {
+    bool have = prepare_next(&src, &dst, &idx);
+    while (have) {
+      launch_loads(0, src);
+      uint8_t* const dst_cur = dst;
+      const int64_t idx_cur = idx;
+      have = prepare_next(&src, &dst, &idx);  // the next item's addresses, while the loads fly
       if (!wait_loaded(0, parity)) {
         failed = true;
         break;
       }
       parity ^= 1u;
-      fold_and_store(0, d, ix);
+      fold_and_store(0, dst_cur, idx_cur);
       bulk_wait_read<0>();
       __syncwarp();
     }
