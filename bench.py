@@ -515,6 +515,8 @@ def run_extra(name, dev, stream, args, peak):
         torch.cuda.empty_cache()
         return out
     if name in ("cfg3", "cfg4"):
+        if args.layers is not None:                      # fewer layers: profiling only
+            spec = wl.with_layers(spec, args.layers)
         w = harness.setup(spec, dev, fill_dst=False)
         ms, pack_ms, unpack_ms, _ = bench_d2d(w, stream, args.steps, args.warmup, nobar)
         traffic = 2.0 * w.n_layer * w.layers
