@@ -59,6 +59,7 @@ extern "C" {
 /* A CUDA stream handle (cudaStream_t). Declared opaquely so that this header
  * compiles without the CUDA toolkit. */
 typedef struct CUstream_st* topkv_stream_t;
+typedef struct CUevent_st* topkv_event_t;   /* opaque cudaEvent_t */
 
 typedef enum topkv_status {
   TOPKV_OK = 0,
@@ -263,6 +264,34 @@ int topkv_unpack_layer_from_host_crc(int layer, void* dst_pool, const topkv_layo
                                      void* d_staging, int64_t staging_capacity_bytes,
                                      void* d_workspace, int64_t workspace_bytes,
                                      topkv_stream_t stream);
+
+/* ---- layer-by-layer issue on a side stream (§5.2, Eq. 3) -------------------------------------
+ * The pipelined transfer as one call per side: for l = first_layer .. first_layer+num_layers-1,
+ * in order, on `side_stream`:
+ *     wait for layer_ready[l - first_layer]     (skipped when layer_ready == NULL or the entry is)
+ *     topkv_pack_layer_to_host(l, ...)          (topkv_unpack_layer_from_host for the receiver)
+ *     record layer_done[l - first_layer]        (skipped when layer_done == NULL or the entry is)
+ * so that the transfer of layer l runs while the caller's main stream computes layers l+1..,
+ * which recorded layer_ready[l] after layer l's K/V were written. A receiver passes the
+ * sender's layer_done events as its layer_ready. Only enqueues; returns after the last layer
+ * has been enqueued. Arguments, forms (d_staging NULL = direct) and errors as for the per-layer
+ * calls; the events are the caller's, created on the stream's device. Everything is validated
+ * for every layer before anything is enqueued, so on an error status nothing was launched,
+ * except TOPKV_ERR_CUDA from the runtime in the middle of the loop (layers before it stay
+ * enqueued). One staging slab serves all layers: they follow each other on one stream. */
+int topkv_pack_layers_to_host_pipelined(int first_layer, int num_layers, const void* src_pool,
+                                        const topkv_layout* layout, const topkv_batch* batch,
+                                        void* h_pinned, int64_t host_capacity_bytes, void* d_staging,
+                                        int64_t staging_capacity_bytes,
+                                        const topkv_event_t* layer_ready,
+                                        const topkv_event_t* layer_done, topkv_stream_t side_stream);
+int topkv_unpack_layers_from_host_pipelined(int first_layer, int num_layers, void* dst_pool,
+                                            const topkv_layout* layout, const topkv_batch* batch,
+                                            const void* h_pinned, int64_t host_bytes, void* d_staging,
+                                            int64_t staging_capacity_bytes,
+                                            const topkv_event_t* layer_ready,
+                                            const topkv_event_t* layer_done,
+                                            topkv_stream_t side_stream);
 
 /* Host-side retry policy of the transfer orchestrator (§3.1: 2 retries, 100 ms exponential
  * backoff): calls attempt(ctx) until it returns TOPKV_OK, at most 1 + retries times, sleeping

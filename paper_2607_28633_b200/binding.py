@@ -42,7 +42,8 @@ EXPORTS = (
     "topkv_header_fill", "topkv_header_check", "topkv_crc64", "topkv_crc_workspace_bytes",
     "topkv_crc_begin", "topkv_pack_layer_crc", "topkv_unpack_layer_crc", "topkv_crc_finish",
     "topkv_retry", "topkv_pack_layer_to_host_crc", "topkv_unpack_layer_from_host_crc",
-    "topkv_set_host_leg_ctas",
+    "topkv_set_host_leg_ctas", "topkv_pack_layers_to_host_pipelined",
+    "topkv_unpack_layers_from_host_pipelined",
 )
 
 
@@ -153,6 +154,9 @@ def lib() -> ctypes.CDLL:
         L.topkv_kernel_launch_count.restype = c_int64
         L.topkv_set_kernel_variant.argtypes = [c_int]
         L.topkv_set_host_leg_ctas.argtypes = [c_int]
+        for fn in (L.topkv_pack_layers_to_host_pipelined, L.topkv_unpack_layers_from_host_pipelined):
+            fn.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p, c_int64,
+                           c_void_p, c_void_p, c_void_p]
         _lib = L
     return _lib
 
@@ -246,6 +250,41 @@ def topkv_unpack_layer_from_host(layer, dst_pool, layout, batch, h_pinned, host_
                                               ctypes.byref(batch), _ptr(h_pinned), host_bytes,
                                               _ptr(d_staging), staging_capacity_bytes,
                                               _stream(stream))
+
+
+def _events(events, n):
+    """torch.cuda.Event list (entries may be None) -> C array of cudaEvent_t, or None."""
+    if events is None:
+        return None
+    assert len(events) == n
+    arr = (c_void_p * n)()
+    for i, e in enumerate(events):
+        if e is None:
+            continue
+        if not e.cuda_event:
+            # torch creates the CUDA event only at its first record(): give it a handle now
+            # (recording on the current stream; the library's own record replaces it)
+            e.record()
+        arr[i] = e.cuda_event
+    return arr
+
+
+def topkv_pack_layers_to_host_pipelined(first_layer, num_layers, src_pool, layout, batch, h_pinned,
+                                        host_capacity_bytes, d_staging, staging_capacity_bytes,
+                                        layer_ready=None, layer_done=None, side_stream=None):
+    return lib().topkv_pack_layers_to_host_pipelined(
+        first_layer, num_layers, _ptr(src_pool), ctypes.byref(layout), ctypes.byref(batch),
+        _ptr(h_pinned), host_capacity_bytes, _ptr(d_staging), staging_capacity_bytes,
+        _events(layer_ready, num_layers), _events(layer_done, num_layers), _stream(side_stream))
+
+
+def topkv_unpack_layers_from_host_pipelined(first_layer, num_layers, dst_pool, layout, batch, h_pinned,
+                                            host_bytes, d_staging, staging_capacity_bytes,
+                                            layer_ready=None, layer_done=None, side_stream=None):
+    return lib().topkv_unpack_layers_from_host_pipelined(
+        first_layer, num_layers, _ptr(dst_pool), ctypes.byref(layout), ctypes.byref(batch),
+        _ptr(h_pinned), host_bytes, _ptr(d_staging), staging_capacity_bytes,
+        _events(layer_ready, num_layers), _events(layer_done, num_layers), _stream(side_stream))
 
 
 def topkv_pack_layer_to_host_noalloc(layer, src_pool, layout, batch, h_pinned,

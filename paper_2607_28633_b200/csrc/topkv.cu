@@ -493,6 +493,64 @@ int crc_host_leg(int layer, const void* pool, const topkv_layout* layout,
 
 }  // namespace
 
+namespace {
+
+// Checks that every layer of the range would be accepted before the first one is enqueued.
+int check_layer_range(int first_layer, int num_layers, const void* pool, const topkv_layout* layout,
+                      const topkv_batch* batch, const void* h_pinned, int64_t host_bytes,
+                      const void* d_staging, int64_t staging_capacity_bytes) {
+  if (num_layers < 0 || first_layer < 0) return TOPKV_ERR_LAYER_RANGE;
+  if (layout == nullptr || batch == nullptr || h_pinned == nullptr) return TOPKV_ERR_INVALID_ARG;
+  KParams kp;
+  Resolved rs;
+  int64_t n_layer;
+  for (int i = 0; i < num_layers; ++i) {
+    const int st = prepare(first_layer + i, pool, layout, batch, h_pinned, host_bytes,
+                           layout->wire_layer_stride, &kp, &rs, &n_layer);
+    if (st != TOPKV_OK) return st;
+  }
+  if (d_staging != nullptr) {
+    if (batch->total_tokens < 0) return TOPKV_ERR_INVALID_ARG;
+    if (layout->wire_plane_stride != 0) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+    if (!mult16p(d_staging)) return TOPKV_ERR_ALIGNMENT;
+    if (staging_capacity_bytes < topkv_wire_layer_bytes(layout, batch->total_tokens)) return TOPKV_ERR_CAPACITY;
+  } else if (num_layers > 0) {
+    void* dev = nullptr;
+    const int st = mapped_device_pointer(h_pinned, &dev);  // refuses pageable memory up front
+    if (st != TOPKV_OK) return st;
+  }
+  return TOPKV_OK;
+}
+
+template <bool PACK>
+int issue_layers(int first_layer, int num_layers, const void* pool, const topkv_layout* layout,
+                 const topkv_batch* batch, const void* h_pinned, int64_t host_bytes, void* d_staging,
+                 int64_t staging_capacity_bytes, const topkv_event_t* layer_ready,
+                 const topkv_event_t* layer_done, topkv_stream_t side_stream) {
+  int st = check_layer_range(first_layer, num_layers, pool, layout, batch, h_pinned, host_bytes, d_staging,
+                             staging_capacity_bytes);
+  if (st != TOPKV_OK) return st;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(side_stream);
+  for (int i = 0; i < num_layers; ++i) {
+    if (layer_ready != nullptr && layer_ready[i] != nullptr) {
+      const cudaError_t e = cudaStreamWaitEvent(s, reinterpret_cast<cudaEvent_t>(layer_ready[i]), 0);
+      if (e != cudaSuccess) return cuda_fail(e);
+    }
+    st = PACK ? topkv_pack_layer_to_host(first_layer + i, pool, layout, batch, const_cast<void*>(h_pinned),
+                                         host_bytes, d_staging, staging_capacity_bytes, side_stream)
+              : topkv_unpack_layer_from_host(first_layer + i, const_cast<void*>(pool), layout, batch, h_pinned,
+                                             host_bytes, d_staging, staging_capacity_bytes, side_stream);
+    if (st != TOPKV_OK) return st;
+    if (layer_done != nullptr && layer_done[i] != nullptr) {
+      const cudaError_t e = cudaEventRecord(reinterpret_cast<cudaEvent_t>(layer_done[i]), s);
+      if (e != cudaSuccess) return cuda_fail(e);
+    }
+  }
+  return TOPKV_OK;
+}
+
+}  // namespace
+
 extern "C" {
 
 int topkv_pack_layer(int layer, const void* src_pool, const topkv_layout* layout,
@@ -591,6 +649,27 @@ int topkv_unpack_layer_from_host(int layer, void* dst_pool, const topkv_layout* 
   }
   kp.wire = static_cast<uint8_t*>(d_staging);
   return launch_copy<false>(kp, rs, (int)layout->kv_factor, s);
+}
+
+int topkv_pack_layers_to_host_pipelined(int first_layer, int num_layers, const void* src_pool,
+                                        const topkv_layout* layout, const topkv_batch* batch,
+                                        void* h_pinned, int64_t host_capacity_bytes, void* d_staging,
+                                        int64_t staging_capacity_bytes,
+                                        const topkv_event_t* layer_ready,
+                                        const topkv_event_t* layer_done, topkv_stream_t side_stream) {
+  return issue_layers<true>(first_layer, num_layers, src_pool, layout, batch, h_pinned, host_capacity_bytes,
+                            d_staging, staging_capacity_bytes, layer_ready, layer_done, side_stream);
+}
+
+int topkv_unpack_layers_from_host_pipelined(int first_layer, int num_layers, void* dst_pool,
+                                            const topkv_layout* layout, const topkv_batch* batch,
+                                            const void* h_pinned, int64_t host_bytes, void* d_staging,
+                                            int64_t staging_capacity_bytes,
+                                            const topkv_event_t* layer_ready,
+                                            const topkv_event_t* layer_done,
+                                            topkv_stream_t side_stream) {
+  return issue_layers<false>(first_layer, num_layers, dst_pool, layout, batch, h_pinned, host_bytes,
+                             d_staging, staging_capacity_bytes, layer_ready, layer_done, side_stream);
 }
 
 int topkv_pack_layer_to_host_noalloc(int layer, const void* src_pool, const topkv_layout* layout,

@@ -29,7 +29,7 @@ class OverlapResult:
     t_main_overlap_ms: float
     t_layer_compute_ms: float
     t_xfer_serial_ms: float
-    t_xfer_overlapped_ms: float
+    t_xfer_overlapped_ms: float | None
     exposed_ms: float
     hidden: float
     hidden_upper_bound: float
@@ -136,15 +136,27 @@ def run_overlap(w: DeviceWorkload, h_pinned: torch.Tensor, staging, prefill: Pre
             prefill.layer()
             done[l].record(main)
         s1.record(main)
-    for l in range(L):
-        side.wait_event(done[l])
-        bo[l].record(side)
-        xfer(l, side)
-        eo[l].record(side)
+    if slots >= L and crc_workspace is None:
+        # the whole side-stream schedule as one library call: wait done[l], ship layer l,
+        # record eo[l] (topkv_pack_layers_to_host_pipelined); bo[l] is not needed for `hidden`
+        cap = 0 if staging is None else staging.numel()
+        tk.check(tk.topkv_pack_layers_to_host_pipelined(
+            0, L, w.src_pool, w.layout, w.src_batch, h_pinned, h_pinned.numel(), staging, cap,
+            done, eo, side))
+        bo = None
+    else:
+        for l in range(L):
+            side.wait_event(done[l])
+            bo[l].record(side)
+            xfer(l, side)
+            eo[l].record(side)
     torch.cuda.synchronize(dev)
     t_main_overlap = s0.elapsed_time(s1)
     exposed = max(0.0, s1.elapsed_time(eo[L - 1]))
-    t_xfer_overlapped = sum(bo[l].elapsed_time(eo[l]) for l in range(L))
+    # sum of the per-layer spans in the overlapped pass (not observable when the schedule was
+    # issued as one library call: no event sits between a layer's wait and its transfer)
+    t_xfer_overlapped = (sum(bo[l].elapsed_time(eo[l]) for l in range(L)) if bo is not None
+                         else None)
     hidden = 1.0 - exposed / t_xfer_serial if t_xfer_serial > 0 else 1.0
     return OverlapResult(
         layers=L, t_main_alone_ms=t_main_alone, t_main_overlap_ms=t_main_overlap,

@@ -1052,6 +1052,61 @@ def test_relay_through_host_on_two_streams(dev):
     torch.cuda.empty_cache()
 
 
+@pytest.mark.parametrize("staged", [True, False])
+def test_pipelined_layer_range_calls(dev, staged):
+    """topkv_pack_layers_to_host_pipelined / topkv_unpack_layers_from_host_pipelined: one call
+    per side enqueues the whole layer-by-layer transfer, gated by per-layer events. Sender and
+    receiver run on two streams; the receiver's layer_ready are the sender's layer_done."""
+    spec = wl.with_layers(wl.CFG2, 4)
+    w = harness.setup(spec, dev, need_wire=False)
+    b = w.batch
+    g = _geom(spec, b.num_pool_pages, 1, 0, 0)
+    L, n = 4, w.n_layer
+    pinned = torch.zeros(L * n, dtype=torch.uint8).pin_memory()
+    st_tx = torch.zeros(n, dtype=torch.uint8, device=dev) if staged else None
+    st_rx = torch.zeros(n, dtype=torch.uint8, device=dev) if staged else None
+    cap = n if staged else 0
+    before = [harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, l) for l in range(L)]
+    main = torch.cuda.current_stream(dev)
+    tx, rx = torch.cuda.Stream(dev, priority=-1), torch.cuda.Stream(dev)
+    x = torch.randn(2048, 2048, device=dev)
+    ready = []
+    for layer in range(L):                               # stands for the prefill of layer l
+        x = (x @ x.T) * 1e-3
+        ev = torch.cuda.Event()
+        ev.record(main)
+        ready.append(ev if layer != 2 else None)         # a missing entry means "no wait"
+    main.synchronize()                                   # layer 2 has no event: it must be ready
+    sent = [torch.cuda.Event() for _ in range(L)]
+    # layers 1..3 first, then layer 0 alone: ranges are independent calls
+    tk.check(tk.topkv_pack_layers_to_host_pipelined(1, 3, w.src_pool, w.layout, w.src_batch, pinned,
+                                                    pinned.numel(), st_tx, cap, ready[1:], sent[1:], tx))
+    tk.check(tk.topkv_pack_layers_to_host_pipelined(0, 1, w.src_pool, w.layout, w.src_batch, pinned,
+                                                    pinned.numel(), st_tx, cap, ready[:1], sent[:1], tx))
+    tk.check(tk.topkv_unpack_layers_from_host_pipelined(0, L, w.dst_pool, w.layout, w.dst_batch, pinned,
+                                                        pinned.numel(), st_rx, cap, sent, None, rx))
+    torch.cuda.synchronize()
+    for layer in range(L):
+        src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, layer)
+        want = oracle.pack(g, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=8)
+        assert np.array_equal(pinned[layer * n:(layer + 1) * n].numpy(), want)
+        oracle.unpack(g, 0, before[layer], b.dst_block_table, b.seq_lens, want, impl="rows", threads=8)
+        assert np.array_equal(harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, layer), before[layer])
+    # errors are found for the whole range before anything is enqueued
+    launches = tk.topkv_kernel_launch_count()
+    assert tk.topkv_pack_layers_to_host_pipelined(2, 3, w.src_pool, w.layout, w.src_batch, pinned,
+                                                  pinned.numel(), st_tx, cap, None, None, tx) \
+        == tk.TOPKV_ERR_LAYER_RANGE
+    assert tk.topkv_pack_layers_to_host_pipelined(0, L, w.src_pool, w.layout, w.src_batch, pinned,
+                                                  pinned.numel() - 16, st_tx, cap, None, None, tx) \
+        == tk.TOPKV_ERR_CAPACITY
+    assert tk.topkv_kernel_launch_count() == launches
+    assert tk.topkv_pack_layers_to_host_pipelined(0, 0, w.src_pool, w.layout, w.src_batch, pinned,
+                                                  pinned.numel(), st_tx, cap, None, None, tx) == tk.TOPKV_OK
+    del w
+    torch.cuda.empty_cache()
+
+
 def test_smoke_entry(dev):
     import __graft_entry__ as entry
     entry.smoke()
