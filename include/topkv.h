@@ -265,6 +265,21 @@ int topkv_unpack_layer_from_host_crc(int layer, void* dst_pool, const topkv_layo
                                      void* d_workspace, int64_t workspace_bytes,
                                      topkv_stream_t stream);
 
+/* Several layers in ONE launch: the layers first_layer .. first_layer + num_layers - 1 of the
+ * same batch, exactly as num_layers calls of topkv_pack_layer / topkv_unpack_layer would move
+ * them (layer l between pool + l*pool_layer_stride and wire + l*wire_layer_stride). For the side
+ * that is not pipelined layer by layer (§5.2 sends per layer; a receiver that gets a whole
+ * payload, a re-send after a failed check, §3.1, small decode-side batches), where the launch
+ * and the ramp of one kernel per layer would dominate. layout->wire_layer_stride must be > 0
+ * when num_layers > 1 (TOPKV_ERR_INVALID_ARG); num_layers <= 65535; num_layers == 0 validates
+ * and launches nothing. Other arguments, flags and errors as for the per-layer calls. */
+int topkv_pack_layers(int first_layer, int num_layers, const void* src_pool,
+                      const topkv_layout* layout, const topkv_batch* batch, void* d_wire,
+                      int64_t wire_capacity_bytes, topkv_stream_t stream);
+int topkv_unpack_layers(int first_layer, int num_layers, void* dst_pool, const topkv_layout* layout,
+                        const topkv_batch* batch, const void* d_wire, int64_t wire_bytes,
+                        topkv_stream_t stream);
+
 /* ---- layer-by-layer issue on a side stream (§5.2, Eq. 3) -------------------------------------
  * The pipelined transfer as one call per side: for l = first_layer .. first_layer+num_layers-1,
  * in order, on `side_stream`:

@@ -43,7 +43,7 @@ EXPORTS = (
     "topkv_crc_begin", "topkv_pack_layer_crc", "topkv_unpack_layer_crc", "topkv_crc_finish",
     "topkv_retry", "topkv_pack_layer_to_host_crc", "topkv_unpack_layer_from_host_crc",
     "topkv_set_host_leg_ctas", "topkv_pack_layers_to_host_pipelined",
-    "topkv_unpack_layers_from_host_pipelined",
+    "topkv_unpack_layers_from_host_pipelined", "topkv_pack_layers", "topkv_unpack_layers",
 )
 
 
@@ -154,6 +154,8 @@ def lib() -> ctypes.CDLL:
         L.topkv_kernel_launch_count.restype = c_int64
         L.topkv_set_kernel_variant.argtypes = [c_int]
         L.topkv_set_host_leg_ctas.argtypes = [c_int]
+        L.topkv_pack_layers.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p]
+        L.topkv_unpack_layers.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p]
         for fn in (L.topkv_pack_layers_to_host_pipelined, L.topkv_unpack_layers_from_host_pipelined):
             fn.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p, c_int64,
                            c_void_p, c_void_p, c_void_p]
@@ -235,6 +237,19 @@ def topkv_pack_layer(layer, src_pool, layout, batch, d_wire, wire_capacity_bytes
 def topkv_unpack_layer(layer, dst_pool, layout, batch, d_wire, wire_bytes, stream=None):
     return lib().topkv_unpack_layer(layer, _ptr(dst_pool), ctypes.byref(layout),
                                     ctypes.byref(batch), _ptr(d_wire), wire_bytes, _stream(stream))
+
+
+def topkv_pack_layers(first_layer, num_layers, src_pool, layout, batch, d_wire, wire_capacity_bytes,
+                      stream=None):
+    return lib().topkv_pack_layers(first_layer, num_layers, _ptr(src_pool), ctypes.byref(layout),
+                                   ctypes.byref(batch), _ptr(d_wire), wire_capacity_bytes,
+                                   _stream(stream))
+
+
+def topkv_unpack_layers(first_layer, num_layers, dst_pool, layout, batch, d_wire, wire_bytes,
+                        stream=None):
+    return lib().topkv_unpack_layers(first_layer, num_layers, _ptr(dst_pool), ctypes.byref(layout),
+                                     ctypes.byref(batch), _ptr(d_wire), wire_bytes, _stream(stream))
 
 
 def topkv_pack_layer_to_host(layer, src_pool, layout, batch, h_pinned, host_capacity_bytes,

@@ -152,6 +152,8 @@ int prepare(int layer, const void* pool, const topkv_layout* lo, const topkv_bat
   kp->num_pages = lo->num_pool_pages;
   kp->wire_limit = (n_layer >= 0 && !spread) ? n_layer : capacity - (int64_t)layer * wire_layer_stride;
   kp->plane_rows = spread ? lo->wire_plane_stride / rs->row_bytes : -1;
+  kp->S_layer = 0;
+  kp->W_layer = 0;
   return TOPKV_OK;
 }
 
@@ -251,12 +253,15 @@ int launch_bulk(const KParams& kp0, const Resolved& rs, int F, cudaStream_t stre
 }
 
 // max_ctas > 0: the wire is host memory behind PCIe; at most that many CTAs walk the spans.
+// layers > 1: one launch covers that many consecutive layers (kp describes the first one and
+// carries the layer strides); the vectorised family only.
 template <bool PACK>
-int launch_copy(KParams kp, const Resolved& rs, int F, cudaStream_t stream, int max_ctas = 0) {
+int launch_copy(KParams kp, const Resolved& rs, int F, cudaStream_t stream, int max_ctas = 0,
+                int layers = 1) {
   const int64_t slots = (int64_t)kp.R * kp.maxp;
-  if (slots == 0) return TOPKV_OK;
+  if (slots == 0 || layers == 0) return TOPKV_OK;
   bool handled = false;
-  if (max_ctas <= 0 && g_variant.load(std::memory_order_relaxed) == 1) {
+  if (max_ctas <= 0 && layers == 1 && g_variant.load(std::memory_order_relaxed) == 1) {
     const int st = launch_bulk<PACK>(kp, rs, F, stream, &handled);
     if (st != TOPKV_OK) return st;
   }
@@ -267,7 +272,7 @@ int launch_copy(KParams kp, const Resolved& rs, int F, cudaStream_t stream, int 
     kp.spr = (kp.maxp + kp.ppc - 1) / kp.ppc;
     const int64_t spans = (int64_t)kp.R * kp.spr;
     const bool walk = max_ctas > 0 && spans > max_ctas;
-    const dim3 grid((unsigned)(walk ? max_ctas : spans));
+    const dim3 grid((unsigned)(walk ? max_ctas : spans), (unsigned)layers);
     // 32-byte vectors when every address the kernel can form is 32-byte aligned
     const bool wide = ((reinterpret_cast<uintptr_t>(kp.pool) | reinterpret_cast<uintptr_t>(kp.wire) |
                         (uintptr_t)kp.S_page | (uintptr_t)kp.S_kv | (uintptr_t)kp.S_tok |
@@ -551,6 +556,41 @@ int issue_layers(int first_layer, int num_layers, const void* pool, const topkv_
 
 }  // namespace
 
+namespace {
+namespace multi {
+
+// One launch for the layers [first_layer, first_layer + num_layers).
+template <bool PACK>
+int copy_layers(int first_layer, int num_layers, const void* pool, const topkv_layout* layout,
+                const topkv_batch* batch, const void* d_wire, int64_t wire_bytes, cudaStream_t s) {
+  if (num_layers < 0 || first_layer < 0) return TOPKV_ERR_LAYER_RANGE;
+  if (num_layers > 65535) return TOPKV_ERR_INVALID_ARG;  // grid.y
+  KParams kp, kp_last;
+  Resolved rs;
+  int64_t n_layer;
+  if (num_layers == 0) {  // still validate the descriptors
+    if (layout == nullptr) return TOPKV_ERR_INVALID_ARG;
+    const int st = check_layout(layout, &rs);
+    return st != TOPKV_OK ? st : check_batch(layout, batch);
+  }
+  int st = prepare(first_layer, pool, layout, batch, d_wire, wire_bytes,
+                   layout ? layout->wire_layer_stride : 0, &kp, &rs, &n_layer);
+  if (st != TOPKV_OK) return st;
+  st = prepare(first_layer + num_layers - 1, pool, layout, batch, d_wire, wire_bytes,
+               layout->wire_layer_stride, &kp_last, &rs, &n_layer);  // range and capacity of the last
+  if (st != TOPKV_OK) return st;
+  if (num_layers > 1) {
+    if (layout->wire_layer_stride <= 0) return TOPKV_ERR_INVALID_ARG;  // all layers on one slab
+    kp.S_layer = layout->pool_layer_stride;
+    kp.W_layer = layout->wire_layer_stride;
+    kp.wire_limit = std::min(kp.wire_limit, kp_last.wire_limit);  // the tightest slab bounds them all
+  }
+  return launch_copy<PACK>(kp, rs, (int)layout->kv_factor, s, 0, num_layers);
+}
+
+}  // namespace multi
+}  // namespace
+
 extern "C" {
 
 int topkv_pack_layer(int layer, const void* src_pool, const topkv_layout* layout,
@@ -575,6 +615,21 @@ int topkv_unpack_layer(int layer, void* dst_pool, const topkv_layout* layout,
                          layout ? layout->wire_layer_stride : 0, &kp, &rs, &n_layer);
   if (st != TOPKV_OK) return st;
   return launch_copy<false>(kp, rs, (int)layout->kv_factor, reinterpret_cast<cudaStream_t>(stream));
+}
+
+
+int topkv_pack_layers(int first_layer, int num_layers, const void* src_pool, const topkv_layout* layout,
+                      const topkv_batch* batch, void* d_wire, int64_t wire_capacity_bytes,
+                      topkv_stream_t stream) {
+  return multi::copy_layers<true>(first_layer, num_layers, src_pool, layout, batch, d_wire, wire_capacity_bytes,
+                                  reinterpret_cast<cudaStream_t>(stream));
+}
+
+int topkv_unpack_layers(int first_layer, int num_layers, void* dst_pool, const topkv_layout* layout,
+                        const topkv_batch* batch, const void* d_wire, int64_t wire_bytes,
+                        topkv_stream_t stream) {
+  return multi::copy_layers<false>(first_layer, num_layers, dst_pool, layout, batch, d_wire, wire_bytes,
+                                   reinterpret_cast<cudaStream_t>(stream));
 }
 
 int topkv_pack_layer_to_host(int layer, const void* src_pool, const topkv_layout* layout,

@@ -32,6 +32,7 @@ struct KParams {
   int64_t num_pages;      // pages per pool slab: every page id is checked against it
   int64_t wire_limit;     // bytes that may be touched behind `wire` (this layer's slab)
   int overlap;            // 1: caller declared this launch independent of the kernels before it
+  int64_t S_layer, W_layer;  // multi-layer launch: bytes from one layer's slab to the next (pool, wire)
 };
 
 // Error bits raised by kernels (never a trap): read back with topkv_device_error_flags().
@@ -61,7 +62,7 @@ __device__ __forceinline__ void pdl_prologue(int overlap) {
   pdl_release_next_grid();
 }
 __device__ __forceinline__ void pdl_epilogue(int overlap) {
-  if (overlap && blockIdx.x == 0 && threadIdx.x == 0) pdl_wait_prior_grid();
+  if (overlap && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) pdl_wait_prior_grid();
 }
 
 // Streaming vector accesses: every byte is touched exactly once, so neither side should

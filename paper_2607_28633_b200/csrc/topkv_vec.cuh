@@ -59,6 +59,9 @@ __device__ __forceinline__ void copy_span(const KParams& p, const int slot) {
   // A span = `ppc` consecutive page columns of one request (one page when pages are large;
   // several small pages, so that every CTA moves a few tens of KiB).
   __shared__ int32_t s_pages[kMaxPagesPerCta];
+  // blockIdx.y = layer of a multi-layer launch (0 and zero strides for a single layer)
+  uint8_t* const pool = p.pool + (int64_t)blockIdx.y * p.S_layer;
+  uint8_t* const wire = p.wire + (int64_t)blockIdx.y * p.W_layer;
   const int r = slot / p.spr;
   const int j0 = (slot - r * p.spr) * p.ppc;
   const int s_r = p.sl[r];
@@ -116,12 +119,12 @@ __device__ __forceinline__ void copy_span(const KParams& p, const int slot) {
       if (s_pages[jj] < 0) continue;
       const int t_lo = max(0, ts0 - jj * p.P), t_hi = min(p.P, ts0 + v - jj * p.P);
       const int n = (t_hi - t_lo) * p.unit_chunks;
-      uint8_t* pool_page = p.pool + (int64_t)s_pages[jj] * p.S_page + (int64_t)t_lo * p.S_tok;
+      uint8_t* pool_page = pool + (int64_t)s_pages[jj] * p.S_page + (int64_t)t_lo * p.S_tok;
 #pragma unroll
       for (int c = 0; c < F; ++c) {
         uint8_t* a = pool_page + c * p.S_kv;
         // not planar => F == 1
-        uint8_t* b = p.wire +
+        uint8_t* b = wire +
                      ((p.planar ? c * PR : 0) + n0 + (int64_t)(jj * p.P + t_lo - ts0)) * unit_bytes;
         const uint8_t* src = PACK ? a : b;
         uint8_t* dst = PACK ? b : a;
@@ -151,9 +154,9 @@ __device__ __forceinline__ void copy_span(const KParams& p, const int slot) {
   const int my_g = tid / tpu;
   const int my_w = tid - my_g * tpu;
   if (my_g >= groups) return;
-  uint8_t* wire_span = p.wire + n0 * F * p.U * unit_bytes;  // TOKEN_KV: the span is one run
+  uint8_t* wire_span = wire + n0 * F * p.U * unit_bytes;  // TOKEN_KV: the span is one run
   if (!MULTI && s_pages[0] < 0) return;                     // single page, unusable: skip it
-  uint8_t* page0 = p.pool + (int64_t)s_pages[0] * p.S_page + (int64_t)ts0 * p.S_tok;
+  uint8_t* page0 = pool + (int64_t)s_pages[0] * p.S_page + (int64_t)ts0 * p.S_tok;
 
   for (int q0 = my_g; q0 < nunits; q0 += groups * kUnroll) {
     for (int w = my_w; w < p.unit_chunks; w += tpu) {
@@ -173,7 +176,7 @@ __device__ __forceinline__ void copy_span(const KParams& p, const int slot) {
         if (p.planar) {
           c = (F > 1 && tc >= v) ? 1 : 0;
           ts = tc - c * v;
-          b = p.wire + (((int64_t)c * PR + n0 + ts) * p.U + h) * unit_bytes + (int64_t)w * VEC;
+          b = wire + (((int64_t)c * PR + n0 + ts) * p.U + h) * unit_bytes + (int64_t)w * VEC;
         } else {
           ts = tc / F;
           c = tc - ts * F;
@@ -183,7 +186,7 @@ __device__ __forceinline__ void copy_span(const KParams& p, const int slot) {
           const int jj = (ts0 + ts) / p.P;
           const int t = ts0 + ts - jj * p.P;
           const int pg = s_pages[jj];
-          a = p.pool + (int64_t)pg * p.S_page + c * p.S_kv + t * p.S_tok + h * p.S_unit +
+          a = pool + (int64_t)pg * p.S_page + c * p.S_kv + t * p.S_tok + h * p.S_unit +
               (int64_t)w * VEC;
           ok[u] = q0 + u * groups < nunits && pg >= 0;
         } else {

@@ -1107,6 +1107,59 @@ def test_pipelined_layer_range_calls(dev, staged):
     torch.cuda.empty_cache()
 
 
+@pytest.mark.parametrize("seed", range(10))
+def test_many_layers_in_one_launch(dev, seed, variant):
+    """topkv_pack_layers / topkv_unpack_layers equal the oracle's per-layer pack / unpack for a
+    range of layers of the layout (random geometries: strided and head-split pools, both wire
+    orders, padded wire slabs, empty batches); the layer outside the range is untouched."""
+    g, sl, bt_s, bt_d, rng = _case(seed)
+    g.L = 3
+    g.W_layer = max(g.W_layer, 16)                     # several layers need distinct slabs
+    lo = _layout_from_geom(g)
+    T = int(sl.sum())
+    src_h = rng.integers(0, 256, g.L * g.S_layer, dtype=np.uint8)
+    fill_h = rng.integers(0, 256, g.L * g.S_layer, dtype=np.uint8)
+    wire_len = g.L * g.W_layer + 32
+    src, dst = torch.from_numpy(src_h).to(dev), torch.from_numpy(fill_h.copy()).to(dev)
+    wire = torch.full((wire_len,), 0x3C, dtype=torch.uint8, device=dev)
+    d_sl = torch.from_numpy(sl).to(dev)
+    d_bs, d_bd = torch.from_numpy(bt_s).to(dev), torch.from_numpy(bt_d).to(dev)
+    know_T = seed % 2 == 0
+    bs = tk.make_batch(d_bs, d_sl, T if know_T else -1)
+    bd = tk.make_batch(d_bd, d_sl, T if know_T else -1)
+    first, count = 1, g.L - 1
+    tk.check(tk.topkv_pack_layers(first, count, src, lo, bs, wire, wire.numel()))
+    want_wire = np.full(wire_len, 0x3C, dtype=np.uint8)
+    want_dst = fill_h.copy()
+    for layer in range(first, first + count):
+        oracle.pack(g, layer, src_h, bt_s, sl, wire=want_wire)
+        oracle.unpack(g, layer, want_dst, bt_d, sl, want_wire)
+    torch.cuda.synchronize()
+    assert np.array_equal(wire.cpu().numpy(), want_wire)
+    tk.check(tk.topkv_unpack_layers(first, count, dst, lo, bd, wire, wire.numel()))
+    torch.cuda.synchronize()
+    assert np.array_equal(dst.cpu().numpy(), want_dst)
+    assert np.array_equal(src.cpu().numpy(), src_h)
+    assert tk.topkv_pack_layers(1, g.L, src, lo, bs, wire, wire.numel()) == tk.TOPKV_ERR_LAYER_RANGE
+    assert tk.topkv_pack_layers(0, 0, src, lo, bs, wire, wire.numel()) == tk.TOPKV_OK
+
+
+def test_many_layers_in_one_launch_cfg1(dev, variant):
+    w = harness.setup(wl.CFG1, dev)
+    b, s = w.batch, wl.CFG1
+    g = _geom(s, b.num_pool_pages, s.L, 0, w.n_layer)
+    src_h, dst_h = w.src_pool.cpu().numpy(), w.dst_pool.cpu().numpy()
+    tk.check(tk.topkv_pack_layers(0, s.L, w.src_pool, w.layout, w.src_batch, w.wire, w.wire.numel()))
+    tk.check(tk.topkv_unpack_layers(0, s.L, w.dst_pool, w.layout, w.dst_batch, w.wire, w.wire.numel()))
+    torch.cuda.synchronize()
+    want = np.zeros(s.L * w.n_layer, dtype=np.uint8)
+    for layer in range(s.L):
+        oracle.pack(g, layer, src_h, b.src_block_table, b.seq_lens, wire=want)
+        oracle.unpack(g, layer, dst_h, b.dst_block_table, b.seq_lens, want)
+    assert np.array_equal(w.wire.cpu().numpy(), want)
+    assert np.array_equal(w.dst_pool.cpu().numpy(), dst_h)
+
+
 def test_smoke_entry(dev):
     import __graft_entry__ as entry
     entry.smoke()
