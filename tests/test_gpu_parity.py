@@ -257,7 +257,8 @@ def test_small_pages_many_per_cta(dev, P, H, D):
             assert np.array_equal(dst.cpu().numpy(), dst_h), (order, F)
 
 
-def test_unusable_tables_are_skipped_not_followed(dev):
+@pytest.mark.parametrize("path", ["per_layer", "layer_range", "checksummed"])
+def test_unusable_tables_are_skipped_not_followed(dev, path, variant):
     """Device-side checks: a page id outside the pool, a length longer than its table row and
     lengths that overflow the wire slab raise status bits; the affected work is skipped, the
     rest is copied, and nothing outside the buffers is touched (guard bands, untouched pool)."""
@@ -277,12 +278,22 @@ def test_unusable_tables_are_skipped_not_followed(dev):
         d_bt, d_sl = torch.from_numpy(bt_dev).to(dev), torch.from_numpy(sl_dev).to(dev)
         b = tk.make_batch(d_bt, d_sl, total)
         tk.check(tk.topkv_reset_device_error_flags())
-        tk.check(tk.topkv_pack_layer(0, src, lo, b, buf[guard:], cap))
+        if path == "per_layer":
+            tk.check(tk.topkv_pack_layer(0, src, lo, b, buf[guard:], cap))
+        elif path == "layer_range":
+            tk.check(tk.topkv_pack_layers(0, 1, src, lo, b, buf[guard:], cap))
+        else:
+            nws = tk.topkv_crc_workspace_bytes(lo, len(sl_dev), bt_dev.shape[1])
+            ws = torch.zeros(nws, dtype=torch.uint8, device=dev)
+            tk.check(tk.topkv_crc_begin(lo, b, ws, nws))
+            tk.check(tk.topkv_pack_layer_crc(0, src, lo, b, buf[guard:], cap, ws, nws))
         flags = tk.topkv_device_error_flags()
         out = buf.cpu().numpy()
         assert (out[:guard] == 0xC3).all() and (out[guard + n:] == 0xC3).all()
         return flags, out[guard:guard + n]
 
+    if path == "checksummed" and variant == 1:
+        pytest.skip("the checksumming copy has one kernel family")
     want = oracle.pack(g, 0, src_h, bt, sl)
     flags, got = run(bt, sl, T, n)
     assert flags == 0 and np.array_equal(got, want)
