@@ -35,6 +35,26 @@ def test_exports_every_declared_symbol():
     assert tk.topkv_version() >= 100
 
 
+def test_plain_c_client_builds_links_and_runs(tmp_path):
+    """The header is valid C99 and the library is usable from C: a small client includes
+    include/topkv.h, links against libtopkv.so and calls the entry points that need no GPU."""
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("gcc not available")
+    tk.lib()
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    libdir = os.path.dirname(tk.LIB_PATH)
+    exe = str(tmp_path / "abi_c_client")
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic",
+                           "-I", os.path.join(root, "include"),
+                           os.path.join(root, "tests", "native", "abi_c_client.c"),
+                           "-o", exe, "-L", libdir, "-l:libtopkv.so", "-Wl,-rpath," + libdir])
+    out = subprocess.run([exe], capture_output=True, text=True, timeout=60)
+    assert out.returncode == 0, out.stderr
+    assert "abi_c_client ok" in out.stdout
+
+
 def test_struct_sizes_match_header():
     # natural alignment of the C structs: 10 x u32 + 8 x i64, and 4 x 32-bit + 3 ptr + i64 + 2 x i32
     assert ctypes.sizeof(tk.topkv_layout) == 104
