@@ -78,6 +78,8 @@ def _load():
         lib.oracle_crc64_iso.argtypes = [vp, i64]
         lib.oracle_kv_plane_crc.restype = u64
         lib.oracle_kv_plane_crc.argtypes = [gp, vp, i64, i64, vp, vp, i64, i64]
+        lib.oracle_kv_plane_crc_layered.restype = u64
+        lib.oracle_kv_plane_crc_layered.argtypes = [gp, vp, i64, i64, vp, vp, i64, i64, vp]
         _lib = lib
     return _lib
 
@@ -253,12 +255,21 @@ def crc64(data, poly_reflected: int = POLY_ISO_REFLECTED) -> int:
     return int(_load().oracle_crc64(a.ctypes.data, a.size, poly_reflected))
 
 
-def kv_plane_crc(g: Geom, pool: np.ndarray, bt: np.ndarray, sl: np.ndarray, r: int, c: int) -> int:
+def kv_plane_crc(g: Geom, pool: np.ndarray, bt: np.ndarray, sl: np.ndarray, r: int, c: int,
+                 layer_windows=None) -> int:
     """CRC-64 of the K (c = 0) or V (c = 1) tensor of request r in the order
-    [layers][seq_len][kv_heads][head_dim], gathered from the paged pool."""
+    [layers][seq_len][kv_heads][head_dim], gathered from the paged pool. ``layer_windows``
+    (one entry per layer, 0 = full) describes a model with windowed layers (§2.2): every layer
+    contributes the tokens it keeps."""
     bt, sl = _tables(bt, sl)
     _u8(pool, False)
     cg = g._c()
+    if layer_windows is not None:
+        lw = np.ascontiguousarray(layer_windows, dtype=np.int64)
+        assert lw.shape == (g.L,)
+        return int(_load().oracle_kv_plane_crc_layered(
+            ctypes.byref(cg), pool.ctypes.data, sl.shape[0], bt.shape[1], bt.ctypes.data,
+            sl.ctypes.data, r, c, lw.ctypes.data))
     return int(_load().oracle_kv_plane_crc(ctypes.byref(cg), pool.ctypes.data, sl.shape[0],
                                            bt.shape[1], bt.ctypes.data, sl.ctypes.data, r, c))
 

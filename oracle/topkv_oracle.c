@@ -220,3 +220,23 @@ uint64_t oracle_kv_plane_crc(const oracle_geom* g, const uint8_t* pool, int64_t 
     }
   return ~crc;
 }
+
+uint64_t oracle_kv_plane_crc_layered(const oracle_geom* g, const uint8_t* pool, int64_t R,
+                                     int64_t maxp, const int32_t* bt, const int32_t* sl, int64_t r,
+                                     int64_t c, const int64_t* layer_window) {
+  (void)R;
+  uint64_t crc = ~(uint64_t)0;
+  for (int64_t l = 0; l < g->L; ++l) {
+    int64_t W = layer_window[l];
+    int64_t i0 = (W > 0 && sl[r] > W) ? sl[r] - W : 0; /* a windowed layer keeps the last W */
+    for (int64_t i = i0; i < sl[r]; ++i) {
+      int64_t page = bt[r * maxp + i / g->P];
+      int64_t t = i % g->P;
+      for (int64_t h = 0; h < g->h_kv; ++h)
+        for (int64_t d = 0; d < g->d_h; ++d)
+          for (int64_t b = 0; b < g->b_p; ++b)
+            crc = crc64_byte(crc, pool[poff(g, l, page, c, t, h, d, b)], ORACLE_POLY_ISO_REFLECTED);
+    }
+  }
+  return ~crc;
+}

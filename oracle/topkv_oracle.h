@@ -74,4 +74,10 @@ uint64_t oracle_crc64_iso(const uint8_t* data, int64_t n);
  * table. A windowed geometry contributes only the tokens it keeps. */
 uint64_t oracle_kv_plane_crc(const oracle_geom* g, const uint8_t* pool, int64_t R, int64_t maxp,
                              const int32_t* bt, const int32_t* sl, int64_t r, int64_t c);
+/* The same for a model whose layers differ in kind (§2.2): layer l keeps all tokens when
+ * layer_window[l] == 0, else the last min(s, layer_window[l]); the tensor that is checksummed
+ * is the concatenation, layer by layer, of what each layer keeps. g->window is not used. */
+uint64_t oracle_kv_plane_crc_layered(const oracle_geom* g, const uint8_t* pool, int64_t R,
+                                     int64_t maxp, const int32_t* bt, const int32_t* sl, int64_t r,
+                                     int64_t c, const int64_t* layer_window);
 #endif

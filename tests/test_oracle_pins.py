@@ -519,6 +519,45 @@ def test_kv_plane_crc_is_the_crc_of_the_paper_payload_order():
     g.wire_order = WIRE_TOKEN_KV
 
 
+def test_layered_kv_plane_crc_is_the_crc_of_what_every_layer_keeps():
+    # a model whose layers alternate full / windowed (§2.2): the checksummed tensor is the
+    # concatenation, layer by layer, of the rows each layer keeps; built here from the windowed
+    # PLANAR pack of each layer (pack with a window is pinned above) and checksummed
+    import copy
+    g, pool, bt, sl = _random_case(33, 2, 2, 8, 4, strided=True)
+    g.L = 4
+    pool = np.random.default_rng(34).integers(0, 256, size=g.L * g.S_layer, dtype=np.uint8)
+    g.W_layer = 0
+    g.wire_order = WIRE_PLANAR
+    windows = [0, 5, 0, 2]
+    R = len(sl)
+    planes, cus = [], []
+    for l in range(g.L):
+        gl = copy.copy(g)
+        gl.window = windows[l]
+        kept = sl.astype(np.int64) if windows[l] == 0 else np.minimum(sl.astype(np.int64), windows[l])
+        cu = np.concatenate([[0], np.cumsum(kept)])
+        planes.append(oracle.pack(gl, l, pool, bt, sl).reshape(g.F, int(cu[-1]), g.row_bytes))
+        cus.append(cu)
+    for r in range(R):
+        for c in range(g.F):
+            tensor = np.concatenate([planes[l][c, cus[l][r]:cus[l][r + 1]].reshape(-1)
+                                     for l in range(g.L)])
+            assert oracle.kv_plane_crc(g, pool, bt, sl, r, c, layer_windows=windows) == \
+                oracle.crc64(tensor.tobytes())
+    # no windows anywhere: the plain routine
+    for r in range(R):
+        assert oracle.kv_plane_crc(g, pool, bt, sl, r, 0, layer_windows=[0] * g.L) == \
+            oracle.kv_plane_crc(g, pool, bt, sl, r, 0)
+    # the same window on every layer: the routine with a windowed geometry
+    gw = copy.copy(g)
+    gw.window = 3
+    for r in range(R):
+        assert oracle.kv_plane_crc(g, pool, bt, sl, r, 1, layer_windows=[3] * g.L) == \
+            oracle.kv_plane_crc(gw, pool, bt, sl, r, 1)
+    g.wire_order = WIRE_TOKEN_KV
+
+
 def test_header_layout():
     g = Geom(L=80, F=2, h_kv=8, d_h=128, b_p=2, P=16, num_pages=1)
     h = oracle.build_header(7, 0xABCDEF, 4096, g, 0x1122334455667788, 0x99AABBCCDDEEFF00)
