@@ -236,10 +236,13 @@ uint64_t topkv_crc64(const void* h_data, int64_t nbytes);
  * 8-byte remainder per 32 runs (of at most 1 KiB) of every request, plane and layer, i.e.
  * about N_layer * L / 4096 bytes (Llama-3-70B shape, 8 x 4096 tokens: 2.6 MB). d_crc_out:
  * DEVICE uint64 [R*F]. batch->cu_seq_lens and total_tokens are optional (the kernel rebuilds
- * the prefix sums from seq_lens), head-split pools are supported; window_tokens must be 0 and
- * num_requests at most 8192 (else TOPKV_ERR_UNSUPPORTED_LAYOUT). TOPKV_FLAG_OVERLAP_PREVIOUS
- * may be set as for the plain calls. The bytes moved are identical to topkv_pack_layer /
- * topkv_unpack_layer. */
+ * the prefix sums from seq_lens), head-split pools are supported; num_requests at most 8192
+ * (else TOPKV_ERR_UNSUPPORTED_LAYOUT). Layers may differ in kind (§2.2): a layer copied with
+ * batch->window_tokens = W contributes the last min(s, W) tokens of every request to the
+ * checksum, exactly the rows it ships; the workspace remembers each layer's window for
+ * topkv_crc_finish, whose own batch argument only supplies the tables (its window_tokens is
+ * ignored). TOPKV_FLAG_OVERLAP_PREVIOUS may be set as for the plain calls. The bytes moved are
+ * identical to topkv_pack_layer / topkv_unpack_layer. */
 int64_t topkv_crc_workspace_bytes(const topkv_layout* layout, int32_t num_requests,
                                   int32_t max_pages_per_req);
 int topkv_crc_begin(const topkv_layout* layout, const topkv_batch* batch, void* d_workspace,

@@ -424,7 +424,6 @@ int crc_copy(int layer, const void* pool, const topkv_layout* lo, const topkv_ba
   if (n_layer_out != nullptr) *n_layer_out = n_layer;
   if (slab_override != nullptr) cp.k.wire = static_cast<uint8_t*>(slab_override);
   if (ws == nullptr || !mult16p(ws)) return TOPKV_ERR_INVALID_ARG;
-  if (b->window_tokens != 0) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
   const int F = (int)lo->kv_factor, R = b->num_requests, maxp = b->max_pages_per_req;
   const int L = (int)lo->num_layers;
   if (R > kCrcMaxR) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
@@ -875,7 +874,6 @@ int topkv_crc_begin(const topkv_layout* layout, const topkv_batch* batch, void* 
   st = check_batch(layout, batch);
   if (st != TOPKV_OK) return st;
   if (d_workspace == nullptr || !mult16p(d_workspace)) return TOPKV_ERR_INVALID_ARG;
-  if (batch->window_tokens != 0) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
   const int F = (int)layout->kv_factor, R = batch->num_requests, maxp = batch->max_pages_per_req;
   const int L = (int)layout->num_layers;
   CrcGeom g;
@@ -884,7 +882,7 @@ int topkv_crc_begin(const topkv_layout* layout, const topkv_batch* batch, void* 
   if (workspace_bytes < 8 * crc_workspace_words(g.kmax, L, R, F)) return TOPKV_ERR_CAPACITY;
   if (R == 0) return TOPKV_OK;
   const CrcWorkspace w = crc_carve(d_workspace, g.kmax, L, R, F);
-  const int64_t total = crc_workspace_words(g.kmax, L, R, F) - (int64_t)L * R * F;
+  const int64_t total = std::max<int64_t>(32 + (int64_t)g.kmax + 1 + R + (int64_t)L * R * g.kmax * F, L);
   const unsigned blocks = (unsigned)std::min<int64_t>((total + 255) / 256, 1024);
   topkv_crc_begin_kernel<<<blocks, 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
       w, g, batch->seq_lens, L, R, maxp, (int)layout->page_tokens, rs.row_bytes, F);
@@ -932,7 +930,8 @@ int topkv_crc_finish(const topkv_layout* layout, const topkv_batch* batch, void*
                                                                      (int)layout->page_tokens);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
-  topkv_crc_finish_kernel<<<(R * F + 127) / 128, 128, 0, s>>>(w, batch->seq_lens, L, R, F, d_crc_out);
+  topkv_crc_finish_kernel<<<(R * F + 127) / 128, 128, 0, s>>>(w, batch->seq_lens, L, R, F, maxp,
+                                                                (int)layout->page_tokens, rs.row_bytes, d_crc_out);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
   g_launches.fetch_add(2, std::memory_order_relaxed);

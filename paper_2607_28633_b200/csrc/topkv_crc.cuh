@@ -166,12 +166,16 @@ __host__ __device__ inline uint64_t gf_powx(uint64_t n) {
 //                               stored (not accumulated) by the copy, so packing a layer again
 //                               just rewrites its entries
 // layer_rem[L * R * F]          written by topkv_crc_finish
+// layer_win[L] (int32)          window with which layer l was last copied (0 = all tokens), cleared
+//                               by topkv_crc_begin: the chain over the layers needs every
+//                               layer's own length
 struct CrcWorkspace {
   uint64_t* c_run;
   uint64_t* c_tail;
   uint64_t* x_req;
   uint64_t* item_rem;
   uint64_t* layer_rem;
+  int32_t* layer_win;
 };
 
 constexpr int kCrcRunsPerItem = 32;  // one run per lane
@@ -194,7 +198,8 @@ struct CrcGeom {
 };
 
 __host__ __device__ inline int64_t crc_workspace_words(int kmax, int L, int R, int F) {
-  return 32 + ((int64_t)kmax + 1) + (int64_t)R + (int64_t)L * R * kmax * F + (int64_t)L * R * F;
+  return 32 + ((int64_t)kmax + 1) + (int64_t)R + (int64_t)L * R * kmax * F + (int64_t)L * R * F +
+         ((int64_t)L + 1) / 2;
 }
 
 __host__ __device__ inline CrcWorkspace crc_carve(void* base, int kmax, int L, int R, int F) {
@@ -204,6 +209,7 @@ __host__ __device__ inline CrcWorkspace crc_carve(void* base, int kmax, int L, i
   w.x_req = w.c_tail + (kmax + 1);
   w.item_rem = w.x_req + R;
   w.layer_rem = w.item_rem + (int64_t)L * R * kmax * F;
+  w.layer_win = reinterpret_cast<int32_t*>(w.layer_rem + (int64_t)L * R * F);
   return w;
 }
 
@@ -229,6 +235,7 @@ topkv_crc_begin_kernel(CrcWorkspace w, CrcGeom g, const int32_t* __restrict__ sl
     } else {
       w.item_rem[k - 32 - n_tail - R] = 0ull;
     }
+    if (k < L) w.layer_win[k] = 0;
   }
 }
 
@@ -273,12 +280,14 @@ __global__ void __launch_bounds__(kCrcMaxWarps * 32, 1) topkv_crc_copy_kernel(co
       raise_error(kErrTable);
       s = s < 0 ? 0 : row_tokens;
     }
+    if (p.window > 0 && s > p.window) s = p.window;  // a windowed layer keeps the last min(s, W)
     s_cu[q + 1] = s;
     s_ic[q + 1] = (int32_t)((s * rpr + kCrcRunsPerItem - 1) / kCrcRunsPerItem);
   }
   if (threadIdx.x == 0) {
     s_cu[0] = 0;
     s_ic[0] = 0;
+    if (blockIdx.x == 0) cp.w.layer_win[cp.layer] = p.window;  // for the chain over the layers
   }
   if (lane == 0)
     for (int q = 0; q < S; ++q) mbar_init(smem_addr(&bars[warp * kCrcMaxStages + q]), 1);
@@ -345,17 +354,21 @@ __global__ void __launch_bounds__(kCrcMaxWarps * 32, 1) topkv_crc_copy_kernel(co
       }
       const int r = lo;
       const int64_t cu_r = s_cu[r];
-      const int64_t n_r = (s_cu[r + 1] - cu_r) * rpr;  // runs of this request's plane
+      const int64_t kept = s_cu[r + 1] - cu_r;          // tokens this layer keeps of request r
+      const int64_t n_r = kept * rpr;                   // runs of this request's plane
       const int k = s_ic[r + 1] - 1 - m;                // full items that follow this one
       const int g = (int)(n_r - (int64_t)kCrcRunsPerItem * (k + 1)) + lane;  // this lane's run
       bool active = g >= 0;
       const uint8_t* src = nullptr;
       uint8_t* dst = nullptr;
       if (active) {
-        const int t = g / rpr;                               // token inside the request
+        const int t = g / rpr;                               // kept token of the request
         const int u = g - t * rpr;                           // run inside the row
         const int h = u / cp.g.rpu, seg = u - h * cp.g.rpu;  // unit (head) and run inside it
-        const int j = t / p.P, tt = t - j * p.P;
+        int64_t s_r = p.sl[r];                               // the kept tokens are the LAST ones
+        s_r = s_r < 0 ? 0 : (s_r > row_tokens ? row_tokens : s_r);
+        const int ta = (int)(s_r - kept) + t;                // token inside the sequence
+        const int j = ta / p.P, tt = ta - j * p.P;
         const int64_t page = p.bt[(int64_t)r * p.maxp + j];
         if (page < 0 || page >= p.num_pages) {  // unusable entry: the run is skipped
           raise_error(kErrTable);
@@ -511,6 +524,8 @@ topkv_crc_layer_kernel(CrcWorkspace w, CrcGeom g, const int32_t* __restrict__ sl
   const int l = (int)(q / ((int64_t)F * R));
   int64_t s = sl[r];
   s = s < 0 ? 0 : (s > (int64_t)maxp * P ? (int64_t)maxp * P : s);
+  const int64_t win = w.layer_win[l];
+  if (win > 0 && s > win) s = win;
   const int K = (int)((s * g.rpr + kCrcRunsPerItem - 1) / kCrcRunsPerItem);
   uint64_t acc = 0;
   for (int k = lane; k < K; k += 32) {
@@ -523,21 +538,34 @@ topkv_crc_layer_kernel(CrcWorkspace w, CrcGeom g, const int32_t* __restrict__ sl
 }
 
 // One thread per (request, plane): chains the layers,
-//   state_0 = ~0,  state_l+1 = state_l * x^(8 * bytes of the plane in one layer) + rem_l,
-// and inverts. A request without tokens has remainder 0 in every layer.
+//   state_0 = ~0,  state_l+1 = state_l * x^(8 * bytes of the plane in layer l) + rem_l,
+// and inverts. A layer copied with a window contributes min(s, window) tokens; a request
+// without tokens has remainder 0 in every layer.
 __global__ void __launch_bounds__(128)
-topkv_crc_finish_kernel(CrcWorkspace w, const int32_t* __restrict__ sl, int L, int R, int F,
-                        uint64_t* __restrict__ out) {
+topkv_crc_finish_kernel(CrcWorkspace w, const int32_t* __restrict__ sl, int L, int R, int F, int maxp,
+                        int P, int64_t row_bytes, uint64_t* __restrict__ out) {
   pdl_prologue(0);
   const int k = blockIdx.x * blockDim.x + threadIdx.x;
   if (k >= R * F) return;
   const int r = k / F, c = k - r * F;
-  const bool empty = sl[r] <= 0;
-  const uint64_t x_req = w.x_req[r];
+  int64_t s = sl[r];
+  s = s < 0 ? 0 : (s > (int64_t)maxp * P ? (int64_t)maxp * P : s);
+  const uint64_t x_full = w.x_req[r];
+  uint64_t x_win = 0;  // x^(8 * bytes of a windowed layer's plane), for the window seen last
+  int64_t seen = -1;
   uint64_t state = ~0ull;
   for (int l = 0; l < L; ++l) {
-    const uint64_t rem = empty ? 0ull : w.layer_rem[((int64_t)l * R + r) * F + c];
-    state = gf_mulmod_clmul(state, x_req) ^ rem;
+    const int64_t win = w.layer_win[l];
+    uint64_t x_len = x_full;
+    if (win > 0 && s > win) {
+      if (win != seen) {
+        x_win = gf_powx(8ull * (uint64_t)win * (uint64_t)row_bytes);
+        seen = win;
+      }
+      x_len = x_win;
+    }
+    const uint64_t rem = s == 0 ? 0ull : w.layer_rem[((int64_t)l * R + r) * F + c];
+    state = gf_mulmod_clmul(state, x_len) ^ rem;
   }
   out[k] = ~state;
 }

@@ -243,14 +243,15 @@ def test_host_crc64_header_and_retry():
         == tk.TOPKV_ERR_CHECKSUM and len(calls) == 3                     # gives up after 1 + 2
     # workspace sizing and unsupported shapes
     # workspace sizing: 32 lane constants, kmax + 1 item constants, R request constants,
-    # L*R*kmax*F item remainders, L*R*F layer remainders, 8 bytes each; kmax = items of 32 runs
+    # L*R*kmax*F item remainders, L*R*F layer remainders, 8 bytes each, and one int32 window per
+    # layer; kmax = items of 32 runs
     # (<= 1 KiB each) that one block-table row can hold
     kmax = 256 * 16 * (2048 // 1024) // 32
     assert tk.topkv_crc_workspace_bytes(lo, 8, 256) == \
-        8 * (32 + kmax + 1 + 8 + 80 * 8 * kmax * 2 + 80 * 8 * 2)
+        8 * (32 + kmax + 1 + 8 + 80 * 8 * kmax * 2 + 80 * 8 * 2 + 40)
     kmax = 128 * 64 * (1152 // 576) // 32                          # 1152-byte rows: 2 runs of 576
     assert tk.topkv_crc_workspace_bytes(mla, 32, 128) == \
-        8 * (32 + kmax + 1 + 32 + 61 * 32 * kmax + 61 * 32)
+        8 * (32 + kmax + 1 + 32 + 61 * 32 * kmax + 61 * 32 + 31)
     assert tk.topkv_crc_workspace_bytes(lo, -1, 4) == tk.TOPKV_ERR_INVALID_ARG
 
 

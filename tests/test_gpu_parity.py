@@ -659,6 +659,74 @@ def test_crc_fused_pack_unpack(dev, seed, variant):
             assert int(crc_rx[r, c]) == want
 
 
+@pytest.mark.parametrize("seed", range(8))
+def test_crc_with_windowed_layers(dev, seed, variant):
+    """A model whose layers differ in kind (§2.2): full layers and windowed layers with two
+    different windows. Every layer is packed / unpacked with its own window; the checksums
+    equal the oracle's CRC over what every layer keeps, the bytes the oracle's windowed pack."""
+    if variant == 1:
+        pytest.skip("the checksumming copy has one kernel family")
+    import copy
+    rng = np.random.default_rng(900 + seed)
+    F = int(rng.integers(1, 3))
+    H, D = [(8, 128), (1, 576), (2, 64), (4, 32)][seed % 4]
+    P = int(rng.choice([1, 4, 16]))
+    R = int(rng.integers(1, 5))
+    sl = rng.integers(0, 12 * P + 2, size=R).astype(np.int32)
+    if seed % 3 == 0:
+        sl[rng.integers(0, R)] = 0
+    L = 5
+    windows = [0, 2 * P + 1, 0, 3, 2 * P + 1]
+    pages = (sl + P - 1) // P
+    maxp = max(int(pages.max()), 1) + 1
+    npages = int(pages.sum()) + 2
+    g = Geom(L=L, F=F, h_kv=H, d_h=D, b_p=2, P=P, num_pages=npages, wire_order=seed % 2)
+    g.W_layer = g.wire_layer_bytes(int(sl.sum()))      # slabs sized for a full layer
+    bt_s = np.full((R, maxp), -1, dtype=np.int32)
+    bt_d = np.full((R, maxp), -1, dtype=np.int32)
+    ps, pd, pos = rng.permutation(npages), rng.permutation(npages), 0
+    for r in range(R):
+        bt_s[r, :pages[r]] = ps[pos:pos + pages[r]]
+        bt_d[r, :pages[r]] = pd[pos:pos + pages[r]]
+        pos += pages[r]
+    src_h = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
+    dst_h = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
+    lo = _layout_from_geom(g)
+    src, dst = torch.from_numpy(src_h).to(dev), torch.from_numpy(dst_h.copy()).to(dev)
+    wire = torch.zeros(max(L * g.W_layer, 16), dtype=torch.uint8, device=dev)
+    d_sl = torch.from_numpy(sl).to(dev)
+    d_bs, d_bd = torch.from_numpy(bt_s).to(dev), torch.from_numpy(bt_d).to(dev)
+    nws = tk.topkv_crc_workspace_bytes(lo, R, maxp)
+    got = []
+    want_wire = np.zeros(max(L * g.W_layer, 16), dtype=np.uint8)
+    want_dst = dst_h.copy()
+    for side, (pool, d_bt, fn) in enumerate(((src, d_bs, tk.topkv_pack_layer_crc),
+                                             (dst, d_bd, tk.topkv_unpack_layer_crc))):
+        ws = torch.full((nws,), 0x77, dtype=torch.uint8, device=dev)
+        crc = torch.zeros(R * F, dtype=torch.int64, device=dev)
+        tk.check(tk.topkv_crc_begin(lo, tk.make_batch(d_bt, d_sl), ws, nws))
+        for layer in range(L):
+            W = windows[layer]
+            kept = int(sl.sum()) if W == 0 else int(np.minimum(sl, W).sum())
+            batch = tk.make_batch(d_bt, d_sl, kept if seed % 2 else -1, None, 0, W)
+            tk.check(fn(layer, pool, lo, batch, wire, wire.numel(), ws, nws))
+        tk.check(tk.topkv_crc_finish(lo, tk.make_batch(d_bt, d_sl), ws, nws, crc))
+        torch.cuda.synchronize()
+        got.append(crc.cpu().numpy().view(np.uint64).reshape(R, F))
+    for layer in range(L):
+        gl = copy.copy(g)
+        gl.window = windows[layer]
+        oracle.pack(gl, layer, src_h, bt_s, sl, wire=want_wire)
+        oracle.unpack(gl, layer, want_dst, bt_d, sl, want_wire)
+    assert np.array_equal(wire.cpu().numpy(), want_wire)
+    assert np.array_equal(dst.cpu().numpy(), want_dst)
+    for r in range(R):
+        for c in range(F):
+            want = oracle.kv_plane_crc(g, src_h, bt_s, sl, r, c, layer_windows=windows)
+            assert int(got[0][r, c]) == want, (r, c)
+            assert int(got[1][r, c]) == want
+
+
 def test_crc_cfg1_header_round_trip_and_corruption(dev, variant):
     """cfg1 end to end: the sender's headers verify on the receiver; one flipped wire bit makes
     exactly the affected request fail with TOPKV_ERR_CHECKSUM, and the retry policy of §3.1
