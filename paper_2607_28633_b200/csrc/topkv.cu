@@ -495,10 +495,7 @@ int crc_host_leg(int layer, const void* pool, const topkv_layout* layout,
   return TOPKV_OK;
 }
 
-}  // namespace
-
-namespace {
-
+// ---- ranges of layers --------------------------------------------------------------------------
 // Checks that every layer of the range would be accepted before the first one is enqueued.
 int check_layer_range(int first_layer, int num_layers, const void* pool, const topkv_layout* layout,
                       const topkv_batch* batch, const void* h_pinned, int64_t host_bytes,
@@ -553,9 +550,6 @@ int issue_layers(int first_layer, int num_layers, const void* pool, const topkv_
   return TOPKV_OK;
 }
 
-}  // namespace
-
-namespace {
 namespace multi {
 
 // One launch for the layers [first_layer, first_layer + num_layers).
