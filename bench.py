@@ -295,33 +295,44 @@ def bench_host_leg(w, stream, pinned, staging, steps, warmup, barrier, slots):
 
 
 def bench_host_relay(w, stream, pinned, staging_tx, staging_rx, steps, warmup, barrier, slots):
-    """The same layers through pinned host memory, pipelined the way a relay would run it: one
-    stream packs layer l to the host while a second stream, gated by a per-layer event, unpacks
-    the layers that have already arrived, so both directions of the PCIe link are busy.
-    Returns ms per step (first pack enqueued to last unpack finished)."""
+    """The same layers through pinned host memory, pipelined the way a relay would run it: layer
+    l is packed to the host while layers that have already arrived are unpacked from it, so both
+    directions of the PCIe link are busy. Each direction alternates between two streams with a
+    staging slab each, so that the copy engine moves layer l while the kernel of layer l + 1
+    runs. Returns ms per step (first pack enqueued to last unpack finished)."""
     import ctypes
     import torch
     from paper_2607_28633_b200 import binding as tk
     L, n = w.layers, w.n_layer
+    dev = w.src_pool.device
     lo = type(w.layout)()
     ctypes.memmove(ctypes.byref(lo), ctypes.byref(w.layout), ctypes.sizeof(lo))
     lo.wire_layer_stride = 0
-    rx = torch.cuda.Stream(w.src_pool.device)
     assert slots >= L, "the relay keeps every layer's slab until it is unpacked"
+    tx = [torch.cuda.Stream(dev), torch.cuda.Stream(dev)]
+    rx = [torch.cuda.Stream(dev), torch.cuda.Stream(dev)]
+    st_tx = [staging_tx, torch.empty_like(staging_tx)]
+    st_rx = [staging_rx, torch.empty_like(staging_rx)]
 
     def step():
+        start = torch.cuda.Event()
+        start.record(stream)
+        for q in tx:
+            q.wait_event(start)
         for l in range(L):
             slab = pinned[l * n:(l + 1) * n]
-            tk.check(tk.topkv_pack_layer_to_host(l, w.src_pool, lo, w.src_batch, slab, n, staging_tx,
-                                                 staging_tx.numel(), stream))
+            a, b = tx[l & 1], rx[l & 1]
+            tk.check(tk.topkv_pack_layer_to_host(l, w.src_pool, lo, w.src_batch, slab, n, st_tx[l & 1],
+                                                 n, a))
             arrived = torch.cuda.Event()
-            arrived.record(stream)
-            rx.wait_event(arrived)
+            arrived.record(a)
+            b.wait_event(arrived)
             tk.check(tk.topkv_unpack_layer_from_host(l, w.dst_pool, lo, w.dst_batch, slab, n,
-                                                     staging_rx, staging_rx.numel(), rx))
-        done = torch.cuda.Event()
-        done.record(rx)
-        stream.wait_event(done)          # the step ends when the last unpack has finished
+                                                     st_rx[l & 1], n, b))
+        for q in rx:                     # the step ends when the last unpacks have finished
+            done = torch.cuda.Event()
+            done.record(q)
+            stream.wait_event(done)
 
     for _ in range(warmup):
         step()

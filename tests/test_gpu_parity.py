@@ -1102,26 +1102,32 @@ def test_side_stream_overlap_run_is_bit_exact(dev, variant):
     torch.cuda.empty_cache()
 
 
-def test_relay_through_host_on_two_streams(dev):
-    """pack_to_host on one stream, unpack_from_host on another, gated per layer by an event:
-    the destination pool ends up as the oracle's unpack of the oracle's pack."""
-    spec = wl.with_layers(wl.CFG2, 3)
+@pytest.mark.parametrize("streams_per_direction", [1, 2])
+def test_relay_through_host_on_two_streams(dev, streams_per_direction):
+    """pack_to_host on one set of streams, unpack_from_host on another, gated per layer by an
+    event (with two streams per direction, each with its own staging slab, the copy engine moves
+    layer l while the kernel of layer l + 1 runs: the configuration bench.py times as e2e): the
+    destination pool ends up as the oracle's unpack of the oracle's pack."""
+    L, k = 5, streams_per_direction
+    spec = wl.with_layers(wl.CFG2, L)
     w = harness.setup(spec, dev)
     b = w.batch
     g = _geom(spec, b.num_pool_pages, 1, 0, 0)
-    tx, rx = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
-    pinned = torch.zeros(3 * w.n_layer, dtype=torch.uint8).pin_memory()
-    st_tx = torch.zeros(w.n_layer, dtype=torch.uint8, device=dev)
-    st_rx = torch.zeros(w.n_layer, dtype=torch.uint8, device=dev)
-    before = [harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, l) for l in range(3)]
-    for layer in range(3):
-        w.pack_to_host(layer, pinned, st_tx, tx)
+    tx = [torch.cuda.Stream(dev) for _ in range(k)]
+    rx = [torch.cuda.Stream(dev) for _ in range(k)]
+    pinned = torch.zeros(L * w.n_layer, dtype=torch.uint8).pin_memory()
+    st_tx = [torch.zeros(w.n_layer, dtype=torch.uint8, device=dev) for _ in range(k)]
+    st_rx = [torch.zeros(w.n_layer, dtype=torch.uint8, device=dev) for _ in range(k)]
+    before = [harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, l) for l in range(L)]
+    for layer in range(L):
+        q = layer % k
+        w.pack_to_host(layer, pinned, st_tx[q], tx[q])
         ev = torch.cuda.Event()
-        ev.record(tx)
-        rx.wait_event(ev)
-        w.unpack_from_host(layer, pinned, st_rx, rx)
+        ev.record(tx[q])
+        rx[q].wait_event(ev)
+        w.unpack_from_host(layer, pinned, st_rx[q], rx[q])
     torch.cuda.synchronize()
-    for layer in range(3):
+    for layer in range(L):
         src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, layer)
         want = oracle.pack(g, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=8)
         assert np.array_equal(pinned[layer * w.n_layer:(layer + 1) * w.n_layer].numpy(), want)
