@@ -250,9 +250,11 @@ def bench_d2d(w, stream, steps, warmup, barrier):
     return total_ms / steps, pack_ms / steps, unpack_ms / steps, launches
 
 
-def bench_host_leg(w, stream, pinned, staging, steps, warmup, barrier, slots):
+def bench_host_leg(w, stream, pinned, staging, steps, warmup, barrier, slots, staging2=None):
     """pack_to_host for all layers then unpack_from_host for all layers, through pinned host
-    memory (``slots`` slabs used as a ring). Returns ms per step and the two phase times."""
+    memory (``slots`` slabs used as a ring). With ``staging2`` the layers alternate between two
+    streams with a staging slab each, so that the copy engine moves layer l while the kernel of
+    layer l + 1 runs. Returns ms per step and the two phase times."""
     import ctypes
     import torch
     from paper_2607_28633_b200 import binding as tk
@@ -261,18 +263,36 @@ def bench_host_leg(w, stream, pinned, staging, steps, warmup, barrier, slots):
     ctypes.memmove(ctypes.byref(lo), ctypes.byref(w.layout), ctypes.sizeof(lo))
     lo.wire_layer_stride = 0
     cap = 0 if staging is None else staging.numel()
+    second = torch.cuda.Stream(w.src_pool.device) if staging2 is not None else None
+
+    def phase(call):
+        """All layers through `call`, on one stream or alternating between two."""
+        if second is None:
+            for l in range(L):
+                call(l, staging, stream)
+            return
+        fork = torch.cuda.Event()
+        fork.record(stream)
+        second.wait_event(fork)
+        for l in range(L):
+            call(l, staging if l % 2 == 0 else staging2, stream if l % 2 == 0 else second)
+        join = torch.cuda.Event()
+        join.record(second)
+        stream.wait_event(join)
+
+    def to_host(l, st, q):
+        slab = pinned[(l % slots) * n:(l % slots + 1) * n]
+        tk.check(tk.topkv_pack_layer_to_host(l, w.src_pool, lo, w.src_batch, slab, n, st, cap, q))
+
+    def from_host(l, st, q):
+        slab = pinned[(l % slots) * n:(l % slots + 1) * n]
+        tk.check(tk.topkv_unpack_layer_from_host(l, w.dst_pool, lo, w.dst_batch, slab, n, st, cap, q))
 
     def step(rec):
         e0 = torch.cuda.Event(enable_timing=True); e0.record(stream)
-        for l in range(L):
-            slab = pinned[(l % slots) * n:(l % slots + 1) * n]
-            tk.check(tk.topkv_pack_layer_to_host(l, w.src_pool, lo, w.src_batch, slab, n, staging,
-                                                 cap, stream))
+        phase(to_host)
         e1 = torch.cuda.Event(enable_timing=True); e1.record(stream)
-        for l in range(L):
-            slab = pinned[(l % slots) * n:(l % slots + 1) * n]
-            tk.check(tk.topkv_unpack_layer_from_host(l, w.dst_pool, lo, w.dst_batch, slab, n,
-                                                     staging, cap, stream))
+        phase(from_host)
         e2 = torch.cuda.Event(enable_timing=True); e2.record(stream)
         if rec is not None:
             rec.append((e0, e1, e2))
@@ -555,8 +575,10 @@ def run_extra(name, dev, stream, args, peak):
             staging = torch.empty(w.n_layer, dtype=torch.uint8, device=dev)
             base = pinned_copy_baseline(dev, stream, w.n_layer)
             hs = max(1, min(args.steps, 3))
-            for form, st in (("staged", staging), ("direct", None)):
-                _, th, fh = bench_host_leg(w, stream, pinned, st, hs, 1, nobar, slots)
+            staging2 = torch.empty(w.n_layer, dtype=torch.uint8, device=dev)
+            for form, st, st2 in (("staged", staging, None), ("staged_two_streams", staging, staging2),
+                                  ("direct", None, None)):
+                _, th, fh = bench_host_leg(w, stream, pinned, st, hs, 1, nobar, slots, st2)
                 d2h = w.n_layer * w.layers / (th * 1e-3) / 1e9
                 h2d = w.n_layer * w.layers / (fh * 1e-3) / 1e9
                 out[f"host_leg_{form}"] = {
@@ -565,7 +587,7 @@ def run_extra(name, dev, stream, args, peak):
                     "from_host_frac_of_pinned_copy": round(h2d / base["h2d"], 4)}
             out["pinned_copy_GBps"] = {k: round(v, 2) for k, v in base.items()}
             out["pinned_slots"] = slots
-            del pinned, staging
+            del pinned, staging, staging2
         del w
     elif name == "cfg5":
         w = harness.setup(spec, dev, need_dst=False, need_wire=False)
