@@ -186,7 +186,8 @@ def run_reference(args):
         vals.append(v)
         times.append(dt / n * spec.L)   # a full step = all L layers at the sampled rate
     value = statistics.mean(vals)
-    sample = f"{n} layer(s) of {spec.L} per step (pack+unpack), rows-memcpy oracle, {cores} threads"
+    sample = (f"one of the {spec.L} layers of this workload, pack+unpack, repeated {n} times per step "
+              f"({per_step:.0f} s), rows-memcpy oracle, {cores} threads")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": UNIT,
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
@@ -777,8 +778,8 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, n, cores, dt = oracle_sample(wl.CFG2, wl.make_batch(wl.CFG2), seconds_target=12.0)
         cpu = {"value": round(v, 3), "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": f"{n} layer(s) of {wl.CFG2.L} of this workload, pack+unpack, "
-                         f"rows-memcpy oracle, {dt:.1f} s"}
+               "sample": f"one of the {wl.CFG2.L} layers of this workload, pack+unpack, repeated "
+                         f"{n} times, rows-memcpy oracle, {dt:.1f} s"}
         # for context: the same oracle on one thread, and the byte-by-byte definition on cfg1
         v1, n1, _, dt1 = oracle_sample(wl.CFG2, wl.make_batch(wl.CFG2), seconds_target=4.0, threads=1)
         vr, nr, _, dtr = oracle_sample(wl.CFG1, wl.make_batch(wl.CFG1), seconds_target=3.0, threads=1,
