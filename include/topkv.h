@@ -42,7 +42,9 @@
  * Stream capture: topkv_pack_layer, topkv_unpack_layer, the two host-leg calls,
  * topkv_repage_layer, topkv_build_plan and the checksummed copies only enqueue kernels and
  * copies, so they may be issued while `stream` is being captured into a CUDA graph (the
- * descriptors are read at call time; the buffers they point to at replay time).
+ * descriptors are read at call time; the buffers they point to at replay time). The first
+ * checksummed copy on a device (and the first call of kernel family 1) also raises that
+ * kernel's shared-memory limit, once per device: make that first call outside a capture.
  *
  * Errors: every int-returning function returns TOPKV_OK (0) or a negative
  * topkv_status. When an error is returned nothing has been launched.

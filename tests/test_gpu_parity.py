@@ -466,6 +466,56 @@ def test_cuda_graph_capture_and_replay(dev):
     assert np.array_equal(w.dst_pool.cpu().numpy(), dst_h)
 
 
+def test_cuda_graph_capture_of_the_checksummed_path_and_layer_ranges(dev, variant):
+    """begin, the checksummed pack of every layer, finish, and a multi-layer unpack captured
+    in one CUDA graph: nothing runs during the capture, and after replays the wire, the pool
+    and the checksums are the oracle's (the remainders are stored, so replays do not add up)."""
+    if variant == 1:
+        pytest.skip("the checksumming copy has one kernel family")
+    w = harness.setup(wl.CFG1, dev)
+    b, s = w.batch, wl.CFG1
+    g = _geom(s, b.num_pool_pages, s.L, 0, w.n_layer)
+    src_h, dst_h = w.src_pool.cpu().numpy(), w.dst_pool.cpu().numpy()
+    nws = tk.topkv_crc_workspace_bytes(w.layout, s.R, b.max_pages_per_req)
+    ws = torch.zeros(nws, dtype=torch.uint8, device=dev)
+    crc = torch.zeros(s.R * s.F, dtype=torch.int64, device=dev)
+    stream = torch.cuda.Stream(dev)
+
+    def enqueue():
+        tk.check(tk.topkv_crc_begin(w.layout, w.src_batch, ws, nws, stream))
+        for layer in range(s.L):
+            tk.check(tk.topkv_pack_layer_crc(layer, w.src_pool, w.layout, w.src_batch, w.wire,
+                                             w.wire.numel(), ws, nws, stream))
+        tk.check(tk.topkv_crc_finish(w.layout, w.src_batch, ws, nws, crc, stream))
+        tk.check(tk.topkv_unpack_layers(0, s.L, w.dst_pool, w.layout, w.dst_batch, w.wire,
+                                        w.wire.numel(), stream))
+
+    with torch.cuda.stream(stream):                      # first use on this device: outside capture
+        enqueue()
+    stream.synchronize()
+    w.wire.zero_()
+    crc.zero_()
+    w.dst_pool.copy_(torch.from_numpy(dst_h))
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        enqueue()
+    assert not w.wire.any() and not crc.any()            # capturing executed nothing
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    want_wire = np.zeros(s.L * w.n_layer, dtype=np.uint8)
+    for layer in range(s.L):
+        oracle.pack(g, layer, src_h, b.src_block_table, b.seq_lens, wire=want_wire)
+        oracle.unpack(g, layer, dst_h, b.dst_block_table, b.seq_lens, want_wire)
+    assert np.array_equal(w.wire.cpu().numpy(), want_wire)
+    assert np.array_equal(w.dst_pool.cpu().numpy(), dst_h)
+    got = crc.cpu().numpy().view(np.uint64).reshape(s.R, s.F)
+    for r in range(s.R):
+        for c in range(s.F):
+            assert int(got[r, c]) == oracle.kv_plane_crc(g, src_h, b.src_block_table, b.seq_lens, r, c)
+
+
 def test_two_batches_on_two_streams(dev):
     """Independent batches issued concurrently on two streams do not disturb each other (the
     library keeps no per-call state)."""
