@@ -112,7 +112,7 @@ typedef struct topkv_batch {
   uint32_t struct_size;          /* = sizeof(topkv_batch)                                   */
   int32_t num_requests;          /* R >= 0                                                  */
   int32_t max_pages_per_req;     /* block-table row width (columns)                         */
-  uint32_t flags;                /* 0 or TOPKV_FLAG_OVERLAP_PREVIOUS                        */
+  uint32_t flags;                /* 0 or TOPKV_FLAG_* bits (below)                          */
   const int32_t* block_table;    /* DEVICE int32 [R][max_pages_per_req]; columns at or past */
                                  /* ceil(s_r/P) are ignored (conventionally -1)             */
   const int32_t* seq_lens;       /* DEVICE int32 [R], each in [0, max_pages_per_req*P]      */
@@ -138,6 +138,15 @@ typedef struct topkv_batch {
  * of layer l. Completion stays in stream order: whatever is enqueued after the call starts
  * only after all of them are done. */
 #define TOPKV_FLAG_OVERLAP_PREVIOUS 1u
+/* TOPKV_FLAG_TABLES_SETTLED: the caller declares that block_table, seq_lens and cu_seq_lens
+ * were NOT written by the kernels enqueued just before this call on `stream` (they were
+ * uploaded or built earlier and something has been waited for since: a copy, an event, a
+ * synchronisation). The kernel then reads its tables and works out its addresses while the
+ * previous kernel still drains and waits for that kernel only before it touches the pool or
+ * the wire, so the data it depends on may still come from that kernel (unpack of layer l right
+ * behind pack of layer l). Honoured by topkv_pack_layer(s) / topkv_unpack_layer(s) and the
+ * host-leg calls in the vectorised kernel family; ignored elsewhere. */
+#define TOPKV_FLAG_TABLES_SETTLED 2u
 
 /* Largest R for which cu_seq_lens may be NULL. */
 #define TOPKV_MAX_INLINE_R 1024

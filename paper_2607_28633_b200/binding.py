@@ -28,6 +28,7 @@ TOPKV_KIND_GQA, TOPKV_KIND_MLA = 0, 1
 TOPKV_WIRE_TOKEN_KV, TOPKV_WIRE_PLANAR = 0, 1
 TOPKV_MAX_INLINE_R = 1024
 TOPKV_FLAG_OVERLAP_PREVIOUS = 1
+TOPKV_FLAG_TABLES_SETTLED = 2
 TOPKV_NOALLOC_STAGING_BYTES = 8 * 1024 * 1024
 
 # every symbol include/topkv.h declares

@@ -90,7 +90,7 @@ int check_layout(const topkv_layout* lo, Resolved* out) {
 
 int check_batch(const topkv_layout* lo, const topkv_batch* b) {
   if (b == nullptr || b->struct_size != sizeof(topkv_batch) ||
-      (b->flags & ~(uint32_t)TOPKV_FLAG_OVERLAP_PREVIOUS) != 0)
+      (b->flags & ~(uint32_t)(TOPKV_FLAG_OVERLAP_PREVIOUS | TOPKV_FLAG_TABLES_SETTLED)) != 0)
     return TOPKV_ERR_INVALID_ARG;
   if (b->num_requests < 0 || b->max_pages_per_req < 0 || b->total_tokens < -1 ||
       b->window_tokens < 0 || b->reserved != 0)
@@ -146,6 +146,7 @@ int prepare(int layer, const void* pool, const topkv_layout* lo, const topkv_bat
   kp->unit_chunks = (int)(rs->unit_bytes / 16);
   kp->planar = lo->wire_order == TOPKV_WIRE_PLANAR;
   kp->overlap = (b->flags & TOPKV_FLAG_OVERLAP_PREVIOUS) ? 1 : 0;
+  kp->late_wait = (!kp->overlap && (b->flags & TOPKV_FLAG_TABLES_SETTLED)) ? 1 : 0;
   kp->ppc = 1;
   kp->spr = kp->maxp;
   kp->window = b->window_tokens;

@@ -32,6 +32,7 @@ struct KParams {
   int64_t num_pages;      // pages per pool slab: every page id is checked against it
   int64_t wire_limit;     // bytes that may be touched behind `wire` (this layer's slab)
   int overlap;            // 1: caller declared this launch independent of the kernels before it
+  int late_wait;          // 1: tables are settled, wait for the previous kernel only before touching data
   int64_t S_layer, W_layer;  // multi-layer launch: bytes from one layer's slab to the next (pool, wire)
 };
 

@@ -111,6 +111,8 @@ __device__ __forceinline__ void copy_span(const KParams& p, const int slot) {
       return;
     }
   }
+  // tables read, addresses known: from here on the pool and the wire are touched
+  if (p.late_wait) pdl_wait_prior_grid();
   constexpr int kUnroll = VEC == 32 ? kUnroll32 : kUnroll16;
 
   if (MERGED) {
@@ -207,9 +209,9 @@ __device__ __forceinline__ void copy_span(const KParams& p, const int slot) {
 template <int F, bool PACK, bool MERGED, int VEC, bool MULTI>
 __global__ void __launch_bounds__(kThreads, kMinCtasPerSm)
 topkv_page_copy_kernel(const KParams p) {
-  pdl_prologue(p.overlap);
+  pdl_prologue(p.overlap | p.late_wait);  // late_wait: copy_span waits once the tables are read
   copy_span<F, PACK, MERGED, VEC, MULTI>(p, blockIdx.x);
-  pdl_epilogue(p.overlap);
+  pdl_epilogue(p.overlap | p.late_wait);  // CTAs without work never reached the wait
 }
 
 // The same copy with a bounded grid: gridDim.x CTAs walk all R * spr spans, CTA b taking spans
@@ -220,13 +222,13 @@ topkv_page_copy_kernel(const KParams p) {
 template <int F, bool PACK, bool MERGED, int VEC, bool MULTI>
 __global__ void __launch_bounds__(kThreads, kMinCtasPerSm)
 topkv_page_copy_walk_kernel(const KParams p) {
-  pdl_prologue(p.overlap);
+  pdl_prologue(p.overlap | p.late_wait);
   const int nslots = p.R * p.spr;
   for (int slot = blockIdx.x; slot < nslots; slot += gridDim.x) {
     copy_span<F, PACK, MERGED, VEC, MULTI>(p, slot);
     __syncthreads();  // the span's page ids in shared memory are re-used by the next span
   }
-  pdl_epilogue(p.overlap);
+  pdl_epilogue(p.overlap | p.late_wait);
 }
 
 // Exclusive prefix sum of seq_lens into int64 [R+1]; one CTA, any R.

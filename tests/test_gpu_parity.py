@@ -432,6 +432,45 @@ def test_overlapped_launches_keep_results_and_order(dev):
     torch.cuda.empty_cache()
 
 
+def test_settled_tables_flag_keeps_data_dependences(dev):
+    """TOPKV_FLAG_TABLES_SETTLED: the kernel reads its tables while its predecessor drains but
+    touches data only after it. A chain in which every kernel depends on the DATA of the one
+    just before it (pack of layer l into ONE shared wire slab, then unpack of that slab, for
+    every layer, then a copy right behind) gives the oracle's result; empty batches and a
+    following kernel without the flag keep stream order too."""
+    spec = wl.with_layers(wl.CFG2, 6)
+    w = harness.setup(spec, dev, need_wire=False)
+    b, s = w.batch, spec
+    g = _geom(s, b.num_pool_pages, 1, 0, 0)
+    stream = torch.cuda.Stream(dev)
+    flag = tk.TOPKV_FLAG_TABLES_SETTLED
+    bs = tk.make_batch(w.src_bt, w.seq_lens, b.total_tokens, w.cu, flag)
+    bd = tk.make_batch(w.dst_bt, w.seq_lens, b.total_tokens, w.cu, flag)
+    lo1 = tk.make_layout(s.L, s.F, s.H, s.D, s.E, s.P, b.num_pool_pages)   # wire_layer_stride 0
+    slab = torch.zeros(w.n_layer, dtype=torch.uint8, device=dev)            # one slab for all layers
+    host_dst = torch.empty(w.dst_pool.numel(), dtype=torch.uint8).pin_memory()
+    dst_before = [harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, l) for l in range(s.L)]
+    zeros = torch.zeros(s.R, dtype=torch.int32, device=dev)
+    empty = tk.make_batch(w.src_bt, zeros, 0, None, flag)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        for l in range(s.L):
+            tk.check(tk.topkv_pack_layer(l, w.src_pool, lo1, bs, slab, slab.numel(), stream))
+            tk.check(tk.topkv_pack_layer(l, w.src_pool, lo1, empty, slab, slab.numel(), stream))
+            tk.check(tk.topkv_unpack_layer(l, w.dst_pool, lo1, bd, slab, slab.numel(), stream))
+        host_dst.copy_(w.dst_pool, non_blocking=True)
+    stream.synchronize()
+    for l in range(s.L):
+        src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, l)
+        want = oracle.pack(g, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=8)
+        oracle.unpack(g, 0, dst_before[l], b.dst_block_table, b.seq_lens, want, impl="rows", threads=8)
+        assert np.array_equal(host_dst[l * w.slab_bytes:(l + 1) * w.slab_bytes].numpy(),
+                              dst_before[l]), l
+    assert tk.topkv_device_error_flags() == 0
+    del w
+    torch.cuda.empty_cache()
+
+
 def test_cuda_graph_capture_and_replay(dev):
     """The hot calls only enqueue work, so a whole layer loop can be captured in a CUDA graph
     and replayed (the launch-bound tiny case is where that pays)."""
