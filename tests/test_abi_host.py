@@ -163,7 +163,7 @@ def test_argument_validation_without_gpu():
     assert P(0, pool, huge, _batch(R=1, maxp=4096, T=-1), wire, cap) == tk.TOPKV_ERR_INVALID_ARG
     bb = _batch(); bb.window_tokens = -1
     assert P(0, pool, lo, bb, wire, cap) == tk.TOPKV_ERR_INVALID_ARG
-    bb = _batch(); bb.flags = 2                              # unknown flag bit
+    bb = _batch(); bb.flags = 4                              # unknown flag bit
     assert P(0, pool, lo, bb, wire, cap) == tk.TOPKV_ERR_INVALID_ARG
     bb = _batch(); bb.seq_lens = None
     assert P(0, pool, lo, bb, wire, cap) == tk.TOPKV_ERR_INVALID_ARG
