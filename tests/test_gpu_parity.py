@@ -1191,6 +1191,48 @@ def test_side_stream_overlap_run_is_bit_exact(dev, variant):
     torch.cuda.empty_cache()
 
 
+def test_cfg5_full_size_overlap_run(dev, variant):
+    """The overlap workload at full size as bench.py runs it: 80 layers, 4 x 4096 tokens, the
+    full-size GEMM stand-in on the main stream, every layer shipped to its own pinned slab by
+    the side stream (staged form, issued with topkv_pack_layers_to_host_pipelined). Three
+    layers are compared in full with the oracle's wire slab, and in every layer sampled tokens
+    with what the oracle computes for them one by one."""
+    if variant == 1:
+        pytest.skip("the overlap driver is kernel-family agnostic; run once")
+    from paper_2607_28633_b200 import overlap
+    spec = wl.CFG5
+    w = harness.setup(spec, dev, need_dst=False, need_wire=False)
+    b, s = w.batch, spec
+    g = _geom(s, b.num_pool_pages, 1, 0, 0)
+    try:
+        pinned = torch.zeros(s.L * w.n_layer, dtype=torch.uint8).pin_memory()
+    except RuntimeError:
+        pytest.skip("this box refuses 5 GiB of pinned memory")
+    staging = torch.zeros(w.n_layer, dtype=torch.uint8, device=dev)
+    pre = overlap.PrefillStandIn(dev, 11)
+    r = overlap.run_overlap(w, pinned, staging, pre)
+    assert r.layers == 80 and r.hidden_upper_bound == pytest.approx(1 - 1 / 80)
+    assert 0.0 <= r.exposed_ms and r.hidden <= 1.0
+    for layer in (0, 41, 79):
+        src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, layer)
+        want = oracle.pack(g, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=8)
+        assert np.array_equal(pinned[layer * w.n_layer:(layer + 1) * w.n_layer].numpy(), want), layer
+    rng = np.random.default_rng(8)
+    cu = np.concatenate([[0], np.cumsum(b.seq_lens.astype(np.int64))])
+    host = pinned.numpy()
+    for layer in range(s.L):
+        for _ in range(3):
+            q = int(rng.integers(0, s.R))
+            i = int(rng.integers(0, b.seq_lens[q]))
+            wo = layer * w.n_layer + (int(cu[q]) + i) * s.tok_bytes
+            po = layer * w.slab_bytes + int(b.src_block_table[q, i // s.P]) * s.page_bytes
+            page_h = w.src_pool[po:po + s.page_bytes].cpu().numpy()
+            assert np.array_equal(_oracle_token(s, page_h, i % s.P), host[wo:wo + s.tok_bytes]), \
+                (layer, q, i)
+    del w, pinned, staging, pre
+    torch.cuda.empty_cache()
+
+
 @pytest.mark.parametrize("streams_per_direction", [1, 2])
 def test_relay_through_host_on_two_streams(dev, streams_per_direction):
     """pack_to_host on one set of streams, unpack_from_host on another, gated per layer by an
