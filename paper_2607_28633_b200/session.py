@@ -39,7 +39,10 @@ class Endpoint:
         self.ws_bytes = tk.check(tk.topkv_crc_workspace_bytes(
             self.layout, R, int(self.block_table.shape[1])))
         self.workspace = torch.empty(self.ws_bytes, dtype=torch.uint8, device=dev)
-        self.staging = torch.empty(max(self.n_layer, 16), dtype=torch.uint8, device=dev)
+        # two staging slabs: consecutive layers alternate between two streams, so that the copy
+        # engine moves layer l while the kernel of layer l + 1 runs
+        self.stagings = [torch.empty(max(self.n_layer, 16), dtype=torch.uint8, device=dev)
+                         for _ in range(2)]
         self.crc = torch.zeros(R * self.layout.kv_factor, dtype=torch.int64, device=dev)
         torch.cuda.current_stream(dev).synchronize()
 
@@ -61,10 +64,11 @@ class TransferSender(Endpoint):
     def begin(self, stream):
         tk.check(tk.topkv_crc_begin(self.layout, self.batch, self.workspace, self.ws_bytes, stream))
 
-    def send_layer(self, layer: int, h_wire: torch.Tensor, stream):
+    def send_layer(self, layer: int, h_wire: torch.Tensor, stream, slot: int = 0):
+        st = self.stagings[slot]
         tk.check(tk.topkv_pack_layer_to_host_crc(
-            layer, self.pool, self.layout, self.batch, h_wire, h_wire.numel(), self.staging,
-            self.staging.numel(), self.workspace, self.ws_bytes, stream))
+            layer, self.pool, self.layout, self.batch, h_wire, h_wire.numel(), st, st.numel(),
+            self.workspace, self.ws_bytes, stream))
 
     def finish(self, stream, request_ids, model_id: int, h_seq_lens) -> list[tk.topkv_wire_header]:
         crc = self._checksums(stream)
@@ -84,10 +88,11 @@ class TransferReceiver(Endpoint):
     def begin(self, stream):
         tk.check(tk.topkv_crc_begin(self.layout, self.batch, self.workspace, self.ws_bytes, stream))
 
-    def recv_layer(self, layer: int, h_wire: torch.Tensor, stream):
+    def recv_layer(self, layer: int, h_wire: torch.Tensor, stream, slot: int = 0):
+        st = self.stagings[slot]
         tk.check(tk.topkv_unpack_layer_from_host_crc(
-            layer, self.pool, self.layout, self.batch, h_wire, h_wire.numel(), self.staging,
-            self.staging.numel(), self.workspace, self.ws_bytes, stream))
+            layer, self.pool, self.layout, self.batch, h_wire, h_wire.numel(), st, st.numel(),
+            self.workspace, self.ws_bytes, stream))
 
     def finish(self, stream, headers, h_seq_lens) -> list[int]:
         """Status per request: TOPKV_OK or TOPKV_ERR_CHECKSUM."""
@@ -101,27 +106,40 @@ class TransferReceiver(Endpoint):
 
 def transfer(sender: TransferSender, receiver: TransferReceiver, h_wire: torch.Tensor,
              request_ids, model_id: int, h_seq_lens, layer_ready=None, corrupt=None):
-    """Runs one whole transfer through pinned host memory on two streams, pipelined per layer
-    (the receiver starts on layer l as soon as it has arrived). ``layer_ready[l]`` is an
+    """Runs one whole transfer through pinned host memory, pipelined per layer (the receiver
+    starts on layer l as soon as it has arrived); each side alternates between two streams. ``layer_ready[l]`` is an
     optional event (e.g. recorded by the prefill) that gates the sending of layer l.
     ``corrupt`` (layer, byte offset) flips one bit of that layer's slab in flight: a test hook
     standing in for a faulty link. Returns (headers, per-request status)."""
     dev = sender.pool.device
-    tx, rx = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    tx = [torch.cuda.Stream(dev), torch.cuda.Stream(dev)]
+    rx = [torch.cuda.Stream(dev), torch.cuda.Stream(dev)]
     L = sender.layout.num_layers
-    sender.begin(tx)
-    receiver.begin(rx)
+
+    def after(first, second):
+        """second starts (continues) only after what first holds so far."""
+        ev = torch.cuda.Event()
+        ev.record(first)
+        second.wait_event(ev)
+
+    sender.begin(tx[0])
+    receiver.begin(rx[0])
+    after(tx[0], tx[1])
+    after(rx[0], rx[1])
     for layer in range(L):
+        q = layer & 1
         if layer_ready is not None:
-            tx.wait_event(layer_ready[layer])
-        sender.send_layer(layer, h_wire, tx)
+            tx[q].wait_event(layer_ready[layer])
+        sender.send_layer(layer, h_wire, tx[q], q)
         arrived = torch.cuda.Event()
-        arrived.record(tx)
+        arrived.record(tx[q])
         if corrupt is not None and corrupt[0] == layer:
             arrived.synchronize()
             h_wire[layer * sender.layout.wire_layer_stride + corrupt[1]] ^= 0x04
-        rx.wait_event(arrived)
-        receiver.recv_layer(layer, h_wire, rx)
-    headers = sender.finish(tx, request_ids, model_id, h_seq_lens)
-    status = receiver.finish(rx, headers, h_seq_lens)
+        rx[q].wait_event(arrived)
+        receiver.recv_layer(layer, h_wire, rx[q], q)
+    after(tx[1], tx[0])
+    after(rx[1], rx[0])
+    headers = sender.finish(tx[0], request_ids, model_id, h_seq_lens)
+    status = receiver.finish(rx[0], headers, h_seq_lens)
     return headers, status
