@@ -47,7 +47,11 @@
  * kernel's shared-memory limit, once per device: make that first call outside a capture.
  *
  * Errors: every int-returning function returns TOPKV_OK (0) or a negative
- * topkv_status. When an error is returned nothing has been launched.
+ * topkv_status. Every argument is checked before anything is enqueued, so when an error is
+ * returned nothing has been launched. The one exception is TOPKV_ERR_CUDA reported by the CUDA
+ * runtime itself in the middle of a call that enqueues more than one operation (the staged
+ * host-leg calls: a kernel and a copy; the pipelined calls: one of each per layer): what was
+ * enqueued before the failing operation stays enqueued.
  */
 #ifndef TOPKV_H_
 #define TOPKV_H_
@@ -256,8 +260,11 @@ uint64_t topkv_crc64(const void* h_data, int64_t nbytes);
  * batch->window_tokens = W contributes the last min(s, W) tokens of every request to the
  * checksum, exactly the rows it ships; the workspace remembers each layer's window for
  * topkv_crc_finish, whose own batch argument only supplies the tables (its window_tokens is
- * ignored). TOPKV_FLAG_OVERLAP_PREVIOUS may be set as for the plain calls. The bytes moved are
- * identical to topkv_pack_layer / topkv_unpack_layer. */
+ * ignored). TOPKV_FLAG_OVERLAP_PREVIOUS may be set as for the plain calls, with one rule that
+ * follows from its definition: the first checksummed copy enqueued after topkv_crc_begin reads
+ * and writes what begin wrote, so that copy must NOT carry the flag (begin's own batch argument
+ * may carry any flags; begin ignores them and never lets a later kernel start early). The bytes
+ * moved are identical to topkv_pack_layer / topkv_unpack_layer. */
 int64_t topkv_crc_workspace_bytes(const topkv_layout* layout, int32_t num_requests,
                                   int32_t max_pages_per_req);
 int topkv_crc_begin(const topkv_layout* layout, const topkv_batch* batch, void* d_workspace,
@@ -425,11 +432,20 @@ int topkv_last_cuda_error(void);
  *      those pages were skipped, nothing outside the pool was touched
  *   4  the lengths found on the device did not fit the wire slab (N_layer when total_tokens is
  *      known, else the capacity passed): that work was skipped, nothing outside was touched
- * topkv_device_error_flags() synchronises the device and returns the bits raised on the current
- * device since the library was loaded or the flags were last reset (0 = none), or a negative
- * topkv_status; topkv_reset_device_error_flags() clears them. */
+ * topkv_device_error_flags() waits for ALL work on the current device (cudaDeviceSynchronize:
+ * every stream, non-blocking ones included; not a hot-path call) and returns the bits raised on
+ * it since the library was loaded or the flags were last reset (0 = none), or a negative
+ * topkv_status; topkv_reset_device_error_flags() waits the same way, then clears them. */
 int topkv_device_error_flags(void);
 int topkv_reset_device_error_flags(void);
+/* Width in bytes (16 or 32) of the global loads and stores that topkv_pack_layers /
+ * topkv_unpack_layers would use for these arguments in the vectorised kernel family (same
+ * arguments, same checks, nothing is launched; 0 for an empty range; a negative topkv_status
+ * when the arguments would be refused). 32 requires every base and every stride the kernel adds,
+ * the two layer strides included when num_layers > 1, to be a multiple of 32 bytes. */
+int topkv_copy_vector_bytes(int first_layer, int num_layers, const void* pool,
+                            const topkv_layout* layout, const topkv_batch* batch,
+                            const void* d_wire, int64_t wire_bytes);
 /* Number of kernels this library has launched in this process (all threads). */
 int64_t topkv_kernel_launch_count(void);
 /* Selects the kernel family used by the four hot calls: 0 = vectorised load/store,

@@ -45,6 +45,7 @@ EXPORTS = (
     "topkv_retry", "topkv_pack_layer_to_host_crc", "topkv_unpack_layer_from_host_crc",
     "topkv_set_host_leg_ctas", "topkv_pack_layers_to_host_pipelined",
     "topkv_unpack_layers_from_host_pipelined", "topkv_pack_layers", "topkv_unpack_layers",
+    "topkv_copy_vector_bytes",
 )
 
 
@@ -157,6 +158,7 @@ def lib() -> ctypes.CDLL:
         L.topkv_set_host_leg_ctas.argtypes = [c_int]
         L.topkv_pack_layers.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p]
         L.topkv_unpack_layers.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p]
+        L.topkv_copy_vector_bytes.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64]
         for fn in (L.topkv_pack_layers_to_host_pipelined, L.topkv_unpack_layers_from_host_pipelined):
             fn.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p, c_int64,
                            c_void_p, c_void_p, c_void_p]
@@ -251,6 +253,11 @@ def topkv_unpack_layers(first_layer, num_layers, dst_pool, layout, batch, d_wire
                         stream=None):
     return lib().topkv_unpack_layers(first_layer, num_layers, _ptr(dst_pool), ctypes.byref(layout),
                                      ctypes.byref(batch), _ptr(d_wire), wire_bytes, _stream(stream))
+
+
+def topkv_copy_vector_bytes(first_layer, num_layers, pool, layout, batch, d_wire, wire_bytes):
+    return lib().topkv_copy_vector_bytes(first_layer, num_layers, _ptr(pool), ctypes.byref(layout),
+                                         ctypes.byref(batch), _ptr(d_wire), wire_bytes)
 
 
 def topkv_pack_layer_to_host(layer, src_pool, layout, batch, h_pinned, host_capacity_bytes,

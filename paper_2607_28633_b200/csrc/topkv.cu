@@ -159,31 +159,28 @@ int prepare(int layer, const void* pool, const topkv_layout* lo, const topkv_bat
 }
 
 template <bool PACK, int VEC, bool MULTI>
-void launch_vec2(const KParams& kp, bool merged, int F, dim3 grid, cudaStream_t stream, bool walk) {
+cudaError_t launch_vec2(const KParams& kp, bool merged, int F, dim3 grid, cudaStream_t stream, bool walk) {
   const dim3 block(kThreads);
   if (walk) {  // bounded grid, every CTA walks several spans
     if (merged) {
-      if (F == 1) launch_pdl(topkv_page_copy_walk_kernel<1, PACK, true, VEC, MULTI>, grid, block, 0, stream, kp);
-      else launch_pdl(topkv_page_copy_walk_kernel<2, PACK, true, VEC, MULTI>, grid, block, 0, stream, kp);
-    } else {
-      if (F == 1) launch_pdl(topkv_page_copy_walk_kernel<1, PACK, false, VEC, MULTI>, grid, block, 0, stream, kp);
-      else launch_pdl(topkv_page_copy_walk_kernel<2, PACK, false, VEC, MULTI>, grid, block, 0, stream, kp);
+      if (F == 1) return launch_pdl(topkv_page_copy_walk_kernel<1, PACK, true, VEC, MULTI>, grid, block, 0, stream, kp);
+      return launch_pdl(topkv_page_copy_walk_kernel<2, PACK, true, VEC, MULTI>, grid, block, 0, stream, kp);
     }
-    return;
+    if (F == 1) return launch_pdl(topkv_page_copy_walk_kernel<1, PACK, false, VEC, MULTI>, grid, block, 0, stream, kp);
+    return launch_pdl(topkv_page_copy_walk_kernel<2, PACK, false, VEC, MULTI>, grid, block, 0, stream, kp);
   }
   if (merged) {
-    if (F == 1) launch_pdl(topkv_page_copy_kernel<1, PACK, true, VEC, MULTI>, grid, block, 0, stream, kp);
-    else launch_pdl(topkv_page_copy_kernel<2, PACK, true, VEC, MULTI>, grid, block, 0, stream, kp);
-  } else {
-    if (F == 1) launch_pdl(topkv_page_copy_kernel<1, PACK, false, VEC, MULTI>, grid, block, 0, stream, kp);
-    else launch_pdl(topkv_page_copy_kernel<2, PACK, false, VEC, MULTI>, grid, block, 0, stream, kp);
+    if (F == 1) return launch_pdl(topkv_page_copy_kernel<1, PACK, true, VEC, MULTI>, grid, block, 0, stream, kp);
+    return launch_pdl(topkv_page_copy_kernel<2, PACK, true, VEC, MULTI>, grid, block, 0, stream, kp);
   }
+  if (F == 1) return launch_pdl(topkv_page_copy_kernel<1, PACK, false, VEC, MULTI>, grid, block, 0, stream, kp);
+  return launch_pdl(topkv_page_copy_kernel<2, PACK, false, VEC, MULTI>, grid, block, 0, stream, kp);
 }
 
 template <bool PACK, int VEC>
-void launch_vec(const KParams& kp, bool merged, int F, dim3 grid, cudaStream_t stream, bool walk) {
-  if (kp.ppc > 1) launch_vec2<PACK, VEC, true>(kp, merged, F, grid, stream, walk);
-  else launch_vec2<PACK, VEC, false>(kp, merged, F, grid, stream, walk);
+cudaError_t launch_vec(const KParams& kp, bool merged, int F, dim3 grid, cudaStream_t stream, bool walk) {
+  if (kp.ppc > 1) return launch_vec2<PACK, VEC, true>(kp, merged, F, grid, stream, walk);
+  return launch_vec2<PACK, VEC, false>(kp, merged, F, grid, stream, walk);
 }
 
 // ---- bulk-async family -------------------------------------------------------------------
@@ -247,10 +244,22 @@ int launch_bulk(const KParams& kp0, const Resolved& rs, int F, cudaStream_t stre
   int st = (F == 1) ? bulk_prepare_device<1, PACK>(&sms) : bulk_prepare_device<2, PACK>(&sms);
   if (st != TOPKV_OK) return st;
   const dim3 grid((unsigned)sms), block(kBulkThreads);
-  if (F == 1) launch_pdl(topkv_bulk_kernel<1, PACK>, grid, block, smem, stream, bp);
-  else launch_pdl(topkv_bulk_kernel<2, PACK>, grid, block, smem, stream, bp);
+  const cudaError_t e = (F == 1) ? launch_pdl(topkv_bulk_kernel<1, PACK>, grid, block, smem, stream, bp)
+                                 : launch_pdl(topkv_bulk_kernel<2, PACK>, grid, block, smem, stream, bp);
+  if (e != cudaSuccess) return cuda_fail(e);
   *handled = true;
   return TOPKV_OK;
+}
+
+// Bytes per access of the vectorised family: 32 only when every address the kernel can form
+// is 32-byte aligned. A launch over several layers also adds multiples of the two layer
+// strides inside the kernel (blockIdx.y), which the ABI only requires to be multiples of 16.
+int copy_vector_bytes(const KParams& kp, int64_t unit_bytes, int layers) {
+  uintptr_t m = reinterpret_cast<uintptr_t>(kp.pool) | reinterpret_cast<uintptr_t>(kp.wire) |
+                (uintptr_t)kp.S_page | (uintptr_t)kp.S_kv | (uintptr_t)kp.S_tok | (uintptr_t)kp.S_unit |
+                (uintptr_t)unit_bytes;
+  if (layers > 1) m |= (uintptr_t)kp.S_layer | (uintptr_t)kp.W_layer;
+  return (m & 31) == 0 ? 32 : 16;
 }
 
 // max_ctas > 0: the wire is host memory behind PCIe; at most that many CTAs walk the spans.
@@ -274,16 +283,17 @@ int launch_copy(KParams kp, const Resolved& rs, int F, cudaStream_t stream, int 
     const int64_t spans = (int64_t)kp.R * kp.spr;
     const bool walk = max_ctas > 0 && spans > max_ctas;
     const dim3 grid((unsigned)(walk ? max_ctas : spans), (unsigned)layers);
-    // 32-byte vectors when every address the kernel can form is 32-byte aligned
-    const bool wide = ((reinterpret_cast<uintptr_t>(kp.pool) | reinterpret_cast<uintptr_t>(kp.wire) |
-                        (uintptr_t)kp.S_page | (uintptr_t)kp.S_kv | (uintptr_t)kp.S_tok |
-                        (uintptr_t)kp.S_unit | (uintptr_t)rs.unit_bytes) & 31) == 0;
-    if (wide) {
+    cudaError_t le;
+    if (copy_vector_bytes(kp, rs.unit_bytes, layers) == 32) {
       kp.unit_chunks = (int)(rs.unit_bytes / 32);
-      launch_vec<PACK, 32>(kp, rs.merged, F, grid, stream, walk);
+      le = launch_vec<PACK, 32>(kp, rs.merged, F, grid, stream, walk);
     } else {
       kp.unit_chunks = (int)(rs.unit_bytes / 16);
-      launch_vec<PACK, 16>(kp, rs.merged, F, grid, stream, walk);
+      le = launch_vec<PACK, 16>(kp, rs.merged, F, grid, stream, walk);
+    }
+    if (le != cudaSuccess) {
+      cudaGetLastError();
+      return cuda_fail(le);
     }
   }
   const cudaError_t e = cudaGetLastError();
@@ -410,19 +420,37 @@ int crc_prepare_device(int* sms_out) {
   return TOPKV_OK;
 }
 
-template <bool PACK>
-int crc_copy(int layer, const void* pool, const topkv_layout* lo, const topkv_batch* b,
-             const void* wire, int64_t cap, void* ws, int64_t ws_bytes, cudaStream_t stream,
-             void* slab_override = nullptr, int64_t* n_layer_out = nullptr, int max_ctas = 0) {
-  // slab_override: device address to use for this layer's wire slab instead of
-  // wire + layer*stride (a staging slab, or the device view of a pinned host slab);
-  // max_ctas > 0: the wire is host memory behind PCIe, at most that many CTAs run
+// A checksummed copy, validated and ready to launch: everything that can be refused is refused
+// by crc_plan, so that a caller with work of its own to enqueue (the host leg's copies) only
+// starts once the whole call is known to be acceptable.
+struct CrcLaunch {
   CrcCopyParams cp;
+  dim3 grid, block;
+  size_t smem = 0;
+  int F = 0;
+  int64_t n_layer = -1;  // bytes of the layer's slab when total_tokens is known
+  bool empty = true;     // nothing to launch (no requests, or no table columns)
+};
+
+// slab_override: device address to use for this layer's wire slab instead of wire + layer*stride
+// (a staging slab, or the device view of a pinned host slab); max_ctas > 0: the wire is host
+// memory behind PCIe, at most that many CTAs run.
+// staging_capacity >= 0: slab_override is the staging slab of the staged host leg, which needs the
+// slab's size on the host, adjacent planes (one contiguous copy) and room for the slab.
+template <bool PACK>
+int crc_plan(int layer, const void* pool, const topkv_layout* lo, const topkv_batch* b, const void* wire,
+             int64_t cap, void* ws, int64_t ws_bytes, void* slab_override, int max_ctas, CrcLaunch* out,
+             int64_t staging_capacity = -1) {
+  CrcCopyParams& cp = out->cp;
   Resolved rs;
-  int64_t n_layer;
-  int st = prepare(layer, pool, lo, b, wire, cap, lo ? lo->wire_layer_stride : 0, &cp.k, &rs, &n_layer);
+  int st = prepare(layer, pool, lo, b, wire, cap, lo ? lo->wire_layer_stride : 0, &cp.k, &rs, &out->n_layer);
   if (st != TOPKV_OK) return st;
-  if (n_layer_out != nullptr) *n_layer_out = n_layer;
+  if (staging_capacity >= 0) {
+    if (out->n_layer < 0) return TOPKV_ERR_INVALID_ARG;
+    if (lo->wire_plane_stride != 0) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+    if (!mult16p(slab_override)) return TOPKV_ERR_ALIGNMENT;
+    if (staging_capacity < out->n_layer) return TOPKV_ERR_CAPACITY;
+  }
   if (slab_override != nullptr) cp.k.wire = static_cast<uint8_t*>(slab_override);
   if (ws == nullptr || !mult16p(ws)) return TOPKV_ERR_INVALID_ARG;
   const int F = (int)lo->kv_factor, R = b->num_requests, maxp = b->max_pages_per_req;
@@ -431,14 +459,15 @@ int crc_copy(int layer, const void* pool, const topkv_layout* lo, const topkv_ba
   st = crc_geometry(lo, rs, maxp, &cp.g);
   if (st != TOPKV_OK) return st;
   if (ws_bytes < 8 * crc_workspace_words(cp.g.kmax, L, R, F)) return TOPKV_ERR_CAPACITY;
-  if (R == 0 || maxp == 0) return TOPKV_OK;
+  out->F = F;
+  out->empty = R == 0 || maxp == 0;
+  if (out->empty) return TOPKV_OK;
   if ((int64_t)R * cp.g.kmax * F > 0x7fffffffll) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
   cp.w = crc_carve(ws, cp.g.kmax, L, R, F);
   cp.layer = layer;
   cp.stages = TOPKV_CRC_STAGES;
   int warps = 0, sms = 0;
-  size_t smem = 0;
-  st = crc_launch_shape(cp.g, R, cp.stages, &warps, &smem);
+  st = crc_launch_shape(cp.g, R, cp.stages, &warps, &out->smem);
   if (st != TOPKV_OK) return st;
   st = (F == 1) ? crc_prepare_device<1, PACK>(&sms) : crc_prepare_device<2, PACK>(&sms);
   if (st != TOPKV_OK) return st;
@@ -446,10 +475,17 @@ int crc_copy(int layer, const void* pool, const topkv_layout* lo, const topkv_ba
   const int64_t items = (int64_t)R * cp.g.kmax * F;  // upper bound
   int64_t ctas = std::min<int64_t>((int64_t)sms * kCrcCtasPerSm, (items + warps - 1) / warps);
   if (max_ctas > 0) ctas = std::min<int64_t>(ctas, max_ctas);
-  const dim3 grid((unsigned)std::max<int64_t>(1, ctas)), block((unsigned)(warps * 32));
+  out->grid = dim3((unsigned)std::max<int64_t>(1, ctas));
+  out->block = dim3((unsigned)(warps * 32));
+  return TOPKV_OK;
+}
+
+template <bool PACK>
+int crc_launch(const CrcLaunch& cl, cudaStream_t stream) {
+  if (cl.empty) return TOPKV_OK;
   cudaError_t e;
-  if (F == 1) e = launch_pdl(topkv_crc_copy_kernel<1, PACK>, grid, block, smem, stream, cp);
-  else e = launch_pdl(topkv_crc_copy_kernel<2, PACK>, grid, block, smem, stream, cp);
+  if (cl.F == 1) e = launch_pdl(topkv_crc_copy_kernel<1, PACK>, cl.grid, cl.block, cl.smem, stream, cl.cp);
+  else e = launch_pdl(topkv_crc_copy_kernel<2, PACK>, cl.grid, cl.block, cl.smem, stream, cl.cp);
   if (e != cudaSuccess) return cuda_fail(e);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
@@ -457,36 +493,46 @@ int crc_copy(int layer, const void* pool, const topkv_layout* lo, const topkv_ba
   return TOPKV_OK;
 }
 
-// Host leg with checksums: the same two forms as the plain host-leg calls.
+template <bool PACK>
+int crc_copy(int layer, const void* pool, const topkv_layout* lo, const topkv_batch* b,
+             const void* wire, int64_t cap, void* ws, int64_t ws_bytes, cudaStream_t stream) {
+  CrcLaunch cl;
+  const int st = crc_plan<PACK>(layer, pool, lo, b, wire, cap, ws, ws_bytes, nullptr, 0, &cl);
+  return st != TOPKV_OK ? st : crc_launch<PACK>(cl, stream);
+}
+
+// Host leg with checksums: the same two forms as the plain host-leg calls. Every argument is
+// checked before the first copy or kernel is enqueued.
 template <bool PACK>
 int crc_host_leg(int layer, const void* pool, const topkv_layout* layout,
                         const topkv_batch* batch, const void* h_pinned, int64_t host_bytes,
                         void* d_staging, int64_t staging_capacity_bytes, void* ws, int64_t ws_bytes,
                         cudaStream_t s) {
   if (layout == nullptr || batch == nullptr || h_pinned == nullptr) return TOPKV_ERR_INVALID_ARG;
+  CrcLaunch cl;
   if (d_staging == nullptr) {  // direct: the kernel works on the mapped pinned slab
-    void* dev = nullptr;
-    int st = mapped_device_pointer(h_pinned, &dev);
+    // validate with the host address first (layer range, capacity, workspace), then map it
+    int st = crc_plan<PACK>(layer, pool, layout, batch, h_pinned, host_bytes, ws, ws_bytes, nullptr,
+                            g_host_leg_ctas.load(std::memory_order_relaxed), &cl);
     if (st != TOPKV_OK) return st;
-    void* slab = static_cast<uint8_t*>(dev) + (int64_t)layer * layout->wire_layer_stride;
-    return crc_copy<PACK>(layer, pool, layout, batch, h_pinned, host_bytes, ws, ws_bytes, s, slab, nullptr,
-                          g_host_leg_ctas.load(std::memory_order_relaxed));
+    void* dev = nullptr;
+    st = mapped_device_pointer(h_pinned, &dev);
+    if (st != TOPKV_OK) return st;
+    cl.cp.k.wire = static_cast<uint8_t*>(dev) + (int64_t)layer * layout->wire_layer_stride;
+    return crc_launch<PACK>(cl, s);
   }
-  if (batch->struct_size == sizeof(topkv_batch) && batch->total_tokens < 0) return TOPKV_ERR_INVALID_ARG;
-  if (layout->struct_size == sizeof(topkv_layout) && layout->wire_plane_stride != 0)
-    return TOPKV_ERR_UNSUPPORTED_LAYOUT;  // one contiguous copy
-  if (!mult16p(d_staging)) return TOPKV_ERR_ALIGNMENT;
+  if (staging_capacity_bytes < 0) return TOPKV_ERR_INVALID_ARG;
+  int st = crc_plan<PACK>(layer, pool, layout, batch, h_pinned, host_bytes, ws, ws_bytes, d_staging, 0, &cl,
+                          staging_capacity_bytes);
+  if (st != TOPKV_OK) return st;
+  const int64_t n_layer = cl.n_layer;  // known: total_tokens >= 0
+  // the layer index and the host capacity have been checked: the slab lies inside h_pinned
   const uint8_t* host_slab = static_cast<const uint8_t*>(h_pinned) + (int64_t)layer * layout->wire_layer_stride;
-  const int64_t n_known = topkv_wire_layer_bytes(layout, batch->total_tokens);
-  if (n_known < 0) return TOPKV_ERR_INVALID_ARG;
-  if (staging_capacity_bytes < n_known) return TOPKV_ERR_CAPACITY;
-  if (!PACK && n_known > 0) {  // bring the slab in first
-    const cudaError_t e = cudaMemcpyAsync(d_staging, host_slab, (size_t)n_known, cudaMemcpyHostToDevice, s);
+  if (!PACK && n_layer > 0) {  // bring the slab in first
+    const cudaError_t e = cudaMemcpyAsync(d_staging, host_slab, (size_t)n_layer, cudaMemcpyHostToDevice, s);
     if (e != cudaSuccess) return cuda_fail(e);
   }
-  int64_t n_layer = -1;
-  const int st = crc_copy<PACK>(layer, pool, layout, batch, h_pinned, host_bytes, ws, ws_bytes, s,
-                                d_staging, &n_layer);
+  st = crc_launch<PACK>(cl, s);
   if (st != TOPKV_OK) return st;
   if (PACK && n_layer > 0) {
     const cudaError_t e = cudaMemcpyAsync(const_cast<uint8_t*>(host_slab), d_staging, (size_t)n_layer,
@@ -553,32 +599,46 @@ int issue_layers(int first_layer, int num_layers, const void* pool, const topkv_
 
 namespace multi {
 
+// Validates a range of layers and fills the parameters of ONE launch that covers it.
+// *launch is false when there is nothing to launch (an empty range).
+int plan_layers(int first_layer, int num_layers, const void* pool, const topkv_layout* layout,
+                const topkv_batch* batch, const void* d_wire, int64_t wire_bytes, KParams* kp,
+                Resolved* rs, bool* launch) {
+  *launch = false;
+  if (num_layers < 0 || first_layer < 0) return TOPKV_ERR_LAYER_RANGE;
+  if (num_layers > 65535) return TOPKV_ERR_INVALID_ARG;  // grid.y
+  KParams kp_last;
+  int64_t n_layer;
+  if (num_layers == 0) {  // still validate the descriptors
+    if (layout == nullptr) return TOPKV_ERR_INVALID_ARG;
+    const int st = check_layout(layout, rs);
+    return st != TOPKV_OK ? st : check_batch(layout, batch);
+  }
+  int st = prepare(first_layer, pool, layout, batch, d_wire, wire_bytes,
+                   layout ? layout->wire_layer_stride : 0, kp, rs, &n_layer);
+  if (st != TOPKV_OK) return st;
+  st = prepare(first_layer + num_layers - 1, pool, layout, batch, d_wire, wire_bytes,
+               layout->wire_layer_stride, &kp_last, rs, &n_layer);  // range and capacity of the last
+  if (st != TOPKV_OK) return st;
+  if (num_layers > 1) {
+    if (layout->wire_layer_stride <= 0) return TOPKV_ERR_INVALID_ARG;  // all layers on one slab
+    kp->S_layer = layout->pool_layer_stride;
+    kp->W_layer = layout->wire_layer_stride;
+    kp->wire_limit = std::min(kp->wire_limit, kp_last.wire_limit);  // the tightest slab bounds them all
+  }
+  *launch = true;
+  return TOPKV_OK;
+}
+
 // One launch for the layers [first_layer, first_layer + num_layers).
 template <bool PACK>
 int copy_layers(int first_layer, int num_layers, const void* pool, const topkv_layout* layout,
                 const topkv_batch* batch, const void* d_wire, int64_t wire_bytes, cudaStream_t s) {
-  if (num_layers < 0 || first_layer < 0) return TOPKV_ERR_LAYER_RANGE;
-  if (num_layers > 65535) return TOPKV_ERR_INVALID_ARG;  // grid.y
-  KParams kp, kp_last;
+  KParams kp;
   Resolved rs;
-  int64_t n_layer;
-  if (num_layers == 0) {  // still validate the descriptors
-    if (layout == nullptr) return TOPKV_ERR_INVALID_ARG;
-    const int st = check_layout(layout, &rs);
-    return st != TOPKV_OK ? st : check_batch(layout, batch);
-  }
-  int st = prepare(first_layer, pool, layout, batch, d_wire, wire_bytes,
-                   layout ? layout->wire_layer_stride : 0, &kp, &rs, &n_layer);
-  if (st != TOPKV_OK) return st;
-  st = prepare(first_layer + num_layers - 1, pool, layout, batch, d_wire, wire_bytes,
-               layout->wire_layer_stride, &kp_last, &rs, &n_layer);  // range and capacity of the last
-  if (st != TOPKV_OK) return st;
-  if (num_layers > 1) {
-    if (layout->wire_layer_stride <= 0) return TOPKV_ERR_INVALID_ARG;  // all layers on one slab
-    kp.S_layer = layout->pool_layer_stride;
-    kp.W_layer = layout->wire_layer_stride;
-    kp.wire_limit = std::min(kp.wire_limit, kp_last.wire_limit);  // the tightest slab bounds them all
-  }
+  bool launch = false;
+  const int st = plan_layers(first_layer, num_layers, pool, layout, batch, d_wire, wire_bytes, &kp, &rs, &launch);
+  if (st != TOPKV_OK || !launch) return st;
   return launch_copy<PACK>(kp, rs, (int)layout->kv_factor, s, 0, num_layers);
 }
 
@@ -815,14 +875,19 @@ int topkv_repage_layer(int layer, const void* src_pool, const topkv_layout* src_
                       (uintptr_t)p.Sd_tok | (uintptr_t)p.Sd_unit | (uintptr_t)unit_bytes) & 31) == 0;
   const dim3 grid((unsigned)((int64_t)p.R * p.spr)), block(kRepageThreads);
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  cudaError_t le;
   if (wide) {
     p.unit_chunks = (int)(unit_bytes / 32);
-    if (F == 1) launch_pdl(topkv_repage_kernel<1, 32>, grid, block, 0, s, p);
-    else launch_pdl(topkv_repage_kernel<2, 32>, grid, block, 0, s, p);
+    le = (F == 1) ? launch_pdl(topkv_repage_kernel<1, 32>, grid, block, 0, s, p)
+                  : launch_pdl(topkv_repage_kernel<2, 32>, grid, block, 0, s, p);
   } else {
     p.unit_chunks = (int)(unit_bytes / 16);
-    if (F == 1) launch_pdl(topkv_repage_kernel<1, 16>, grid, block, 0, s, p);
-    else launch_pdl(topkv_repage_kernel<2, 16>, grid, block, 0, s, p);
+    le = (F == 1) ? launch_pdl(topkv_repage_kernel<1, 16>, grid, block, 0, s, p)
+                  : launch_pdl(topkv_repage_kernel<2, 16>, grid, block, 0, s, p);
+  }
+  if (le != cudaSuccess) {
+    cudaGetLastError();
+    return cuda_fail(le);
   }
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
@@ -951,18 +1016,35 @@ int topkv_last_cuda_error(void) { return g_last_cuda_error; }
 
 int topkv_reset_device_error_flags(void) {
   const int zero = 0;
-  const cudaError_t e = cudaMemcpyToSymbol(g_device_error_flags, &zero, sizeof(int));
+  cudaError_t e = cudaDeviceSynchronize();  // no kernel may still raise a bit behind the reset
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = cudaMemcpyToSymbol(g_device_error_flags, &zero, sizeof(int));
   if (e != cudaSuccess) return cuda_fail(e);
   return TOPKV_OK;
 }
 
 int topkv_device_error_flags(void) {
   int flags = 0;
-  const cudaError_t e = cudaMemcpyFromSymbol(&flags, g_device_error_flags, sizeof(int));
+  // every stream of the device, the non-blocking ones included, has to be done: the copy below
+  // runs on the legacy default stream, which orders against blocking streams only
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = cudaMemcpyFromSymbol(&flags, g_device_error_flags, sizeof(int));
   if (e != cudaSuccess) return cuda_fail(e);
   return flags;
 }
 int64_t topkv_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int topkv_copy_vector_bytes(int first_layer, int num_layers, const void* pool, const topkv_layout* layout,
+                            const topkv_batch* batch, const void* d_wire, int64_t wire_bytes) {
+  KParams kp;
+  Resolved rs;
+  bool launch = false;
+  const int st = multi::plan_layers(first_layer, num_layers, pool, layout, batch, d_wire, wire_bytes, &kp, &rs,
+                                    &launch);
+  if (st != TOPKV_OK) return st;
+  return launch ? copy_vector_bytes(kp, rs.unit_bytes, num_layers) : 0;
+}
 
 int topkv_set_host_leg_ctas(int ctas) {
   if (ctas < 0 || ctas > 65535) return TOPKV_ERR_INVALID_ARG;

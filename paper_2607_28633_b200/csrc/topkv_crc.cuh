@@ -5,7 +5,7 @@
 // Everything is linear over GF(2). With rem(M) = M(x) * x^64 mod P (no initial value, no
 // inversion) and "||" concatenation:   rem(A || B) = rem(A) * x^(8|B|) + rem(B)   (mod P).
 // The tensor of one request and one plane, [layers][seq_len][kv_heads][head_dim], is cut,
-// layer by layer, into runs (a fraction of a token row, at most 512 bytes) and the runs into
+// layer by layer, into runs (a fraction of a token row, at most 1 KiB) and the runs into
 // items of 32 consecutive runs counted from the END of the request's plane, so that every item
 // but the first of a request is full and k full items follow item k. One warp takes one item,
 // one lane one run:
@@ -217,7 +217,10 @@ __host__ __device__ inline CrcWorkspace crc_carve(void* base, int kmax, int L, i
 __global__ void __launch_bounds__(256)
 topkv_crc_begin_kernel(CrcWorkspace w, CrcGeom g, const int32_t* __restrict__ sl, int L, int R,
                        int maxp, int P, int64_t row_bytes, int F) {
-  pdl_prologue(0);
+  // No early release of the next kernel: a checksummed copy launched behind this kernel reads
+  // the tables built here and writes the words cleared here, so it may only become resident
+  // once every CTA of this kernel has finished.
+  pdl_wait_prior_grid();
   const int64_t n_tail = (int64_t)g.kmax + 1;
   const int64_t n_items = (int64_t)L * R * g.kmax * F;
   const int64_t total = 32 + n_tail + R + n_items;

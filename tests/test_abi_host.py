@@ -293,3 +293,73 @@ def test_validate_batch_host():
     short = sl.copy(); short[0] = 16                               # ignores the unused column
     ok = bt.copy(); ok[0, 1] = -1
     assert V(lo, 3, 2, ok, short, 1) == tk.TOPKV_OK
+
+
+def test_vector_width_of_layer_range_launches():
+    """A launch over several layers adds multiples of the two layer strides inside the kernel,
+    and the ABI only asks those to be multiples of 16: 32-byte accesses are chosen only when the
+    strides allow them, whatever the alignment of the first layer's slabs."""
+    n = 1_785_856                                           # cfg1's slab, a multiple of 32
+    b = _batch()
+    pool, wire = 0x7000000, 0x9000000                       # 32-byte aligned bases
+    V = tk.topkv_copy_vector_bytes
+    lo = _gqa(wire_layer_stride=n)
+    assert V(0, 1, pool, lo, b, wire, 8 * n) == 32
+    assert V(0, 4, pool, lo, b, wire, 8 * n) == 32
+    assert V(0, 1, pool + 16, lo, b, wire, 8 * n) == 16     # a 16-byte-only base
+    assert V(0, 1, pool, lo, b, wire + 16, 8 * n) == 16
+    pad = _gqa(wire_layer_stride=n + 16)                    # padded wire slabs: 16 mod 32
+    assert V(0, 1, pool, pad, b, wire, 8 * n) == 32         # layer 0 alone never adds the stride
+    assert V(0, 2, pool, pad, b, wire, 8 * n) == 16         # layer 1's slab is only 16-aligned
+    assert V(2, 1, pool, pad, b, wire, 8 * n) == 32         # 2 * (n + 16) is a multiple of 32
+    assert V(1, 1, pool, pad, b, wire, 8 * n) == 16         # the base of layer 1 shows it already
+    assert V(2, 2, pool, pad, b, wire, 8 * n) == 16         # aligned first layer, odd stride
+    odd = _gqa(wire_layer_stride=n)
+    odd.pool_layer_stride += 16                             # e.g. a plane-major pool with padding
+    assert V(0, 1, pool, odd, b, wire, 8 * n) == 32
+    assert V(0, 3, pool, odd, b, wire, 8 * n) == 16
+    assert V(2, 2, pool, odd, b, wire, 8 * n) == 16
+    small = tk.make_layout(4, 2, 1, 8, 2, 16, 64, wire_layer_stride=n)   # 16-byte rows
+    assert V(0, 2, pool, small, b, wire, 8 * n) == 16
+    # the same checks as the launching calls, and nothing is launched
+    before = tk.topkv_kernel_launch_count()
+    assert V(0, 0, pool, lo, b, wire, 8 * n) == 0
+    assert V(3, 2, pool, lo, b, wire, 8 * n) == tk.TOPKV_ERR_LAYER_RANGE
+    assert V(0, 4, pool, lo, b, wire, 4 * n - 1) == tk.TOPKV_ERR_CAPACITY
+    assert V(0, 2, pool, _gqa(wire_layer_stride=0), b, wire, 8 * n) == tk.TOPKV_ERR_INVALID_ARG
+    assert tk.topkv_kernel_launch_count() == before
+
+
+def test_checksummed_host_leg_validates_before_it_enqueues():
+    """Every argument of the checksummed host-leg calls is checked before the first copy or
+    kernel is enqueued: a bad layer, a short host buffer, a short or missing workspace, a
+    misaligned or short staging slab return their status with nothing launched (the addresses
+    here are fakes: had anything been enqueued with them, the call could not have returned a
+    validation status)."""
+    n = 1_785_856
+    lo, b = _gqa(wire_layer_stride=n), _batch()
+    pool, host, staging, ws = 0x7000000, 0x9000000, 0xA000000, 0xB000000
+    nws = tk.topkv_crc_workspace_bytes(lo, 4, 16)
+    assert nws > 0
+    before = tk.topkv_kernel_launch_count()
+    for fn in (tk.topkv_pack_layer_to_host_crc, tk.topkv_unpack_layer_from_host_crc):
+        for st_ptr, st_cap in ((staging, n), (None, 0)):            # staged and direct forms
+            assert fn(4, pool, lo, b, host, 4 * n, st_ptr, st_cap, ws, nws) == tk.TOPKV_ERR_LAYER_RANGE
+            assert fn(-1, pool, lo, b, host, 4 * n, st_ptr, st_cap, ws, nws) == tk.TOPKV_ERR_LAYER_RANGE
+            assert fn(3, pool, lo, b, host, 4 * n - 1, st_ptr, st_cap, ws, nws) == tk.TOPKV_ERR_CAPACITY
+            assert fn(0, pool, lo, b, host, 4 * n, st_ptr, st_cap, ws, nws - 8) == tk.TOPKV_ERR_CAPACITY
+            assert fn(0, pool, lo, b, host, 4 * n, st_ptr, st_cap, None, nws) == tk.TOPKV_ERR_INVALID_ARG
+            assert fn(0, pool, lo, b, host, 4 * n, st_ptr, st_cap, ws + 8, nws) == tk.TOPKV_ERR_INVALID_ARG
+            assert fn(0, pool + 8, lo, b, host, 4 * n, st_ptr, st_cap, ws, nws) == tk.TOPKV_ERR_ALIGNMENT
+            assert fn(0, pool, lo, b, None, 4 * n, st_ptr, st_cap, ws, nws) == tk.TOPKV_ERR_INVALID_ARG
+        assert fn(0, pool, lo, b, host, 4 * n, staging + 8, n, ws, nws) == tk.TOPKV_ERR_ALIGNMENT
+        assert fn(0, pool, lo, b, host, 4 * n, staging, n - 1, ws, nws) == tk.TOPKV_ERR_CAPACITY
+        assert fn(0, pool, lo, _batch(T=-1), host, 4 * n, staging, n, ws, nws) == tk.TOPKV_ERR_INVALID_ARG
+        planar = _gqa(wire_order=tk.TOPKV_WIRE_PLANAR, wire_layer_stride=n)
+        planar.wire_plane_stride = 2048 * 1000
+        assert fn(0, pool, planar, b, host, 1 << 40, staging, 1 << 40, ws, nws) \
+            == tk.TOPKV_ERR_UNSUPPORTED_LAYOUT
+    # the plain staged calls keep the same order
+    assert tk.topkv_unpack_layer_from_host(4, pool, lo, b, host, 4 * n, staging, n) == tk.TOPKV_ERR_LAYER_RANGE
+    assert tk.topkv_unpack_layer_from_host(3, pool, lo, b, host, 4 * n - 1, staging, n) == tk.TOPKV_ERR_CAPACITY
+    assert tk.topkv_kernel_launch_count() == before
