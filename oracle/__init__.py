@@ -80,6 +80,17 @@ def _load():
         lib.oracle_kv_plane_crc.argtypes = [gp, vp, i64, i64, vp, vp, i64, i64]
         lib.oracle_kv_plane_crc_layered.restype = u64
         lib.oracle_kv_plane_crc_layered.argtypes = [gp, vp, i64, i64, vp, vp, i64, i64, vp]
+        for name in ("oracle_pack_layered", "oracle_unpack_layered"):
+            fn = getattr(lib, name)
+            fn.restype = None
+            fn.argtypes = [gp, i64, vp, vp, vp, i64, i64, vp, vp, vp, i64, i64, vp, vp]
+        lib.oracle_layered_offsets.restype = None
+        lib.oracle_layered_offsets.argtypes = [gp, i64, vp, vp, i64, vp, vp]
+        cp, ci = ctypes.c_char_p, ctypes.c_int
+        lib.oracle_select_transport.restype = ci
+        lib.oracle_select_transport.argtypes = [ci, cp, ci, cp, cp, ci, cp, ci]
+        lib.oracle_planning_rate.restype = f64
+        lib.oracle_planning_rate.argtypes = [ci]
         _lib = lib
     return _lib
 
@@ -238,6 +249,102 @@ def unpack(g: Geom, layer: int, pool: np.ndarray, bt: np.ndarray, sl: np.ndarray
     else:
         raise ValueError(impl)
     return pool
+
+
+# ---- layers of different kinds on the data path (§2.2) ----------------------------------------
+
+_KIND = {"full": 0, "window": 1, "state": 2}
+
+
+def _kinds(kinds):
+    k = np.array([_KIND[x[0]] for x in kinds], dtype=np.int64)
+    prm = np.array([x[1] if len(x) > 1 else 0 for x in kinds], dtype=np.int64)
+    return k, prm
+
+
+def layered_offsets(g: Geom, kinds, sl) -> np.ndarray:
+    """Where every layer's slab starts on the wire of a model whose layers differ in kind
+    (``kinds`` as for kv_bytes_layered, one entry per model layer); the last entry is the total,
+    the sum over the requests of Eq. 1 per layer kind."""
+    k, prm = _kinds(kinds)
+    sl = np.ascontiguousarray(sl, dtype=np.int32)
+    off = np.zeros(len(kinds) + 1, dtype=np.int64)
+    cg = g._c()
+    _load().oracle_layered_offsets(ctypes.byref(cg), len(kinds), k.ctypes.data, prm.ctypes.data,
+                                   sl.shape[0], sl.ctypes.data, off.ctypes.data)
+    return off
+
+
+def _layered_args(g, kinds, pool, bt, sl, state_pool, S_state_layer, S_slot, slots, wire):
+    k, prm = _kinds(kinds)
+    bt, sl = _tables(bt, sl)
+    n_att = int((k != 2).sum())
+    assert n_att <= g.L, "the paged pool holds one layer per attention layer of the model"
+    off = layered_offsets(g, kinds, sl)
+    assert wire.size >= int(off[-1]), (wire.size, int(off[-1]))
+    # extent guards for the C loops: every attention layer like a per-layer call
+    for a, l in enumerate(np.flatnonzero(k != 2)):
+        gl = Geom(**{**g.__dict__, "window": int(prm[l]) if k[l] == 1 else 0, "W_layer": 0, "W_plane": 0})
+        _check_extent(gl, a, pool, bt, sl, wire[int(off[l]):])
+    n_state = int((k == 2).sum())
+    if n_state:
+        slots = np.ascontiguousarray(slots, dtype=np.int32)
+        assert slots.shape == sl.shape and slots.min() >= 0
+        need = (n_state - 1) * S_state_layer + int(slots.max()) * S_slot + int(prm[k == 2].max())
+        assert state_pool is not None and state_pool.size >= need, (need,)
+        assert int(prm[k == 2].max()) <= S_slot
+    else:
+        slots = np.zeros(sl.shape, dtype=np.int32)
+        state_pool = np.zeros(1, dtype=np.uint8) if state_pool is None else state_pool
+    cg = g._c()
+    return (cg, k, prm, bt, sl, slots, state_pool, off,
+            (ctypes.byref(cg), len(kinds), k.ctypes.data, prm.ctypes.data, pool.ctypes.data,
+             sl.shape[0], bt.shape[1], bt.ctypes.data, sl.ctypes.data, state_pool.ctypes.data,
+             S_state_layer, S_slot, slots.ctypes.data, wire.ctypes.data))
+
+
+def pack_layered(g: Geom, kinds, pool, bt, sl, state_pool=None, S_state_layer: int = 0,
+                 S_slot: int = 0, slots=None, wire=None):
+    """All layers of a model whose layers differ in kind onto one wire, slab after slab in model
+    order. Returns (wire, offsets)."""
+    off = layered_offsets(g, kinds, sl)
+    if wire is None:
+        wire = np.zeros(max(int(off[-1]), 1), dtype=np.uint8)
+    _u8(pool, False), _u8(wire, True)
+    keep = _layered_args(g, kinds, pool, bt, sl, state_pool, S_state_layer, S_slot, slots, wire)
+    _load().oracle_pack_layered(*keep[-1])
+    return wire, off
+
+
+def unpack_layered(g: Geom, kinds, pool, bt, sl, wire, state_pool=None, S_state_layer: int = 0,
+                   S_slot: int = 0, slots=None):
+    """The inverse, in place: pool (and state_pool) <- wire; untouched bytes keep their value."""
+    _u8(pool, True), _u8(wire, False)
+    if state_pool is not None:
+        _u8(state_pool, True)
+    keep = _layered_args(g, kinds, pool, bt, sl, state_pool, S_state_layer, S_slot, slots, wire)
+    _load().oracle_unpack_layered(*keep[-1])
+    return pool
+
+
+# ---- transport selection (Alg. 1) and planning rates (§3.3) -----------------------------------
+
+MODES = {"nvlink": 1, "pcie": 2, "rdma": 3, "tcp": 4}
+MODE_NAMES = {v: k for k, v in MODES.items()}
+
+
+def select_transport(s, t, cluster_has_rdma: bool, override: str | None = None) -> str:
+    """Alg. 1. ``s`` and ``t`` are (nvlink_domain, has_nvlink, node_ip) of the source and the
+    target instance. Returns "nvlink", "pcie", "rdma" or "tcp"."""
+    m = _load().oracle_select_transport(
+        MODES[override] if override else 0, s[0].encode(), int(bool(s[1])), s[2].encode(),
+        t[0].encode(), int(bool(t[1])), t[2].encode(), int(bool(cluster_has_rdma)))
+    return MODE_NAMES[m]
+
+
+def planning_rate(mode: str) -> float:
+    """Bytes per second the orchestrator plans with for a mode (§3.3)."""
+    return float(_load().oracle_planning_rate(MODES[mode]))
 
 
 # ---- integrity check and header of the serialised cache (§3.4) --------------------------------

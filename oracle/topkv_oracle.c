@@ -4,6 +4,9 @@
  * Pinned by tests/test_oracle_*.py against: the values of Table 1 and Table 4, the §5.2
  * worked example, a hand-derived miniature, an independently derived inverse index map,
  * memcpy / row-gather special cases, and round-trip and permutation invariants.
+ * The layered pack / unpack (layers of different kinds, §2.2) is pinned against numpy slices of
+ * the full pack and a fancy-index gather of the state slots, and its size against Eq. 1 per
+ * layer kind; the transport selector against every branch of Alg. 1 and, with Eq. 2, Table 4.
  * The CRC routine is pinned against liblzma (ECMA-182 polynomial), both catalogue check values
  * and a polynomial-remainder derivation.
  * parity unpinned: WHICH CRC-64 the paper means (it names no polynomial; the ISO 3309 one is
@@ -182,6 +185,94 @@ void oracle_unpack_rows(const oracle_geom* g, int64_t layer, uint8_t* pool, int6
                         int64_t maxp, const int32_t* bt, const int32_t* sl, const uint8_t* wire,
                         int threads) {
   run_rows(g, layer, pool, R, maxp, bt, sl, (uint8_t*)wire, threads, 0);
+}
+
+/* ---- layers of different kinds on the data path (§2.2) ---------------------------------- */
+
+static int64_t kept_by_kind(int64_t kind, int64_t param, int64_t s) {
+  return (kind == 1 && param < s) ? param : s; /* a windowed layer is capped at its window */
+}
+
+void oracle_layered_offsets(const oracle_geom* g, int64_t n_layers, const int64_t* kind,
+                            const int64_t* param, int64_t R, const int32_t* sl, int64_t* offsets) {
+  int64_t tok_bytes = g->F * g->h_kv * g->d_h * g->b_p;
+  int64_t off = 0;
+  for (int64_t l = 0; l < n_layers; ++l) {
+    offsets[l] = off;
+    for (int64_t r = 0; r < R; ++r)
+      off += (kind[l] == 2) ? param[l] : tok_bytes * kept_by_kind(kind[l], param[l], sl[r]);
+  }
+  offsets[n_layers] = off;
+}
+
+static void layered(const oracle_geom* g, int64_t n_layers, const int64_t* kind, const int64_t* param,
+                    uint8_t* pool, int64_t R, int64_t maxp, const int32_t* bt, const int32_t* sl,
+                    uint8_t* state_pool, int64_t S_state_layer, int64_t S_slot, const int32_t* slot,
+                    uint8_t* wire, int pack) {
+  int64_t* off = (int64_t*)malloc(sizeof(int64_t) * (size_t)(n_layers + 1));
+  oracle_layered_offsets(g, n_layers, kind, param, R, sl, off);
+  int64_t a = 0, j = 0; /* attention layers and state layers seen so far */
+  for (int64_t l = 0; l < n_layers; ++l) {
+    uint8_t* slab = wire + off[l];
+    if (kind[l] == 2) {
+      for (int64_t r = 0; r < R; ++r)
+        for (int64_t b = 0; b < param[l]; ++b) {
+          uint8_t* st = state_pool + j * S_state_layer + (int64_t)slot[r] * S_slot + b;
+          if (pack) slab[r * param[l] + b] = *st;
+          else *st = slab[r * param[l] + b];
+        }
+      ++j;
+    } else {
+      oracle_geom gl = *g; /* this layer's view: its window, its slab as the whole wire */
+      gl.window = (kind[l] == 1) ? param[l] : 0;
+      gl.W_layer = 0;
+      gl.W_plane = 0;
+      if (pack) oracle_pack_ref(&gl, a, pool, R, maxp, bt, sl, slab);
+      else oracle_unpack_ref(&gl, a, pool, R, maxp, bt, sl, slab);
+      ++a;
+    }
+  }
+  free(off);
+}
+
+void oracle_pack_layered(const oracle_geom* g, int64_t n_layers, const int64_t* kind,
+                         const int64_t* param, const uint8_t* pool, int64_t R, int64_t maxp,
+                         const int32_t* bt, const int32_t* sl, const uint8_t* state_pool,
+                         int64_t S_state_layer, int64_t S_slot, const int32_t* slot, uint8_t* wire) {
+  layered(g, n_layers, kind, param, (uint8_t*)pool, R, maxp, bt, sl, (uint8_t*)state_pool, S_state_layer,
+          S_slot, slot, wire, 1);
+}
+
+void oracle_unpack_layered(const oracle_geom* g, int64_t n_layers, const int64_t* kind,
+                           const int64_t* param, uint8_t* pool, int64_t R, int64_t maxp,
+                           const int32_t* bt, const int32_t* sl, uint8_t* state_pool,
+                           int64_t S_state_layer, int64_t S_slot, const int32_t* slot,
+                           const uint8_t* wire) {
+  layered(g, n_layers, kind, param, pool, R, maxp, bt, sl, state_pool, S_state_layer, S_slot, slot,
+          (uint8_t*)wire, 0);
+}
+
+/* ---- transport selection (Alg. 1), planning rates (§3.3) ---------------------------------- */
+
+int oracle_select_transport(int override_mode, const char* s_domain, int s_has_nvlink,
+                            const char* s_ip, const char* t_domain, int t_has_nvlink,
+                            const char* t_ip, int cluster_has_rdma) {
+  if (override_mode != 0) return override_mode;                 /* manual override configured   */
+  int has_nvlink = s_has_nvlink && t_has_nvlink && strcmp(s_domain, t_domain) == 0;
+  if (has_nvlink) return ORACLE_MODE_NVLINK;                    /* same NVLink domain           */
+  if (strcmp(s_ip, t_ip) == 0) return ORACLE_MODE_PCIE;         /* same node, cross-domain      */
+  if (cluster_has_rdma) return ORACLE_MODE_RDMA;                /* cross-node, RDMA available   */
+  return ORACLE_MODE_TCP;                                       /* fallback                     */
+}
+
+double oracle_planning_rate(int mode) {
+  switch (mode) {
+    case ORACLE_MODE_NVLINK: return 450e9; /* NVLink 4.0, 18 links, unidirectional       */
+    case ORACLE_MODE_PCIE: return 50e9;    /* Gen5 x16 practical throughput              */
+    case ORACLE_MODE_RDMA: return 25e9;    /* 400 Gbps InfiniBand NDR less protocol cost */
+    case ORACLE_MODE_TCP: return 10e9;     /* 100 Gbps Ethernet with gRPC framing        */
+    default: return 0.0;
+  }
 }
 
 /* ---- CRC-64 (§3.4) -------------------------------------------------------------------- */

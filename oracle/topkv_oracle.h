@@ -59,6 +59,41 @@ void oracle_unpack_rows(const oracle_geom* g, int64_t layer, uint8_t* pool, int6
                         int64_t maxp, const int32_t* bt, const int32_t* sl, const uint8_t* wire,
                         int threads);
 
+/* ---- a model whose layers differ in kind, on the data path (§2.2) ---------------------------
+ * kind[l] / param[l] as for oracle_kv_bytes_layered. Attention layers (full, windowed) live in
+ * the paged pool and are numbered among themselves in model order: the a-th attention layer is
+ * layer a of the pool (g->L of them). Constant-state layers keep one fixed-size state per
+ * request in a pool of slots and are numbered among themselves too: byte b of the state of
+ * request r in the j-th state layer is state_pool[j*S_state_layer + slot[r]*S_slot + b].
+ * The wire holds the layers' slabs back to back in model order (the order in which the
+ * pipelined transfer sends them, §5.2): an attention layer's slab is the pack of the tokens it
+ * keeps (all, or the last min(s, window)), a state layer's slab the R states in request order.
+ * offsets[l] is where slab l starts, offsets[n_layers] the total: the sum over the requests of
+ * Eq. 1 per layer kind. g->window, g->W_layer and g->W_plane are not used. */
+void oracle_layered_offsets(const oracle_geom* g, int64_t n_layers, const int64_t* kind,
+                            const int64_t* param, int64_t R, const int32_t* sl, int64_t* offsets);
+void oracle_pack_layered(const oracle_geom* g, int64_t n_layers, const int64_t* kind,
+                         const int64_t* param, const uint8_t* pool, int64_t R, int64_t maxp,
+                         const int32_t* bt, const int32_t* sl, const uint8_t* state_pool,
+                         int64_t S_state_layer, int64_t S_slot, const int32_t* slot, uint8_t* wire);
+void oracle_unpack_layered(const oracle_geom* g, int64_t n_layers, const int64_t* kind,
+                           const int64_t* param, uint8_t* pool, int64_t R, int64_t maxp,
+                           const int32_t* bt, const int32_t* sl, uint8_t* state_pool,
+                           int64_t S_state_layer, int64_t S_slot, const int32_t* slot,
+                           const uint8_t* wire);
+
+/* ---- transport selection (Alg. 1) and the planning rates of §3.3 -------------------------
+ * Modes in the order Alg. 1 tries them. override_mode 0 = no manual override configured.
+ * HasNVLink(s, t): both instances report NVLink and are registered in the same NVLink domain
+ * (the paper compares node names: an 8-GPU domain is a node); IsSameNode(s, t): equal node IP
+ * addresses; HasRDMA(): a cluster-level flag. */
+enum { ORACLE_MODE_NVLINK = 1, ORACLE_MODE_PCIE = 2, ORACLE_MODE_RDMA = 3, ORACLE_MODE_TCP = 4 };
+int oracle_select_transport(int override_mode, const char* s_domain, int s_has_nvlink,
+                            const char* s_ip, const char* t_domain, int t_has_nvlink,
+                            const char* t_ip, int cluster_has_rdma);
+/* Achievable rate the orchestrator plans with, bytes per second (§3.3); 0 for an unknown mode. */
+double oracle_planning_rate(int mode);
+
 /* ---- integrity check of the serialised tensors (§3.4) -----------------------------------
  * The paper's header carries "CRC-64 checksums for both key and value tensors" and does not
  * name the polynomial. Reading taken: the reflected CRC-64 with all-ones initial value and
