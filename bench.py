@@ -3,10 +3,12 @@
 
 A "step" is one pass of the hot path over one synthetic batch: the plan (prefix sums), then
 pack of every layer, then unpack of every layer, device to device. The headline workload is
-the Llama-3-8B-shaped cache (16 requests, 512..4096 tokens, 32 layers). The same JSON line
-also carries the host-leg (PCIe) figure as ``e2e``, the live roofline of the pack kernel, the
-CPU oracle timed on this machine as ``cpu_baseline``, and, at one GPU, the other benchmark shapes
-(70B GQA with its host leg, DeepSeek-V3 MLA) and the side-stream overlap run under ``extra``.
+the largest single-GPU configuration: the Llama-3-70B-shaped cache (8 requests of 4096
+tokens, 80 layers, 10 GiB of wire). The same JSON line also carries the host-leg (PCIe) figure
+as ``e2e`` (all 80 layers through pinned host memory), the live roofline of the pack kernel,
+the CPU oracle timed on this machine as ``cpu_baseline``, and, at one GPU, the other benchmark
+shapes (8B GQA, DeepSeek-V3 MLA), the side-stream overlap runs and the checksummed copy under
+``extra``.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--extras ...]
 
@@ -32,10 +34,26 @@ METRIC = "kv_pack_unpack_GBps"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM traffic of one pack launch relative to its algorithmic bytes, from a steady-state ncu
-# capture of this kernel at the same per-launch size (--cache-control none, six launches):
-# (dram__bytes_read.sum + dram__bytes_write.sum) / (2*N_layer).
-NCU_TRAFFIC_RATIO = 0.995
+# DRAM traffic of one pack launch relative to its algorithmic bytes comes from an ncu capture
+# of this kernel at the same per-launch size, summarised under profiles/: the summary carries
+# a line "traffic_ratio = <(dram__bytes_read.sum + dram__bytes_write.sum) / (2*N_layer)>" and
+# the date and command of the capture, which are stamped into the bench line beside the number.
+TRAFFIC_PROFILE = os.path.join("profiles", "page_copy_kernel_pack_cfg3_4layers.md")
+
+
+def ncu_traffic(bytes_per_launch):
+    """(traffic bytes per launch or None, where the figure comes from)."""
+    import re
+    path = os.path.join(ROOT, TRAFFIC_PROFILE)
+    try:
+        text = open(path).read()
+        ratio = float(re.search(r"^traffic_ratio\s*=\s*([0-9.]+)", text, re.M).group(1))
+        when = re.search(r"^captured\s*=\s*(\S+)", text, re.M)
+        src = f"{TRAFFIC_PROFILE} (ncu capture of {when.group(1) if when else 'unknown date'}, " \
+              f"ratio {ratio} x algorithmic bytes; not re-measured in this run)"
+        return int(ratio * bytes_per_launch), src
+    except Exception:
+        return None, f"{TRAFFIC_PROFILE} not found or without a traffic_ratio line"
 
 
 def measured_peak_gbs():
@@ -175,7 +193,7 @@ def run_reference(args):
     if rank != 0:
         return
     from paper_2607_28633_b200 import workloads as wl
-    spec = wl.CFG2
+    spec = HEADLINE(wl)
     batch = wl.make_batch(spec)
     per_step = max(1.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
     for _ in range(args.warmup):
@@ -199,6 +217,34 @@ def run_reference(args):
         "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0,
                 "d2h_bytes_per_step": 0},
     }))
+
+
+def HEADLINE(wl):
+    """The workload the N = 1 line is quoted on: the largest single-GPU configuration."""
+    return wl.CFG3
+
+
+_PINNED = {}
+
+
+def pinned_buffer(nbytes, fallback_bytes=None):
+    """One pinned host buffer for the whole run, grown on demand and handed out as views (pinning
+    10 GiB takes seconds, and the host allocator rounds sizes up). Returns a uint8 tensor of
+    nbytes, or of fallback_bytes when the box refuses the larger size."""
+    import torch
+    have = _PINNED.get("buf")
+    if have is not None and have.numel() >= nbytes:
+        return have[:nbytes]
+    try:
+        _PINNED["buf"] = None
+        del have
+        _PINNED["buf"] = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
+        return _PINNED["buf"][:nbytes]
+    except Exception:
+        if fallback_bytes is None:
+            raise
+        _PINNED["buf"] = torch.empty(fallback_bytes, dtype=torch.uint8, pin_memory=True)
+        return _PINNED["buf"][:fallback_bytes]
 
 
 def workload_config(spec, batch):
@@ -493,6 +539,58 @@ def device_copy_baseline(dev, stream, nbytes, reps=10):
     return 2 * nbytes / (best * 1e-3) / 1e9
 
 
+def bench_chain(w, stream, steps, flags=0):
+    """The dependent order of a relay without a host hop: for every layer, pack into ONE shared
+    wire slab, then unpack that slab, so that every kernel depends on the data of the kernel
+    just before it and no launch may be declared independent. GB/s of read + write traffic."""
+    import ctypes
+    import torch
+    from paper_2607_28633_b200 import binding as tk
+    lo = type(w.layout)()
+    ctypes.memmove(ctypes.byref(lo), ctypes.byref(w.layout), ctypes.sizeof(lo))
+    lo.wire_layer_stride = 0
+    slab = w.wire[:w.n_layer]
+    bs = tk.make_batch(w.src_bt, w.seq_lens, w.batch.total_tokens, w.cu, flags)
+    bd = tk.make_batch(w.dst_bt, w.seq_lens, w.batch.total_tokens, w.cu, flags)
+
+    def run():
+        for l in range(w.layers):
+            tk.check(tk.topkv_pack_layer(l, w.src_pool, lo, bs, slab, w.n_layer, stream))
+            tk.check(tk.topkv_unpack_layer(l, w.dst_pool, lo, bd, slab, w.n_layer, stream))
+    run()
+    stream.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(steps):
+        run()
+    b.record(stream)
+    stream.synchronize()
+    ms = a.elapsed_time(b) / steps
+    return 4.0 * w.n_layer * w.layers / (ms * 1e-3) / 1e9, ms / (2 * w.layers) * 1e3
+
+
+def host_leg_forms(w, dev, stream, pinned, slots, steps):
+    """The host leg of the workload in its three forms against a pinned cudaMemcpyAsync of one
+    slab measured in the same run."""
+    import torch
+    nobar = lambda: None
+    staging = torch.empty(w.n_layer, dtype=torch.uint8, device=dev)
+    staging2 = torch.empty(w.n_layer, dtype=torch.uint8, device=dev)
+    base = pinned_copy_baseline(dev, stream, w.n_layer)
+    out = {}
+    for form, st, st2 in (("staged", staging, None), ("staged_two_streams", staging, staging2),
+                          ("direct", None, None)):
+        _, th, fh = bench_host_leg(w, stream, pinned, st, steps, 1, nobar, slots, st2)
+        d2h = w.n_layer * w.layers / (th * 1e-3) / 1e9
+        h2d = w.n_layer * w.layers / (fh * 1e-3) / 1e9
+        out[form] = {"to_host_GBps": round(d2h, 2), "from_host_GBps": round(h2d, 2),
+                     "to_host_frac_of_pinned_copy": round(d2h / base["d2h"], 4),
+                     "from_host_frac_of_pinned_copy": round(h2d / base["h2d"], 4)}
+    out["pinned_copy_GBps"] = {k: round(v, 2) for k, v in base.items()}
+    out["pinned_slots"] = slots
+    return out
+
+
 def run_extra(name, dev, stream, args, peak):
     """Other benchmark shapes at one GPU; returns a dict for the ``extra`` object."""
     import torch
@@ -554,7 +652,7 @@ def run_extra(name, dev, stream, args, peak):
         b = w.batch
         tx = session.TransferSender(w.src_pool, w.layout, w.src_bt, w.seq_lens, b.total_tokens)
         rx = session.TransferReceiver(w.dst_pool, w.layout, w.dst_bt, w.seq_lens, b.total_tokens)
-        h_wire = torch.empty(w.layers * w.n_layer, dtype=torch.uint8, pin_memory=True)
+        h_wire = pinned_buffer(w.layers * w.n_layer)
         ids = list(range(spec.R))
         best, ok = 1e30, True
         for it in range(3):
@@ -575,15 +673,76 @@ def run_extra(name, dev, stream, args, peak):
         torch.cuda.empty_cache()
         return out
     if name == "crc":
-        spec = wl.CFG2 if args.layers is None else wl.with_layers(wl.CFG2, args.layers)
-        w = harness.setup(spec, dev, fill_dst=False)
-        out = {"workload": spec.name}
-        out.update(bench_crc(w, stream, max(1, min(args.steps, 5))))
-        out["frac_of_hbm_peak"] = round(out["pack_crc_GBps"] / peak, 4)
-        del w
-        torch.cuda.empty_cache()
+        # the checksummed copy on the three benchmark shapes (16 layers of the two large ones)
+        out = {}
+        for base, layers in ((wl.CFG2, None), (wl.CFG3, 16), (wl.CFG4, 16)):
+            layers = args.layers if args.layers is not None else layers
+            spec = base if layers is None else wl.with_layers(base, layers)
+            w = harness.setup(spec, dev, fill_dst=False)
+            r = {"layers": w.layers}
+            r.update(bench_crc(w, stream, max(1, min(args.steps, 5))))
+            r["frac_of_hbm_peak"] = round(r["pack_crc_GBps"] / peak, 4)
+            r["unpack_frac_of_hbm_peak"] = round(r["unpack_crc_GBps"] / peak, 4)
+            out[base.name] = r
+            del w
+            torch.cuda.empty_cache()
+        out["workload"] = wl.CFG2.name
+        out["frac_of_hbm_peak"] = out[wl.CFG2.name]["frac_of_hbm_peak"]
         return out
-    if name in ("cfg3", "cfg4"):
+    if name == "chain":
+        # pack(l) -> unpack(l) per layer through one shared slab: every launch depends on the one
+        # before it (the order of a device-to-device relay), so TOPKV_FLAG_OVERLAP_PREVIOUS is
+        # not available; plain launches and TOPKV_FLAG_TABLES_SETTLED
+        out = {"workload": "cfg2_llama3_8b, cfg4_dsv3_mla", "order": "pack(l), unpack(l), pack(l+1), ..."}
+        for base in (wl.CFG2, wl.CFG4):
+            spec = base if args.layers is None else wl.with_layers(base, args.layers)
+            w = harness.setup(spec, dev, fill_dst=False)
+            r = {}
+            for label, flags in (("plain", 0), ("tables_settled", tk.TOPKV_FLAG_TABLES_SETTLED)):
+                gbs, us = bench_chain(w, stream, max(1, min(args.steps, 5)), flags)
+                r[label] = {"GBps": round(gbs, 1), "us_per_launch": round(us, 2),
+                            "frac_of_hbm_peak": round(gbs / peak, 4),
+                            "frac_of_8000_spec": round(gbs / 8000.0, 4)}
+            out[base.name] = r
+            del w
+            torch.cuda.empty_cache()
+        return out
+    if name == "overlap_curve":
+        # three points on the Eq. 3 curve (§5.2) and the interference §5.5 could not validate:
+        # slack (64 MiB per layer under a 2.8 ms layer), near-saturated (128 MiB per layer, about
+        # 2.4 ms on the link, under the same layer) and oversubscribed (128 MiB per layer under
+        # a halved stand-in, so that T_xfer > T_rem and Eq. 3 predicts hidden < 1)
+        points = (("slack", wl.CFG5, wl.GEMM_FFN), ("near_saturated", wl.CFG3, wl.GEMM_FFN),
+                  ("oversubscribed", wl.CFG3, wl.GEMM_FFN // 2))
+        out = {"workload": "cfg5 / cfg3 batches under the GEMM stand-in"}
+        for label, base, ffn in points:
+            spec = base if args.layers is None else wl.with_layers(base, args.layers)
+            w = harness.setup(spec, dev, need_dst=False, need_wire=False)
+            slots = w.layers
+            pinned = pinned_buffer(slots * w.n_layer, 8 * w.n_layer)
+            slots = min(slots, pinned.numel() // w.n_layer)
+            staging = torch.empty(w.n_layer, dtype=torch.uint8, device=dev)
+            pre = overlap.PrefillStandIn(dev, w.batch.seeds["data"] + 50, ffn=ffn)
+            pt = {"requests": spec.R, "bytes_per_layer": w.n_layer, "gemm_ffn": ffn}
+            for form, st in (("staged", staging), ("direct", None)):
+                r = overlap.run_overlap(w, pinned, st, pre, slots=slots)
+                model = tk.topkv_model_hidden_fraction(r.layers, r.t_layer_compute_ms * 1e-3,
+                                                       r.t_xfer_serial_ms * 1e-3)
+                # what Eq. 3 allows at best: the last slab's transfer can never be hidden
+                bound = min(model, 1.0 - 1.0 / r.layers)
+                pt[form] = {"hidden": round(r.hidden, 4), "hidden_model": round(model, 4),
+                            "hidden_model_minus_last_slab": round(bound, 4),
+                            "slowdown": round(r.slowdown, 4),
+                            "t_layer_compute_ms": round(r.t_layer_compute_ms, 4),
+                            "t_xfer_serial_ms": round(r.t_xfer_serial_ms, 3),
+                            "t_main_overlap_ms": round(r.t_main_overlap_ms, 3),
+                            "exposed_ms": round(r.exposed_ms, 3),
+                            "xfer_gbs_serial": round(r.xfer_gbs_serial, 2)}
+            out[label] = pt
+            del w, pinned, staging, pre
+            torch.cuda.empty_cache()
+        return out
+    if name in ("cfg2", "cfg3", "cfg4"):
         if args.layers is not None:                      # fewer layers: profiling only
             spec = wl.with_layers(spec, args.layers)
         w = harness.setup(spec, dev, fill_dst=False)
@@ -595,38 +754,14 @@ def run_extra(name, dev, stream, args, peak):
                     "unpack_frac_of_peak": round(traffic / (unpack_ms * 1e-3) / 1e9 / peak, 4),
                     "ms_per_step": round(ms, 4), "wire_bytes_per_layer": w.n_layer,
                     "layers": w.layers})
-        if name == "cfg3":
-            slots = w.layers
-            try:
-                pinned = torch.empty(slots * w.n_layer, dtype=torch.uint8, pin_memory=True)
-            except Exception:
-                slots = 4
-                pinned = torch.empty(slots * w.n_layer, dtype=torch.uint8, pin_memory=True)
-            staging = torch.empty(w.n_layer, dtype=torch.uint8, device=dev)
-            base = pinned_copy_baseline(dev, stream, w.n_layer)
-            hs = max(1, min(args.steps, 3))
-            staging2 = torch.empty(w.n_layer, dtype=torch.uint8, device=dev)
-            for form, st, st2 in (("staged", staging, None), ("staged_two_streams", staging, staging2),
-                                  ("direct", None, None)):
-                _, th, fh = bench_host_leg(w, stream, pinned, st, hs, 1, nobar, slots, st2)
-                d2h = w.n_layer * w.layers / (th * 1e-3) / 1e9
-                h2d = w.n_layer * w.layers / (fh * 1e-3) / 1e9
-                out[f"host_leg_{form}"] = {
-                    "to_host_GBps": round(d2h, 2), "from_host_GBps": round(h2d, 2),
-                    "to_host_frac_of_pinned_copy": round(d2h / base["d2h"], 4),
-                    "from_host_frac_of_pinned_copy": round(h2d / base["h2d"], 4)}
-            out["pinned_copy_GBps"] = {k: round(v, 2) for k, v in base.items()}
-            out["pinned_slots"] = slots
-            del pinned, staging, staging2
+        if name == "cfg2":
+            out["repage_GBps"] = round(bench_repage(w, stream, max(1, min(args.steps, 5))), 1)
         del w
     elif name == "cfg5":
         w = harness.setup(spec, dev, need_dst=False, need_wire=False)
         slots = w.layers
-        try:
-            pinned = torch.empty(slots * w.n_layer, dtype=torch.uint8, pin_memory=True)
-        except Exception:
-            slots = 8
-            pinned = torch.empty(slots * w.n_layer, dtype=torch.uint8, pin_memory=True)
+        pinned = pinned_buffer(slots * w.n_layer, 8 * w.n_layer)
+        slots = min(slots, pinned.numel() // w.n_layer)
         staging = torch.empty(w.n_layer, dtype=torch.uint8, device=dev)
         pre = overlap.PrefillStandIn(dev, w.batch.seeds["data"] + 50)
         best = None
@@ -672,7 +807,7 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="topkv", choices=["topkv", "reference"])
-    ap.add_argument("--extras", default="cfg5,cfg3,cfg4,crc,session,cfg1",
+    ap.add_argument("--extras", default="cfg5,overlap_curve,cfg2,cfg4,chain,crc,session,cfg1",
                     help="comma list of extra workloads measured at one GPU ('' for none)")
     ap.add_argument("--variant", type=int, default=None, help="kernel family (see topkv.h)")
     ap.add_argument("--layers", type=int, default=None, help="fewer layers (profiling only)")
@@ -731,7 +866,8 @@ def main():
         return dist_util.sum_over_ranks(dist, x, dev)
 
     peak, peak_src = measured_peak_gbs()
-    spec = wl.CFG2 if args.layers is None else wl.with_layers(wl.CFG2, args.layers)
+    head = HEADLINE(wl)
+    spec = head if args.layers is None else wl.with_layers(head, args.layers)
     w = harness.setup(spec, dev, rank=rank, fill_dst=False)
     stream = torch.cuda.Stream(dev)
     L, n_layer = w.layers, w.n_layer
@@ -753,45 +889,52 @@ def main():
     achieved_unpack = 2.0 * n_layer / (unpack_launch_ms * 1e-3) / 1e9
 
     e2e = None
+    extra = {}
     if not args.no_e2e:
-        slots = L
-        try:
-            pinned = torch.empty(slots * n_layer, dtype=torch.uint8, pin_memory=True)
-        except Exception:
-            slots = 4
-            pinned = torch.empty(slots * n_layer, dtype=torch.uint8, pin_memory=True)
+        # every layer through pinned host memory with the C-ABI host-leg calls: one slab per
+        # layer (10 GiB for the 70B shape), or a ring of 4 slabs when the box refuses that much
+        pinned = pinned_buffer(L * n_layer, 4 * n_layer)
+        slots = min(L, pinned.numel() // n_layer)
         staging = torch.empty(n_layer, dtype=torch.uint8, device=dev)
         hs = max(1, min(args.steps, 3))
         ems, th, fh = bench_host_leg(w, stream, pinned, staging, hs, 1, barrier, slots)
         form = "staged (kernel + copy engine), pack of all layers then unpack of all layers"
+        if slots < L:
+            form += f"; ring of {slots} pinned slabs (the box refused one slab per layer)"
         if slots >= L:   # both link directions at once: unpack layer l while later layers pack
             staging_rx = torch.empty(n_layer, dtype=torch.uint8, device=dev)
             rms = bench_host_relay(w, stream, pinned, staging, staging_rx, hs, 1, barrier, slots)
             if rms < ems:
-                sequential_ms, ems = ems, rms
+                ems = rms
                 form = ("staged (kernel + copy engine), pipelined relay: layer l is unpacked from "
-                        "the host while later layers are still packed to it")
+                        "the host while later layers are still packed to it; one pinned slab per layer")
             del staging_rx
         ems_max = max_over_ranks(ems)
         e2e = {"value": round(bytes_step_all / (ems_max * 1e-3) / 1e9, 3), "unit": UNIT,
                "h2d_bytes_per_step": n_layer * L, "d2h_bytes_per_step": n_layer * L,
                "form": form, "steps": hs, "ms_per_step": round(ems_max, 3),
+               "pinned_slots": slots,
                "sequential_ms_per_step": round(th + fh, 3),
                "to_host_link_GBps": round(n_layer * L / (th * 1e-3) / 1e9, 2),
                "from_host_link_GBps": round(n_layer * L / (fh * 1e-3) / 1e9, 2)}
-        del pinned, staging
-        if rank == 0 and world == 1 and slots >= L:
-            # what the link gives each direction while both are busy: plain pinned copies
-            bidir = pinned_copy_bidirectional_baseline(dev, n_layer)
-            e2e["pinned_copy_both_directions_GBps_each"] = round(bidir, 2)
-            e2e["link_GBps_each_direction"] = round(n_layer * L / (ems_max * 1e-3) / 1e9, 2)
-            e2e["frac_of_pinned_copy_both_directions"] = round(
-                n_layer * L / (ems_max * 1e-3) / 1e9 / bidir, 4)
+        del staging
+        if rank == 0 and world == 1:
+            if slots >= L:
+                # what the link gives each direction while both are busy: plain pinned copies
+                bidir = pinned_copy_bidirectional_baseline(dev, n_layer)
+                e2e["pinned_copy_both_directions_GBps_each"] = round(bidir, 2)
+                e2e["link_GBps_each_direction"] = round(n_layer * L / (ems_max * 1e-3) / 1e9, 2)
+                e2e["frac_of_pinned_copy_both_directions"] = round(
+                    n_layer * L / (ems_max * 1e-3) / 1e9 / bidir, 4)
+            # the host leg one direction at a time, in its three forms, against a pinned copy
+            hl = host_leg_forms(w, dev, stream, pinned, slots, hs)
+            e2e["host_leg"] = hl
+            e2e["to_host_frac_of_pinned_copy"] = hl["staged"]["to_host_frac_of_pinned_copy"]
+            e2e["from_host_frac_of_pinned_copy"] = hl["staged"]["from_host_frac_of_pinned_copy"]
+        del pinned
 
-    extra = {}
     if rank == 0 and world == 1:
         extra["device_copy_GBps_same_bytes"] = round(device_copy_baseline(dev, stream, n_layer), 1)
-        extra["repage_GBps"] = round(bench_repage(w, stream, max(1, min(args.steps, 5))), 1)
     batch = w.batch
     del w
     torch.cuda.empty_cache()
@@ -805,18 +948,19 @@ def main():
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v, n, cores, dt = oracle_sample(wl.CFG2, wl.make_batch(wl.CFG2), seconds_target=12.0)
+        v, n, cores, dt = oracle_sample(head, wl.make_batch(head), seconds_target=12.0)
         cpu = {"value": round(v, 3), "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": f"one of the {wl.CFG2.L} layers of this workload, pack+unpack, repeated "
+               "sample": f"one of the {head.L} layers of this workload, pack+unpack, repeated "
                          f"{n} times, rows-memcpy oracle, {dt:.1f} s"}
         # for context: the same oracle on one thread, and the byte-by-byte definition on cfg1
-        v1, n1, _, dt1 = oracle_sample(wl.CFG2, wl.make_batch(wl.CFG2), seconds_target=4.0, threads=1)
+        v1, n1, _, dt1 = oracle_sample(head, wl.make_batch(head), seconds_target=4.0, threads=1)
         vr, nr, _, dtr = oracle_sample(wl.CFG1, wl.make_batch(wl.CFG1), seconds_target=3.0, threads=1,
                                        impl="ref")
         cpu["one_thread_GBps"] = round(v1, 3)
         cpu["byte_loop_definition_cfg1_GBps"] = round(vr, 4)
 
     if rank == 0:
+        traffic, traffic_src = ncu_traffic(2 * n_layer)
         line = {
             "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(ms_max, 4),
@@ -829,10 +973,10 @@ def main():
                          "frac_of_8000_spec": round(achieved / 8000.0, 4),
                          "bytes_per_launch": 2 * n_layer,
                          "launch_ms": round(pack_launch_ms, 5),
-                         "traffic": (None if NCU_TRAFFIC_RATIO is None
-                                     else int(NCU_TRAFFIC_RATIO * 2 * n_layer)),
+                         "traffic": traffic, "traffic_source": traffic_src,
                          "unpack_achieved": round(achieved_unpack, 1),
-                         "unpack_frac": round(achieved_unpack / peak, 4)},
+                         "unpack_frac": round(achieved_unpack / peak, 4),
+                         "unpack_launch_ms": round(unpack_launch_ms, 5)},
             "e2e": e2e, "cpu_baseline": cpu, "extra": extra,
         }
         print(json.dumps(line))

@@ -419,6 +419,38 @@ double topkv_model_t_eff_s(double t_last_s, double t_xfer_s, double t_rem_s);
  * layer's cache is ready (§5.2 worked example): min(1, (layers-1)*t_layer / t_xfer). */
 double topkv_model_hidden_fraction(int layers, double t_layer_compute_s, double t_xfer_total_s);
 
+/* ---- transport selection (Alg. 1) and planning rates (§3.3): host only, context -------------
+ * What the transfer manager decides BEFORE any byte moves: which transport carries the cache
+ * from the source instance to the target instance. This library implements one of those
+ * transports on one GPU (the pinned-host PCIe leg); the selector is here so that a caller can
+ * apply the paper's rule and its latency model (Eq. 2) to size a transfer. It moves no data
+ * and opens no connection. */
+enum {
+  TOPKV_TRANSPORT_NVLINK = 1, /* same NVLink domain: 450 GB/s unidirectional (NVLink 4.0, 18 links) */
+  TOPKV_TRANSPORT_PCIE = 2,   /* same node, cross-domain: 50 GB/s (Gen5 x16, practical)             */
+  TOPKV_TRANSPORT_RDMA = 3,   /* cross-node, RDMA available: 25 GB/s (InfiniBand NDR)               */
+  TOPKV_TRANSPORT_TCP = 4     /* fallback: 10 GB/s (100 GbE with gRPC framing)                      */
+};
+/* What a worker instance reports when it registers (§3.2). Strings are NUL-terminated, HOST. */
+typedef struct topkv_endpoint {
+  uint32_t struct_size;      /* = sizeof(topkv_endpoint)                                          */
+  uint32_t has_nvlink;       /* the instance reports HasNVLink = true                             */
+  const char* nvlink_domain; /* the NVLink domain it is registered in; the paper compares node    */
+                             /* names (an 8-GPU domain is a node); may be NULL when has_nvlink = 0 */
+  const char* node_ip;       /* IsSameNode compares node IP addresses                             */
+} topkv_endpoint;
+/* Alg. 1, in its order: a configured override (override_mode != 0) wins; else NVLINK when both
+ * instances report NVLink and sit in the same domain; else PCIE on the same node; else RDMA when
+ * the cluster has it (cluster_has_rdma != 0); else TCP. Returns a TOPKV_TRANSPORT_* value, or
+ * TOPKV_ERR_INVALID_ARG (NULL, struct_size mismatch, unknown override, missing node_ip). */
+int topkv_select_transport(const topkv_endpoint* source, const topkv_endpoint* target,
+                           int cluster_has_rdma, int override_mode);
+/* The achievable rate the orchestrator plans with for a mode, bytes per second (§3.3: 450, 50,
+ * 25, 10 GB/s); 0.0 for an unknown mode. Table 4 = topkv_model_transfer_s(1.3e9, rate, 0). */
+double topkv_planning_rate(int mode);
+/* "nvlink", "pcie", "rdma", "tcp", or "unknown". */
+const char* topkv_transport_name(int mode);
+
 /* ---- diagnostics ------------------------------------------------------------------------ */
 
 const char* topkv_strerror(int status);

@@ -45,7 +45,8 @@ EXPORTS = (
     "topkv_retry", "topkv_pack_layer_to_host_crc", "topkv_unpack_layer_from_host_crc",
     "topkv_set_host_leg_ctas", "topkv_pack_layers_to_host_pipelined",
     "topkv_unpack_layers_from_host_pipelined", "topkv_pack_layers", "topkv_unpack_layers",
-    "topkv_copy_vector_bytes",
+    "topkv_copy_vector_bytes", "topkv_select_transport", "topkv_planning_rate",
+    "topkv_transport_name",
 )
 
 
@@ -75,6 +76,21 @@ class topkv_layer_spec(ctypes.Structure):
 
 
 TOPKV_LAYER_FULL, TOPKV_LAYER_WINDOW, TOPKV_LAYER_STATE = 0, 1, 2
+TOPKV_TRANSPORT_NVLINK, TOPKV_TRANSPORT_PCIE, TOPKV_TRANSPORT_RDMA, TOPKV_TRANSPORT_TCP = 1, 2, 3, 4
+
+
+class topkv_endpoint(ctypes.Structure):
+    _fields_ = [("struct_size", c_uint32), ("has_nvlink", c_uint32),
+                ("nvlink_domain", ctypes.c_char_p), ("node_ip", ctypes.c_char_p)]
+
+
+def make_endpoint(nvlink_domain, has_nvlink, node_ip) -> topkv_endpoint:
+    e = topkv_endpoint()
+    e.struct_size = ctypes.sizeof(topkv_endpoint)
+    e.has_nvlink = 1 if has_nvlink else 0
+    e.nvlink_domain = None if nvlink_domain is None else nvlink_domain.encode()
+    e.node_ip = None if node_ip is None else node_ip.encode()
+    return e
 
 
 class topkv_wire_header(ctypes.Structure):
@@ -158,6 +174,12 @@ def lib() -> ctypes.CDLL:
         L.topkv_set_host_leg_ctas.argtypes = [c_int]
         L.topkv_pack_layers.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p]
         L.topkv_unpack_layers.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p]
+        ep = ctypes.POINTER(topkv_endpoint)
+        L.topkv_select_transport.argtypes = [ep, ep, c_int, c_int]
+        L.topkv_planning_rate.argtypes = [c_int]
+        L.topkv_planning_rate.restype = c_double
+        L.topkv_transport_name.argtypes = [c_int]
+        L.topkv_transport_name.restype = ctypes.c_char_p
         L.topkv_copy_vector_bytes.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64]
         for fn in (L.topkv_pack_layers_to_host_pipelined, L.topkv_unpack_layers_from_host_pipelined):
             fn.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p, c_int64,
@@ -441,6 +463,19 @@ def topkv_model_t_eff_s(t_last_s, t_xfer_s, t_rem_s):
 
 def topkv_model_hidden_fraction(layers, t_layer_compute_s, t_xfer_total_s):
     return lib().topkv_model_hidden_fraction(layers, t_layer_compute_s, t_xfer_total_s)
+
+
+def topkv_select_transport(source, target, cluster_has_rdma, override_mode=0):
+    return lib().topkv_select_transport(ctypes.byref(source), ctypes.byref(target),
+                                        int(bool(cluster_has_rdma)), override_mode)
+
+
+def topkv_planning_rate(mode):
+    return lib().topkv_planning_rate(mode)
+
+
+def topkv_transport_name(mode):
+    return lib().topkv_transport_name(mode).decode()
 
 
 def topkv_strerror(status):

@@ -76,6 +76,37 @@ double topkv_model_hidden_fraction(int layers, double t_layer_compute_s, double 
   return covered < 1.0 ? covered : 1.0;
 }
 
+// ---- transport selection (Alg. 1), planning rates (§3.3) ----------------------------------------
+int topkv_select_transport(const topkv_endpoint* s, const topkv_endpoint* t, int cluster_has_rdma,
+                           int override_mode) {
+  if (s == nullptr || t == nullptr || s->struct_size != sizeof(topkv_endpoint) ||
+      t->struct_size != sizeof(topkv_endpoint))
+    return TOPKV_ERR_INVALID_ARG;
+  if (override_mode != 0) {  // a manual override is returned as configured
+    if (override_mode < TOPKV_TRANSPORT_NVLINK || override_mode > TOPKV_TRANSPORT_TCP)
+      return TOPKV_ERR_INVALID_ARG;
+    return override_mode;
+  }
+  if (s->node_ip == nullptr || t->node_ip == nullptr) return TOPKV_ERR_INVALID_ARG;
+  const bool both_report = s->has_nvlink != 0 && t->has_nvlink != 0;
+  if (both_report && (s->nvlink_domain == nullptr || t->nvlink_domain == nullptr))
+    return TOPKV_ERR_INVALID_ARG;
+  if (both_report && std::strcmp(s->nvlink_domain, t->nvlink_domain) == 0) return TOPKV_TRANSPORT_NVLINK;
+  if (std::strcmp(s->node_ip, t->node_ip) == 0) return TOPKV_TRANSPORT_PCIE;
+  return cluster_has_rdma != 0 ? TOPKV_TRANSPORT_RDMA : TOPKV_TRANSPORT_TCP;
+}
+
+double topkv_planning_rate(int mode) {
+  static const double kGBps[5] = {0.0, 450.0, 50.0, 25.0, 10.0};
+  if (mode < TOPKV_TRANSPORT_NVLINK || mode > TOPKV_TRANSPORT_TCP) return 0.0;
+  return kGBps[mode] * 1e9;
+}
+
+const char* topkv_transport_name(int mode) {
+  static const char* const kNames[5] = {"unknown", "nvlink", "pcie", "rdma", "tcp"};
+  return (mode >= TOPKV_TRANSPORT_NVLINK && mode <= TOPKV_TRANSPORT_TCP) ? kNames[mode] : kNames[0];
+}
+
 int topkv_validate_batch_host(const topkv_layout* lo, int32_t R, int32_t maxp,
                               const int32_t* h_bt, const int32_t* h_sl, int require_disjoint) {
   if (!layout_header_ok(lo) || R < 0 || maxp < 0) return TOPKV_ERR_INVALID_ARG;

@@ -79,9 +79,10 @@ def setup(spec: wl.WorkloadSpec, device, layers: int | None = None, rank: int = 
     seeded pattern, so that untouched bytes are part of any comparison) and builds the plan."""
     batch = wl.make_batch(spec, rank=rank)
     L = spec.L if layers is None else layers
-    n_layer = batch.total_tokens * spec.tok_bytes
     lo = tk.make_layout(L, spec.F, spec.H, spec.D, spec.E, spec.P, batch.num_pool_pages,
-                        wire_order=wire_order, wire_layer_stride=n_layer)
+                        wire_order=wire_order)
+    n_layer = tk.check(tk.topkv_wire_layer_bytes(lo, batch.total_tokens))   # N_layer, from the library
+    lo.wire_layer_stride = n_layer
     nbytes = L * lo.pool_layer_stride
     src = wl.fill_torch(nbytes, batch.seeds["data"], device, raw_bits=spec.raw_bits)
     dst = None

@@ -363,3 +363,39 @@ def test_checksummed_host_leg_validates_before_it_enqueues():
     assert tk.topkv_unpack_layer_from_host(4, pool, lo, b, host, 4 * n, staging, n) == tk.TOPKV_ERR_LAYER_RANGE
     assert tk.topkv_unpack_layer_from_host(3, pool, lo, b, host, 4 * n - 1, staging, n) == tk.TOPKV_ERR_CAPACITY
     assert tk.topkv_kernel_launch_count() == before
+
+
+def test_transport_selection_and_planning_rates(golden):
+    """topkv_select_transport against the oracle's Alg. 1 on every combination of the inputs,
+    and the planning rates with Eq. 2 against Table 4."""
+    import itertools
+    import oracle
+    g = golden("paper_values.txt")
+    E = tk.make_endpoint
+    names = {tk.TOPKV_TRANSPORT_NVLINK: "nvlink", tk.TOPKV_TRANSPORT_PCIE: "pcie",
+             tk.TOPKV_TRANSPORT_RDMA: "rdma", tk.TOPKV_TRANSPORT_TCP: "tcp"}
+    doms, ips = ("node-a", "node-b"), ("10.0.0.1", "10.0.0.2")
+    n = 0
+    for ds, dt, hs, ht, ips_, ipt, rdma in itertools.product(doms, doms, (0, 1), (0, 1), ips, ips, (0, 1)):
+        got = tk.topkv_select_transport(E(ds, hs, ips_), E(dt, ht, ipt), rdma)
+        assert names[got] == oracle.select_transport((ds, hs, ips_), (dt, ht, ipt), rdma)
+        assert tk.topkv_transport_name(got) == names[got]
+        n += 1
+    assert n == 128
+    a, b = E("node-a", 1, "10.0.0.1"), E("node-b", 1, "10.0.0.2")
+    for mode, name in names.items():
+        assert tk.topkv_select_transport(a, b, 0, mode) == mode            # the override wins
+        assert tk.topkv_planning_rate(mode) == float(g[f"plan.{name}.gbps"]) * 1e9
+        assert tk.topkv_planning_rate(mode) == oracle.planning_rate(name)
+        ms = tk.topkv_model_transfer_s(1.3e9, tk.topkv_planning_rate(mode), 0.0) * 1e3
+        want = float(g[f"table4.{name}.ms"])
+        assert round(ms, 1 if want < 10 else 0) == want
+    assert tk.topkv_planning_rate(0) == 0.0 and tk.topkv_planning_rate(5) == 0.0
+    assert tk.topkv_transport_name(9) == "unknown"
+    assert tk.topkv_select_transport(a, b, 0, 7) == tk.TOPKV_ERR_INVALID_ARG
+    bad = E("node-a", 1, "10.0.0.1"); bad.struct_size = 4
+    assert tk.topkv_select_transport(bad, b, 0) == tk.TOPKV_ERR_INVALID_ARG
+    assert tk.topkv_select_transport(E("x", 1, None), b, 0) == tk.TOPKV_ERR_INVALID_ARG
+    assert tk.topkv_select_transport(E(None, 1, "10.0.0.1"), a, 0) == tk.TOPKV_ERR_INVALID_ARG
+    # an instance without NVLink needs no domain
+    assert tk.topkv_select_transport(E(None, 0, "10.0.0.1"), a, 0) == tk.TOPKV_TRANSPORT_PCIE

@@ -82,13 +82,17 @@ def test_build_plan(dev):
 
 def _case(seed):
     """Random geometry, including strided pools, head-split rows, 16-byte-only alignment,
-    empty requests, full last pages and single tokens."""
+    1-byte and 2-byte elements, empty requests, full last pages and single tokens."""
     rng = np.random.default_rng(seed)
     F = int(rng.integers(1, 3))
     H = int(rng.choice([1, 2, 4, 8]))
     D = int(rng.choice([8, 24, 64, 72, 128, 576]))
     P = int(rng.choice([1, 3, 16, 64]))
-    E = 2
+    # element width b_p: 2 bytes (FP16 / bf16) or 1 byte (FP8), every pool style with both;
+    # a 1-byte head must still be a multiple of 16 bytes
+    E = 1 if (seed // 4) % 2 == 1 else 2
+    if E == 1 and D % 16:
+        D *= 2
     L = 2
     R = int(rng.integers(1, 7))
     sl = rng.integers(0, 4 * P + 2, size=R).astype(np.int32)
@@ -360,46 +364,162 @@ def _oracle_token(spec, page_host, t):
     return wire[t * spec.tok_bytes:(t + 1) * spec.tok_bytes]
 
 
-@pytest.mark.parametrize("name,full_layers", [("cfg2", (0, 17, 31)), ("cfg3", (0, 79)), ("cfg4", (0, 60))])
-def test_full_size_in_the_bench_launch_configuration(dev, name, full_layers):
+@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4"])
+def test_full_size_in_the_bench_launch_configuration(dev, name):
     """The workloads at full size, all layers resident, issued as bench.py issues them (one
-    stream, TOPKV_FLAG_OVERLAP_PREVIOUS after the first layer of each phase). A few layers are
-    compared in full with the oracle; in every layer sampled tokens are compared with what the
-    oracle computes for them one by one, on the wire and in the destination pool."""
+    stream, TOPKV_FLAG_OVERLAP_PREVIOUS after the first layer of each phase). EVERY layer's wire
+    slab and EVERY layer's destination slab (untouched bytes included) is compared in full with
+    the oracle; a few sampled tokens are also checked one by one through a one-page oracle
+    problem, which ties the batch-level comparison to the per-token definition."""
     spec = wl.ALL[name]
     w = harness.setup(spec, dev)
     b, s = w.batch, spec
     stream = torch.cuda.Stream(dev)
     g1 = _geom(s, b.num_pool_pages, 1, 0, 0)
-    dst_before = {l: harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, l) for l in full_layers}
+    dst_before = w.dst_pool.clone()                       # on the device: a host copy is 20 GiB
     for layer in range(s.L):
         w.pack(layer, stream, overlap=layer > 0)
     for layer in range(s.L):
         w.unpack(layer, stream, overlap=layer > 0)
     stream.synchronize()
-    for layer in full_layers:
+    assert tk.topkv_device_error_flags() == 0
+    for layer in range(s.L):
         src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, layer)
-        want = oracle.pack(g1, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=8)
+        want = oracle.pack(g1, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=16)
         got = w.wire[layer * w.n_layer:(layer + 1) * w.n_layer].cpu().numpy()
         assert np.array_equal(got, want), f"pack layer {layer}"
-        dst_h = dst_before[layer]
-        oracle.unpack(g1, 0, dst_h, b.dst_block_table, b.seq_lens, want, impl="rows", threads=8)
+        dst_h = harness.layer_slab_to_numpy(dst_before, w.slab_bytes, layer)
+        oracle.unpack(g1, 0, dst_h, b.dst_block_table, b.seq_lens, want, impl="rows", threads=16)
         assert np.array_equal(harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, layer), dst_h), \
             f"unpack layer {layer}"
     rng = np.random.default_rng(7)
     cu = np.concatenate([[0], np.cumsum(b.seq_lens.astype(np.int64))])
+    for layer in rng.choice(s.L, size=min(8, s.L), replace=False):
+        layer = int(layer)
+        r = int(rng.integers(0, s.R))
+        i = int(rng.integers(0, b.seq_lens[r]))
+        wo = layer * w.n_layer + (int(cu[r]) + i) * s.tok_bytes
+        got_wire = w.wire[wo:wo + s.tok_bytes].cpu().numpy()
+        for pool, table in ((w.src_pool, b.src_block_table), (w.dst_pool, b.dst_block_table)):
+            po = layer * w.slab_bytes + int(table[r, i // s.P]) * s.page_bytes
+            page_h = pool[po:po + s.page_bytes].cpu().numpy()
+            assert np.array_equal(_oracle_token(s, page_h, i % s.P), got_wire), (layer, r, i)
+    del w, dst_before
+    torch.cuda.empty_cache()
+
+
+def test_cfg3_host_leg_full_size(dev):
+    """Configuration 3 as stated: all 80 layers of the 70B-shaped cache packed to pinned host
+    memory over PCIe (staged form, one 128 MiB slab per layer, 10 GiB in all), then unpacked from
+    the host into the destination pool. Every pinned slab and every destination slab is
+    compared in full with the oracle."""
+    spec = wl.CFG3
+    w = harness.setup(spec, dev, need_wire=False)
+    b, s = w.batch, spec
+    g1 = _geom(s, b.num_pool_pages, 1, 0, 0)
+    try:
+        pinned = torch.empty(s.L * w.n_layer, dtype=torch.uint8).pin_memory()
+    except RuntimeError:
+        pytest.skip("this box refuses 10 GiB of pinned memory")
+    pinned.fill_(0x6B)
+    dst_before = w.dst_pool.clone()
+    staging = torch.empty(w.n_layer, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.Stream(dev)
+    stream.wait_stream(torch.cuda.current_stream(dev))
     for layer in range(s.L):
-        for _ in range(4):
-            r = int(rng.integers(0, s.R))
-            i = int(rng.integers(0, b.seq_lens[r]))
-            wo = layer * w.n_layer + (int(cu[r]) + i) * s.tok_bytes
-            got_wire = w.wire[wo:wo + s.tok_bytes].cpu().numpy()
-            for pool, table in ((w.src_pool, b.src_block_table), (w.dst_pool, b.dst_block_table)):
-                po = layer * w.slab_bytes + int(table[r, i // s.P]) * s.page_bytes
-                page_h = pool[po:po + s.page_bytes].cpu().numpy()
-                assert np.array_equal(_oracle_token(s, page_h, i % s.P), got_wire), (layer, r, i)
+        w.pack_to_host(layer, pinned, staging, stream)
+    for layer in range(s.L):
+        w.unpack_from_host(layer, pinned, staging, stream)
+    stream.synchronize()
+    assert tk.topkv_device_error_flags() == 0
+    host = pinned.numpy()
+    for layer in range(s.L):
+        src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, layer)
+        want = oracle.pack(g1, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=16)
+        assert np.array_equal(host[layer * w.n_layer:(layer + 1) * w.n_layer], want), f"to host, layer {layer}"
+        dst_h = harness.layer_slab_to_numpy(dst_before, w.slab_bytes, layer)
+        oracle.unpack(g1, 0, dst_h, b.dst_block_table, b.seq_lens, want, impl="rows", threads=16)
+        assert np.array_equal(harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, layer), dst_h), \
+            f"from host, layer {layer}"
+    del w, dst_before, pinned, staging
+    torch.cuda.empty_cache()
+
+
+def test_fp8_elements_bench_shape(dev):
+    """1-byte elements (b_p = 1 in Eq. 1) on the 70B batch: 8 x 128 x 1 = 1 KiB rows, 32 KiB
+    pages, two layers, compared in full with the oracle built with b_p = 1."""
+    from dataclasses import replace
+    spec = replace(wl.with_layers(wl.CFG3, 2), E=1, name="cfg3_fp8")
+    w = harness.setup(spec, dev, fill_dst=True)
+    assert w.layout.elem_bytes == 1 and w.n_layer == 8 * 4096 * 2 * 1024
+    stream = torch.cuda.Stream(dev)
+    stream.wait_stream(torch.cuda.current_stream(dev))
+    dst_before = [harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, l) for l in range(2)]
+    for layer in range(2):
+        w.pack(layer, stream, overlap=layer > 0)
+    for layer in range(2):
+        w.unpack(layer, stream, overlap=layer > 0)
+    stream.synchronize()
+    b = w.batch
+    g1 = _geom(spec, b.num_pool_pages, 1, 0, 0)
+    assert g1.b_p == 1 and g1.row_bytes == 1024
+    for layer in range(2):
+        src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, layer)
+        want = oracle.pack(g1, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=16)
+        assert np.array_equal(w.wire[layer * w.n_layer:(layer + 1) * w.n_layer].cpu().numpy(), want)
+        oracle.unpack(g1, 0, dst_before[layer], b.dst_block_table, b.seq_lens, want, impl="rows", threads=16)
+        assert np.array_equal(harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, layer), dst_before[layer])
     del w
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("pieces", [1, 16])
+def test_constant_state_layer_as_a_one_row_layout(dev, pieces):
+    """A linear-attention layer carries a fixed-size state per request instead of per-token
+    rows (§2.2). It goes through the same calls as a one-plane layout with one-token pages:
+    F = 1, H = 1, P = 1, and either the whole state slot as ONE page of `state` bytes
+    (pieces = 1) or the slot described as `pieces` consecutive pages of state / pieces bytes
+    (table row = slot * pieces + 0 .. pieces - 1), so that `pieces` CTAs share a large state.
+    The bytes shipped per request and layer are exactly the ("state", n) term of Eq. 1 per layer
+    kind, and they equal the oracle's pack of that geometry."""
+    rng = np.random.default_rng(31 + pieces)
+    state = 32 * 128 * 128 * 2                            # 32 heads of 128 x 128 bf16 = 1 MiB
+    L, R, slots = 3, 5, 9                                 # state layers, requests, pool slots
+    assert oracle.kv_bytes_layered(1, 1, 4096, [("state", state)] * L) == L * state
+    E = 2
+    g = Geom(L=L, F=1, h_kv=1, d_h=state // pieces // E, b_p=E, P=1, num_pages=slots * pieces)
+    assert g.S_page * pieces == state and g.S_layer == slots * state
+    sl = np.full(R, pieces, dtype=np.int32)               # every request has exactly one state
+    sub = np.arange(pieces, dtype=np.int32)[None, :]
+    slot_s = rng.permutation(slots)[:R].astype(np.int32).reshape(R, 1) * pieces + sub
+    slot_d = rng.permutation(slots)[:R].astype(np.int32).reshape(R, 1) * pieces + sub
+    T = int(sl.sum())
+    g.W_layer = g.wire_layer_bytes(T)
+    assert g.W_layer == R * state                         # R states per layer on the wire
+    lo = _layout_from_geom(g)
+    assert tk.topkv_kv_bytes_layered(lo, [(tk.TOPKV_LAYER_STATE, state)] * L, 4096) == L * state
+    assert tk.topkv_wire_layer_bytes(lo, T) == R * state
+    src_h = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
+    dst_h = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
+    src, dst = torch.from_numpy(src_h).to(dev), torch.from_numpy(dst_h).to(dev)
+    wire = torch.zeros(L * g.W_layer, dtype=torch.uint8, device=dev)
+    d_sl = torch.from_numpy(sl).to(dev)
+    bs = tk.make_batch(torch.from_numpy(slot_s).to(dev), d_sl, T)
+    bd = tk.make_batch(torch.from_numpy(slot_d).to(dev), d_sl, T)
+    want = np.zeros(L * g.W_layer, dtype=np.uint8)
+    for layer in range(L):
+        tk.check(tk.topkv_pack_layer(layer, src, lo, bs, wire, wire.numel()))
+        tk.check(tk.topkv_unpack_layer(layer, dst, lo, bd, wire, wire.numel()))
+        oracle.pack(g, layer, src_h, slot_s, sl, wire=want, impl="rows")
+        oracle.unpack(g, layer, dst_h, slot_d, sl, want, impl="rows")
+    torch.cuda.synchronize()
+    assert np.array_equal(wire.cpu().numpy(), want)
+    assert np.array_equal(dst.cpu().numpy(), dst_h)
+    # the wire is the requests' states in request order: the plain definition, written out
+    for layer in range(L):
+        for r in range(R):
+            a = layer * g.S_layer + int(slot_s[r, 0]) * g.S_page
+            assert np.array_equal(want[layer * g.W_layer + r * state:][:state], src_h[a:a + state])
 
 
 def test_overlapped_launches_keep_results_and_order(dev):
@@ -1194,9 +1314,9 @@ def test_side_stream_overlap_run_is_bit_exact(dev, variant):
 def test_cfg5_full_size_overlap_run(dev, variant):
     """The overlap workload at full size as bench.py runs it: 80 layers, 4 x 4096 tokens, the
     full-size GEMM stand-in on the main stream, every layer shipped to its own pinned slab by
-    the side stream (staged form, issued with topkv_pack_layers_to_host_pipelined). Three
-    layers are compared in full with the oracle's wire slab, and in every layer sampled tokens
-    with what the oracle computes for them one by one."""
+    the side stream (staged form, issued with topkv_pack_layers_to_host_pipelined). Every
+    layer's pinned slab is compared in full with the oracle's wire slab, and a few sampled
+    tokens with what the oracle computes for them one by one."""
     if variant == 1:
         pytest.skip("the overlap driver is kernel-family agnostic; run once")
     from paper_2607_28633_b200 import overlap
@@ -1213,14 +1333,14 @@ def test_cfg5_full_size_overlap_run(dev, variant):
     r = overlap.run_overlap(w, pinned, staging, pre)
     assert r.layers == 80 and r.hidden_upper_bound == pytest.approx(1 - 1 / 80)
     assert 0.0 <= r.exposed_ms and r.hidden <= 1.0
-    for layer in (0, 41, 79):
-        src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, layer)
-        want = oracle.pack(g, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=8)
-        assert np.array_equal(pinned[layer * w.n_layer:(layer + 1) * w.n_layer].numpy(), want), layer
-    rng = np.random.default_rng(8)
-    cu = np.concatenate([[0], np.cumsum(b.seq_lens.astype(np.int64))])
     host = pinned.numpy()
     for layer in range(s.L):
+        src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, layer)
+        want = oracle.pack(g, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=16)
+        assert np.array_equal(host[layer * w.n_layer:(layer + 1) * w.n_layer], want), layer
+    rng = np.random.default_rng(8)
+    cu = np.concatenate([[0], np.cumsum(b.seq_lens.astype(np.int64))])
+    for layer in (0, 37, 79):
         for _ in range(3):
             q = int(rng.integers(0, s.R))
             i = int(rng.integers(0, b.seq_lens[q]))
@@ -1331,6 +1451,8 @@ def test_many_layers_in_one_launch(dev, seed, variant):
     g, sl, bt_s, bt_d, rng = _case(seed)
     g.L = 3
     g.W_layer = max(g.W_layer, 16)                     # several layers need distinct slabs
+    if seed % 2:                                       # slab strides that are 16 mod 32: layer 1's
+        g.W_layer += 16 if g.W_layer % 32 == 0 else 0  # slabs are then only 16-byte aligned
     lo = _layout_from_geom(g)
     T = int(sl.sum())
     src_h = rng.integers(0, 256, g.L * g.S_layer, dtype=np.uint8)
@@ -1343,7 +1465,9 @@ def test_many_layers_in_one_launch(dev, seed, variant):
     know_T = seed % 2 == 0
     bs = tk.make_batch(d_bs, d_sl, T if know_T else -1)
     bd = tk.make_batch(d_bd, d_sl, T if know_T else -1)
-    first, count = 1, g.L - 1
+    first, count = (1, g.L - 1) if seed % 3 else (0, g.L)
+    if count > 1 and (g.W_layer % 32 or g.S_layer % 32):
+        assert tk.topkv_copy_vector_bytes(first, count, src, lo, bs, wire, wire.numel()) == 16
     tk.check(tk.topkv_pack_layers(first, count, src, lo, bs, wire, wire.numel()))
     want_wire = np.full(wire_len, 0x3C, dtype=np.uint8)
     want_dst = fill_h.copy()
@@ -1358,6 +1482,50 @@ def test_many_layers_in_one_launch(dev, seed, variant):
     assert np.array_equal(src.cpu().numpy(), src_h)
     assert tk.topkv_pack_layers(1, g.L, src, lo, bs, wire, wire.numel()) == tk.TOPKV_ERR_LAYER_RANGE
     assert tk.topkv_pack_layers(0, 0, src, lo, bs, wire, wire.numel()) == tk.TOPKV_OK
+
+
+def test_many_layers_in_one_launch_with_padded_slabs(dev, variant):
+    """32-byte aligned buffers and a first layer of 0, but layer strides that are 16 mod 32 (a
+    padded wire slab, a padded pool slab): every later layer's slab is only 16-byte aligned, so
+    the launch must use 16-byte accesses; bytes equal the oracle's."""
+    rng = np.random.default_rng(4242)
+    L, R, P = 4, 3, 16
+    sl = np.array([40, 16, 33], dtype=np.int32)
+    pages = (sl + P - 1) // P
+    npages = int(pages.sum()) + 2
+    for pad_wire, pad_pool in ((16, 0), (0, 16), (16, 16), (48, 80)):
+        g = Geom(L=L, F=2, h_kv=2, d_h=64, b_p=2, P=P, num_pages=npages)
+        g.S_layer += pad_pool
+        T = int(sl.sum())
+        g.W_layer = g.wire_layer_bytes(T) + pad_wire
+        assert g.wire_layer_bytes(T) % 32 == 0
+        bt_s = np.full((R, 3), -1, dtype=np.int32)
+        bt_d = np.full((R, 3), -1, dtype=np.int32)
+        ps, pd, pos = rng.permutation(npages), rng.permutation(npages), 0
+        for r in range(R):
+            bt_s[r, :pages[r]] = ps[pos:pos + pages[r]]
+            bt_d[r, :pages[r]] = pd[pos:pos + pages[r]]
+            pos += pages[r]
+        lo = _layout_from_geom(g)
+        src_h = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
+        dst_h = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
+        src, dst = torch.from_numpy(src_h).to(dev), torch.from_numpy(dst_h).to(dev)
+        wire = torch.full((L * g.W_layer,), 0x5C, dtype=torch.uint8, device=dev)
+        assert src.data_ptr() % 32 == 0 and dst.data_ptr() % 32 == 0 and wire.data_ptr() % 32 == 0
+        d_sl = torch.from_numpy(sl).to(dev)
+        bs = tk.make_batch(torch.from_numpy(bt_s).to(dev), d_sl, T)
+        bd = tk.make_batch(torch.from_numpy(bt_d).to(dev), d_sl, T)
+        assert tk.topkv_copy_vector_bytes(0, L, src, lo, bs, wire, wire.numel()) == 16
+        assert tk.topkv_copy_vector_bytes(0, 1, src, lo, bs, wire, wire.numel()) == 32
+        tk.check(tk.topkv_pack_layers(0, L, src, lo, bs, wire, wire.numel()))
+        tk.check(tk.topkv_unpack_layers(0, L, dst, lo, bd, wire, wire.numel()))
+        torch.cuda.synchronize()
+        want = np.full(L * g.W_layer, 0x5C, dtype=np.uint8)
+        for layer in range(L):
+            oracle.pack(g, layer, src_h, bt_s, sl, wire=want)
+            oracle.unpack(g, layer, dst_h, bt_d, sl, want)
+        assert np.array_equal(wire.cpu().numpy(), want), (pad_wire, pad_pool)
+        assert np.array_equal(dst.cpu().numpy(), dst_h), (pad_wire, pad_pool)
 
 
 def test_many_layers_in_one_launch_cfg1(dev, variant):
