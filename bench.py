@@ -165,6 +165,7 @@ def oracle_sample(spec, batch, seconds_target=12.0, threads=None, impl="rows"):
     import oracle
     from paper_2607_28633_b200 import workloads as wl
     cores = host_cores() if threads is None else threads
+    cores = max(1, min(cores, spec.R))   # the rows form splits by request: the threads it really uses
     g = oracle.Geom(L=1, F=spec.F, h_kv=spec.H, d_h=spec.D, b_p=spec.E, P=spec.P,
                     num_pages=batch.num_pool_pages)
     src = wl.fill_numpy(g.pool_bytes(), batch.seeds["data"], raw_bits=True)
@@ -539,24 +540,34 @@ def device_copy_baseline(dev, stream, nbytes, reps=10):
     return 2 * nbytes / (best * 1e-3) / 1e9
 
 
-def bench_chain(w, stream, steps, flags=0):
-    """The dependent order of a relay without a host hop: for every layer, pack into ONE shared
-    wire slab, then unpack that slab, so that every kernel depends on the data of the kernel
-    just before it and no launch may be declared independent. GB/s of read + write traffic."""
+def bench_chain(w, stream, steps, unpack_flags=0, slabs=1):
+    """The dependent order of a relay without a host hop: pack(l), unpack(l), pack(l+1), ...
+    where every unpack needs the slab that the pack just before it wrote, so an unpack can never
+    be declared independent. With ``slabs`` = 1 all layers go through ONE wire slab, so pack(l+1)
+    also has to wait for unpack(l) to have read it and no launch may overlap its predecessor.
+    With 2 slabs the layers alternate between them: pack(l+1) then touches nothing that
+    unpack(l) or pack(l) touch and carries TOPKV_FLAG_OVERLAP_PREVIOUS within the flag's
+    contract, while every unpack still waits for its pack. GB/s of read + write traffic, and
+    microseconds per launch."""
     import ctypes
     import torch
     from paper_2607_28633_b200 import binding as tk
     lo = type(w.layout)()
     ctypes.memmove(ctypes.byref(lo), ctypes.byref(w.layout), ctypes.sizeof(lo))
     lo.wire_layer_stride = 0
-    slab = w.wire[:w.n_layer]
-    bs = tk.make_batch(w.src_bt, w.seq_lens, w.batch.total_tokens, w.cu, flags)
-    bd = tk.make_batch(w.dst_bt, w.seq_lens, w.batch.total_tokens, w.cu, flags)
+    n = w.n_layer
+    slab = [w.wire[k * n:(k + 1) * n] for k in range(slabs)]
+    T = w.batch.total_tokens
+    ov = tk.TOPKV_FLAG_OVERLAP_PREVIOUS if slabs > 1 else 0
+    bs0 = tk.make_batch(w.src_bt, w.seq_lens, T, w.cu, 0)
+    bs = tk.make_batch(w.src_bt, w.seq_lens, T, w.cu, ov)
+    bd = tk.make_batch(w.dst_bt, w.seq_lens, T, w.cu, unpack_flags)
 
     def run():
         for l in range(w.layers):
-            tk.check(tk.topkv_pack_layer(l, w.src_pool, lo, bs, slab, w.n_layer, stream))
-            tk.check(tk.topkv_unpack_layer(l, w.dst_pool, lo, bd, slab, w.n_layer, stream))
+            q = slab[l % slabs]
+            tk.check(tk.topkv_pack_layer(l, w.src_pool, lo, bs if l else bs0, q, n, stream))
+            tk.check(tk.topkv_unpack_layer(l, w.dst_pool, lo, bd, q, n, stream))
     run()
     stream.synchronize()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -690,16 +701,19 @@ def run_extra(name, dev, stream, args, peak):
         out["frac_of_hbm_peak"] = out[wl.CFG2.name]["frac_of_hbm_peak"]
         return out
     if name == "chain":
-        # pack(l) -> unpack(l) per layer through one shared slab: every launch depends on the one
-        # before it (the order of a device-to-device relay), so TOPKV_FLAG_OVERLAP_PREVIOUS is
-        # not available; plain launches and TOPKV_FLAG_TABLES_SETTLED
+        # pack(l) -> unpack(l) per layer, the order of a device-to-device relay: every unpack
+        # depends on the pack before it. One shared slab (nothing may overlap) or two alternating
+        # slabs (pack(l+1) is independent of unpack(l) and says so); unpack plain or with
+        # TOPKV_FLAG_TABLES_SETTLED
         out = {"workload": "cfg2_llama3_8b, cfg4_dsv3_mla", "order": "pack(l), unpack(l), pack(l+1), ..."}
         for base in (wl.CFG2, wl.CFG4):
             spec = base if args.layers is None else wl.with_layers(base, args.layers)
             w = harness.setup(spec, dev, fill_dst=False)
             r = {}
-            for label, flags in (("plain", 0), ("tables_settled", tk.TOPKV_FLAG_TABLES_SETTLED)):
-                gbs, us = bench_chain(w, stream, max(1, min(args.steps, 5)), flags)
+            ts = tk.TOPKV_FLAG_TABLES_SETTLED
+            for label, flags, slabs in (("one_slab_plain", 0, 1), ("one_slab_tables_settled", ts, 1),
+                                        ("two_slabs_plain", 0, 2), ("two_slabs_tables_settled", ts, 2)):
+                gbs, us = bench_chain(w, stream, max(1, min(args.steps, 5)), flags, slabs)
                 r[label] = {"GBps": round(gbs, 1), "us_per_launch": round(us, 2),
                             "frac_of_hbm_peak": round(gbs / peak, 4),
                             "frac_of_8000_spec": round(gbs / 8000.0, 4)}
@@ -811,6 +825,8 @@ def main():
                     help="comma list of extra workloads measured at one GPU ('' for none)")
     ap.add_argument("--variant", type=int, default=None, help="kernel family (see topkv.h)")
     ap.add_argument("--layers", type=int, default=None, help="fewer layers (profiling only)")
+    ap.add_argument("--workload", default=None, choices=["cfg2", "cfg3", "cfg4"],
+                    help="time another benchmark shape in place of the headline one (profiling only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -866,7 +882,7 @@ def main():
         return dist_util.sum_over_ranks(dist, x, dev)
 
     peak, peak_src = measured_peak_gbs()
-    head = HEADLINE(wl)
+    head = HEADLINE(wl) if args.workload is None else wl.ALL[args.workload]
     spec = head if args.layers is None else wl.with_layers(head, args.layers)
     w = harness.setup(spec, dev, rank=rank, fill_dst=False)
     stream = torch.cuda.Stream(dev)
