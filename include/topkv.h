@@ -407,6 +407,82 @@ typedef struct topkv_layer_spec {
 int64_t topkv_kv_bytes_layered(const topkv_layout* layout, const topkv_layer_spec* specs,
                                int64_t seq_len);
 
+/* ---- a model whose layers differ in kind, on the data path (§2.2) ---------------------------
+ * Hybrid models mix layer kinds: full-attention layers cache every token, windowed layers only
+ * the last W, linear-attention layers a fixed-size state per request. A layer table describes
+ * such a model to the data path, one topkv_layer_spec per MODEL layer, so that the range calls
+ * and the side-stream schedule of §5.2 can run it:
+ *   FULL, WINDOW  live in the paged pool and share the batch's block table. They are numbered
+ *                 among themselves in model order: the a-th attention layer of the model is
+ *                 layer a of the pool (layout->num_layers counts attention layers only). A
+ *                 WINDOW layer ships the last min(s_r, param) tokens of every request.
+ *   STATE         one state of `param` bytes per request, in a pool of slots: the state of
+ *                 request r in the j-th STATE layer of the model (numbered among themselves)
+ *                 starts at state_pool + j*state_layer_stride + state_slots[r]*state_slot_stride.
+ *                 param, both strides and the pool base must be multiples of 16 bytes.
+ * The wire holds the layers' slabs back to back in model order (the order in which they are
+ * sent): an attention layer's slab is exactly what topkv_pack_layer produces for that layer
+ * with that window (wire order as in the layout), a STATE layer's slab the R states in request
+ * order. Slab l starts at h_offsets[l] of topkv_layer_table_offsets; the total,
+ * h_offsets[num_layers], is Eq. 1 per layer kind summed over the requests.
+ * Rules: batch->window_tokens must be 0 (the table decides per layer); batch->cu_seq_lens, when
+ * given, serves the FULL layers, WINDOW layers derive their prefix sums in the kernel, so a
+ * model with WINDOW layers needs num_requests <= TOPKV_MAX_INLINE_R; h_seq_lens must hold the
+ * values of batch->seq_lens (if batch->total_tokens is given it must equal their sum). */
+typedef struct topkv_layer_table {
+  uint32_t struct_size;           /* = sizeof(topkv_layer_table)                                */
+  uint32_t num_layers;            /* layers of the model, every kind                            */
+  const topkv_layer_spec* specs;  /* HOST [num_layers]                                          */
+  const int32_t* h_seq_lens;      /* HOST int32 [R]: the lengths, to size every slab on the host */
+  void* state_pool;               /* DEVICE: slots of the STATE layers; NULL if there are none  */
+  const int32_t* state_slots;     /* DEVICE int32 [R]: slot of request r                        */
+  int64_t state_layer_stride;     /* bytes from one STATE layer's slots to the next one's       */
+  int64_t state_slot_stride;      /* bytes between two slots (>= the largest state)             */
+  int64_t num_state_slots;        /* every slot id is checked against it on the device          */
+} topkv_layer_table;
+
+/* h_offsets: HOST int64 [table->num_layers + 1]. */
+int topkv_layer_table_offsets(const topkv_layout* layout, const topkv_layer_table* table,
+                              int32_t num_requests, int64_t* h_offsets);
+
+/* Model layers first_layer .. first_layer + num_layers - 1 between the pools and the wire buffer
+ * behind d_wire (slab l at d_wire + h_offsets[l]), device to device, one kernel per layer on
+ * `stream`. The layers of one call touch different slabs and different pool layers, so every
+ * launch after the first is allowed to overlap its predecessor; batch->flags applies to the
+ * first. Everything is validated for every layer before anything is launched. For unpack,
+ * `dst_pool` and table->state_pool are the destination pools, batch->block_table and
+ * table->state_slots the destination's tables. */
+int topkv_pack_model_layers(int first_layer, int num_layers, const void* src_pool,
+                            const topkv_layout* layout, const topkv_batch* batch,
+                            const topkv_layer_table* table, void* d_wire,
+                            int64_t wire_capacity_bytes, topkv_stream_t stream);
+int topkv_unpack_model_layers(int first_layer, int num_layers, void* dst_pool,
+                              const topkv_layout* layout, const topkv_batch* batch,
+                              const topkv_layer_table* table, const void* d_wire,
+                              int64_t wire_bytes, topkv_stream_t stream);
+
+/* The layer-by-layer side-stream schedule (see topkv_pack_layers_to_host_pipelined) for such a
+ * model: per model layer, wait for layer_ready[i], ship the layer's slab to (from) h_pinned +
+ * h_offsets[l] over PCIe, record layer_done[i]. d_staging != NULL: staged form, the slab must
+ * hold the largest slab of the range; NULL: direct form. Errors as for the plain pipelined
+ * calls. */
+int topkv_pack_model_layers_to_host_pipelined(int first_layer, int num_layers, const void* src_pool,
+                                              const topkv_layout* layout, const topkv_batch* batch,
+                                              const topkv_layer_table* table, void* h_pinned,
+                                              int64_t host_capacity_bytes, void* d_staging,
+                                              int64_t staging_capacity_bytes,
+                                              const topkv_event_t* layer_ready,
+                                              const topkv_event_t* layer_done,
+                                              topkv_stream_t side_stream);
+int topkv_unpack_model_layers_from_host_pipelined(int first_layer, int num_layers, void* dst_pool,
+                                                  const topkv_layout* layout, const topkv_batch* batch,
+                                                  const topkv_layer_table* table, const void* h_pinned,
+                                                  int64_t host_bytes, void* d_staging,
+                                                  int64_t staging_capacity_bytes,
+                                                  const topkv_event_t* layer_ready,
+                                                  const topkv_event_t* layer_done,
+                                                  topkv_stream_t side_stream);
+
 /* ---- CPU-side analytic helpers (context only; no GPU work) ------------------------------- */
 
 /* Eq. 2: bytes / bandwidth + setup latency, in seconds. */

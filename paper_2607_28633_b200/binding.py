@@ -46,7 +46,9 @@ EXPORTS = (
     "topkv_set_host_leg_ctas", "topkv_pack_layers_to_host_pipelined",
     "topkv_unpack_layers_from_host_pipelined", "topkv_pack_layers", "topkv_unpack_layers",
     "topkv_copy_vector_bytes", "topkv_select_transport", "topkv_planning_rate",
-    "topkv_transport_name",
+    "topkv_transport_name", "topkv_layer_table_offsets", "topkv_pack_model_layers",
+    "topkv_unpack_model_layers", "topkv_pack_model_layers_to_host_pipelined",
+    "topkv_unpack_model_layers_from_host_pipelined",
 )
 
 
@@ -76,6 +78,35 @@ class topkv_layer_spec(ctypes.Structure):
 
 
 TOPKV_LAYER_FULL, TOPKV_LAYER_WINDOW, TOPKV_LAYER_STATE = 0, 1, 2
+
+
+class topkv_layer_table(ctypes.Structure):
+    _fields_ = [("struct_size", c_uint32), ("num_layers", c_uint32), ("specs", c_void_p),
+                ("h_seq_lens", c_void_p), ("state_pool", c_void_p), ("state_slots", c_void_p),
+                ("state_layer_stride", c_int64), ("state_slot_stride", c_int64),
+                ("num_state_slots", c_int64)]
+
+
+def make_layer_table(specs, h_seq_lens, state_pool=None, state_slots=None, state_layer_stride=0,
+                     state_slot_stride=0, num_state_slots=0) -> topkv_layer_table:
+    """specs: sequence of (kind, param) per model layer; h_seq_lens: numpy int32 [R] on the host;
+    state_pool / state_slots: device tensors (or None). The table keeps what it points to alive."""
+    import numpy as np
+    arr = (topkv_layer_spec * len(specs))()
+    for i, (kind, param) in enumerate(specs):
+        arr[i].kind, arr[i].param = kind, param
+    lens = np.ascontiguousarray(h_seq_lens, dtype=np.int32)
+    t = topkv_layer_table()
+    t.struct_size = ctypes.sizeof(topkv_layer_table)
+    t.num_layers = len(specs)
+    t.specs = ctypes.addressof(arr)
+    t.h_seq_lens = lens.ctypes.data
+    t.state_pool = _ptr(state_pool)
+    t.state_slots = _ptr(state_slots)
+    t.state_layer_stride, t.state_slot_stride = state_layer_stride, state_slot_stride
+    t.num_state_slots = num_state_slots
+    t._keepalive = (arr, lens, state_pool, state_slots)
+    return t
 TOPKV_TRANSPORT_NVLINK, TOPKV_TRANSPORT_PCIE, TOPKV_TRANSPORT_RDMA, TOPKV_TRANSPORT_TCP = 1, 2, 3, 4
 
 
@@ -174,6 +205,14 @@ def lib() -> ctypes.CDLL:
         L.topkv_set_host_leg_ctas.argtypes = [c_int]
         L.topkv_pack_layers.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p]
         L.topkv_unpack_layers.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p]
+        tp = ctypes.POINTER(topkv_layer_table)
+        L.topkv_layer_table_offsets.argtypes = [lp, tp, c_int32, c_void_p]
+        L.topkv_pack_model_layers.argtypes = [c_int, c_int, c_void_p, lp, bp, tp, c_void_p, c_int64, c_void_p]
+        L.topkv_unpack_model_layers.argtypes = [c_int, c_int, c_void_p, lp, bp, tp, c_void_p, c_int64, c_void_p]
+        for fn in (L.topkv_pack_model_layers_to_host_pipelined,
+                   L.topkv_unpack_model_layers_from_host_pipelined):
+            fn.argtypes = [c_int, c_int, c_void_p, lp, bp, tp, c_void_p, c_int64, c_void_p, c_int64,
+                           c_void_p, c_void_p, c_void_p]
         ep = ctypes.POINTER(topkv_endpoint)
         L.topkv_select_transport.argtypes = [ep, ep, c_int, c_int]
         L.topkv_planning_rate.argtypes = [c_int]
@@ -329,6 +368,49 @@ def topkv_unpack_layers_from_host_pipelined(first_layer, num_layers, dst_pool, l
     return lib().topkv_unpack_layers_from_host_pipelined(
         first_layer, num_layers, _ptr(dst_pool), ctypes.byref(layout), ctypes.byref(batch),
         _ptr(h_pinned), host_bytes, _ptr(d_staging), staging_capacity_bytes,
+        _events(layer_ready, num_layers), _events(layer_done, num_layers), _stream(side_stream))
+
+
+def topkv_layer_table_offsets(layout, table, num_requests):
+    """Returns (status, offsets) with offsets a numpy int64 [num_layers + 1]."""
+    import numpy as np
+    off = np.zeros(table.num_layers + 1, dtype=np.int64)
+    st = lib().topkv_layer_table_offsets(ctypes.byref(layout), ctypes.byref(table), num_requests,
+                                         off.ctypes.data)
+    return st, off
+
+
+def topkv_pack_model_layers(first_layer, num_layers, src_pool, layout, batch, table, d_wire,
+                            wire_capacity_bytes, stream=None):
+    return lib().topkv_pack_model_layers(first_layer, num_layers, _ptr(src_pool), ctypes.byref(layout),
+                                         ctypes.byref(batch), ctypes.byref(table), _ptr(d_wire),
+                                         wire_capacity_bytes, _stream(stream))
+
+
+def topkv_unpack_model_layers(first_layer, num_layers, dst_pool, layout, batch, table, d_wire,
+                              wire_bytes, stream=None):
+    return lib().topkv_unpack_model_layers(first_layer, num_layers, _ptr(dst_pool), ctypes.byref(layout),
+                                           ctypes.byref(batch), ctypes.byref(table), _ptr(d_wire),
+                                           wire_bytes, _stream(stream))
+
+
+def topkv_pack_model_layers_to_host_pipelined(first_layer, num_layers, src_pool, layout, batch, table,
+                                              h_pinned, host_capacity_bytes, d_staging,
+                                              staging_capacity_bytes, layer_ready=None, layer_done=None,
+                                              side_stream=None):
+    return lib().topkv_pack_model_layers_to_host_pipelined(
+        first_layer, num_layers, _ptr(src_pool), ctypes.byref(layout), ctypes.byref(batch),
+        ctypes.byref(table), _ptr(h_pinned), host_capacity_bytes, _ptr(d_staging), staging_capacity_bytes,
+        _events(layer_ready, num_layers), _events(layer_done, num_layers), _stream(side_stream))
+
+
+def topkv_unpack_model_layers_from_host_pipelined(first_layer, num_layers, dst_pool, layout, batch, table,
+                                                  h_pinned, host_bytes, d_staging,
+                                                  staging_capacity_bytes, layer_ready=None,
+                                                  layer_done=None, side_stream=None):
+    return lib().topkv_unpack_model_layers_from_host_pipelined(
+        first_layer, num_layers, _ptr(dst_pool), ctypes.byref(layout), ctypes.byref(batch),
+        ctypes.byref(table), _ptr(h_pinned), host_bytes, _ptr(d_staging), staging_capacity_bytes,
         _events(layer_ready, num_layers), _events(layer_done, num_layers), _stream(side_stream))
 
 

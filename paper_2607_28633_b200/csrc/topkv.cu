@@ -149,6 +149,9 @@ int prepare(int layer, const void* pool, const topkv_layout* lo, const topkv_bat
   kp->late_wait = (!kp->overlap && (b->flags & TOPKV_FLAG_TABLES_SETTLED)) ? 1 : 0;
   kp->ppc = 1;
   kp->spr = kp->maxp;
+  kp->cpp = 1;
+  kp->tps = 0;
+  kp->const_len = 0;
   kp->window = b->window_tokens;
   kp->num_pages = lo->num_pool_pages;
   kp->wire_limit = (n_layer >= 0 && !spread) ? n_layer : capacity - (int64_t)layer * wire_layer_stride;
@@ -222,7 +225,7 @@ int bulk_prepare_device(int* sms_out) {
 template <bool PACK>
 int launch_bulk(const KParams& kp0, const Resolved& rs, int F, cudaStream_t stream, bool* handled) {
   *handled = false;
-  if (kp0.R > kBulkMaxR || kp0.window > 0) return TOPKV_OK;
+  if (kp0.R > kBulkMaxR || kp0.window > 0 || kp0.const_len > 0) return TOPKV_OK;
   if ((int64_t)kp0.R * kp0.maxp * kp0.P > 0x7fffffffll) return TOPKV_OK;  // its prefix sums are int32
   const int64_t tok_bytes = (int64_t)F * rs.row_bytes;
   if (tok_bytes > kStageTarget || rs.unit_bytes > 0x7fffffff) return TOPKV_OK;
@@ -280,6 +283,19 @@ int launch_copy(KParams kp, const Resolved& rs, int F, cudaStream_t stream, int 
     kp.ppc = (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(kMaxPagesPerCta, kp.maxp),
                                                         kSpanTargetBytes / page_bytes));
     kp.spr = (kp.maxp + kp.ppc - 1) / kp.ppc;
+    kp.cpp = 1;
+    kp.tps = 0;
+    if (page_bytes >= 2 * kSpanTargetBytes && kp.P > 1) {  // huge pages: several CTAs per page
+      const int64_t tok_bytes = (int64_t)F * rs.row_bytes;
+      kp.tps = (int)std::max<int64_t>(1, std::min<int64_t>(kp.P, kSpanTargetBytes / tok_bytes));
+      kp.cpp = (kp.P + kp.tps - 1) / kp.tps;
+      if ((int64_t)kp.maxp * kp.cpp > 0x7fffffffll / std::max(1, kp.R)) {  // keep R * spr an int
+        kp.cpp = 1;
+        kp.tps = 0;
+      } else if (kp.cpp > 1) {
+        kp.spr = kp.maxp * kp.cpp;
+      }
+    }
     const int64_t spans = (int64_t)kp.R * kp.spr;
     const bool walk = max_ctas > 0 && spans > max_ctas;
     const dim3 grid((unsigned)(walk ? max_ctas : spans), (unsigned)layers);
@@ -643,6 +659,256 @@ int copy_layers(int first_layer, int num_layers, const void* pool, const topkv_l
 }
 
 }  // namespace multi
+
+// ---- a model whose layers differ in kind (§2.2) -------------------------------------------------
+namespace model {
+
+struct LayerPlan {
+  KParams kp;
+  Resolved rs;
+  int F = 0;
+  int64_t offset = 0;   // where the layer's slab starts in the wire buffer
+  int64_t n_slab = 0;   // its size in bytes
+  bool empty = false;   // nothing to launch
+};
+
+int check_table(const topkv_layout* lo, const topkv_batch* b, const topkv_layer_table* t) {
+  if (t == nullptr || t->struct_size != sizeof(topkv_layer_table) || t->specs == nullptr)
+    return TOPKV_ERR_INVALID_ARG;
+  if (lo == nullptr || b == nullptr) return TOPKV_ERR_INVALID_ARG;
+  if (b->struct_size != sizeof(topkv_batch) || b->window_tokens != 0) return TOPKV_ERR_INVALID_ARG;
+  if (b->num_requests > 0 && t->h_seq_lens == nullptr) return TOPKV_ERR_INVALID_ARG;
+  return TOPKV_OK;
+}
+
+// Tokens of the batch that a layer of this kind keeps, from the host copy of the lengths.
+int64_t kept_tokens(const topkv_layer_table* t, int R, const topkv_layer_spec& sp) {
+  int64_t total = 0;
+  for (int r = 0; r < R; ++r) {
+    const int64_t s = t->h_seq_lens[r];
+    total += (sp.kind == TOPKV_LAYER_WINDOW && sp.param < s) ? sp.param : s;
+  }
+  return total;
+}
+
+int slab_bytes(const topkv_layout* lo, const topkv_layer_table* t, int R, uint32_t l, int64_t* out) {
+  const topkv_layer_spec& sp = t->specs[l];
+  if (sp.reserved != 0 || sp.param < 0) return TOPKV_ERR_INVALID_ARG;
+  const int64_t tok_bytes = (int64_t)lo->kv_factor * lo->num_kv_heads * lo->head_dim * lo->elem_bytes;
+  switch (sp.kind) {
+    case TOPKV_LAYER_FULL:
+    case TOPKV_LAYER_WINDOW: *out = tok_bytes * kept_tokens(t, R, sp); return TOPKV_OK;
+    case TOPKV_LAYER_STATE: *out = (int64_t)R * sp.param; return TOPKV_OK;
+    default: return TOPKV_ERR_INVALID_ARG;
+  }
+}
+
+// Plans model layer l: validates it and fills the kernel parameters, exactly as the per-layer
+// calls would for the view this layer has of the pools. `wire_base` / `capacity` describe the
+// whole wire buffer (device, or pinned host); `offset` is the layer's place in it.
+int plan_layer(uint32_t l, const void* pool, const topkv_layout* lo, const topkv_batch* b,
+               const topkv_layer_table* t, const void* wire_base, int64_t capacity, int64_t offset,
+               uint32_t flags, LayerPlan* out) {
+  const int R = b->num_requests;
+  const topkv_layer_spec& sp = t->specs[l];
+  int st = slab_bytes(lo, t, R, l, &out->n_slab);
+  if (st != TOPKV_OK) return st;
+  out->offset = offset;
+  if (wire_base == nullptr || capacity < 0) return TOPKV_ERR_INVALID_ARG;
+  if (offset + out->n_slab > capacity) return TOPKV_ERR_CAPACITY;
+  uint32_t ord = 0;  // this layer's number among the layers of its own pool
+  for (uint32_t q = 0; q < l; ++q)
+    ord += (t->specs[q].kind == TOPKV_LAYER_STATE) == (sp.kind == TOPKV_LAYER_STATE) ? 1u : 0u;
+  const uint8_t* slab = static_cast<const uint8_t*>(wire_base) + offset;
+  if (sp.kind != TOPKV_LAYER_STATE) {
+    topkv_layout lo2 = *lo;
+    lo2.wire_layer_stride = 0;  // the slab is addressed directly
+    topkv_batch b2 = *b;
+    b2.flags = flags;
+    b2.window_tokens = sp.kind == TOPKV_LAYER_WINDOW ? (int32_t)std::min<int64_t>(sp.param, 0x7fffffff) : 0;
+    if (sp.kind == TOPKV_LAYER_WINDOW && sp.param == 0) return TOPKV_ERR_INVALID_ARG;  // a window of no tokens
+    b2.total_tokens = R > 0 ? kept_tokens(t, R, sp) : 0;
+    if (b2.window_tokens != 0) b2.cu_seq_lens = nullptr;  // the plan's prefix sums count whole sequences
+    if (b->total_tokens >= 0 && R > 0) {                  // the two descriptions of the batch must agree
+      topkv_layer_spec full = {TOPKV_LAYER_FULL, 0, 0};
+      if (kept_tokens(t, R, full) != b->total_tokens) return TOPKV_ERR_INVALID_ARG;
+    }
+    int64_t n_layer = 0;
+    st = prepare((int)ord, pool, &lo2, &b2, slab, capacity - offset, 0, &out->kp, &out->rs, &n_layer);
+    if (st != TOPKV_OK) return st;
+    out->F = (int)lo->kv_factor;
+    out->empty = (int64_t)out->kp.R * out->kp.maxp == 0;
+    return TOPKV_OK;
+  }
+  // a constant-state layer: R states of sp.param bytes, one slot each, shipped in request order.
+  // The copy kernel sees the slot as one page of `k` rows, every request having exactly k tokens.
+  const int64_t B = sp.param;
+  out->F = 1;
+  out->empty = R == 0 || B == 0;
+  if (out->empty) return TOPKV_OK;
+  if (t->state_pool == nullptr || t->state_slots == nullptr || t->num_state_slots <= 0)
+    return TOPKV_ERR_INVALID_ARG;
+  if (t->state_slot_stride < B || t->state_layer_stride <= 0) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  if (!mult16(B) || !mult16(t->state_slot_stride) || !mult16(t->state_layer_stride) ||
+      !mult16p(t->state_pool) || !mult16p(slab))
+    return TOPKV_ERR_ALIGNMENT;
+  int64_t row = 4096;  // the largest power of two up to 4 KiB that divides the state
+  while (B % row) row >>= 1;
+  const int64_t k = B / row;
+  if (k * (int64_t)R > 0x7fffffffll) return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  KParams& kp = out->kp;
+  kp = KParams{};
+  kp.pool = static_cast<uint8_t*>(t->state_pool) + (int64_t)ord * t->state_layer_stride;
+  kp.wire = const_cast<uint8_t*>(slab);
+  kp.bt = t->state_slots;  // [R][1]: the slot is the request's only "page"
+  kp.sl = nullptr;
+  kp.cu = nullptr;
+  kp.T = (int64_t)R * k;
+  kp.S_page = t->state_slot_stride;
+  kp.S_kv = 0;
+  kp.S_tok = row;
+  kp.S_unit = 0;
+  kp.R = R;
+  kp.maxp = 1;
+  kp.P = (int)k;
+  kp.U = 1;
+  kp.unit_chunks = (int)(row / 16);
+  kp.planar = 0;
+  kp.plane_rows = -1;
+  kp.window = 0;
+  kp.ppc = 1;
+  kp.spr = 1;
+  kp.cpp = 1;
+  kp.tps = 0;
+  kp.const_len = (int)k;
+  kp.num_pages = t->num_state_slots;
+  kp.wire_limit = out->n_slab;
+  kp.overlap = (flags & TOPKV_FLAG_OVERLAP_PREVIOUS) ? 1 : 0;
+  kp.late_wait = (!kp.overlap && (flags & TOPKV_FLAG_TABLES_SETTLED)) ? 1 : 0;
+  kp.S_layer = 0;
+  kp.W_layer = 0;
+  out->rs.row_bytes = row;
+  out->rs.unit_bytes = row;
+  out->rs.U = 1;
+  out->rs.merged = true;
+  return TOPKV_OK;
+}
+
+int check_range(const topkv_layer_table* t, int first_layer, int num_layers) {
+  if (first_layer < 0 || num_layers < 0 || (int64_t)first_layer + num_layers > (int64_t)t->num_layers)
+    return TOPKV_ERR_LAYER_RANGE;
+  return TOPKV_OK;
+}
+
+// Offset of layer `first` and, through `visit`, every layer of the range with its offset.
+template <typename Visit>
+int for_layers(int first_layer, int num_layers, const topkv_layout* lo, const topkv_batch* b,
+               const topkv_layer_table* t, Visit visit) {
+  int64_t off = 0;
+  for (uint32_t l = 0; l < (uint32_t)(first_layer + num_layers); ++l) {
+    int64_t n = 0;
+    const int st = slab_bytes(lo, t, b->num_requests, l, &n);
+    if (st != TOPKV_OK) return st;
+    if (l >= (uint32_t)first_layer) {
+      const int sv = visit(l, off);
+      if (sv != TOPKV_OK) return sv;
+    }
+    off += n;
+  }
+  return TOPKV_OK;
+}
+
+// Device to device: one launch per layer; the layers of one call touch different slabs and
+// different pool layers, so every launch after the first may overlap its predecessor.
+template <bool PACK>
+int copy_layers(int first_layer, int num_layers, const void* pool, const topkv_layout* lo,
+                const topkv_batch* b, const topkv_layer_table* t, const void* d_wire, int64_t wire_bytes,
+                cudaStream_t s) {
+  int st = check_table(lo, b, t);
+  if (st != TOPKV_OK) return st;
+  st = check_range(t, first_layer, num_layers);
+  if (st != TOPKV_OK) return st;
+  LayerPlan lp;
+  st = for_layers(first_layer, num_layers, lo, b, t, [&](uint32_t l, int64_t off) {  // validate all first
+    return plan_layer(l, pool, lo, b, t, d_wire, wire_bytes, off, b->flags, &lp);
+  });
+  if (st != TOPKV_OK) return st;
+  bool launched = false;
+  return for_layers(first_layer, num_layers, lo, b, t, [&](uint32_t l, int64_t off) {
+    const uint32_t flags = launched ? (b->flags | TOPKV_FLAG_OVERLAP_PREVIOUS) : b->flags;
+    int sv = plan_layer(l, pool, lo, b, t, d_wire, wire_bytes, off, flags, &lp);
+    if (sv != TOPKV_OK || lp.empty) return sv;
+    sv = launch_copy<PACK>(lp.kp, lp.rs, lp.F, s);
+    launched = launched || sv == TOPKV_OK;
+    return sv;
+  });
+}
+
+// The side-stream schedule of §5.2 for such a model: per layer wait, ship over PCIe, record.
+template <bool PACK>
+int issue_layers(int first_layer, int num_layers, const void* pool, const topkv_layout* lo,
+                 const topkv_batch* b, const topkv_layer_table* t, const void* h_pinned, int64_t host_bytes,
+                 void* d_staging, int64_t staging_capacity_bytes, const topkv_event_t* layer_ready,
+                 const topkv_event_t* layer_done, cudaStream_t s) {
+  int st = check_table(lo, b, t);
+  if (st != TOPKV_OK) return st;
+  st = check_range(t, first_layer, num_layers);
+  if (st != TOPKV_OK) return st;
+  if (h_pinned == nullptr) return TOPKV_ERR_INVALID_ARG;
+  if (d_staging != nullptr && !mult16p(d_staging)) return TOPKV_ERR_ALIGNMENT;
+  LayerPlan lp;
+  st = for_layers(first_layer, num_layers, lo, b, t, [&](uint32_t l, int64_t off) {  // validate all first
+    const int sv = plan_layer(l, pool, lo, b, t, h_pinned, host_bytes, off, b->flags, &lp);
+    if (sv != TOPKV_OK) return sv;
+    if (d_staging != nullptr && staging_capacity_bytes < lp.n_slab) return (int)TOPKV_ERR_CAPACITY;
+    return (int)TOPKV_OK;
+  });
+  if (st != TOPKV_OK) return st;
+  uint8_t* dev_view = nullptr;  // the pinned buffer as the GPU sees it (direct form)
+  if (d_staging == nullptr && num_layers > 0) {
+    void* dev = nullptr;
+    st = mapped_device_pointer(h_pinned, &dev);  // refuses pageable memory before anything is enqueued
+    if (st != TOPKV_OK) return st;
+    dev_view = static_cast<uint8_t*>(dev);
+  }
+  const int host_ctas = g_host_leg_ctas.load(std::memory_order_relaxed);
+  return for_layers(first_layer, num_layers, lo, b, t, [&](uint32_t l, int64_t off) {
+    const int i = (int)l - first_layer;
+    if (layer_ready != nullptr && layer_ready[i] != nullptr) {
+      const cudaError_t e = cudaStreamWaitEvent(s, reinterpret_cast<cudaEvent_t>(layer_ready[i]), 0);
+      if (e != cudaSuccess) return cuda_fail(e);
+    }
+    int sv = plan_layer(l, pool, lo, b, t, h_pinned, host_bytes, off, b->flags, &lp);
+    if (sv != TOPKV_OK) return sv;
+    uint8_t* host_slab = const_cast<uint8_t*>(static_cast<const uint8_t*>(h_pinned)) + off;
+    if (!lp.empty && lp.n_slab > 0) {
+      if (d_staging == nullptr) {  // direct: mapped stores / loads from a bounded grid
+        lp.kp.wire = dev_view + off;
+        sv = launch_copy<PACK>(lp.kp, lp.rs, lp.F, s, host_ctas);
+        if (sv != TOPKV_OK) return sv;
+      } else {
+        lp.kp.wire = static_cast<uint8_t*>(d_staging);
+        if (!PACK) {
+          const cudaError_t e = cudaMemcpyAsync(d_staging, host_slab, (size_t)lp.n_slab, cudaMemcpyHostToDevice, s);
+          if (e != cudaSuccess) return cuda_fail(e);
+        }
+        sv = launch_copy<PACK>(lp.kp, lp.rs, lp.F, s);
+        if (sv != TOPKV_OK) return sv;
+        if (PACK) {
+          const cudaError_t e = cudaMemcpyAsync(host_slab, d_staging, (size_t)lp.n_slab, cudaMemcpyDeviceToHost, s);
+          if (e != cudaSuccess) return cuda_fail(e);
+        }
+      }
+    }
+    if (layer_done != nullptr && layer_done[i] != nullptr) {
+      const cudaError_t e = cudaEventRecord(reinterpret_cast<cudaEvent_t>(layer_done[i]), s);
+      if (e != cudaSuccess) return cuda_fail(e);
+    }
+    return (int)TOPKV_OK;
+  });
+}
+
+}  // namespace model
 }  // namespace
 
 extern "C" {
@@ -779,6 +1045,61 @@ int topkv_unpack_layers_from_host_pipelined(int first_layer, int num_layers, voi
                                             topkv_stream_t side_stream) {
   return issue_layers<false>(first_layer, num_layers, dst_pool, layout, batch, h_pinned, host_bytes,
                              d_staging, staging_capacity_bytes, layer_ready, layer_done, side_stream);
+}
+
+int topkv_layer_table_offsets(const topkv_layout* layout, const topkv_layer_table* table,
+                              int32_t num_requests, int64_t* h_offsets) {
+  if (layout == nullptr || layout->struct_size != sizeof(topkv_layout) || table == nullptr ||
+      table->struct_size != sizeof(topkv_layer_table) || table->specs == nullptr || h_offsets == nullptr ||
+      num_requests < 0 || (num_requests > 0 && table->h_seq_lens == nullptr))
+    return TOPKV_ERR_INVALID_ARG;
+  int64_t off = 0;
+  for (uint32_t l = 0; l < table->num_layers; ++l) {
+    h_offsets[l] = off;
+    int64_t n = 0;
+    const int st = model::slab_bytes(layout, table, num_requests, l, &n);
+    if (st != TOPKV_OK) return st;
+    off += n;
+  }
+  h_offsets[table->num_layers] = off;
+  return TOPKV_OK;
+}
+
+int topkv_pack_model_layers(int first_layer, int num_layers, const void* src_pool, const topkv_layout* layout,
+                            const topkv_batch* batch, const topkv_layer_table* table, void* d_wire,
+                            int64_t wire_capacity_bytes, topkv_stream_t stream) {
+  return model::copy_layers<true>(first_layer, num_layers, src_pool, layout, batch, table, d_wire,
+                                  wire_capacity_bytes, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int topkv_unpack_model_layers(int first_layer, int num_layers, void* dst_pool, const topkv_layout* layout,
+                              const topkv_batch* batch, const topkv_layer_table* table, const void* d_wire,
+                              int64_t wire_bytes, topkv_stream_t stream) {
+  return model::copy_layers<false>(first_layer, num_layers, dst_pool, layout, batch, table, d_wire, wire_bytes,
+                                   reinterpret_cast<cudaStream_t>(stream));
+}
+
+int topkv_pack_model_layers_to_host_pipelined(int first_layer, int num_layers, const void* src_pool,
+                                              const topkv_layout* layout, const topkv_batch* batch,
+                                              const topkv_layer_table* table, void* h_pinned,
+                                              int64_t host_capacity_bytes, void* d_staging,
+                                              int64_t staging_capacity_bytes, const topkv_event_t* layer_ready,
+                                              const topkv_event_t* layer_done, topkv_stream_t side_stream) {
+  return model::issue_layers<true>(first_layer, num_layers, src_pool, layout, batch, table, h_pinned,
+                                   host_capacity_bytes, d_staging, staging_capacity_bytes, layer_ready,
+                                   layer_done, reinterpret_cast<cudaStream_t>(side_stream));
+}
+
+int topkv_unpack_model_layers_from_host_pipelined(int first_layer, int num_layers, void* dst_pool,
+                                                  const topkv_layout* layout, const topkv_batch* batch,
+                                                  const topkv_layer_table* table, const void* h_pinned,
+                                                  int64_t host_bytes, void* d_staging,
+                                                  int64_t staging_capacity_bytes,
+                                                  const topkv_event_t* layer_ready,
+                                                  const topkv_event_t* layer_done, topkv_stream_t side_stream) {
+  return model::issue_layers<false>(first_layer, num_layers, dst_pool, layout, batch, table, h_pinned, host_bytes,
+                                    d_staging, staging_capacity_bytes, layer_ready, layer_done,
+                                    reinterpret_cast<cudaStream_t>(side_stream));
 }
 
 int topkv_pack_layer_to_host_noalloc(int layer, const void* src_pool, const topkv_layout* layout,

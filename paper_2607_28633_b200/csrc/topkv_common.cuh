@@ -29,6 +29,10 @@ struct KParams {
   int64_t plane_rows;     // PLANAR: rows between the planes of a slab, or -1 = total tokens T
   int window;             // 0, or the layer keeps only the last min(s, window) tokens
   int ppc, spr;           // vectorised family: page columns per CTA, CTAs per request
+  int cpp, tps;           // pages far larger than a CTA's span are split: CTAs per page (1 = whole
+                          // pages), tokens per CTA of a split page
+  int const_len;          // > 0: every request has exactly this many tokens; sl and cu are not read
+                          // (the fixed-size state of a linear-attention layer, cut into rows)
   int64_t num_pages;      // pages per pool slab: every page id is checked against it
   int64_t wire_limit;     // bytes that may be touched behind `wire` (this layer's slab)
   int overlap;            // 1: caller declared this launch independent of the kernels before it

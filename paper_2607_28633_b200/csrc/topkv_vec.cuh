@@ -63,25 +63,39 @@ __device__ __forceinline__ void copy_span(const KParams& p, const int slot) {
   uint8_t* const pool = p.pool + (int64_t)blockIdx.y * p.S_layer;
   uint8_t* const wire = p.wire + (int64_t)blockIdx.y * p.W_layer;
   const int r = slot / p.spr;
-  const int j0 = (slot - r * p.spr) * p.ppc;
-  const int s_r = p.sl[r];
+  const int sidx = slot - r * p.spr;  // span of request r
+  // The span: `ppc` whole page columns from column j0 on, or, when pages are far larger than a
+  // CTA's share, `tps` tokens of page column j0 (`cpp` CTAs per page).
+  int j0, first, span_tokens;
+  if (p.cpp > 1) {
+    j0 = sidx / p.cpp;
+    first = j0 * p.P + (sidx - j0 * p.cpp) * p.tps;
+    span_tokens = min(p.tps, (j0 + 1) * p.P - first);
+  } else {
+    j0 = sidx * p.ppc;
+    first = j0 * p.P;  // first token of the span's page columns
+    span_tokens = p.ppc * p.P;
+  }
+  const int s_r = p.const_len > 0 ? p.const_len : p.sl[r];
   // first token this layer keeps: 0, or s_r - window for a windowed layer (§2.2)
   const int b_r = (p.window > 0 && s_r > p.window) ? s_r - p.window : 0;
-  const int first = j0 * p.P;  // first token of the span's page columns
   const int tid = threadIdx.x;
-  int hi = min(first + p.ppc * p.P, s_r);
+  int hi = min(first + span_tokens, s_r);
   if (s_r > p.maxp * p.P) {  // length longer than its block-table row: copy what the row holds
     hi = min(hi, p.maxp * p.P);
-    if (tid == 0 && j0 == 0) raise_error(kErrTable);
+    if (tid == 0 && sidx == 0) raise_error(kErrTable);
   }
   const int lo = max(first, b_r);
   if (lo >= hi) return;
-  const int v = hi - lo;       // kept tokens in this span
-  const int ts0 = lo - first;  // where they start inside the span
-  const int jlo = ts0 / p.P, jhi = (ts0 + v - 1) / p.P;  // page columns (relative) they touch
+  const int v = hi - lo;                // kept tokens in this span
+  const int ts0 = lo - j0 * p.P;        // where they start, counted from the start of page column j0
+  const int jlo = ts0 / p.P, jhi = (ts0 + v - 1) / p.P;  // page columns (relative to j0) they touch
 
   int64_t cu_r, T = p.T;
-  if (p.cu != nullptr) {
+  if (p.const_len > 0) {
+    cu_r = (int64_t)r * p.const_len;
+    if (T < 0) T = (int64_t)p.R * p.const_len;
+  } else if (p.cu != nullptr) {
     cu_r = p.cu[r];
     if (p.planar && p.plane_rows < 0 && T < 0) T = p.cu[p.R];
   } else {

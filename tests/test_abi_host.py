@@ -399,3 +399,81 @@ def test_transport_selection_and_planning_rates(golden):
     assert tk.topkv_select_transport(E(None, 1, "10.0.0.1"), a, 0) == tk.TOPKV_ERR_INVALID_ARG
     # an instance without NVLink needs no domain
     assert tk.topkv_select_transport(E(None, 0, "10.0.0.1"), a, 0) == tk.TOPKV_TRANSPORT_PCIE
+
+
+def test_layer_table_offsets_and_validation_without_gpu(golden):
+    """Host side of the layer table (§2.2): slab offsets equal Eq. 1 per layer kind, and the
+    calls refuse bad tables, ranges, capacities and state geometry before anything is launched."""
+    import oracle
+    g = golden("paper_values.txt")
+    s = int(g["seq_len"])
+    F_, W_, S_ = tk.TOPKV_LAYER_FULL, tk.TOPKV_LAYER_WINDOW, tk.TOPKV_LAYER_STATE
+    # gpt-oss shape: 36 layers, every other one windowed at 128
+    lo = tk.make_layout(36, 2, 8, 64, 2, 16, 64)
+    specs = [(W_, 128) if l % 2 == 0 else (F_, 0) for l in range(36)]
+    lens = np.array([s, 100, 128, 129, 0], dtype=np.int32)
+    t = tk.make_layer_table(specs, lens)
+    st, off = tk.topkv_layer_table_offsets(lo, t, len(lens))
+    assert st == tk.TOPKV_OK
+    kinds = [("window", 128) if l % 2 == 0 else ("full",) for l in range(36)]
+    og = oracle.Geom(L=36, F=2, h_kv=8, d_h=64, b_p=2, P=16, num_pages=64)
+    assert np.array_equal(off, oracle.layered_offsets(og, kinds, lens))
+    assert off[-1] == sum(tk.topkv_kv_bytes_layered(lo, specs, int(x)) for x in lens)
+    one = tk.make_layer_table(specs, np.array([s], dtype=np.int32))
+    st, off1 = tk.topkv_layer_table_offsets(lo, one, 1)
+    assert round(int(off1[-1]) / 2**30, 2) == float(g["layered.gpt_oss_120b.gb"])
+    # a model with state layers
+    state = 4096
+    sq = [(F_, 0) if l % 4 == 3 else (S_, state) for l in range(8)]
+    lq = tk.make_layout(2, 2, 2, 256, 2, 16, 64)
+    R = 3
+    lens3 = np.array([40, 0, 17], dtype=np.int32)
+    pool, wire, sp, slots = 0x7000000, 0x9000000, 0xB000000, 0xC000000
+    tq = tk.make_layer_table(sq, lens3, sp, slots, 64 * state, state, 64)
+    st, offq = tk.topkv_layer_table_offsets(lq, tq, R)
+    assert st == tk.TOPKV_OK and offq[1] - offq[0] == R * state
+    assert offq[4] - offq[3] == 57 * 2 * 2 * 256 * 2
+    total = int(offq[-1])
+    b = tk.make_batch(_FakeTensor(0x10000, (R, 4)), _FakeTensor(0x20000, (R,)), 57)
+    P = tk.topkv_pack_model_layers
+    before = tk.topkv_kernel_launch_count()
+    assert P(0, 9, pool, lq, b, tq, wire, total) == tk.TOPKV_ERR_LAYER_RANGE
+    assert P(-1, 1, pool, lq, b, tq, wire, total) == tk.TOPKV_ERR_LAYER_RANGE
+    assert P(0, 8, pool, lq, b, tq, wire, total - 1) == tk.TOPKV_ERR_CAPACITY
+    assert P(0, 8, pool, lq, b, tq, None, total) == tk.TOPKV_ERR_INVALID_ARG
+    assert P(0, 8, pool, lq, b, tq, wire + 8, total + 8) == tk.TOPKV_ERR_ALIGNMENT
+    bw = tk.make_batch(_FakeTensor(0x10000, (R, 4)), _FakeTensor(0x20000, (R,)), 57, None, 0, 16)
+    assert P(0, 8, pool, lq, bw, tq, wire, total) == tk.TOPKV_ERR_INVALID_ARG       # the table sets windows
+    bt_ = tk.make_batch(_FakeTensor(0x10000, (R, 4)), _FakeTensor(0x20000, (R,)), 58)
+    assert P(0, 8, pool, lq, bt_, tq, wire, total) == tk.TOPKV_ERR_INVALID_ARG      # lengths disagree
+    bad = tk.make_layer_table(sq, lens3, sp, slots, 64 * state, state, 64); bad.struct_size = 8
+    assert P(0, 8, pool, lq, b, bad, wire, total) == tk.TOPKV_ERR_INVALID_ARG
+    bad = tk.make_layer_table(sq, lens3, None, slots, 64 * state, state, 64)        # no state pool
+    assert P(0, 8, pool, lq, b, bad, wire, total) == tk.TOPKV_ERR_INVALID_ARG
+    bad = tk.make_layer_table(sq, lens3, sp, slots, 64 * state, state - 16, 64)     # slot < state
+    assert P(0, 8, pool, lq, b, bad, wire, total) == tk.TOPKV_ERR_UNSUPPORTED_LAYOUT
+    bad = tk.make_layer_table(sq, lens3, sp + 8, slots, 64 * state, state, 64)
+    assert P(0, 8, pool, lq, b, bad, wire, total) == tk.TOPKV_ERR_ALIGNMENT
+    odd = [(S_, 24)] + sq[1:]                                                        # state not x16
+    bad = tk.make_layer_table(odd, lens3, sp, slots, 64 * state, state, 64)
+    st, off_odd = tk.topkv_layer_table_offsets(lq, bad, R)
+    assert P(0, 1, pool, lq, b, bad, wire, int(off_odd[-1])) == tk.TOPKV_ERR_ALIGNMENT
+    bad = tk.make_layer_table([(9, 0)] + sq[1:], lens3, sp, slots, 64 * state, state, 64)
+    assert tk.topkv_layer_table_offsets(lq, bad, R)[0] == tk.TOPKV_ERR_INVALID_ARG
+    assert P(0, 1, pool, lq, b, bad, wire, total) == tk.TOPKV_ERR_INVALID_ARG
+    # the attention layers of the model must fit the pool (3 attention layers, pool of 2)
+    three = [(F_, 0), (S_, state), (W_, 4), (F_, 0)]
+    t3 = tk.make_layer_table(three, lens3, sp, slots, 64 * state, state, 64)
+    st, off3 = tk.topkv_layer_table_offsets(lq, t3, R)
+    assert P(0, 4, pool, lq, b, t3, wire, int(off3[-1])) == tk.TOPKV_ERR_LAYER_RANGE
+    # pipelined form: the staging slab must hold the largest slab of the range
+    H = tk.topkv_pack_model_layers_to_host_pipelined
+    biggest = int(np.diff(offq).max())
+    assert H(0, 8, pool, lq, b, tq, wire, total, 0xA000000, biggest - 16) == tk.TOPKV_ERR_CAPACITY
+    assert H(0, 8, pool, lq, b, tq, wire, total - 16, 0xA000000, biggest) == tk.TOPKV_ERR_CAPACITY
+    assert H(0, 8, pool, lq, b, tq, wire, total, 0xA000008, biggest) == tk.TOPKV_ERR_ALIGNMENT
+    assert H(0, 8, pool, lq, b, tq, None, total, 0xA000000, biggest) == tk.TOPKV_ERR_INVALID_ARG
+    assert tk.topkv_unpack_model_layers_from_host_pipelined(
+        7, 2, pool, lq, b, tq, wire, total, 0xA000000, biggest) == tk.TOPKV_ERR_LAYER_RANGE
+    assert tk.topkv_kernel_launch_count() == before
+    assert P(0, 0, pool, lq, b, tq, wire, total) == tk.TOPKV_OK                     # empty range

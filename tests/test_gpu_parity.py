@@ -1547,3 +1547,223 @@ def test_many_layers_in_one_launch_cfg1(dev, variant):
 def test_smoke_entry(dev):
     import __graft_entry__ as entry
     entry.smoke()
+
+
+# -------------------------------------------------------------------- huge pages, hybrid models (§2.2)
+
+@pytest.mark.parametrize("F,H,D,P", [(2, 8, 128, 256), (1, 1, 576, 512), (2, 2, 64, 300), (2, 8, 128, 64)])
+def test_pages_far_larger_than_a_span_are_split_between_ctas(dev, F, H, D, P):
+    """Pages of 256 KiB to 1 MiB: several CTAs share a page, each taking a run of its tokens;
+    ragged lengths end in the middle of a CTA's run, windows start in the middle of one."""
+    rng = np.random.default_rng(P + D)
+    sl = np.array([P + 37, 0, 3 * P, 1, 2 * P - 1], dtype=np.int32)
+    R = len(sl)
+    pages = (sl + P - 1) // P
+    maxp = int(pages.max()) + 1
+    npages = int(pages.sum()) + 2
+    for order in (0, 1):
+        for window in (0, P // 2 + 5):
+            g = Geom(L=2, F=F, h_kv=H, d_h=D, b_p=2, P=P, num_pages=npages, wire_order=order,
+                     window=window)
+            T = g.kept_tokens(sl)
+            g.W_layer = g.wire_layer_bytes(T)
+            bt_s = np.full((R, maxp), -1, dtype=np.int32)
+            bt_d = np.full((R, maxp), -1, dtype=np.int32)
+            ps, pd, pos = rng.permutation(npages), rng.permutation(npages), 0
+            for r in range(R):
+                bt_s[r, :pages[r]] = ps[pos:pos + pages[r]]
+                bt_d[r, :pages[r]] = pd[pos:pos + pages[r]]
+                pos += pages[r]
+            lo = _layout_from_geom(g)
+            src_h = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
+            dst_h = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
+            src, dst = torch.from_numpy(src_h).to(dev), torch.from_numpy(dst_h).to(dev)
+            wire = torch.zeros(2 * g.W_layer, dtype=torch.uint8, device=dev)
+            d_sl = torch.from_numpy(sl).to(dev)
+            bs = tk.make_batch(torch.from_numpy(bt_s).to(dev), d_sl, T, None, 0, window)
+            bd = tk.make_batch(torch.from_numpy(bt_d).to(dev), d_sl, T, None, 0, window)
+            want = np.zeros(2 * g.W_layer, dtype=np.uint8)
+            for layer in range(2):
+                tk.check(tk.topkv_pack_layer(layer, src, lo, bs, wire, wire.numel()))
+                tk.check(tk.topkv_unpack_layer(layer, dst, lo, bd, wire, wire.numel()))
+                oracle.pack(g, layer, src_h, bt_s, sl, wire=want, impl="rows")
+                oracle.unpack(g, layer, dst_h, bt_d, sl, want, impl="rows")
+            torch.cuda.synchronize()
+            assert np.array_equal(wire.cpu().numpy(), want), (order, window)
+            assert np.array_equal(dst.cpu().numpy(), dst_h), (order, window)
+
+
+def _hybrid(dev, kinds, H, D, P, sl, state_slot_stride, rng, F=2, wire_order=0):
+    """Device and host side of a hybrid model: paged pools for the attention layers, slot pools
+    for the state layers, source and destination each with their own tables and slots."""
+    R = len(sl)
+    n_att = sum(k[0] != "state" for k in kinds)
+    n_state = len(kinds) - n_att
+    pages = (sl + P - 1) // P
+    maxp = max(int(pages.max()), 1)
+    npages = int(pages.sum()) + 3
+    g = Geom(L=max(n_att, 1), F=F, h_kv=H, d_h=D, b_p=2, P=P, num_pages=npages, wire_order=wire_order)
+    n_slots = R + 2
+    S_sl = n_slots * state_slot_stride + 32
+    side = {}
+    for name in ("src", "dst"):
+        bt = np.full((R, maxp), -1, dtype=np.int32)
+        perm, pos = rng.permutation(npages), 0
+        for r in range(R):
+            bt[r, :pages[r]] = perm[pos:pos + pages[r]]
+            pos += pages[r]
+        pool = rng.integers(0, 256, g.pool_bytes(), dtype=np.uint8)
+        sp = rng.integers(0, 256, max(n_state * S_sl, 16), dtype=np.uint8)
+        slots = rng.permutation(n_slots)[:R].astype(np.int32)
+        side[name] = dict(bt=bt, pool=pool, sp=sp, slots=slots,
+                          d_bt=torch.from_numpy(bt).to(dev), d_pool=torch.from_numpy(pool).to(dev),
+                          d_sp=torch.from_numpy(sp).to(dev), d_slots=torch.from_numpy(slots).to(dev))
+    code = {"full": tk.TOPKV_LAYER_FULL, "window": tk.TOPKV_LAYER_WINDOW, "state": tk.TOPKV_LAYER_STATE}
+    specs = [(code[k[0]], k[1] if len(k) > 1 else 0) for k in kinds]
+    lo = _layout_from_geom(g)
+    d_sl = torch.from_numpy(sl).to(dev)
+    T = int(sl.sum())
+    for name in ("src", "dst"):
+        s = side[name]
+        s["batch"] = tk.make_batch(s["d_bt"], d_sl, T)
+        s["table"] = tk.make_layer_table(specs, sl, s["d_sp"] if n_state else None,
+                                         s["d_slots"] if n_state else None, S_sl, state_slot_stride,
+                                         n_slots)
+    return g, lo, side, S_sl
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_hybrid_model_layers_device_to_device(dev, seed):
+    """Full, windowed and constant-state layers in mixed order through topkv_pack_model_layers /
+    topkv_unpack_model_layers: the wire is the oracle's layered pack (slabs back to back in model
+    order, offsets equal), the destination pools the oracle's layered unpack, untouched bytes
+    included; ranges of layers leave the other slabs alone."""
+    rng = np.random.default_rng(3100 + seed)
+    H, D, P = [(8, 64, 16), (1, 128, 4), (2, 64, 1)][seed % 3]
+    F = 1 if seed == 4 else 2
+    state_a, state_b = 48 * 1024 + 16 * (seed % 3), 300 * 1024      # one below, one above a CTA's span
+    kinds = [("full",), ("window", 5), ("state", state_a), ("window", 1), ("state", state_b),
+             ("full",), ("window", 1000)]
+    if seed % 2:
+        kinds = kinds[::-1]
+    R = int(rng.integers(1, 6))
+    sl = rng.integers(0, 5 * P + 3, size=R).astype(np.int32)
+    if seed % 3 == 0:
+        sl[int(rng.integers(0, R))] = 0
+    slot_stride = 304 * 1024
+    g, lo, side, S_sl = _hybrid(dev, kinds, H, D, P, sl, slot_stride, rng, F=F, wire_order=seed % 2)
+    s, d = side["src"], side["dst"]
+    want, off = oracle.pack_layered(g, kinds, s["pool"], s["bt"], sl, s["sp"], S_sl, slot_stride, s["slots"])
+    st, got_off = tk.topkv_layer_table_offsets(lo, s["table"], R)
+    assert st == tk.TOPKV_OK and np.array_equal(got_off, off)
+    assert int(off[-1]) == sum(oracle.kv_bytes_layered(H, D, int(x), kinds, F=F) for x in sl)
+    L = len(kinds)
+    total = int(off[-1])
+    wire = torch.full((total + 64,), 0x3C, dtype=torch.uint8, device=dev)
+    # in two ranges, the later one first
+    tk.check(tk.topkv_pack_model_layers(3, L - 3, s["d_pool"], lo, s["batch"], s["table"], wire, total))
+    torch.cuda.synchronize()
+    assert (wire[:int(off[3])] == 0x3C).all()
+    tk.check(tk.topkv_pack_model_layers(0, 3, s["d_pool"], lo, s["batch"], s["table"], wire, total))
+    torch.cuda.synchronize()
+    got = wire.cpu().numpy()
+    assert np.array_equal(got[:total], want[:total]) and (got[total:] == 0x3C).all()
+    tk.check(tk.topkv_unpack_model_layers(0, L, d["d_pool"], lo, d["batch"], d["table"], wire, total))
+    torch.cuda.synchronize()
+    oracle.unpack_layered(g, kinds, d["pool"], d["bt"], sl, want, d["sp"], S_sl, slot_stride, d["slots"])
+    assert np.array_equal(d["d_pool"].cpu().numpy(), d["pool"])
+    assert np.array_equal(d["d_sp"].cpu().numpy(), d["sp"])
+    assert np.array_equal(s["d_pool"].cpu().numpy(), s["pool"])          # sources untouched
+    assert np.array_equal(s["d_sp"].cpu().numpy(), s["sp"])
+    # errors are found for the whole range before anything is launched
+    before = tk.topkv_kernel_launch_count()
+    assert tk.topkv_pack_model_layers(0, L + 1, s["d_pool"], lo, s["batch"], s["table"], wire, total) \
+        == tk.TOPKV_ERR_LAYER_RANGE
+    assert tk.topkv_pack_model_layers(0, L, s["d_pool"], lo, s["batch"], s["table"], wire, total - 16) \
+        == tk.TOPKV_ERR_CAPACITY
+    assert tk.topkv_kernel_launch_count() == before
+
+
+@pytest.mark.parametrize("staged", [True, False])
+def test_gpt_oss_shaped_hybrid_through_the_side_stream_schedule(dev, staged, golden):
+    """A gpt-oss-shaped model (§2.2: 36 layers, every other one windowed at 128 tokens, 8 KV
+    heads of 64) through the pipelined side-stream calls: the sender ships model layer l after
+    its event, the receiver places it after the sender's done-event. What lands in pinned memory
+    is the oracle's layered wire, its size Eq. 1 per layer kind (0.15 binary GB per 4K-token
+    request), and the destination pool the oracle's layered unpack."""
+    rng = np.random.default_rng(77)
+    gd = golden("paper_values.txt")
+    L, nw = int(gd["layered.gpt_oss_120b.layers"]), int(gd["layered.gpt_oss_120b.windowed"])
+    kinds = [("window", 128) if l % 2 == 0 else ("full",) for l in range(L)]
+    assert sum(k[0] == "window" for k in kinds) == nw
+    sl = np.array([4096, 700, 128, 129, 2049], dtype=np.int32)
+    R = len(sl)
+    g, lo, side, _ = _hybrid(dev, kinds, 8, 64, 16, sl, 16, rng)
+    s, d = side["src"], side["dst"]
+    want, off = oracle.pack_layered(g, kinds, s["pool"], s["bt"], sl)
+    total = int(off[-1])
+    per_request = [oracle.kv_bytes_layered(8, 64, int(x), kinds) for x in sl]
+    assert total == sum(per_request)
+    assert round(per_request[0] / 2**30, 2) == float(gd["layered.gpt_oss_120b.gb"])
+    st, got_off = tk.topkv_layer_table_offsets(lo, s["table"], R)
+    assert st == tk.TOPKV_OK and np.array_equal(got_off, off)
+    pinned = torch.full((total,), 0x99, dtype=torch.uint8).pin_memory()
+    biggest = int(np.diff(off).max())
+    st_tx = torch.empty(biggest, dtype=torch.uint8, device=dev) if staged else None
+    st_rx = torch.empty(biggest, dtype=torch.uint8, device=dev) if staged else None
+    cap = biggest if staged else 0
+    main = torch.cuda.current_stream(dev)
+    tx, rx = torch.cuda.Stream(dev, priority=-1), torch.cuda.Stream(dev)
+    x = torch.randn(1024, 1024, device=dev)
+    ready = []
+    for layer in range(L):                               # stands for the prefill of layer l
+        x = (x @ x.T) * 1e-3
+        ev = torch.cuda.Event()
+        ev.record(main)
+        ready.append(ev)
+    sent = [torch.cuda.Event() for _ in range(L)]
+    tk.check(tk.topkv_pack_model_layers_to_host_pipelined(
+        0, L, s["d_pool"], lo, s["batch"], s["table"], pinned, total, st_tx, cap, ready, sent, tx))
+    tk.check(tk.topkv_unpack_model_layers_from_host_pipelined(
+        0, L, d["d_pool"], lo, d["batch"], d["table"], pinned, total, st_rx, cap, sent, None, rx))
+    torch.cuda.synchronize()
+    assert np.array_equal(pinned.numpy(), want[:total])
+    oracle.unpack_layered(g, kinds, d["pool"], d["bt"], sl, want)
+    assert np.array_equal(d["d_pool"].cpu().numpy(), d["pool"])
+    # a staging slab smaller than the largest slab of the range is refused before any launch
+    if staged:
+        before = tk.topkv_kernel_launch_count()
+        assert tk.topkv_pack_model_layers_to_host_pipelined(
+            0, L, s["d_pool"], lo, s["batch"], s["table"], pinned, total, st_tx, biggest - 16, None,
+            None, tx) == tk.TOPKV_ERR_CAPACITY
+        assert tk.topkv_kernel_launch_count() == before
+
+
+def test_qwen_shaped_hybrid_with_state_layers_through_the_host(dev):
+    """Three of every four layers carry a constant state (§2.2's 45-of-60 split, shortened to 12
+    layers): staged side-stream transfer of attention and state slabs alike."""
+    rng = np.random.default_rng(78)
+    state = 512 * 1024
+    kinds = [("full",) if l % 4 == 3 else ("state", state) for l in range(12)]
+    sl = np.array([333, 64, 1000], dtype=np.int32)
+    g, lo, side, S_sl = _hybrid(dev, kinds, 2, 256, 16, sl, state, rng)
+    s, d = side["src"], side["dst"]
+    want, off = oracle.pack_layered(g, kinds, s["pool"], s["bt"], sl, s["sp"], S_sl, state, s["slots"])
+    total = int(off[-1])
+    assert total == sum(oracle.kv_bytes_layered(2, 256, int(x), kinds) for x in sl)
+    assert off[1] - off[0] == len(sl) * state
+    pinned = torch.zeros(total, dtype=torch.uint8).pin_memory()
+    biggest = int(np.diff(off).max())
+    staging = torch.empty(biggest, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.Stream(dev)
+    stream.wait_stream(torch.cuda.current_stream(dev))
+    L = len(kinds)
+    tk.check(tk.topkv_pack_model_layers_to_host_pipelined(
+        0, L, s["d_pool"], lo, s["batch"], s["table"], pinned, total, staging, biggest, None, None, stream))
+    tk.check(tk.topkv_unpack_model_layers_from_host_pipelined(
+        0, L, d["d_pool"], lo, d["batch"], d["table"], pinned, total, None, 0, None, None, stream))
+    stream.synchronize()
+    assert np.array_equal(pinned.numpy(), want[:total])
+    oracle.unpack_layered(g, kinds, d["pool"], d["bt"], sl, want, d["sp"], S_sl, state, d["slots"])
+    assert np.array_equal(d["d_pool"].cpu().numpy(), d["pool"])
+    assert np.array_equal(d["d_sp"].cpu().numpy(), d["sp"])
