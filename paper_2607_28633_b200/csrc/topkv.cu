@@ -1311,7 +1311,7 @@ int topkv_crc_finish(const topkv_layout* layout, const topkv_batch* batch, void*
                                                                      (int)layout->page_tokens);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);
-  topkv_crc_finish_kernel<<<(R * F + 127) / 128, 128, 0, s>>>(w, batch->seq_lens, L, R, F, maxp,
+  topkv_crc_finish_kernel<<<(R * F + 3) / 4, 128, 0, s>>>(w, batch->seq_lens, L, R, F, maxp,  // a warp each
                                                                 (int)layout->page_tokens, rs.row_bytes, d_crc_out);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e);

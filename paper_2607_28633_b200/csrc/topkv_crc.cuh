@@ -146,8 +146,9 @@ __host__ __device__ __forceinline__ uint64_t gf_fold64(uint64_t rem, const uint3
   return ((uint64_t)rh << 32) | rl;
 }
 
-// x^n mod P by square and multiply.
-__host__ __device__ inline uint64_t gf_powx(uint64_t n) {
+// x^n mod P, bit-serial square and multiply: the plain definition, kept as the reference that
+// gf_powx is checked against on the host.
+__host__ __device__ inline uint64_t gf_powx_ref(uint64_t n) {
   uint64_t result = kGfOne, base = kGfX;
   while (n) {
     if (n & 1) result = gf_mulmod(result, base);
@@ -155,6 +156,31 @@ __host__ __device__ inline uint64_t gf_powx(uint64_t n) {
     n >>= 1;
   }
   return result;
+}
+
+// x^n mod P, left to right over the bits of n below the leading one: square (one carry-less
+// product), then one more factor x where the bit is set (a shift). About 26 products for the
+// exponents met here, against several thousand dependent shift-and-add steps of the
+// bit-serial form.
+__host__ __device__ inline uint64_t gf_powx(uint64_t n) {
+  if (n == 0) return kGfOne;
+  int top = 63;
+  while (!((n >> top) & 1)) --top;
+  uint64_t result = kGfX;  // the leading one
+  for (int b = top - 1; b >= 0; --b) {
+    result = gf_mulmod_clmul(result, result);
+    if ((n >> b) & 1) result = gf_mulx(result);
+  }
+  return result;
+}
+
+// The chain over the layers is a composition of affine maps s -> s * A + V over GF(2)[x]/P.
+// then(f, g) is "f first, then g".
+struct GfAffine {
+  uint64_t A, V;
+};
+__host__ __device__ __forceinline__ GfAffine gf_then(GfAffine f, GfAffine g) {
+  return {gf_mulmod_clmul(f.A, g.A), gf_mulmod_clmul(f.V, g.A) ^ g.V};
 }
 
 // ---- workspace (device memory owned by the caller), in 8-byte words ------------------------------
@@ -540,37 +566,55 @@ topkv_crc_layer_kernel(CrcWorkspace w, CrcGeom g, const int32_t* __restrict__ sl
   if (lane == 0) w.layer_rem[((int64_t)l * R + r) * F + c] = acc;
 }
 
-// One thread per (request, plane): chains the layers,
+// One warp per (request, plane): chains the layers,
 //   state_0 = ~0,  state_l+1 = state_l * x^(8 * bytes of the plane in layer l) + rem_l,
 // and inverts. A layer copied with a window contributes min(s, window) tokens; a request
-// without tokens has remainder 0 in every layer.
+// without tokens has remainder 0 in every layer. Every step is the affine map
+// s -> s * A_l + rem_l; the maps of 32 consecutive layers, one per lane, are composed by a
+// shuffle tree (five levels) instead of one after the other.
 __global__ void __launch_bounds__(128)
 topkv_crc_finish_kernel(CrcWorkspace w, const int32_t* __restrict__ sl, int L, int R, int F, int maxp,
                         int P, int64_t row_bytes, uint64_t* __restrict__ out) {
   pdl_prologue(0);
-  const int k = blockIdx.x * blockDim.x + threadIdx.x;
-  if (k >= R * F) return;
+  const int lane = threadIdx.x & 31;
+  const int k = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (k >= R * F) return;  // uniform across the warp
   const int r = k / F, c = k - r * F;
   int64_t s = sl[r];
   s = s < 0 ? 0 : (s > (int64_t)maxp * P ? (int64_t)maxp * P : s);
   const uint64_t x_full = w.x_req[r];
-  uint64_t x_win = 0;  // x^(8 * bytes of a windowed layer's plane), for the window seen last
+  uint64_t x_win = 0;  // x^(8 * bytes of a windowed layer's plane), for the window this lane saw last
   int64_t seen = -1;
   uint64_t state = ~0ull;
-  for (int l = 0; l < L; ++l) {
-    const int64_t win = w.layer_win[l];
-    uint64_t x_len = x_full;
-    if (win > 0 && s > win) {
-      if (win != seen) {
-        x_win = gf_powx(8ull * (uint64_t)win * (uint64_t)row_bytes);
-        seen = win;
+  for (int base = 0; base < L; base += 32) {
+    const int l = base + lane;
+    GfAffine f = {kGfOne, 0ull};  // identity for lanes past the last layer
+    if (l < L) {
+      const int64_t win = w.layer_win[l];
+      f.A = x_full;
+      if (win > 0 && s > win) {
+        if (win != seen) {
+          x_win = gf_powx(8ull * (uint64_t)win * (uint64_t)row_bytes);
+          seen = win;
+        }
+        f.A = x_win;
       }
-      x_len = x_win;
+      f.V = s == 0 ? 0ull : w.layer_rem[((int64_t)l * R + r) * F + c];
     }
-    const uint64_t rem = s == 0 ? 0ull : w.layer_rem[((int64_t)l * R + r) * F + c];
-    state = gf_mulmod_clmul(state, x_len) ^ rem;
+    // after the step with offset o, every lane that is a multiple of 2o holds the composition of
+    // the maps of lanes [lane, lane + 2o); other lanes hold values that nobody reads any more
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      GfAffine g;
+      g.A = __shfl_down_sync(0xffffffffu, f.A, o);
+      g.V = __shfl_down_sync(0xffffffffu, f.V, o);
+      f = gf_then(f, g);
+    }
+    f.A = __shfl_sync(0xffffffffu, f.A, 0);
+    f.V = __shfl_sync(0xffffffffu, f.V, 0);
+    state = gf_mulmod_clmul(state, f.A) ^ f.V;
   }
-  out[k] = ~state;
+  if (lane == 0) out[k] = ~state;
 }
 
 }  // namespace topkv

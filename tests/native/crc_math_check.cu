@@ -60,6 +60,30 @@ int main(int argc, char** argv) {
     memcpy(ww, w, 64);
     if (gf_fold64(s, ww) != ref) ++bad;
   }
+  // x^n by repeated squaring with the carry-less product against the bit-serial definition
+  for (int i = 0; i < 3000; ++i) {
+    uint64_t n = splitmix(seed) >> (i % 64);
+    if (i < 200) n = (uint64_t)i;
+    if (i % 11 == 0) n = 8ull * 1024 * 32 * (uint64_t)(i + 1);
+    if (gf_powx(n) != gf_powx_ref(n)) ++bad;
+  }
+  // a chain of affine steps composed pairwise (as the shuffle tree of topkv_crc_finish does it,
+  // 32 steps at a time, identity padded) against the steps taken one after the other
+  for (int i = 0; i < 200; ++i) {
+    const int n = 1 + (int)(splitmix(seed) % 100);
+    std::vector<GfAffine> f(n);
+    for (auto& x : f) x = {splitmix(seed), splitmix(seed)};
+    uint64_t seq = ~0ull, tree = ~0ull;
+    for (int l = 0; l < n; ++l) seq = gf_mulmod(seq, f[l].A) ^ f[l].V;
+    for (int base = 0; base < n; base += 32) {
+      GfAffine lane[32];
+      for (int q = 0; q < 32; ++q) lane[q] = base + q < n ? f[base + q] : GfAffine{kGfOne, 0ull};
+      for (int o = 1; o < 32; o <<= 1)
+        for (int q = 0; q + o < 32; q += 2 * o) lane[q] = gf_then(lane[q], lane[q + o]);
+      tree = gf_mulmod_clmul(tree, lane[0].A) ^ lane[0].V;
+    }
+    if (seq != tree) ++bad;
+  }
   if (bad) {
     printf("mismatches %d\n", bad);
     return 1;
