@@ -83,6 +83,22 @@ int main(void) {
   attempts_left = 10;
   if (topkv_retry(attempt, NULL, 2, 1) != TOPKV_ERR_CHECKSUM) return 11;
   if (topkv_model_hidden_fraction(80, 0.5e-3, 52e-3) < 0.75) return 12;
+  {
+    topkv_endpoint a, b;
+    memset(&a, 0, sizeof a);
+    memset(&b, 0, sizeof b);
+    a.struct_size = b.struct_size = (uint32_t)sizeof(topkv_endpoint);
+    a.has_nvlink = b.has_nvlink = 1;
+    a.nvlink_domain = "node-a"; a.node_ip = "10.0.0.1";
+    b.nvlink_domain = "node-a"; b.node_ip = "10.0.0.1";
+    if (topkv_select_transport(&a, &b, 0, 0) != TOPKV_TRANSPORT_NVLINK) return 14;
+    b.nvlink_domain = "node-b"; b.node_ip = "10.0.0.2";
+    if (topkv_select_transport(&a, &b, 1, 0) != TOPKV_TRANSPORT_RDMA) return 15;
+    if (topkv_select_transport(&a, &b, 0, 0) != TOPKV_TRANSPORT_TCP) return 16;
+    if (topkv_select_transport(&a, &b, 0, TOPKV_TRANSPORT_PCIE) != TOPKV_TRANSPORT_PCIE) return 17;
+    if (topkv_planning_rate(TOPKV_TRANSPORT_NVLINK) != 450e9 || topkv_planning_rate(9) != 0.0) return 18;
+    if (strcmp(topkv_transport_name(TOPKV_TRANSPORT_TCP), "tcp") != 0) return 19;
+  }
   for (int s = -12; s <= 1; ++s)
     if (topkv_strerror(s) == NULL) return 13;
   printf("sanitized host shims ok\n");

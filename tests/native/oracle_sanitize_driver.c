@@ -50,8 +50,33 @@ int main(void) {
       for (int64_t c = 0; c < g.F; ++c)
         if (oracle_kv_plane_crc(&g, pool, R, maxp, bt, sl, r, c) !=
             oracle_kv_plane_crc(&g, back, R, maxp, bt, sl, r, c)) { puts("crc differs"); return 1; }
+    /* the same batch as a model whose layers differ in kind: windowed, state, full, state */
+    {
+      int64_t kind[4] = {1, 2, 0, 2}, param[4] = {2, 48, 0, 16}, off[5];
+      int64_t S_slot = 64, S_state_layer = (R + 1) * S_slot + 16;
+      int32_t slot[4];
+      for (int64_t r = 0; r < R; ++r) slot[r] = (int32_t)(R - r); /* slots 1..R of R + 1 */
+      oracle_geom gm = g;
+      gm.window = 0;
+      oracle_layered_offsets(&gm, 4, kind, param, R, sl, off);
+      uint8_t* sp = malloc((size_t)(2 * S_state_layer));
+      uint8_t* sp_back = malloc((size_t)(2 * S_state_layer));
+      for (int64_t k = 0; k < 2 * S_state_layer; ++k) sp[k] = (uint8_t)(lcg(&seed) >> 24);
+      memset(sp_back, 0x33, (size_t)(2 * S_state_layer));
+      uint8_t* lw = calloc((size_t)(off[4] + 1), 1);
+      uint8_t* lw2 = calloc((size_t)(off[4] + 1), 1);
+      memset(back, 0x5A, (size_t)(g.L * g.S_layer));
+      oracle_pack_layered(&gm, 4, kind, param, pool, R, maxp, bt, sl, sp, S_state_layer, S_slot, slot, lw);
+      oracle_unpack_layered(&gm, 4, kind, param, back, R, maxp, bt, sl, sp_back, S_state_layer, S_slot, slot, lw);
+      oracle_pack_layered(&gm, 4, kind, param, back, R, maxp, bt, sl, sp_back, S_state_layer, S_slot, slot, lw2);
+      if (memcmp(lw, lw2, (size_t)off[4]) != 0) { puts("layered round trip differs"); return 1; }
+      free(sp); free(sp_back); free(lw); free(lw2);
+    }
     free(pool); free(back); free(wire_a); free(wire_b);
   }
+  if (oracle_select_transport(0, "a", 1, "1.1.1.1", "a", 1, "1.1.1.1", 0) != ORACLE_MODE_NVLINK ||
+      oracle_select_transport(0, "a", 1, "1.1.1.1", "b", 1, "1.1.1.2", 0) != ORACLE_MODE_TCP ||
+      oracle_planning_rate(ORACLE_MODE_PCIE) != 50e9) { puts("selector"); return 1; }
   if (oracle_crc64_iso((const uint8_t*)"123456789", 9) != 0xB90956C775A41001ull) { puts("check value"); return 1; }
   puts("sanitized oracle ok");
   return 0;

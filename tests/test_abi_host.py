@@ -91,6 +91,11 @@ def test_layered_sizes(golden):
     specs = [(W, 128) if l % 2 == 0 else (F, 0) for l in range(36)]
     got = tk.topkv_kv_bytes_layered(oss, specs, s)
     assert got == 18 * 2 * 8 * 64 * 2 * (4096 + 128)
+    # A thin pin, stated as such: 155,713,536 B is 0.14502 binary GB, which rounds to the printed
+    # 0.15 with a margin of 2e-5 (in decimal GB it would be 0.156). The reading (binary GB, as
+    # Table 1's 0.27 requires; heads, head dim and window from the model's public configuration)
+    # is what is pinned, not an independent measurement of the paper's figure.
+    assert 0.145 <= got / 2**30 < 0.1451
     assert round(got / 2**30, 2) == float(g["layered.gpt_oss_120b.gb"])
     l70 = tk.make_layout(80, 2, 8, 128, 2, 16, 1)
     assert tk.topkv_kv_bytes_layered(l70, [(F, 0)] * 80, s) == tk.topkv_kv_bytes(l70, s)
