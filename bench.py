@@ -722,6 +722,64 @@ def run_extra(name, dev, stream, args, peak):
             del w
             torch.cuda.empty_cache()
         return out
+    if name == "hybrid":
+        # models whose layers differ in kind (§2.2) through the layer-table calls, device to
+        # device: a gpt-oss-shaped one (36 layers, every other one windowed at 128 tokens, 8 KV
+        # heads of 64) and a Qwen3.5-shaped one (60 layers, 45 of them a constant 1 MiB state
+        # per request, 15 full layers of 2 KV heads of 256), both on cfg2's 16 requests of
+        # 512..4096 tokens. GB/s of read + write traffic over all slabs of the model.
+        import numpy as np
+        from dataclasses import replace
+        out = {"workload": "cfg2 batch; gpt-oss-shaped and Qwen3.5-shaped layer tables"}
+        F_, W_, S_ = tk.TOPKV_LAYER_FULL, tk.TOPKV_LAYER_WINDOW, tk.TOPKV_LAYER_STATE
+        state = 1 << 20
+        models = (("gpt_oss_shaped", replace(wl.CFG2, L=36, H=8, D=64),
+                   [(W_, 128) if l % 2 == 0 else (F_, 0) for l in range(36)]),
+                  ("qwen35_shaped", replace(wl.CFG2, L=15, H=2, D=256),
+                   [(F_, 0) if l % 4 == 3 else (S_, state) for l in range(60)]))
+        for label, spec, specs in models:
+            w = harness.setup(spec, dev, fill_dst=False, need_wire=False)
+            R = spec.R
+            n_state = sum(1 for k, _ in specs if k == S_)
+            slots = R + 4
+            sp_s = wl.fill_torch(max(n_state * slots * state, 16), 77, dev, raw_bits=True)
+            sp_d = torch.zeros_like(sp_s)
+            g = np.random.Generator(np.random.PCG64(78))
+            sl_s = torch.from_numpy(g.permutation(slots)[:R].astype(np.int32)).to(dev)
+            sl_d = torch.from_numpy(g.permutation(slots)[:R].astype(np.int32)).to(dev)
+            ts = tk.make_layer_table(specs, w.batch.seq_lens, sp_s, sl_s, slots * state, state, slots)
+            td = tk.make_layer_table(specs, w.batch.seq_lens, sp_d, sl_d, slots * state, state, slots)
+            st, off = tk.topkv_layer_table_offsets(w.layout, ts, R)
+            tk.check(st)
+            total = int(off[-1])
+            wire = torch.empty(total, dtype=torch.uint8, device=dev)
+            nl = len(specs)
+
+            def run():
+                tk.check(tk.topkv_pack_model_layers(0, nl, w.src_pool, w.layout, w.src_batch, ts, wire,
+                                                    total, stream))
+                tk.check(tk.topkv_unpack_model_layers(0, nl, w.dst_pool, w.layout, w.dst_batch, td, wire,
+                                                      total, stream))
+            run()
+            stream.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            steps = max(1, min(args.steps, 5))
+            a.record(stream)
+            for _ in range(steps):
+                run()
+            b.record(stream)
+            stream.synchronize()
+            ms = a.elapsed_time(b) / steps
+            gbs = 4.0 * total / (ms * 1e-3) / 1e9
+            out[label] = {"model_layers": nl, "wire_bytes_all_layers": total,
+                          "largest_slab_bytes": int(np.diff(off).max()),
+                          "smallest_slab_bytes": int(np.diff(off).min()),
+                          "ms_pack_plus_unpack": round(ms, 4), "GBps": round(gbs, 1),
+                          "frac_of_hbm_peak": round(gbs / peak, 4),
+                          "device_error_flags": tk.topkv_device_error_flags()}
+            del w, sp_s, sp_d, wire
+            torch.cuda.empty_cache()
+        return out
     if name == "overlap_curve":
         # three points on the Eq. 3 curve (§5.2) and the interference §5.5 could not validate:
         # slack (64 MiB per layer under a 2.8 ms layer), near-saturated (128 MiB per layer, about
@@ -822,7 +880,7 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="topkv", choices=["topkv", "reference"])
-    ap.add_argument("--extras", default="cfg5,overlap_curve,cfg2,cfg4,chain,crc,session,cfg1",
+    ap.add_argument("--extras", default="cfg5,overlap_curve,cfg2,cfg4,chain,crc,hybrid,session,cfg1",
                     help="comma list of extra workloads measured at one GPU ('' for none)")
     ap.add_argument("--variant", type=int, default=None, help="kernel family (see topkv.h)")
     ap.add_argument("--layers", type=int, default=None, help="fewer layers (profiling only)")
