@@ -446,10 +446,13 @@ int topkv_layer_table_offsets(const topkv_layout* layout, const topkv_layer_tabl
                               int32_t num_requests, int64_t* h_offsets);
 
 /* Model layers first_layer .. first_layer + num_layers - 1 between the pools and the wire buffer
- * behind d_wire (slab l at d_wire + h_offsets[l]), device to device, one kernel per layer on
- * `stream`. The layers of one call touch different slabs and different pool layers, so every
- * launch after the first is allowed to overlap its predecessor; batch->flags applies to the
- * first. Everything is validated for every layer before anything is launched. For unpack,
+ * behind d_wire (slab l at d_wire + h_offsets[l]), device to device, on `stream`. Layers of the
+ * same kind and parameter that lie at a constant stride in their pool and in the wire (every
+ * other layer of a model that alternates windowed and full layers, the state layers between
+ * the full ones) share one launch; otherwise one kernel per layer. The layers of one call touch
+ * different slabs and different pool layers, so every launch after the first is allowed to
+ * overlap its predecessor (and the layers are moved in no particular order); batch->flags
+ * applies to the first. Everything is validated for every layer before anything is launched. For unpack,
  * `dst_pool` and table->state_pool are the destination pools, batch->block_table and
  * table->state_slots the destination's tables. */
 int topkv_pack_model_layers(int first_layer, int num_layers, const void* src_pool,

@@ -22,6 +22,7 @@
 #include <cstdint>
 #include <cstring>
 #include <mutex>
+#include <vector>
 
 namespace {
 
@@ -818,8 +819,12 @@ int for_layers(int first_layer, int num_layers, const topkv_layout* lo, const to
   return TOPKV_OK;
 }
 
-// Device to device: one launch per layer; the layers of one call touch different slabs and
-// different pool layers, so every launch after the first may overlap its predecessor.
+// Device to device. The layers of one call touch different slabs and different pool layers, so
+// every launch after the first may overlap its predecessor, and layers of the same kind and
+// parameter whose places in their pool and in the wire form an arithmetic progression (every
+// other layer of a model that alternates windowed and full layers; the state layers between the
+// full ones) are equal slabs at a constant stride on both sides: they go into ONE launch, the
+// layer being blockIdx.y, instead of one launch-bound kernel each.
 template <bool PACK>
 int copy_layers(int first_layer, int num_layers, const void* pool, const topkv_layout* lo,
                 const topkv_batch* b, const topkv_layer_table* t, const void* d_wire, int64_t wire_bytes,
@@ -828,20 +833,57 @@ int copy_layers(int first_layer, int num_layers, const void* pool, const topkv_l
   if (st != TOPKV_OK) return st;
   st = check_range(t, first_layer, num_layers);
   if (st != TOPKV_OK) return st;
+  struct Info {
+    int64_t off;
+    uint32_t ord;
+    bool done;
+  };
+  std::vector<Info> info((size_t)num_layers);
   LayerPlan lp;
   st = for_layers(first_layer, num_layers, lo, b, t, [&](uint32_t l, int64_t off) {  // validate all first
+    uint32_t ord = 0;
+    for (uint32_t q = 0; q < l; ++q)
+      ord += (t->specs[q].kind == TOPKV_LAYER_STATE) == (t->specs[l].kind == TOPKV_LAYER_STATE) ? 1u : 0u;
+    info[l - first_layer] = {off, ord, false};
     return plan_layer(l, pool, lo, b, t, d_wire, wire_bytes, off, b->flags, &lp);
   });
   if (st != TOPKV_OK) return st;
   bool launched = false;
-  return for_layers(first_layer, num_layers, lo, b, t, [&](uint32_t l, int64_t off) {
+  for (int i = 0; i < num_layers; ++i) {
+    if (info[i].done) continue;
+    const topkv_layer_spec& sp = t->specs[first_layer + i];
+    const bool is_state = sp.kind == TOPKV_LAYER_STATE;
+    // the run that starts at layer i: same kind and parameter, constant stride in pool and wire
+    int count = 1, last = i;
+    int64_t d_off = 0, d_ord = 0;
+    for (int j = i + 1; j < num_layers && count < 65535; ++j) {
+      const topkv_layer_spec& sq = t->specs[first_layer + j];
+      if (info[j].done || sq.kind != sp.kind || sq.param != sp.param) continue;
+      const int64_t o = info[j].off - info[last].off, r = (int64_t)info[j].ord - info[last].ord;
+      if (count == 1) {
+        d_off = o;
+        d_ord = r;
+      } else if (o != d_off || r != d_ord) {
+        continue;
+      }
+      info[j].done = true;
+      last = j;
+      ++count;
+    }
+    info[i].done = true;
     const uint32_t flags = launched ? (b->flags | TOPKV_FLAG_OVERLAP_PREVIOUS) : b->flags;
-    int sv = plan_layer(l, pool, lo, b, t, d_wire, wire_bytes, off, flags, &lp);
-    if (sv != TOPKV_OK || lp.empty) return sv;
-    sv = launch_copy<PACK>(lp.kp, lp.rs, lp.F, s);
-    launched = launched || sv == TOPKV_OK;
-    return sv;
-  });
+    st = plan_layer((uint32_t)(first_layer + i), pool, lo, b, t, d_wire, wire_bytes, info[i].off, flags, &lp);
+    if (st != TOPKV_OK) return st;
+    if (lp.empty) continue;
+    if (count > 1) {
+      lp.kp.S_layer = d_ord * (is_state ? t->state_layer_stride : lo->pool_layer_stride);
+      lp.kp.W_layer = d_off;
+    }
+    st = launch_copy<PACK>(lp.kp, lp.rs, lp.F, s, 0, count);
+    if (st != TOPKV_OK) return st;
+    launched = true;
+  }
+  return TOPKV_OK;
 }
 
 // The side-stream schedule of §5.2 for such a model: per layer wait, ship over PCIe, record.
