@@ -580,6 +580,49 @@ def bench_chain(w, stream, steps, unpack_flags=0, slabs=1):
     return 4.0 * w.n_layer * w.layers / (ms * 1e-3) / 1e9, ms / (2 * w.layers) * 1e3
 
 
+def bench_chain_linked(w, stream, steps, slabs=1):
+    """The same dependent order with span links (topkv_pack_layer_linked /
+    topkv_unpack_layer_linked): unpack(l) waits span by span for pack(l), pack(l + slabs) span by
+    span for unpack(l) to have read the slab, and no launch waits for its predecessor as a whole."""
+    import ctypes
+    import torch
+    from paper_2607_28633_b200 import binding as tk
+    lo = type(w.layout)()
+    ctypes.memmove(ctypes.byref(lo), ctypes.byref(w.layout), ctypes.sizeof(lo))
+    lo.wire_layer_stride = 0
+    n = w.n_layer
+    slab = [w.wire[k * n:(k + 1) * n] for k in range(slabs)]
+    T = w.batch.total_tokens
+    bs = tk.make_batch(w.src_bt, w.seq_lens, T, w.cu)
+    bd = tk.make_batch(w.dst_bt, w.seq_lens, T, w.cu)
+    words = tk.check(tk.topkv_span_link_words(lo, bs))
+    dev = w.src_pool.device
+    fp = [torch.zeros(words, dtype=torch.int32, device=dev) for _ in range(slabs)]
+    fu = [torch.zeros(words, dtype=torch.int32, device=dev) for _ in range(slabs)]
+    uses = [0] * slabs           # how often each slab has been through a pack / unpack pair
+
+    def run():
+        for l in range(w.layers):
+            q = l % slabs
+            e = uses[q]
+            lp = tk.make_span_link(fu[q] if e else None, e, fp[q], e + 1)
+            tk.check(tk.topkv_pack_layer_linked(l, w.src_pool, lo, bs, slab[q], n, lp, stream))
+            lu = tk.make_span_link(fp[q], e + 1, fu[q], e + 1)
+            tk.check(tk.topkv_unpack_layer_linked(l, w.dst_pool, lo, bd, slab[q], n, lu, stream))
+            uses[q] = e + 1
+    run()
+    stream.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(steps):
+        run()
+    b.record(stream)
+    stream.synchronize()
+    assert tk.topkv_device_error_flags() == 0
+    ms = a.elapsed_time(b) / steps
+    return 4.0 * w.n_layer * w.layers / (ms * 1e-3) / 1e9, ms / (2 * w.layers) * 1e3
+
+
 def host_leg_forms(w, dev, stream, pinned, slots, steps):
     """The host leg of the workload in its three forms against a pinned cudaMemcpyAsync of one
     slab measured in the same run."""
@@ -715,6 +758,11 @@ def run_extra(name, dev, stream, args, peak):
             for label, flags, slabs in (("one_slab_plain", 0, 1), ("one_slab_tables_settled", ts, 1),
                                         ("two_slabs_plain", 0, 2), ("two_slabs_tables_settled", ts, 2)):
                 gbs, us = bench_chain(w, stream, max(1, min(args.steps, 5)), flags, slabs)
+                r[label] = {"GBps": round(gbs, 1), "us_per_launch": round(us, 2),
+                            "frac_of_hbm_peak": round(gbs / peak, 4),
+                            "frac_of_8000_spec": round(gbs / 8000.0, 4)}
+            for label, slabs in (("one_slab_span_linked", 1), ("two_slabs_span_linked", 2)):
+                gbs, us = bench_chain_linked(w, stream, max(1, min(args.steps, 5)), slabs)
                 r[label] = {"GBps": round(gbs, 1), "us_per_launch": round(us, 2),
                             "frac_of_hbm_peak": round(gbs / peak, 4),
                             "frac_of_8000_spec": round(gbs / 8000.0, 4)}

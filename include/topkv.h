@@ -195,6 +195,48 @@ int topkv_unpack_layer_from_host(int layer, void* dst_pool, const topkv_layout* 
                                  int64_t host_bytes, void* d_staging,
                                  int64_t staging_capacity_bytes, topkv_stream_t stream);
 
+/* ---- span links: dependent launches that do not wait for each other as a whole (§5.2) -------
+ * In a relay, the unpack of layer l reads what the pack of layer l has just written (§5.2 sends
+ * a layer as soon as it exists), so that launch can never be declared independent, and as an
+ * ordinary launch it waits for the LAST CTA of the pack before its first CTA may touch memory.
+ * A span link orders the two kernels span by span instead: both cut the batch into the same
+ * spans (one CTA each; the same lengths, page_tokens, row size and max_pages_per_req on both
+ * sides, whatever the block tables), every CTA of the first kernel publishes its span's flag
+ * when its stores are issued, and every CTA of the second waits for the flag of ITS span only,
+ * so the second kernel runs under the first one's tail like an independent launch.
+ *   d_signal : flags this call publishes (value signal_epoch), or NULL
+ *   d_await  : flags this call waits for (until they hold await_epoch), or NULL
+ * Both are DEVICE int32 arrays of topkv_span_link_words() entries, owned by the caller, that
+ * must not already hold the epochs of the calls about to use them (zero them once and use
+ * epochs 1, 2, 3, ...: an array is reused by giving every pair of calls its own epoch).
+ * A linked call never waits for the previous kernel as a whole and reads its tables at once,
+ * as if TOPKV_FLAG_OVERLAP_PREVIOUS were set: the caller promises that the tables were not
+ * written by kernels still running and that EVERY conflict with kernels enqueued before it on
+ * `stream` is covered by the link. For pack(l) -> unpack(l) -> pack(l+1) -> ... through one slab:
+ * pack(l+1) awaits the flags unpack(l) publishes (the slab has been read) and publishes the
+ * flags unpack(l+1) awaits. Kernels still complete in stream order. Waits are bounded (about
+ * half a second): a flag that never arrives raises bit 1 of topkv_device_error_flags() and skips the
+ * span. Linked launches are safe because a kernel's CTAs are scheduled only after every CTA of
+ * the earlier kernels of the stream has started: enqueue the linked calls on ONE stream, in
+ * producer-before-consumer order, with no other work between them. Vectorised kernel family,
+ * one layer per call. */
+typedef struct topkv_span_link {
+  uint32_t struct_size;   /* = sizeof(topkv_span_link)               */
+  uint32_t await_epoch;   /* value the awaited flags must reach      */
+  uint32_t signal_epoch;  /* value written into the published flags  */
+  uint32_t reserved;      /* must be 0                               */
+  const int32_t* d_await; /* DEVICE int32 [words] or NULL            */
+  int32_t* d_signal;      /* DEVICE int32 [words] or NULL            */
+} topkv_span_link;
+/* Number of flags (spans) of one layer of this batch, or a negative topkv_status. */
+int64_t topkv_span_link_words(const topkv_layout* layout, const topkv_batch* batch);
+int topkv_pack_layer_linked(int layer, const void* src_pool, const topkv_layout* layout,
+                            const topkv_batch* batch, void* d_wire, int64_t wire_capacity_bytes,
+                            const topkv_span_link* link, topkv_stream_t stream);
+int topkv_unpack_layer_linked(int layer, void* dst_pool, const topkv_layout* layout,
+                              const topkv_batch* batch, const void* d_wire, int64_t wire_bytes,
+                              const topkv_span_link* link, topkv_stream_t stream);
+
 /* ---- direct re-paging (no wire slab) -------------------------------------------------------- */
 
 /* Moves layer `layer` of the batch from one paged pool straight into another paged pool with

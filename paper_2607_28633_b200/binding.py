@@ -48,7 +48,8 @@ EXPORTS = (
     "topkv_copy_vector_bytes", "topkv_select_transport", "topkv_planning_rate",
     "topkv_transport_name", "topkv_layer_table_offsets", "topkv_pack_model_layers",
     "topkv_unpack_model_layers", "topkv_pack_model_layers_to_host_pipelined",
-    "topkv_unpack_model_layers_from_host_pipelined",
+    "topkv_unpack_model_layers_from_host_pipelined", "topkv_span_link_words",
+    "topkv_pack_layer_linked", "topkv_unpack_layer_linked",
 )
 
 
@@ -78,6 +79,20 @@ class topkv_layer_spec(ctypes.Structure):
 
 
 TOPKV_LAYER_FULL, TOPKV_LAYER_WINDOW, TOPKV_LAYER_STATE = 0, 1, 2
+
+
+class topkv_span_link(ctypes.Structure):
+    _fields_ = [("struct_size", c_uint32), ("await_epoch", c_uint32), ("signal_epoch", c_uint32),
+                ("reserved", c_uint32), ("d_await", c_void_p), ("d_signal", c_void_p)]
+
+
+def make_span_link(d_await=None, await_epoch=0, d_signal=None, signal_epoch=0) -> topkv_span_link:
+    k = topkv_span_link()
+    k.struct_size = ctypes.sizeof(topkv_span_link)
+    k.await_epoch, k.signal_epoch = await_epoch, signal_epoch
+    k.d_await, k.d_signal = _ptr(d_await), _ptr(d_signal)
+    k._keepalive = (d_await, d_signal)
+    return k
 
 
 class topkv_layer_table(ctypes.Structure):
@@ -205,6 +220,11 @@ def lib() -> ctypes.CDLL:
         L.topkv_set_host_leg_ctas.argtypes = [c_int]
         L.topkv_pack_layers.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p]
         L.topkv_unpack_layers.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p]
+        kp_ = ctypes.POINTER(topkv_span_link)
+        L.topkv_span_link_words.argtypes = [lp, bp]
+        L.topkv_span_link_words.restype = c_int64
+        L.topkv_pack_layer_linked.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64, kp_, c_void_p]
+        L.topkv_unpack_layer_linked.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64, kp_, c_void_p]
         tp = ctypes.POINTER(topkv_layer_table)
         L.topkv_layer_table_offsets.argtypes = [lp, tp, c_int32, c_void_p]
         L.topkv_pack_model_layers.argtypes = [c_int, c_int, c_void_p, lp, bp, tp, c_void_p, c_int64, c_void_p]
@@ -369,6 +389,23 @@ def topkv_unpack_layers_from_host_pipelined(first_layer, num_layers, dst_pool, l
         first_layer, num_layers, _ptr(dst_pool), ctypes.byref(layout), ctypes.byref(batch),
         _ptr(h_pinned), host_bytes, _ptr(d_staging), staging_capacity_bytes,
         _events(layer_ready, num_layers), _events(layer_done, num_layers), _stream(side_stream))
+
+
+def topkv_span_link_words(layout, batch):
+    return lib().topkv_span_link_words(ctypes.byref(layout), ctypes.byref(batch))
+
+
+def topkv_pack_layer_linked(layer, src_pool, layout, batch, d_wire, wire_capacity_bytes, link,
+                            stream=None):
+    return lib().topkv_pack_layer_linked(layer, _ptr(src_pool), ctypes.byref(layout),
+                                         ctypes.byref(batch), _ptr(d_wire), wire_capacity_bytes,
+                                         ctypes.byref(link), _stream(stream))
+
+
+def topkv_unpack_layer_linked(layer, dst_pool, layout, batch, d_wire, wire_bytes, link, stream=None):
+    return lib().topkv_unpack_layer_linked(layer, _ptr(dst_pool), ctypes.byref(layout),
+                                           ctypes.byref(batch), _ptr(d_wire), wire_bytes,
+                                           ctypes.byref(link), _stream(stream))
 
 
 def topkv_layer_table_offsets(layout, table, num_requests):

@@ -159,6 +159,10 @@ int prepare(int layer, const void* pool, const topkv_layout* lo, const topkv_bat
   kp->plane_rows = spread ? lo->wire_plane_stride / rs->row_bytes : -1;
   kp->S_layer = 0;
   kp->W_layer = 0;
+  kp->link_await = nullptr;
+  kp->link_signal = nullptr;
+  kp->await_epoch = 0;
+  kp->signal_epoch = 0;
   return TOPKV_OK;
 }
 
@@ -266,6 +270,29 @@ int copy_vector_bytes(const KParams& kp, int64_t unit_bytes, int layers) {
   return (m & 31) == 0 ? 32 : 16;
 }
 
+// How the vectorised family cuts a block-table row into spans (one CTA each): `ppc` whole page
+// columns per span when pages are small, `cpp` CTAs per page when pages are far larger than a
+// CTA's share, one page otherwise. Fills ppc, spr, cpp, tps.
+void span_geometry(KParams* kp, int F, int64_t row_bytes) {
+  const int64_t page_bytes = (int64_t)kp->P * F * row_bytes;
+  kp->ppc = (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(kMaxPagesPerCta, kp->maxp),
+                                                       kSpanTargetBytes / page_bytes));
+  kp->spr = (kp->maxp + kp->ppc - 1) / kp->ppc;
+  kp->cpp = 1;
+  kp->tps = 0;
+  if (page_bytes >= 2 * kSpanTargetBytes && kp->P > 1) {  // huge pages: several CTAs per page
+    const int64_t tok_bytes = (int64_t)F * row_bytes;
+    kp->tps = (int)std::max<int64_t>(1, std::min<int64_t>(kp->P, kSpanTargetBytes / tok_bytes));
+    kp->cpp = (kp->P + kp->tps - 1) / kp->tps;
+    if ((int64_t)kp->maxp * kp->cpp > 0x7fffffffll / std::max(1, kp->R)) {  // keep R * spr an int
+      kp->cpp = 1;
+      kp->tps = 0;
+    } else if (kp->cpp > 1) {
+      kp->spr = kp->maxp * kp->cpp;
+    }
+  }
+}
+
 // max_ctas > 0: the wire is host memory behind PCIe; at most that many CTAs walk the spans.
 // layers > 1: one launch covers that many consecutive layers (kp describes the first one and
 // carries the layer strides); the vectorised family only.
@@ -275,28 +302,13 @@ int launch_copy(KParams kp, const Resolved& rs, int F, cudaStream_t stream, int 
   const int64_t slots = (int64_t)kp.R * kp.maxp;
   if (slots == 0 || layers == 0) return TOPKV_OK;
   bool handled = false;
-  if (max_ctas <= 0 && layers == 1 && g_variant.load(std::memory_order_relaxed) == 1) {
+  const bool linked = kp.link_await != nullptr || kp.link_signal != nullptr;
+  if (max_ctas <= 0 && layers == 1 && !linked && g_variant.load(std::memory_order_relaxed) == 1) {
     const int st = launch_bulk<PACK>(kp, rs, F, stream, &handled);
     if (st != TOPKV_OK) return st;
   }
   if (!handled) {
-    const int64_t page_bytes = (int64_t)kp.P * F * rs.row_bytes;
-    kp.ppc = (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(kMaxPagesPerCta, kp.maxp),
-                                                        kSpanTargetBytes / page_bytes));
-    kp.spr = (kp.maxp + kp.ppc - 1) / kp.ppc;
-    kp.cpp = 1;
-    kp.tps = 0;
-    if (page_bytes >= 2 * kSpanTargetBytes && kp.P > 1) {  // huge pages: several CTAs per page
-      const int64_t tok_bytes = (int64_t)F * rs.row_bytes;
-      kp.tps = (int)std::max<int64_t>(1, std::min<int64_t>(kp.P, kSpanTargetBytes / tok_bytes));
-      kp.cpp = (kp.P + kp.tps - 1) / kp.tps;
-      if ((int64_t)kp.maxp * kp.cpp > 0x7fffffffll / std::max(1, kp.R)) {  // keep R * spr an int
-        kp.cpp = 1;
-        kp.tps = 0;
-      } else if (kp.cpp > 1) {
-        kp.spr = kp.maxp * kp.cpp;
-      }
-    }
+    span_geometry(&kp, F, rs.row_bytes);
     const int64_t spans = (int64_t)kp.R * kp.spr;
     const bool walk = max_ctas > 0 && spans > max_ctas;
     const dim3 grid((unsigned)(walk ? max_ctas : spans), (unsigned)layers);
@@ -979,6 +991,68 @@ int topkv_unpack_layer(int layer, void* dst_pool, const topkv_layout* layout,
   return launch_copy<false>(kp, rs, (int)layout->kv_factor, reinterpret_cast<cudaStream_t>(stream));
 }
 
+
+namespace {
+// Checks a span link and puts it into the kernel parameters: a linked launch orders itself
+// span by span, so it never waits for the previous kernel as a whole (kp->overlap).
+int apply_link(const topkv_span_link* link, KParams* kp) {
+  if (link == nullptr || link->struct_size != sizeof(topkv_span_link) || link->reserved != 0)
+    return TOPKV_ERR_INVALID_ARG;
+  if (link->d_await == nullptr && link->d_signal == nullptr) return TOPKV_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(link->d_await) | reinterpret_cast<uintptr_t>(link->d_signal)) & 3)
+    return TOPKV_ERR_ALIGNMENT;
+  kp->link_await = link->d_await;
+  kp->link_signal = link->d_signal;
+  kp->await_epoch = (int)link->await_epoch;
+  kp->signal_epoch = (int)link->signal_epoch;
+  kp->overlap = 1;
+  kp->late_wait = 0;
+  return TOPKV_OK;
+}
+}  // namespace
+
+int64_t topkv_span_link_words(const topkv_layout* layout, const topkv_batch* batch) {
+  Resolved rs;
+  int st = check_layout(layout, &rs);
+  if (st != TOPKV_OK) return st;
+  st = check_batch(layout, batch);
+  if (st != TOPKV_OK) return st;
+  KParams kp = {};
+  kp.R = batch->num_requests;
+  kp.maxp = batch->max_pages_per_req;
+  kp.P = (int)layout->page_tokens;
+  if ((int64_t)kp.R * kp.maxp == 0) return 0;
+  span_geometry(&kp, (int)layout->kv_factor, rs.row_bytes);
+  return (int64_t)kp.R * kp.spr;
+}
+
+int topkv_pack_layer_linked(int layer, const void* src_pool, const topkv_layout* layout,
+                            const topkv_batch* batch, void* d_wire, int64_t wire_capacity_bytes,
+                            const topkv_span_link* link, topkv_stream_t stream) {
+  KParams kp;
+  Resolved rs;
+  int64_t n_layer;
+  int st = prepare(layer, src_pool, layout, batch, d_wire, wire_capacity_bytes,
+                   layout ? layout->wire_layer_stride : 0, &kp, &rs, &n_layer);
+  if (st != TOPKV_OK) return st;
+  st = apply_link(link, &kp);
+  if (st != TOPKV_OK) return st;
+  return launch_copy<true>(kp, rs, (int)layout->kv_factor, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int topkv_unpack_layer_linked(int layer, void* dst_pool, const topkv_layout* layout,
+                              const topkv_batch* batch, const void* d_wire, int64_t wire_bytes,
+                              const topkv_span_link* link, topkv_stream_t stream) {
+  KParams kp;
+  Resolved rs;
+  int64_t n_layer;
+  int st = prepare(layer, dst_pool, layout, batch, d_wire, wire_bytes,
+                   layout ? layout->wire_layer_stride : 0, &kp, &rs, &n_layer);
+  if (st != TOPKV_OK) return st;
+  st = apply_link(link, &kp);
+  if (st != TOPKV_OK) return st;
+  return launch_copy<false>(kp, rs, (int)layout->kv_factor, reinterpret_cast<cudaStream_t>(stream));
+}
 
 int topkv_pack_layers(int first_layer, int num_layers, const void* src_pool, const topkv_layout* layout,
                       const topkv_batch* batch, void* d_wire, int64_t wire_capacity_bytes,

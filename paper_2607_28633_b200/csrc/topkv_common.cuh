@@ -38,6 +38,10 @@ struct KParams {
   int overlap;            // 1: caller declared this launch independent of the kernels before it
   int late_wait;          // 1: tables are settled, wait for the previous kernel only before touching data
   int64_t S_layer, W_layer;  // multi-layer launch: bytes from one layer's slab to the next (pool, wire)
+  // span links: ordering against an earlier kernel span by span instead of grid by grid
+  const int32_t* link_await;  // flags this launch waits for, one per span, or nullptr
+  int32_t* link_signal;       // flags this launch publishes, one per span, or nullptr
+  int await_epoch, signal_epoch;
 };
 
 // Error bits raised by kernels (never a trap): read back with topkv_device_error_flags().
@@ -68,6 +72,21 @@ __device__ __forceinline__ void pdl_prologue(int overlap) {
 }
 __device__ __forceinline__ void pdl_epilogue(int overlap) {
   if (overlap && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) pdl_wait_prior_grid();
+}
+
+// Span links. A linked launch does not wait for the kernel before it as a whole: every CTA waits
+// (bounded) until the flag of ITS span holds the epoch it expects, and publishes its own span's
+// flag once its stores are issued. Programmatic dependent launch makes this safe: a kernel's
+// CTAs are only scheduled once every CTA of all earlier kernels of the stream has started, so
+// the CTA that a waiter depends on is resident or finished and never waits for the waiter.
+constexpr uint32_t kLinkPollLimit = 1u << 19;  // a poll is a 100 ns pause and one load: gives up after about half a second
+__device__ __forceinline__ int ld_acquire_gpu(const int32_t* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_gpu(int32_t* p, int v) {
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
 // Streaming vector accesses: every byte is touched exactly once, so neither side should

@@ -54,11 +54,13 @@ __device__ __forceinline__ int64_t block_prefix(const int32_t* __restrict__ sl, 
 // One CTA per (request, page column). F: planes per token; PACK: pool -> wire, else
 // wire -> pool; MERGED: the valid tokens of a page form one contiguous run per plane on
 // both sides (MLA rows, or PLANAR wire with a token-contiguous pool).
+// Returns (uniformly over the CTA) whether the span holds any token this layer keeps.
 template <int F, bool PACK, bool MERGED, int VEC, bool MULTI>
-__device__ __forceinline__ void copy_span(const KParams& p, const int slot) {
+__device__ __forceinline__ bool copy_span_work(const KParams& p, const int slot) {
   // A span = `ppc` consecutive page columns of one request (one page when pages are large;
   // several small pages, so that every CTA moves a few tens of KiB).
   __shared__ int32_t s_pages[kMaxPagesPerCta];
+  __shared__ int s_link_failed;
   // blockIdx.y = layer of a multi-layer launch (0 and zero strides for a single layer)
   uint8_t* const pool = p.pool + (int64_t)blockIdx.y * p.S_layer;
   uint8_t* const wire = p.wire + (int64_t)blockIdx.y * p.W_layer;
@@ -86,7 +88,14 @@ __device__ __forceinline__ void copy_span(const KParams& p, const int slot) {
     if (tid == 0 && sidx == 0) raise_error(kErrTable);
   }
   const int lo = max(first, b_r);
-  if (lo >= hi) return;
+  if (lo >= hi) return false;
+  // linked launch: ask for this span's flag now, so that the answer travels while the rest of
+  // the tables is read; it is looked at (and asked for again, if need be) just before data is
+  // touched
+  const int32_t* const link_flag =
+      p.link_await != nullptr ? p.link_await + ((int64_t)blockIdx.y * gridDim.x + slot) : nullptr;
+  int link_seen = 0;
+  if (link_flag != nullptr && tid == 0) link_seen = ld_acquire_gpu(link_flag);
   const int v = hi - lo;                // kept tokens in this span
   const int ts0 = lo - j0 * p.P;        // where they start, counted from the start of page column j0
   const int jlo = ts0 / p.P, jhi = (ts0 + v - 1) / p.P;  // page columns (relative to j0) they touch
@@ -122,11 +131,31 @@ __device__ __forceinline__ void copy_span(const KParams& p, const int slot) {
                                : (n0 >= 0 && (n0 + v) * F * row <= p.wire_limit);
     if (!fits) {
       if (tid == 0) raise_error(kErrWire);
-      return;
+      return true;
     }
   }
   // tables read, addresses known: from here on the pool and the wire are touched
   if (p.late_wait) pdl_wait_prior_grid();
+  if (p.link_await != nullptr) {  // wait for this span's flag, not for the whole kernel before
+    if (tid == 0) {
+      uint32_t polls = 0;
+      int failed = 0;
+      while (link_seen != p.await_epoch) {
+        if (++polls > kLinkPollLimit) {
+          failed = 1;
+          break;
+        }
+        __nanosleep(100);
+        link_seen = ld_acquire_gpu(link_flag);
+      }
+      s_link_failed = failed;
+    }
+    __syncthreads();
+    if (s_link_failed) {  // the span is skipped and reported; nothing was touched
+      if (tid == 0) raise_error(kErrWait);
+      return true;
+    }
+  }
   constexpr int kUnroll = VEC == 32 ? kUnroll32 : kUnroll16;
 
   if (MERGED) {
@@ -159,7 +188,7 @@ __device__ __forceinline__ void copy_span(const KParams& p, const int slot) {
         }
       }
     }
-    return;
+    return true;
   }
 
   // Units of the span in wire order: q = (ts*F + c)*U + h (TOKEN_KV) or q = (c*v + ts)*U + h
@@ -169,9 +198,9 @@ __device__ __forceinline__ void copy_span(const KParams& p, const int slot) {
   const int groups = kThreads / tpu;
   const int my_g = tid / tpu;
   const int my_w = tid - my_g * tpu;
-  if (my_g >= groups) return;
+  if (my_g >= groups) return true;
   uint8_t* wire_span = wire + n0 * F * p.U * unit_bytes;  // TOKEN_KV: the span is one run
-  if (!MULTI && s_pages[0] < 0) return;                     // single page, unusable: skip it
+  if (!MULTI && s_pages[0] < 0) return true;                // single page, unusable: skip it
   uint8_t* page0 = pool + (int64_t)s_pages[0] * p.S_page + (int64_t)ts0 * p.S_tok;
 
   for (int q0 = my_g; q0 < nunits; q0 += groups * kUnroll) {
@@ -217,6 +246,20 @@ __device__ __forceinline__ void copy_span(const KParams& p, const int slot) {
         if (ok[u]) buf[u].store(dstp[u]);
       }
     }
+  }
+  return true;
+}
+
+// One span, and, for a linked launch, the publication of its flag once every thread of the CTA
+// has issued its stores (spans without kept tokens publish nothing: their consumers, which see
+// the same lengths, do not wait for them either).
+template <int F, bool PACK, bool MERGED, int VEC, bool MULTI>
+__device__ __forceinline__ void copy_span(const KParams& p, const int slot) {
+  const bool nonempty = copy_span_work<F, PACK, MERGED, VEC, MULTI>(p, slot);
+  if (p.link_signal != nullptr && nonempty) {
+    __syncthreads();  // every thread's stores are ordered before thread 0's release below
+    if (threadIdx.x == 0)
+      st_release_gpu(p.link_signal + ((int64_t)blockIdx.y * gridDim.x + slot), p.signal_epoch);
   }
 }
 

@@ -482,3 +482,27 @@ def test_layer_table_offsets_and_validation_without_gpu(golden):
         7, 2, pool, lq, b, tq, wire, total, 0xA000000, biggest) == tk.TOPKV_ERR_LAYER_RANGE
     assert tk.topkv_kernel_launch_count() == before
     assert P(0, 0, pool, lq, b, tq, wire, total) == tk.TOPKV_OK                     # empty range
+
+
+def test_span_link_validation_without_gpu():
+    lo, b = _gqa(wire_layer_stride=1_785_856), _batch()
+    pool, wire, cap = 0x7000000, 0x9000000, 4 * 1_785_856
+    assert tk.topkv_span_link_words(lo, b) == 4 * 16                    # one 64 KiB page per span
+    small = tk.make_layout(4, 2, 1, 128, 2, 16, 64)                     # 8 KiB pages: 8 per span
+    assert tk.topkv_span_link_words(small, b) == 4 * 2
+    huge = tk.make_layout(4, 2, 8, 128, 2, 256, 64)                     # 1 MiB pages: 16 CTAs each
+    assert tk.topkv_span_link_words(huge, _batch(maxp=2, T=-1)) == 4 * 2 * 16
+    assert tk.topkv_span_link_words(lo, tk.make_batch(_FakeTensor(0, (0, 16)), _FakeTensor(0, (0,)), 0)) == 0
+    P, U = tk.topkv_pack_layer_linked, tk.topkv_unpack_layer_linked
+    flags = 0xC000000
+    before = tk.topkv_kernel_launch_count()
+    ok = tk.make_span_link(None, 0, flags, 1)
+    assert P(4, pool, lo, b, wire, cap, ok) == tk.TOPKV_ERR_LAYER_RANGE
+    assert U(3, pool, lo, b, wire, cap - 1, ok) == tk.TOPKV_ERR_CAPACITY
+    assert P(0, pool, lo, b, wire, cap, tk.make_span_link(None, 0, None, 0)) == tk.TOPKV_ERR_INVALID_ARG
+    bad = tk.make_span_link(flags, 1, None, 0); bad.struct_size = 4
+    assert U(0, pool, lo, b, wire, cap, bad) == tk.TOPKV_ERR_INVALID_ARG
+    bad = tk.make_span_link(flags, 1, None, 0); bad.reserved = 1
+    assert U(0, pool, lo, b, wire, cap, bad) == tk.TOPKV_ERR_INVALID_ARG
+    assert U(0, pool, lo, b, wire, cap, tk.make_span_link(flags + 2, 1, None, 0)) == tk.TOPKV_ERR_ALIGNMENT
+    assert tk.topkv_kernel_launch_count() == before

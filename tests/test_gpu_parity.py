@@ -1767,3 +1767,122 @@ def test_qwen_shaped_hybrid_with_state_layers_through_the_host(dev):
     oracle.unpack_layered(g, kinds, d["pool"], d["bt"], sl, want, d["sp"], S_sl, state, d["slots"])
     assert np.array_equal(d["d_pool"].cpu().numpy(), d["pool"])
     assert np.array_equal(d["d_sp"].cpu().numpy(), d["sp"])
+
+
+# -------------------------------------------------------------------- span links
+
+def _linked_chain(w, lo1, slab, stream, flags_p, flags_u, epoch0, layers):
+    """pack(l) -> unpack(l) -> pack(l+1) -> ... through ONE slab, every launch linked span by span
+    to the one it depends on: unpack(l) awaits pack(l); pack(l+1) awaits unpack(l)."""
+    b = w.batch
+    bs = tk.make_batch(w.src_bt, w.seq_lens, b.total_tokens, w.cu)
+    bd = tk.make_batch(w.dst_bt, w.seq_lens, b.total_tokens, w.cu)
+    e = epoch0
+    for k, l in enumerate(layers):
+        lp = tk.make_span_link(flags_u if e else None, e, flags_p, e + 1)   # e = 0: nothing before it
+        tk.check(tk.topkv_pack_layer_linked(l, w.src_pool, lo1, bs, slab, slab.numel(), lp, stream))
+        lu = tk.make_span_link(flags_p, e + 1, flags_u, e + 1)
+        tk.check(tk.topkv_unpack_layer_linked(l, w.dst_pool, lo1, bd, slab, slab.numel(), lu, stream))
+        e += 1
+    return e
+
+
+def test_span_linked_chain_through_one_slab(dev, variant):
+    """Every kernel of the chain depends on the DATA of the kernel just before it (one shared
+    wire slab), none waits for its predecessor as a whole: they are ordered span by span. The
+    destination pool is the oracle's unpack of the oracle's pack for every layer, twice over
+    (the flag arrays are reused with increasing epochs), with a copy right behind the chain."""
+    if variant == 1:
+        pytest.skip("span links belong to the vectorised family")
+    spec = wl.with_layers(wl.CFG2, 6)
+    w = harness.setup(spec, dev, need_wire=False)
+    b, s = w.batch, spec
+    g = _geom(s, b.num_pool_pages, 1, 0, 0)
+    stream = torch.cuda.Stream(dev)
+    lo1 = tk.make_layout(s.L, s.F, s.H, s.D, s.E, s.P, b.num_pool_pages)   # wire_layer_stride 0
+    slab = torch.zeros(w.n_layer, dtype=torch.uint8, device=dev)
+    words = tk.topkv_span_link_words(lo1, w.src_batch)
+    assert words == s.R * b.max_pages_per_req                            # one 64 KiB page per span
+    flags_p = torch.zeros(words, dtype=torch.int32, device=dev)
+    flags_u = torch.zeros(words, dtype=torch.int32, device=dev)
+    host_dst = torch.empty(w.dst_pool.numel(), dtype=torch.uint8).pin_memory()
+    dst_before = [harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, l) for l in range(s.L)]
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        e = _linked_chain(w, lo1, slab, stream, flags_p, flags_u, 0, range(s.L))
+        e = _linked_chain(w, lo1, slab, stream, flags_p, flags_u, e, reversed(range(s.L)))
+        host_dst.copy_(w.dst_pool, non_blocking=True)
+    stream.synchronize()
+    assert tk.topkv_device_error_flags() == 0
+    assert int(flags_p.max()) == e and int(flags_u.max()) == e
+    for l in range(s.L):
+        src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, l)
+        want = oracle.pack(g, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=8)
+        oracle.unpack(g, 0, dst_before[l], b.dst_block_table, b.seq_lens, want, impl="rows", threads=8)
+        assert np.array_equal(host_dst[l * w.slab_bytes:(l + 1) * w.slab_bytes].numpy(), dst_before[l]), l
+    del w
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_span_linked_pairs_random_geometries(dev, seed, variant):
+    """Linked pack -> unpack pairs on small random geometries (empty requests and empty spans
+    publish and await nothing, windows, strided pools, grouped small pages, both wire orders)."""
+    if variant == 1:
+        pytest.skip("span links belong to the vectorised family")
+    g, sl, bt_s, bt_d, rng = _case(seed)
+    if seed % 2:
+        g.window = int(rng.choice([1, g.P, 2 * g.P + 1]))
+    T = g.kept_tokens(sl)
+    g.W_layer = g.wire_layer_bytes(T) + 16
+    lo = _layout_from_geom(g)
+    src_h = rng.integers(0, 256, g.L * g.S_layer, dtype=np.uint8)
+    dst_h = rng.integers(0, 256, g.L * g.S_layer, dtype=np.uint8)
+    src, dst = torch.from_numpy(src_h).to(dev), torch.from_numpy(dst_h).to(dev)
+    wire = torch.full((g.L * g.W_layer + 32,), 0x3C, dtype=torch.uint8, device=dev)
+    d_sl = torch.from_numpy(sl).to(dev)
+    bs = tk.make_batch(torch.from_numpy(bt_s).to(dev), d_sl, T, None, 0, g.window)
+    bd = tk.make_batch(torch.from_numpy(bt_d).to(dev), d_sl, T, None, 0, g.window)
+    words = tk.topkv_span_link_words(lo, bs)
+    assert words >= 0
+    flags = torch.zeros(max(words, 1) * g.L, dtype=torch.int32, device=dev)
+    stream = torch.cuda.Stream(dev)
+    stream.wait_stream(torch.cuda.current_stream(dev))
+    want = np.full(g.L * g.W_layer + 32, 0x3C, dtype=np.uint8)
+    for layer in range(g.L):
+        f = flags[layer * max(words, 1):(layer + 1) * max(words, 1)]
+        tk.check(tk.topkv_pack_layer_linked(layer, src, lo, bs, wire, wire.numel(),
+                                            tk.make_span_link(None, 0, f, 7), stream))
+        tk.check(tk.topkv_unpack_layer_linked(layer, dst, lo, bd, wire, wire.numel(),
+                                              tk.make_span_link(f, 7, None, 0), stream))
+        oracle.pack(g, layer, src_h, bt_s, sl, wire=want)
+        oracle.unpack(g, layer, dst_h, bt_d, sl, want)
+    stream.synchronize()
+    assert np.array_equal(wire.cpu().numpy(), want)
+    assert np.array_equal(dst.cpu().numpy(), dst_h)
+
+
+def test_span_link_that_never_arrives_gives_up_and_reports(dev, variant):
+    """An unpack linked to flags that nothing publishes: every CTA's bounded wait runs out (about
+    half a second), the spans are skipped, bit 1 of the device status word is raised, the destination
+    pool is untouched and the context stays usable."""
+    if variant == 1:
+        pytest.skip("span links belong to the vectorised family")
+    w = harness.setup(wl.CFG1, dev)
+    before = w.dst_pool.cpu().numpy()
+    words = tk.topkv_span_link_words(w.layout, w.dst_batch)
+    flags = torch.zeros(words, dtype=torch.int32, device=dev)
+    torch.cuda.synchronize()
+    tk.check(tk.topkv_unpack_layer_linked(0, w.dst_pool, w.layout, w.dst_batch, w.wire, w.wire.numel(),
+                                          tk.make_span_link(flags, 5, None, 0)))
+    assert tk.topkv_device_error_flags() == 1
+    assert np.array_equal(w.dst_pool.cpu().numpy(), before)
+    tk.check(tk.topkv_reset_device_error_flags())
+    # the same call with the flags in place goes through
+    flags.fill_(5)
+    torch.cuda.synchronize()
+    tk.check(tk.topkv_pack_layer(0, w.src_pool, w.layout, w.src_batch, w.wire, w.wire.numel()))
+    tk.check(tk.topkv_unpack_layer_linked(0, w.dst_pool, w.layout, w.dst_batch, w.wire, w.wire.numel(),
+                                          tk.make_span_link(flags, 5, None, 0)))
+    assert tk.topkv_device_error_flags() == 0
+    assert not np.array_equal(w.dst_pool.cpu().numpy(), before)
