@@ -1063,11 +1063,16 @@ def main():
     torch.cuda.empty_cache()
     if world == 1 and args.extras:
         for name in [x for x in args.extras.split(",") if x]:
+            xs = ClockSampler(local)      # every extra carries the clocks seen while it ran
+            xs.start()
             try:
                 extra[name] = run_extra(name, dev, stream, args, peak)
             except Exception as e:  # an extra must not take the headline line down
                 extra[name] = {"error": f"{type(e).__name__}: {e}"}
                 torch.cuda.empty_cache()
+            c = xs.stop()
+            if isinstance(extra[name], dict):
+                extra[name]["clocks"] = {"sm_mhz": c.get("sm_mhz"), "reasons": c.get("reasons")}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

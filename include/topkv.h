@@ -218,8 +218,10 @@ int topkv_unpack_layer_from_host(int layer, void* dst_pool, const topkv_layout* 
  * half a second): a flag that never arrives raises bit 1 of topkv_device_error_flags() and skips the
  * span. Linked launches are safe because a kernel's CTAs are scheduled only after every CTA of
  * the earlier kernels of the stream has started: enqueue the linked calls on ONE stream, in
- * producer-before-consumer order, with no other work between them. Vectorised kernel family,
- * one layer per call. */
+ * producer-before-consumer order, with no other work between them. The epochs are plain
+ * arguments: a CUDA graph that captured linked calls replays the epochs of the capture, so such
+ * a graph must clear the flag arrays (a memset node) ahead of the linked calls of every replay.
+ * Vectorised kernel family, one layer per call. */
 typedef struct topkv_span_link {
   uint32_t struct_size;   /* = sizeof(topkv_span_link)               */
   uint32_t await_epoch;   /* value the awaited flags must reach      */
