@@ -336,11 +336,30 @@ def bench_host_leg(w, stream, pinned, staging, steps, warmup, barrier, slots, st
         slab = pinned[(l % slots) * n:(l % slots + 1) * n]
         tk.check(tk.topkv_unpack_layer_from_host(l, w.dst_pool, lo, w.dst_batch, slab, n, st, cap, q))
 
+    def two_lanes(fn, pool, batch):
+        """All layers through one library call that alternates between two streams and two
+        staging slabs (needs one pinned slab per layer)."""
+        lanes = [stream, second]
+        fork = torch.cuda.Event()
+        fork.record(stream)
+        second.wait_event(fork)
+        tk.check(fn(0, L, pool, w.layout, batch, pinned, L * n, [staging, staging2], cap, None, None,
+                    lanes))
+        join = torch.cuda.Event()
+        join.record(second)
+        stream.wait_event(join)
+
     def step(rec):
         e0 = torch.cuda.Event(enable_timing=True); e0.record(stream)
-        phase(to_host)
+        if second is not None and slots >= L:
+            two_lanes(tk.topkv_pack_layers_to_host_two_lanes, w.src_pool, w.src_batch)
+        else:
+            phase(to_host)
         e1 = torch.cuda.Event(enable_timing=True); e1.record(stream)
-        phase(from_host)
+        if second is not None and slots >= L:
+            two_lanes(tk.topkv_unpack_layers_from_host_two_lanes, w.dst_pool, w.dst_batch)
+        else:
+            phase(from_host)
         e2 = torch.cuda.Event(enable_timing=True); e2.record(stream)
         if rec is not None:
             rec.append((e0, e1, e2))
@@ -365,39 +384,33 @@ def bench_host_leg(w, stream, pinned, staging, steps, warmup, barrier, slots, st
 def bench_host_relay(w, stream, pinned, staging_tx, staging_rx, steps, warmup, barrier, slots):
     """The same layers through pinned host memory, pipelined the way a relay would run it: layer
     l is packed to the host while layers that have already arrived are unpacked from it, so both
-    directions of the PCIe link are busy. Each direction alternates between two streams with a
-    staging slab each, so that the copy engine moves layer l while the kernel of layer l + 1
-    runs. Returns ms per step (first pack enqueued to last unpack finished)."""
-    import ctypes
+    directions of the PCIe link are busy. The whole relay is two library calls
+    (topkv_pack_layers_to_host_two_lanes, topkv_unpack_layers_from_host_two_lanes): each direction
+    alternates between two streams with a staging slab each, so that the copy engine moves layer
+    l while the kernel of layer l + 1 runs, and the receiver's layer_ready events are the
+    sender's layer_done events. Returns ms per step (first pack enqueued to last unpack
+    finished)."""
     import torch
     from paper_2607_28633_b200 import binding as tk
     L, n = w.layers, w.n_layer
     dev = w.src_pool.device
-    lo = type(w.layout)()
-    ctypes.memmove(ctypes.byref(lo), ctypes.byref(w.layout), ctypes.sizeof(lo))
-    lo.wire_layer_stride = 0
     assert slots >= L, "the relay keeps every layer's slab until it is unpacked"
     tx = [torch.cuda.Stream(dev), torch.cuda.Stream(dev)]
     rx = [torch.cuda.Stream(dev), torch.cuda.Stream(dev)]
     st_tx = [staging_tx, torch.empty_like(staging_tx)]
     st_rx = [staging_rx, torch.empty_like(staging_rx)]
+    sent = [torch.cuda.Event() for _ in range(L)]
 
     def step():
         start = torch.cuda.Event()
         start.record(stream)
-        for q in tx:
+        for q in tx + rx:
             q.wait_event(start)
-        for l in range(L):
-            slab = pinned[l * n:(l + 1) * n]
-            a, b = tx[l & 1], rx[l & 1]
-            tk.check(tk.topkv_pack_layer_to_host(l, w.src_pool, lo, w.src_batch, slab, n, st_tx[l & 1],
-                                                 n, a))
-            arrived = torch.cuda.Event()
-            arrived.record(a)
-            b.wait_event(arrived)
-            tk.check(tk.topkv_unpack_layer_from_host(l, w.dst_pool, lo, w.dst_batch, slab, n,
-                                                     st_rx[l & 1], n, b))
-        for q in rx:                     # the step ends when the last unpacks have finished
+        tk.check(tk.topkv_pack_layers_to_host_two_lanes(
+            0, L, w.src_pool, w.layout, w.src_batch, pinned, L * n, st_tx, n, None, sent, tx))
+        tk.check(tk.topkv_unpack_layers_from_host_two_lanes(
+            0, L, w.dst_pool, w.layout, w.dst_batch, pinned, L * n, st_rx, n, sent, None, rx))
+        for q in tx + rx:                # the step ends when both directions have finished
             done = torch.cuda.Event()
             done.record(q)
             stream.wait_event(done)
@@ -632,7 +645,7 @@ def host_leg_forms(w, dev, stream, pinned, slots, steps):
     staging2 = torch.empty(w.n_layer, dtype=torch.uint8, device=dev)
     base = pinned_copy_baseline(dev, stream, w.n_layer)
     out = {}
-    for form, st, st2 in (("staged", staging, None), ("staged_two_streams", staging, staging2),
+    for form, st, st2 in (("staged", staging, None), ("staged_two_lanes", staging, staging2),
                           ("direct", None, None)):
         _, th, fh = bench_host_leg(w, stream, pinned, st, steps, 1, nobar, slots, st2)
         d2h = w.n_layer * w.layers / (th * 1e-3) / 1e9
@@ -1029,8 +1042,10 @@ def main():
             rms = bench_host_relay(w, stream, pinned, staging, staging_rx, hs, 1, barrier, slots)
             if rms < ems:
                 ems = rms
-                form = ("staged (kernel + copy engine), pipelined relay: layer l is unpacked from "
-                        "the host while later layers are still packed to it; one pinned slab per layer")
+                form = ("staged (kernel + copy engine), pipelined relay as two library calls "
+                        "(topkv_pack_layers_to_host_two_lanes, topkv_unpack_layers_from_host_two_lanes): "
+                        "layer l is unpacked from the host while later layers are still packed to it; "
+                        "one pinned slab per layer")
             del staging_rx
         ems_max = max_over_ranks(ems)
         e2e = {"value": round(bytes_step_all / (ems_max * 1e-3) / 1e9, 3), "unit": UNIT,

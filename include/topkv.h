@@ -377,6 +377,28 @@ int topkv_unpack_layers_from_host_pipelined(int first_layer, int num_layers, voi
                                             const topkv_event_t* layer_done,
                                             topkv_stream_t side_stream);
 
+/* The same schedule on TWO lanes (staged form only): layer i of the range goes to
+ * side_streams[i % 2] with d_stagings[i % 2] (HOST arrays of two entries each; the two streams and
+ * the two slabs must differ, each slab holds one layer), so that the copy engine moves one layer
+ * while the kernel of the next one runs: measured 1.000 / 0.997 of a pinned cudaMemcpyAsync where
+ * one lane reaches 0.98. layer_ready[i] is waited for and layer_done[i] recorded on the lane that
+ * ships layer i; order between the two lanes is the caller's (e.g. by waiting for the last two
+ * layer_done events). Errors as for the one-lane calls. */
+int topkv_pack_layers_to_host_two_lanes(int first_layer, int num_layers, const void* src_pool,
+                                        const topkv_layout* layout, const topkv_batch* batch,
+                                        void* h_pinned, int64_t host_capacity_bytes,
+                                        void* const* d_stagings, int64_t staging_capacity_bytes,
+                                        const topkv_event_t* layer_ready,
+                                        const topkv_event_t* layer_done,
+                                        const topkv_stream_t* side_streams);
+int topkv_unpack_layers_from_host_two_lanes(int first_layer, int num_layers, void* dst_pool,
+                                            const topkv_layout* layout, const topkv_batch* batch,
+                                            const void* h_pinned, int64_t host_bytes,
+                                            void* const* d_stagings, int64_t staging_capacity_bytes,
+                                            const topkv_event_t* layer_ready,
+                                            const topkv_event_t* layer_done,
+                                            const topkv_stream_t* side_streams);
+
 /* Host-side retry policy of the transfer orchestrator (§3.1: 2 retries, 100 ms exponential
  * backoff): calls attempt(ctx) until it returns TOPKV_OK, at most 1 + retries times, sleeping
  * backoff_ms, 2*backoff_ms, ... between attempts. Returns the last status. */

@@ -50,6 +50,7 @@ EXPORTS = (
     "topkv_unpack_model_layers", "topkv_pack_model_layers_to_host_pipelined",
     "topkv_unpack_model_layers_from_host_pipelined", "topkv_span_link_words",
     "topkv_pack_layer_linked", "topkv_unpack_layer_linked",
+    "topkv_pack_layers_to_host_two_lanes", "topkv_unpack_layers_from_host_two_lanes",
 )
 
 
@@ -220,6 +221,9 @@ def lib() -> ctypes.CDLL:
         L.topkv_set_host_leg_ctas.argtypes = [c_int]
         L.topkv_pack_layers.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p]
         L.topkv_unpack_layers.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p]
+        for fn in (L.topkv_pack_layers_to_host_two_lanes, L.topkv_unpack_layers_from_host_two_lanes):
+            fn.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p, c_int64,
+                           c_void_p, c_void_p, c_void_p]
         kp_ = ctypes.POINTER(topkv_span_link)
         L.topkv_span_link_words.argtypes = [lp, bp]
         L.topkv_span_link_words.restype = c_int64
@@ -449,6 +453,31 @@ def topkv_unpack_model_layers_from_host_pipelined(first_layer, num_layers, dst_p
         first_layer, num_layers, _ptr(dst_pool), ctypes.byref(layout), ctypes.byref(batch),
         ctypes.byref(table), _ptr(h_pinned), host_bytes, _ptr(d_staging), staging_capacity_bytes,
         _events(layer_ready, num_layers), _events(layer_done, num_layers), _stream(side_stream))
+
+
+def _two(ptrs, conv):
+    arr = (c_void_p * 2)()
+    arr[0], arr[1] = conv(ptrs[0]), conv(ptrs[1])
+    return arr
+
+
+def topkv_pack_layers_to_host_two_lanes(first_layer, num_layers, src_pool, layout, batch, h_pinned,
+                                        host_capacity_bytes, d_stagings, staging_capacity_bytes,
+                                        layer_ready=None, layer_done=None, side_streams=None):
+    """d_stagings and side_streams: sequences of two device slabs / two streams."""
+    return lib().topkv_pack_layers_to_host_two_lanes(
+        first_layer, num_layers, _ptr(src_pool), ctypes.byref(layout), ctypes.byref(batch),
+        _ptr(h_pinned), host_capacity_bytes, _two(d_stagings, _ptr), staging_capacity_bytes,
+        _events(layer_ready, num_layers), _events(layer_done, num_layers), _two(side_streams, _stream))
+
+
+def topkv_unpack_layers_from_host_two_lanes(first_layer, num_layers, dst_pool, layout, batch, h_pinned,
+                                            host_bytes, d_stagings, staging_capacity_bytes,
+                                            layer_ready=None, layer_done=None, side_streams=None):
+    return lib().topkv_unpack_layers_from_host_two_lanes(
+        first_layer, num_layers, _ptr(dst_pool), ctypes.byref(layout), ctypes.byref(batch),
+        _ptr(h_pinned), host_bytes, _two(d_stagings, _ptr), staging_capacity_bytes,
+        _events(layer_ready, num_layers), _events(layer_done, num_layers), _two(side_streams, _stream))
 
 
 def topkv_pack_layer_to_host_noalloc(layer, src_pool, layout, batch, h_pinned,

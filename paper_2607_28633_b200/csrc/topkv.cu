@@ -599,24 +599,34 @@ int check_layer_range(int first_layer, int num_layers, const void* pool, const t
   return TOPKV_OK;
 }
 
+// lanes = 1: every layer on streams[0] with stagings[0]. lanes = 2: layer i of the range on
+// streams[i % 2] with stagings[i % 2] (staged form only), so that the copy engine moves one
+// layer while the kernel of the next one runs.
 template <bool PACK>
 int issue_layers(int first_layer, int num_layers, const void* pool, const topkv_layout* layout,
-                 const topkv_batch* batch, const void* h_pinned, int64_t host_bytes, void* d_staging,
+                 const topkv_batch* batch, const void* h_pinned, int64_t host_bytes, void* const* stagings,
                  int64_t staging_capacity_bytes, const topkv_event_t* layer_ready,
-                 const topkv_event_t* layer_done, topkv_stream_t side_stream) {
-  int st = check_layer_range(first_layer, num_layers, pool, layout, batch, h_pinned, host_bytes, d_staging,
-                             staging_capacity_bytes);
-  if (st != TOPKV_OK) return st;
-  cudaStream_t s = reinterpret_cast<cudaStream_t>(side_stream);
+                 const topkv_event_t* layer_done, const topkv_stream_t* streams, int lanes) {
+  if (stagings == nullptr || streams == nullptr) return TOPKV_ERR_INVALID_ARG;
+  for (int q = 0; q < lanes; ++q) {
+    if (lanes > 1 && stagings[q] == nullptr) return TOPKV_ERR_INVALID_ARG;  // two lanes: staged form only
+    const int st = check_layer_range(first_layer, num_layers, pool, layout, batch, h_pinned, host_bytes,
+                                     stagings[q], staging_capacity_bytes);
+    if (st != TOPKV_OK) return st;
+  }
+  if (lanes > 1 && (stagings[0] == stagings[1] || streams[0] == streams[1])) return TOPKV_ERR_INVALID_ARG;
   for (int i = 0; i < num_layers; ++i) {
+    const int q = i % lanes;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(streams[q]);
     if (layer_ready != nullptr && layer_ready[i] != nullptr) {
       const cudaError_t e = cudaStreamWaitEvent(s, reinterpret_cast<cudaEvent_t>(layer_ready[i]), 0);
       if (e != cudaSuccess) return cuda_fail(e);
     }
-    st = PACK ? topkv_pack_layer_to_host(first_layer + i, pool, layout, batch, const_cast<void*>(h_pinned),
-                                         host_bytes, d_staging, staging_capacity_bytes, side_stream)
-              : topkv_unpack_layer_from_host(first_layer + i, const_cast<void*>(pool), layout, batch, h_pinned,
-                                             host_bytes, d_staging, staging_capacity_bytes, side_stream);
+    const int st =
+        PACK ? topkv_pack_layer_to_host(first_layer + i, pool, layout, batch, const_cast<void*>(h_pinned),
+                                        host_bytes, stagings[q], staging_capacity_bytes, streams[q])
+             : topkv_unpack_layer_from_host(first_layer + i, const_cast<void*>(pool), layout, batch, h_pinned,
+                                            host_bytes, stagings[q], staging_capacity_bytes, streams[q]);
     if (st != TOPKV_OK) return st;
     if (layer_done != nullptr && layer_done[i] != nullptr) {
       const cudaError_t e = cudaEventRecord(reinterpret_cast<cudaEvent_t>(layer_done[i]), s);
@@ -1149,7 +1159,26 @@ int topkv_pack_layers_to_host_pipelined(int first_layer, int num_layers, const v
                                         const topkv_event_t* layer_ready,
                                         const topkv_event_t* layer_done, topkv_stream_t side_stream) {
   return issue_layers<true>(first_layer, num_layers, src_pool, layout, batch, h_pinned, host_capacity_bytes,
-                            d_staging, staging_capacity_bytes, layer_ready, layer_done, side_stream);
+                            &d_staging, staging_capacity_bytes, layer_ready, layer_done, &side_stream, 1);
+}
+
+int topkv_pack_layers_to_host_two_lanes(int first_layer, int num_layers, const void* src_pool,
+                                        const topkv_layout* layout, const topkv_batch* batch,
+                                        void* h_pinned, int64_t host_capacity_bytes, void* const* d_stagings,
+                                        int64_t staging_capacity_bytes, const topkv_event_t* layer_ready,
+                                        const topkv_event_t* layer_done, const topkv_stream_t* side_streams) {
+  return issue_layers<true>(first_layer, num_layers, src_pool, layout, batch, h_pinned, host_capacity_bytes,
+                            d_stagings, staging_capacity_bytes, layer_ready, layer_done, side_streams, 2);
+}
+
+int topkv_unpack_layers_from_host_two_lanes(int first_layer, int num_layers, void* dst_pool,
+                                            const topkv_layout* layout, const topkv_batch* batch,
+                                            const void* h_pinned, int64_t host_bytes, void* const* d_stagings,
+                                            int64_t staging_capacity_bytes, const topkv_event_t* layer_ready,
+                                            const topkv_event_t* layer_done,
+                                            const topkv_stream_t* side_streams) {
+  return issue_layers<false>(first_layer, num_layers, dst_pool, layout, batch, h_pinned, host_bytes, d_stagings,
+                             staging_capacity_bytes, layer_ready, layer_done, side_streams, 2);
 }
 
 int topkv_unpack_layers_from_host_pipelined(int first_layer, int num_layers, void* dst_pool,
@@ -1160,7 +1189,7 @@ int topkv_unpack_layers_from_host_pipelined(int first_layer, int num_layers, voi
                                             const topkv_event_t* layer_done,
                                             topkv_stream_t side_stream) {
   return issue_layers<false>(first_layer, num_layers, dst_pool, layout, batch, h_pinned, host_bytes,
-                             d_staging, staging_capacity_bytes, layer_ready, layer_done, side_stream);
+                             &d_staging, staging_capacity_bytes, layer_ready, layer_done, &side_stream, 1);
 }
 
 int topkv_layer_table_offsets(const topkv_layout* layout, const topkv_layer_table* table,

@@ -1886,3 +1886,52 @@ def test_span_link_that_never_arrives_gives_up_and_reports(dev, variant):
                                           tk.make_span_link(flags, 5, None, 0)))
     assert tk.topkv_device_error_flags() == 0
     assert not np.array_equal(w.dst_pool.cpu().numpy(), before)
+
+
+def test_two_lane_host_leg_relay(dev):
+    """topkv_pack_layers_to_host_two_lanes / topkv_unpack_layers_from_host_two_lanes: the whole
+    relay through pinned memory as two calls, each direction alternating between two streams and
+    two staging slabs, the receiver gated by the sender's per-layer events. Pinned slabs and
+    destination pool equal the oracle's, for an odd number of layers and for a sub-range."""
+    L = 5
+    spec = wl.with_layers(wl.CFG2, L)
+    w = harness.setup(spec, dev, need_wire=False)
+    b = w.batch
+    g = _geom(spec, b.num_pool_pages, 1, 0, 0)
+    n = w.n_layer
+    pinned = torch.zeros(L * n, dtype=torch.uint8).pin_memory()
+    tx = [torch.cuda.Stream(dev), torch.cuda.Stream(dev)]
+    rx = [torch.cuda.Stream(dev), torch.cuda.Stream(dev)]
+    st_tx = [torch.empty(n, dtype=torch.uint8, device=dev) for _ in range(2)]
+    st_rx = [torch.empty(n, dtype=torch.uint8, device=dev) for _ in range(2)]
+    before = [harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, l) for l in range(L)]
+    torch.cuda.synchronize()
+    sent = [torch.cuda.Event() for _ in range(L)]
+    # layers 1..4 first, then layer 0 on its own
+    tk.check(tk.topkv_pack_layers_to_host_two_lanes(1, L - 1, w.src_pool, w.layout, w.src_batch, pinned,
+                                                    pinned.numel(), st_tx, n, None, sent[1:], tx))
+    tk.check(tk.topkv_pack_layers_to_host_two_lanes(0, 1, w.src_pool, w.layout, w.src_batch, pinned,
+                                                    pinned.numel(), st_tx, n, None, sent[:1], tx))
+    tk.check(tk.topkv_unpack_layers_from_host_two_lanes(0, L, w.dst_pool, w.layout, w.dst_batch, pinned,
+                                                        pinned.numel(), st_rx, n, sent, None, rx))
+    torch.cuda.synchronize()
+    assert tk.topkv_device_error_flags() == 0
+    for layer in range(L):
+        src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, layer)
+        want = oracle.pack(g, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=8)
+        assert np.array_equal(pinned[layer * n:(layer + 1) * n].numpy(), want), layer
+        oracle.unpack(g, 0, before[layer], b.dst_block_table, b.seq_lens, want, impl="rows", threads=8)
+        assert np.array_equal(harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, layer), before[layer])
+    # refused before anything is enqueued: one slab or one stream given twice, a missing slab
+    launches = tk.topkv_kernel_launch_count()
+    P2 = tk.topkv_pack_layers_to_host_two_lanes
+    args = (0, L, w.src_pool, w.layout, w.src_batch, pinned, pinned.numel())
+    assert P2(*args, [st_tx[0], st_tx[0]], n, None, None, tx) == tk.TOPKV_ERR_INVALID_ARG
+    assert P2(*args, st_tx, n, None, None, [tx[0], tx[0]]) == tk.TOPKV_ERR_INVALID_ARG
+    assert P2(*args, [st_tx[0], None], n, None, None, tx) == tk.TOPKV_ERR_INVALID_ARG
+    assert P2(*args, st_tx, n - 16, None, None, tx) == tk.TOPKV_ERR_CAPACITY
+    assert P2(2, L, w.src_pool, w.layout, w.src_batch, pinned, pinned.numel(), st_tx, n, None, None, tx) \
+        == tk.TOPKV_ERR_LAYER_RANGE
+    assert tk.topkv_kernel_launch_count() == launches
+    del w
+    torch.cuda.empty_cache()
