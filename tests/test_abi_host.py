@@ -506,3 +506,23 @@ def test_span_link_validation_without_gpu():
     assert U(0, pool, lo, b, wire, cap, bad) == tk.TOPKV_ERR_INVALID_ARG
     assert U(0, pool, lo, b, wire, cap, tk.make_span_link(flags + 2, 1, None, 0)) == tk.TOPKV_ERR_ALIGNMENT
     assert tk.topkv_kernel_launch_count() == before
+
+
+def test_two_lane_host_leg_validation_without_gpu():
+    n = 1_785_856
+    lo, b = _gqa(wire_layer_stride=n), _batch()
+    pool, host = 0x7000000, 0x9000000
+    st, streams = [0xA000000, 0xA800000], [0x1000, 0x2000]
+    before = tk.topkv_kernel_launch_count()
+    for fn in (tk.topkv_pack_layers_to_host_two_lanes, tk.topkv_unpack_layers_from_host_two_lanes):
+        args = (pool, lo, b, host, 4 * n)
+        assert fn(0, 5, *args, st, n, None, None, streams) == tk.TOPKV_ERR_LAYER_RANGE
+        assert fn(0, 4, pool, lo, b, host, 4 * n - 1, st, n, None, None, streams) == tk.TOPKV_ERR_CAPACITY
+        assert fn(0, 4, *args, st, n - 1, None, None, streams) == tk.TOPKV_ERR_CAPACITY
+        assert fn(0, 4, *args, [st[0], st[0]], n, None, None, streams) == tk.TOPKV_ERR_INVALID_ARG
+        assert fn(0, 4, *args, [st[0], None], n, None, None, streams) == tk.TOPKV_ERR_INVALID_ARG
+        assert fn(0, 4, *args, st, n, None, None, [streams[0], streams[0]]) == tk.TOPKV_ERR_INVALID_ARG
+        assert fn(0, 4, *args, [st[0], st[1] + 8], n, None, None, streams) == tk.TOPKV_ERR_ALIGNMENT
+        assert fn(0, 4, pool, lo, _batch(T=-1), host, 4 * n, st, n, None, None, streams) \
+            == tk.TOPKV_ERR_INVALID_ARG
+    assert tk.topkv_kernel_launch_count() == before
