@@ -1030,7 +1030,9 @@ def main():
         # every layer through pinned host memory with the C-ABI host-leg calls: one slab per
         # layer (10 GiB for the 70B shape), or a ring of 4 slabs when the box refuses that much
         pinned = pinned_buffer(L * n_layer, 4 * n_layer)
-        slots = min(L, pinned.numel() // n_layer)
+        # every rank takes the same path (the barriers inside the timed legs must match): the
+        # smallest number of slabs any rank obtained decides
+        slots = int(round(-max_over_ranks(-float(min(L, pinned.numel() // n_layer)))))
         staging = torch.empty(n_layer, dtype=torch.uint8, device=dev)
         hs = max(1, min(args.steps, 3))
         ems, th, fh = bench_host_leg(w, stream, pinned, staging, hs, 1, barrier, slots)
