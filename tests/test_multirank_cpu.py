@@ -28,6 +28,9 @@ WORKER = textwrap.dedent("""
     gbs, ms = dist_util.aggregate_throughput(dist, bytes_rank, ms_rank)
     # every rank must also see the other's token count through the reduction
     tot_tokens = dist_util.sum_over_ranks(dist, float(b.total_tokens))
+    # bench.py's ranks agree on the smallest number of pinned slabs any of them obtained
+    slots = int(round(-dist_util.max_over_ranks(dist, -float(80 if rank == 0 else 4))))
+    assert slots == 4
     dist.barrier()
     print(json.dumps({{"rank": rank, "tokens": b.total_tokens, "gbs": gbs, "ms": ms,
                       "tot_tokens": tot_tokens,
