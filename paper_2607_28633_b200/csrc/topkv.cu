@@ -699,8 +699,12 @@ int check_table(const topkv_layout* lo, const topkv_batch* b, const topkv_layer_
   if (t == nullptr || t->struct_size != sizeof(topkv_layer_table) || t->specs == nullptr)
     return TOPKV_ERR_INVALID_ARG;
   if (lo == nullptr || b == nullptr) return TOPKV_ERR_INVALID_ARG;
+  if (lo->struct_size != sizeof(topkv_layout)) return TOPKV_ERR_INVALID_ARG;  // fields are read below
   if (b->struct_size != sizeof(topkv_batch) || b->window_tokens != 0) return TOPKV_ERR_INVALID_ARG;
+  if (b->num_requests < 0) return TOPKV_ERR_INVALID_ARG;
   if (b->num_requests > 0 && t->h_seq_lens == nullptr) return TOPKV_ERR_INVALID_ARG;
+  for (int r = 0; r < b->num_requests; ++r)
+    if (t->h_seq_lens[r] < 0) return TOPKV_ERR_INVALID_ARG;
   return TOPKV_OK;
 }
 
@@ -1198,6 +1202,8 @@ int topkv_layer_table_offsets(const topkv_layout* layout, const topkv_layer_tabl
       table->struct_size != sizeof(topkv_layer_table) || table->specs == nullptr || h_offsets == nullptr ||
       num_requests < 0 || (num_requests > 0 && table->h_seq_lens == nullptr))
     return TOPKV_ERR_INVALID_ARG;
+  for (int32_t r = 0; r < num_requests; ++r)
+    if (table->h_seq_lens[r] < 0) return TOPKV_ERR_INVALID_ARG;
   int64_t off = 0;
   for (uint32_t l = 0; l < table->num_layers; ++l) {
     h_offsets[l] = off;

@@ -451,6 +451,11 @@ def test_layer_table_offsets_and_validation_without_gpu(golden):
     assert P(0, 8, pool, lq, bw, tq, wire, total) == tk.TOPKV_ERR_INVALID_ARG       # the table sets windows
     bt_ = tk.make_batch(_FakeTensor(0x10000, (R, 4)), _FakeTensor(0x20000, (R,)), 58)
     assert P(0, 8, pool, lq, bt_, tq, wire, total) == tk.TOPKV_ERR_INVALID_ARG      # lengths disagree
+    neg = tk.make_layer_table(sq, np.array([40, -1, 17], dtype=np.int32), sp, slots, 64 * state, state, 64)
+    assert P(0, 8, pool, lq, b, neg, wire, total) == tk.TOPKV_ERR_INVALID_ARG      # a negative length
+    assert tk.topkv_layer_table_offsets(lq, neg, R)[0] == tk.TOPKV_ERR_INVALID_ARG
+    old = tk.make_layout(2, 2, 2, 256, 2, 16, 64); old.struct_size = 8
+    assert P(0, 8, pool, old, b, tq, wire, total) == tk.TOPKV_ERR_INVALID_ARG
     bad = tk.make_layer_table(sq, lens3, sp, slots, 64 * state, state, 64); bad.struct_size = 8
     assert P(0, 8, pool, lq, b, bad, wire, total) == tk.TOPKV_ERR_INVALID_ARG
     bad = tk.make_layer_table(sq, lens3, None, slots, 64 * state, state, 64)        # no state pool
