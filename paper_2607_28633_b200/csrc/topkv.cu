@@ -22,6 +22,7 @@
 #include <cstdint>
 #include <cstring>
 #include <mutex>
+#include <utility>
 #include <vector>
 
 namespace {
@@ -695,6 +696,22 @@ struct LayerPlan {
   bool empty = false;   // nothing to launch
 };
 
+// The tokens of the batch that a layer of a given kind keeps come from the host copy of the
+// lengths. Scratch of the call in progress on this thread (cleared at every entry point): the
+// sums are remembered per distinct window (a model has a handful), so a call costs one pass
+// over the lengths per window, not one per layer.
+thread_local struct {
+  const int32_t* lens = nullptr;
+  int R = -1;
+  std::vector<std::pair<int64_t, int64_t>> sums;  // (window or -1 for all tokens, tokens kept)
+} g_token_sums;
+
+void reset_token_sums(const topkv_layer_table* t, int R) {
+  g_token_sums.lens = t->h_seq_lens;
+  g_token_sums.R = R;
+  g_token_sums.sums.clear();
+}
+
 int check_table(const topkv_layout* lo, const topkv_batch* b, const topkv_layer_table* t) {
   if (t == nullptr || t->struct_size != sizeof(topkv_layer_table) || t->specs == nullptr)
     return TOPKV_ERR_INVALID_ARG;
@@ -705,16 +722,23 @@ int check_table(const topkv_layout* lo, const topkv_batch* b, const topkv_layer_
   if (b->num_requests > 0 && t->h_seq_lens == nullptr) return TOPKV_ERR_INVALID_ARG;
   for (int r = 0; r < b->num_requests; ++r)
     if (t->h_seq_lens[r] < 0) return TOPKV_ERR_INVALID_ARG;
+  if (lo->wire_plane_stride != 0) return TOPKV_ERR_UNSUPPORTED_LAYOUT;  // slabs lie back to back
+  reset_token_sums(t, b->num_requests);  // the lengths may have changed in place since the last call
   return TOPKV_OK;
 }
 
-// Tokens of the batch that a layer of this kind keeps, from the host copy of the lengths.
+// Tokens of the batch that a layer of this kind keeps (see g_token_sums).
 int64_t kept_tokens(const topkv_layer_table* t, int R, const topkv_layer_spec& sp) {
+  const int64_t key = sp.kind == TOPKV_LAYER_WINDOW ? sp.param : -1;
+  if (g_token_sums.lens != t->h_seq_lens || g_token_sums.R != R) reset_token_sums(t, R);
+  for (const auto& kv : g_token_sums.sums)
+    if (kv.first == key) return kv.second;
   int64_t total = 0;
   for (int r = 0; r < R; ++r) {
     const int64_t s = t->h_seq_lens[r];
-    total += (sp.kind == TOPKV_LAYER_WINDOW && sp.param < s) ? sp.param : s;
+    total += (key >= 0 && key < s) ? key : s;
   }
+  g_token_sums.sums.emplace_back(key, total);
   return total;
 }
 
@@ -1204,6 +1228,7 @@ int topkv_layer_table_offsets(const topkv_layout* layout, const topkv_layer_tabl
     return TOPKV_ERR_INVALID_ARG;
   for (int32_t r = 0; r < num_requests; ++r)
     if (table->h_seq_lens[r] < 0) return TOPKV_ERR_INVALID_ARG;
+  model::reset_token_sums(table, num_requests);
   int64_t off = 0;
   for (uint32_t l = 0; l < table->num_layers; ++l) {
     h_offsets[l] = off;
