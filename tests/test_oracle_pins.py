@@ -772,7 +772,7 @@ def test_transport_selection_reproduces_table4(golden):
         ratio = ms["rdma"] / ms[mode]
         want = float(g[f"table4.{mode}.vs_rdma"])
         assert round(ratio, 1 if want < 1 else 0) == want, (mode, ratio)
-    # §5.1's "3 to 18x over uniform RDMA": the upper end is the NVLink row; the lower end is
+    # §5.1 claims a reduction of 3x to 18x over RDMA everywhere: the upper end is the NVLink row; the lower end is
     # not reproducible from the paper's own table, whose PCIe row gives 52 / 26 = 2x
     assert round(ms["rdma"] / ms["nvlink"]) == int(g["s51.reduction_hi"])
     assert round(ms["rdma"] / ms["pcie"]) == 2 != int(g["s51.reduction_lo"])
