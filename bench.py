@@ -1073,6 +1073,22 @@ def main():
             e2e["from_host_frac_of_pinned_copy"] = hl["staged"]["from_host_frac_of_pinned_copy"]
         del pinned
 
+    if rank == 0:
+        # the paper's own quoted link rates and the rates its orchestrator plans with (§3.3,
+        # Table 2, Table 4): context for the figures above, measured on other hardware or not at
+        # all, never a target of this run
+        modes = (tk.TOPKV_TRANSPORT_NVLINK, tk.TOPKV_TRANSPORT_PCIE, tk.TOPKV_TRANSPORT_RDMA,
+                 tk.TOPKV_TRANSPORT_TCP)
+        extra["paper_context"] = {
+            "published_link_GBps": {"nvlink4_h100_domain": 900, "nvlink5_per_gpu": 1800,
+                                    "pcie_gen5_x16": 128, "infiniband_ndr": 50, "tcp_100gbe": 12.5},
+            "planning_GBps": {tk.topkv_transport_name(m): tk.topkv_planning_rate(m) / 1e9 for m in modes},
+            "eq2_ms_for_this_workload_per_request": {
+                tk.topkv_transport_name(m): round(tk.topkv_model_transfer_s(
+                    float(tk.topkv_kv_bytes(w.layout, 4096)) * head.L / max(1, w.layers),
+                    tk.topkv_planning_rate(m), 0.0) * 1e3, 2) for m in modes},
+            "note": "analytic or vendor figures quoted by the paper (H100-era hardware); no measured "
+                    "number for this path exists in the paper"}
     if rank == 0 and world == 1:
         extra["device_copy_GBps_same_bytes"] = round(device_copy_baseline(dev, stream, n_layer), 1)
     batch = w.batch
