@@ -779,6 +779,32 @@ def run_extra(name, dev, stream, args, peak):
                 r[label] = {"GBps": round(gbs, 1), "us_per_launch": round(us, 2),
                             "frac_of_hbm_peak": round(gbs / peak, 4),
                             "frac_of_8000_spec": round(gbs / 8000.0, 4)}
+            # the same one-slab linked chain as ONE library call per pass
+            words = tk.check(tk.topkv_span_link_words(w.layout, w.src_batch))
+            flags = torch.zeros(2 * words, dtype=torch.int32, device=dev)
+            slab = w.wire[:w.n_layer]
+            done, reps = 0, max(1, min(args.steps, 5))
+
+            def relay():
+                nonlocal done
+                tk.check(tk.topkv_relay_layers_linked(0, w.layers, w.src_pool, w.layout, w.src_batch,
+                                                      w.dst_pool, w.layout, w.dst_batch, slab, w.n_layer,
+                                                      flags, flags.numel(), done, stream))
+                done += w.layers
+            relay()
+            stream.synchronize()
+            ea, eb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ea.record(stream)
+            for _ in range(reps):
+                relay()
+            eb.record(stream)
+            stream.synchronize()
+            rms = ea.elapsed_time(eb) / reps
+            gbs = 4.0 * w.n_layer * w.layers / (rms * 1e-3) / 1e9
+            r["one_slab_relay_call"] = {"GBps": round(gbs, 1), "us_per_launch": round(rms / (2 * w.layers) * 1e3, 2),
+                                        "frac_of_hbm_peak": round(gbs / peak, 4),
+                                        "frac_of_8000_spec": round(gbs / 8000.0, 4)}
+            del flags
             out[base.name] = r
             del w
             torch.cuda.empty_cache()

@@ -239,6 +239,27 @@ int topkv_unpack_layer_linked(int layer, void* dst_pool, const topkv_layout* lay
                               const topkv_batch* batch, const void* d_wire, int64_t wire_bytes,
                               const topkv_span_link* link, topkv_stream_t stream);
 
+/* The whole relay of a range of layers through ONE wire slab as one call: for every layer,
+ * pack (source pool -> slab) and unpack (slab -> destination pool), all 2 * num_layers launches
+ * span-linked: unpack(l) follows pack(l) span by span, pack(l+1) overwrites a span of the slab as
+ * soon as unpack(l) has read it. This is the shape a transfer to another GPU has (pack into the
+ * receiver's slab, unpack there, §5.2) run on one GPU; where both pools are on this GPU and no
+ * wire is wanted, topkv_repage_layer moves half the bytes.
+ * The two sides must describe the same requests and cut them into the same spans: equal
+ * num_requests, max_pages_per_req, window_tokens, page_tokens, kv_factor, heads, head_dim,
+ * elem_bytes and wire order (else TOPKV_ERR_UNSUPPORTED_LAYOUT); block tables, strides and pool
+ * sizes may differ. wire_layer_stride of both layouts is ignored: d_slab (slab_bytes >= N_layer)
+ * is the slab of every layer. d_flags: DEVICE int32 [2 * topkv_span_link_words()], zeroed once by
+ * the caller; first_epoch = the number of layers already relayed through these flags since they
+ * were zeroed (0 the first time; the call uses epochs first_epoch + 1 .. first_epoch +
+ * num_layers). Everything is validated for every layer before the first launch. */
+int topkv_relay_layers_linked(int first_layer, int num_layers, const void* src_pool,
+                              const topkv_layout* src_layout, const topkv_batch* src_batch,
+                              void* dst_pool, const topkv_layout* dst_layout,
+                              const topkv_batch* dst_batch, void* d_slab, int64_t slab_bytes,
+                              int32_t* d_flags, int64_t flags_words, uint32_t first_epoch,
+                              topkv_stream_t stream);
+
 /* ---- direct re-paging (no wire slab) -------------------------------------------------------- */
 
 /* Moves layer `layer` of the batch from one paged pool straight into another paged pool with

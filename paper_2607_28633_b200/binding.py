@@ -51,6 +51,7 @@ EXPORTS = (
     "topkv_unpack_model_layers_from_host_pipelined", "topkv_span_link_words",
     "topkv_pack_layer_linked", "topkv_unpack_layer_linked",
     "topkv_pack_layers_to_host_two_lanes", "topkv_unpack_layers_from_host_two_lanes",
+    "topkv_relay_layers_linked",
 )
 
 
@@ -229,6 +230,8 @@ def lib() -> ctypes.CDLL:
         L.topkv_span_link_words.restype = c_int64
         L.topkv_pack_layer_linked.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64, kp_, c_void_p]
         L.topkv_unpack_layer_linked.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64, kp_, c_void_p]
+        L.topkv_relay_layers_linked.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, lp, bp, c_void_p,
+                                                c_int64, c_void_p, c_int64, c_uint32, c_void_p]
         tp = ctypes.POINTER(topkv_layer_table)
         L.topkv_layer_table_offsets.argtypes = [lp, tp, c_int32, c_void_p]
         L.topkv_pack_model_layers.argtypes = [c_int, c_int, c_void_p, lp, bp, tp, c_void_p, c_int64, c_void_p]
@@ -410,6 +413,15 @@ def topkv_unpack_layer_linked(layer, dst_pool, layout, batch, d_wire, wire_bytes
     return lib().topkv_unpack_layer_linked(layer, _ptr(dst_pool), ctypes.byref(layout),
                                            ctypes.byref(batch), _ptr(d_wire), wire_bytes,
                                            ctypes.byref(link), _stream(stream))
+
+
+def topkv_relay_layers_linked(first_layer, num_layers, src_pool, src_layout, src_batch, dst_pool,
+                              dst_layout, dst_batch, d_slab, slab_bytes, d_flags, flags_words,
+                              first_epoch, stream=None):
+    return lib().topkv_relay_layers_linked(
+        first_layer, num_layers, _ptr(src_pool), ctypes.byref(src_layout), ctypes.byref(src_batch),
+        _ptr(dst_pool), ctypes.byref(dst_layout), ctypes.byref(dst_batch), _ptr(d_slab), slab_bytes,
+        _ptr(d_flags), flags_words, first_epoch, _stream(stream))
 
 
 def topkv_layer_table_offsets(layout, table, num_requests):

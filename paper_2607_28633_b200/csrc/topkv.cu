@@ -1092,6 +1092,59 @@ int topkv_unpack_layer_linked(int layer, void* dst_pool, const topkv_layout* lay
   return launch_copy<false>(kp, rs, (int)layout->kv_factor, reinterpret_cast<cudaStream_t>(stream));
 }
 
+int topkv_relay_layers_linked(int first_layer, int num_layers, const void* src_pool,
+                              const topkv_layout* src_layout, const topkv_batch* src_batch, void* dst_pool,
+                              const topkv_layout* dst_layout, const topkv_batch* dst_batch, void* d_slab,
+                              int64_t slab_bytes, int32_t* d_flags, int64_t flags_words,
+                              uint32_t first_epoch, topkv_stream_t stream) {
+  if (first_layer < 0 || num_layers < 0) return TOPKV_ERR_LAYER_RANGE;
+  if (src_layout == nullptr || dst_layout == nullptr || src_layout->struct_size != sizeof(topkv_layout) ||
+      dst_layout->struct_size != sizeof(topkv_layout))
+    return TOPKV_ERR_INVALID_ARG;
+  const int64_t ws = topkv_span_link_words(src_layout, src_batch);
+  const int64_t wd = topkv_span_link_words(dst_layout, dst_batch);
+  if (ws < 0) return (int)ws;
+  if (wd < 0) return (int)wd;
+  // both sides must cut the batch into the same spans and agree on what a wire row is
+  if (ws != wd || src_layout->page_tokens != dst_layout->page_tokens ||
+      src_batch->num_requests != dst_batch->num_requests ||
+      src_batch->max_pages_per_req != dst_batch->max_pages_per_req ||
+      src_batch->window_tokens != dst_batch->window_tokens ||
+      src_layout->kv_factor != dst_layout->kv_factor || src_layout->num_kv_heads != dst_layout->num_kv_heads ||
+      src_layout->head_dim != dst_layout->head_dim || src_layout->elem_bytes != dst_layout->elem_bytes ||
+      src_layout->wire_order != dst_layout->wire_order ||
+      src_layout->wire_plane_stride != dst_layout->wire_plane_stride)
+    return TOPKV_ERR_UNSUPPORTED_LAYOUT;
+  if (ws > 0 && (d_flags == nullptr || flags_words < 2 * ws)) return d_flags == nullptr ? TOPKV_ERR_INVALID_ARG
+                                                                                        : TOPKV_ERR_CAPACITY;
+  if ((uint64_t)first_epoch + (uint64_t)num_layers > 0x7fffffffull) return TOPKV_ERR_INVALID_ARG;
+  topkv_layout ls = *src_layout, ld = *dst_layout;
+  ls.wire_layer_stride = 0;  // every layer goes through the one slab
+  ld.wire_layer_stride = 0;
+  // validate every layer on both sides before the first launch
+  KParams kp;
+  Resolved rs;
+  int64_t n_layer;
+  for (int i = 0; i < num_layers; ++i) {
+    int st = prepare(first_layer + i, src_pool, &ls, src_batch, d_slab, slab_bytes, 0, &kp, &rs, &n_layer);
+    if (st != TOPKV_OK) return st;
+    st = prepare(first_layer + i, dst_pool, &ld, dst_batch, d_slab, slab_bytes, 0, &kp, &rs, &n_layer);
+    if (st != TOPKV_OK) return st;
+  }
+  int32_t* packed = d_flags;         // span s of the slab holds the layer of epoch e
+  int32_t* consumed = d_flags + ws;  // span s of the slab has been read for the layer of epoch e
+  for (int i = 0; i < num_layers; ++i) {
+    const uint32_t e = first_epoch + (uint32_t)i;
+    topkv_span_link lp = {sizeof(topkv_span_link), e, e + 1, 0, e ? consumed : nullptr, packed};
+    int st = topkv_pack_layer_linked(first_layer + i, src_pool, &ls, src_batch, d_slab, slab_bytes, &lp, stream);
+    if (st != TOPKV_OK) return st;
+    topkv_span_link lu = {sizeof(topkv_span_link), e + 1, e + 1, 0, packed, consumed};
+    st = topkv_unpack_layer_linked(first_layer + i, dst_pool, &ld, dst_batch, d_slab, slab_bytes, &lu, stream);
+    if (st != TOPKV_OK) return st;
+  }
+  return TOPKV_OK;
+}
+
 int topkv_pack_layers(int first_layer, int num_layers, const void* src_pool, const topkv_layout* layout,
                       const topkv_batch* batch, void* d_wire, int64_t wire_capacity_bytes,
                       topkv_stream_t stream) {

@@ -531,3 +531,25 @@ def test_two_lane_host_leg_validation_without_gpu():
         assert fn(0, 4, pool, lo, _batch(T=-1), host, 4 * n, st, n, None, None, streams) \
             == tk.TOPKV_ERR_INVALID_ARG
     assert tk.topkv_kernel_launch_count() == before
+
+
+def test_relay_linked_validation_without_gpu():
+    n = 1_785_856
+    lo, b = _gqa(wire_layer_stride=n), _batch()
+    src, dst, slab, flags = 0x7000000, 0x8000000, 0x9000000, 0xC000000
+    words = tk.topkv_span_link_words(lo, b)
+    R = tk.topkv_relay_layers_linked
+    before = tk.topkv_kernel_launch_count()
+    assert R(0, 5, src, lo, b, dst, lo, b, slab, n, flags, 2 * words, 0) == tk.TOPKV_ERR_LAYER_RANGE
+    assert R(-1, 1, src, lo, b, dst, lo, b, slab, n, flags, 2 * words, 0) == tk.TOPKV_ERR_LAYER_RANGE
+    assert R(0, 4, src, lo, b, dst, lo, b, slab, n - 1, flags, 2 * words, 0) == tk.TOPKV_ERR_CAPACITY
+    assert R(0, 4, src, lo, b, dst, lo, b, slab, n, flags, 2 * words - 1, 0) == tk.TOPKV_ERR_CAPACITY
+    assert R(0, 4, src, lo, b, dst, lo, b, slab, n, None, 2 * words, 0) == tk.TOPKV_ERR_INVALID_ARG
+    assert R(0, 4, src, lo, b, dst + 8, lo, b, slab, n, flags, 2 * words, 0) == tk.TOPKV_ERR_ALIGNMENT
+    assert R(0, 4, src, lo, b, dst, lo, _batch(R=5), slab, n, flags, 2 * words, 0) == tk.TOPKV_ERR_UNSUPPORTED_LAYOUT
+    p32 = tk.make_layout(4, 2, 8, 128, 2, 32, 64)
+    assert R(0, 4, src, lo, b, dst, p32, _batch(maxp=8), slab, n, flags, 2 * words, 0) \
+        == tk.TOPKV_ERR_UNSUPPORTED_LAYOUT
+    assert R(0, 4, src, lo, b, dst, lo, b, slab, n, flags, 2 * words, 0x7fffffff) == tk.TOPKV_ERR_INVALID_ARG
+    assert R(0, 0, src, lo, b, dst, lo, b, slab, n, flags, 2 * words, 0) == tk.TOPKV_OK
+    assert tk.topkv_kernel_launch_count() == before

@@ -1935,3 +1935,44 @@ def test_two_lane_host_leg_relay(dev):
     assert tk.topkv_kernel_launch_count() == launches
     del w
     torch.cuda.empty_cache()
+
+
+def test_relay_layers_linked_one_call(dev, variant):
+    """topkv_relay_layers_linked: a range of layers from one paged pool into another through ONE
+    slab as a single call (2 launches per layer, all span-linked), twice with continuing epochs;
+    the destination is the oracle's unpack of the oracle's pack, the source is untouched."""
+    if variant == 1:
+        pytest.skip("span links belong to the vectorised family")
+    for name, L in (("cfg2", 5), ("cfg4", 3)):
+        spec = wl.with_layers(wl.ALL[name], L)
+        w = harness.setup(spec, dev, need_wire=False)
+        b = w.batch
+        g = _geom(spec, b.num_pool_pages, 1, 0, 0)
+        slab = torch.zeros(w.n_layer, dtype=torch.uint8, device=dev)
+        words = tk.topkv_span_link_words(w.layout, w.src_batch)
+        flags = torch.zeros(2 * words, dtype=torch.int32, device=dev)
+        before = [harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, l) for l in range(L)]
+        stream = torch.cuda.Stream(dev)
+        stream.wait_stream(torch.cuda.current_stream(dev))
+        args = (w.src_pool, w.layout, w.src_batch, w.dst_pool, w.layout, w.dst_batch, slab, slab.numel(),
+                flags, flags.numel())
+        tk.check(tk.topkv_relay_layers_linked(0, 2, *args, 0, stream))
+        tk.check(tk.topkv_relay_layers_linked(2, L - 2, *args, 2, stream))      # epochs continue
+        stream.synchronize()
+        assert tk.topkv_device_error_flags() == 0 and int(flags.max()) == L
+        for l in range(L):
+            src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, l)
+            want = oracle.pack(g, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=8)
+            oracle.unpack(g, 0, before[l], b.dst_block_table, b.seq_lens, want, impl="rows", threads=8)
+            assert np.array_equal(harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, l), before[l]), (name, l)
+        # refused before anything is launched
+        launches = tk.topkv_kernel_launch_count()
+        assert tk.topkv_relay_layers_linked(0, L + 1, *args, 0, stream) == tk.TOPKV_ERR_LAYER_RANGE
+        assert tk.topkv_relay_layers_linked(0, L, *args[:8], flags, words, 0, stream) == tk.TOPKV_ERR_CAPACITY
+        other = tk.make_layout(L, spec.F, spec.H, spec.D, spec.E, spec.P * 2, b.num_pool_pages)
+        assert tk.topkv_relay_layers_linked(0, L, w.src_pool, w.layout, w.src_batch, w.dst_pool, other,
+                                            w.dst_batch, slab, slab.numel(), flags, flags.numel(), 0,
+                                            stream) == tk.TOPKV_ERR_UNSUPPORTED_LAYOUT
+        assert tk.topkv_kernel_launch_count() == launches
+        del w
+        torch.cuda.empty_cache()
