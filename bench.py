@@ -636,6 +636,86 @@ def bench_chain_linked(w, stream, steps, slabs=1):
     return 4.0 * w.n_layer * w.layers / (ms * 1e-3) / 1e9, ms / (2 * w.layers) * 1e3
 
 
+def launch_modes(w, stream, peak):
+    """The pack and the unpack of every layer of the workload in the ways a caller can issue them,
+    each layer into its own slab of the wire (every launch touches memory no earlier one touched,
+    so L2 holds nothing for it): one call alone between two synchronisations (what the side
+    stream of §5.2 issues after a layer's event; the median over the layers, CUDA events around
+    each call), all layers back to back with no flag (every launch waits for the one before it),
+    with TOPKV_FLAG_TABLES_SETTLED, and with TOPKV_FLAG_OVERLAP_PREVIOUS (the headline's form).
+    GB/s of read + write traffic per launch."""
+    import statistics
+    import torch
+    from paper_2607_28633_b200 import binding as tk
+    L, n, T = w.layers, w.n_layer, w.batch.total_tokens
+    tk.check(tk.topkv_build_plan(tk.make_batch(w.src_bt, w.seq_lens), w.cu, stream))
+    stream.synchronize()
+    out = {}
+    for what, fn, pool, bt in (("pack", tk.topkv_pack_layer, w.src_pool, w.src_bt),
+                               ("unpack", tk.topkv_unpack_layer, w.dst_pool, w.dst_bt)):
+        def batch(flags):
+            return tk.make_batch(bt, w.seq_lens, T, w.cu, flags)
+
+        def call(l, b):
+            tk.check(fn(l, pool, w.layout, b, w.wire, w.wire.numel(), stream))
+        r = {}
+        b0 = batch(0)
+        for l in range(min(L, 3)):
+            call(l, b0)
+        stream.synchronize()
+        times = []
+        for l in range(L):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            call(l, b0)
+            b.record(stream)
+            stream.synchronize()
+            times.append(a.elapsed_time(b) * 1e3)
+        us = statistics.median(times)
+        r["one_call_alone"] = {"us_per_launch_median": round(us, 2), "us_min": round(min(times), 2),
+                               "us_max": round(max(times), 2), "calls": L,
+                               "GBps": round(2.0 * n / (us * 1e-6) / 1e9, 1)}
+        for label, first, rest in (("back_to_back_no_flag", 0, 0),
+                                   ("back_to_back_tables_settled", 0, tk.TOPKV_FLAG_TABLES_SETTLED),
+                                   ("back_to_back_overlap_previous", 0, tk.TOPKV_FLAG_OVERLAP_PREVIOUS)):
+            bf, br = batch(first), batch(rest)
+            best = None
+            for _ in range(3):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                for l in range(L):
+                    call(l, br if l else bf)
+                b.record(stream)
+                stream.synchronize()
+                t = a.elapsed_time(b) * 1e3 / L
+                best = t if best is None else min(best, t)
+            r[label] = {"us_per_launch": round(best, 2), "GBps": round(2.0 * n / (best * 1e-6) / 1e9, 1)}
+        for v in r.values():
+            v["frac_of_hbm_peak"] = round(v["GBps"] / peak, 4)
+            v["frac_of_8000_spec"] = round(v["GBps"] / 8000.0, 4)
+        out[what] = r
+    if L >= 2:
+        # for scale: a plain device copy of one slab (torch copy_, N_layer read + N_layer written)
+        # issued the same way, alone between two synchronisations
+        times = []
+        with torch.cuda.stream(stream):
+            for k in range(max(20, L)):
+                i, j = k % L, (k + L // 2) % L
+                if i == j:
+                    continue
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                w.wire[i * n:(i + 1) * n].copy_(w.wire[j * n:(j + 1) * n])
+                b.record(stream)
+                stream.synchronize()
+                times.append(a.elapsed_time(b) * 1e3)
+        us = statistics.median(times[3:])
+        out["plain_copy_one_call_alone"] = {"us_per_launch_median": round(us, 2),
+                                            "GBps": round(2.0 * n / (us * 1e-6) / 1e9, 1),
+                                            "frac_of_hbm_peak": round(2.0 * n / (us * 1e-6) / 1e9 / peak, 4)}
+    return out
+
+
 def host_leg_forms(w, dev, stream, pinned, slots, steps):
     """The host leg of the workload in its three forms against a pinned cudaMemcpyAsync of one
     slab measured in the same run."""
@@ -967,6 +1047,8 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="topkv", choices=["topkv", "reference"])
+    ap.add_argument("--no-launch-modes", action="store_true",
+                    help="skip the one-call-alone / back-to-back comparison of the headline workload")
     ap.add_argument("--extras", default="cfg5,overlap_curve,cfg2,cfg4,chain,crc,hybrid,session,cfg1",
                     help="comma list of extra workloads measured at one GPU ('' for none)")
     ap.add_argument("--variant", type=int, default=None, help="kernel family (see topkv.h)")
@@ -1117,6 +1199,8 @@ def main():
                     "number for this path exists in the paper"}
     if rank == 0 and world == 1:
         extra["device_copy_GBps_same_bytes"] = round(device_copy_baseline(dev, stream, n_layer), 1)
+        if not args.no_launch_modes:
+            extra["launch_modes"] = launch_modes(w, stream, peak)
     batch = w.batch
     del w
     torch.cuda.empty_cache()

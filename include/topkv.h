@@ -212,7 +212,12 @@ int topkv_unpack_layer_from_host(int layer, void* dst_pool, const topkv_layout* 
  * A linked call never waits for the previous kernel as a whole and reads its tables at once,
  * as if TOPKV_FLAG_OVERLAP_PREVIOUS were set: the caller promises that the tables were not
  * written by kernels still running and that EVERY conflict with kernels enqueued before it on
- * `stream` is covered by the link. For pack(l) -> unpack(l) -> pack(l+1) -> ... through one slab:
+ * `stream` is covered by the link. The FIRST call of a chain usually cannot promise that (the
+ * kernel before it wrote the pool, or the plan): give it TOPKV_LINK_WAIT_PREVIOUS, which makes
+ * it an ordinary launch towards everything before it (it waits for the previous kernel to
+ * finish before it reads anything, and only then lets the next linked kernel in, so that the
+ * calls after it are ordered behind that kernel too) and a linked one towards what follows.
+ * For pack(l) -> unpack(l) -> pack(l+1) -> ... through one slab:
  * pack(l+1) awaits the flags unpack(l) publishes (the slab has been read) and publishes the
  * flags unpack(l+1) awaits. Kernels still complete in stream order. Waits are bounded (about
  * half a second): a flag that never arrives raises bit 1 of topkv_device_error_flags() and skips the
@@ -222,11 +227,12 @@ int topkv_unpack_layer_from_host(int layer, void* dst_pool, const topkv_layout* 
  * arguments: a CUDA graph that captured linked calls replays the epochs of the capture, so such
  * a graph must clear the flag arrays (a memset node) ahead of the linked calls of every replay.
  * Vectorised kernel family, one layer per call. */
+#define TOPKV_LINK_WAIT_PREVIOUS 1u /* also wait for the previous kernel of the stream as a whole */
 typedef struct topkv_span_link {
   uint32_t struct_size;   /* = sizeof(topkv_span_link)               */
   uint32_t await_epoch;   /* value the awaited flags must reach      */
   uint32_t signal_epoch;  /* value written into the published flags  */
-  uint32_t reserved;      /* must be 0                               */
+  uint32_t flags;         /* 0 or TOPKV_LINK_WAIT_PREVIOUS           */
   const int32_t* d_await; /* DEVICE int32 [words] or NULL            */
   int32_t* d_signal;      /* DEVICE int32 [words] or NULL            */
 } topkv_span_link;
@@ -252,7 +258,10 @@ int topkv_unpack_layer_linked(int layer, void* dst_pool, const topkv_layout* lay
  * is the slab of every layer. d_flags: DEVICE int32 [2 * topkv_span_link_words()], zeroed once by
  * the caller; first_epoch = the number of layers already relayed through these flags since they
  * were zeroed (0 the first time; the call uses epochs first_epoch + 1 .. first_epoch +
- * num_layers). Everything is validated for every layer before the first launch. */
+ * num_layers). The first pack of the call waits for the kernel enqueued before the call as a
+ * whole (TOPKV_LINK_WAIT_PREVIOUS), unless src_batch carries TOPKV_FLAG_OVERLAP_PREVIOUS; all
+ * later launches are ordered behind it through their links. Everything is validated for every
+ * layer before the first launch. */
 int topkv_relay_layers_linked(int first_layer, int num_layers, const void* src_pool,
                               const topkv_layout* src_layout, const topkv_batch* src_batch,
                               void* dst_pool, const topkv_layout* dst_layout,

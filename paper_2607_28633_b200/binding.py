@@ -29,6 +29,7 @@ TOPKV_WIRE_TOKEN_KV, TOPKV_WIRE_PLANAR = 0, 1
 TOPKV_MAX_INLINE_R = 1024
 TOPKV_FLAG_OVERLAP_PREVIOUS = 1
 TOPKV_FLAG_TABLES_SETTLED = 2
+TOPKV_LINK_WAIT_PREVIOUS = 1
 TOPKV_NOALLOC_STAGING_BYTES = 8 * 1024 * 1024
 
 # every symbol include/topkv.h declares
@@ -85,13 +86,14 @@ TOPKV_LAYER_FULL, TOPKV_LAYER_WINDOW, TOPKV_LAYER_STATE = 0, 1, 2
 
 class topkv_span_link(ctypes.Structure):
     _fields_ = [("struct_size", c_uint32), ("await_epoch", c_uint32), ("signal_epoch", c_uint32),
-                ("reserved", c_uint32), ("d_await", c_void_p), ("d_signal", c_void_p)]
+                ("flags", c_uint32), ("d_await", c_void_p), ("d_signal", c_void_p)]
 
 
-def make_span_link(d_await=None, await_epoch=0, d_signal=None, signal_epoch=0) -> topkv_span_link:
+def make_span_link(d_await=None, await_epoch=0, d_signal=None, signal_epoch=0,
+                   flags: int = 0) -> topkv_span_link:
     k = topkv_span_link()
     k.struct_size = ctypes.sizeof(topkv_span_link)
-    k.await_epoch, k.signal_epoch = await_epoch, signal_epoch
+    k.await_epoch, k.signal_epoch, k.flags = await_epoch, signal_epoch, flags
     k.d_await, k.d_signal = _ptr(d_await), _ptr(d_signal)
     k._keepalive = (d_await, d_signal)
     return k

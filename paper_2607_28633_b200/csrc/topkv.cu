@@ -1032,9 +1032,12 @@ int topkv_unpack_layer(int layer, void* dst_pool, const topkv_layout* layout,
 
 namespace {
 // Checks a span link and puts it into the kernel parameters: a linked launch orders itself
-// span by span, so it never waits for the previous kernel as a whole (kp->overlap).
+// span by span, so it never waits for the previous kernel as a whole (kp->overlap) unless the
+// link asks for that too; then it waits before it reads anything and releases the next kernel
+// only afterwards, which orders every later linked launch behind the previous kernel as well.
 int apply_link(const topkv_span_link* link, KParams* kp) {
-  if (link == nullptr || link->struct_size != sizeof(topkv_span_link) || link->reserved != 0)
+  if (link == nullptr || link->struct_size != sizeof(topkv_span_link) ||
+      (link->flags & ~TOPKV_LINK_WAIT_PREVIOUS) != 0)
     return TOPKV_ERR_INVALID_ARG;
   if (link->d_await == nullptr && link->d_signal == nullptr) return TOPKV_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(link->d_await) | reinterpret_cast<uintptr_t>(link->d_signal)) & 3)
@@ -1043,7 +1046,7 @@ int apply_link(const topkv_span_link* link, KParams* kp) {
   kp->link_signal = link->d_signal;
   kp->await_epoch = (int)link->await_epoch;
   kp->signal_epoch = (int)link->signal_epoch;
-  kp->overlap = 1;
+  kp->overlap = (link->flags & TOPKV_LINK_WAIT_PREVIOUS) ? 0 : 1;
   kp->late_wait = 0;
   return TOPKV_OK;
 }
@@ -1135,7 +1138,8 @@ int topkv_relay_layers_linked(int first_layer, int num_layers, const void* src_p
   int32_t* consumed = d_flags + ws;  // span s of the slab has been read for the layer of epoch e
   for (int i = 0; i < num_layers; ++i) {
     const uint32_t e = first_epoch + (uint32_t)i;
-    topkv_span_link lp = {sizeof(topkv_span_link), e, e + 1, 0, e ? consumed : nullptr, packed};
+    const uint32_t lf = (i == 0 && !(src_batch->flags & TOPKV_FLAG_OVERLAP_PREVIOUS)) ? TOPKV_LINK_WAIT_PREVIOUS : 0u;
+    topkv_span_link lp = {sizeof(topkv_span_link), e, e + 1, lf, e ? consumed : nullptr, packed};
     int st = topkv_pack_layer_linked(first_layer + i, src_pool, &ls, src_batch, d_slab, slab_bytes, &lp, stream);
     if (st != TOPKV_OK) return st;
     topkv_span_link lu = {sizeof(topkv_span_link), e + 1, e + 1, 0, packed, consumed};

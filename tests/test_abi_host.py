@@ -507,7 +507,7 @@ def test_span_link_validation_without_gpu():
     assert P(0, pool, lo, b, wire, cap, tk.make_span_link(None, 0, None, 0)) == tk.TOPKV_ERR_INVALID_ARG
     bad = tk.make_span_link(flags, 1, None, 0); bad.struct_size = 4
     assert U(0, pool, lo, b, wire, cap, bad) == tk.TOPKV_ERR_INVALID_ARG
-    bad = tk.make_span_link(flags, 1, None, 0); bad.reserved = 1
+    bad = tk.make_span_link(flags, 1, None, 0, flags=2)   # only TOPKV_LINK_WAIT_PREVIOUS is defined
     assert U(0, pool, lo, b, wire, cap, bad) == tk.TOPKV_ERR_INVALID_ARG
     assert U(0, pool, lo, b, wire, cap, tk.make_span_link(flags + 2, 1, None, 0)) == tk.TOPKV_ERR_ALIGNMENT
     assert tk.topkv_kernel_launch_count() == before

@@ -1976,3 +1976,62 @@ def test_relay_layers_linked_one_call(dev, variant):
         assert tk.topkv_kernel_launch_count() == launches
         del w
         torch.cuda.empty_cache()
+
+
+def test_relay_call_right_behind_a_kernel_that_writes_its_source(dev, variant):
+    """The first launch of topkv_relay_layers_linked is an ordinary launch towards what precedes
+    the call (TOPKV_LINK_WAIT_PREVIOUS): kernels that rewrite the source pool and the plan are
+    enqueued on the same stream right before it, with nothing in between, and the destination
+    must hold the NEW source contents. The same with hand-made links whose first one carries
+    the flag."""
+    if variant == 1:
+        pytest.skip("span links belong to the vectorised family")
+    L = 3
+    spec = wl.with_layers(wl.CFG2, L)
+    w = harness.setup(spec, dev, need_wire=False)
+    b = w.batch
+    g = _geom(spec, b.num_pool_pages, 1, 0, 0)
+    n = w.n_layer
+    fresh = wl.fill_torch(2 * L * n, 4242, dev, raw_bits=True)          # two new contents for the source
+    slab = torch.zeros(n, dtype=torch.uint8, device=dev)
+    words = tk.topkv_span_link_words(w.layout, w.src_batch)
+    cu = torch.zeros_like(w.cu)
+    T = b.total_tokens
+    bs = tk.make_batch(w.src_bt, w.seq_lens, T, cu)
+    bd = tk.make_batch(w.dst_bt, w.seq_lens, T, cu)
+    stream = torch.cuda.Stream(dev)
+    lo1 = tk.make_layout(spec.L, spec.F, spec.H, spec.D, spec.E, spec.P, b.num_pool_pages)
+    for round_, by_hand in enumerate((False, True)):
+        flags = torch.zeros(2 * words, dtype=torch.int32, device=dev)
+        cu.zero_()
+        src_h = [harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, l) for l in range(L)]
+        dst_h = [harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, l) for l in range(L)]
+        wire_in = fresh[round_ * L * n:(round_ + 1) * L * n]
+        torch.cuda.synchronize()
+        # the producers: the plan both sides read, and new contents for every source layer
+        tk.check(tk.topkv_build_plan(tk.make_batch(w.src_bt, w.seq_lens), cu, stream))
+        for l in range(L):
+            tk.check(tk.topkv_unpack_layer(l, w.src_pool, w.layout, w.src_batch, wire_in, wire_in.numel(), stream))
+        if not by_hand:
+            tk.check(tk.topkv_relay_layers_linked(0, L, w.src_pool, w.layout, bs, w.dst_pool, w.layout, bd, slab,
+                                                  n, flags, flags.numel(), 0, stream))
+        else:
+            fp, fu = flags[:words], flags[words:]
+            for l in range(L):
+                lp = tk.make_span_link(fu if l else None, l, fp, l + 1,
+                                       tk.TOPKV_LINK_WAIT_PREVIOUS if l == 0 else 0)
+                tk.check(tk.topkv_pack_layer_linked(l, w.src_pool, lo1, bs, slab, n, lp, stream))
+                tk.check(tk.topkv_unpack_layer_linked(l, w.dst_pool, lo1, bd, slab, n,
+                                                      tk.make_span_link(fp, l + 1, fu, l + 1), stream))
+        stream.synchronize()
+        assert tk.topkv_device_error_flags() == 0
+        win = wire_in.cpu().numpy()
+        for l in range(L):
+            oracle.unpack(g, 0, src_h[l], b.src_block_table, b.seq_lens, win[l * n:(l + 1) * n],
+                          impl="rows", threads=8)
+            assert np.array_equal(harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, l), src_h[l]), l
+            want = oracle.pack(g, 0, src_h[l], b.src_block_table, b.seq_lens, impl="rows", threads=8)
+            oracle.unpack(g, 0, dst_h[l], b.dst_block_table, b.seq_lens, want, impl="rows", threads=8)
+            assert np.array_equal(harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, l), dst_h[l]), (by_hand, l)
+    del w
+    torch.cuda.empty_cache()
