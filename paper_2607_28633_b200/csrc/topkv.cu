@@ -294,6 +294,18 @@ void span_geometry(KParams* kp, int F, int64_t row_bytes) {
   }
 }
 
+// A windowed layer keeps at most `window` tokens per request, wherever they lie in its row: the
+// window touches at most ceil(window / span) + 1 spans, so only that many CTAs per request are
+// launched and each finds its span from the request's length (a 128-token window of a
+// 4,096-token row: 5 CTAs instead of 128, of which 123 would find nothing to do).
+void window_spans(KParams* kp) {
+  kp->wspr = 0;
+  if (kp->window <= 0 || kp->cpp != 1 || kp->const_len > 0) return;
+  const int64_t span_tokens = (int64_t)kp->ppc * kp->P;
+  const int64_t need = (kp->window + span_tokens - 1) / span_tokens + 1;
+  if (need < kp->spr) kp->wspr = (int)need;
+}
+
 // max_ctas > 0: the wire is host memory behind PCIe; at most that many CTAs walk the spans.
 // layers > 1: one launch covers that many consecutive layers (kp describes the first one and
 // carries the layer strides); the vectorised family only.
@@ -310,7 +322,8 @@ int launch_copy(KParams kp, const Resolved& rs, int F, cudaStream_t stream, int 
   }
   if (!handled) {
     span_geometry(&kp, F, rs.row_bytes);
-    const int64_t spans = (int64_t)kp.R * kp.spr;
+    window_spans(&kp);
+    const int64_t spans = (int64_t)kp.R * (kp.wspr > 0 ? kp.wspr : kp.spr);
     const bool walk = max_ctas > 0 && spans > max_ctas;
     const dim3 grid((unsigned)(walk ? max_ctas : spans), (unsigned)layers);
     cudaError_t le;
@@ -898,12 +911,15 @@ int copy_layers(int first_layer, int num_layers, const void* pool, const topkv_l
     return plan_layer(l, pool, lo, b, t, d_wire, wire_bytes, off, b->flags, &lp);
   });
   if (st != TOPKV_OK) return st;
-  bool launched = false;
+  // the runs: same kind and parameter, constant stride in pool and wire
+  struct Run {
+    int first, count;
+    int64_t d_off, d_ord, bytes;
+  };
+  std::vector<Run> runs;
   for (int i = 0; i < num_layers; ++i) {
     if (info[i].done) continue;
     const topkv_layer_spec& sp = t->specs[first_layer + i];
-    const bool is_state = sp.kind == TOPKV_LAYER_STATE;
-    // the run that starts at layer i: same kind and parameter, constant stride in pool and wire
     int count = 1, last = i;
     int64_t d_off = 0, d_ord = 0;
     for (int j = i + 1; j < num_layers && count < 65535; ++j) {
@@ -921,15 +937,28 @@ int copy_layers(int first_layer, int num_layers, const void* pool, const topkv_l
       ++count;
     }
     info[i].done = true;
+    int64_t n = 0;
+    st = slab_bytes(lo, t, b->num_requests, (uint32_t)(first_layer + i), &n);
+    if (st != TOPKV_OK) return st;
+    runs.push_back({i, count, d_off, d_ord, n * count});
+  }
+  // The launches of one call are independent of each other, so their order is free: the largest
+  // run goes first and the small ones (the 4 MiB slabs of windowed layers) run under its tail
+  // instead of standing alone, launch-bound, between two large ones.
+  std::stable_sort(runs.begin(), runs.end(), [](const Run& a, const Run& c) { return a.bytes > c.bytes; });
+  bool launched = false;
+  for (const Run& run : runs) {
+    const bool is_state = t->specs[first_layer + run.first].kind == TOPKV_LAYER_STATE;
     const uint32_t flags = launched ? (b->flags | TOPKV_FLAG_OVERLAP_PREVIOUS) : b->flags;
-    st = plan_layer((uint32_t)(first_layer + i), pool, lo, b, t, d_wire, wire_bytes, info[i].off, flags, &lp);
+    st = plan_layer((uint32_t)(first_layer + run.first), pool, lo, b, t, d_wire, wire_bytes, info[run.first].off,
+                    flags, &lp);
     if (st != TOPKV_OK) return st;
     if (lp.empty) continue;
-    if (count > 1) {
-      lp.kp.S_layer = d_ord * (is_state ? t->state_layer_stride : lo->pool_layer_stride);
-      lp.kp.W_layer = d_off;
+    if (run.count > 1) {
+      lp.kp.S_layer = run.d_ord * (is_state ? t->state_layer_stride : lo->pool_layer_stride);
+      lp.kp.W_layer = run.d_off;
     }
-    st = launch_copy<PACK>(lp.kp, lp.rs, lp.F, s, 0, count);
+    st = launch_copy<PACK>(lp.kp, lp.rs, lp.F, s, 0, run.count);
     if (st != TOPKV_OK) return st;
     launched = true;
   }

@@ -29,6 +29,8 @@ struct KParams {
   int64_t plane_rows;     // PLANAR: rows between the planes of a slab, or -1 = total tokens T
   int window;             // 0, or the layer keeps only the last min(s, window) tokens
   int ppc, spr;           // vectorised family: page columns per CTA, CTAs per request
+  int wspr;               // windowed layer: only the `wspr` spans per request that the window can touch get
+                          // a CTA, counted from the span of the first kept token (0 = all `spr` spans)
   int cpp, tps;           // pages far larger than a CTA's span are split: CTAs per page (1 = whole
                           // pages), tokens per CTA of a split page
   int const_len;          // > 0: every request has exactly this many tokens; sl and cu are not read

@@ -64,8 +64,16 @@ __device__ __forceinline__ bool copy_span_work(const KParams& p, const int slot)
   // blockIdx.y = layer of a multi-layer launch (0 and zero strides for a single layer)
   uint8_t* const pool = p.pool + (int64_t)blockIdx.y * p.S_layer;
   uint8_t* const wire = p.wire + (int64_t)blockIdx.y * p.W_layer;
-  const int r = slot / p.spr;
-  const int sidx = slot - r * p.spr;  // span of request r
+  const int gspr = p.wspr > 0 ? p.wspr : p.spr;  // spans per request that have a CTA
+  const int r = slot / gspr;
+  const int s_r = p.const_len > 0 ? p.const_len : p.sl[r];
+  // first token this layer keeps: 0, or s_r - window for a windowed layer (§2.2)
+  const int b_r = (p.window > 0 && s_r > p.window) ? s_r - p.window : 0;
+  int sidx = slot - r * gspr;  // span of request r
+  if (p.wspr > 0) {            // counted from the span that holds the first kept token
+    sidx += b_r / (p.ppc * p.P);
+    if (sidx >= p.spr) return false;
+  }
   // The span: `ppc` whole page columns from column j0 on, or, when pages are far larger than a
   // CTA's share, `tps` tokens of page column j0 (`cpp` CTAs per page).
   int j0, first, span_tokens;
@@ -78,9 +86,6 @@ __device__ __forceinline__ bool copy_span_work(const KParams& p, const int slot)
     first = j0 * p.P;  // first token of the span's page columns
     span_tokens = p.ppc * p.P;
   }
-  const int s_r = p.const_len > 0 ? p.const_len : p.sl[r];
-  // first token this layer keeps: 0, or s_r - window for a windowed layer (§2.2)
-  const int b_r = (p.window > 0 && s_r > p.window) ? s_r - p.window : 0;
   const int tid = threadIdx.x;
   int hi = min(first + span_tokens, s_r);
   if (s_r > p.maxp * p.P) {  // length longer than its block-table row: copy what the row holds
@@ -280,7 +285,7 @@ template <int F, bool PACK, bool MERGED, int VEC, bool MULTI>
 __global__ void __launch_bounds__(kThreads, kMinCtasPerSm)
 topkv_page_copy_walk_kernel(const KParams p) {
   pdl_prologue(p.overlap | p.late_wait);
-  const int nslots = p.R * p.spr;
+  const int nslots = p.R * (p.wspr > 0 ? p.wspr : p.spr);
   for (int slot = blockIdx.x; slot < nslots; slot += gridDim.x) {
     copy_span<F, PACK, MERGED, VEC, MULTI>(p, slot);
     __syncthreads();  // the span's page ids in shared memory are re-used by the next span

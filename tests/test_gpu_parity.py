@@ -742,6 +742,76 @@ def test_windowed_layers(dev, seed):
     assert np.array_equal(dst.cpu().numpy(), dst_h)
 
 
+@pytest.mark.parametrize("P,H,D", [(4, 1, 64), (16, 8, 128), (1, 2, 64)])
+def test_window_spans_counted_from_the_first_kept_token(dev, variant, P, H, D):
+    """Long rows with a short window: only the few spans a window can touch get a CTA, each
+    placed from the request's own length. Lengths and windows sit on and around span borders
+    (a span = 64 KiB worth of page columns: 64 pages of 4 tokens here, one page of 16, 64 pages
+    of one token), with empty requests, requests shorter than the window and stale (-1)
+    columns before every window. Pack, unpack and a linked pack -> unpack pair."""
+    rng = np.random.default_rng(900 + P)
+    E, F = 2, 2
+    page_bytes = P * F * H * D * E
+    ppc = max(1, min(64, 65536 // page_bytes))
+    span = ppc * P
+    maxp = (12 * span) // P + 3
+    for W in (1, span - 1, span, span + 1, 2 * span + 1, 3 * span):
+        if W <= 0:
+            continue
+        lens = [0, 1, max(1, W - 1), W, W + 1, 5 * span, 5 * span + 1, 5 * span - 1, 7 * span + W // 2,
+                12 * span, 12 * span - W + 1, int(rng.integers(1, 12 * span))]
+        sl = np.array(lens, dtype=np.int32)
+        R = len(sl)
+        pages = (sl + P - 1) // P
+        npages = int(pages.sum()) + 3
+        g = Geom(L=1, F=F, h_kv=H, d_h=D, b_p=E, P=P, num_pages=npages)
+        g.window = W
+        T = g.kept_tokens(sl)
+        g.W_layer = g.wire_layer_bytes(T)
+        bt_s = np.full((R, maxp), -1, dtype=np.int32)
+        bt_d = np.full((R, maxp), -1, dtype=np.int32)
+        ps, pd, pos = rng.permutation(npages), rng.permutation(npages), 0
+        for r in range(R):
+            bt_s[r, :pages[r]] = ps[pos:pos + pages[r]]
+            bt_d[r, :pages[r]] = pd[pos:pos + pages[r]]
+            pos += pages[r]
+            stale = max(0, int(sl[r]) - W) // P                 # columns wholly before the window
+            bt_s[r, :stale] = -1
+            bt_d[r, :stale] = -1
+        lo = _layout_from_geom(g)
+        src_h = rng.integers(0, 256, g.S_layer, dtype=np.uint8)
+        dst_h = rng.integers(0, 256, g.S_layer, dtype=np.uint8)
+        src = torch.from_numpy(src_h).to(dev)
+        dst, dst2 = torch.from_numpy(dst_h).to(dev), torch.from_numpy(dst_h).to(dev)
+        wire = torch.full((g.W_layer + 64,), 0x3C, dtype=torch.uint8, device=dev)
+        wire2 = torch.full((g.W_layer + 64,), 0x3C, dtype=torch.uint8, device=dev)
+        d_sl = torch.from_numpy(sl).to(dev)
+        bs = tk.make_batch(torch.from_numpy(bt_s).to(dev), d_sl, T, None, 0, W)
+        bd = tk.make_batch(torch.from_numpy(bt_d).to(dev), d_sl, T, None, 0, W)
+        tk.check(tk.topkv_pack_layer(0, src, lo, bs, wire, wire.numel()))
+        tk.check(tk.topkv_unpack_layer(0, dst, lo, bd, wire, wire.numel()))
+        want = np.full(g.W_layer + 64, 0x3C, dtype=np.uint8)
+        oracle.pack(g, 0, src_h, bt_s, sl, wire=want)
+        oracle.unpack(g, 0, dst_h, bt_d, sl, want)
+        torch.cuda.synchronize()
+        assert tk.topkv_device_error_flags() == 0
+        assert np.array_equal(wire.cpu().numpy(), want), W
+        assert np.array_equal(dst.cpu().numpy(), dst_h), W
+        if variant == 0:
+            words = tk.topkv_span_link_words(lo, bs)
+            flags = torch.zeros(max(1, words), dtype=torch.int32, device=dev)
+            stream = torch.cuda.Stream(dev)
+            stream.wait_stream(torch.cuda.current_stream(dev))
+            tk.check(tk.topkv_pack_layer_linked(0, src, lo, bs, wire2, wire2.numel(),
+                                                tk.make_span_link(None, 0, flags, 3), stream))
+            tk.check(tk.topkv_unpack_layer_linked(0, dst2, lo, bd, wire2, wire2.numel(),
+                                                  tk.make_span_link(flags, 3, None, 0), stream))
+            stream.synchronize()
+            assert tk.topkv_device_error_flags() == 0
+            assert np.array_equal(wire2.cpu().numpy(), want), W
+            assert np.array_equal(dst2.cpu().numpy(), dst_h), W
+
+
 def test_windowed_layer_bench_shape(dev):
     """gpt-oss-like windowed layer on the 8B batch: window 128 of up to 4096 tokens."""
     w = harness.setup(wl.CFG2, dev, layers=2)
