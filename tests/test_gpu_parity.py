@@ -408,22 +408,26 @@ def test_full_size_in_the_bench_launch_configuration(dev, name):
     torch.cuda.empty_cache()
 
 
-def test_cfg3_host_leg_full_size(dev):
+def test_cfg3_host_leg_full_size(dev, variant):
     """Configuration 3 as stated: all 80 layers of the 70B-shaped cache packed to pinned host
     memory over PCIe (staged form, one 128 MiB slab per layer, 10 GiB in all), then unpacked from
     the host into the destination pool. Every pinned slab and every destination slab is
-    compared in full with the oracle."""
+    compared in full with the oracle. In the vectorised family the same layers then go through
+    the form bench.py times as its end-to-end number: the pipelined relay of the two two-lane
+    calls (each direction alternating between two streams and two staging slabs, the receiver's
+    layer_ready events being the sender's layer_done), compared with the same oracle slabs."""
     spec = wl.CFG3
     w = harness.setup(spec, dev, need_wire=False)
     b, s = w.batch, spec
     g1 = _geom(s, b.num_pool_pages, 1, 0, 0)
+    n = w.n_layer
     try:
-        pinned = torch.empty(s.L * w.n_layer, dtype=torch.uint8).pin_memory()
+        pinned = torch.empty(s.L * n, dtype=torch.uint8).pin_memory()
     except RuntimeError:
         pytest.skip("this box refuses 10 GiB of pinned memory")
     pinned.fill_(0x6B)
     dst_before = w.dst_pool.clone()
-    staging = torch.empty(w.n_layer, dtype=torch.uint8, device=dev)
+    staging = torch.empty(n, dtype=torch.uint8, device=dev)
     stream = torch.cuda.Stream(dev)
     stream.wait_stream(torch.cuda.current_stream(dev))
     for layer in range(s.L):
@@ -432,16 +436,40 @@ def test_cfg3_host_leg_full_size(dev):
         w.unpack_from_host(layer, pinned, staging, stream)
     stream.synchronize()
     assert tk.topkv_device_error_flags() == 0
-    host = pinned.numpy()
+    relay = variant == 0
+    if relay:   # keep the first form's results aside and run the relay into the same buffers
+        host_seq = pinned.clone()                       # pageable copy
+        dst_seq = w.dst_pool.clone()
+        w.dst_pool.copy_(dst_before)
+        pinned.fill_(0x6B)
+        tx = [torch.cuda.Stream(dev), torch.cuda.Stream(dev)]
+        rx = [torch.cuda.Stream(dev), torch.cuda.Stream(dev)]
+        st_tx = [staging, torch.empty_like(staging)]
+        st_rx = [torch.empty_like(staging), torch.empty_like(staging)]
+        sent = [torch.cuda.Event() for _ in range(s.L)]
+        torch.cuda.synchronize()
+        tk.check(tk.topkv_pack_layers_to_host_two_lanes(
+            0, s.L, w.src_pool, w.layout, w.src_batch, pinned, s.L * n, st_tx, n, None, sent, tx))
+        tk.check(tk.topkv_unpack_layers_from_host_two_lanes(
+            0, s.L, w.dst_pool, w.layout, w.dst_batch, pinned, s.L * n, st_rx, n, sent, None, rx))
+        torch.cuda.synchronize()
+        assert tk.topkv_device_error_flags() == 0
+    else:
+        host_seq, dst_seq = pinned, w.dst_pool
+    host, host1 = pinned.numpy(), host_seq.numpy()
     for layer in range(s.L):
         src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, layer)
         want = oracle.pack(g1, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=16)
-        assert np.array_equal(host[layer * w.n_layer:(layer + 1) * w.n_layer], want), f"to host, layer {layer}"
+        assert np.array_equal(host1[layer * n:(layer + 1) * n], want), f"to host, layer {layer}"
         dst_h = harness.layer_slab_to_numpy(dst_before, w.slab_bytes, layer)
         oracle.unpack(g1, 0, dst_h, b.dst_block_table, b.seq_lens, want, impl="rows", threads=16)
-        assert np.array_equal(harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, layer), dst_h), \
+        assert np.array_equal(harness.layer_slab_to_numpy(dst_seq, w.slab_bytes, layer), dst_h), \
             f"from host, layer {layer}"
-    del w, dst_before, pinned, staging
+        if relay:
+            assert np.array_equal(host[layer * n:(layer + 1) * n], want), f"relay to host, layer {layer}"
+            assert np.array_equal(harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, layer), dst_h), \
+                f"relay from host, layer {layer}"
+    del w, dst_before, pinned, staging, host_seq, dst_seq
     torch.cuda.empty_cache()
 
 
