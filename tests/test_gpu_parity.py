@@ -365,12 +365,18 @@ def _oracle_token(spec, page_host, t):
 
 
 @pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4"])
-def test_full_size_in_the_bench_launch_configuration(dev, name):
+def test_full_size_in_the_bench_launch_configuration(dev, name, variant):
     """The workloads at full size, all layers resident, issued as bench.py issues them (one
     stream, TOPKV_FLAG_OVERLAP_PREVIOUS after the first layer of each phase). EVERY layer's wire
     slab and EVERY layer's destination slab (untouched bytes included) is compared in full with
     the oracle; a few sampled tokens are also checked one by one through a one-page oracle
-    problem, which ties the batch-level comparison to the per-token definition."""
+    problem, which ties the batch-level comparison to the per-token definition.
+    Once per shape the checksummed chain runs beside it, again as bench.py issues it (begin, one
+    checksummed copy per layer with the flag after the first, finish; pack, then unpack, into a
+    second wire and a second destination pool): its slabs are compared with the same oracle
+    slabs, and the CRC-64 of every request's K and V tensor over ALL layers, from both
+    directions, with the oracle's bit-by-bit CRC of the tensor gathered from the source pool."""
+    from concurrent.futures import ThreadPoolExecutor
     spec = wl.ALL[name]
     w = harness.setup(spec, dev)
     b, s = w.batch, spec
@@ -383,6 +389,25 @@ def test_full_size_in_the_bench_launch_configuration(dev, name):
         w.unpack(layer, stream, overlap=layer > 0)
     stream.synchronize()
     assert tk.topkv_device_error_flags() == 0
+    with_crc = variant == 0
+    if with_crc:
+        wire2 = torch.zeros_like(w.wire)
+        dst2 = dst_before.clone()
+        nws = tk.topkv_crc_workspace_bytes(w.layout, s.R, b.max_pages_per_req)
+        ws = torch.empty(nws, dtype=torch.uint8, device=dev)
+        crcs = {}
+        for what, fn, pool, batch in (("pack", tk.topkv_pack_layer_crc, w.src_pool, w.src_batch),
+                                      ("unpack", tk.topkv_unpack_layer_crc, dst2, w.dst_batch)):
+            crc = torch.zeros(s.R * s.F, dtype=torch.int64, device=dev)
+            tk.check(tk.topkv_crc_begin(w.layout, batch, ws, nws, stream))
+            for layer in range(s.L):
+                tk.check(fn(layer, pool, w.layout, w._flagged(batch, layer > 0), wire2, wire2.numel(), ws,
+                            nws, stream))
+            tk.check(tk.topkv_crc_finish(w.layout, batch, ws, nws, crc, stream))
+            stream.synchronize()
+            crcs[what] = crc.cpu().numpy().view(np.uint64).reshape(s.R, s.F)
+        assert tk.topkv_device_error_flags() == 0
+        pool_h = np.empty(s.L * w.slab_bytes, dtype=np.uint8)      # the whole source pool, for the CRCs
     for layer in range(s.L):
         src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, layer)
         want = oracle.pack(g1, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=16)
@@ -392,6 +417,22 @@ def test_full_size_in_the_bench_launch_configuration(dev, name):
         oracle.unpack(g1, 0, dst_h, b.dst_block_table, b.seq_lens, want, impl="rows", threads=16)
         assert np.array_equal(harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, layer), dst_h), \
             f"unpack layer {layer}"
+        if with_crc:
+            got2 = wire2[layer * w.n_layer:(layer + 1) * w.n_layer].cpu().numpy()
+            assert np.array_equal(got2, want), f"checksummed pack, layer {layer}"
+            assert np.array_equal(harness.layer_slab_to_numpy(dst2, w.slab_bytes, layer), dst_h), \
+                f"checksummed unpack, layer {layer}"
+            pool_h[layer * w.slab_bytes:(layer + 1) * w.slab_bytes] = src_h
+    if with_crc:
+        gL = _geom(s, b.num_pool_pages, s.L, 0, 0)
+        pairs = [(r, c) for r in range(s.R) for c in range(s.F)]
+        with ThreadPoolExecutor(max_workers=16) as ex:     # the C routine runs without the GIL
+            want_crc = list(ex.map(lambda rc: oracle.kv_plane_crc(gL, pool_h, b.src_block_table, b.seq_lens,
+                                                                  rc[0], rc[1]), pairs))
+        for (r, c), v in zip(pairs, want_crc):
+            assert int(crcs["pack"][r, c]) == v, ("pack", r, c)
+            assert int(crcs["unpack"][r, c]) == v, ("unpack", r, c)
+        del wire2, dst2, ws, pool_h
     rng = np.random.default_rng(7)
     cu = np.concatenate([[0], np.cumsum(b.seq_lens.astype(np.int64))])
     for layer in rng.choice(s.L, size=min(8, s.L), replace=False):
