@@ -123,7 +123,11 @@ typedef struct topkv_batch {
   const int64_t* cu_seq_lens;    /* DEVICE int64 [R+1] from topkv_build_plan, or NULL: then */
                                  /* each CTA derives it (allowed for R <= TOPKV_MAX_INLINE_R)*/
   int64_t total_tokens;          /* T if the host knows it, else -1. When -1 the capacity   */
-                                 /* checks are skipped and the caller guarantees them.      */
+                                 /* checks are skipped and the caller guarantees them. A    */
+                                 /* stated total must equal the sum of seq_lens: it bounds  */
+                                 /* the slab and, for a ragged batch, the number of CTAs    */
+                                 /* (T / span + R instead of one per block-table column); a */
+                                 /* total below the device lengths raises error bit 4.      */
   int32_t window_tokens;         /* 0 = every token. W > 0 = a windowed layer (§2.2): only  */
                                  /* the last min(s_r, W) tokens of each request are kept,   */
                                  /* so only they are packed / unpacked; T, cu_seq_lens and  */

@@ -323,8 +323,22 @@ int launch_copy(KParams kp, const Resolved& rs, int F, cudaStream_t stream, int 
   if (!handled) {
     span_geometry(&kp, F, rs.row_bytes);
     window_spans(&kp);
-    const int64_t spans = (int64_t)kp.R * (kp.wspr > 0 ? kp.wspr : kp.spr);
+    int64_t spans = (int64_t)kp.R * (kp.wspr > 0 ? kp.wspr : kp.spr);
     const bool walk = max_ctas > 0 && spans > max_ctas;
+    // A ragged batch fills far fewer block-table columns than R * max_pages_per_req: when the
+    // caller has stated the total, total / span + R CTAs are enough for every span that can hold
+    // tokens, and each finds its place from the lengths (worth it from 10 % fewer CTAs on). The
+    // search runs before the kernel's wait for its predecessor where the flags allow that; a
+    // launch that must wait first would only lengthen its start by it, and keeps the plain grid.
+    kp.compact = 0;
+    if (!walk && !linked && (kp.overlap || kp.late_wait) && kp.T >= 0 && kp.window == 0 && kp.cpp == 1 && kp.const_len == 0 &&
+        kp.R <= kThreads) {
+      const int64_t bound = kp.T / ((int64_t)kp.ppc * kp.P) + kp.R;
+      if (bound * 10 < spans * 9) {
+        kp.compact = 1;
+        spans = bound;
+      }
+    }
     const dim3 grid((unsigned)(walk ? max_ctas : spans), (unsigned)layers);
     cudaError_t le;
     if (copy_vector_bytes(kp, rs.unit_bytes, layers) == 32) {

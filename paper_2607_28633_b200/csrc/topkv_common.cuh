@@ -31,6 +31,9 @@ struct KParams {
   int ppc, spr;           // vectorised family: page columns per CTA, CTAs per request
   int wspr;               // windowed layer: only the `wspr` spans per request that the window can touch get
                           // a CTA, counted from the span of the first kept token (0 = all `spr` spans)
+  int compact;            // 1: the grid holds one CTA per span that CAN hold tokens (total_tokens / span + R of
+                          // them) instead of one per block-table column; each CTA finds its request and
+                          // span from the lengths (ragged batches: nearly half the columns are empty)
   int cpp, tps;           // pages far larger than a CTA's span are split: CTAs per page (1 = whole
                           // pages), tokens per CTA of a split page
   int const_len;          // > 0: every request has exactly this many tokens; sl and cu are not read

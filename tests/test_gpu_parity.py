@@ -325,6 +325,84 @@ def test_unusable_tables_are_skipped_not_followed(dev, path, variant):
     tk.check(tk.topkv_reset_device_error_flags())
 
 
+@pytest.mark.parametrize("R", [1, 7, 33, 256, 257])
+def test_compact_grid_for_ragged_batches(dev, R, variant):
+    """One long request among many short and empty ones: the block-table row is long, most of
+    its columns are empty for most requests, and with the total stated the grid holds one CTA
+    per span that can hold tokens (total / span + R) instead of one per column, each CTA finding
+    its request from the lengths (up to 256 requests; beyond that, and with an unknown total,
+    one CTA per column as before). Pack and unpack against the oracle for every form; a stated
+    total below what the device lengths add up to raises the wire bit and touches nothing
+    outside the slab."""
+    rng = np.random.default_rng(1000 + R)
+    for P, H, D in ((16, 8, 128), (4, 1, 64)):
+        F, E = 2, 2
+        sl = rng.integers(0, 3 * P + 2, size=R).astype(np.int32)
+        if R > 2:
+            sl[rng.integers(0, R, size=max(1, R // 5))] = 0
+        sl[rng.integers(0, R)] = 645                               # one long request: a long row
+        pages = (sl + P - 1) // P
+        maxp = int(pages.max()) + 2
+        npages = int(pages.sum()) + 3
+        g = Geom(L=2, F=F, h_kv=H, d_h=D, b_p=E, P=P, num_pages=npages)
+        T = int(sl.sum())
+        g.W_layer = g.wire_layer_bytes(T) + 32
+        bt_s = np.full((R, maxp), -1, dtype=np.int32)
+        bt_d = np.full((R, maxp), -1, dtype=np.int32)
+        ps, pd, pos = rng.permutation(npages), rng.permutation(npages), 0
+        for r in range(R):
+            bt_s[r, :pages[r]] = ps[pos:pos + pages[r]]
+            bt_d[r, :pages[r]] = pd[pos:pos + pages[r]]
+            pos += pages[r]
+        lo = _layout_from_geom(g)
+        src_h = rng.integers(0, 256, g.L * g.S_layer, dtype=np.uint8)
+        dst_h0 = rng.integers(0, 256, g.L * g.S_layer, dtype=np.uint8)
+        src = torch.from_numpy(src_h).to(dev)
+        d_sl = torch.from_numpy(sl).to(dev)
+        d_bs, d_bd = torch.from_numpy(bt_s).to(dev), torch.from_numpy(bt_d).to(dev)
+        want = np.full(g.L * g.W_layer + 64, 0x3C, dtype=np.uint8)
+        want_dst = dst_h0.copy()
+        for layer in range(g.L):
+            oracle.pack(g, layer, src_h, bt_s, sl, wire=want)
+            oracle.unpack(g, layer, want_dst, bt_d, sl, want)
+        for total in (T, -1):
+            cu = None
+            wire = torch.full((g.L * g.W_layer + 64,), 0x3C, dtype=torch.uint8, device=dev)
+            dst = torch.from_numpy(dst_h0).to(dev)
+            # the compact grid is taken by launches that may read their tables before they wait
+            # for the kernel before them; the tables here were uploaded long before
+            ts = tk.TOPKV_FLAG_TABLES_SETTLED
+            bs, bd = tk.make_batch(d_bs, d_sl, total, cu, ts), tk.make_batch(d_bd, d_sl, total, cu, ts)
+            for layer in range(g.L):
+                tk.check(tk.topkv_pack_layer(layer, src, lo, bs, wire, wire.numel()))
+                tk.check(tk.topkv_unpack_layer(layer, dst, lo, bd, wire, wire.numel()))
+            torch.cuda.synchronize()
+            assert tk.topkv_device_error_flags() == 0
+            assert np.array_equal(wire.cpu().numpy(), want), (P, total)
+            assert np.array_equal(dst.cpu().numpy(), want_dst), (P, total)
+            # both layers in one launch
+            wire.fill_(0x3C)
+            tk.check(tk.topkv_pack_layers(0, g.L, src, lo, bs, wire, wire.numel()))
+            torch.cuda.synchronize()
+            assert np.array_equal(wire.cpu().numpy(), want), (P, total, "range")
+        # a total that understates the device lengths: reported, nothing outside the slab touched
+        if T > 4 * P:
+            short = T - 3 * P
+            n_short = g.wire_layer_bytes(short)
+            guard = 4096
+            buf = torch.full((guard + n_short + guard,), 0xC3, dtype=torch.uint8, device=dev)
+            lo1 = _layout_from_geom(g)
+            lo1.wire_layer_stride = 0
+            tk.check(tk.topkv_reset_device_error_flags())
+            tk.check(tk.topkv_pack_layer(0, src, lo1, tk.make_batch(d_bs, d_sl, short, None,
+                                                                    tk.TOPKV_FLAG_TABLES_SETTLED),
+                                         buf[guard:], n_short))
+            assert tk.topkv_device_error_flags() & 4
+            out = buf.cpu().numpy()
+            assert (out[:guard] == 0xC3).all() and (out[guard + n_short:] == 0xC3).all()
+            tk.check(tk.topkv_reset_device_error_flags())
+
+
 # -------------------------------------------------------------------- benchmark shapes
 
 def _check_layers(w, layers, dev, threads=8):
