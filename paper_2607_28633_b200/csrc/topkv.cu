@@ -331,7 +331,7 @@ int launch_copy(KParams kp, const Resolved& rs, int F, cudaStream_t stream, int 
     // search runs before the kernel's wait for its predecessor where the flags allow that; a
     // launch that must wait first would only lengthen its start by it, and keeps the plain grid.
     kp.compact = 0;
-    if (!walk && !linked && (kp.overlap || kp.late_wait) && kp.T >= 0 && kp.window == 0 && kp.cpp == 1 && kp.const_len == 0 &&
+    if (!walk && (kp.overlap || kp.late_wait) && kp.T >= 0 && kp.window == 0 && kp.cpp == 1 && kp.const_len == 0 &&
         kp.R <= kThreads) {
       const int64_t bound = kp.T / ((int64_t)kp.ppc * kp.P) + kp.R;
       if (bound * 10 < spans * 9) {

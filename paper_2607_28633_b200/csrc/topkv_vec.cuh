@@ -54,9 +54,11 @@ __device__ __forceinline__ int64_t block_prefix(const int32_t* __restrict__ sl, 
 // One CTA per (request, page column). F: planes per token; PACK: pool -> wire, else
 // wire -> pool; MERGED: the valid tokens of a page form one contiguous run per plane on
 // both sides (MLA rows, or PLANAR wire with a token-contiguous pool).
-// Returns (uniformly over the CTA) whether the span holds any token this layer keeps.
+// Returns (uniformly over the CTA) -1 when the span holds no token this layer keeps, else the
+// span's number r * spr + (span of request r), whichever CTA of whichever grid form took it:
+// that number indexes the flags of a span link.
 template <int F, bool PACK, bool MERGED, int VEC, bool MULTI>
-__device__ __forceinline__ bool copy_span_work(const KParams& p, const int slot) {
+__device__ __forceinline__ int copy_span_work(const KParams& p, const int slot) {
   // A span = `ppc` consecutive page columns of one request (one page when pages are large;
   // several small pages, so that every CTA moves a few tens of KiB).
   __shared__ int32_t s_pages[kMaxPagesPerCta];
@@ -101,14 +103,14 @@ __device__ __forceinline__ bool copy_span_work(const KParams& p, const int slot)
     __syncthreads();
     r = s_hit[0];
     sidx = s_hit[1];
-    if (r < 0) return false;
+    if (r < 0) return -1;
   }
   const int s_r = p.const_len > 0 ? p.const_len : p.sl[r];
   // first token this layer keeps: 0, or s_r - window for a windowed layer (§2.2)
   const int b_r = (p.window > 0 && s_r > p.window) ? s_r - p.window : 0;
   if (p.wspr > 0) {            // counted from the span that holds the first kept token
     sidx += b_r / (p.ppc * p.P);
-    if (sidx >= p.spr) return false;
+    if (sidx >= p.spr) return -1;
   }
   // The span: `ppc` whole page columns from column j0 on, or, when pages are far larger than a
   // CTA's share, `tps` tokens of page column j0 (`cpp` CTAs per page).
@@ -129,12 +131,13 @@ __device__ __forceinline__ bool copy_span_work(const KParams& p, const int slot)
     if (tid == 0 && sidx == 0) raise_error(kErrTable);
   }
   const int lo = max(first, b_r);
-  if (lo >= hi) return false;
+  if (lo >= hi) return -1;
+  const int span_id = r * p.spr + sidx;
   // linked launch: ask for this span's flag now, so that the answer travels while the rest of
   // the tables is read; it is looked at (and asked for again, if need be) just before data is
   // touched
   const int32_t* const link_flag =
-      p.link_await != nullptr ? p.link_await + ((int64_t)blockIdx.y * gridDim.x + slot) : nullptr;
+      p.link_await != nullptr ? p.link_await + ((int64_t)blockIdx.y * p.R * p.spr + span_id) : nullptr;
   int link_seen = 0;
   if (link_flag != nullptr && tid == 0) link_seen = ld_acquire_gpu(link_flag);
   const int v = hi - lo;                // kept tokens in this span
@@ -172,7 +175,7 @@ __device__ __forceinline__ bool copy_span_work(const KParams& p, const int slot)
                                : (n0 >= 0 && (n0 + v) * F * row <= p.wire_limit);
     if (!fits) {
       if (tid == 0) raise_error(kErrWire);
-      return true;
+      return span_id;
     }
   }
   // tables read, addresses known: from here on the pool and the wire are touched
@@ -194,7 +197,7 @@ __device__ __forceinline__ bool copy_span_work(const KParams& p, const int slot)
     __syncthreads();
     if (s_link_failed) {  // the span is skipped and reported; nothing was touched
       if (tid == 0) raise_error(kErrWait);
-      return true;
+      return span_id;
     }
   }
   constexpr int kUnroll = VEC == 32 ? kUnroll32 : kUnroll16;
@@ -229,7 +232,7 @@ __device__ __forceinline__ bool copy_span_work(const KParams& p, const int slot)
         }
       }
     }
-    return true;
+    return span_id;
   }
 
   // Units of the span in wire order: q = (ts*F + c)*U + h (TOKEN_KV) or q = (c*v + ts)*U + h
@@ -239,9 +242,9 @@ __device__ __forceinline__ bool copy_span_work(const KParams& p, const int slot)
   const int groups = kThreads / tpu;
   const int my_g = tid / tpu;
   const int my_w = tid - my_g * tpu;
-  if (my_g >= groups) return true;
+  if (my_g >= groups) return span_id;
   uint8_t* wire_span = wire + n0 * F * p.U * unit_bytes;  // TOKEN_KV: the span is one run
-  if (!MULTI && s_pages[0] < 0) return true;                // single page, unusable: skip it
+  if (!MULTI && s_pages[0] < 0) return span_id;                // single page, unusable: skip it
   uint8_t* page0 = pool + (int64_t)s_pages[0] * p.S_page + (int64_t)ts0 * p.S_tok;
 
   for (int q0 = my_g; q0 < nunits; q0 += groups * kUnroll) {
@@ -288,7 +291,7 @@ __device__ __forceinline__ bool copy_span_work(const KParams& p, const int slot)
       }
     }
   }
-  return true;
+  return span_id;
 }
 
 // One span, and, for a linked launch, the publication of its flag once every thread of the CTA
@@ -296,11 +299,11 @@ __device__ __forceinline__ bool copy_span_work(const KParams& p, const int slot)
 // the same lengths, do not wait for them either).
 template <int F, bool PACK, bool MERGED, int VEC, bool MULTI>
 __device__ __forceinline__ void copy_span(const KParams& p, const int slot) {
-  const bool nonempty = copy_span_work<F, PACK, MERGED, VEC, MULTI>(p, slot);
-  if (p.link_signal != nullptr && nonempty) {
+  const int span_id = copy_span_work<F, PACK, MERGED, VEC, MULTI>(p, slot);
+  if (p.link_signal != nullptr && span_id >= 0) {
     __syncthreads();  // every thread's stores are ordered before thread 0's release below
     if (threadIdx.x == 0)
-      st_release_gpu(p.link_signal + ((int64_t)blockIdx.y * gridDim.x + slot), p.signal_epoch);
+      st_release_gpu(p.link_signal + ((int64_t)blockIdx.y * p.R * p.spr + span_id), p.signal_epoch);
   }
 }
 
