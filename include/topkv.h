@@ -282,7 +282,9 @@ int topkv_relay_layers_linked(int first_layer, int num_layers, const void* src_p
  * role (§3.5) and the cache must move into the other role's pool.
  * The two layouts must agree in kv_factor, num_kv_heads, head_dim and elem_bytes; everything
  * else may differ. Lengths are read from src_batch->seq_lens (dst_batch->seq_lens must hold
- * the same values); cu_seq_lens and total_tokens are not used. The launch overlaps the
+ * the same values); cu_seq_lens is not used; src_batch->total_tokens, when stated (>= 0), must
+ * be the sum of the lengths and lets a ragged batch launch one CTA per span that can hold
+ * tokens (a total below the device lengths raises error bit 4). The launch overlaps the
  * previous kernel only if BOTH batches carry TOPKV_FLAG_OVERLAP_PREVIOUS. Preconditions as for
  * unpack: no two requests share a destination page; the pools do not overlap. */
 int topkv_repage_layer(int layer, const void* src_pool, const topkv_layout* src_layout,

@@ -1470,7 +1470,17 @@ int topkv_repage_layer(int layer, const void* src_pool, const topkv_layout* src_
                       (uintptr_t)p.Ss_page | (uintptr_t)p.Ss_kv | (uintptr_t)p.Ss_tok |
                       (uintptr_t)p.Ss_unit | (uintptr_t)p.Sd_page | (uintptr_t)p.Sd_kv |
                       (uintptr_t)p.Sd_tok | (uintptr_t)p.Sd_unit | (uintptr_t)unit_bytes) & 31) == 0;
-  const dim3 grid((unsigned)((int64_t)p.R * p.spr)), block(kRepageThreads);
+  // a ragged batch whose total the caller has stated: one CTA per span that can hold tokens
+  int64_t spans = (int64_t)p.R * p.spr;
+  p.compact = 0;
+  if (p.overlap && src_batch->total_tokens >= 0 && p.R <= kRepageThreads) {
+    const int64_t bound = src_batch->total_tokens / p.span_tokens + p.R;
+    if (bound * 10 < spans * 9) {
+      p.compact = 1;
+      spans = bound;
+    }
+  }
+  const dim3 grid((unsigned)spans), block(kRepageThreads);
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   cudaError_t le;
   if (wide) {

@@ -94,6 +94,46 @@ __device__ __forceinline__ void st_release_gpu(int32_t* p, int v) {
   asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
+// The compact grid of a ragged batch: CTA `slot` takes the slot-th span that holds tokens,
+// counted request by request (request q has ceil(min(s_q, row_tokens) / span_tokens) of them).
+// An inclusive scan of those counts over the CTA (R <= THREADS), then the one thread whose
+// request contains that span says so. Returns false (uniformly) when `slot` lies past the last
+// span. If there are more spans than CTAs, the lengths on the device exceed the total the grid
+// was sized from: CTA 0 raises the wire bit.
+template <int THREADS>
+__device__ __forceinline__ bool find_span(const int32_t* __restrict__ sl, int R, int row_tokens,
+                                          int span_tokens, int slot, int* r_out, int* sidx_out) {
+  __shared__ int s_scan[THREADS / 32];
+  __shared__ int s_hit[2];
+  const int t = threadIdx.x, lane = t & 31, wid = t >> 5;
+  int n_q = 0;
+  if (t < R) n_q = (min(max(sl[t], 0), row_tokens) + span_tokens - 1) / span_tokens;
+  int incl = n_q;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int up = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += up;
+  }
+  if (lane == 31) s_scan[wid] = incl;
+  if (t == 0) s_hit[0] = -1;
+  __syncthreads();
+  int total = 0;
+#pragma unroll
+  for (int w = 0; w < THREADS / 32; ++w) {
+    if (w < wid) incl += s_scan[w];
+    total += s_scan[w];
+  }
+  if (n_q > 0 && slot >= incl - n_q && slot < incl) {
+    s_hit[0] = t;
+    s_hit[1] = slot - (incl - n_q);
+  }
+  if (t == 0 && slot == 0 && total > (int)gridDim.x) raise_error(kErrWire);
+  __syncthreads();
+  *r_out = s_hit[0];
+  *sidx_out = s_hit[1];
+  return s_hit[0] >= 0;
+}
+
 // Streaming vector accesses: every byte is touched exactly once, so neither side should
 // displace anything useful from L1 / L2. Vec<32> uses the 256-bit global accesses of sm_100.
 template <int VEC>

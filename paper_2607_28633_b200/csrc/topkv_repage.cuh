@@ -27,6 +27,7 @@ struct RepageParams {
   int unit_chunks;  // VEC-byte chunks per unit
   int span_tokens;  // tokens per CTA
   int spr;          // CTAs per request
+  int compact;      // 1: one CTA per span that can hold tokens (see find_span), not per (request, span) slot
   int overlap;
 };
 
@@ -38,10 +39,16 @@ __global__ void __launch_bounds__(kRepageThreads, 3) topkv_repage_kernel(const R
   constexpr int kUnroll = VEC == 32 ? 4 : 8;
   const int tid = threadIdx.x;
   const int slot = blockIdx.x;
-  const int r = slot / p.spr;
-  const int first = (slot - r * p.spr) * p.span_tokens;
-  int s_r = p.sl[r];
   const int64_t row_tokens = min((int64_t)p.maxp_s * p.Ps, (int64_t)p.maxp_d * p.Pd);
+  int r = slot / p.spr;
+  int sidx = slot - r * p.spr;
+  if (p.compact &&
+      !find_span<kRepageThreads>(p.sl, p.R, (int)min(row_tokens, (int64_t)0x7fffffff), p.span_tokens, slot, &r, &sidx)) {
+    pdl_epilogue(p.overlap);
+    return;
+  }
+  const int first = sidx * p.span_tokens;
+  int s_r = p.sl[r];
   if (s_r > row_tokens) {  // longer than a block-table row: copy what both rows describe
     s_r = (int)row_tokens;
     if (tid == 0 && first == 0) raise_error(kErrTable);

@@ -69,42 +69,7 @@ __device__ __forceinline__ int copy_span_work(const KParams& p, const int slot) 
   const int gspr = p.wspr > 0 ? p.wspr : p.spr;  // spans per request that have a CTA
   int r = slot / gspr;
   int sidx = slot - r * gspr;  // span of request r
-  if (p.compact) {
-    // CTA `slot` takes the slot-th span that holds tokens, counted request by request: an
-    // inclusive scan of the spans per request over the CTA (R <= kThreads), then the one thread
-    // whose request contains that span says so.
-    __shared__ int s_scan[kThreads / 32];
-    __shared__ int s_hit[2];
-    const int t = threadIdx.x, lane = t & 31, wid = t >> 5;
-    const int st = p.ppc * p.P;
-    int n_q = 0;
-    if (t < p.R) n_q = (min(max(p.sl[t], 0), p.maxp * p.P) + st - 1) / st;
-    int incl = n_q;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int up = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += up;
-    }
-    if (lane == 31) s_scan[wid] = incl;
-    if (t == 0) s_hit[0] = -1;
-    __syncthreads();
-    int total = 0;
-#pragma unroll
-    for (int w = 0; w < kThreads / 32; ++w) {
-      if (w < wid) incl += s_scan[w];
-      total += s_scan[w];
-    }
-    if (n_q > 0 && slot >= incl - n_q && slot < incl) {
-      s_hit[0] = t;
-      s_hit[1] = slot - (incl - n_q);
-    }
-    // more spans than CTAs: the lengths on the device exceed the total the caller stated
-    if (t == 0 && slot == 0 && total > (int)gridDim.x) raise_error(kErrWire);
-    __syncthreads();
-    r = s_hit[0];
-    sidx = s_hit[1];
-    if (r < 0) return -1;
-  }
+  if (p.compact && !find_span<kThreads>(p.sl, p.R, p.maxp * p.P, p.ppc * p.P, slot, &r, &sidx)) return -1;
   const int s_r = p.const_len > 0 ? p.const_len : p.sl[r];
   // first token this layer keeps: 0, or s_r - window for a windowed layer (§2.2)
   const int b_r = (p.window > 0 && s_r > p.window) ? s_r - p.window : 0;
