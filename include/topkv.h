@@ -659,6 +659,16 @@ int topkv_reset_device_error_flags(void);
 int topkv_copy_vector_bytes(int first_layer, int num_layers, const void* pool,
                             const topkv_layout* layout, const topkv_batch* batch,
                             const void* d_wire, int64_t wire_bytes);
+/* Number of CTAs per layer that topkv_pack_layer / topkv_unpack_layer would launch for these
+ * arguments in the vectorised kernel family (same arguments, same checks, nothing is launched;
+ * a negative topkv_status when they would be refused). One CTA per span of a block-table row
+ * (R * spans per row), or, for a ragged batch whose total is stated and whose launch may read
+ * its tables before it waits for its predecessor (either flag), total_tokens / span_tokens + R
+ * CTAs: *compact (may be NULL) says which. Whatever the lengths, as long as they add up to
+ * total_tokens, that many CTAs cover every span that holds tokens. */
+int64_t topkv_copy_grid_ctas(int layer, const void* pool, const topkv_layout* layout,
+                             const topkv_batch* batch, const void* d_wire, int64_t wire_bytes,
+                             int32_t* compact);
 /* Number of kernels this library has launched in this process (all threads). */
 int64_t topkv_kernel_launch_count(void);
 /* Selects the kernel family used by the four hot calls: 0 = vectorised load/store,

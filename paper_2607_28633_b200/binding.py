@@ -46,7 +46,7 @@ EXPORTS = (
     "topkv_retry", "topkv_pack_layer_to_host_crc", "topkv_unpack_layer_from_host_crc",
     "topkv_set_host_leg_ctas", "topkv_pack_layers_to_host_pipelined",
     "topkv_unpack_layers_from_host_pipelined", "topkv_pack_layers", "topkv_unpack_layers",
-    "topkv_copy_vector_bytes", "topkv_select_transport", "topkv_planning_rate",
+    "topkv_copy_vector_bytes", "topkv_copy_grid_ctas", "topkv_select_transport", "topkv_planning_rate",
     "topkv_transport_name", "topkv_layer_table_offsets", "topkv_pack_model_layers",
     "topkv_unpack_model_layers", "topkv_pack_model_layers_to_host_pipelined",
     "topkv_unpack_model_layers_from_host_pipelined", "topkv_span_link_words",
@@ -249,6 +249,8 @@ def lib() -> ctypes.CDLL:
         L.topkv_transport_name.argtypes = [c_int]
         L.topkv_transport_name.restype = ctypes.c_char_p
         L.topkv_copy_vector_bytes.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64]
+        L.topkv_copy_grid_ctas.restype = c_int64
+        L.topkv_copy_grid_ctas.argtypes = [c_int, c_void_p, lp, bp, c_void_p, c_int64, ctypes.POINTER(c_int32)]
         for fn in (L.topkv_pack_layers_to_host_pipelined, L.topkv_unpack_layers_from_host_pipelined):
             fn.argtypes = [c_int, c_int, c_void_p, lp, bp, c_void_p, c_int64, c_void_p, c_int64,
                            c_void_p, c_void_p, c_void_p]
@@ -343,6 +345,14 @@ def topkv_unpack_layers(first_layer, num_layers, dst_pool, layout, batch, d_wire
                         stream=None):
     return lib().topkv_unpack_layers(first_layer, num_layers, _ptr(dst_pool), ctypes.byref(layout),
                                      ctypes.byref(batch), _ptr(d_wire), wire_bytes, _stream(stream))
+
+
+def topkv_copy_grid_ctas(layer, pool, layout, batch, d_wire, wire_bytes):
+    """(CTAs per layer or a negative status, compact grid or not)."""
+    compact = c_int32(0)
+    n = lib().topkv_copy_grid_ctas(layer, _ptr(pool), ctypes.byref(layout), ctypes.byref(batch), _ptr(d_wire),
+                                   wire_bytes, ctypes.byref(compact))
+    return int(n), bool(compact.value)
 
 
 def topkv_copy_vector_bytes(first_layer, num_layers, pool, layout, batch, d_wire, wire_bytes):

@@ -306,6 +306,32 @@ void window_spans(KParams* kp) {
   if (need < kp->spr) kp->wspr = (int)need;
 }
 
+// Cuts the batch into spans and decides how many CTAs per layer the vectorised family launches
+// (fills ppc, spr, cpp, tps, wspr, compact). *walk: the grid is bounded by max_ctas and every CTA
+// walks several spans.
+int64_t grid_spans(KParams* kp, int F, int64_t row_bytes, int max_ctas, bool* walk) {
+  span_geometry(kp, F, row_bytes);
+  window_spans(kp);
+  int64_t spans = (int64_t)kp->R * (kp->wspr > 0 ? kp->wspr : kp->spr);
+  *walk = max_ctas > 0 && spans > max_ctas;
+  // A ragged batch fills far fewer block-table columns than R * max_pages_per_req: when the
+  // caller has stated the total, total / span + R CTAs are enough for every span that can hold
+  // tokens (request q has ceil(s_q / span) <= s_q / span + 1 of them), and each finds its place
+  // from the lengths (worth it from 10 % fewer CTAs on). The search runs before the kernel's
+  // wait for its predecessor where the flags allow that; a launch that must wait first would
+  // only lengthen its start by it, and keeps the plain grid.
+  kp->compact = 0;
+  if (!*walk && (kp->overlap || kp->late_wait) && kp->T >= 0 && kp->window == 0 && kp->cpp == 1 &&
+      kp->const_len == 0 && kp->R <= kThreads) {
+    const int64_t bound = kp->T / ((int64_t)kp->ppc * kp->P) + kp->R;
+    if (bound * 10 < spans * 9) {
+      kp->compact = 1;
+      spans = bound;
+    }
+  }
+  return spans;
+}
+
 // max_ctas > 0: the wire is host memory behind PCIe; at most that many CTAs walk the spans.
 // layers > 1: one launch covers that many consecutive layers (kp describes the first one and
 // carries the layer strides); the vectorised family only.
@@ -321,24 +347,8 @@ int launch_copy(KParams kp, const Resolved& rs, int F, cudaStream_t stream, int 
     if (st != TOPKV_OK) return st;
   }
   if (!handled) {
-    span_geometry(&kp, F, rs.row_bytes);
-    window_spans(&kp);
-    int64_t spans = (int64_t)kp.R * (kp.wspr > 0 ? kp.wspr : kp.spr);
-    const bool walk = max_ctas > 0 && spans > max_ctas;
-    // A ragged batch fills far fewer block-table columns than R * max_pages_per_req: when the
-    // caller has stated the total, total / span + R CTAs are enough for every span that can hold
-    // tokens, and each finds its place from the lengths (worth it from 10 % fewer CTAs on). The
-    // search runs before the kernel's wait for its predecessor where the flags allow that; a
-    // launch that must wait first would only lengthen its start by it, and keeps the plain grid.
-    kp.compact = 0;
-    if (!walk && (kp.overlap || kp.late_wait) && kp.T >= 0 && kp.window == 0 && kp.cpp == 1 && kp.const_len == 0 &&
-        kp.R <= kThreads) {
-      const int64_t bound = kp.T / ((int64_t)kp.ppc * kp.P) + kp.R;
-      if (bound * 10 < spans * 9) {
-        kp.compact = 1;
-        spans = bound;
-      }
-    }
+    bool walk = false;
+    const int64_t spans = grid_spans(&kp, F, rs.row_bytes, max_ctas, &walk);
     const dim3 grid((unsigned)(walk ? max_ctas : spans), (unsigned)layers);
     cudaError_t le;
     if (copy_vector_bytes(kp, rs.unit_bytes, layers) == 32) {
@@ -1651,6 +1661,22 @@ int topkv_copy_vector_bytes(int first_layer, int num_layers, const void* pool, c
                                     &launch);
   if (st != TOPKV_OK) return st;
   return launch ? copy_vector_bytes(kp, rs.unit_bytes, num_layers) : 0;
+}
+
+int64_t topkv_copy_grid_ctas(int layer, const void* pool, const topkv_layout* layout, const topkv_batch* batch,
+                             const void* d_wire, int64_t wire_bytes, int32_t* compact) {
+  KParams kp;
+  Resolved rs;
+  int64_t n_layer;
+  const int st = prepare(layer, pool, layout, batch, d_wire, wire_bytes, layout ? layout->wire_layer_stride : 0,
+                         &kp, &rs, &n_layer);
+  if (st != TOPKV_OK) return st;
+  if (compact != nullptr) *compact = 0;
+  if ((int64_t)kp.R * kp.maxp == 0) return 0;
+  bool walk = false;
+  const int64_t spans = grid_spans(&kp, (int)layout->kv_factor, rs.row_bytes, 0, &walk);
+  if (compact != nullptr) *compact = kp.compact;
+  return spans;
 }
 
 int topkv_set_host_leg_ctas(int ctas) {

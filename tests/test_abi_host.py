@@ -553,3 +553,67 @@ def test_relay_linked_validation_without_gpu():
     assert R(0, 4, src, lo, b, dst, lo, b, slab, n, flags, 2 * words, 0x7fffffff) == tk.TOPKV_ERR_INVALID_ARG
     assert R(0, 0, src, lo, b, dst, lo, b, slab, n, flags, 2 * words, 0) == tk.TOPKV_OK
     assert tk.topkv_kernel_launch_count() == before
+
+
+def test_compact_grid_covers_every_span_that_can_hold_tokens():
+    """The grid of a ragged batch whose total is stated: total / span + R CTAs. Whatever lengths
+    add up to that total, the spans that hold tokens (request q: ceil(s_q / span)) are never more
+    than the CTAs launched; the compact form is taken only by launches that may read their tables
+    before they wait (either flag), with a stated total, no window, at most 256 requests, and
+    only when it saves a tenth of the CTAs. Host logic only: nothing is launched."""
+    import numpy as np
+    rng = np.random.default_rng(5)
+    pool, wire = 0x7000000, 0x9000000
+    ov, ts = tk.TOPKV_FLAG_OVERLAP_PREVIOUS, tk.TOPKV_FLAG_TABLES_SETTLED
+    G = tk.topkv_copy_grid_ctas
+    before = tk.topkv_kernel_launch_count()
+    seen_compact = 0
+    for trial in range(300):
+        P = int(rng.choice([1, 4, 16, 64]))
+        H, D = int(rng.choice([1, 2, 8])), int(rng.choice([64, 128]))
+        R = int(rng.choice([1, 2, 7, 16, 64, 256]))
+        lo = tk.make_layout(2, 2, H, D, 2, P, 1 << 20)
+        page_bytes = P * 2 * H * D * 2
+        ppc_max = max(1, 65536 // page_bytes)
+        shape = rng.choice(["ragged", "equal", "one_long"])
+        if shape == "equal":
+            sl = np.full(R, int(rng.integers(1, 40 * P + 1)))
+        elif shape == "one_long":
+            sl = rng.integers(0, 3, size=R)
+            sl[rng.integers(0, R)] = int(rng.integers(100, 4000))
+        else:
+            sl = rng.integers(0, 60 * P, size=R)
+        maxp = int(max(1, -(-int(sl.max()) // P))) + int(rng.integers(0, 3))
+        ppc = max(1, min(64, maxp, ppc_max))
+        span = ppc * P                                    # tokens per CTA
+        spr = -(-maxp // ppc)
+        T = int(sl.sum())
+        filled = int((-(-sl // span)).sum())              # spans that hold tokens
+        split = page_bytes >= 2 * 65536 and P > 1         # pages far larger than a span: CTAs per page
+        if split:
+            tps = max(1, min(P, 65536 // (2 * H * D * 2)))
+            spr = maxp * (-(-P // tps))
+            filled = int(sum((s // P) * (-(-P // tps)) + -(-(s % P) // tps) for s in sl.tolist()))
+        n_layer = tk.topkv_wire_layer_bytes(lo, T)
+        for flags in (0, ov, ts):
+            b = tk.make_batch(_FakeTensor(0x10000, (R, maxp)), _FakeTensor(0x20000, (R,)), T, None, flags)
+            ctas, compact = G(0, pool, lo, b, wire, max(n_layer, 16))
+            assert ctas >= filled, (trial, P, R, maxp, T)
+            if flags == 0 or split:
+                assert not compact and ctas == R * spr
+            if compact:
+                seen_compact += 1
+                assert ctas == T // span + R and ctas * 10 < R * spr * 9
+            else:
+                assert ctas == R * spr
+        # an unknown total, a window, or more than 256 requests keep one CTA per block-table column
+        b = tk.make_batch(_FakeTensor(0x10000, (R, maxp)), _FakeTensor(0x20000, (R,)), -1, None, ov)
+        assert G(0, pool, lo, b, wire, 1 << 40) == (R * spr, False)
+    assert seen_compact > 50
+    big = tk.make_batch(_FakeTensor(0x10000, (257, 64)), _FakeTensor(0x20000, (257,)), 300, None, ov)
+    lo = tk.make_layout(2, 2, 8, 128, 2, 16, 1 << 20)
+    assert G(0, pool, lo, big, wire, 1 << 30) == (257 * 64, False)
+    b256 = tk.make_batch(_FakeTensor(0x10000, (256, 64)), _FakeTensor(0x20000, (256,)), 300, None, ov)
+    assert G(0, pool, lo, b256, wire, 1 << 30) == (300 // 16 + 256, True)
+    assert G(2, pool, lo, b256, wire, 1 << 30)[0] == tk.TOPKV_ERR_LAYER_RANGE
+    assert tk.topkv_kernel_launch_count() == before
