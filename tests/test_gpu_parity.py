@@ -2309,3 +2309,124 @@ def test_relay_call_right_behind_a_kernel_that_writes_its_source(dev, variant):
             assert np.array_equal(harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, l), dst_h[l]), (by_hand, l)
     del w
     torch.cuda.empty_cache()
+
+
+# -------------------------------------------------------------------- random call sequences
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_call_sequences_against_an_oracle_model(dev, seed, variant):
+    """A random sequence of calls on one stream (pack, unpack, layer ranges, re-paging, linked
+    pairs, staged and direct host legs; lengths from a plan or not, total stated or not, a
+    window or not) with the flags a caller may legitimately set: TOPKV_FLAG_OVERLAP_PREVIOUS only
+    when the call touches nothing that the calls since the last unflagged one touch,
+    TOPKV_FLAG_TABLES_SETTLED always (the tables are never written by a kernel here). The same
+    sequence is applied to numpy copies with the oracle; every buffer must agree at the end."""
+    g, sl, bt_s, bt_d, rng = _case(seed)
+    rng = np.random.default_rng(7000 + seed)
+    W = int(rng.choice([0, 0, 1, g.P + 1, 3 * g.P]))
+    g.window = W
+    T = g.kept_tokens(sl)
+    g.W_layer = g.wire_layer_bytes(T) + 16 * int(rng.integers(0, 3))
+    lo = _layout_from_geom(g)
+    nbytes = g.L * g.S_layer
+    wire_len = g.L * g.W_layer + 32
+    h = {"src": rng.integers(0, 256, nbytes, dtype=np.uint8), "dst": rng.integers(0, 256, nbytes, dtype=np.uint8),
+         "wire": rng.integers(0, 256, wire_len, dtype=np.uint8), "host": rng.integers(0, 256, wire_len, dtype=np.uint8)}
+    d = {k: torch.from_numpy(v.copy()).to(dev) for k, v in h.items() if k != "host"}
+    pinned = torch.from_numpy(h["host"].copy()).pin_memory()
+    staging = torch.zeros(max(g.W_layer, 16), dtype=torch.uint8, device=dev)
+    d_sl = torch.from_numpy(sl).to(dev)
+    d_bt = {"src": torch.from_numpy(bt_s).to(dev), "dst": torch.from_numpy(bt_d).to(dev)}
+    h_bt = {"src": bt_s, "dst": bt_d}
+    R = len(sl)
+    cu = torch.zeros(R + 1, dtype=torch.int64, device=dev)
+    tk.check(tk.topkv_build_plan(tk.make_batch(d_bt["src"], d_sl, window_tokens=W), cu))
+    words = max(1, tk.topkv_span_link_words(lo, tk.make_batch(d_bt["src"], d_sl, T, None, 0, W)))
+    link_flags = torch.zeros(words, dtype=torch.int32, device=dev)
+    epoch = 0
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream(dev)
+    since_unflagged = []          # (reads, writes) of the kernels since the last call without the flag
+
+    def batch(side, flags):
+        total = T if rng.integers(0, 2) else -1
+        plan = cu if rng.integers(0, 2) else None
+        return tk.make_batch(d_bt[side], d_sl, total, plan, flags, W)
+
+    def flags_for(reads, writes, may_overlap=True):
+        free = all(not (writes & (r2 | w2)) and not (reads & w2) for r2, w2 in since_unflagged)
+        if may_overlap and since_unflagged and free and rng.integers(0, 2):
+            since_unflagged.append((reads, writes))
+            return tk.TOPKV_FLAG_OVERLAP_PREVIOUS
+        since_unflagged[:] = [(reads, writes)]
+        return tk.TOPKV_FLAG_TABLES_SETTLED if rng.integers(0, 2) else 0
+
+    kinds = ["pack", "unpack", "pack_range", "unpack_range", "to_host", "from_host"]
+    if W == 0:
+        kinds.append("repage")
+    if variant == 0:
+        kinds.append("linked")
+    for step in range(14):
+        kind = str(rng.choice(kinds))
+        layer = int(rng.integers(0, g.L))
+        pool = str(rng.choice(["src", "dst"]))
+        if kind == "pack":
+            f = flags_for({(pool, layer)}, {("wire", layer)})
+            tk.check(tk.topkv_pack_layer(layer, d[pool], lo, batch(pool, f), d["wire"], wire_len, stream))
+            oracle.pack(g, layer, h[pool], h_bt[pool], sl, wire=h["wire"])
+        elif kind == "unpack":
+            f = flags_for({("wire", layer)}, {(pool, layer)})
+            tk.check(tk.topkv_unpack_layer(layer, d[pool], lo, batch(pool, f), d["wire"], wire_len, stream))
+            oracle.unpack(g, layer, h[pool], h_bt[pool], sl, h["wire"])
+        elif kind in ("pack_range", "unpack_range"):
+            first = int(rng.integers(0, g.L))
+            n = int(rng.integers(1, g.L - first + 1))
+            pools, wires = {(pool, l) for l in range(first, first + n)}, {("wire", l) for l in range(first, first + n)}
+            if kind == "pack_range":
+                f = flags_for(pools, wires)
+                tk.check(tk.topkv_pack_layers(first, n, d[pool], lo, batch(pool, f), d["wire"], wire_len, stream))
+                for l in range(first, first + n):
+                    oracle.pack(g, l, h[pool], h_bt[pool], sl, wire=h["wire"])
+            else:
+                f = flags_for(wires, pools)
+                tk.check(tk.topkv_unpack_layers(first, n, d[pool], lo, batch(pool, f), d["wire"], wire_len, stream))
+                for l in range(first, first + n):
+                    oracle.unpack(g, l, h[pool], h_bt[pool], sl, h["wire"])
+        elif kind == "repage":
+            other = "dst" if pool == "src" else "src"
+            f = flags_for({(pool, layer)}, {(other, layer)})
+            tk.check(tk.topkv_repage_layer(layer, d[pool], lo, batch(pool, f), d[other], lo, batch(other, f), stream))
+            tmp = np.zeros(wire_len, dtype=np.uint8)
+            oracle.pack(g, layer, h[pool], h_bt[pool], sl, wire=tmp)
+            oracle.unpack(g, layer, h[other], h_bt[other], sl, tmp)
+        elif kind == "linked":
+            other = "dst" if pool == "src" else "src"
+            since_unflagged[:] = []       # the first linked call waits for everything before it
+            lp = tk.make_span_link(None, 0, link_flags, epoch + 1, tk.TOPKV_LINK_WAIT_PREVIOUS)
+            tk.check(tk.topkv_pack_layer_linked(layer, d[pool], lo, batch(pool, 0), d["wire"], wire_len, lp, stream))
+            lu = tk.make_span_link(link_flags, epoch + 1, None, 0)
+            tk.check(tk.topkv_unpack_layer_linked(layer, d[other], lo, batch(other, 0), d["wire"], wire_len, lu,
+                                                  stream))
+            epoch += 1
+            oracle.pack(g, layer, h[pool], h_bt[pool], sl, wire=h["wire"])
+            oracle.unpack(g, layer, h[other], h_bt[other], sl, h["wire"])
+            # the next call must not carry the overlap flag: make it see both kernels as unflagged work
+            since_unflagged[:] = [({(pool, layer), ("wire", layer)}, {("wire", layer), (other, layer)})]
+        else:
+            staged = bool(rng.integers(0, 2))
+            st, cap = (staging, staging.numel()) if staged else (None, 0)
+            b = tk.make_batch(d_bt[pool], d_sl, T, cu if rng.integers(0, 2) else None, 0, W)
+            since_unflagged[:] = []       # a copy, or a kernel without the flag
+            if kind == "to_host":
+                tk.check(tk.topkv_pack_layer_to_host(layer, d[pool], lo, b, pinned, wire_len, st, cap, stream))
+                oracle.pack(g, layer, h[pool], h_bt[pool], sl, wire=h["host"])
+                since_unflagged[:] = [({(pool, layer)}, {("host", layer)})]
+            else:
+                tk.check(tk.topkv_unpack_layer_from_host(layer, d[pool], lo, b, pinned, wire_len, st, cap, stream))
+                oracle.unpack(g, layer, h[pool], h_bt[pool], sl, h["host"])
+                since_unflagged[:] = [({("host", layer)}, {(pool, layer)})]
+    stream.synchronize()
+    assert tk.topkv_device_error_flags() == 0
+    for k in ("src", "dst", "wire"):
+        assert np.array_equal(d[k].cpu().numpy(), h[k]), k
+    assert np.array_equal(pinned.numpy(), h["host"])
