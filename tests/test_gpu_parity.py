@@ -2252,6 +2252,53 @@ def test_relay_layers_linked_one_call(dev, variant):
         torch.cuda.empty_cache()
 
 
+def test_linked_relay_captured_in_a_cuda_graph(dev, variant):
+    """The linked relay of several layers through one slab captured in a CUDA graph together
+    with the clearing of its flag array (the epochs are plain arguments, so every replay starts
+    from cleared flags): nothing runs during the capture; after every replay, with new source
+    contents each time, the destination is the oracle's unpack of the oracle's pack."""
+    if variant == 1:
+        pytest.skip("span links belong to the vectorised family")
+    L = 4
+    spec = wl.with_layers(wl.CFG2, L)
+    w = harness.setup(spec, dev, need_wire=False)
+    b = w.batch
+    g = _geom(spec, b.num_pool_pages, 1, 0, 0)
+    n = w.n_layer
+    slab = torch.zeros(n, dtype=torch.uint8, device=dev)
+    words = tk.topkv_span_link_words(w.layout, w.src_batch)
+    flags = torch.zeros(2 * words, dtype=torch.int32, device=dev)
+    stream = torch.cuda.Stream(dev)
+    args = (w.src_pool, w.layout, w.src_batch, w.dst_pool, w.layout, w.dst_batch, slab, n, flags, flags.numel())
+    with torch.cuda.stream(stream):                      # warm up outside the capture
+        tk.check(tk.topkv_relay_layers_linked(0, 1, *args, 0, stream))
+    stream.synchronize()
+    dst0 = w.dst_pool.clone()
+    flags.zero_()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        flags.zero_()
+        tk.check(tk.topkv_relay_layers_linked(0, L, *args, 0, stream))
+    assert not flags.any()                               # capturing executed nothing
+    fresh = wl.fill_torch(2 * L * w.slab_bytes, 99, dev, raw_bits=True)
+    for rep in range(2):
+        w.src_pool.copy_(fresh[rep * L * w.slab_bytes:(rep + 1) * L * w.slab_bytes])
+        w.dst_pool.copy_(dst0)
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert tk.topkv_device_error_flags() == 0 and int(flags.max()) == L
+        for l in range(L):
+            src_h = harness.layer_slab_to_numpy(w.src_pool, w.slab_bytes, l)
+            want = oracle.pack(g, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=8)
+            dst_h = harness.layer_slab_to_numpy(dst0, w.slab_bytes, l)
+            oracle.unpack(g, 0, dst_h, b.dst_block_table, b.seq_lens, want, impl="rows", threads=8)
+            assert np.array_equal(harness.layer_slab_to_numpy(w.dst_pool, w.slab_bytes, l), dst_h), (rep, l)
+    del w, graph
+    torch.cuda.empty_cache()
+
+
 def test_relay_call_right_behind_a_kernel_that_writes_its_source(dev, variant):
     """The first launch of topkv_relay_layers_linked is an ordinary launch towards what precedes
     the call (TOPKV_LINK_WAIT_PREVIOUS): kernels that rewrite the source pool and the plan are
