@@ -212,6 +212,6 @@ const char* topkv_strerror(int status) {
   }
 }
 
-int topkv_version(void) { return 110; }
+int topkv_version(void) { return 120; }
 
 }  // extern "C"
