@@ -73,6 +73,10 @@ __device__ __forceinline__ int copy_span_work(const KParams& p, const int slot) 
   const int s_r = p.const_len > 0 ? p.const_len : p.sl[r];
   // first token this layer keeps: 0, or s_r - window for a windowed layer (§2.2)
   const int b_r = (p.window > 0 && s_r > p.window) ? s_r - p.window : 0;
+  // a length longer than its block-table row: reported by every CTA of the request (a windowed
+  // layer may run none for its first spans), and only what the row holds is copied
+  const bool over_long = s_r > p.maxp * p.P;
+  if (over_long && threadIdx.x == 0) raise_error(kErrTable);
   if (p.wspr > 0) {            // counted from the span that holds the first kept token
     sidx += b_r / (p.ppc * p.P);
     if (sidx >= p.spr) return -1;
@@ -91,10 +95,7 @@ __device__ __forceinline__ int copy_span_work(const KParams& p, const int slot) 
   }
   const int tid = threadIdx.x;
   int hi = min(first + span_tokens, s_r);
-  if (s_r > p.maxp * p.P) {  // length longer than its block-table row: copy what the row holds
-    hi = min(hi, p.maxp * p.P);
-    if (tid == 0 && sidx == 0) raise_error(kErrTable);
-  }
+  if (over_long) hi = min(hi, p.maxp * p.P);
   const int lo = max(first, b_r);
   if (lo >= hi) return -1;
   const int span_id = r * p.spr + sidx;

@@ -315,6 +315,14 @@ def test_unusable_tables_are_skipped_not_followed(dev, path, variant):
     long = sl.copy(); long[1] = 65
     flags, _ = run(bt, long, T, n)
     assert flags & 2
+    if path != "checksummed":                # the same under a window, however far past the row the length is
+        for s_long in (65, 200):
+            long[1] = s_long
+            d_bt, d_sl = torch.from_numpy(bt).to(dev), torch.from_numpy(long).to(dev)
+            buf = torch.full((n + 4096,), 0xC3, dtype=torch.uint8, device=dev)
+            tk.check(tk.topkv_reset_device_error_flags())
+            tk.check(tk.topkv_pack_layer(0, src, lo, tk.make_batch(d_bt, d_sl, -1, None, 0, 16), buf, n))
+            assert tk.topkv_device_error_flags() & 2, s_long
     # (c) device lengths that need more wire than the slab has
     more = sl.copy(); more[2] = 48
     bt48 = bt.copy(); bt48[2, 2] = 5
