@@ -93,6 +93,13 @@ def test_entry_points_survive_random_descriptors(seed):
             lambda: tk.topkv_pack_layer_linked(layer, pool, lo, b, wire, cap,
                                                tk.make_span_link(0xE000000, 1, 0xE100000 + off, 2)),
             lambda: tk.topkv_pack_layer_to_host_noalloc(layer, pool, lo, b, host, cap),
+            lambda: tk.topkv_unpack_layer_linked(layer, pool, lo, b, wire, cap,
+                                                 tk.make_span_link(0xE000000, 1, None, 0, int(rng.integers(0, 3)))),
+            lambda: tk.topkv_relay_layers_linked(layer, int(rng.integers(0, 4)), pool, lo, b, pool + (1 << 30), lo,
+                                                 b, wire, cap, 0xE000000, int(rng.choice([0, 64, 1 << 30])),
+                                                 int(rng.integers(0, 5)), None),
+            lambda: tk.topkv_unpack_layers_from_host_two_lanes(layer, 3, pool, lo, b, host, cap, [st, st + 4096],
+                                                               cap, None, None, [0x100, 0x200]),
         ]
         for fn in calls:
             st_code = fn()
@@ -102,6 +109,8 @@ def test_entry_points_survive_random_descriptors(seed):
         tk.topkv_wire_layer_bytes(lo, int(rng.integers(-2, 1 << 20)))
         tk.topkv_crc_workspace_bytes(lo, b.num_requests, b.max_pages_per_req)
         tk.topkv_span_link_words(lo, b)
+        n, compact = tk.topkv_copy_grid_ctas(layer, pool, lo, b, wire, cap)
+        assert n >= 0 or n in KNOWN, n
         kinds = [(int(rng.integers(0, 4)), int(rng.choice([0, 16, 128, 24, -1]))) for _ in range(4)]
         lens = np.asarray(rng.integers(0, 300, size=max(b.num_requests, 1)), dtype=np.int32)
         t = tk.make_layer_table(kinds, lens, 0xF000000, 0xF100000, 1 << 20, 4096, 64)
