@@ -978,6 +978,17 @@ def run_extra(name, dev, stream, args, peak):
                             "t_main_overlap_ms": round(r.t_main_overlap_ms, 3),
                             "exposed_ms": round(r.exposed_ms, 3),
                             "xfer_gbs_serial": round(r.xfer_gbs_serial, 2)}
+            if label == "oversubscribed":
+                # the direct form's interference against the number of CTAs that walk the spans
+                # (every one of them holds an SM for the whole run once the link is always busy)
+                sweep = {}
+                for ctas in (4, 8, 16):
+                    prev = tk.topkv_set_host_leg_ctas(ctas)
+                    r = overlap.run_overlap(w, pinned, None, pre, slots=slots)
+                    tk.topkv_set_host_leg_ctas(prev)
+                    sweep[str(ctas)] = {"hidden": round(r.hidden, 4), "slowdown": round(r.slowdown, 4),
+                                        "xfer_gbs_serial": round(r.xfer_gbs_serial, 2)}
+                pt["direct_by_host_leg_ctas"] = sweep
             out[label] = pt
             del w, pinned, staging, pre
             torch.cuda.empty_cache()
@@ -1005,7 +1016,7 @@ def run_extra(name, dev, stream, args, peak):
         staging = torch.empty(w.n_layer, dtype=torch.uint8, device=dev)
         pre = overlap.PrefillStandIn(dev, w.batch.seeds["data"] + 50)
         best = None
-        # direct = mapped stores from a bounded grid (the library's default, 16 CTAs);
+        # direct = mapped stores from a bounded grid (the library's default, 8 CTAs);
         # direct_cta_per_span = the same stores from one CTA per page span, for contrast
         for form, st, ctas in (("staged", staging, None), ("direct", None, None),
                                ("direct_cta_per_span", None, 0)):

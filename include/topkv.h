@@ -679,10 +679,13 @@ int topkv_set_kernel_variant(int variant);
  * d_staging == NULL), the PCIe transport of §3.3 / Table 4: n > 0 = at most n CTAs walk all
  * spans of pages (default TOPKV_DEFAULT_HOST_LEG_CTAS); 0 = one CTA per span, as for a device
  * wire. The PCIe link sets the pace of that leg, so a few CTAs keep it full while the rest of
- * the GPU stays with the prefill that runs beside the transfer (§5.2). Returns the previous
+ * the GPU stays with the prefill that runs beside the transfer (§5.2): on a B200 4 CTAs fill the
+ * link with stores and 6 with loads, and when the link is busy all the time every CTA beyond
+ * that holds an SM that a GEMM beside it cannot use (8 CTAs: 7 % slower prefill, 16: 40 %).
+ * Returns the previous
  * value, or TOPKV_ERR_INVALID_ARG for n < 0 or n > 65535. Process-wide; takes effect for calls
  * made after it returns. The bytes moved are the same for every setting. */
-#define TOPKV_DEFAULT_HOST_LEG_CTAS 16
+#define TOPKV_DEFAULT_HOST_LEG_CTAS 8
 int topkv_set_host_leg_ctas(int ctas);
 
 #ifdef __cplusplus

@@ -1447,7 +1447,7 @@ def test_host_leg_cta_bound_setter(dev):
     assert tk.topkv_set_host_leg_ctas(-1) == tk.TOPKV_ERR_INVALID_ARG
     assert tk.topkv_set_host_leg_ctas(1 << 16) == tk.TOPKV_ERR_INVALID_ARG
     prev = tk.topkv_set_host_leg_ctas(5)
-    assert prev == 16                                  # the documented default
+    assert prev == 8                                   # the documented default
     assert tk.topkv_set_host_leg_ctas(prev) == 5
 
 
