@@ -2307,6 +2307,51 @@ def test_linked_relay_captured_in_a_cuda_graph(dev, variant):
     torch.cuda.empty_cache()
 
 
+def test_linked_relay_many_calls_alternating_sources(dev, variant):
+    """The linked relay called 120 times in a row through the same slab and the same flag arrays
+    (epochs continuing), the source alternating at random between two pools with different
+    contents: a span read before it was rewritten, or rewritten before it was read, would leave
+    bytes of the other source in the destination. Checked against the oracle's result for the
+    source of the last call, every few calls."""
+    if variant == 1:
+        pytest.skip("span links belong to the vectorised family")
+    L = 3
+    spec = wl.with_layers(wl.CFG2, L)
+    w = harness.setup(spec, dev, need_wire=False)
+    b = w.batch
+    g = _geom(spec, b.num_pool_pages, 1, 0, 0)
+    n = w.n_layer
+    srcs = [w.src_pool, wl.fill_torch(w.src_pool.numel(), 4321, dev, raw_bits=True)]
+    want = []                                             # the oracle's destination pool per source
+    for src in srcs:
+        pool = w.dst_pool.cpu().numpy().copy()
+        for l in range(L):
+            src_h = harness.layer_slab_to_numpy(src, w.slab_bytes, l)
+            wire = oracle.pack(g, 0, src_h, b.src_block_table, b.seq_lens, impl="rows", threads=8)
+            oracle.unpack(g, 0, pool[l * w.slab_bytes:(l + 1) * w.slab_bytes], b.dst_block_table, b.seq_lens,
+                          wire, impl="rows", threads=8)
+        want.append(torch.from_numpy(pool).to(dev))
+    assert not torch.equal(want[0], want[1])
+    slab = torch.zeros(n, dtype=torch.uint8, device=dev)
+    words = tk.topkv_span_link_words(w.layout, w.src_batch)
+    flags = torch.zeros(2 * words, dtype=torch.int32, device=dev)
+    stream = torch.cuda.Stream(dev)
+    stream.wait_stream(torch.cuda.current_stream(dev))
+    rng = np.random.default_rng(3)
+    epoch = 0
+    for it in range(120):
+        k = int(rng.integers(0, 2))
+        tk.check(tk.topkv_relay_layers_linked(0, L, srcs[k], w.layout, w.src_batch, w.dst_pool, w.layout,
+                                              w.dst_batch, slab, n, flags, flags.numel(), epoch, stream))
+        epoch += L
+        if it % 7 == 6 or it == 119:
+            stream.synchronize()
+            assert torch.equal(w.dst_pool, want[k]), it
+    assert tk.topkv_device_error_flags() == 0 and int(flags.max()) == epoch
+    del w, srcs, want
+    torch.cuda.empty_cache()
+
+
 def test_relay_call_right_behind_a_kernel_that_writes_its_source(dev, variant):
     """The first launch of topkv_relay_layers_linked is an ordinary launch towards what precedes
     the call (TOPKV_LINK_WAIT_PREVIOUS): kernels that rewrite the source pool and the plan are
