@@ -78,3 +78,26 @@ def test_a_plain_c_program_links_and_calls_the_library(built, tmp_path):
     out = subprocess.run([str(exe)], capture_output=True, text=True)
     assert out.returncode == 0, out.stdout + out.stderr
     assert "bad 0" in out.stdout and f"version {tk.topkv_version()}" in out.stdout
+
+
+@pytest.mark.gpu
+def test_a_c_program_runs_pack_and_unpack_on_the_gpu(built, tmp_path):
+    """tests/c_caller/roundtrip.c (plain C, gcc): CUDA runtime + the library + the oracle, nothing else. Packs
+    and unpacks three layers of a ragged batch and compares wire and destination pool with the
+    oracle byte for byte (its exit status says so)."""
+    import oracle
+    cuda = os.environ.get("CUDA_HOME", "/usr/local/cuda")
+    if shutil.which("gcc") is None or not os.path.exists(os.path.join(cuda, "include", "cuda_runtime.h")):
+        pytest.skip("gcc or the CUDA runtime headers are not installed")
+    exe = tmp_path / "roundtrip"
+    libdir = os.path.dirname(built)
+    oracle_so = oracle.build()
+    odir = os.path.dirname(oracle_so)
+    subprocess.run(["gcc", "-std=c99", "-O1", "-Wall", "-Wextra", os.path.join(ROOT, "tests", "c_caller", "roundtrip.c"),
+                    "-o", str(exe), "-I", INCLUDE, "-I", odir, "-I", os.path.join(cuda, "include"),
+                    "-L", libdir, "-ltopkv", oracle_so, "-L", os.path.join(cuda, "lib64"), "-lcudart",
+                    f"-Wl,-rpath,{libdir}", f"-Wl,-rpath,{odir}", f"-Wl,-rpath,{os.path.join(cuda, 'lib64')}"],
+                   check=True)
+    out = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert out.returncode == 0, out.stdout + out.stderr
+    assert "wire identical, destination pool identical" in out.stdout
